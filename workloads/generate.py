@@ -1,0 +1,270 @@
+"""Counter-based seeded tensors for the workloads C1..C5.
+
+Every tensor is drawn from its own Philox stream keyed by (seed, tensor id),
+so changing one tensor's shape never changes another tensor's values.  Values
+are rounded once to their storage type (fp32, or bf16 with round-to-nearest-
+even); `Tensor.store` holds exactly the bytes a device buffer receives and
+`Tensor.f64()` widens those same bytes, without further rounding, for the CPU
+oracle.
+
+Distribution notation follows the workload list: "N(0, 1/fan_in)" gives the
+variance, "N(0, 0.02)" / "N(1, 0.02)" give the standard deviation (the usual
+GPT-style init), U(a, b) is uniform on the open interval.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+
+import numpy as np
+
+
+# --------------------------------------------------------------------------
+# storage formats
+# --------------------------------------------------------------------------
+def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
+    """fp32 -> bf16 bit patterns (uint16), round-to-nearest-even."""
+    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
+    rounding = ((u >> np.uint32(16)) & np.uint32(1)) + np.uint32(0x7FFF)
+    return ((u + rounding) >> np.uint32(16)).astype(np.uint16)
+
+
+def bf16_bits_to_f32(b: np.ndarray) -> np.ndarray:
+    return (b.astype(np.uint32) << np.uint32(16)).view(np.float32)
+
+
+def bf16_bits_to_f64(b: np.ndarray) -> np.ndarray:
+    return bf16_bits_to_f32(b).astype(np.float64)
+
+
+@dataclass
+class Tensor:
+    """One named tensor in its storage format.
+
+    dtype "f32": `store` is float32.  dtype "bf16": `store` is uint16 holding
+    bf16 bit patterns.  Shapes are logical, row-major, innermost last.
+    """
+
+    name: str
+    dtype: str
+    store: np.ndarray
+
+    @property
+    def shape(self):
+        return tuple(self.store.shape)
+
+    def f64(self) -> np.ndarray:
+        if self.dtype == "bf16":
+            return bf16_bits_to_f64(self.store)
+        return self.store.astype(np.float64)
+
+    def nbytes(self) -> int:
+        return int(self.store.nbytes)
+
+
+def make(name: str, dtype: str, values_f32: np.ndarray) -> Tensor:
+    """Round fp32 values to the storage type and wrap them."""
+    v = np.ascontiguousarray(values_f32, dtype=np.float32)
+    if dtype == "bf16":
+        return Tensor(name, "bf16", f32_to_bf16_bits(v))
+    if dtype == "f32":
+        return Tensor(name, "f32", v)
+    raise ValueError(f"unknown dtype {dtype!r}")
+
+
+# --------------------------------------------------------------------------
+# draws
+# --------------------------------------------------------------------------
+def _rng(seed: int, tensor_id: int) -> np.random.Generator:
+    return np.random.Generator(np.random.Philox(key=[int(seed), int(tensor_id)]))
+
+
+def _normal(seed, tid, shape, mean=0.0, std=1.0) -> np.ndarray:
+    x = _rng(seed, tid).standard_normal(size=shape, dtype=np.float32)
+    if std != 1.0:
+        x *= np.float32(std)
+    if mean != 0.0:
+        x += np.float32(mean)
+    return x
+
+
+def _uniform(seed, tid, shape, lo, hi) -> np.ndarray:
+    u = _rng(seed, tid).random(size=shape, dtype=np.float32)  # [0, 1)
+    # open interval: move exact 0 draws half a step inside
+    u = np.where(u == 0.0, np.float32(2.0 ** -25), u)
+    return (np.float32(lo) + (np.float32(hi) - np.float32(lo)) * u).astype(np.float32)
+
+
+def int_valued(seed: int, tid: int, shape, lo: int, hi: int, dtype: str, name="t") -> Tensor:
+    """Integers in [lo, hi]: exact in bf16, fp32 and fp64 alike, so a
+    contraction over them has one exact answer in every precision."""
+    v = _rng(seed, tid).integers(lo, hi + 1, size=shape).astype(np.float32)
+    return make(name, dtype, v)
+
+
+@dataclass
+class Workload:
+    """Inputs and parameters of one composed module, plus its op sequence.
+
+    `ops` is declarative: each entry names an operator kind, the values it
+    reads, the parameters it uses and its scalar attributes.  `partitions`
+    maps a decomposition name to the list of first-op indices of its
+    submodules.
+    """
+
+    name: str
+    dtype: str
+    inputs: dict = field(default_factory=dict)
+    params: dict = field(default_factory=dict)
+    ops: list = field(default_factory=list)
+    partitions: dict = field(default_factory=dict)
+    flops: float = 0.0
+    min_bytes: float = 0.0
+
+
+def _op(kind, out, ins, params=None, **attrs):
+    return {"kind": kind, "out": out, "in": list(ins), "params": dict(params or {}), "attrs": attrs}
+
+
+# --------------------------------------------------------------------------
+# C1: fp32 linear -> +bias -> ReLU -> row LayerNorm
+# --------------------------------------------------------------------------
+def c1(seed=0, M=64, K=256, N=128, dtype="f32") -> Workload:
+    w = Workload("c1", dtype)
+    w.inputs["x"] = make("x", dtype, _normal(seed, 0, (M, K)))
+    w.params["W"] = make("W", dtype, _normal(seed, 1, (K, N), std=(1.0 / K) ** 0.5))
+    w.params["b"] = make("b", dtype, _uniform(seed, 2, (N,), -0.1, 0.1))
+    w.params["gamma"] = make("gamma", dtype, np.ones((N,), np.float32))
+    w.params["beta"] = make("beta", dtype, np.zeros((N,), np.float32))
+    w.ops = [
+        _op("linear", "y0", ["x"], {"w": "W"}),
+        _op("bias_add", "y1", ["y0"], {"b": "b"}),
+        _op("relu", "y2", ["y1"]),
+        _op("layernorm", "y3", ["y2"], {"gamma": "gamma", "beta": "beta"}, eps=1e-5),
+    ]
+    w.partitions = {"fused": [0], "split": [0, 2, 3], "per_op": [0, 1, 2, 3]}
+    w.flops = 2.0 * M * K * N
+    esz = 4 if dtype == "f32" else 2
+    w.min_bytes = esz * (M * K + K * N + N + M * N)
+    return w
+
+
+# --------------------------------------------------------------------------
+# C2: bf16 GEMM -> +bias -> GELU(tanh) -> x0.5 -> clamp[-1, 1]
+# --------------------------------------------------------------------------
+def c2(seed=0, M=4096, K=4096, N=4096, dtype="bf16") -> Workload:
+    w = Workload("c2", dtype)
+    w.inputs["x"] = make("x", dtype, _normal(seed, 0, (M, K)))
+    w.params["W"] = make("W", dtype, _normal(seed, 1, (K, N), std=(1.0 / K) ** 0.5))
+    w.params["bias"] = make("bias", dtype, _normal(seed, 2, (N,), std=0.02))
+    w.ops = [
+        _op("linear", "y0", ["x"], {"w": "W"}),
+        _op("bias_add", "y1", ["y0"], {"b": "bias"}),
+        _op("gelu_tanh", "y2", ["y1"]),
+        _op("scale", "y3", ["y2"], s=0.5),
+        _op("clamp", "y4", ["y3"], lo=-1.0, hi=1.0),
+    ]
+    w.partitions = {"fused": [0], "split": [0, 2, 3, 4]}
+    w.flops = 2.0 * M * K * N
+    esz = 4 if dtype == "f32" else 2
+    w.min_bytes = esz * (M * K + K * N + N + M * N)
+    return w
+
+
+# --------------------------------------------------------------------------
+# C3: bf16 NHWC conv3x3 -> +bias -> ReLU -> GroupNorm
+# --------------------------------------------------------------------------
+def c3(seed=0, NB=32, H=56, W=56, C=128, CO=128, G=32, dtype="bf16") -> Workload:
+    w = Workload("c3", dtype)
+    w.inputs["x"] = make("x", dtype, _normal(seed, 0, (NB, H, W, C)))
+    # logical weight layout [C_out, kh, kw, C_in]
+    w.params["Wc"] = make("Wc", dtype, _normal(seed, 1, (CO, 3, 3, C), std=(1.0 / (9 * C)) ** 0.5))
+    w.params["bias"] = make("bias", dtype, _normal(seed, 2, (CO,), std=0.02))
+    w.params["gamma"] = make("gamma", dtype, _normal(seed, 3, (CO,), mean=1.0, std=0.02))
+    w.params["beta"] = make("beta", dtype, _normal(seed, 4, (CO,), std=0.02))
+    w.ops = [
+        _op("conv2d_3x3", "y0", ["x"], {"w": "Wc"}),
+        _op("bias_add", "y1", ["y0"], {"b": "bias"}),
+        _op("relu", "y2", ["y1"]),
+        _op("groupnorm", "y3", ["y2"], {"gamma": "gamma", "beta": "beta"}, groups=G, eps=1e-5),
+    ]
+    w.partitions = {"fused": [0], "split2": [0, 3], "split3": [0, 2, 3]}
+    w.flops = 2.0 * NB * H * W * CO * 9 * C
+    w.min_bytes = 2 * (NB * H * W * C + CO * 9 * C + 3 * CO + NB * H * W * CO)
+    return w
+
+
+# --------------------------------------------------------------------------
+# C4: bf16 causal attention -> out-proj + residual -> RMSNorm
+# --------------------------------------------------------------------------
+def c4(seed=0, B=16, H=16, S=2048, D=128, dtype="bf16") -> Workload:
+    w = Workload("c4", dtype)
+    E = H * D
+    w.inputs["q"] = make("q", dtype, _normal(seed, 0, (B, H, S, D)))
+    w.inputs["k"] = make("k", dtype, _normal(seed, 1, (B, H, S, D)))
+    w.inputs["v"] = make("v", dtype, _normal(seed, 2, (B, H, S, D)))
+    w.inputs["r"] = make("r", dtype, _normal(seed, 3, (B * S, E)))
+    w.params["Wo"] = make("Wo", dtype, _normal(seed, 4, (E, E), std=0.02))
+    w.params["gamma"] = make("gamma", dtype, np.ones((E,), np.float32))
+    w.ops = [
+        # attention output is logically [B*S, H*D], head-major columns
+        _op("attention_causal", "a", ["q", "k", "v"], layout="bhsd", heads=H, head_dim=D),
+        _op("linear", "p", ["a"], {"w": "Wo"}),
+        _op("residual_add", "h", ["p", "r"]),
+        _op("rmsnorm", "y", ["h"], {"gamma": "gamma"}, eps=1e-6),
+    ]
+    w.partitions = {"split3": [0, 1, 3], "per_op": [0, 1, 2, 3], "fused": [0]}
+    w.flops = 4.0 * B * H * D * (S * (S + 1) / 2) + 2.0 * B * S * E * E
+    w.min_bytes = 2 * (3 * B * H * S * D + B * S * E + E * E + E + B * S * E)
+    return w
+
+
+# --------------------------------------------------------------------------
+# C5: bf16 4-layer pre-norm decoder (RMSNorm, causal MHA, SwiGLU FFN)
+# --------------------------------------------------------------------------
+def c5(seed=0, B=8, S=1024, E=2048, H=16, F=8192, L=4, dtype="bf16") -> Workload:
+    w = Workload("c5", dtype)
+    D = E // H
+    w.inputs["x"] = make("x", dtype, _normal(seed, 0, (B * S, E)))
+    w.params["ones"] = make("ones", dtype, np.ones((E,), np.float32))
+    cur = "x"
+    tid = 1
+    layer_starts = []
+    for l in range(L):
+        layer_starts.append(len(w.ops))
+        # W_qkv columns are [Q | K | V], each head-major; W_gu columns are [gate | up]
+        w.params[f"Wqkv{l}"] = make(f"Wqkv{l}", dtype, _normal(seed, tid + 0, (E, 3 * E), std=0.02))
+        w.params[f"Wo{l}"] = make(f"Wo{l}", dtype, _normal(seed, tid + 1, (E, E), std=0.02))
+        w.params[f"Wgu{l}"] = make(f"Wgu{l}", dtype, _normal(seed, tid + 2, (E, 2 * F), std=0.02))
+        w.params[f"Wd{l}"] = make(f"Wd{l}", dtype, _normal(seed, tid + 3, (F, E), std=0.02))
+        tid += 4
+        w.ops += [
+            _op("rmsnorm", f"n1_{l}", [cur], {"gamma": "ones"}, eps=1e-6),
+            _op("linear", f"qkv_{l}", [f"n1_{l}"], {"w": f"Wqkv{l}"}),
+            _op("attention_causal", f"att_{l}", [f"qkv_{l}"], layout="packed_qkv", heads=H,
+                head_dim=D, batch=B, seq=S),
+            _op("linear", f"o_{l}", [f"att_{l}"], {"w": f"Wo{l}"}),
+            _op("residual_add", f"x1_{l}", [f"o_{l}", cur]),
+            _op("rmsnorm", f"n2_{l}", [f"x1_{l}"], {"gamma": "ones"}, eps=1e-6),
+            _op("linear", f"gu_{l}", [f"n2_{l}"], {"w": f"Wgu{l}"}),
+            _op("swiglu", f"hid_{l}", [f"gu_{l}"]),
+            _op("linear", f"d_{l}", [f"hid_{l}"], {"w": f"Wd{l}"}),
+            _op("residual_add", f"x2_{l}", [f"d_{l}", f"x1_{l}"]),
+        ]
+        cur = f"x2_{l}"
+    w.ops.append(_op("rmsnorm", "y", [cur], {"gamma": "ones"}, eps=1e-6))
+    n_ops = len(w.ops)
+    # default decomposition: GEMMs carry their elementwise tails, norms and attention stand alone
+    fused_cuts = []
+    for s in layer_starts:
+        fused_cuts += [s + 0, s + 1, s + 2, s + 3, s + 5, s + 6, s + 8]
+    fused_cuts.append(n_ops - 1)
+    w.partitions = {"fused_tails": fused_cuts, "per_op": list(range(n_ops)), "fused": [0]}
+    T = B * S
+    per_layer = (2.0 * T * E * 3 * E + 4.0 * B * H * D * (S * (S + 1) / 2) + 2.0 * T * E * E
+                 + 2.0 * T * E * 2 * F + 2.0 * T * F * E)
+    w.flops = L * per_layer
+    w.min_bytes = 2 * (2 * T * E + L * (3 * E * E + E * E + 3 * E * F))
+    return w
+
+
+WORKLOADS = {"c1": c1, "c2": c2, "c3": c3, "c4": c4, "c5": c5}
