@@ -1,0 +1,238 @@
+/*
+ * mk.h — C ABI of the composed-subkernel library (sm_100a).
+ *
+ * The library executes a PyTorch-style module as a programmatic composition of
+ * subkernels.  The calls follow the paper's statement of the problem
+ * (Methodology; Algorithms 1 and 2):
+ *
+ *   1. describe the module as an operator sequence            mk_module_create
+ *   2. register / edit its decomposition into submodules,     mk_module_set_decomposition,
+ *      each with a fixed input/output contract                mk_module_split / _fuse / _total_fuse,
+ *                                                             mk_module_get_contract
+ *   3. bind one subkernel implementation per submodule,       mk_impl_count / mk_impl_name,
+ *      and swap it without touching the neighbours            mk_module_bind
+ *   4. run the composed forward                               mk_module_set_param,
+ *                                                             mk_module_workspace_size,
+ *                                                             mk_module_forward
+ *   5. observe: per-subkernel time, boundary tensors          mk_module_profile,
+ *                                                             mk_module_intermediate
+ *
+ * Conventions
+ *   - Every pointer named dev_* / in_ptrs[i] / out_ptrs[i] / workspace is a DEVICE pointer
+ *     owned by the caller; the library borrows it and never allocates, frees or copies
+ *     device memory.  All other pointers are HOST pointers.
+ *   - Tensors are dense, row-major, innermost dimension last.  Device pointers must be
+ *     16-byte aligned.
+ *   - Every function returns an mk_status (0 = MK_OK, negative = error) and never throws or
+ *     aborts.  A failed edit or bind leaves the module exactly as it was (the paper's
+ *     Split/Fuse agents return the previous decomposition on failure).
+ *   - mk_module_forward is asynchronous on the given stream: no host synchronisation, no
+ *     allocation and no host<->device copy.
+ *   - There is no CPU fallback.  A submodule with no matching implementation yields
+ *     MK_ERR_NO_IMPL; a device that is not sm_100 yields MK_ERR_UNSUPPORTED_ARCH.
+ *   - One thread uses a module at a time.
+ */
+#ifndef MK_H_
+#define MK_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define MK_API __attribute__((visibility("default")))
+#else
+#define MK_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t mk_status;
+enum {
+  MK_OK = 0,
+  MK_ERR_INVALID_ARG = -1,
+  MK_ERR_SHAPE_MISMATCH = -2,
+  MK_ERR_NO_IMPL = -3,
+  MK_ERR_CONTRACT_VIOLATION = -4,
+  MK_ERR_WORKSPACE_TOO_SMALL = -5,
+  MK_ERR_UNSUPPORTED_ARCH = -6,
+  MK_ERR_CUDA = -7,
+  MK_ERR_DEVICE_TIMEOUT = -8,
+  MK_ERR_NO_DEVICE = -9,
+  MK_ERR_PARAM_MISSING = -10
+};
+
+typedef enum { MK_F32 = 0, MK_BF16 = 1 } mk_dtype;
+
+/* Physical layout of a rank-2 tensor.  MK_LAYOUT_TRANSPOSED stores the logical [R, C] matrix
+ * as its transpose, i.e. a dense row-major [C, R] array (a linear weight kept [out, in]). */
+typedef enum { MK_LAYOUT_ROW_MAJOR = 0, MK_LAYOUT_TRANSPOSED = 1 } mk_layout;
+
+#define MK_MAX_RANK 4
+typedef struct mk_tensor_spec {
+  int32_t dtype;               /* mk_dtype */
+  int32_t rank;                /* 1..MK_MAX_RANK */
+  int64_t shape[MK_MAX_RANK];  /* logical shape */
+  int32_t layout;              /* mk_layout (rank 2 only; 0 otherwise) */
+  int32_t reserved;
+} mk_tensor_spec;
+
+/* Operator kinds.  "x" is the operator's first input.
+ *   LINEAR          y[M,N] = x[M,K] @ W[K,N]            param 0 = W (logical [K,N]); i[0] = N,
+ *                                                       i[1] = mk_layout of W's storage
+ *   CONV2D_3X3      NHWC cross-correlation, stride 1, zero pad 1; param 0 = W [C_out,3,3,C_in];
+ *                                                       i[0] = C_out
+ *   BIAS_ADD        y = x + b[last dim]                 param 0 = b
+ *   RELU, GELU_TANH, SILU                               elementwise
+ *   SCALE           y = f[0] * x
+ *   CLAMP           y = min(max(x, f[0]), f[1])
+ *   RESIDUAL_ADD    y = x + in[1]                       (same shape)
+ *   SWIGLU          x[..., 2F] = [gate | up]; y[..., F] = silu(gate) * up
+ *   LAYERNORM       rows over the last dim, biased variance, f[0] = eps inside the root;
+ *                                                       param 0 = gamma, param 1 = beta (either may be absent)
+ *   RMSNORM         y = x / sqrt(mean(x^2) + f[0]) * gamma;  param 0 = gamma (may be absent)
+ *   GROUPNORM       NHWC, i[0] = groups of adjacent channels, f[0] = eps; params as LAYERNORM
+ *   SOFTMAX         safe softmax over the last dim
+ *   ATTENTION_CAUSAL  softmax(mask_{j<=i}(Q K^T / sqrt(D))) V, diagonal kept.
+ *                   i[0] = heads H, i[1] = head_dim D.
+ *                   i[2] = 0: three inputs q, k, v, each [B, H, S, D];
+ *                   i[2] = B > 0: one input, packed [B*S, 3*H*D] with columns [Q | K | V],
+ *                                 each head-major, and i[3] = S.
+ *                   Output is the logical [B*S, H*D] matrix (head-major columns).
+ * Definitions: the paper's subkernel listings (linear with W stored [K, N]; LayerNorm; online-
+ * softmax attention) and its correctness appendix (safe softmax, tril(diagonal=0) mask, fp32
+ * accumulation); RMSNorm, GroupNorm, SwiGLU, tanh-GELU and the 3x3 convolution follow the
+ * workload list.
+ */
+typedef enum {
+  MK_OP_LINEAR = 1,
+  MK_OP_CONV2D_3X3 = 2,
+  MK_OP_BIAS_ADD = 3,
+  MK_OP_RELU = 4,
+  MK_OP_GELU_TANH = 5,
+  MK_OP_SILU = 6,
+  MK_OP_SCALE = 7,
+  MK_OP_CLAMP = 8,
+  MK_OP_RESIDUAL_ADD = 9,
+  MK_OP_SWIGLU = 10,
+  MK_OP_LAYERNORM = 11,
+  MK_OP_RMSNORM = 12,
+  MK_OP_GROUPNORM = 13,
+  MK_OP_SOFTMAX = 14,
+  MK_OP_ATTENTION_CAUSAL = 15
+} mk_op_kind;
+
+/* Value numbering: module input k has id k; operator j produces id n_inputs + j.
+ * MK_PREV names the previous operator's output (module input 0 for operator 0).
+ * The last operator's output is the module's output. */
+#define MK_PREV (-1)
+#define MK_NONE (-2)
+
+typedef struct mk_op_desc {
+  int32_t kind;   /* mk_op_kind */
+  int32_t in[3];  /* value ids read; unused entries MK_NONE */
+  double f[2];    /* scalar attributes, see the table above */
+  int32_t i[4];   /* integer attributes, see the table above */
+} mk_op_desc;
+
+typedef struct mk_ctx mk_ctx;
+typedef struct mk_module mk_module;
+
+/* ---- context ------------------------------------------------------------------------------
+ * device >= 0: binds the context to that CUDA device (must be compute capability 10.x, else
+ * MK_ERR_UNSUPPORTED_ARCH; MK_ERR_NO_DEVICE if there is none).  device = -1: a host-only
+ * planning context — describing, decomposing, binding and contract queries work, launching
+ * returns MK_ERR_NO_DEVICE.  *out is written only on success. */
+MK_API mk_status mk_ctx_create(int32_t device, mk_ctx** out);
+MK_API void mk_ctx_destroy(mk_ctx* ctx);
+MK_API const char* mk_status_str(mk_status s);
+/* Text of the last error raised through this context ("" if none).  Valid until the next call. */
+MK_API const char* mk_last_error(const mk_ctx* ctx);
+/* Synchronises the context's device and reports a bounded-wait expiry inside a kernel
+ * (MK_ERR_DEVICE_TIMEOUT) or a CUDA error (MK_ERR_CUDA).  Clears the timeout flag. */
+MK_API mk_status mk_ctx_check(mk_ctx* ctx);
+
+/* ---- 1. describe a module as an operator sequence -------------------------------------------
+ * ops[n_ops] and inputs[n_inputs] are copied.  Shapes of all values are inferred here;
+ * an inconsistent sequence gives MK_ERR_SHAPE_MISMATCH / MK_ERR_INVALID_ARG.  The initial
+ * decomposition is one submodule per operator, each bound to the composer's default choice. */
+MK_API mk_status mk_module_create(mk_ctx* ctx, const mk_op_desc* ops, int32_t n_ops,
+                           const mk_tensor_spec* inputs, int32_t n_inputs, mk_module** out);
+MK_API void mk_module_destroy(mk_module* m);
+MK_API mk_status mk_module_n_ops(const mk_module* m, int32_t* n);
+/* Spec of value `value_id` (inputs first, then one per operator). */
+MK_API mk_status mk_module_value_spec(const mk_module* m, int32_t value_id, mk_tensor_spec* out);
+
+/* ---- 2. the decomposition: a partition of [0, n_ops) into contiguous submodules -----------
+ * first_op_of_sub[n_sub] must start at 0 and increase strictly; every operator then lies in
+ * exactly one submodule ("fully and exclusively cover").  Every new submodule is bound to
+ * the composer's default choice; MK_ERR_NO_IMPL if some submodule cannot be implemented. */
+MK_API mk_status mk_module_set_decomposition(mk_module* m, const int32_t* first_op_of_sub, int32_t n_sub);
+MK_API mk_status mk_module_n_sub(const mk_module* m, int32_t* n);
+/* Writes n_sub entries into first_op_of_sub (capacity checked against *n_sub on entry). */
+MK_API mk_status mk_module_get_decomposition(const mk_module* m, int32_t* first_op_of_sub, int32_t* n_sub);
+/* Split submodule `sub` into exactly two at operator `at_op` (first_op < at_op <= last op). */
+MK_API mk_status mk_module_split(mk_module* m, int32_t sub, int32_t at_op);
+/* Fuse `count` >= 2 adjacent submodules starting at `first_sub` into one. */
+MK_API mk_status mk_module_fuse(mk_module* m, int32_t first_sub, int32_t count);
+/* Collapse to the monolithic problem: one submodule holding every operator. */
+MK_API mk_status mk_module_total_fuse(mk_module* m);
+/* The submodule's I/O contract: value ids and specs it reads from outside and those it
+ * produces for later submodules or as the module output.  On entry *n_in / *n_out hold the
+ * capacities of the arrays (ids and specs may each be NULL); on return the counts. */
+MK_API mk_status mk_module_get_contract(const mk_module* m, int32_t sub, int32_t* in_ids,
+                                 mk_tensor_spec* in_specs, int32_t* n_in, int32_t* out_ids,
+                                 mk_tensor_spec* out_specs, int32_t* n_out);
+
+/* ---- 3. implementations: list, bind, swap ----------------------------------------------------
+ * mk_impl_count/_name enumerate the registered single-kernel-family implementations whose
+ * legality predicate accepts submodule `sub` as a whole.  mk_module_bind(sub, name) binds one
+ * of them (MK_ERR_NO_IMPL if it does not accept the submodule; the old binding stays).
+ * name = NULL asks the composer: it takes the widest legal fused implementation, and if no
+ * single one covers the submodule it covers it with a chain of them (longest match first),
+ * keeping the chain's intermediates in the workspace.  mk_module_bound_impl returns the bound
+ * name (a chain reads "a+b+c"); the string lives until the next edit or bind. */
+MK_API mk_status mk_impl_count(const mk_module* m, int32_t sub, int32_t* n);
+MK_API mk_status mk_impl_name(const mk_module* m, int32_t sub, int32_t i, const char** name);
+MK_API mk_status mk_module_bind(mk_module* m, int32_t sub, const char* impl_name);
+MK_API mk_status mk_module_bound_impl(const mk_module* m, int32_t sub, const char** name);
+
+/* ---- 4. parameters, workspace, run --------------------------------------------------------------
+ * set_param: operator `op`, slot as listed per kind; dev_ptr is borrowed and must stay valid;
+ * spec must equal what the operator expects (MK_ERR_SHAPE_MISMATCH otherwise). */
+MK_API mk_status mk_module_set_param(mk_module* m, int32_t op, int32_t slot, const void* dev_ptr,
+                              const mk_tensor_spec* spec);
+/* keep != 0: every submodule-boundary tensor keeps its own workspace range so that
+ * mk_module_intermediate can read it after a forward; keep = 0 (default) lets boundary
+ * tensors whose lifetimes do not overlap share memory. */
+MK_API mk_status mk_module_keep_intermediates(mk_module* m, int32_t keep);
+/* Bytes of workspace the current decomposition and bindings need (boundary tensors plus
+ * kernel scratch). */
+MK_API mk_status mk_module_workspace_size(mk_module* m, size_t* bytes);
+/* Kernel launches one forward issues under the current decomposition and bindings. */
+MK_API mk_status mk_module_launch_count(mk_module* m, int32_t* n);
+/* Composed forward.  in_ptrs[n_inputs], out_ptrs[1]: device tensors matching the specs.
+ * workspace: device memory of at least workspace_size bytes, 256-byte aligned, may be NULL
+ * when the size is 0.  cuda_stream: a cudaStream_t (NULL = the default stream).
+ * Errors: MK_ERR_PARAM_MISSING, MK_ERR_WORKSPACE_TOO_SMALL, MK_ERR_NO_DEVICE, MK_ERR_CUDA. */
+MK_API mk_status mk_module_forward(mk_module* m, const void* const* in_ptrs, void* const* out_ptrs,
+                            void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* ---- 5. observability ---------------------------------------------------------------------------
+ * profile: runs `iters` forwards with a CUDA event pair around every submodule, synchronises,
+ * and writes the mean milliseconds per submodule into ms_per_sub[n_sub] (the per-subkernel
+ * runtime the paper's budget allocation and Swap step read). */
+MK_API mk_status mk_module_profile(mk_module* m, const void* const* in_ptrs, void* const* out_ptrs,
+                            void* workspace, size_t workspace_bytes, void* cuda_stream,
+                            int32_t iters, float* ms_per_sub);
+/* Device pointer and spec of the tensor produced by value `value_id` at a submodule boundary
+ * during the last forward (requires keep_intermediates; MK_ERR_INVALID_ARG if the value is
+ * internal to a submodule or no forward has run). */
+MK_API mk_status mk_module_intermediate(const mk_module* m, int32_t value_id, const void** dev_ptr,
+                                 mk_tensor_spec* spec);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MK_H_ */

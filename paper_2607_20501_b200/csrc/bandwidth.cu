@@ -1,0 +1,480 @@
+// HBM-bound subkernels: elementwise chains, row reductions (LayerNorm / RMSNorm / softmax) and
+// NHWC GroupNorm.  All global traffic is 128-bit wide on the vector paths; statistics are fp32;
+// rows stay in registers between the reduction and the normalising pass, so each element is read
+// once and written once.
+#include "device_common.cuh"
+
+namespace mk {
+
+static inline int ceil_div_i64(int64_t a, int64_t b) { return (int)((a + b - 1) / b); }
+
+// =====================================================================================================
+// elementwise chain
+// =====================================================================================================
+template <typename T, bool SWIGLU>
+__global__ void __launch_bounds__(256) eltwise_vec_kernel(const T* __restrict__ x, T* __restrict__ y, int64_t rows,
+                                                          int64_t cols, const __grid_constant__ EpiProgram p) {
+  constexpr int VE = Elem<T>::VEC;
+  constexpr int UNROLL = 4;
+  const int64_t vpr = cols / VE;
+  const int64_t total = rows * vpr;
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  const int64_t in_ld = SWIGLU ? 2 * cols : cols;
+  for (int64_t base = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; base < total; base += stride * UNROLL) {
+    float v[UNROLL][VE];
+    float u[UNROLL][VE];
+    int64_t row[UNROLL], col[UNROLL];
+#pragma unroll
+    for (int q = 0; q < UNROLL; ++q) {
+      const int64_t i = base + q * stride;
+      if (i < total) {
+        row[q] = i / vpr;
+        col[q] = (i - row[q] * vpr) * VE;
+        ld_vec(x + row[q] * in_ld + col[q], v[q]);
+        if (SWIGLU) ld_vec(x + row[q] * in_ld + cols + col[q], u[q]);
+      }
+    }
+#pragma unroll
+    for (int q = 0; q < UNROLL; ++q) {
+      const int64_t i = base + q * stride;
+      if (i < total) {
+        if (SWIGLU) {
+#pragma unroll
+          for (int e = 0; e < VE; ++e) v[q][e] = silu_f(v[q][e]) * u[q][e];
+        }
+        epi_apply_vec<T, VE>(p, v[q], row[q], col[q], cols);
+        st_vec(y + row[q] * cols + col[q], v[q]);
+      }
+    }
+  }
+}
+
+template <typename T, bool SWIGLU>
+__global__ void __launch_bounds__(256) eltwise_scalar_kernel(const T* __restrict__ x, T* __restrict__ y, int64_t rows,
+                                                             int64_t cols, const __grid_constant__ EpiProgram p) {
+  const int64_t total = rows * cols;
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  const int64_t in_ld = SWIGLU ? 2 * cols : cols;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+    const int64_t r = i / cols, c = i - r * cols;
+    float v = Elem<T>::ld(x + r * in_ld + c);
+    if (SWIGLU) v = silu_f(v) * Elem<T>::ld(x + r * in_ld + cols + c);
+    Elem<T>::st(y + i, epi_apply(p, v, r, c, cols));
+  }
+}
+
+template <typename T>
+static cudaError_t eltwise_dispatch(const void* x, void* y, int64_t rows, int64_t cols, bool swiglu, const EpiProgram& p,
+                                    int sm_count, cudaStream_t s) {
+  constexpr int VE = Elem<T>::VEC;
+  const T* xp = (const T*)x;
+  T* yp = (T*)y;
+  if (rows * cols == 0) return cudaSuccess;
+  if (cols % VE == 0) {
+    const int64_t total = rows * (cols / VE);
+    int grid = ceil_div_i64(total, 256 * 4);
+    grid = grid < 1 ? 1 : (grid > sm_count * 8 ? sm_count * 8 : grid);
+    if (swiglu) eltwise_vec_kernel<T, true><<<grid, 256, 0, s>>>(xp, yp, rows, cols, p);
+    else eltwise_vec_kernel<T, false><<<grid, 256, 0, s>>>(xp, yp, rows, cols, p);
+  } else {
+    int grid = ceil_div_i64(rows * cols, 256);
+    grid = grid > sm_count * 8 ? sm_count * 8 : grid;
+    if (swiglu) eltwise_scalar_kernel<T, true><<<grid, 256, 0, s>>>(xp, yp, rows, cols, p);
+    else eltwise_scalar_kernel<T, false><<<grid, 256, 0, s>>>(xp, yp, rows, cols, p);
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_eltwise(int dtype, const void* x, void* y, int64_t rows, int64_t cols, bool swiglu, const EpiProgram& p,
+                           int sm_count, cudaStream_t s) {
+  return dtype == DT_F32 ? eltwise_dispatch<float>(x, y, rows, cols, swiglu, p, sm_count, s)
+                         : eltwise_dispatch<__nv_bfloat16>(x, y, rows, cols, swiglu, p, sm_count, s);
+}
+
+// =====================================================================================================
+// row reductions: one warp per row, the row lives in registers
+// =====================================================================================================
+template <typename T, int VPL, int MODE>
+__global__ void __launch_bounds__(128) rowop_warp_kernel(const T* __restrict__ x, T* __restrict__ y, int64_t rows, int n,
+                                                         const T* __restrict__ gamma, const T* __restrict__ beta, float eps,
+                                                         const __grid_constant__ EpiProgram pre) {
+  constexpr int VE = Elem<T>::VEC;
+  const int lane = threadIdx.x & 31;
+  const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (row >= rows) return;
+  const int nvec = n / VE;
+  const T* xr = x + row * n;
+  float v[VPL][VE];
+#pragma unroll
+  for (int i = 0; i < VPL; ++i) {
+    const int vi = lane + 32 * i;
+    if (vi < nvec) {
+      ld_vec(xr + vi * VE, v[i]);
+      epi_apply_vec<T, VE>(pre, v[i], row, (int64_t)vi * VE, n);
+    } else {
+#pragma unroll
+      for (int e = 0; e < VE; ++e) v[i][e] = (MODE == ROW_SOFTMAX) ? -INFINITY : 0.0f;
+    }
+  }
+  const float inv_n = 1.0f / (float)n;
+  float mean = 0.0f, mul = 1.0f;
+  if (MODE == ROW_LAYERNORM) {
+    float s = 0.0f;
+#pragma unroll
+    for (int i = 0; i < VPL; ++i)
+#pragma unroll
+      for (int e = 0; e < VE; ++e) s += v[i][e];
+    mean = warp_sum(s) * inv_n;
+    float q = 0.0f;
+#pragma unroll
+    for (int i = 0; i < VPL; ++i)
+      if (lane + 32 * i < nvec) {
+#pragma unroll
+        for (int e = 0; e < VE; ++e) { const float d = v[i][e] - mean; q += d * d; }
+      }
+    mul = rsqrtf(warp_sum(q) * inv_n + eps);
+  } else if (MODE == ROW_RMSNORM) {
+    float q = 0.0f;
+#pragma unroll
+    for (int i = 0; i < VPL; ++i)
+#pragma unroll
+      for (int e = 0; e < VE; ++e) q += v[i][e] * v[i][e];
+    mul = rsqrtf(warp_sum(q) * inv_n + eps);
+  } else {
+    float mx = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < VPL; ++i)
+#pragma unroll
+      for (int e = 0; e < VE; ++e) mx = fmaxf(mx, v[i][e]);
+    mx = warp_max(mx);
+    float s = 0.0f;
+#pragma unroll
+    for (int i = 0; i < VPL; ++i)
+#pragma unroll
+      for (int e = 0; e < VE; ++e) { v[i][e] = __expf(v[i][e] - mx); s += v[i][e]; }
+    mul = 1.0f / warp_sum(s);
+  }
+  T* yr = y + row * n;
+#pragma unroll
+  for (int i = 0; i < VPL; ++i) {
+    const int vi = lane + 32 * i;
+    if (vi < nvec) {
+      float o[VE];
+#pragma unroll
+      for (int e = 0; e < VE; ++e) o[e] = (v[i][e] - mean) * mul;
+      if (MODE != ROW_SOFTMAX) {
+        if (gamma) {
+          float g[VE];
+          ld_vec(gamma + vi * VE, g);
+#pragma unroll
+          for (int e = 0; e < VE; ++e) o[e] *= g[e];
+        }
+        if (MODE == ROW_LAYERNORM && beta) {
+          float b[VE];
+          ld_vec(beta + vi * VE, b);
+#pragma unroll
+          for (int e = 0; e < VE; ++e) o[e] += b[e];
+        }
+      }
+      st_vec(yr + vi * VE, o);
+    }
+  }
+}
+
+// Fallback for rows that do not fit the register path or are not a multiple of the vector width:
+// one CTA per row, three passes over the row (it stays in L1/L2 between them).
+template <int MODE>
+__device__ __forceinline__ float block_reduce(float v, float* sh) {
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  v = (MODE == 1) ? warp_max(v) : warp_sum(v);
+  __syncthreads();
+  if (lane == 0) sh[w] = v;
+  __syncthreads();
+  float r = (MODE == 1) ? -INFINITY : 0.0f;
+  for (int i = 0; i < nw; ++i) r = (MODE == 1) ? fmaxf(r, sh[i]) : r + sh[i];
+  return r;
+}
+
+template <typename T, int MODE>
+__global__ void __launch_bounds__(256) rowop_block_kernel(const T* __restrict__ x, T* __restrict__ y, int64_t rows, int64_t n,
+                                                          const T* __restrict__ gamma, const T* __restrict__ beta, float eps,
+                                                          const __grid_constant__ EpiProgram pre) {
+  __shared__ float sh[32];
+  const int64_t row = blockIdx.x;
+  const T* xr = x + row * n;
+  T* yr = y + row * n;
+  const float inv_n = 1.0f / (float)n;
+  float mean = 0.0f, mul = 1.0f, mx = 0.0f;
+  if (MODE == ROW_LAYERNORM) {
+    float s = 0.0f;
+    for (int64_t c = threadIdx.x; c < n; c += blockDim.x) s += epi_apply(pre, Elem<T>::ld(xr + c), row, c, n);
+    mean = block_reduce<0>(s, sh) * inv_n;
+    float q = 0.0f;
+    for (int64_t c = threadIdx.x; c < n; c += blockDim.x) { const float d = epi_apply(pre, Elem<T>::ld(xr + c), row, c, n) - mean; q += d * d; }
+    mul = rsqrtf(block_reduce<0>(q, sh) * inv_n + eps);
+  } else if (MODE == ROW_RMSNORM) {
+    float q = 0.0f;
+    for (int64_t c = threadIdx.x; c < n; c += blockDim.x) { const float d = epi_apply(pre, Elem<T>::ld(xr + c), row, c, n); q += d * d; }
+    mul = rsqrtf(block_reduce<0>(q, sh) * inv_n + eps);
+  } else {
+    float m = -INFINITY;
+    for (int64_t c = threadIdx.x; c < n; c += blockDim.x) m = fmaxf(m, epi_apply(pre, Elem<T>::ld(xr + c), row, c, n));
+    mx = block_reduce<1>(m, sh);
+    float s = 0.0f;
+    for (int64_t c = threadIdx.x; c < n; c += blockDim.x) s += __expf(epi_apply(pre, Elem<T>::ld(xr + c), row, c, n) - mx);
+    mul = 1.0f / block_reduce<0>(s, sh);
+  }
+  for (int64_t c = threadIdx.x; c < n; c += blockDim.x) {
+    const float v = epi_apply(pre, Elem<T>::ld(xr + c), row, c, n);
+    float o;
+    if (MODE == ROW_SOFTMAX) {
+      o = __expf(v - mx) * mul;
+    } else {
+      o = (v - mean) * mul;
+      if (gamma) o *= Elem<T>::ld(gamma + c);
+      if (MODE == ROW_LAYERNORM && beta) o += Elem<T>::ld(beta + c);
+    }
+    Elem<T>::st(yr + c, o);
+  }
+}
+
+template <typename T, int MODE>
+static cudaError_t rowop_mode(const T* x, T* y, int64_t rows, int64_t n, const T* g, const T* b, float eps,
+                              const EpiProgram& pre, cudaStream_t s) {
+  constexpr int VE = Elem<T>::VEC;
+  if (rows == 0) return cudaSuccess;
+  const int64_t nvec = n / VE;
+  if (n % VE == 0 && nvec <= 32 * 16) {
+    const int grid = ceil_div_i64(rows, 4);
+    const int ni = (int)n;
+    if (nvec <= 32) rowop_warp_kernel<T, 1, MODE><<<grid, 128, 0, s>>>(x, y, rows, ni, g, b, eps, pre);
+    else if (nvec <= 64) rowop_warp_kernel<T, 2, MODE><<<grid, 128, 0, s>>>(x, y, rows, ni, g, b, eps, pre);
+    else if (nvec <= 128) rowop_warp_kernel<T, 4, MODE><<<grid, 128, 0, s>>>(x, y, rows, ni, g, b, eps, pre);
+    else if (nvec <= 256) rowop_warp_kernel<T, 8, MODE><<<grid, 128, 0, s>>>(x, y, rows, ni, g, b, eps, pre);
+    else rowop_warp_kernel<T, 16, MODE><<<grid, 128, 0, s>>>(x, y, rows, ni, g, b, eps, pre);
+  } else {
+    rowop_block_kernel<T, MODE><<<(unsigned)rows, 256, 0, s>>>(x, y, rows, n, g, b, eps, pre);
+  }
+  return cudaGetLastError();
+}
+
+template <typename T>
+static cudaError_t rowop_dispatch(int mode, const void* x, void* y, int64_t rows, int64_t n, const void* g, const void* b,
+                                  float eps, const EpiProgram& pre, cudaStream_t s) {
+  const T* xp = (const T*)x; T* yp = (T*)y; const T* gp = (const T*)g; const T* bp = (const T*)b;
+  switch (mode) {
+    case ROW_LAYERNORM: return rowop_mode<T, ROW_LAYERNORM>(xp, yp, rows, n, gp, bp, eps, pre, s);
+    case ROW_RMSNORM: return rowop_mode<T, ROW_RMSNORM>(xp, yp, rows, n, gp, bp, eps, pre, s);
+    default: return rowop_mode<T, ROW_SOFTMAX>(xp, yp, rows, n, gp, bp, eps, pre, s);
+  }
+}
+
+cudaError_t launch_rowop(int dtype, int mode, const void* x, void* y, int64_t rows, int64_t n, const void* gamma,
+                         const void* beta, float eps, const EpiProgram& pre, cudaStream_t s) {
+  return dtype == DT_F32 ? rowop_dispatch<float>(mode, x, y, rows, n, gamma, beta, eps, pre, s)
+                         : rowop_dispatch<__nv_bfloat16>(mode, x, y, rows, n, gamma, beta, eps, pre, s);
+}
+
+// =====================================================================================================
+// GroupNorm NHWC: the statistics of one (image, group) span the whole image, a global
+// synchronisation, so it takes two launches: partial sums per (image, pixel chunk, group), then a
+// pass that reduces the partials (a few dozen values) and normalises.
+// scratch layout: float [nb][chunks][groups][2] = (sum, sum of squares)
+// =====================================================================================================
+int groupnorm_chunks(int64_t nb, int64_t hw, int sm_count) {
+  // enough CTAs to fill the machine twice over, at least 32 pixels each
+  int64_t want = (2 * (int64_t)sm_count + nb - 1) / nb;
+  int64_t maxc = hw / 32 > 0 ? hw / 32 : 1;
+  int64_t c = want < 1 ? 1 : want;
+  if (c > maxc) c = maxc;
+  if (c > 64) c = 64;
+  return (int)c;
+}
+size_t groupnorm_scratch_bytes(int64_t nb, int64_t hw, int64_t, int groups, int sm_count) {
+  return (size_t)nb * groupnorm_chunks(nb, hw, sm_count) * groups * 2 * sizeof(float);
+}
+
+constexpr int GN_THREADS = 256;
+constexpr int GN_MAX_C = 2048;
+
+template <typename T>
+__host__ __device__ inline bool gn_fast_ok(int64_t c) {
+  const int64_t vpp = c / Elem<T>::VEC;
+  return c % Elem<T>::VEC == 0 && vpp >= 1 && vpp <= GN_THREADS && (GN_THREADS % vpp) == 0 && c <= GN_MAX_C;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(GN_THREADS) groupnorm_stats_kernel(const T* __restrict__ x, int64_t hw, int c, int groups,
+                                                                     const __grid_constant__ EpiProgram pre,
+                                                                     float* __restrict__ scratch) {
+  constexpr int VE = Elem<T>::VEC;
+  __shared__ float sh_s[GN_THREADS * VE];
+  __shared__ float sh_q[GN_THREADS * VE];
+  const int chunks = gridDim.x, chunk = blockIdx.x;
+  const int64_t img = blockIdx.y;
+  const int vpp = c / VE;
+  const int vcol = threadIdx.x % vpp, prow = threadIdx.x / vpp, pstride = GN_THREADS / vpp;
+  const int64_t p0 = hw * chunk / chunks, p1 = hw * (chunk + 1) / chunks;
+  float s[VE], q[VE];
+#pragma unroll
+  for (int e = 0; e < VE; ++e) { s[e] = 0.0f; q[e] = 0.0f; }
+  for (int64_t pix = p0 + prow; pix < p1; pix += pstride) {
+    float v[VE];
+    const int64_t r = img * hw + pix;
+    ld_vec(x + r * c + vcol * VE, v);
+    epi_apply_vec<T, VE>(pre, v, r, (int64_t)vcol * VE, c);
+#pragma unroll
+    for (int e = 0; e < VE; ++e) { s[e] += v[e]; q[e] += v[e] * v[e]; }
+  }
+#pragma unroll
+  for (int e = 0; e < VE; ++e) {
+    sh_s[prow * c + vcol * VE + e] = s[e];
+    sh_q[prow * c + vcol * VE + e] = q[e];
+  }
+  __syncthreads();
+  const int cg = c / groups;
+  for (int g = threadIdx.x; g < groups; g += GN_THREADS) {
+    float ts = 0.0f, tq = 0.0f;
+    for (int ch = g * cg; ch < (g + 1) * cg; ++ch)
+      for (int r = 0; r < pstride; ++r) { ts += sh_s[r * c + ch]; tq += sh_q[r * c + ch]; }
+    float* o = scratch + ((img * chunks + chunk) * groups + g) * 2;
+    o[0] = ts;
+    o[1] = tq;
+  }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(GN_THREADS) groupnorm_apply_kernel(const T* __restrict__ x, T* __restrict__ y, int64_t hw,
+                                                                     int c, int groups, const T* __restrict__ gamma,
+                                                                     const T* __restrict__ beta, float eps,
+                                                                     const __grid_constant__ EpiProgram pre,
+                                                                     const float* __restrict__ scratch) {
+  constexpr int VE = Elem<T>::VEC;
+  __shared__ float sh_scale[GN_MAX_C];
+  __shared__ float sh_shift[GN_MAX_C];
+  const int chunks = gridDim.x, chunk = blockIdx.x;
+  const int64_t img = blockIdx.y;
+  const int cg = c / groups;
+  const float inv_cnt = 1.0f / ((float)hw * (float)cg);
+  for (int ch = threadIdx.x; ch < c; ch += GN_THREADS) {
+    const int g = ch / cg;
+    float ts = 0.0f, tq = 0.0f;
+    for (int k = 0; k < chunks; ++k) {
+      const float* o = scratch + ((img * chunks + k) * groups + g) * 2;
+      ts += o[0];
+      tq += o[1];
+    }
+    const float mean = ts * inv_cnt;
+    const float var = fmaxf(tq * inv_cnt - mean * mean, 0.0f);
+    const float rstd = rsqrtf(var + eps);
+    const float ga = gamma ? Elem<T>::ld(gamma + ch) : 1.0f;
+    const float be = beta ? Elem<T>::ld(beta + ch) : 0.0f;
+    sh_scale[ch] = rstd * ga;
+    sh_shift[ch] = be - mean * rstd * ga;
+  }
+  __syncthreads();
+  const int vpp = c / VE;
+  const int vcol = threadIdx.x % vpp, prow = threadIdx.x / vpp, pstride = GN_THREADS / vpp;
+  const int64_t p0 = hw * chunk / chunks, p1 = hw * (chunk + 1) / chunks;
+  for (int64_t pix = p0 + prow; pix < p1; pix += pstride) {
+    float v[VE];
+    const int64_t r = img * hw + pix;
+    ld_vec(x + r * c + vcol * VE, v);
+    epi_apply_vec<T, VE>(pre, v, r, (int64_t)vcol * VE, c);
+#pragma unroll
+    for (int e = 0; e < VE; ++e) v[e] = v[e] * sh_scale[vcol * VE + e] + sh_shift[vcol * VE + e];
+    st_vec(y + r * c + vcol * VE, v);
+  }
+}
+
+// Any channel count: scalar accesses, shared-memory atomics for the group sums.
+template <typename T>
+__global__ void __launch_bounds__(GN_THREADS) groupnorm_stats_generic(const T* __restrict__ x, int64_t hw, int64_t c, int groups,
+                                                                      const __grid_constant__ EpiProgram pre,
+                                                                      float* __restrict__ scratch) {
+  const int chunks = gridDim.x, chunk = blockIdx.x;
+  const int64_t img = blockIdx.y;
+  const int64_t cg = c / groups;
+  const int64_t p0 = hw * chunk / chunks, p1 = hw * (chunk + 1) / chunks;
+  float* out = scratch + (img * chunks + chunk) * groups * 2;
+  for (int g = 0; g < groups; ++g) {  // one group at a time keeps shared memory constant-size
+    __shared__ float sh[32];
+    float s = 0.0f, q = 0.0f;
+    const int64_t cnt = (p1 - p0) * cg;
+    for (int64_t i = threadIdx.x; i < cnt; i += GN_THREADS) {
+      const int64_t pix = p0 + i / cg, ch = g * cg + i % cg;
+      const int64_t r = img * hw + pix;
+      const float v = epi_apply(pre, Elem<T>::ld(x + r * c + ch), r, ch, c);
+      s += v;
+      q += v * v;
+    }
+    s = block_reduce<0>(s, sh);
+    q = block_reduce<0>(q, sh);
+    if (threadIdx.x == 0) { out[g * 2] = s; out[g * 2 + 1] = q; }
+  }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(GN_THREADS) groupnorm_apply_generic(const T* __restrict__ x, T* __restrict__ y, int64_t hw,
+                                                                      int64_t c, int groups, const T* __restrict__ gamma,
+                                                                      const T* __restrict__ beta, float eps,
+                                                                      const __grid_constant__ EpiProgram pre,
+                                                                      const float* __restrict__ scratch) {
+  const int chunks = gridDim.x, chunk = blockIdx.x;
+  const int64_t img = blockIdx.y;
+  const int64_t cg = c / groups;
+  const float inv_cnt = 1.0f / ((float)hw * (float)cg);
+  const int64_t p0 = hw * chunk / chunks, p1 = hw * (chunk + 1) / chunks;
+  for (int64_t i = threadIdx.x; i < (p1 - p0) * c; i += GN_THREADS) {
+    const int64_t pix = p0 + i / c, ch = i % c;
+    const int g = (int)(ch / cg);
+    float ts = 0.0f, tq = 0.0f;
+    for (int k = 0; k < chunks; ++k) {
+      const float* o = scratch + ((img * chunks + k) * groups + g) * 2;
+      ts += o[0];
+      tq += o[1];
+    }
+    const float mean = ts * inv_cnt;
+    const float rstd = rsqrtf(fmaxf(tq * inv_cnt - mean * mean, 0.0f) + eps);
+    const int64_t r = img * hw + pix;
+    float v = (epi_apply(pre, Elem<T>::ld(x + r * c + ch), r, ch, c) - mean) * rstd;
+    if (gamma) v *= Elem<T>::ld(gamma + ch);
+    if (beta) v += Elem<T>::ld(beta + ch);
+    Elem<T>::st(y + r * c + ch, v);
+  }
+}
+
+template <typename T>
+static cudaError_t gn_stats(const void* x, int64_t nb, int64_t hw, int64_t c, int groups, const EpiProgram& pre, float* scratch,
+                            int chunks, cudaStream_t s) {
+  if (nb == 0) return cudaSuccess;
+  dim3 grid(chunks, (unsigned)nb);
+  if (gn_fast_ok<T>(c)) groupnorm_stats_kernel<T><<<grid, GN_THREADS, 0, s>>>((const T*)x, hw, (int)c, groups, pre, scratch);
+  else groupnorm_stats_generic<T><<<grid, GN_THREADS, 0, s>>>((const T*)x, hw, c, groups, pre, scratch);
+  return cudaGetLastError();
+}
+template <typename T>
+static cudaError_t gn_apply(const void* x, void* y, int64_t nb, int64_t hw, int64_t c, int groups, const void* g, const void* b,
+                            float eps, const EpiProgram& pre, const float* scratch, int chunks, cudaStream_t s) {
+  if (nb == 0) return cudaSuccess;
+  dim3 grid(chunks, (unsigned)nb);
+  if (gn_fast_ok<T>(c))
+    groupnorm_apply_kernel<T><<<grid, GN_THREADS, 0, s>>>((const T*)x, (T*)y, hw, (int)c, groups, (const T*)g, (const T*)b, eps, pre, scratch);
+  else
+    groupnorm_apply_generic<T><<<grid, GN_THREADS, 0, s>>>((const T*)x, (T*)y, hw, c, groups, (const T*)g, (const T*)b, eps, pre, scratch);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_groupnorm_stats(int dtype, const void* x, int64_t nb, int64_t hw, int64_t c, int groups, const EpiProgram& pre,
+                                   float* scratch, int chunks, cudaStream_t s) {
+  return dtype == DT_F32 ? gn_stats<float>(x, nb, hw, c, groups, pre, scratch, chunks, s)
+                         : gn_stats<__nv_bfloat16>(x, nb, hw, c, groups, pre, scratch, chunks, s);
+}
+cudaError_t launch_groupnorm_apply(int dtype, const void* x, void* y, int64_t nb, int64_t hw, int64_t c, int groups,
+                                   const void* gamma, const void* beta, float eps, const EpiProgram& pre, const float* scratch,
+                                   int chunks, cudaStream_t s) {
+  return dtype == DT_F32 ? gn_apply<float>(x, y, nb, hw, c, groups, gamma, beta, eps, pre, scratch, chunks, s)
+                         : gn_apply<__nv_bfloat16>(x, y, nb, hw, c, groups, gamma, beta, eps, pre, scratch, chunks, s);
+}
+
+}  // namespace mk

@@ -1,0 +1,151 @@
+// Device helpers shared by the kernels: storage conversion, 128-bit access, warp reductions and the
+// elementwise-program interpreter.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "kernels.h"
+
+namespace mk {
+
+template <typename T> struct Elem;
+template <> struct Elem<float> {
+  static constexpr int VEC = 4;  // elements per 128-bit access
+  __device__ __forceinline__ static float ld(const float* p) { return *p; }
+  __device__ __forceinline__ static void st(float* p, float v) { *p = v; }
+};
+template <> struct Elem<__nv_bfloat16> {
+  static constexpr int VEC = 8;
+  __device__ __forceinline__ static float ld(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+  __device__ __forceinline__ static void st(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
+};
+
+// 128-bit load of VEC consecutive elements into fp32 registers (pointer 16-byte aligned)
+__device__ __forceinline__ void ld_vec(const float* p, float (&v)[4]) {
+  const float4 t = *reinterpret_cast<const float4*>(p);
+  v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+}
+__device__ __forceinline__ void ld_vec(const __nv_bfloat16* p, float (&v)[8]) {
+  const uint4 t = *reinterpret_cast<const uint4*>(p);
+  const uint32_t w[4] = {t.x, t.y, t.z, t.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    v[2 * i] = __uint_as_float(w[i] << 16);
+    v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+  }
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&t);
+}
+__device__ __forceinline__ void st_vec(float* p, const float (&v)[4]) {
+  *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
+}
+__device__ __forceinline__ void st_vec(__nv_bfloat16* p, const float (&v)[8]) {
+  uint4 t;
+  t.x = pack_bf16x2(v[0], v[1]);
+  t.y = pack_bf16x2(v[2], v[3]);
+  t.z = pack_bf16x2(v[4], v[5]);
+  t.w = pack_bf16x2(v[6], v[7]);
+  *reinterpret_cast<uint4*>(p) = t;
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+__device__ __forceinline__ float gelu_tanh_f(float x) {
+  const float u = 0.7978845608028654f * (x + 0.044715f * x * x * x);
+  return 0.5f * x * (1.0f + tanhf(u));
+}
+__device__ __forceinline__ float silu_f(float x) { return x / (1.0f + __expf(-x)); }
+
+__device__ __forceinline__ float epi_ptr_ld(const void* p, int dtype, int64_t i) {
+  return dtype == DT_F32 ? reinterpret_cast<const float*>(p)[i]
+                         : __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p)[i]);
+}
+
+// Run the program on one value sitting at (row, col) of a [*, ld] output.
+__device__ __forceinline__ float epi_apply(const EpiProgram& p, float v, int64_t row, int64_t col, int64_t ld) {
+  for (int i = 0; i < p.n; ++i) {
+    const EpiOp& o = p.op[i];
+    switch (o.kind) {
+      case EPI_BIAS: v += epi_ptr_ld(o.ptr, p.dtype, col); break;
+      case EPI_RELU: v = fmaxf(v, 0.0f); break;
+      case EPI_GELU_TANH: v = gelu_tanh_f(v); break;
+      case EPI_SILU: v = silu_f(v); break;
+      case EPI_SCALE: v *= o.a; break;
+      case EPI_CLAMP: v = fminf(fmaxf(v, o.a), o.b); break;
+      case EPI_RESIDUAL: v += epi_ptr_ld(o.ptr, p.dtype, row * ld + col); break;
+      default: break;
+    }
+  }
+  return v;
+}
+
+// Run the program on NV consecutive columns of one row; col0 is a multiple of NV and the program's
+// pointers are 16-byte aligned, so bias and residual are fetched with 128-bit loads.
+template <typename T, int NV>
+__device__ __forceinline__ void epi_apply_vec(const EpiProgram& p, float (&v)[NV], int64_t row, int64_t col0, int64_t ld) {
+  static_assert(NV % Elem<T>::VEC == 0, "vector width");
+  constexpr int VE = Elem<T>::VEC;
+  for (int i = 0; i < p.n; ++i) {
+    const EpiOp& o = p.op[i];
+    switch (o.kind) {
+      case EPI_BIAS: {
+        const T* b = reinterpret_cast<const T*>(o.ptr) + col0;
+#pragma unroll
+        for (int j = 0; j < NV; j += VE) {
+          float t[VE];
+          ld_vec(b + j, t);
+#pragma unroll
+          for (int q = 0; q < VE; ++q) v[j + q] += t[q];
+        }
+        break;
+      }
+      case EPI_RESIDUAL: {
+        const T* r = reinterpret_cast<const T*>(o.ptr) + row * ld + col0;
+#pragma unroll
+        for (int j = 0; j < NV; j += VE) {
+          float t[VE];
+          ld_vec(r + j, t);
+#pragma unroll
+          for (int q = 0; q < VE; ++q) v[j + q] += t[q];
+        }
+        break;
+      }
+      case EPI_RELU:
+#pragma unroll
+        for (int j = 0; j < NV; ++j) v[j] = fmaxf(v[j], 0.0f);
+        break;
+      case EPI_GELU_TANH:
+#pragma unroll
+        for (int j = 0; j < NV; ++j) v[j] = gelu_tanh_f(v[j]);
+        break;
+      case EPI_SILU:
+#pragma unroll
+        for (int j = 0; j < NV; ++j) v[j] = silu_f(v[j]);
+        break;
+      case EPI_SCALE:
+#pragma unroll
+        for (int j = 0; j < NV; ++j) v[j] *= o.a;
+        break;
+      case EPI_CLAMP:
+#pragma unroll
+        for (int j = 0; j < NV; ++j) v[j] = fminf(fmaxf(v[j], o.a), o.b);
+        break;
+      default: break;
+    }
+  }
+}
+
+}  // namespace mk

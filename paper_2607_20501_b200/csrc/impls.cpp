@@ -1,0 +1,244 @@
+// Implementation registry: each entry is a kernel family with the legality predicate that says
+// which operator ranges it can run as ONE fused piece, following the paper's fusion rules
+// (appendix "Prompts", decomposition: GEMM + elementwise tail, elementwise chains, bias after
+// matmul and residual add fuse; a reduction that needs the whole row / group before its result is
+// used blocks fusion unless one CTA owns the whole row).
+//
+// Order = the composer's preference among implementations that accept the same range.
+#include "mk_internal.h"
+
+namespace mk {
+namespace {
+
+int dt(const Module& m) { return m.values[0].spec.dtype == MK_F32 ? DT_F32 : DT_BF16; }
+
+// ops lo+1.. read their predecessor as first input; nothing but the last value leaves the piece;
+// residual operands come from outside the piece.
+bool is_chain(const Module& m, int lo, int hi) {
+  if (hi <= lo) return false;
+  for (int j = lo + 1; j < hi; ++j)
+    if (m.ops[j].in_id[0] != m.ops[j - 1].out_id) return false;
+  for (int j = lo; j < hi - 1; ++j)
+    if (m.escapes(j, lo, hi)) return false;
+  for (int j = lo; j < hi; ++j)
+    if (m.ops[j].d.kind == MK_OP_RESIDUAL_ADD) {
+      const int prod = m.values[m.ops[j].in_id[1]].producer;
+      if (prod >= lo && prod < hi) return false;
+    }
+  return true;
+}
+bool all_eltwise(const Module& m, int a, int b) {
+  if (b - a > EPI_MAX) return false;
+  for (int j = a; j < b; ++j)
+    if (!is_eltwise(m.ops[j].d.kind)) return false;
+  return true;
+}
+size_t no_scratch(const Module&, int, int) { return 0; }
+
+int64_t last_dim(const mk_tensor_spec& s) { return s.shape[s.rank - 1]; }
+int64_t rows_of(const mk_tensor_spec& s) { return numel(s) / last_dim(s); }
+
+// ------------------------------------------------------------------ eltwise chain
+bool eltwise_match(const Module& m, int lo, int hi) {
+  if (!is_chain(m, lo, hi)) return false;
+  const bool sw = m.ops[lo].d.kind == MK_OP_SWIGLU;
+  return all_eltwise(m, lo + (sw ? 1 : 0), hi);
+}
+mk_status eltwise_emit(const Module& m, int lo, int hi, const Resolved& r, std::vector<Launch>& out, std::string& err) {
+  const bool sw = m.ops[lo].d.kind == MK_OP_SWIGLU;
+  EpiProgram p;
+  mk_status st = build_epi(m, lo + (sw ? 1 : 0), hi, r, p, err);
+  if (st != MK_OK) return st;
+  const void* x = r.value_ptr[m.ops[lo].in_id[0]];
+  void* y = r.value_ptr[m.ops[hi - 1].out_id];
+  const mk_tensor_spec& ys = m.vspec(m.ops[hi - 1].out_id);
+  const int64_t rows = rows_of(ys), cols = last_dim(ys);
+  const int d = dt(m), sms = m.ctx->sm_count;
+  out.push_back([=](cudaStream_t s) { return launch_eltwise(d, x, y, rows, cols, sw, p, sms, s); });
+  return MK_OK;
+}
+
+// ------------------------------------------------------------------ row reductions
+bool is_rowop(int32_t k) { return k == MK_OP_LAYERNORM || k == MK_OP_RMSNORM || k == MK_OP_SOFTMAX; }
+int row_mode(int32_t k) { return k == MK_OP_LAYERNORM ? ROW_LAYERNORM : k == MK_OP_RMSNORM ? ROW_RMSNORM : ROW_SOFTMAX; }
+
+bool rowop_match(const Module& m, int lo, int hi) {
+  return is_chain(m, lo, hi) && is_rowop(m.ops[hi - 1].d.kind) && all_eltwise(m, lo, hi - 1);
+}
+mk_status rowop_emit(const Module& m, int lo, int hi, const Resolved& r, std::vector<Launch>& out, std::string& err) {
+  EpiProgram p;
+  mk_status st = build_epi(m, lo, hi - 1, r, p, err);
+  if (st != MK_OK) return st;
+  const Op& op = m.ops[hi - 1];
+  const void* x = r.value_ptr[m.ops[lo].in_id[0]];
+  void* y = r.value_ptr[op.out_id];
+  const mk_tensor_spec& ys = m.vspec(op.out_id);
+  const int64_t rows = rows_of(ys), n = last_dim(ys);
+  const void* g = op.param[0].set ? op.param[0].ptr : nullptr;
+  const void* b = op.param[1].set ? op.param[1].ptr : nullptr;
+  const float eps = (float)op.d.f[0];
+  const int mode = row_mode(op.d.kind), d = dt(m);
+  out.push_back([=](cudaStream_t s) { return launch_rowop(d, mode, x, y, rows, n, g, b, eps, p, s); });
+  return MK_OK;
+}
+
+// ------------------------------------------------------------------ GroupNorm (two launches + scratch)
+bool groupnorm_match(const Module& m, int lo, int hi) {
+  return is_chain(m, lo, hi) && m.ops[hi - 1].d.kind == MK_OP_GROUPNORM && all_eltwise(m, lo, hi - 1);
+}
+size_t groupnorm_scratch(const Module& m, int, int hi) {
+  const mk_tensor_spec& s = m.vspec(m.ops[hi - 1].out_id);
+  return groupnorm_scratch_bytes(s.shape[0], s.shape[1] * s.shape[2], s.shape[3], m.ops[hi - 1].d.i[0], m.ctx->sm_count);
+}
+mk_status groupnorm_emit(const Module& m, int lo, int hi, const Resolved& r, std::vector<Launch>& out, std::string& err) {
+  EpiProgram p;
+  mk_status st = build_epi(m, lo, hi - 1, r, p, err);
+  if (st != MK_OK) return st;
+  const Op& op = m.ops[hi - 1];
+  const void* x = r.value_ptr[m.ops[lo].in_id[0]];
+  void* y = r.value_ptr[op.out_id];
+  const mk_tensor_spec& s = m.vspec(op.out_id);
+  const int64_t nb = s.shape[0], hw = s.shape[1] * s.shape[2], c = s.shape[3];
+  const int groups = op.d.i[0];
+  const void* g = op.param[0].set ? op.param[0].ptr : nullptr;
+  const void* b = op.param[1].set ? op.param[1].ptr : nullptr;
+  const float eps = (float)op.d.f[0];
+  const int d = dt(m);
+  const int chunks = groupnorm_chunks(nb, hw, m.ctx->sm_count);
+  float* scratch = (float*)r.scratch;
+  out.push_back([=](cudaStream_t st_) { return launch_groupnorm_stats(d, x, nb, hw, c, groups, p, scratch, chunks, st_); });
+  out.push_back([=](cudaStream_t st_) { return launch_groupnorm_apply(d, x, y, nb, hw, c, groups, g, b, eps, p, scratch, chunks, st_); });
+  return MK_OK;
+}
+
+// ------------------------------------------------------------------ GEMM family
+// LINEAR [SWIGLU] [elementwise]*
+bool gemm_shape(const Module& m, int lo, int hi, bool* swiglu, int* tail_lo) {
+  if (!is_chain(m, lo, hi) || m.ops[lo].d.kind != MK_OP_LINEAR) return false;
+  int t = lo + 1;
+  *swiglu = t < hi && m.ops[t].d.kind == MK_OP_SWIGLU;
+  if (*swiglu) ++t;
+  *tail_lo = t;
+  return all_eltwise(m, t, hi);
+}
+bool gemm_simt_match(const Module& m, int lo, int hi) {
+  bool sw; int t;
+  return gemm_shape(m, lo, hi, &sw, &t);
+}
+mk_status gemm_simt_emit(const Module& m, int lo, int hi, const Resolved& r, std::vector<Launch>& out, std::string& err) {
+  bool sw; int t;
+  gemm_shape(m, lo, hi, &sw, &t);
+  EpiProgram p;
+  mk_status st = build_epi(m, t, hi, r, p, err);
+  if (st != MK_OK) return st;
+  const Op& op = m.ops[lo];
+  const void* a = r.value_ptr[op.in_id[0]];
+  const void* w = op.param[0].ptr;
+  void* y = r.value_ptr[m.ops[hi - 1].out_id];
+  const mk_tensor_spec& xs = m.vspec(op.in_id[0]);
+  const int64_t M = xs.shape[0], K = xs.shape[1], N = last_dim(m.vspec(m.ops[hi - 1].out_id));
+  const bool wt = op.d.i[1] == MK_LAYOUT_TRANSPOSED;
+  const int d = dt(m);
+  out.push_back([=](cudaStream_t s) { return launch_gemm_simt(d, a, w, wt, y, M, N, K, sw, p, s); });
+  return MK_OK;
+}
+
+// LINEAR [elementwise]* (LAYERNORM | RMSNORM), fp32, one CTA owns whole rows
+bool linear_rownorm_match(const Module& m, int lo, int hi) {
+  if (hi - lo < 2 || !is_chain(m, lo, hi) || m.ops[lo].d.kind != MK_OP_LINEAR) return false;
+  const int32_t k = m.ops[hi - 1].d.kind;
+  if (k != MK_OP_LAYERNORM && k != MK_OP_RMSNORM) return false;
+  if (!all_eltwise(m, lo + 1, hi - 1)) return false;
+  if (m.values[0].spec.dtype != MK_F32) return false;
+  return m.ops[lo].d.i[0] <= 1024;
+}
+mk_status linear_rownorm_emit(const Module& m, int lo, int hi, const Resolved& r, std::vector<Launch>& out, std::string& err) {
+  EpiProgram p;
+  mk_status st = build_epi(m, lo + 1, hi - 1, r, p, err);
+  if (st != MK_OK) return st;
+  const Op& op = m.ops[lo];
+  const Op& nop = m.ops[hi - 1];
+  const void* a = r.value_ptr[op.in_id[0]];
+  const void* w = op.param[0].ptr;
+  void* y = r.value_ptr[nop.out_id];
+  const mk_tensor_spec& xs = m.vspec(op.in_id[0]);
+  const int64_t M = xs.shape[0], K = xs.shape[1], N = op.d.i[0];
+  const bool wt = op.d.i[1] == MK_LAYOUT_TRANSPOSED;
+  const void* g = nop.param[0].set ? nop.param[0].ptr : nullptr;
+  const void* b = nop.param[1].set ? nop.param[1].ptr : nullptr;
+  const float eps = (float)nop.d.f[0];
+  const int mode = row_mode(nop.d.kind), d = dt(m);
+  out.push_back([=](cudaStream_t s) { return launch_linear_rownorm_simt(d, a, w, wt, y, M, N, K, p, mode, g, b, eps, s); });
+  return MK_OK;
+}
+
+// ------------------------------------------------------------------ convolution
+bool conv_simt_match(const Module& m, int lo, int hi) {
+  return is_chain(m, lo, hi) && m.ops[lo].d.kind == MK_OP_CONV2D_3X3 && all_eltwise(m, lo + 1, hi);
+}
+mk_status conv_simt_emit(const Module& m, int lo, int hi, const Resolved& r, std::vector<Launch>& out, std::string& err) {
+  EpiProgram p;
+  mk_status st = build_epi(m, lo + 1, hi, r, p, err);
+  if (st != MK_OK) return st;
+  const Op& op = m.ops[lo];
+  const void* x = r.value_ptr[op.in_id[0]];
+  const void* w = op.param[0].ptr;
+  void* y = r.value_ptr[m.ops[hi - 1].out_id];
+  const mk_tensor_spec& xs = m.vspec(op.in_id[0]);
+  const int64_t nb = xs.shape[0], h = xs.shape[1], wd = xs.shape[2], c = xs.shape[3], co = op.d.i[0];
+  const int d = dt(m);
+  out.push_back([=](cudaStream_t s) { return launch_conv3x3_simt(d, x, w, y, nb, h, wd, c, co, p, s); });
+  return MK_OK;
+}
+
+// ------------------------------------------------------------------ attention
+AttnView attn_view(const Module& m, const Op& op, const Resolved& r) {
+  AttnView a{};
+  const int64_t H = op.d.i[0], D = op.d.i[1];
+  const size_t es = dtype_size(m.values[0].spec.dtype);
+  if (op.d.i[2] == 0) {
+    const mk_tensor_spec& q = m.vspec(op.in_id[0]);
+    a.q = r.value_ptr[op.in_id[0]];
+    a.k = r.value_ptr[op.in_id[1]];
+    a.v = r.value_ptr[op.in_id[2]];
+    a.B = q.shape[0]; a.H = H; a.S = q.shape[2]; a.D = D;
+    a.sb = H * a.S * D; a.sh = a.S * D; a.ss = D;
+  } else {
+    const char* base = (const char*)r.value_ptr[op.in_id[0]];
+    const int64_t E = H * D;
+    a.q = base;
+    a.k = base + E * es;
+    a.v = base + 2 * E * es;
+    a.B = op.d.i[2]; a.H = H; a.S = op.d.i[3]; a.D = D;
+    a.sb = a.S * 3 * E; a.sh = D; a.ss = 3 * E;
+  }
+  return a;
+}
+bool attn_simt_match(const Module& m, int lo, int hi) {
+  return hi - lo == 1 && m.ops[lo].d.kind == MK_OP_ATTENTION_CAUSAL && m.ops[lo].d.i[1] <= 256;
+}
+mk_status attn_simt_emit(const Module& m, int lo, int, const Resolved& r, std::vector<Launch>& out, std::string&) {
+  const Op& op = m.ops[lo];
+  const AttnView a = attn_view(m, op, r);
+  void* o = r.value_ptr[op.out_id];
+  const int d = dt(m);
+  out.push_back([=](cudaStream_t s) { return launch_attention_simt(d, a, o, s); });
+  return MK_OK;
+}
+
+}  // namespace
+
+const std::vector<Impl>& registry() {
+  static const std::vector<Impl> reg = {
+      {"linear_rownorm_simt", linear_rownorm_match, no_scratch, linear_rownorm_emit},
+      {"gemm_simt", gemm_simt_match, no_scratch, gemm_simt_emit},
+      {"conv3x3_simt", conv_simt_match, no_scratch, conv_simt_emit},
+      {"attention_simt", attn_simt_match, no_scratch, attn_simt_emit},
+      {"rowop", rowop_match, no_scratch, rowop_emit},
+      {"groupnorm_nhwc", groupnorm_match, groupnorm_scratch, groupnorm_emit},
+      {"eltwise", eltwise_match, no_scratch, eltwise_emit},
+  };
+  return reg;
+}
+
+}  // namespace mk

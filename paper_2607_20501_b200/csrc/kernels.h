@@ -1,0 +1,94 @@
+// Host-callable launchers of the sm_100a kernels.  One function = one kernel launch on the
+// given stream; none of them allocates, synchronises or copies.  Pointers are device pointers.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+namespace mk {
+
+// dtype codes mirror mk_dtype
+constexpr int DT_F32 = 0;
+constexpr int DT_BF16 = 1;
+
+// ---- elementwise program: the tail a producing kernel applies before its store -----------------
+// (paper, decomposition rules: GEMM + elementwise, elementwise chains, bias after matmul and the
+// residual add are fused into one subkernel)
+enum EpiKind : int32_t {
+  EPI_BIAS = 1,      // v += bias[col]            ptr = bias vector
+  EPI_RELU = 2,
+  EPI_GELU_TANH = 3,
+  EPI_SILU = 4,
+  EPI_SCALE = 5,     // v *= a
+  EPI_CLAMP = 6,     // v = min(max(v, a), b)
+  EPI_RESIDUAL = 7   // v += res[row * ld + col]  ptr = residual tensor, ld = output width
+};
+constexpr int EPI_MAX = 8;
+struct EpiOp {
+  int32_t kind;
+  float a, b;
+  int32_t pad;
+  const void* ptr;
+};
+struct EpiProgram {
+  int32_t n = 0;
+  int32_t dtype = DT_BF16;  // element type behind ptr
+  EpiOp op[EPI_MAX];
+};
+
+// ---- device status word (bounded-wait expiry codes) --------------------------------------------------
+unsigned int* kernel_status_ptr();   // device address, nullptr without a device
+cudaError_t kernel_status_fetch_and_clear(unsigned int* out);
+
+// ---- HBM-bound kernels ------------------------------------------------------------------------------
+// y[rows, cols] = program(x).  swiglu: x is [rows, 2*cols] = [gate | up] and the program runs on
+// silu(gate) * up.
+cudaError_t launch_eltwise(int dtype, const void* x, void* y, int64_t rows, int64_t cols, bool swiglu,
+                           const EpiProgram& p, int sm_count, cudaStream_t s);
+
+enum RowMode : int32_t { ROW_LAYERNORM = 0, ROW_RMSNORM = 1, ROW_SOFTMAX = 2 };
+// Row-wise reduction over the last dimension of program(x)[rows, n]; gamma/beta may be null.
+cudaError_t launch_rowop(int dtype, int mode, const void* x, void* y, int64_t rows, int64_t n,
+                         const void* gamma, const void* beta, float eps, const EpiProgram& pre,
+                         cudaStream_t s);
+
+// GroupNorm over NHWC [nb, hw, c]: stats writes per-(image, chunk, group) partial sums into
+// scratch, apply reduces them and normalises.  scratch must hold groupnorm_scratch_bytes().
+int groupnorm_chunks(int64_t nb, int64_t hw, int sm_count);
+size_t groupnorm_scratch_bytes(int64_t nb, int64_t hw, int64_t c, int groups, int sm_count);
+cudaError_t launch_groupnorm_stats(int dtype, const void* x, int64_t nb, int64_t hw, int64_t c,
+                                   int groups, const EpiProgram& pre, float* scratch, int chunks,
+                                   cudaStream_t s);
+cudaError_t launch_groupnorm_apply(int dtype, const void* x, void* y, int64_t nb, int64_t hw,
+                                   int64_t c, int groups, const void* gamma, const void* beta,
+                                   float eps, const EpiProgram& pre, const float* scratch, int chunks,
+                                   cudaStream_t s);
+
+// ---- plain-ALU (SIMT) kernels: any shape, fp32 or bf16, fp32 accumulation -------------------------
+// Y[M, N] = program(A[M, K] @ W); W is [K, N] row-major, or [N, K] when w_transposed.
+// swiglu: W has 2N logical columns [gate | up] and Y = program(silu(A Wg) * (A Wu)).
+cudaError_t launch_gemm_simt(int dtype, const void* a, const void* w, bool w_transposed, void* y,
+                             int64_t m, int64_t n, int64_t k, bool swiglu, const EpiProgram& p,
+                             cudaStream_t s);
+// Small-shape fused chain: one CTA owns whole rows, so the row norm follows the GEMM in-kernel.
+// Y = rownorm(program(A @ W)); n <= 1024.
+cudaError_t launch_linear_rownorm_simt(int dtype, const void* a, const void* w, bool w_transposed,
+                                       void* y, int64_t m, int64_t n, int64_t k, const EpiProgram& p,
+                                       int mode, const void* gamma, const void* beta, float eps,
+                                       cudaStream_t s);
+cudaError_t launch_conv3x3_simt(int dtype, const void* x, const void* w, void* y, int64_t nb, int64_t h,
+                                int64_t wd, int64_t c, int64_t co, const EpiProgram& p, cudaStream_t s);
+
+// Strided view of Q, K, V: element (b, h, s, d) sits at base + b*sb + h*sh + s*ss + d (elements).
+struct AttnView {
+  const void* q;
+  const void* k;
+  const void* v;
+  int64_t sb, sh, ss;
+  int64_t B, H, S, D;
+};
+// O is the dense [B*S, H*D] matrix.
+cudaError_t launch_attention_simt(int dtype, const AttnView& a, void* o, cudaStream_t s);
+
+}  // namespace mk

@@ -1,0 +1,312 @@
+// Plain-ALU subkernels: any shape, fp32 or bf16 storage, fp32 FMA accumulation (no TF32: the fp32
+// tolerance rtol 1e-4 / atol 1e-5 rules it out, as the paper's own fp32 setting does).  They are the
+// always-legal implementations the composer falls back to for shapes the tensor-core kernels do
+// not take, the alternatives a submodule can be swapped to, and — for the small fp32 chain — the
+// fused single-launch kernel in which one CTA owns whole rows so the row norm needs no second pass
+// over memory.
+#include "device_common.cuh"
+
+namespace mk {
+
+// =====================================================================================================
+// tiled GEMM, 64x64 tile, 16x16 threads, 4x4 micro-tile
+// =====================================================================================================
+template <typename T, bool SWIGLU>
+__global__ void __launch_bounds__(256) gemm_simt_kernel(const T* __restrict__ a, const T* __restrict__ w, bool wt,
+                                                        T* __restrict__ y, int64_t M, int64_t N, int64_t K,
+                                                        const __grid_constant__ EpiProgram p) {
+  constexpr int BM = 64, BN = 64, BK = 16;
+  __shared__ float As[BK][BM + 1];
+  __shared__ float Ws[SWIGLU ? 2 : 1][BK][BN + 1];
+  const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;
+  const int64_t m0 = (int64_t)blockIdx.y * BM, n0 = (int64_t)blockIdx.x * BN;
+  const int64_t ldw = SWIGLU ? 2 * N : N;  // logical columns of W
+  float acc[4][4] = {};
+  float acc2[SWIGLU ? 4 : 1][4] = {};
+  for (int64_t k0 = 0; k0 < K; k0 += BK) {
+    for (int i = threadIdx.x; i < BM * BK; i += 256) {
+      const int mm = i / BK, kk = i % BK;
+      const int64_t gm = m0 + mm, gk = k0 + kk;
+      As[kk][mm] = (gm < M && gk < K) ? Elem<T>::ld(a + gm * K + gk) : 0.0f;
+    }
+    for (int i = threadIdx.x; i < BN * BK; i += 256) {
+      int nn, kk;
+      if (wt) { nn = i / BK; kk = i % BK; } else { kk = i / BN; nn = i % BN; }
+      const int64_t gn = n0 + nn, gk = k0 + kk;
+      const bool ok = gn < N && gk < K;
+      Ws[0][kk][nn] = ok ? Elem<T>::ld(wt ? w + gn * K + gk : w + gk * ldw + gn) : 0.0f;
+      if (SWIGLU) Ws[1][kk][nn] = ok ? Elem<T>::ld(wt ? w + (N + gn) * K + gk : w + gk * ldw + N + gn) : 0.0f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < BK; ++kk) {
+      float av[4], bv[4], cv[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) av[i] = As[kk][ty * 4 + i];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        bv[j] = Ws[0][kk][tx * 4 + j];
+        if (SWIGLU) cv[j] = Ws[1][kk][tx * 4 + j];
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+          if (SWIGLU) acc2[i][j] = fmaf(av[i], cv[j], acc2[i][j]);
+        }
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int64_t gm = m0 + ty * 4 + i, gn = n0 + tx * 4 + j;
+      if (gm < M && gn < N) {
+        float v = acc[i][j];
+        if (SWIGLU) v = silu_f(v) * acc2[i][j];
+        Elem<T>::st(y + gm * N + gn, epi_apply(p, v, gm, gn, N));
+      }
+    }
+}
+
+template <typename T>
+static cudaError_t gemm_simt_dispatch(const void* a, const void* w, bool wt, void* y, int64_t m, int64_t n, int64_t k, bool swiglu,
+                                      const EpiProgram& p, cudaStream_t s) {
+  if (m == 0 || n == 0) return cudaSuccess;
+  dim3 grid((unsigned)((n + 63) / 64), (unsigned)((m + 63) / 64));
+  if (swiglu) gemm_simt_kernel<T, true><<<grid, 256, 0, s>>>((const T*)a, (const T*)w, wt, (T*)y, m, n, k, p);
+  else gemm_simt_kernel<T, false><<<grid, 256, 0, s>>>((const T*)a, (const T*)w, wt, (T*)y, m, n, k, p);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_gemm_simt(int dtype, const void* a, const void* w, bool w_transposed, void* y, int64_t m, int64_t n, int64_t k,
+                             bool swiglu, const EpiProgram& p, cudaStream_t s) {
+  return dtype == DT_F32 ? gemm_simt_dispatch<float>(a, w, w_transposed, y, m, n, k, swiglu, p, s)
+                         : gemm_simt_dispatch<__nv_bfloat16>(a, w, w_transposed, y, m, n, k, swiglu, p, s);
+}
+
+// =====================================================================================================
+// small-shape fused chain: linear -> elementwise tail -> row norm, one launch
+// CTA = LR_ROWS rows x all N columns; K is split over LR_THREADS / NT thread groups whose partial
+// sums meet in shared memory; then one warp per row normalises.
+// =====================================================================================================
+constexpr int LR_ROWS = 2;
+constexpr int LR_THREADS = 512;
+constexpr int LR_MAXC = 4;  // columns per thread: N <= NT * LR_MAXC
+
+template <typename T>
+__global__ void __launch_bounds__(LR_THREADS) linear_rownorm_kernel(const T* __restrict__ a, const T* __restrict__ w, bool wt,
+                                                                    T* __restrict__ y, int M, int N, int K, int NT,
+                                                                    const __grid_constant__ EpiProgram p, int mode,
+                                                                    const T* __restrict__ gamma, const T* __restrict__ beta,
+                                                                    float eps) {
+  extern __shared__ float smem[];
+  float* xs = smem;                         // [LR_ROWS][K]
+  float* part = smem + LR_ROWS * K;         // [KS][LR_ROWS][N]
+  const int KS = LR_THREADS / NT;
+  const int ct = threadIdx.x % NT, ks = threadIdx.x / NT;
+  const int m0 = blockIdx.x * LR_ROWS;
+  for (int i = threadIdx.x; i < LR_ROWS * K; i += LR_THREADS) {
+    const int r = i / K, k = i - r * K;
+    xs[i] = (m0 + r < M) ? Elem<T>::ld(a + (int64_t)(m0 + r) * K + k) : 0.0f;
+  }
+  __syncthreads();
+  const int kper = (K + KS - 1) / KS;
+  const int kb = ks * kper, ke = min(K, kb + kper);
+  float acc[LR_ROWS][LR_MAXC] = {};
+  if (ks < KS) {
+#pragma unroll 8
+    for (int k = kb; k < ke; ++k) {
+      float wv[LR_MAXC];
+#pragma unroll
+      for (int j = 0; j < LR_MAXC; ++j) {
+        const int c = ct + j * NT;
+        wv[j] = (c < N) ? Elem<T>::ld(wt ? w + (int64_t)c * K + k : w + (int64_t)k * N + c) : 0.0f;
+      }
+#pragma unroll
+      for (int r = 0; r < LR_ROWS; ++r)
+#pragma unroll
+        for (int j = 0; j < LR_MAXC; ++j) acc[r][j] = fmaf(xs[r * K + k], wv[j], acc[r][j]);
+    }
+#pragma unroll
+    for (int r = 0; r < LR_ROWS; ++r)
+#pragma unroll
+      for (int j = 0; j < LR_MAXC; ++j) {
+        const int c = ct + j * NT;
+        if (c < N) part[(ks * LR_ROWS + r) * N + c] = acc[r][j];
+      }
+  }
+  __syncthreads();
+  // sum the K-slices in a fixed order, apply the elementwise tail; result overwrites slice 0
+  for (int i = threadIdx.x; i < LR_ROWS * N; i += LR_THREADS) {
+    const int r = i / N, c = i - r * N;
+    float v = 0.0f;
+    for (int q = 0; q < KS; ++q) v += part[(q * LR_ROWS + r) * N + c];
+    part[r * N + c] = epi_apply(p, v, m0 + r, c, N);
+  }
+  __syncthreads();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (warp < LR_ROWS && m0 + warp < M) {
+    const float* row = part + warp * N;
+    const float inv_n = 1.0f / (float)N;
+    float mean = 0.0f;
+    if (mode == ROW_LAYERNORM) {
+      float s = 0.0f;
+      for (int c = lane; c < N; c += 32) s += row[c];
+      mean = warp_sum(s) * inv_n;
+    }
+    float q = 0.0f;
+    for (int c = lane; c < N; c += 32) { const float d = row[c] - mean; q += d * d; }
+    const float rstd = rsqrtf(warp_sum(q) * inv_n + eps);
+    T* yr = y + (int64_t)(m0 + warp) * N;
+    for (int c = lane; c < N; c += 32) {
+      float o = (row[c] - mean) * rstd;
+      if (gamma) o *= Elem<T>::ld(gamma + c);
+      if (mode == ROW_LAYERNORM && beta) o += Elem<T>::ld(beta + c);
+      Elem<T>::st(yr + c, o);
+    }
+  }
+}
+
+template <typename T>
+static cudaError_t linear_rownorm_dispatch(const void* a, const void* w, bool wt, void* y, int64_t m, int64_t n, int64_t k,
+                                           const EpiProgram& p, int mode, const void* g, const void* b, float eps,
+                                           cudaStream_t s) {
+  if (m == 0) return cudaSuccess;
+  int NT = 32;
+  while (NT < n && NT < 256) NT *= 2;
+  if ((int64_t)NT * LR_MAXC < n) return cudaErrorInvalidValue;
+  const int KS = LR_THREADS / NT;
+  const size_t smem = sizeof(float) * ((size_t)LR_ROWS * k + (size_t)KS * LR_ROWS * n);
+  if (smem > 200 * 1024) return cudaErrorInvalidValue;
+  static bool attr_f32 = false, attr_bf16 = false;
+  bool& done = sizeof(T) == 4 ? attr_f32 : attr_bf16;
+  if (!done) {
+    cudaError_t e = cudaFuncSetAttribute(linear_rownorm_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e != cudaSuccess) return e;
+    done = true;
+  }
+  const int grid = (int)((m + LR_ROWS - 1) / LR_ROWS);
+  linear_rownorm_kernel<T><<<grid, LR_THREADS, smem, s>>>((const T*)a, (const T*)w, wt, (T*)y, (int)m, (int)n, (int)k, NT, p, mode,
+                                                          (const T*)g, (const T*)b, eps);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_linear_rownorm_simt(int dtype, const void* a, const void* w, bool w_transposed, void* y, int64_t m, int64_t n,
+                                       int64_t k, const EpiProgram& p, int mode, const void* gamma, const void* beta, float eps,
+                                       cudaStream_t s) {
+  return dtype == DT_F32 ? linear_rownorm_dispatch<float>(a, w, w_transposed, y, m, n, k, p, mode, gamma, beta, eps, s)
+                         : linear_rownorm_dispatch<__nv_bfloat16>(a, w, w_transposed, y, m, n, k, p, mode, gamma, beta, eps, s);
+}
+
+// =====================================================================================================
+// direct 3x3 convolution, NHWC, one thread per output element
+// =====================================================================================================
+template <typename T>
+__global__ void __launch_bounds__(256) conv3x3_simt_kernel(const T* __restrict__ x, const T* __restrict__ w, T* __restrict__ y,
+                                                           int64_t nb, int h, int wd, int c, int co,
+                                                           const __grid_constant__ EpiProgram p) {
+  const int64_t total = nb * h * wd * co;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    const int o = (int)(i % co);
+    const int64_t pix = i / co;
+    const int px = (int)(pix % wd);
+    const int py = (int)((pix / wd) % h);
+    const int64_t n = pix / ((int64_t)wd * h);
+    float acc = 0.0f;
+    for (int a = 0; a < 3; ++a) {
+      const int iy = py + a - 1;
+      if (iy < 0 || iy >= h) continue;
+      for (int b = 0; b < 3; ++b) {
+        const int ix = px + b - 1;
+        if (ix < 0 || ix >= wd) continue;
+        const T* xp = x + ((n * h + iy) * wd + ix) * c;
+        const T* wp = w + ((int64_t)(o * 3 + a) * 3 + b) * c;
+        for (int ch = 0; ch < c; ++ch) acc = fmaf(Elem<T>::ld(xp + ch), Elem<T>::ld(wp + ch), acc);
+      }
+    }
+    Elem<T>::st(y + i, epi_apply(p, acc, pix, o, co));
+  }
+}
+
+cudaError_t launch_conv3x3_simt(int dtype, const void* x, const void* w, void* y, int64_t nb, int64_t h, int64_t wd, int64_t c,
+                                int64_t co, const EpiProgram& p, cudaStream_t s) {
+  const int64_t total = nb * h * wd * co;
+  if (total == 0) return cudaSuccess;
+  int64_t g = (total + 255) / 256;
+  if (g > 148 * 64) g = 148 * 64;
+  if (dtype == DT_F32)
+    conv3x3_simt_kernel<float><<<(unsigned)g, 256, 0, s>>>((const float*)x, (const float*)w, (float*)y, nb, (int)h, (int)wd, (int)c, (int)co, p);
+  else
+    conv3x3_simt_kernel<__nv_bfloat16><<<(unsigned)g, 256, 0, s>>>((const __nv_bfloat16*)x, (const __nv_bfloat16*)w, (__nv_bfloat16*)y, nb,
+                                                                   (int)h, (int)wd, (int)c, (int)co, p);
+  return cudaGetLastError();
+}
+
+// =====================================================================================================
+// causal attention, one warp per (batch, head, query); online softmax over the keys j <= i
+// =====================================================================================================
+template <typename T>
+__global__ void __launch_bounds__(128) attention_simt_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
+                                                             T* __restrict__ o, int64_t sb, int64_t sh, int64_t ss, int64_t B, int H,
+                                                             int S, int D) {
+  constexpr int MAXE = 8;  // D <= 256
+  const int lane = threadIdx.x & 31;
+  const int64_t wid = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (wid >= B * H * S) return;
+  const int i = (int)(wid % S);
+  const int h = (int)((wid / S) % H);
+  const int64_t b = wid / ((int64_t)S * H);
+  const int64_t base = b * sb + h * sh;
+  float qv[MAXE], acc[MAXE];
+#pragma unroll
+  for (int e = 0; e < MAXE; ++e) {
+    const int d = lane + 32 * e;
+    qv[e] = d < D ? Elem<T>::ld(q + base + i * ss + d) : 0.0f;
+    acc[e] = 0.0f;
+  }
+  const float scale = rsqrtf((float)D);
+  float m = -INFINITY, l = 0.0f;
+  for (int j = 0; j <= i; ++j) {
+    float dot = 0.0f;
+#pragma unroll
+    for (int e = 0; e < MAXE; ++e) {
+      const int d = lane + 32 * e;
+      if (d < D) dot = fmaf(qv[e], Elem<T>::ld(k + base + j * ss + d), dot);
+    }
+    const float sc = warp_sum(dot) * scale;
+    const float mn = fmaxf(m, sc);
+    const float alpha = expf(m - mn), pj = expf(sc - mn);
+    l = l * alpha + pj;
+#pragma unroll
+    for (int e = 0; e < MAXE; ++e) {
+      const int d = lane + 32 * e;
+      if (d < D) acc[e] = acc[e] * alpha + pj * Elem<T>::ld(v + base + j * ss + d);
+    }
+    m = mn;
+  }
+  const float inv = 1.0f / l;
+  T* orow = o + ((b * S + i) * H + h) * D;
+#pragma unroll
+  for (int e = 0; e < MAXE; ++e) {
+    const int d = lane + 32 * e;
+    if (d < D) Elem<T>::st(orow + d, acc[e] * inv);
+  }
+}
+
+cudaError_t launch_attention_simt(int dtype, const AttnView& a, void* o, cudaStream_t s) {
+  const int64_t warps = a.B * a.H * a.S;
+  if (warps == 0) return cudaSuccess;
+  const unsigned grid = (unsigned)((warps + 3) / 4);
+  if (dtype == DT_F32)
+    attention_simt_kernel<float><<<grid, 128, 0, s>>>((const float*)a.q, (const float*)a.k, (const float*)a.v, (float*)o, a.sb, a.sh, a.ss, a.B,
+                                                      (int)a.H, (int)a.S, (int)a.D);
+  else
+    attention_simt_kernel<__nv_bfloat16><<<grid, 128, 0, s>>>((const __nv_bfloat16*)a.q, (const __nv_bfloat16*)a.k, (const __nv_bfloat16*)a.v,
+                                                              (__nv_bfloat16*)o, a.sb, a.sh, a.ss, a.B, (int)a.H, (int)a.S, (int)a.D);
+  return cudaGetLastError();
+}
+
+}  // namespace mk

@@ -136,7 +136,7 @@ def c1(seed=0, M=64, K=256, N=128, dtype="f32") -> Workload:
     w.params["gamma"] = make("gamma", dtype, np.ones((N,), np.float32))
     w.params["beta"] = make("beta", dtype, np.zeros((N,), np.float32))
     w.ops = [
-        _op("linear", "y0", ["x"], {"w": "W"}),
+        _op("linear", "y0", ["x"], {"w": "W"}, n=N),
         _op("bias_add", "y1", ["y0"], {"b": "b"}),
         _op("relu", "y2", ["y1"]),
         _op("layernorm", "y3", ["y2"], {"gamma": "gamma", "beta": "beta"}, eps=1e-5),
@@ -157,7 +157,7 @@ def c2(seed=0, M=4096, K=4096, N=4096, dtype="bf16") -> Workload:
     w.params["W"] = make("W", dtype, _normal(seed, 1, (K, N), std=(1.0 / K) ** 0.5))
     w.params["bias"] = make("bias", dtype, _normal(seed, 2, (N,), std=0.02))
     w.ops = [
-        _op("linear", "y0", ["x"], {"w": "W"}),
+        _op("linear", "y0", ["x"], {"w": "W"}, n=N),
         _op("bias_add", "y1", ["y0"], {"b": "bias"}),
         _op("gelu_tanh", "y2", ["y1"]),
         _op("scale", "y3", ["y2"], s=0.5),
@@ -182,7 +182,7 @@ def c3(seed=0, NB=32, H=56, W=56, C=128, CO=128, G=32, dtype="bf16") -> Workload
     w.params["gamma"] = make("gamma", dtype, _normal(seed, 3, (CO,), mean=1.0, std=0.02))
     w.params["beta"] = make("beta", dtype, _normal(seed, 4, (CO,), std=0.02))
     w.ops = [
-        _op("conv2d_3x3", "y0", ["x"], {"w": "Wc"}),
+        _op("conv2d_3x3", "y0", ["x"], {"w": "Wc"}, c_out=CO),
         _op("bias_add", "y1", ["y0"], {"b": "bias"}),
         _op("relu", "y2", ["y1"]),
         _op("groupnorm", "y3", ["y2"], {"gamma": "gamma", "beta": "beta"}, groups=G, eps=1e-5),
@@ -208,7 +208,7 @@ def c4(seed=0, B=16, H=16, S=2048, D=128, dtype="bf16") -> Workload:
     w.ops = [
         # attention output is logically [B*S, H*D], head-major columns
         _op("attention_causal", "a", ["q", "k", "v"], layout="bhsd", heads=H, head_dim=D),
-        _op("linear", "p", ["a"], {"w": "Wo"}),
+        _op("linear", "p", ["a"], {"w": "Wo"}, n=E),
         _op("residual_add", "h", ["p", "r"]),
         _op("rmsnorm", "y", ["h"], {"gamma": "gamma"}, eps=1e-6),
     ]
@@ -239,15 +239,15 @@ def c5(seed=0, B=8, S=1024, E=2048, H=16, F=8192, L=4, dtype="bf16") -> Workload
         tid += 4
         w.ops += [
             _op("rmsnorm", f"n1_{l}", [cur], {"gamma": "ones"}, eps=1e-6),
-            _op("linear", f"qkv_{l}", [f"n1_{l}"], {"w": f"Wqkv{l}"}),
+            _op("linear", f"qkv_{l}", [f"n1_{l}"], {"w": f"Wqkv{l}"}, n=3 * E),
             _op("attention_causal", f"att_{l}", [f"qkv_{l}"], layout="packed_qkv", heads=H,
                 head_dim=D, batch=B, seq=S),
-            _op("linear", f"o_{l}", [f"att_{l}"], {"w": f"Wo{l}"}),
+            _op("linear", f"o_{l}", [f"att_{l}"], {"w": f"Wo{l}"}, n=E),
             _op("residual_add", f"x1_{l}", [f"o_{l}", cur]),
             _op("rmsnorm", f"n2_{l}", [f"x1_{l}"], {"gamma": "ones"}, eps=1e-6),
-            _op("linear", f"gu_{l}", [f"n2_{l}"], {"w": f"Wgu{l}"}),
+            _op("linear", f"gu_{l}", [f"n2_{l}"], {"w": f"Wgu{l}"}, n=2 * F),
             _op("swiglu", f"hid_{l}", [f"gu_{l}"]),
-            _op("linear", f"d_{l}", [f"hid_{l}"], {"w": f"Wd{l}"}),
+            _op("linear", f"d_{l}", [f"hid_{l}"], {"w": f"Wd{l}"}, n=E),
             _op("residual_add", f"x2_{l}", [f"d_{l}", f"x1_{l}"]),
         ]
         cur = f"x2_{l}"
