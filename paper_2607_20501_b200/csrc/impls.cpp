@@ -5,7 +5,10 @@
 // used blocks fusion unless one CTA owns the whole row).
 //
 // Order = the composer's preference among implementations that accept the same range.
+#include <memory>
+
 #include "mk_internal.h"
+#include "tc_plans.h"
 
 namespace mk {
 namespace {
@@ -143,6 +146,34 @@ mk_status gemm_simt_emit(const Module& m, int lo, int hi, const Resolved& r, std
   return MK_OK;
 }
 
+// tcgen05 GEMM: bf16, W stored [N, K], 16-byte rows
+bool gemm_tc_match(const Module& m, int lo, int hi) {
+  bool sw; int t;
+  if (!gemm_shape(m, lo, hi, &sw, &t)) return false;
+  if (m.values[0].spec.dtype != MK_BF16) return false;
+  const Op& op = m.ops[lo];
+  if (op.d.i[1] != MK_LAYOUT_TRANSPOSED) return false;
+  const int64_t K = m.vspec(op.in_id[0]).shape[1];
+  const int64_t N = last_dim(m.vspec(m.ops[hi - 1].out_id));
+  return K % 8 == 0 && N % 8 == 0;
+}
+mk_status gemm_tc_emit(const Module& m, int lo, int hi, const Resolved& r, std::vector<Launch>& out, std::string& err) {
+  bool sw; int t;
+  gemm_shape(m, lo, hi, &sw, &t);
+  EpiProgram p;
+  mk_status st = build_epi(m, t, hi, r, p, err);
+  if (st != MK_OK) return st;
+  const Op& op = m.ops[lo];
+  const mk_tensor_spec& xs = m.vspec(op.in_id[0]);
+  const int64_t M = xs.shape[0], K = xs.shape[1], N = last_dim(m.vspec(m.ops[hi - 1].out_id));
+  auto plan = std::make_shared<GemmTcPlan>();
+  cudaError_t e = gemm_tc_plan(plan.get(), r.value_ptr[op.in_id[0]], op.param[0].ptr, r.value_ptr[m.ops[hi - 1].out_id], M, N, K, sw, p,
+                               m.ctx->sm_count);
+  if (e != cudaSuccess) { err = std::string("gemm_tc plan: ") + cudaGetErrorString(e); return MK_ERR_CUDA; }
+  out.push_back([plan](cudaStream_t s) { return launch_gemm_tc(*plan, s); });
+  return MK_OK;
+}
+
 // LINEAR [elementwise]* (LAYERNORM | RMSNORM), fp32, one CTA owns whole rows
 bool linear_rownorm_match(const Module& m, int lo, int hi) {
   if (hi - lo < 2 || !is_chain(m, lo, hi) || m.ops[lo].d.kind != MK_OP_LINEAR) return false;
@@ -231,6 +262,7 @@ mk_status attn_simt_emit(const Module& m, int lo, int, const Resolved& r, std::v
 const std::vector<Impl>& registry() {
   static const std::vector<Impl> reg = {
       {"linear_rownorm_simt", linear_rownorm_match, no_scratch, linear_rownorm_emit},
+      {"gemm_tc", gemm_tc_match, no_scratch, gemm_tc_emit},
       {"gemm_simt", gemm_simt_match, no_scratch, gemm_simt_emit},
       {"conv3x3_simt", conv_simt_match, no_scratch, conv_simt_emit},
       {"attention_simt", attn_simt_match, no_scratch, attn_simt_emit},
