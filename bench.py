@@ -1,0 +1,365 @@
+#!/usr/bin/env python
+"""Benchmark of the composed forward (one JSON line on stdout).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload c2]
+
+A step is one composed forward of the workload's module (every submodule of its default
+decomposition) over one batch of seeded synthetic input.  `value` is the whole-job throughput in
+TFLOP/s of algorithmic work with inputs resident in HBM; `e2e` repeats the measurement with the
+step's inputs copied from pinned host memory and its result copied back inside the timed region.
+Each step works on a different copy of the inputs and outputs (a rotation larger than L2), so no
+step finds its operands in L2 from the step before.
+
+Under torchrun every rank runs the same workload on its own GPU (independent batches, no
+collective on the data path: weak scaling); times are device times, max over ranks.
+
+`--impl reference` times the fp64 CPU oracle, as it stands, on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "composed-module fwd latency, TFLOP/s & GB/s as % of B200 roofline, per subkernel"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
+# capture summarised under profiles/ (null until a capture of that workload exists)
+NCU_TRAFFIC_BYTES = {}
+
+DEFAULT_STEPS = {"c1": 2000, "c2": 1000, "c3": 1000, "c4": 200, "c5": 50}
+
+
+def full_workload(name, seed=0):
+    import workloads as W
+    return W.generate.WORKLOADS[name](seed)
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        d["_source"] = "measured"
+        return d
+    d = dict(FALLBACK_PEAKS)
+    d["_source"] = "fallback"
+    return d
+
+
+# ----------------------------------------------------------------------------------------------------
+# clocks: sampled on a thread while the timed region runs (read-only NVML queries)
+# ----------------------------------------------------------------------------------------------------
+class ClockSampler:
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
+
+    def __init__(self, index):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._t = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _once(self):
+        try:
+            self.samples.append(self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM))
+            try:
+                r = self.nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+            except Exception:
+                r = self.nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+            for bit, name in self.REASONS.items():
+                if r & bit:
+                    self.reasons.add(name)
+        except Exception:
+            pass
+
+    def _run(self):
+        while not self._stop.is_set():
+            self._once()
+            self._stop.wait(0.02)
+
+    def start(self):
+        if self.nv:
+            self._t = threading.Thread(target=self._run, daemon=True)
+            self._t.start()
+
+    def stop(self):
+        if self._t:
+            self._once()
+            self._stop.set()
+            self._t.join()
+        s = sorted(self.samples)
+        return {"sm_mhz": s[len(s) // 2] if s else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(s)}
+
+
+# ----------------------------------------------------------------------------------------------------
+# CPU oracle legs
+# ----------------------------------------------------------------------------------------------------
+def oracle_sample(name, w, budget_s=12.0):
+    """Time the fp64 oracle on a bounded sample of the workload: a leading block of independent
+    rows / images / batch elements, sized from a short probe to take about `budget_s` seconds.
+    Returns (flops_done, seconds, description)."""
+    import numpy as np
+    from oracle import modules as OM
+
+    def sub(frac_units):
+        import copy
+        s = copy.copy(w)
+        s.inputs = dict(w.inputs)
+        s.ops = [dict(o, attrs=dict(o["attrs"])) for o in w.ops]
+        from workloads.generate import Tensor
+        if name in ("c1", "c2"):
+            rows = frac_units
+            s.inputs["x"] = Tensor("x", w.dtype, w.inputs["x"].store[:rows])
+            total = w.inputs["x"].shape[0]
+            what = f"first {rows} of {total} rows of X"
+        elif name == "c3":
+            s.inputs["x"] = Tensor("x", w.dtype, w.inputs["x"].store[:frac_units])
+            total = w.inputs["x"].shape[0]
+            what = f"first {frac_units} of {total} images"
+        elif name == "c4":
+            b_total, h, sq, d = w.inputs["q"].shape
+            for k in ("q", "k", "v"):
+                s.inputs[k] = Tensor(k, w.dtype, w.inputs[k].store[:frac_units])
+            s.inputs["r"] = Tensor("r", w.dtype, w.inputs["r"].store[: frac_units * sq])
+            total = b_total
+            what = f"first {frac_units} of {total} batch elements"
+        else:
+            attn = [o for o in w.ops if o["kind"] == "attention_causal"][0]["attrs"]
+            sq, total = attn["seq"], attn["batch"]
+            s.inputs["x"] = Tensor("x", w.dtype, w.inputs["x"].store[: frac_units * sq])
+            for o in s.ops:
+                if o["kind"] == "attention_causal":
+                    o["attrs"]["batch"] = frac_units
+            what = f"first {frac_units} of {total} batch elements"
+        return s, total, what
+
+    probe_units = {"c1": 64, "c2": 64, "c3": 1, "c4": 1, "c5": 1}[name]
+    s, total, _ = sub(probe_units)
+    t0 = time.perf_counter()
+    OM.run_workload(s, [0])
+    probe = max(time.perf_counter() - t0, 1e-4)
+    units = int(min(total, max(probe_units, probe_units * budget_s / probe)))
+    if units > probe_units:
+        s, total, what = sub(units)
+        t0 = time.perf_counter()
+        OM.run_workload(s, [0])
+        secs = time.perf_counter() - t0
+    else:
+        s, total, what = sub(probe_units)
+        units, secs = probe_units, probe
+    return w.flops * units / total, secs, what
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = full_workload(args.workload)
+    t_all = []
+    flops = 0.0
+    what = ""
+    budget = max(2.0, min(12.0, 120.0 / max(1, args.steps + args.warmup)))
+    for i in range(args.warmup + args.steps):
+        f, s, what = oracle_sample(args.workload, w, budget_s=budget)
+        if i >= args.warmup:
+            t_all.append(s)
+            flops = f
+    mean_s = sum(t_all) / len(t_all)
+    val = flops / mean_s / 1e12
+    cores = os.cpu_count()
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": "TFLOP/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": mean_s * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload, "sample": what},
+        "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": what},
+        "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------------------------------
+# GPU arm
+# ----------------------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback for the product path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    from paper_2607_20501_b200 import Context
+    from paper_2607_20501_b200.runner import DeviceWorkload
+
+    name = args.workload
+    w = full_workload(name)
+    ctx = Context(local)
+    # rotation: enough independent copies that a pass over all of them exceeds L2 (126 MB) twice over
+    per_copy = sum(t.nbytes() for t in w.inputs.values()) + sum(t.nbytes() for t in w.params.values())
+    rot = int(max(2, min(8, -(-300e6 // max(per_copy, 1)))))
+    sets = [DeviceWorkload(ctx, w, device=f"cuda:{local}") for _ in range(rot)]
+    part = args.decomposition or ("fused" if "fused" in w.partitions else None)
+    for dw in sets:
+        if part:
+            dw.module.set_decomposition(w.partitions[part])
+        dw.ensure_workspace()
+    impls = [sets[0].module.bound_impl(s) for s in range(sets[0].module.n_sub())]
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(max(args.warmup, 3)):
+        sets[i % rot].forward()
+    barrier()
+    launches_per_step = sets[0].module.launch_count()
+
+    # ---- timed region: K steps, device time, per-step event pairs for the kernel duration
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local)
+    sampler.start()
+    barrier()
+    t_begin.record(stream)
+    for i in range(args.steps):
+        ev[i][0].record(stream)
+        sets[i % rot].forward()
+        ev[i][1].record(stream)
+    t_end.record(stream)
+    barrier()
+    clocks = sampler.stop()
+    ctx.check()
+    total_ms = t_begin.elapsed_time(t_end)
+    step_ms = sorted(a.elapsed_time(b) for a, b in ev)
+    kernel_ms = sum(step_ms) / len(step_ms)
+
+    # ---- end to end: pinned host inputs in, result out, every step
+    host_in = {k: torch.empty(t.shape, dtype=sets[0].inputs[k].dtype).pin_memory() for k, t in w.inputs.items()}
+    for k in host_in:
+        host_in[k].copy_(sets[0].inputs[k].cpu())
+    host_out = torch.empty(sets[0].out.shape, dtype=sets[0].out.dtype).pin_memory()
+    h2d = sum(t.numel() * t.element_size() for t in host_in.values())
+    d2h = host_out.numel() * host_out.element_size()
+    e2e_steps = max(3, min(args.steps, 50))
+
+    def e2e_step(dw):
+        for k in host_in:
+            dw.inputs[k].copy_(host_in[k], non_blocking=True)
+        dw.forward()
+        host_out.copy_(dw.out, non_blocking=True)
+
+    e2e_step(sets[0])
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(e2e_steps):
+        e2e_step(sets[i % rot])
+    e1.record(stream)
+    barrier()
+    e2e_ms = e0.elapsed_time(e1) / e2e_steps
+
+    # ---- per-subkernel breakdown of the split decomposition (time shares)
+    breakdown = None
+    split_name = {"c1": "split", "c2": "split", "c3": "split2", "c4": "split3", "c5": "fused_tails"}.get(name)
+    if rank == 0 and split_name in w.partitions:
+        dw = sets[0]
+        dw.module.set_decomposition(w.partitions[split_name])
+        dw.ensure_workspace()
+        dw.forward()
+        torch.cuda.synchronize()
+        ms = dw.profile(iters=20)
+        tot = sum(ms)
+        names = [dw.module.bound_impl(s) for s in range(dw.module.n_sub())]
+        agg = {}
+        for n_, t_ in zip(names, ms):
+            agg[n_] = agg.get(n_, 0.0) + t_
+        breakdown = {"decomposition": split_name, "ms_total": tot,
+                     "share": {k: round(v / tot, 4) for k, v in agg.items()},
+                     "ms": {k: round(v, 5) for k, v in agg.items()}}
+
+    # ---- max over ranks
+    t = torch.tensor([total_ms, kernel_ms, e2e_ms], dtype=torch.float64, device=f"cuda:{local}")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms, kernel_ms, e2e_ms = (float(v) for v in t.tolist())
+
+    if rank == 0:
+        pk = peaks()
+        ms_per_step = total_ms / args.steps
+        value = world * w.flops / (ms_per_step * 1e-3) / 1e12
+        achieved = w.flops / (kernel_ms * 1e-3) / 1e12
+        peak = pk["bf16_tflops"] if ms_per_step < 1.0 else pk.get("bf16_tflops_sustained", pk["bf16_tflops"])
+        t_roof_ms = max(w.flops / (peak * 1e12), w.min_bytes / (pk["hbm_gbs"] * 1e9)) * 1e3
+        line = {
+            "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
+            "config": {"workload": name, "decomposition": part, "impls": impls,
+                       "l2": f"rotation over {rot} independent input/output sets ({rot * per_copy / 1e6:.0f} MB > L2)",
+                       "shapes": {k: list(t.shape) for k, t in w.inputs.items()}},
+            "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                         "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES.get(name),
+                         "peak_source": pk["_source"], "kernel_ms": kernel_ms, "module_t_roof_ms": t_roof_ms,
+                         "module_frac": t_roof_ms / ms_per_step, "min_step_ms": step_ms[0]},
+            "e2e": {"value": world * w.flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
+            "gpu_launches": launches_per_step * args.steps,
+            "clocks": clocks,
+            "per_subkernel": breakdown,
+        }
+        if not args.no_cpu and world == 1:
+            f, s, what = oracle_sample(name, w, budget_s=args.cpu_seconds)
+            line["cpu_baseline"] = {"value": f / s / 1e12, "unit": "TFLOP/s", "cores": os.cpu_count(), "kind": "oracle",
+                                    "sample": what, "seconds": s}
+        else:
+            line["cpu_baseline"] = None
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c2", choices=["c1", "c2", "c3", "c4", "c5"])
+    ap.add_argument("--decomposition", default=None)
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle leg")
+    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    args = ap.parse_args()
+    if args.steps is None:
+        args.steps = DEFAULT_STEPS[args.workload] if args.impl == "ours" else 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
