@@ -18,6 +18,7 @@
 #include "device_common.cuh"
 #include "tc_common.cuh"
 #include "tc_plans.h"
+#include "tc_epilogue.cuh"
 
 namespace mk {
 
@@ -37,64 +38,6 @@ struct Shared {
   uint32_t tmem_base;
   int abort_flag;
 };
-
-__device__ __forceinline__ float gelu_fast(float x) {
-  const float u = 0.7978845608028654f * (x + 0.044715f * x * x * x);
-  return 0.5f * x * (1.0f + tc::tanh_fast(u));
-}
-__device__ __forceinline__ float silu_fast(float x) { return __fdividef(x, 1.0f + tc::ex2_fast(-1.4426950408889634f * x)); }
-
-// elementwise program on 32 consecutive columns of one row, fast transcendental forms (bf16 output)
-__device__ __forceinline__ void epi32(const EpiProgram& p, float (&v)[32], int64_t row, int64_t col0, int64_t ld) {
-  for (int i = 0; i < p.n; ++i) {
-    const EpiOp& o = p.op[i];
-    switch (o.kind) {
-      case EPI_BIAS: {
-        const __nv_bfloat16* b = reinterpret_cast<const __nv_bfloat16*>(o.ptr) + col0;
-#pragma unroll
-        for (int j = 0; j < 32; j += 8) {
-          float t[8];
-          ld_vec(b + j, t);
-#pragma unroll
-          for (int q = 0; q < 8; ++q) v[j + q] += t[q];
-        }
-        break;
-      }
-      case EPI_RESIDUAL: {
-        const __nv_bfloat16* r = reinterpret_cast<const __nv_bfloat16*>(o.ptr) + row * ld + col0;
-#pragma unroll
-        for (int j = 0; j < 32; j += 8) {
-          float t[8];
-          ld_vec(r + j, t);
-#pragma unroll
-          for (int q = 0; q < 8; ++q) v[j + q] += t[q];
-        }
-        break;
-      }
-      case EPI_RELU:
-#pragma unroll
-        for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.0f);
-        break;
-      case EPI_GELU_TANH:
-#pragma unroll
-        for (int j = 0; j < 32; ++j) v[j] = gelu_fast(v[j]);
-        break;
-      case EPI_SILU:
-#pragma unroll
-        for (int j = 0; j < 32; ++j) v[j] = silu_fast(v[j]);
-        break;
-      case EPI_SCALE:
-#pragma unroll
-        for (int j = 0; j < 32; ++j) v[j] *= o.a;
-        break;
-      case EPI_CLAMP:
-#pragma unroll
-        for (int j = 0; j < 32; ++j) v[j] = fminf(fmaxf(v[j], o.a), o.b);
-        break;
-      default: break;
-    }
-  }
-}
 
 __device__ __forceinline__ void tile_coords(int t, int num_m, int num_n, int& mi, int& ni) {
   const int per_group = GROUP_M * num_n;

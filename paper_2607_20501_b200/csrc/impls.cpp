@@ -157,7 +157,7 @@ bool gemm_tc_match(const Module& m, int lo, int hi) {
   const int64_t N = last_dim(m.vspec(m.ops[hi - 1].out_id));
   return K % 8 == 0 && N % 8 == 0;
 }
-mk_status gemm_tc_emit(const Module& m, int lo, int hi, const Resolved& r, std::vector<Launch>& out, std::string& err) {
+mk_status gemm_tc_emit_impl(const Module& m, int lo, int hi, const Resolved& r, std::vector<Launch>& out, std::string& err, bool pair) {
   bool sw; int t;
   gemm_shape(m, lo, hi, &sw, &t);
   EpiProgram p;
@@ -167,11 +167,24 @@ mk_status gemm_tc_emit(const Module& m, int lo, int hi, const Resolved& r, std::
   const mk_tensor_spec& xs = m.vspec(op.in_id[0]);
   const int64_t M = xs.shape[0], K = xs.shape[1], N = last_dim(m.vspec(m.ops[hi - 1].out_id));
   auto plan = std::make_shared<GemmTcPlan>();
-  cudaError_t e = gemm_tc_plan(plan.get(), r.value_ptr[op.in_id[0]], op.param[0].ptr, r.value_ptr[m.ops[hi - 1].out_id], M, N, K, sw, p,
-                               m.ctx->sm_count);
+  const void* a = r.value_ptr[op.in_id[0]];
+  void* y = r.value_ptr[m.ops[hi - 1].out_id];
+  cudaError_t e = pair ? gemm_tc2_plan(plan.get(), a, op.param[0].ptr, y, M, N, K, sw, p, m.ctx->sm_count)
+                       : gemm_tc_plan(plan.get(), a, op.param[0].ptr, y, M, N, K, sw, p, m.ctx->sm_count);
   if (e != cudaSuccess) { err = std::string("gemm_tc plan: ") + cudaGetErrorString(e); return MK_ERR_CUDA; }
-  out.push_back([plan](cudaStream_t s) { return launch_gemm_tc(*plan, s); });
+  if (pair) out.push_back([plan](cudaStream_t s) { return launch_gemm_tc2(*plan, s); });
+  else out.push_back([plan](cudaStream_t s) { return launch_gemm_tc(*plan, s); });
   return MK_OK;
+}
+mk_status gemm_tc_emit(const Module& m, int lo, int hi, const Resolved& r, std::vector<Launch>& out, std::string& err) {
+  return gemm_tc_emit_impl(m, lo, hi, r, out, err, false);
+}
+// two-SM form: worth it once a tile pair has more than one CTA's worth of rows
+bool gemm_tc2_match(const Module& m, int lo, int hi) {
+  return gemm_tc_match(m, lo, hi) && m.vspec(m.ops[lo].in_id[0]).shape[0] > 128;
+}
+mk_status gemm_tc2_emit(const Module& m, int lo, int hi, const Resolved& r, std::vector<Launch>& out, std::string& err) {
+  return gemm_tc_emit_impl(m, lo, hi, r, out, err, true);
 }
 
 // LINEAR [elementwise]* (LAYERNORM | RMSNORM), fp32, one CTA owns whole rows
@@ -262,6 +275,7 @@ mk_status attn_simt_emit(const Module& m, int lo, int, const Resolved& r, std::v
 const std::vector<Impl>& registry() {
   static const std::vector<Impl> reg = {
       {"linear_rownorm_simt", linear_rownorm_match, no_scratch, linear_rownorm_emit},
+      {"gemm_tc2", gemm_tc2_match, no_scratch, gemm_tc2_emit},
       {"gemm_tc", gemm_tc_match, no_scratch, gemm_tc_emit},
       {"gemm_simt", gemm_simt_match, no_scratch, gemm_simt_emit},
       {"conv3x3_simt", conv_simt_match, no_scratch, conv_simt_emit},

@@ -23,3 +23,10 @@ cudaError_t gemm_tc_plan(GemmTcPlan* p, const void* a, const void* w_nk, void* y
 cudaError_t launch_gemm_tc(const GemmTcPlan& p, cudaStream_t s);
 
 }  // namespace mk
+
+namespace mk {
+// Two-SM form (CTA pairs, tcgen05 cta_group::2, 256x256 tiles); same contract as gemm_tc_plan.
+cudaError_t gemm_tc2_plan(GemmTcPlan* p, const void* a, const void* w_nk, void* y, int64_t m, int64_t n, int64_t k, bool swiglu,
+                          const EpiProgram& epi, int sm_count);
+cudaError_t launch_gemm_tc2(const GemmTcPlan& p, cudaStream_t s);
+}  // namespace mk
