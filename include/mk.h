@@ -232,6 +232,31 @@ MK_API mk_status mk_module_profile(mk_module* m, const void* const* in_ptrs, voi
 MK_API mk_status mk_module_intermediate(const mk_module* m, int32_t value_id, const void** dev_ptr,
                                  mk_tensor_spec* spec);
 
+/* ---- allocation-free GroupNorm ----------------------------------------------------------------
+ * (The paper has no counterpart: this entry point exists for callers, not for the method.)
+ * NHWC GroupNorm, the same two kernels the composed path launches, for callers that cannot
+ * allocate device memory where they call the library and so cannot provide a workspace: code
+ * inside a memory-planned region of a framework, a plugin that is handed only its input and
+ * output buffers, a latency-critical loop that must not hit cudaMalloc's implicit
+ * synchronisation.  The partial sums live in a 1 MiB array inside the library image, resident
+ * on every GPU that loads the library until the process exits.
+ *   dev_x, dev_y       [n, h, w, c] tensors of `dtype` (mk_dtype), 16-byte aligned, caller-owned
+ *   dev_gamma/dev_beta [c] or NULL
+ *   groups             must divide c; eps >= 0, inside the square root
+ * The call allocates nothing, is asynchronous on `cuda_stream` and does not synchronise.
+ * The first call on each device looks up the array's device address (a host-side query, made
+ * with that device current): make that first call before starting any stream capture.
+ * All calls share the one array and it keeps the last call's contents; the kernels overwrite
+ * every slot they later read, so nothing needs clearing, but two calls whose kernels overlap on
+ * the GPU (different streams, no dependency) race on it — order them.
+ * Errors: MK_ERR_WORKSPACE_TOO_SMALL if n * chunks * groups * 8 bytes exceeds 1 MiB (chunks <= 64
+ * pixel chunks per image; e.g. n = 32, groups = 32 needs 80 KiB), MK_ERR_SHAPE_MISMATCH,
+ * MK_ERR_INVALID_ARG, MK_ERR_NO_DEVICE, MK_ERR_CUDA. */
+MK_API mk_status mk_groupnorm_nhwc_noalloc(int32_t dtype, const void* dev_x, void* dev_y,
+                                           const void* dev_gamma, const void* dev_beta, int64_t n,
+                                           int64_t h, int64_t w, int64_t c, int32_t groups,
+                                           double eps, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -88,6 +88,8 @@ _sig("mk_module_launch_count", C.c_int32, _P, _I32P)
 _sig("mk_module_forward", C.c_int32, _P, _PP, _PP, _P, C.c_size_t, _P)
 _sig("mk_module_profile", C.c_int32, _P, _PP, _PP, _P, C.c_size_t, _P, C.c_int32, C.POINTER(C.c_float))
 _sig("mk_module_intermediate", C.c_int32, _P, C.c_int32, _PP, _SPECP)
+_sig("mk_groupnorm_nhwc_noalloc", C.c_int32, C.c_int32, _P, _P, _P, _P, C.c_int64, C.c_int64, C.c_int64,
+     C.c_int64, C.c_int32, C.c_double, _P)
 
 EXPORTS = [n for n in dir() if n.startswith("mk_") and callable(globals()[n]) and n not in
            ("mk_tensor_spec", "mk_op_desc")]
