@@ -135,9 +135,12 @@ class Context:
             raise MkError(st, self.last_error())
 
     def __del__(self):
-        if getattr(self, "h", None):
-            mk_ctx_destroy(self.h)
-            self.h = None
+        try:
+            if getattr(self, "h", None):
+                mk_ctx_destroy(self.h)
+                self.h = None
+        except Exception:       # interpreter shutdown: the module globals may already be gone
+            pass
 
 
 def _ptr(t):
@@ -209,9 +212,12 @@ class Module:
             raise MkError(st, self.ctx.last_error())
 
     def __del__(self):
-        if getattr(self, "h", None):
-            mk_module_destroy(self.h)
-            self.h = None
+        try:
+            if getattr(self, "h", None):
+                mk_module_destroy(self.h)
+                self.h = None
+        except Exception:       # interpreter shutdown: the module globals may already be gone
+            pass
 
     # -- description ---------------------------------------------------------------------------------
     def n_ops(self):

@@ -38,7 +38,7 @@ def _headers_mtime():
 
 
 def _compile(src, obj, verbose):
-    cmd = [NVCC, *FLAGS, "-x", "cu", "-c", src, "-o", obj]
+    cmd = [NVCC, *FLAGS, *os.environ.get("MK_NVCC_FLAGS", "").split(), "-x", "cu", "-c", src, "-o", obj]
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")

@@ -2,35 +2,54 @@
 //
 //   D[M, N] = tail(A[M, K] @ W[K, N])        A row-major (K-major), W stored [N, K] (K-major)
 //
-// One persistent CTA per SM, 6 warps:
-//   warp 0        TMA producer: A tile 128x64 and W tile 256x64 per stage, 128-byte swizzle,
-//                 4-stage mbarrier ring (192 KB of shared memory)
-//   warp 1        allocates TMEM (512 columns = two 128x256 fp32 accumulators) and issues
-//                 tcgen05.mma 128x256x16, four per stage; tcgen05.commit frees the stage and,
-//                 after the last K block, publishes the accumulator
-//   warps 2..5    epilogue: tcgen05.ld 32 lanes x 32 columns, the elementwise program in fp32
-//                 registers, bf16 pack, 16-byte global stores; runs on accumulator t while the
-//                 tensor cores fill accumulator t+1
-// SwiGLU mode: the 256 accumulator columns are 128 gate columns and the matching 128 up columns
-// (two TMA boxes of W), and the tile's output is silu(gate) * up, 128 columns wide.
+// Two forms of one kernel:
+//   CTAS = 2  a cluster of two CTAs (two SMs) shares one tcgen05.mma.cta_group::2 of shape 256x256x16.
+//             Each CTA stages its own 128 rows of A and its own 128 of the tile's 256 W rows (32 KB per
+//             stage, 6 stages), so each W byte crosses L2 -> SM once per pair.  No TMA multicast: each
+//             CTA issues plain tile loads for its halves and both CTAs' loads complete on the leader's
+//             "full" barrier; the leader's tcgen05.commit (multicast of a barrier arrival, not of data)
+//             frees the stage in both CTAs and publishes the accumulator to both epilogues.
+//   CTAS = 1  one CTA per 128x256 tile (48 KB per stage, 4 stages), for M <= 128.
 //
-// Every mbarrier wait is bounded; see tc_common.cuh.
+// Per CTA, 10 warps:
+//   warp 0        TMA producer (one lane): 128-byte-swizzled tiles into an mbarrier ring
+//   warp 1        TMEM allocation (512 columns = two 128x256 fp32 accumulators); one lane of the leader
+//                 CTA issues the MMAs.  The issue loop is kept to a few instructions per MMA: a single
+//                 thread issuing dependent instructions can starve the tensor pipe (a 256x256x16 MMA
+//                 lasts 128 cycles)
+//   warps 2..9    epilogue of this CTA's 128 rows (two warps per TMEM lane quarter, alternating 32-column
+//                 chunks): tcgen05.ld, elementwise program in fp32, bf16 pack, shared-memory transpose,
+//                 coalesced stores; overlaps the next tile's MMAs through the second accumulator
+// SwiGLU mode: accumulator columns [0,128) are gate columns and [128,256) the matching up columns
+// (two TMA boxes of W; in the pair form the leader holds gate rows, the peer up rows); the tile's
+// output is silu(gate) * up, 128 columns wide.
+// Ragged M / N / K: TMA zero-fills out-of-range rows and K columns; stores are guarded.
+// Every mbarrier wait is bounded (tc_common.cuh); a CTA pair leaves through a cluster barrier.
 #include "device_common.cuh"
 #include "tc_common.cuh"
-#include "tc_plans.h"
 #include "tc_epilogue.cuh"
+#include "tc_plans.h"
 
 namespace mk {
 
 namespace {
 
-constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4, UMMA_K = 16;
-constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
-constexpr int GEMM_THREADS = 192;
-constexpr int GROUP_M = 16;
-constexpr size_t GEMM_SMEM = (size_t)STAGES * STAGE_BYTES + 1024 /*alignment*/ + 256 /*barriers*/;
+constexpr int BM = 128;   // rows per CTA
+constexpr int BN = 256;   // accumulator columns
+constexpr int BK = 64, UMMA_K = 16;
+constexpr int EPI_WARPS = 8;
+constexpr int THREADS = 64 + 32 * EPI_WARPS;
+constexpr int GROUP_M = 8;  // tile rows walked together for L2 reuse
 
-struct Shared {
+template <int CTAS> struct Cfg {
+  static constexpr int STAGES = CTAS == 2 ? 6 : 4;
+  static constexpr int A_BYTES = BM * BK * 2;
+  static constexpr int B_BYTES = (BN / CTAS) * BK * 2;
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr size_t SMEM = (size_t)STAGES * STAGE_BYTES + EPI_WARPS * EPI_WARP_BYTES + 1024 /*alignment*/ + 256 /*barriers*/;
+};
+
+template <int STAGES> struct Shared {
   uint64_t full[STAGES];
   uint64_t empty[STAGES];
   uint64_t tfull[2];
@@ -49,117 +68,168 @@ __device__ __forceinline__ void tile_coords(int t, int num_m, int num_n, int& mi
   ni = r / gsz;
 }
 
-template <bool SWIGLU>
-__global__ void __launch_bounds__(GEMM_THREADS, 1)
+template <int CTAS, bool SWIGLU>
+__global__ void __launch_bounds__(THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, __nv_bfloat16* __restrict__ out, int M,
                int N, int K, int up_row_offset, const __grid_constant__ EpiProgram epi, unsigned int* status) {
+  using C = Cfg<CTAS>;
+  constexpr int STAGES = C::STAGES;
   constexpr int OUT_N = SWIGLU ? BN / 2 : BN;  // output columns per tile
   extern __shared__ uint8_t smem_raw[];
   uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  Shared* sh = reinterpret_cast<Shared*>(tiles + (size_t)STAGES * STAGE_BYTES);
+  uint8_t* staging = tiles + (size_t)STAGES * C::STAGE_BYTES;
+  Shared<STAGES>* sh = reinterpret_cast<Shared<STAGES>*>(staging + EPI_WARPS * EPI_WARP_BYTES);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int num_m = (M + BM - 1) / BM, num_n = (N + OUT_N - 1) / OUT_N;
+  const uint32_t rank = CTAS == 2 ? tc::cluster_ctarank() : 0;
+  const bool leader = rank == 0;
+  const int unit_id = blockIdx.x / CTAS, num_units = gridDim.x / CTAS;   // a unit = a CTA or a CTA pair
+  const int num_m = (M + CTAS * BM - 1) / (CTAS * BM), num_n = (N + OUT_N - 1) / OUT_N;
   const int total_tiles = num_m * num_n;
   const int num_kb = (K + BK - 1) / BK;
   volatile int* abort_flag = &sh->abort_flag;
+  MK_TR_DECL
+  MK_TR_INIT;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { tc::mbar_init(&sh->full[s], 1); tc::mbar_init(&sh->empty[s], 1); }
-    for (int b = 0; b < 2; ++b) { tc::mbar_init(&sh->tfull[b], 1); tc::mbar_init(&sh->tempty[b], 4); }
+    for (int b = 0; b < 2; ++b) { tc::mbar_init(&sh->tfull[b], 1); tc::mbar_init(&sh->tempty[b], EPI_WARPS * CTAS); }
     sh->abort_flag = 0;
     tc::fence_barrier_init();
     tc::tma_prefetch_desc(&tmA);
     tc::tma_prefetch_desc(&tmB);
   }
   if (warp == 1) {
-    tc::tmem_alloc(&sh->tmem_base, 512);
-    tc::tmem_relinquish();
+    if (CTAS == 2) tc::tmem_alloc_pair(&sh->tmem_base, 512);
+    else { tc::tmem_alloc(&sh->tmem_base, 512); tc::tmem_relinquish(); }
   }
   tc::tc_fence_before();
   __syncthreads();
+  if (CTAS == 2) tc::cluster_sync();  // both CTAs' barriers exist before anything remote touches them
   tc::tc_fence_after();
   const uint32_t tmem_base = sh->tmem_base;
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
-    int stage = 0;
-    uint32_t phase = 0;
-    bool ok = true;
-    for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-      int mi, ni;
-      tile_coords(t, num_m, num_n, mi, ni);
-      for (int kb = 0; kb < num_kb && ok; ++kb) {
-        if (lane == 0) {
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int t = unit_id; t < total_tiles && ok; t += num_units) {
+        int mi, ni;
+        tile_coords(t, num_m, num_n, mi, ni);
+        const int m0 = (mi * CTAS + (int)rank) * BM;
+        const int n0 = ni * OUT_N;
+#ifdef MK_TRACE
+        unsigned long long esum = 0;
+#endif
+        for (int kb = 0; kb < num_kb; ++kb) {
+#ifdef MK_TRACE
+          const unsigned long long w0_ = tc::gtime();
+#endif
           ok = tc::mbar_wait(&sh->empty[stage], phase ^ 1, abort_flag, status, tc::WAIT_SMEM_EMPTY);
-          if (ok) {
-            uint8_t* a_dst = tiles + (size_t)stage * STAGE_BYTES;
-            uint8_t* b_dst = a_dst + A_BYTES;
-            tc::mbar_expect_tx(&sh->full[stage], STAGE_BYTES);
-            tc::tma_load_2d(a_dst, &tmA, &sh->full[stage], kb * BK, mi * BM);
-            const int n0 = ni * OUT_N;
+#ifdef MK_TRACE
+          esum += tc::gtime() - w0_;
+          if (kb == num_kb - 1 && blockIdx.x == 0) mk_tr[70 + (t - unit_id) / num_units] = mk_tr[0] + esum;
+#endif
+          if (!ok) break;
+          uint8_t* a_dst = tiles + (size_t)stage * C::STAGE_BYTES;
+          uint8_t* b_dst = a_dst + C::A_BYTES;
+          if (CTAS == 2) {
+            const uint32_t full_leader = tc::map_to_cta(tc::smem_u32(&sh->full[stage]), 0);
+            if (leader) tc::mbar_expect_tx(&sh->full[stage], 2 * C::STAGE_BYTES);
+            const int b_row = SWIGLU ? (leader ? n0 : up_row_offset + n0) : n0 + (int)rank * (BN / 2);
+            tc::tma_load_2d_pair(a_dst, &tmA, full_leader, kb * BK, m0);
+            tc::tma_load_2d_pair(b_dst, &tmB, full_leader, kb * BK, b_row);
+          } else {
+            tc::mbar_expect_tx(&sh->full[stage], C::STAGE_BYTES);
+            tc::tma_load_2d(a_dst, &tmA, &sh->full[stage], kb * BK, m0);
             tc::tma_load_2d(b_dst, &tmB, &sh->full[stage], kb * BK, n0);
-            tc::tma_load_2d(b_dst + B_BYTES / 2, &tmB, &sh->full[stage], kb * BK, SWIGLU ? up_row_offset + n0 : n0 + BN / 2);
+            tc::tma_load_2d(b_dst + C::B_BYTES / 2, &tmB, &sh->full[stage], kb * BK, SWIGLU ? up_row_offset + n0 : n0 + BN / 2);
           }
+          if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
-        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-        if (++stage == STAGES) { stage = 0; phase ^= 1; }
       }
     }
+    __syncwarp();
   } else if (warp == 1) {
-    // ------------------------------------------------------------ MMA issuer
-    constexpr uint32_t idesc = tc::idesc_bf16_f32(BM, BN, 0, 0);
-    int stage = 0;
-    uint32_t phase = 0;
-    bool ok = true;
-    int it = 0;
-    for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
-      const int acc = it & 1;
-      const uint32_t acc_phase = (it >> 1) & 1;
-      const uint32_t d_tmem = tmem_base + acc * BN;
-      if (lane == 0) {
-        ok = tc::mbar_wait(&sh->tempty[acc], acc_phase ^ 1, abort_flag, status, tc::WAIT_TMEM_EMPTY);
+    // ------------------------------------------------------------ MMA issuer (one lane of the leader)
+    if (leader && lane == 0) {
+      constexpr uint32_t idesc = tc::idesc_bf16_f32(CTAS * BM, BN, 0, 0);
+      const uint32_t a_lo0 = tc::desc_lo_sw128(tc::smem_u32(tiles));
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      int it = 0;
+      for (int t = unit_id; t < total_tiles && ok; t += num_units, ++it) {
+        const int acc = it & 1;
+        const uint32_t d_tmem = tmem_base + acc * BN;
+        ok = tc::mbar_wait(&sh->tempty[acc], ((it >> 1) & 1) ^ 1, abort_flag, status, tc::WAIT_TMEM_EMPTY);
+        if (!ok) break;
         tc::tc_fence_after();
-      }
-      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-      for (int kb = 0; kb < num_kb && ok; ++kb) {
-        if (lane == 0) {
+        MK_TR(1 + it * 8);                       // MMA: accumulator free, tile starts
+        uint32_t accumulate = 0;
+#ifdef MK_TRACE
+        unsigned long long wsum = 0;
+#endif
+        for (int kb = 0; kb < num_kb; ++kb) {
+#ifdef MK_TRACE
+          const unsigned long long w0_ = tc::gtime();
+#endif
           ok = tc::mbar_wait(&sh->full[stage], phase, abort_flag, status, tc::WAIT_SMEM_FULL);
-          if (ok) {
-            tc::tc_fence_after();
-            const uint32_t a_addr = tc::smem_u32(tiles + (size_t)stage * STAGE_BYTES);
-            const uint64_t adesc = tc::smem_desc_sw128(a_addr, 16, 1024);
-            const uint64_t bdesc = tc::smem_desc_sw128(a_addr + A_BYTES, 16, 1024);
+#ifdef MK_TRACE
+          wsum += tc::gtime() - w0_;
+          if (kb == num_kb - 1 && blockIdx.x == 0) mk_tr[60 + it] = mk_tr[0] + wsum;
+#endif
+          if (!ok) break;
+          tc::tc_fence_after();
+          const uint32_t a_lo = a_lo0 + (uint32_t)stage * (C::STAGE_BYTES >> 4);
+          const uint32_t b_lo = a_lo + (C::A_BYTES >> 4);
 #pragma unroll
-            for (int k = 0; k < BK / UMMA_K; ++k)
-              tc::umma_ss(d_tmem, adesc + (uint64_t)(k * UMMA_K * 2 / 16), bdesc + (uint64_t)(k * UMMA_K * 2 / 16), idesc,
-                          (kb > 0 || k > 0) ? 1u : 0u);
-            tc::umma_commit(&sh->empty[stage]);
-            if (kb == num_kb - 1) tc::umma_commit(&sh->tfull[acc]);
+          for (int k = 0; k < BK / UMMA_K; ++k) {
+            if (CTAS == 2) tc::umma_ss_pair_lohi(d_tmem, a_lo + 2 * k, b_lo + 2 * k, idesc, accumulate);
+            else tc::umma_ss_lohi(d_tmem, a_lo + 2 * k, b_lo + 2 * k, idesc, accumulate);
+            accumulate = 1;
           }
+          if (CTAS == 2) tc::umma_commit_pair(&sh->empty[stage]);
+          else tc::umma_commit(&sh->empty[stage]);
+          if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
-        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-        if (++stage == STAGES) { stage = 0; phase ^= 1; }
+        if (!ok) break;
+        MK_TR(2 + it * 8);                       // MMA: last MMA of the tile issued
+        if (CTAS == 2) tc::umma_commit_pair(&sh->tfull[acc]);
+        else tc::umma_commit(&sh->tfull[acc]);
       }
     }
+    __syncwarp();
   } else {
-    // ------------------------------------------------------------ epilogue
-    const int q = warp & 3;  // TMEM lane quarter this warp may read
+    // ------------------------------------------------------------ epilogue: this CTA's 128 rows
+    // eight warps: warp w reads TMEM lane quarter w % 4 (the hardware's rule) and takes every other
+    // 32-column chunk, so each scheduler has two epilogue warps to interleave
+    const int q = warp & 3;
+    const int half = (warp - 2) >> 2;
+    constexpr int CHUNKS = OUT_N / 32;
+    EpiWarp ew;
+    ew.init(staging + (warp - 2) * EPI_WARP_BYTES, epi, lane);
     bool ok = true;
     int it = 0;
-    for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
+    for (int t = unit_id; t < total_tiles && ok; t += num_units, ++it) {
       int mi, ni;
       tile_coords(t, num_m, num_n, mi, ni);
       const int acc = it & 1;
-      const uint32_t acc_phase = (it >> 1) & 1;
-      ok = tc::mbar_wait(&sh->tfull[acc], acc_phase, abort_flag, status, tc::WAIT_TMEM_FULL);
+      const int64_t row0 = (int64_t)(mi * CTAS + (int)rank) * BM + q * 32;
+      auto rowmap = [&](int r) -> int64_t { const int64_t g = row0 + r; return g < M ? g : -1; };
+      const int64_t col_base = (int64_t)ni * OUT_N;
+      uint4 res_regs[4];
+      ew.load_bias(epi, col_base, OUT_N, N);
+      ew.prefetch_res(epi, rowmap, col_base + half * 32, N, res_regs);
+      ok = tc::mbar_wait(&sh->tfull[acc], (it >> 1) & 1, abort_flag, status, tc::WAIT_TMEM_FULL);
       ok = __all_sync(0xffffffffu, ok ? 1 : 0) != 0;
       if (!ok) break;
+      if (threadIdx.x == 64) MK_TR(3 + it * 8);  // epilogue: accumulator ready
       tc::tc_fence_after();
-      const int64_t row = (int64_t)mi * BM + q * 32 + lane;
       const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN;
-      __nv_bfloat16* orow = out + row * N;
 #pragma unroll 1
-      for (int c = 0; c < OUT_N / 32; ++c) {
+      for (int c = half; c < CHUNKS; c += 2) {
         uint32_t r[32];
         float v[32];
         tc::tmem_ld32(t_row + c * 32, r);
@@ -172,30 +242,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
           for (int j = 0; j < 32; ++j) v[j] = silu_fast(v[j]) * __uint_as_float(r[j]);
         }
-        const int64_t col0 = (int64_t)ni * OUT_N + c * 32;
-        if (row < M && col0 < N) {
-          if (col0 + 32 <= N) {
-            epi32(epi, v, row, col0, N);
-#pragma unroll
-            for (int j = 0; j < 32; j += 8) {
-              uint4 pk;
-              pk.x = pack_bf16x2(v[j], v[j + 1]);
-              pk.y = pack_bf16x2(v[j + 2], v[j + 3]);
-              pk.z = pack_bf16x2(v[j + 4], v[j + 5]);
-              pk.w = pack_bf16x2(v[j + 6], v[j + 7]);
-              *reinterpret_cast<uint4*>(orow + col0 + j) = pk;
-            }
-          } else {
-            for (int j = 0; j < 32 && col0 + j < N; ++j) orow[col0 + j] = __float2bfloat16_rn(epi_apply(epi, v[j], row, col0 + j, N));
-          }
-        }
+        ew.chunk_out(epi, v, rowmap, out, col_base + c * 32, c * 32, (int64_t)N, res_regs, c + 2 < CHUNKS ? col_base + (c + 2) * 32 : -1);
       }
       tc::tc_fence_before();
       __syncwarp();
-      if (lane == 0) tc::mbar_arrive(&sh->tempty[acc]);
+      if (threadIdx.x == 64) MK_TR(4 + it * 8);  // epilogue: tile stored
+      if (lane == 0) {
+        if (CTAS == 2) tc::mbar_arrive_cluster(tc::map_to_cta(tc::smem_u32(&sh->tempty[acc]), 0));
+        else tc::mbar_arrive(&sh->tempty[acc]);
+      }
     }
   }
 
+  MK_TR_PRINT("gemm");
   // common exit: on an aborted run give copies in flight time to land before the CTA retires
   if (*abort_flag) {
     const long long t0 = clock64();
@@ -203,16 +262,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   }
   tc::tc_fence_before();
   __syncthreads();
+  if (CTAS == 2) tc::cluster_sync();  // the peer's shared memory and barriers stay alive until both are done
   if (warp == 1) {
     tc::tc_fence_after();
-    tc::tmem_dealloc(tmem_base, 512);
+    if (CTAS == 2) tc::tmem_dealloc_pair(tmem_base, 512);
+    else tc::tmem_dealloc(tmem_base, 512);
   }
 }
 
-}  // namespace
-
-cudaError_t gemm_tc_plan(GemmTcPlan* p, const void* a, const void* w_nk, void* y, int64_t m, int64_t n, int64_t k, bool swiglu,
-                         const EpiProgram& epi, int sm_count) {
+template <int CTAS>
+cudaError_t plan_impl(GemmTcPlan* p, const void* a, const void* w_nk, void* y, int64_t m, int64_t n, int64_t k, bool swiglu,
+                      const EpiProgram& epi, int sm_count) {
   if (k % 8 || n % 8 || m < 1 || n < 1 || k < 1) return cudaErrorInvalidValue;
   if (m > INT32_MAX || n > INT32_MAX || k > INT32_MAX) return cudaErrorInvalidValue;
   const int64_t w_rows = swiglu ? 2 * n : n;
@@ -225,25 +285,50 @@ cudaError_t gemm_tc_plan(GemmTcPlan* p, const void* a, const void* w_nk, void* y
   p->swiglu = swiglu;
   p->epi = epi;
   const int out_n = swiglu ? BN / 2 : BN;
-  const int64_t tiles = ((m + BM - 1) / BM) * ((n + out_n - 1) / out_n);
-  p->grid = (int)(tiles < sm_count ? tiles : sm_count);
+  const int64_t tiles = ((m + CTAS * BM - 1) / (CTAS * BM)) * ((n + out_n - 1) / out_n);
+  const int64_t units = tiles < sm_count / CTAS ? tiles : sm_count / CTAS;
+  p->grid = (int)(CTAS * units);
   return cudaSuccess;
 }
 
-cudaError_t launch_gemm_tc(const GemmTcPlan& p, cudaStream_t s) {
+template <int CTAS>
+cudaError_t launch_impl(const GemmTcPlan& p, cudaStream_t s) {
   static bool attr_done = false;
   if (!attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM_SMEM);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM_SMEM);
+    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<CTAS, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<CTAS>::SMEM);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<CTAS, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<CTAS>::SMEM);
     if (e != cudaSuccess) return e;
     attr_done = true;
   }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)p.grid);
+  cfg.blockDim = dim3(THREADS);
+  cfg.dynamicSmemBytes = Cfg<CTAS>::SMEM;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = CTAS;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
   unsigned int* status = kernel_status_ptr();
-  if (p.swiglu)
-    gemm_tc_kernel<true><<<p.grid, GEMM_THREADS, GEMM_SMEM, s>>>(p.tm_a, p.tm_b, (__nv_bfloat16*)p.out, p.m, p.n, p.k, p.n, p.epi, status);
-  else
-    gemm_tc_kernel<false><<<p.grid, GEMM_THREADS, GEMM_SMEM, s>>>(p.tm_a, p.tm_b, (__nv_bfloat16*)p.out, p.m, p.n, p.k, 0, p.epi, status);
-  return cudaGetLastError();
+  __nv_bfloat16* out = (__nv_bfloat16*)p.out;
+  if (p.swiglu) return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<CTAS, true>, p.tm_a, p.tm_b, out, p.m, p.n, p.k, p.n, p.epi, status);
+  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<CTAS, false>, p.tm_a, p.tm_b, out, p.m, p.n, p.k, 0, p.epi, status);
 }
+
+}  // namespace
+
+cudaError_t gemm_tc_plan(GemmTcPlan* p, const void* a, const void* w_nk, void* y, int64_t m, int64_t n, int64_t k, bool swiglu,
+                         const EpiProgram& epi, int sm_count) {
+  return plan_impl<1>(p, a, w_nk, y, m, n, k, swiglu, epi, sm_count);
+}
+cudaError_t launch_gemm_tc(const GemmTcPlan& p, cudaStream_t s) { return launch_impl<1>(p, s); }
+cudaError_t gemm_tc2_plan(GemmTcPlan* p, const void* a, const void* w_nk, void* y, int64_t m, int64_t n, int64_t k, bool swiglu,
+                          const EpiProgram& epi, int sm_count) {
+  return plan_impl<2>(p, a, w_nk, y, m, n, k, swiglu, epi, sm_count);
+}
+cudaError_t launch_gemm_tc2(const GemmTcPlan& p, cudaStream_t s) { return launch_impl<2>(p, s); }
 
 }  // namespace mk

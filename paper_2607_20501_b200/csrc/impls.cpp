@@ -235,6 +235,26 @@ mk_status conv_simt_emit(const Module& m, int lo, int hi, const Resolved& r, std
   return MK_OK;
 }
 
+// tcgen05 implicit GEMM, weights resident in shared memory
+bool conv_tc2_match(const Module& m, int lo, int hi) {
+  if (!conv_simt_match(m, lo, hi) || m.values[0].spec.dtype != MK_BF16) return false;
+  const mk_tensor_spec& xs = m.vspec(m.ops[lo].in_id[0]);
+  return conv3x3_tc2_supported(xs.shape[0], xs.shape[1], xs.shape[2], xs.shape[3], m.ops[lo].d.i[0]);
+}
+mk_status conv_tc2_emit(const Module& m, int lo, int hi, const Resolved& r, std::vector<Launch>& out, std::string& err) {
+  EpiProgram p;
+  mk_status st = build_epi(m, lo + 1, hi, r, p, err);
+  if (st != MK_OK) return st;
+  const Op& op = m.ops[lo];
+  const mk_tensor_spec& xs = m.vspec(op.in_id[0]);
+  auto plan = std::make_shared<ConvTcPlan>();
+  cudaError_t e = conv3x3_tc2_plan(plan.get(), r.value_ptr[op.in_id[0]], op.param[0].ptr, r.value_ptr[m.ops[hi - 1].out_id], xs.shape[0],
+                                   xs.shape[1], xs.shape[2], xs.shape[3], op.d.i[0], p, m.ctx->sm_count);
+  if (e != cudaSuccess) { err = std::string("conv3x3_tc2 plan: ") + cudaGetErrorString(e); return MK_ERR_CUDA; }
+  out.push_back([plan](cudaStream_t s) { return launch_conv3x3_tc2(*plan, s); });
+  return MK_OK;
+}
+
 // ------------------------------------------------------------------ attention
 AttnView attn_view(const Module& m, const Op& op, const Resolved& r) {
   AttnView a{};
@@ -278,6 +298,7 @@ const std::vector<Impl>& registry() {
       {"gemm_tc2", gemm_tc2_match, no_scratch, gemm_tc2_emit},
       {"gemm_tc", gemm_tc_match, no_scratch, gemm_tc_emit},
       {"gemm_simt", gemm_simt_match, no_scratch, gemm_simt_emit},
+      {"conv3x3_tc2", conv_tc2_match, no_scratch, conv_tc2_emit},
       {"conv3x3_simt", conv_simt_match, no_scratch, conv_simt_emit},
       {"attention_simt", attn_simt_match, no_scratch, attn_simt_emit},
       {"rowop", rowop_match, no_scratch, rowop_emit},

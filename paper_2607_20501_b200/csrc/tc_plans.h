@@ -30,3 +30,21 @@ cudaError_t gemm_tc2_plan(GemmTcPlan* p, const void* a, const void* w_nk, void* 
                           const EpiProgram& epi, int sm_count);
 cudaError_t launch_gemm_tc2(const GemmTcPlan& p, cudaStream_t s);
 }  // namespace mk
+
+namespace mk {
+struct ConvTcPlan {
+  CUtensorMap tm_x, tm_w;
+  void* y = nullptr;
+  int nb = 0, h = 0, w = 0, c_in = 0, c_out = 0;
+  int grid = 0;
+  size_t smem = 0;
+  EpiProgram epi;
+};
+// NHWC bf16 3x3 conv (stride 1, pad 1) + elementwise tail; weights [C_out, 3, 3, C_in].
+// Supported: C_in in {64, 128}, C_out multiple of 32 up to 256, W <= 62, and half the weights
+// plus two input patches must fit one SM's shared memory.
+bool conv3x3_tc2_supported(int64_t nb, int64_t h, int64_t w, int64_t c_in, int64_t c_out);
+cudaError_t conv3x3_tc2_plan(ConvTcPlan* p, const void* x, const void* w, void* y, int64_t nb, int64_t h, int64_t wd, int64_t c_in,
+                             int64_t c_out, const EpiProgram& epi, int sm_count);
+cudaError_t launch_conv3x3_tc2(const ConvTcPlan& p, cudaStream_t s);
+}  // namespace mk

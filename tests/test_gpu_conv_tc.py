@@ -1,0 +1,58 @@
+"""tcgen05 implicit-GEMM convolution (K2) against the fp64 oracle: exact on integer inputs (any
+mismatch is an indexing bug: tap offsets, padding, row wrap, channel blocks), within tolerance on
+random inputs with every fused tail, swap against the plain-ALU kernel."""
+import numpy as np
+import pytest
+
+import workloads as W
+from workloads import generate as G
+from tests.parity import assert_parity, oracle, run_gpu
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    from paper_2607_20501_b200 import Context
+    return Context(0)
+
+
+def _bf16_round(x):
+    return W.bf16_bits_to_f64(W.f32_to_bf16_bits(np.asarray(x, np.float32)))
+
+
+SHAPES = [(1, 4, 4, 64, 32), (2, 8, 8, 64, 64), (3, 9, 7, 128, 128), (2, 13, 62, 64, 96), (1, 56, 56, 128, 128),
+          (5, 6, 10, 64, 256)]
+
+
+@pytest.mark.parametrize("nb,h,w,c,co", SHAPES)
+def test_integer_inputs_are_exact(ctx, nb, h, w, c, co):
+    wl = G.c3(0, NB=nb, H=h, W=w, C=c, CO=co, G=4)
+    wl.inputs["x"] = G.int_valued(1, 0, (nb, h, w, c), -2, 2, "bf16", "x")
+    wl.params["Wc"] = G.int_valued(1, 1, (co, 3, 3, c), -2, 2, "bf16", "Wc")
+    wl.ops = wl.ops[:1]
+    ref, _ = oracle(wl, [0])
+    dw, out = run_gpu(ctx, wl, [0], binds={0: "conv3x3_tc2"})
+    want = _bf16_round(ref)
+    bad = np.argwhere(out != want)
+    assert bad.size == 0, f"{len(bad)} of {out.size} mismatches, first at {bad[:6].tolist()}: got {out[tuple(bad[0])]}, want {want[tuple(bad[0])]}"
+
+
+@pytest.mark.parametrize("nb,h,w,c,co", [(3, 9, 7, 128, 128), (2, 56, 56, 128, 128)])
+def test_conv_chain_matches_the_oracle(ctx, nb, h, w, c, co):
+    for seed in range(2):
+        wl = W.c3(seed, NB=nb, H=h, W=w, C=c, CO=co, G=32)
+        ref, _ = oracle(wl, [0])
+        for part in ("fused", "split2", "split3"):
+            dw, out = run_gpu(ctx, wl, wl.partitions[part])
+            assert dw.module.bound_impl(0).startswith("conv3x3_tc2"), dw.module.bound_impl(0)
+            assert_parity(out, ref, "bf16", f"{part} seed {seed}")
+
+
+def test_swap_conv_kernels(ctx):
+    wl = W.c3(0, NB=2, H=12, W=12, C=64, CO=64, G=8)
+    ref, _ = oracle(wl, [0])
+    for impl in ("conv3x3_tc2", "conv3x3_simt"):
+        dw, out = run_gpu(ctx, wl, wl.partitions["split2"], binds={0: impl})
+        assert dw.module.bound_impl(0) == impl
+        assert_parity(out, ref, "bf16", impl)
