@@ -33,9 +33,8 @@ __device__ __forceinline__ float silu_fast(float x) { return __fdividef(x, 1.0f 
 // residual for these columns in shared memory (null: read them from global memory).
 __device__ __forceinline__ void epi32(const EpiProgram& p, float (&v)[32], int64_t row, int64_t col0, int64_t ld, const uint8_t* bias32,
                                       const uint8_t* res_row) {
-#pragma unroll
-  for (int i = 0; i < EPI_MAX; ++i) {
-    if (i >= p.n) break;
+#pragma unroll 1
+  for (int i = 0; i < p.n; ++i) {
     const EpiOp& o = p.op[i];
     switch (o.kind) {
       case EPI_BIAS: {
