@@ -48,3 +48,18 @@ cudaError_t conv3x3_tc2_plan(ConvTcPlan* p, const void* x, const void* w, void* 
                              int64_t c_out, const EpiProgram& epi, int sm_count);
 cudaError_t launch_conv3x3_tc2(const ConvTcPlan& p, cudaStream_t s);
 }  // namespace mk
+
+namespace mk {
+struct AttnTcPlan {
+  CUtensorMap tm_q, tm_k, tm_v;
+  void* out = nullptr;
+  int B = 0, H = 0, S = 0;
+  float scale_log2 = 0.f;
+  int grid = 0;
+};
+// Causal attention, bf16, head_dim 128, any strided [B, H, S, D] view whose strides are multiples of
+// 16 bytes; output the dense [B*S, H*D] matrix.
+bool attention_tc_supported(const AttnView& a);
+cudaError_t attention_tc_plan(AttnTcPlan* p, const AttnView& a, void* o);
+cudaError_t launch_attention_tc(const AttnTcPlan& p, cudaStream_t s);
+}  // namespace mk

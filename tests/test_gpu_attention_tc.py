@@ -1,0 +1,68 @@
+"""tcgen05 causal attention (K7) against the fp64 oracle: one tile, several key tiles, ragged
+sequence lengths, several heads and batches, the packed-QKV view, closed forms, swap against the
+plain-ALU kernel."""
+import numpy as np
+import pytest
+
+import workloads as W
+from workloads import generate as G
+from tests.parity import assert_parity, oracle, run_gpu
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    from paper_2607_20501_b200 import Context
+    return Context(0)
+
+
+def _attn_only(w):
+    w.ops = w.ops[:1]
+    return w
+
+
+@pytest.mark.parametrize("b,h,s", [(1, 1, 128), (1, 2, 256), (2, 3, 384), (1, 2, 200), (1, 1, 1000), (2, 2, 64), (1, 1, 1),
+                                   (1, 4, 2048)])
+def test_attention_matches_the_oracle(ctx, b, h, s):
+    for seed in range(2 if s <= 512 else 1):
+        w = _attn_only(W.c4(seed, B=b, H=h, S=s, D=128))
+        ref, _ = oracle(w, [0])
+        dw, out = run_gpu(ctx, w, [0], binds={0: "attention_tc"})
+        assert dw.module.bound_impl(0) == "attention_tc"
+        assert_parity(out, ref, "bf16", f"B{b} H{h} S{s} seed{seed}")
+
+
+def test_closed_forms(ctx):
+    b, h, s, d = 1, 2, 300, 128
+    w = _attn_only(W.c4(0, B=b, H=h, S=s, D=d))
+    k = w.inputs["k"].store
+    w.inputs["k"] = G.Tensor("k", "bf16", np.broadcast_to(k[:, :, :1], k.shape).copy())   # identical keys
+    dw, out = run_gpu(ctx, w, [0], binds={0: "attention_tc"})
+    v = w.inputs["v"].f64()
+    pm = np.cumsum(v, axis=2) / np.arange(1, s + 1)[None, None, :, None]     # prefix means of V
+    assert_parity(out, pm.transpose(0, 2, 1, 3).reshape(b * s, h * d), "bf16", "uniform weights")
+    # first query sees only the first key (the diagonal is kept)
+    assert np.array_equal(out[0].reshape(h, d), v[0, :, 0, :])
+
+
+def test_packed_qkv_view_and_swap(ctx):
+    w = W.c5(0, B=2, S=160, E=256, H=2, F=64, L=1)
+    w.ops = w.ops[:3]            # rmsnorm -> qkv linear -> attention on the packed tensor
+    ref, _ = oracle(w, [0])
+    outs = {}
+    for impl in ("attention_tc", "attention_simt"):
+        dw, out = run_gpu(ctx, w, [0, 1, 2], binds={2: impl})
+        assert dw.module.bound_impl(2) == impl
+        assert_parity(out, ref, "bf16", impl)
+        outs[impl] = out
+    assert np.abs(outs["attention_tc"] - outs["attention_simt"]).max() <= 4e-2
+
+
+def test_c4_block_at_reduced_size(ctx):
+    w = W.c4(0, B=2, H=4, S=512, D=128)
+    ref, inter = oracle(w, None)
+    for part in ("split3", "per_op", "fused"):
+        dw, out = run_gpu(ctx, w, w.partitions[part])
+        assert "attention_tc" in dw.module.bound_impl(0)
+        assert_parity(out, ref, "bf16", part)
