@@ -11,39 +11,43 @@ static inline int ceil_div_i64(int64_t a, int64_t b) { return (int)((a + b - 1) 
 // =====================================================================================================
 // elementwise chain
 // =====================================================================================================
+// Thread (cx, ry) of a block owns one 16-byte column vector and walks down the rows, four rows in
+// flight at a time: no per-element index arithmetic (a 64-bit division per vector made the first
+// version of this kernel ALU-bound), the bias slice of a thread never changes, and every access of a
+// warp is a contiguous run of a row.  tx = threads along a row (power of two <= 256).
 template <typename T, bool SWIGLU>
 __global__ void __launch_bounds__(256) eltwise_vec_kernel(const T* __restrict__ x, T* __restrict__ y, int64_t rows,
-                                                          int64_t cols, const __grid_constant__ EpiProgram p) {
+                                                          int64_t cols, int tx, const __grid_constant__ EpiProgram p) {
   constexpr int VE = Elem<T>::VEC;
   constexpr int UNROLL = 4;
-  const int64_t vpr = cols / VE;
-  const int64_t total = rows * vpr;
-  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  const int vpr = (int)(cols / VE);
+  const int cx = threadIdx.x & (tx - 1), ry = threadIdx.x / tx, rpb = 256 / tx;
+  const int vc = blockIdx.x * tx + cx;
+  if (vc >= vpr) return;
+  const int64_t col = (int64_t)vc * VE;
   const int64_t in_ld = SWIGLU ? 2 * cols : cols;
-  for (int64_t base = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; base < total; base += stride * UNROLL) {
+  const int64_t rstride = (int64_t)gridDim.y * rpb;
+  for (int64_t r0 = (int64_t)blockIdx.y * rpb + ry; r0 < rows; r0 += rstride * UNROLL) {
     float v[UNROLL][VE];
     float u[UNROLL][VE];
-    int64_t row[UNROLL], col[UNROLL];
 #pragma unroll
     for (int q = 0; q < UNROLL; ++q) {
-      const int64_t i = base + q * stride;
-      if (i < total) {
-        row[q] = i / vpr;
-        col[q] = (i - row[q] * vpr) * VE;
-        ld_vec(x + row[q] * in_ld + col[q], v[q]);
-        if (SWIGLU) ld_vec(x + row[q] * in_ld + cols + col[q], u[q]);
+      const int64_t r = r0 + q * rstride;
+      if (r < rows) {
+        ld_vec(x + r * in_ld + col, v[q]);
+        if (SWIGLU) ld_vec(x + r * in_ld + cols + col, u[q]);
       }
     }
 #pragma unroll
     for (int q = 0; q < UNROLL; ++q) {
-      const int64_t i = base + q * stride;
-      if (i < total) {
+      const int64_t r = r0 + q * rstride;
+      if (r < rows) {
         if (SWIGLU) {
 #pragma unroll
           for (int e = 0; e < VE; ++e) v[q][e] = silu_f(v[q][e]) * u[q][e];
         }
-        epi_apply_vec<T, VE>(p, v[q], row[q], col[q], cols);
-        st_vec(y + row[q] * cols + col[q], v[q]);
+        epi_apply_vec<T, VE>(p, v[q], r, col, cols);
+        st_vec(y + r * cols + col, v[q]);
       }
     }
   }
@@ -70,12 +74,21 @@ static cudaError_t eltwise_dispatch(const void* x, void* y, int64_t rows, int64_
   const T* xp = (const T*)x;
   T* yp = (T*)y;
   if (rows * cols == 0) return cudaSuccess;
-  if (cols % VE == 0) {
-    const int64_t total = rows * (cols / VE);
-    int grid = ceil_div_i64(total, 256 * 4);
-    grid = grid < 1 ? 1 : (grid > sm_count * 8 ? sm_count * 8 : grid);
-    if (swiglu) eltwise_vec_kernel<T, true><<<grid, 256, 0, s>>>(xp, yp, rows, cols, p);
-    else eltwise_vec_kernel<T, false><<<grid, 256, 0, s>>>(xp, yp, rows, cols, p);
+  if (cols % VE == 0 && cols / VE <= INT32_MAX / 2) {
+    const int vpr = (int)(cols / VE);
+    int tx = 1;
+    while (tx < vpr && tx < 256) tx *= 2;
+    const int rpb = 256 / tx;
+    const int gx = (vpr + tx - 1) / tx;
+    // enough row blocks to fill the machine 8 CTAs deep, each thread taking >= 4 rows when there are that many
+    int64_t gy = (rows + (int64_t)rpb * 4 - 1) / ((int64_t)rpb * 4);
+    const int64_t cap = ((int64_t)sm_count * 8 + gx - 1) / gx;
+    if (gy > cap) gy = cap;
+    if (gy < 1) gy = 1;
+    if (gy > 65535) gy = 65535;
+    dim3 grid((unsigned)gx, (unsigned)gy);
+    if (swiglu) eltwise_vec_kernel<T, true><<<grid, 256, 0, s>>>(xp, yp, rows, cols, tx, p);
+    else eltwise_vec_kernel<T, false><<<grid, 256, 0, s>>>(xp, yp, rows, cols, tx, p);
   } else {
     int grid = ceil_div_i64(rows * cols, 256);
     grid = grid > sm_count * 8 ? sm_count * 8 : grid;
@@ -92,29 +105,41 @@ cudaError_t launch_eltwise(int dtype, const void* x, void* y, int64_t rows, int6
 }
 
 // =====================================================================================================
-// row reductions: one warp per row, the row lives in registers
+// row reductions: one warp per row at a time, the row lives in registers; warps walk the rows with a
+// grid-wide stride so a launch is a few resident waves, not one block per handful of rows
 // =====================================================================================================
 template <typename T, int VPL, int MODE>
-__global__ void __launch_bounds__(128) rowop_warp_kernel(const T* __restrict__ x, T* __restrict__ y, int64_t rows, int n,
+__global__ void __launch_bounds__(256) rowop_warp_kernel(const T* __restrict__ x, T* __restrict__ y, int64_t rows, int n,
                                                          const T* __restrict__ gamma, const T* __restrict__ beta, float eps,
                                                          const __grid_constant__ EpiProgram pre) {
   constexpr int VE = Elem<T>::VEC;
   const int lane = threadIdx.x & 31;
-  const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  if (row >= rows) return;
   const int nvec = n / VE;
-  const T* xr = x + row * n;
+  const int64_t wstride = (int64_t)gridDim.x * (blockDim.x >> 5);
+  const int64_t row_first = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  uint4 raw[VPL];   // the NEXT row, in flight while the current one is reduced
+  if (row_first < rows) {
+#pragma unroll
+    for (int i = 0; i < VPL; ++i)
+      if (lane + 32 * i < nvec) raw[i] = ld_raw(x + row_first * n + (lane + 32 * i) * VE);
+  }
+  for (int64_t row = row_first; row < rows; row += wstride) {
   float v[VPL][VE];
 #pragma unroll
   for (int i = 0; i < VPL; ++i) {
     const int vi = lane + 32 * i;
     if (vi < nvec) {
-      ld_vec(xr + vi * VE, v[i]);
+      unpack_raw(raw[i], v[i]);
       epi_apply_vec<T, VE>(pre, v[i], row, (int64_t)vi * VE, n);
     } else {
 #pragma unroll
       for (int e = 0; e < VE; ++e) v[i][e] = (MODE == ROW_SOFTMAX) ? -INFINITY : 0.0f;
     }
+  }
+  if (row + wstride < rows) {
+#pragma unroll
+    for (int i = 0; i < VPL; ++i)
+      if (lane + 32 * i < nvec) raw[i] = ld_raw(x + (row + wstride) * n + (lane + 32 * i) * VE);
   }
   const float inv_n = 1.0f / (float)n;
   float mean = 0.0f, mul = 1.0f;
@@ -179,6 +204,7 @@ __global__ void __launch_bounds__(128) rowop_warp_kernel(const T* __restrict__ x
       st_vec(yr + vi * VE, o);
     }
   }
+  }  // row loop
 }
 
 // Fallback for rows that do not fit the register path or are not a multiple of the vector width:
@@ -245,13 +271,14 @@ static cudaError_t rowop_mode(const T* x, T* y, int64_t rows, int64_t n, const T
   if (rows == 0) return cudaSuccess;
   const int64_t nvec = n / VE;
   if (n % VE == 0 && nvec <= 32 * 16) {
-    const int grid = ceil_div_i64(rows, 4);
+    int grid = ceil_div_i64(rows, 8);
+    if (grid > 148 * 8) grid = 148 * 8;
     const int ni = (int)n;
-    if (nvec <= 32) rowop_warp_kernel<T, 1, MODE><<<grid, 128, 0, s>>>(x, y, rows, ni, g, b, eps, pre);
-    else if (nvec <= 64) rowop_warp_kernel<T, 2, MODE><<<grid, 128, 0, s>>>(x, y, rows, ni, g, b, eps, pre);
-    else if (nvec <= 128) rowop_warp_kernel<T, 4, MODE><<<grid, 128, 0, s>>>(x, y, rows, ni, g, b, eps, pre);
-    else if (nvec <= 256) rowop_warp_kernel<T, 8, MODE><<<grid, 128, 0, s>>>(x, y, rows, ni, g, b, eps, pre);
-    else rowop_warp_kernel<T, 16, MODE><<<grid, 128, 0, s>>>(x, y, rows, ni, g, b, eps, pre);
+    if (nvec <= 32) rowop_warp_kernel<T, 1, MODE><<<grid, 256, 0, s>>>(x, y, rows, ni, g, b, eps, pre);
+    else if (nvec <= 64) rowop_warp_kernel<T, 2, MODE><<<grid, 256, 0, s>>>(x, y, rows, ni, g, b, eps, pre);
+    else if (nvec <= 128) rowop_warp_kernel<T, 4, MODE><<<grid, 256, 0, s>>>(x, y, rows, ni, g, b, eps, pre);
+    else if (nvec <= 256) rowop_warp_kernel<T, 8, MODE><<<grid, 256, 0, s>>>(x, y, rows, ni, g, b, eps, pre);
+    else rowop_warp_kernel<T, 16, MODE><<<grid, 256, 0, s>>>(x, y, rows, ni, g, b, eps, pre);
   } else {
     rowop_block_kernel<T, MODE><<<(unsigned)rows, 256, 0, s>>>(x, y, rows, n, g, b, eps, pre);
   }

@@ -36,6 +36,20 @@ __device__ __forceinline__ void ld_vec(const __nv_bfloat16* p, float (&v)[8]) {
     v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
   }
 }
+// raw 128-bit load now, conversion later (software pipelining: the next row's loads are in flight
+// while the current row is reduced)
+__device__ __forceinline__ uint4 ld_raw(const void* p) { return *reinterpret_cast<const uint4*>(p); }
+__device__ __forceinline__ void unpack_raw(const uint4& t, float (&v)[4]) {
+  v[0] = __uint_as_float(t.x); v[1] = __uint_as_float(t.y); v[2] = __uint_as_float(t.z); v[3] = __uint_as_float(t.w);
+}
+__device__ __forceinline__ void unpack_raw(const uint4& t, float (&v)[8]) {
+  const uint32_t w[4] = {t.x, t.y, t.z, t.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    v[2 * i] = __uint_as_float(w[i] << 16);
+    v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+  }
+}
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&t);
@@ -68,6 +82,13 @@ __device__ __forceinline__ float gelu_tanh_f(float x) {
   return 0.5f * x * (1.0f + tanhf(u));
 }
 __device__ __forceinline__ float silu_f(float x) { return x / (1.0f + __expf(-x)); }
+// hardware tanh (relative error ~2^-11): only where the result is stored as bf16 (half-ulp 2^-9)
+__device__ __forceinline__ float gelu_tanh_bf16_f(float x) {
+  const float u = 0.7978845608028654f * (x + 0.044715f * x * x * x);
+  float t;
+  asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(u));
+  return 0.5f * x * (1.0f + t);
+}
 
 __device__ __forceinline__ float epi_ptr_ld(const void* p, int dtype, int64_t i) {
   return dtype == DT_F32 ? reinterpret_cast<const float*>(p)[i]
@@ -129,7 +150,7 @@ __device__ __forceinline__ void epi_apply_vec(const EpiProgram& p, float (&v)[NV
         break;
       case EPI_GELU_TANH:
 #pragma unroll
-        for (int j = 0; j < NV; ++j) v[j] = gelu_tanh_f(v[j]);
+        for (int j = 0; j < NV; ++j) v[j] = sizeof(T) == 2 ? gelu_tanh_bf16_f(v[j]) : gelu_tanh_f(v[j]);
         break;
       case EPI_SILU:
 #pragma unroll
