@@ -87,7 +87,10 @@ typedef struct mk_tensor_spec {
  *   RELU, GELU_TANH, SILU                               elementwise
  *   SCALE           y = f[0] * x
  *   CLAMP           y = min(max(x, f[0]), f[1])
- *   RESIDUAL_ADD    y = x + in[1]                       (same shape)
+ *   RESIDUAL_ADD    y = x + in[1]                       (same shape).  i[0] = 1: the sum is stored as fp32
+ *                                                       whatever the module dtype (an fp32 residual
+ *                                                       stream); such a value may only feed another
+ *                                                       RESIDUAL_ADD (either operand), LAYERNORM or RMSNORM
  *   SWIGLU          x[..., 2F] = [gate | up]; y[..., F] = silu(gate) * up
  *   LAYERNORM       rows over the last dim, biased variance, f[0] = eps inside the root;
  *                                                       param 0 = gamma, param 1 = beta (either may be absent)

@@ -184,6 +184,8 @@ class Module:
             elif kind == "groupnorm":
                 d.f[0] = a["eps"]
                 d.i[0] = a["groups"]
+            elif kind == "residual_add":
+                d.i[0] = 1 if a.get("store") == "f32" else 0
             elif kind == "linear":
                 d.i[0] = int(a["n"])
                 d.i[1] = weight_layout

@@ -275,7 +275,7 @@ mk_status mk_module_set_param(mk_module* m, int32_t op, int32_t slot, const void
   const mk_tensor_spec& x = m->values[o.in_id[0]].spec;
   const int64_t last = x.shape[x.rank - 1];
   mk_tensor_spec want{};
-  want.dtype = x.dtype;
+  want.dtype = m->values[0].spec.dtype;   // parameters always have the module's storage type
   bool ok = false;
   switch (o.d.kind) {
     case MK_OP_LINEAR:

@@ -279,11 +279,11 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       EpiProgram none;
       none.n = 0;
       EpiWarp ew;
-      ew.init(staging + q * EPI_WARP_BYTES, none, lane);
+      ew.init(staging + q * EPI_WARP_BYTES, none, lane, false);
       const int64_t row0 = (int64_t)b * S + (int64_t)qt * BQ + q * 32;
       const int64_t row_end = (int64_t)b * S + S;
       auto rowmap = [&](int r) -> int64_t { const int64_t g = row0 + r; return g < row_end ? g : -1; };
-      uint4 none_regs[4];
+      uint4 none_regs[8];
       const int64_t n_cols = (int64_t)H * HD;
 #pragma unroll
       for (int c = 0; c < 4; ++c) {

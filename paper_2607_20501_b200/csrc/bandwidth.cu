@@ -15,8 +15,8 @@ static inline int ceil_div_i64(int64_t a, int64_t b) { return (int)((a + b - 1) 
 // flight at a time: no per-element index arithmetic (a 64-bit division per vector made the first
 // version of this kernel ALU-bound), the bias slice of a thread never changes, and every access of a
 // warp is a contiguous run of a row.  tx = threads along a row (power of two <= 256).
-template <typename T, bool SWIGLU>
-__global__ void __launch_bounds__(256) eltwise_vec_kernel(const T* __restrict__ x, T* __restrict__ y, int64_t rows,
+template <typename T, typename TO, bool SWIGLU>
+__global__ void __launch_bounds__(256) eltwise_vec_kernel(const T* __restrict__ x, TO* __restrict__ y, int64_t rows,
                                                           int64_t cols, int tx, const __grid_constant__ EpiProgram p) {
   constexpr int VE = Elem<T>::VEC;
   constexpr int UNROLL = 4;
@@ -47,14 +47,14 @@ __global__ void __launch_bounds__(256) eltwise_vec_kernel(const T* __restrict__ 
           for (int e = 0; e < VE; ++e) v[q][e] = silu_f(v[q][e]) * u[q][e];
         }
         epi_apply_vec<T, VE>(p, v[q], r, col, cols);
-        st_vec(y + r * cols + col, v[q]);
+        st_vec_as<TO, VE>(y + r * cols + col, v[q]);
       }
     }
   }
 }
 
-template <typename T, bool SWIGLU>
-__global__ void __launch_bounds__(256) eltwise_scalar_kernel(const T* __restrict__ x, T* __restrict__ y, int64_t rows,
+template <typename T, typename TO, bool SWIGLU>
+__global__ void __launch_bounds__(256) eltwise_scalar_kernel(const T* __restrict__ x, TO* __restrict__ y, int64_t rows,
                                                              int64_t cols, const __grid_constant__ EpiProgram p) {
   const int64_t total = rows * cols;
   const int64_t stride = (int64_t)gridDim.x * blockDim.x;
@@ -63,16 +63,16 @@ __global__ void __launch_bounds__(256) eltwise_scalar_kernel(const T* __restrict
     const int64_t r = i / cols, c = i - r * cols;
     float v = Elem<T>::ld(x + r * in_ld + c);
     if (SWIGLU) v = silu_f(v) * Elem<T>::ld(x + r * in_ld + cols + c);
-    Elem<T>::st(y + i, epi_apply(p, v, r, c, cols));
+    Elem<TO>::st(y + i, epi_apply(p, v, r, c, cols));
   }
 }
 
-template <typename T>
+template <typename T, typename TO>
 static cudaError_t eltwise_dispatch(const void* x, void* y, int64_t rows, int64_t cols, bool swiglu, const EpiProgram& p,
                                     int sm_count, cudaStream_t s) {
   constexpr int VE = Elem<T>::VEC;
   const T* xp = (const T*)x;
-  T* yp = (T*)y;
+  TO* yp = (TO*)y;
   if (rows * cols == 0) return cudaSuccess;
   if (cols % VE == 0 && cols / VE <= INT32_MAX / 2) {
     const int vpr = (int)(cols / VE);
@@ -87,29 +87,30 @@ static cudaError_t eltwise_dispatch(const void* x, void* y, int64_t rows, int64_
     if (gy < 1) gy = 1;
     if (gy > 65535) gy = 65535;
     dim3 grid((unsigned)gx, (unsigned)gy);
-    if (swiglu) eltwise_vec_kernel<T, true><<<grid, 256, 0, s>>>(xp, yp, rows, cols, tx, p);
-    else eltwise_vec_kernel<T, false><<<grid, 256, 0, s>>>(xp, yp, rows, cols, tx, p);
+    if (swiglu) eltwise_vec_kernel<T, TO, true><<<grid, 256, 0, s>>>(xp, yp, rows, cols, tx, p);
+    else eltwise_vec_kernel<T, TO, false><<<grid, 256, 0, s>>>(xp, yp, rows, cols, tx, p);
   } else {
     int grid = ceil_div_i64(rows * cols, 256);
     grid = grid > sm_count * 8 ? sm_count * 8 : grid;
-    if (swiglu) eltwise_scalar_kernel<T, true><<<grid, 256, 0, s>>>(xp, yp, rows, cols, p);
-    else eltwise_scalar_kernel<T, false><<<grid, 256, 0, s>>>(xp, yp, rows, cols, p);
+    if (swiglu) eltwise_scalar_kernel<T, TO, true><<<grid, 256, 0, s>>>(xp, yp, rows, cols, p);
+    else eltwise_scalar_kernel<T, TO, false><<<grid, 256, 0, s>>>(xp, yp, rows, cols, p);
   }
   return cudaGetLastError();
 }
 
-cudaError_t launch_eltwise(int dtype, const void* x, void* y, int64_t rows, int64_t cols, bool swiglu, const EpiProgram& p,
-                           int sm_count, cudaStream_t s) {
-  return dtype == DT_F32 ? eltwise_dispatch<float>(x, y, rows, cols, swiglu, p, sm_count, s)
-                         : eltwise_dispatch<__nv_bfloat16>(x, y, rows, cols, swiglu, p, sm_count, s);
+cudaError_t launch_eltwise(int dtype, int out_dtype, const void* x, void* y, int64_t rows, int64_t cols, bool swiglu,
+                           const EpiProgram& p, int sm_count, cudaStream_t s) {
+  if (dtype == DT_F32) return out_dtype == DT_F32 ? eltwise_dispatch<float, float>(x, y, rows, cols, swiglu, p, sm_count, s) : cudaErrorInvalidValue;
+  return out_dtype == DT_F32 ? eltwise_dispatch<__nv_bfloat16, float>(x, y, rows, cols, swiglu, p, sm_count, s)
+                             : eltwise_dispatch<__nv_bfloat16, __nv_bfloat16>(x, y, rows, cols, swiglu, p, sm_count, s);
 }
 
 // =====================================================================================================
 // row reductions: one warp per row at a time, the row lives in registers; warps walk the rows with a
 // grid-wide stride so a launch is a few resident waves, not one block per handful of rows
 // =====================================================================================================
-template <typename T, int VPL, int MODE>
-__global__ void __launch_bounds__(256) rowop_warp_kernel(const T* __restrict__ x, T* __restrict__ y, int64_t rows, int n,
+template <typename TI, typename T, int VPL, int MODE>
+__global__ void __launch_bounds__(256) rowop_warp_kernel(const TI* __restrict__ x, T* __restrict__ y, int64_t rows, int n,
                                                          const T* __restrict__ gamma, const T* __restrict__ beta, float eps,
                                                          const __grid_constant__ EpiProgram pre) {
   constexpr int VE = Elem<T>::VEC;
@@ -117,11 +118,11 @@ __global__ void __launch_bounds__(256) rowop_warp_kernel(const T* __restrict__ x
   const int nvec = n / VE;
   const int64_t wstride = (int64_t)gridDim.x * (blockDim.x >> 5);
   const int64_t row_first = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  uint4 raw[VPL];   // the NEXT row, in flight while the current one is reduced
+  RawVec<TI, VE> raw[VPL];   // the NEXT row, in flight while the current one is reduced
   if (row_first < rows) {
 #pragma unroll
     for (int i = 0; i < VPL; ++i)
-      if (lane + 32 * i < nvec) raw[i] = ld_raw(x + row_first * n + (lane + 32 * i) * VE);
+      if (lane + 32 * i < nvec) raw[i].load(x + row_first * n + (lane + 32 * i) * VE);
   }
   for (int64_t row = row_first; row < rows; row += wstride) {
   float v[VPL][VE];
@@ -129,7 +130,7 @@ __global__ void __launch_bounds__(256) rowop_warp_kernel(const T* __restrict__ x
   for (int i = 0; i < VPL; ++i) {
     const int vi = lane + 32 * i;
     if (vi < nvec) {
-      unpack_raw(raw[i], v[i]);
+      raw[i].unpack(v[i]);
       epi_apply_vec<T, VE>(pre, v[i], row, (int64_t)vi * VE, n);
     } else {
 #pragma unroll
@@ -139,7 +140,7 @@ __global__ void __launch_bounds__(256) rowop_warp_kernel(const T* __restrict__ x
   if (row + wstride < rows) {
 #pragma unroll
     for (int i = 0; i < VPL; ++i)
-      if (lane + 32 * i < nvec) raw[i] = ld_raw(x + (row + wstride) * n + (lane + 32 * i) * VE);
+      if (lane + 32 * i < nvec) raw[i].load(x + (row + wstride) * n + (lane + 32 * i) * VE);
   }
   const float inv_n = 1.0f / (float)n;
   float mean = 0.0f, mul = 1.0f;
@@ -221,37 +222,37 @@ __device__ __forceinline__ float block_reduce(float v, float* sh) {
   return r;
 }
 
-template <typename T, int MODE>
-__global__ void __launch_bounds__(256) rowop_block_kernel(const T* __restrict__ x, T* __restrict__ y, int64_t rows, int64_t n,
+template <typename TI, typename T, int MODE>
+__global__ void __launch_bounds__(256) rowop_block_kernel(const TI* __restrict__ x, T* __restrict__ y, int64_t rows, int64_t n,
                                                           const T* __restrict__ gamma, const T* __restrict__ beta, float eps,
                                                           const __grid_constant__ EpiProgram pre) {
   __shared__ float sh[32];
   const int64_t row = blockIdx.x;
-  const T* xr = x + row * n;
+  const TI* xr = x + row * n;
   T* yr = y + row * n;
   const float inv_n = 1.0f / (float)n;
   float mean = 0.0f, mul = 1.0f, mx = 0.0f;
   if (MODE == ROW_LAYERNORM) {
     float s = 0.0f;
-    for (int64_t c = threadIdx.x; c < n; c += blockDim.x) s += epi_apply(pre, Elem<T>::ld(xr + c), row, c, n);
+    for (int64_t c = threadIdx.x; c < n; c += blockDim.x) s += epi_apply(pre, Elem<TI>::ld(xr + c), row, c, n);
     mean = block_reduce<0>(s, sh) * inv_n;
     float q = 0.0f;
-    for (int64_t c = threadIdx.x; c < n; c += blockDim.x) { const float d = epi_apply(pre, Elem<T>::ld(xr + c), row, c, n) - mean; q += d * d; }
+    for (int64_t c = threadIdx.x; c < n; c += blockDim.x) { const float d = epi_apply(pre, Elem<TI>::ld(xr + c), row, c, n) - mean; q += d * d; }
     mul = rsqrtf(block_reduce<0>(q, sh) * inv_n + eps);
   } else if (MODE == ROW_RMSNORM) {
     float q = 0.0f;
-    for (int64_t c = threadIdx.x; c < n; c += blockDim.x) { const float d = epi_apply(pre, Elem<T>::ld(xr + c), row, c, n); q += d * d; }
+    for (int64_t c = threadIdx.x; c < n; c += blockDim.x) { const float d = epi_apply(pre, Elem<TI>::ld(xr + c), row, c, n); q += d * d; }
     mul = rsqrtf(block_reduce<0>(q, sh) * inv_n + eps);
   } else {
     float m = -INFINITY;
-    for (int64_t c = threadIdx.x; c < n; c += blockDim.x) m = fmaxf(m, epi_apply(pre, Elem<T>::ld(xr + c), row, c, n));
+    for (int64_t c = threadIdx.x; c < n; c += blockDim.x) m = fmaxf(m, epi_apply(pre, Elem<TI>::ld(xr + c), row, c, n));
     mx = block_reduce<1>(m, sh);
     float s = 0.0f;
-    for (int64_t c = threadIdx.x; c < n; c += blockDim.x) s += __expf(epi_apply(pre, Elem<T>::ld(xr + c), row, c, n) - mx);
+    for (int64_t c = threadIdx.x; c < n; c += blockDim.x) s += __expf(epi_apply(pre, Elem<TI>::ld(xr + c), row, c, n) - mx);
     mul = 1.0f / block_reduce<0>(s, sh);
   }
   for (int64_t c = threadIdx.x; c < n; c += blockDim.x) {
-    const float v = epi_apply(pre, Elem<T>::ld(xr + c), row, c, n);
+    const float v = epi_apply(pre, Elem<TI>::ld(xr + c), row, c, n);
     float o;
     if (MODE == ROW_SOFTMAX) {
       o = __expf(v - mx) * mul;
@@ -264,8 +265,8 @@ __global__ void __launch_bounds__(256) rowop_block_kernel(const T* __restrict__ 
   }
 }
 
-template <typename T, int MODE>
-static cudaError_t rowop_mode(const T* x, T* y, int64_t rows, int64_t n, const T* g, const T* b, float eps,
+template <typename TI, typename T, int MODE>
+static cudaError_t rowop_mode(const TI* x, T* y, int64_t rows, int64_t n, const T* g, const T* b, float eps,
                               const EpiProgram& pre, cudaStream_t s) {
   constexpr int VE = Elem<T>::VEC;
   if (rows == 0) return cudaSuccess;
@@ -274,32 +275,33 @@ static cudaError_t rowop_mode(const T* x, T* y, int64_t rows, int64_t n, const T
     int grid = ceil_div_i64(rows, 8);
     if (grid > 148 * 8) grid = 148 * 8;
     const int ni = (int)n;
-    if (nvec <= 32) rowop_warp_kernel<T, 1, MODE><<<grid, 256, 0, s>>>(x, y, rows, ni, g, b, eps, pre);
-    else if (nvec <= 64) rowop_warp_kernel<T, 2, MODE><<<grid, 256, 0, s>>>(x, y, rows, ni, g, b, eps, pre);
-    else if (nvec <= 128) rowop_warp_kernel<T, 4, MODE><<<grid, 256, 0, s>>>(x, y, rows, ni, g, b, eps, pre);
-    else if (nvec <= 256) rowop_warp_kernel<T, 8, MODE><<<grid, 256, 0, s>>>(x, y, rows, ni, g, b, eps, pre);
-    else rowop_warp_kernel<T, 16, MODE><<<grid, 256, 0, s>>>(x, y, rows, ni, g, b, eps, pre);
+    if (nvec <= 32) rowop_warp_kernel<TI, T, 1, MODE><<<grid, 256, 0, s>>>(x, y, rows, ni, g, b, eps, pre);
+    else if (nvec <= 64) rowop_warp_kernel<TI, T, 2, MODE><<<grid, 256, 0, s>>>(x, y, rows, ni, g, b, eps, pre);
+    else if (nvec <= 128) rowop_warp_kernel<TI, T, 4, MODE><<<grid, 256, 0, s>>>(x, y, rows, ni, g, b, eps, pre);
+    else if (nvec <= 256) rowop_warp_kernel<TI, T, 8, MODE><<<grid, 256, 0, s>>>(x, y, rows, ni, g, b, eps, pre);
+    else rowop_warp_kernel<TI, T, 16, MODE><<<grid, 256, 0, s>>>(x, y, rows, ni, g, b, eps, pre);
   } else {
-    rowop_block_kernel<T, MODE><<<(unsigned)rows, 256, 0, s>>>(x, y, rows, n, g, b, eps, pre);
+    rowop_block_kernel<TI, T, MODE><<<(unsigned)rows, 256, 0, s>>>(x, y, rows, n, g, b, eps, pre);
   }
   return cudaGetLastError();
 }
 
-template <typename T>
+template <typename TI, typename T>
 static cudaError_t rowop_dispatch(int mode, const void* x, void* y, int64_t rows, int64_t n, const void* g, const void* b,
                                   float eps, const EpiProgram& pre, cudaStream_t s) {
-  const T* xp = (const T*)x; T* yp = (T*)y; const T* gp = (const T*)g; const T* bp = (const T*)b;
+  const TI* xp = (const TI*)x; T* yp = (T*)y; const T* gp = (const T*)g; const T* bp = (const T*)b;
   switch (mode) {
-    case ROW_LAYERNORM: return rowop_mode<T, ROW_LAYERNORM>(xp, yp, rows, n, gp, bp, eps, pre, s);
-    case ROW_RMSNORM: return rowop_mode<T, ROW_RMSNORM>(xp, yp, rows, n, gp, bp, eps, pre, s);
-    default: return rowop_mode<T, ROW_SOFTMAX>(xp, yp, rows, n, gp, bp, eps, pre, s);
+    case ROW_LAYERNORM: return rowop_mode<TI, T, ROW_LAYERNORM>(xp, yp, rows, n, gp, bp, eps, pre, s);
+    case ROW_RMSNORM: return rowop_mode<TI, T, ROW_RMSNORM>(xp, yp, rows, n, gp, bp, eps, pre, s);
+    default: return rowop_mode<TI, T, ROW_SOFTMAX>(xp, yp, rows, n, gp, bp, eps, pre, s);
   }
 }
 
-cudaError_t launch_rowop(int dtype, int mode, const void* x, void* y, int64_t rows, int64_t n, const void* gamma,
+cudaError_t launch_rowop(int dtype, int in_dtype, int mode, const void* x, void* y, int64_t rows, int64_t n, const void* gamma,
                          const void* beta, float eps, const EpiProgram& pre, cudaStream_t s) {
-  return dtype == DT_F32 ? rowop_dispatch<float>(mode, x, y, rows, n, gamma, beta, eps, pre, s)
-                         : rowop_dispatch<__nv_bfloat16>(mode, x, y, rows, n, gamma, beta, eps, pre, s);
+  if (dtype == DT_F32) return in_dtype == DT_F32 ? rowop_dispatch<float, float>(mode, x, y, rows, n, gamma, beta, eps, pre, s) : cudaErrorInvalidValue;
+  return in_dtype == DT_F32 ? rowop_dispatch<float, __nv_bfloat16>(mode, x, y, rows, n, gamma, beta, eps, pre, s)
+                            : rowop_dispatch<__nv_bfloat16, __nv_bfloat16>(mode, x, y, rows, n, gamma, beta, eps, pre, s);
 }
 
 // =====================================================================================================

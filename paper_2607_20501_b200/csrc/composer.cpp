@@ -23,6 +23,12 @@ bool same_spec(const mk_tensor_spec& a, const mk_tensor_spec& b) {
     if (a.shape[i] != b.shape[i]) return false;
   return true;
 }
+static bool same_shape(const mk_tensor_spec& a, const mk_tensor_spec& b) {
+  if (a.rank != b.rank || a.layout != b.layout) return false;
+  for (int i = 0; i < a.rank; ++i)
+    if (a.shape[i] != b.shape[i]) return false;
+  return true;
+}
 bool is_eltwise(int32_t kind) {
   switch (kind) {
     case MK_OP_BIAS_ADD:
@@ -83,6 +89,11 @@ mk_status infer_shapes(Module& m, std::string& err) {
     const mk_tensor_spec x = m.values[op.in_id[0]].spec;
     const int64_t last = x.shape[x.rank - 1];
     mk_tensor_spec y = x;
+    y.dtype = dtype;
+    // an fp32 value inside a bf16 module (an fp32 residual stream) may only feed a residual add or a row norm
+    const bool takes_f32 = d.kind == MK_OP_RESIDUAL_ADD || d.kind == MK_OP_RMSNORM || d.kind == MK_OP_LAYERNORM;
+    for (int k = 0; k < op.n_in; ++k)
+      if (m.values[op.in_id[k]].spec.dtype != dtype && !takes_f32) { err = at + "this operator does not take an fp32 residual-stream value"; return MK_ERR_SHAPE_MISMATCH; }
     switch (d.kind) {
       case MK_OP_LINEAR: {
         if (x.rank != 2) { err = at + "LINEAR takes a rank-2 input"; return MK_ERR_SHAPE_MISMATCH; }
@@ -107,7 +118,9 @@ mk_status infer_shapes(Module& m, std::string& err) {
         if (!(d.f[0] <= d.f[1])) { err = at + "CLAMP needs f[0] <= f[1]"; return MK_ERR_INVALID_ARG; }
         break;
       case MK_OP_RESIDUAL_ADD:
-        if (!same_spec(x, m.values[op.in_id[1]].spec)) { err = at + "RESIDUAL_ADD operands differ in shape"; return MK_ERR_SHAPE_MISMATCH; }
+        if (!same_shape(x, m.values[op.in_id[1]].spec)) { err = at + "RESIDUAL_ADD operands differ in shape"; return MK_ERR_SHAPE_MISMATCH; }
+        if (d.i[0] != 0 && d.i[0] != 1) { err = at + "RESIDUAL_ADD i[0] must be 0 (module dtype) or 1 (fp32 store)"; return MK_ERR_INVALID_ARG; }
+        if (d.i[0] == 1) y.dtype = MK_F32;
         break;
       case MK_OP_SWIGLU:
         if (last % 2) { err = at + "SWIGLU needs an even last dimension"; return MK_ERR_SHAPE_MISMATCH; }
@@ -356,7 +369,7 @@ mk_status build_epi(const Module& m, int lo, int hi, const Resolved& r, EpiProgr
     switch (op.d.kind) {
       case MK_OP_BIAS_ADD:
         if (!op.param[0].set) { err = "op " + std::to_string(j) + ": bias has not been set"; return MK_ERR_PARAM_MISSING; }
-        e.kind = EPI_BIAS; e.ptr = op.param[0].ptr; break;
+        e.kind = EPI_BIAS; e.ptr = op.param[0].ptr; e.ptr_dtype = p.dtype; break;
       case MK_OP_RELU: e.kind = EPI_RELU; break;
       case MK_OP_GELU_TANH: e.kind = EPI_GELU_TANH; break;
       case MK_OP_SILU: e.kind = EPI_SILU; break;
@@ -364,6 +377,7 @@ mk_status build_epi(const Module& m, int lo, int hi, const Resolved& r, EpiProgr
       case MK_OP_CLAMP: e.kind = EPI_CLAMP; e.a = (float)op.d.f[0]; e.b = (float)op.d.f[1]; break;
       case MK_OP_RESIDUAL_ADD:
         e.kind = EPI_RESIDUAL; e.ptr = r.value_ptr[op.in_id[1]];
+        e.ptr_dtype = m.values[op.in_id[1]].spec.dtype == MK_F32 ? DT_F32 : DT_BF16;
         if (!e.ptr) { err = "residual operand is not materialised"; return MK_ERR_CONTRACT_VIOLATION; }
         break;
       default:

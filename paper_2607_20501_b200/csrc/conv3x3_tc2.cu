@@ -165,7 +165,7 @@ conv3x3_tc2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     // ------------------------------------------------------------ epilogue: 128 tile rows = 2 output rows x 64 pitch
     const int q = warp & 3;
     EpiWarp ew;
-    ew.init(staging + q * EPI_WARP_BYTES, epi, lane);
+    ew.init(staging + q * EPI_WARP_BYTES, epi, lane, false);
     ew.load_bias(epi, 0, C_OUT, C_OUT);          // the bias slice is the same for every tile: once
     const int chunks = C_OUT / 32;
     bool ok = true;
@@ -179,7 +179,7 @@ conv3x3_tc2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
       const int64_t pix0 = ((int64_t)n * H + h) * W;
       const bool row_ok = h < H;
       auto rowmap = [&](int r) -> int64_t { return (row_ok && w0 + r < W) ? pix0 + w0 + r : -1; };
-      uint4 res_regs[4];
+      uint4 res_regs[8];
       ew.prefetch_res(epi, rowmap, 0, C_OUT, res_regs);
       ok = tc::mbar_wait(&sh->tfull[acc], (it >> 1) & 1, abort_flag, status, tc::WAIT_TMEM_FULL);
       ok = __all_sync(0xffffffffu, ok ? 1 : 0) != 0;

@@ -66,6 +66,53 @@ __device__ __forceinline__ void st_vec(__nv_bfloat16* p, const float (&v)[8]) {
   *reinterpret_cast<uint4*>(p) = t;
 }
 
+// NV fp32 registers -> NV consecutive elements of type TO (16-byte aligned destination)
+template <typename TO, int NV>
+__device__ __forceinline__ void st_vec_as(TO* p, const float (&v)[NV]) {
+  if constexpr (sizeof(TO) == 4) {
+#pragma unroll
+    for (int j = 0; j < NV; j += 4) *reinterpret_cast<float4*>(reinterpret_cast<float*>(p) + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+  } else {
+#pragma unroll
+    for (int j = 0; j < NV; j += 8) {
+      uint4 t;
+      t.x = pack_bf16x2(v[j], v[j + 1]);
+      t.y = pack_bf16x2(v[j + 2], v[j + 3]);
+      t.z = pack_bf16x2(v[j + 4], v[j + 5]);
+      t.w = pack_bf16x2(v[j + 6], v[j + 7]);
+      *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p) + j) = t;
+    }
+  }
+}
+// NV consecutive elements of type TI, raw (16-byte pieces), and their later conversion to fp32
+template <typename TI, int NV> struct RawVec {
+  static constexpr int N16 = NV * (int)sizeof(TI) / 16;
+  uint4 r[N16];
+  __device__ __forceinline__ void load(const TI* p) {
+#pragma unroll
+    for (int i = 0; i < N16; ++i) r[i] = *reinterpret_cast<const uint4*>(reinterpret_cast<const uint8_t*>(p) + 16 * i);
+  }
+  __device__ __forceinline__ void unpack(float (&v)[NV]) const {
+    if constexpr (sizeof(TI) == 4) {
+#pragma unroll
+      for (int i = 0; i < N16; ++i) {
+        v[4 * i] = __uint_as_float(r[i].x); v[4 * i + 1] = __uint_as_float(r[i].y);
+        v[4 * i + 2] = __uint_as_float(r[i].z); v[4 * i + 3] = __uint_as_float(r[i].w);
+      }
+    } else {
+#pragma unroll
+      for (int i = 0; i < N16; ++i) {
+        const uint32_t w[4] = {r[i].x, r[i].y, r[i].z, r[i].w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          v[8 * i + 2 * k] = __uint_as_float(w[k] << 16);
+          v[8 * i + 2 * k + 1] = __uint_as_float(w[k] & 0xffff0000u);
+        }
+      }
+    }
+  }
+};
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
@@ -106,7 +153,7 @@ __device__ __forceinline__ float epi_apply(const EpiProgram& p, float v, int64_t
       case EPI_SILU: v = silu_f(v); break;
       case EPI_SCALE: v *= o.a; break;
       case EPI_CLAMP: v = fminf(fmaxf(v, o.a), o.b); break;
-      case EPI_RESIDUAL: v += epi_ptr_ld(o.ptr, p.dtype, row * ld + col); break;
+      case EPI_RESIDUAL: v += epi_ptr_ld(o.ptr, o.ptr_dtype, row * ld + col); break;
       default: break;
     }
   }
@@ -134,13 +181,24 @@ __device__ __forceinline__ void epi_apply_vec(const EpiProgram& p, float (&v)[NV
         break;
       }
       case EPI_RESIDUAL: {
-        const T* r = reinterpret_cast<const T*>(o.ptr) + row * ld + col0;
+        if (o.ptr_dtype == DT_F32) {   // an fp32 residual stream next to bf16 activations
+          const float* r = reinterpret_cast<const float*>(o.ptr) + row * ld + col0;
 #pragma unroll
-        for (int j = 0; j < NV; j += VE) {
-          float t[VE];
-          ld_vec(r + j, t);
+          for (int j = 0; j < NV; j += 4) {
+            float t[4];
+            ld_vec(r + j, t);
 #pragma unroll
-          for (int q = 0; q < VE; ++q) v[j + q] += t[q];
+            for (int q = 0; q < 4; ++q) v[j + q] += t[q];
+          }
+        } else {
+          const T* r = reinterpret_cast<const T*>(o.ptr) + row * ld + col0;
+#pragma unroll
+          for (int j = 0; j < NV; j += VE) {
+            float t[VE];
+            ld_vec(r + j, t);
+#pragma unroll
+            for (int q = 0; q < VE; ++q) v[j + q] += t[q];
+          }
         }
         break;
       }

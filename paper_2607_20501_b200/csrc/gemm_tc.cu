@@ -70,7 +70,7 @@ __device__ __forceinline__ void tile_coords(int t, int num_m, int num_n, int& mi
 
 template <int CTAS, bool SWIGLU>
 __global__ void __launch_bounds__(THREADS, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, __nv_bfloat16* __restrict__ out, int M,
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, void* __restrict__ out, int out_f32, int M,
                int N, int K, int up_row_offset, const __grid_constant__ EpiProgram epi, unsigned int* status) {
   using C = Cfg<CTAS>;
   constexpr int STAGES = C::STAGES;
@@ -209,7 +209,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int half = (warp - 2) >> 2;
     constexpr int CHUNKS = OUT_N / 32;
     EpiWarp ew;
-    ew.init(staging + (warp - 2) * EPI_WARP_BYTES, epi, lane);
+    ew.init(staging + (warp - 2) * EPI_WARP_BYTES, epi, lane, out_f32 != 0);
     bool ok = true;
     int it = 0;
     for (int t = unit_id; t < total_tiles && ok; t += num_units, ++it) {
@@ -219,7 +219,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int64_t row0 = (int64_t)(mi * CTAS + (int)rank) * BM + q * 32;
       auto rowmap = [&](int r) -> int64_t { const int64_t g = row0 + r; return g < M ? g : -1; };
       const int64_t col_base = (int64_t)ni * OUT_N;
-      uint4 res_regs[4];
+      uint4 res_regs[8];
       ew.load_bias(epi, col_base, OUT_N, N);
       ew.prefetch_res(epi, rowmap, col_base + half * 32, N, res_regs);
       ok = tc::mbar_wait(&sh->tfull[acc], (it >> 1) & 1, abort_flag, status, tc::WAIT_TMEM_FULL);
@@ -271,7 +271,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 }
 
 template <int CTAS>
-cudaError_t plan_impl(GemmTcPlan* p, const void* a, const void* w_nk, void* y, int64_t m, int64_t n, int64_t k, bool swiglu,
+cudaError_t plan_impl(GemmTcPlan* p, const void* a, const void* w_nk, void* y, bool out_f32, int64_t m, int64_t n, int64_t k, bool swiglu,
                       const EpiProgram& epi, int sm_count) {
   if (k % 8 || n % 8 || m < 1 || n < 1 || k < 1) return cudaErrorInvalidValue;
   if (m > INT32_MAX || n > INT32_MAX || k > INT32_MAX) return cudaErrorInvalidValue;
@@ -281,6 +281,7 @@ cudaError_t plan_impl(GemmTcPlan* p, const void* a, const void* w_nk, void* y, i
   e = encode_tmap_2d_bf16(&p->tm_b, w_nk, (uint64_t)w_rows, (uint64_t)k, (uint64_t)k, BN / 2, BK);
   if (e != cudaSuccess) return e;
   p->out = y;
+  p->out_f32 = out_f32;
   p->m = (int)m; p->n = (int)n; p->k = (int)k;
   p->swiglu = swiglu;
   p->epi = epi;
@@ -313,21 +314,21 @@ cudaError_t launch_impl(const GemmTcPlan& p, cudaStream_t s) {
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   unsigned int* status = kernel_status_ptr();
-  __nv_bfloat16* out = (__nv_bfloat16*)p.out;
-  if (p.swiglu) return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<CTAS, true>, p.tm_a, p.tm_b, out, p.m, p.n, p.k, p.n, p.epi, status);
-  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<CTAS, false>, p.tm_a, p.tm_b, out, p.m, p.n, p.k, 0, p.epi, status);
+  const int out_f32 = p.out_f32 ? 1 : 0;
+  if (p.swiglu) return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<CTAS, true>, p.tm_a, p.tm_b, p.out, out_f32, p.m, p.n, p.k, p.n, p.epi, status);
+  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<CTAS, false>, p.tm_a, p.tm_b, p.out, out_f32, p.m, p.n, p.k, 0, p.epi, status);
 }
 
 }  // namespace
 
-cudaError_t gemm_tc_plan(GemmTcPlan* p, const void* a, const void* w_nk, void* y, int64_t m, int64_t n, int64_t k, bool swiglu,
+cudaError_t gemm_tc_plan(GemmTcPlan* p, const void* a, const void* w_nk, void* y, bool out_f32, int64_t m, int64_t n, int64_t k, bool swiglu,
                          const EpiProgram& epi, int sm_count) {
-  return plan_impl<1>(p, a, w_nk, y, m, n, k, swiglu, epi, sm_count);
+  return plan_impl<1>(p, a, w_nk, y, out_f32, m, n, k, swiglu, epi, sm_count);
 }
 cudaError_t launch_gemm_tc(const GemmTcPlan& p, cudaStream_t s) { return launch_impl<1>(p, s); }
-cudaError_t gemm_tc2_plan(GemmTcPlan* p, const void* a, const void* w_nk, void* y, int64_t m, int64_t n, int64_t k, bool swiglu,
+cudaError_t gemm_tc2_plan(GemmTcPlan* p, const void* a, const void* w_nk, void* y, bool out_f32, int64_t m, int64_t n, int64_t k, bool swiglu,
                           const EpiProgram& epi, int sm_count) {
-  return plan_impl<2>(p, a, w_nk, y, m, n, k, swiglu, epi, sm_count);
+  return plan_impl<2>(p, a, w_nk, y, out_f32, m, n, k, swiglu, epi, sm_count);
 }
 cudaError_t launch_gemm_tc2(const GemmTcPlan& p, cudaStream_t s) { return launch_impl<2>(p, s); }
 

@@ -14,6 +14,10 @@ namespace mk {
 namespace {
 
 int dt(const Module& m) { return m.values[0].spec.dtype == MK_F32 ? DT_F32 : DT_BF16; }
+int dt_of(const mk_tensor_spec& s) { return s.dtype == MK_F32 ? DT_F32 : DT_BF16; }
+// the piece's first input / its output stored in the module's dtype (not an fp32 residual stream)
+bool in_is_module_dtype(const Module& m, int lo) { return m.vspec(m.ops[lo].in_id[0]).dtype == m.values[0].spec.dtype; }
+bool out_is_module_dtype(const Module& m, int hi) { return m.vspec(m.ops[hi - 1].out_id).dtype == m.values[0].spec.dtype; }
 
 // ops lo+1.. read their predecessor as first input; nothing but the last value leaves the piece;
 // residual operands come from outside the piece.
@@ -43,7 +47,7 @@ int64_t rows_of(const mk_tensor_spec& s) { return numel(s) / last_dim(s); }
 
 // ------------------------------------------------------------------ eltwise chain
 bool eltwise_match(const Module& m, int lo, int hi) {
-  if (!is_chain(m, lo, hi)) return false;
+  if (!is_chain(m, lo, hi) || !in_is_module_dtype(m, lo)) return false;
   const bool sw = m.ops[lo].d.kind == MK_OP_SWIGLU;
   return all_eltwise(m, lo + (sw ? 1 : 0), hi);
 }
@@ -56,8 +60,8 @@ mk_status eltwise_emit(const Module& m, int lo, int hi, const Resolved& r, std::
   void* y = r.value_ptr[m.ops[hi - 1].out_id];
   const mk_tensor_spec& ys = m.vspec(m.ops[hi - 1].out_id);
   const int64_t rows = rows_of(ys), cols = last_dim(ys);
-  const int d = dt(m), sms = m.ctx->sm_count;
-  out.push_back([=](cudaStream_t s) { return launch_eltwise(d, x, y, rows, cols, sw, p, sms, s); });
+  const int d = dt(m), od = dt_of(ys), sms = m.ctx->sm_count;
+  out.push_back([=](cudaStream_t s) { return launch_eltwise(d, od, x, y, rows, cols, sw, p, sms, s); });
   return MK_OK;
 }
 
@@ -66,7 +70,9 @@ bool is_rowop(int32_t k) { return k == MK_OP_LAYERNORM || k == MK_OP_RMSNORM || 
 int row_mode(int32_t k) { return k == MK_OP_LAYERNORM ? ROW_LAYERNORM : k == MK_OP_RMSNORM ? ROW_RMSNORM : ROW_SOFTMAX; }
 
 bool rowop_match(const Module& m, int lo, int hi) {
-  return is_chain(m, lo, hi) && is_rowop(m.ops[hi - 1].d.kind) && all_eltwise(m, lo, hi - 1);
+  if (!is_chain(m, lo, hi) || !is_rowop(m.ops[hi - 1].d.kind) || !all_eltwise(m, lo, hi - 1)) return false;
+  // an fp32 residual-stream input is taken by the norm itself, not through an elementwise prefix
+  return in_is_module_dtype(m, lo) || hi - lo == 1;
 }
 mk_status rowop_emit(const Module& m, int lo, int hi, const Resolved& r, std::vector<Launch>& out, std::string& err) {
   EpiProgram p;
@@ -80,14 +86,14 @@ mk_status rowop_emit(const Module& m, int lo, int hi, const Resolved& r, std::ve
   const void* g = op.param[0].set ? op.param[0].ptr : nullptr;
   const void* b = op.param[1].set ? op.param[1].ptr : nullptr;
   const float eps = (float)op.d.f[0];
-  const int mode = row_mode(op.d.kind), d = dt(m);
-  out.push_back([=](cudaStream_t s) { return launch_rowop(d, mode, x, y, rows, n, g, b, eps, p, s); });
+  const int mode = row_mode(op.d.kind), d = dt(m), id = dt_of(m.vspec(m.ops[lo].in_id[0]));
+  out.push_back([=](cudaStream_t s) { return launch_rowop(d, id, mode, x, y, rows, n, g, b, eps, p, s); });
   return MK_OK;
 }
 
 // ------------------------------------------------------------------ GroupNorm (two launches + scratch)
 bool groupnorm_match(const Module& m, int lo, int hi) {
-  return is_chain(m, lo, hi) && m.ops[hi - 1].d.kind == MK_OP_GROUPNORM && all_eltwise(m, lo, hi - 1);
+  return is_chain(m, lo, hi) && m.ops[hi - 1].d.kind == MK_OP_GROUPNORM && all_eltwise(m, lo, hi - 1) && in_is_module_dtype(m, lo);
 }
 size_t groupnorm_scratch(const Module& m, int, int hi) {
   const mk_tensor_spec& s = m.vspec(m.ops[hi - 1].out_id);
@@ -117,7 +123,7 @@ mk_status groupnorm_emit(const Module& m, int lo, int hi, const Resolved& r, std
 // ------------------------------------------------------------------ GEMM family
 // LINEAR [SWIGLU] [elementwise]*
 bool gemm_shape(const Module& m, int lo, int hi, bool* swiglu, int* tail_lo) {
-  if (!is_chain(m, lo, hi) || m.ops[lo].d.kind != MK_OP_LINEAR) return false;
+  if (!is_chain(m, lo, hi) || m.ops[lo].d.kind != MK_OP_LINEAR || !in_is_module_dtype(m, lo)) return false;
   int t = lo + 1;
   *swiglu = t < hi && m.ops[t].d.kind == MK_OP_SWIGLU;
   if (*swiglu) ++t;
@@ -141,8 +147,8 @@ mk_status gemm_simt_emit(const Module& m, int lo, int hi, const Resolved& r, std
   const mk_tensor_spec& xs = m.vspec(op.in_id[0]);
   const int64_t M = xs.shape[0], K = xs.shape[1], N = last_dim(m.vspec(m.ops[hi - 1].out_id));
   const bool wt = op.d.i[1] == MK_LAYOUT_TRANSPOSED;
-  const int d = dt(m);
-  out.push_back([=](cudaStream_t s) { return launch_gemm_simt(d, a, w, wt, y, M, N, K, sw, p, s); });
+  const int d = dt(m), od = dt_of(m.vspec(m.ops[hi - 1].out_id));
+  out.push_back([=](cudaStream_t s) { return launch_gemm_simt(d, od, a, w, wt, y, M, N, K, sw, p, s); });
   return MK_OK;
 }
 
@@ -169,8 +175,9 @@ mk_status gemm_tc_emit_impl(const Module& m, int lo, int hi, const Resolved& r, 
   auto plan = std::make_shared<GemmTcPlan>();
   const void* a = r.value_ptr[op.in_id[0]];
   void* y = r.value_ptr[m.ops[hi - 1].out_id];
-  cudaError_t e = pair ? gemm_tc2_plan(plan.get(), a, op.param[0].ptr, y, M, N, K, sw, p, m.ctx->sm_count)
-                       : gemm_tc_plan(plan.get(), a, op.param[0].ptr, y, M, N, K, sw, p, m.ctx->sm_count);
+  const bool of32 = m.vspec(m.ops[hi - 1].out_id).dtype == MK_F32;
+  cudaError_t e = pair ? gemm_tc2_plan(plan.get(), a, op.param[0].ptr, y, of32, M, N, K, sw, p, m.ctx->sm_count)
+                       : gemm_tc_plan(plan.get(), a, op.param[0].ptr, y, of32, M, N, K, sw, p, m.ctx->sm_count);
   if (e != cudaSuccess) { err = std::string("gemm_tc plan: ") + cudaGetErrorString(e); return MK_ERR_CUDA; }
   if (pair) out.push_back([plan](cudaStream_t s) { return launch_gemm_tc2(*plan, s); });
   else out.push_back([plan](cudaStream_t s) { return launch_gemm_tc(*plan, s); });
@@ -218,7 +225,7 @@ mk_status linear_rownorm_emit(const Module& m, int lo, int hi, const Resolved& r
 
 // ------------------------------------------------------------------ convolution
 bool conv_simt_match(const Module& m, int lo, int hi) {
-  return is_chain(m, lo, hi) && m.ops[lo].d.kind == MK_OP_CONV2D_3X3 && all_eltwise(m, lo + 1, hi);
+  return is_chain(m, lo, hi) && m.ops[lo].d.kind == MK_OP_CONV2D_3X3 && all_eltwise(m, lo + 1, hi) && out_is_module_dtype(m, hi);
 }
 mk_status conv_simt_emit(const Module& m, int lo, int hi, const Resolved& r, std::vector<Launch>& out, std::string& err) {
   EpiProgram p;

@@ -28,12 +28,12 @@ constexpr int EPI_MAX = 8;
 struct EpiOp {
   int32_t kind;
   float a, b;
-  int32_t pad;
+  int32_t ptr_dtype;  // element type behind ptr (a residual may be fp32 in a bf16 module)
   const void* ptr;
 };
 struct EpiProgram {
   int32_t n = 0;
-  int32_t dtype = DT_BF16;  // element type behind ptr
+  int32_t dtype = DT_BF16;  // the module's storage type (bias vectors, default for everything)
   EpiOp op[EPI_MAX];
 };
 
@@ -43,13 +43,14 @@ cudaError_t kernel_status_fetch_and_clear(unsigned int* out);
 
 // ---- HBM-bound kernels ------------------------------------------------------------------------------
 // y[rows, cols] = program(x).  swiglu: x is [rows, 2*cols] = [gate | up] and the program runs on
-// silu(gate) * up.
-cudaError_t launch_eltwise(int dtype, const void* x, void* y, int64_t rows, int64_t cols, bool swiglu,
+// silu(gate) * up.  x has the module dtype; y has out_dtype (fp32 for an fp32 residual stream).
+cudaError_t launch_eltwise(int dtype, int out_dtype, const void* x, void* y, int64_t rows, int64_t cols, bool swiglu,
                            const EpiProgram& p, int sm_count, cudaStream_t s);
 
 enum RowMode : int32_t { ROW_LAYERNORM = 0, ROW_RMSNORM = 1, ROW_SOFTMAX = 2 };
 // Row-wise reduction over the last dimension of program(x)[rows, n]; gamma/beta may be null.
-cudaError_t launch_rowop(int dtype, int mode, const void* x, void* y, int64_t rows, int64_t n,
+// x has in_dtype (fp32 when it is an fp32 residual stream), y / gamma / beta have dtype.
+cudaError_t launch_rowop(int dtype, int in_dtype, int mode, const void* x, void* y, int64_t rows, int64_t n,
                          const void* gamma, const void* beta, float eps, const EpiProgram& pre,
                          cudaStream_t s);
 
@@ -68,7 +69,7 @@ cudaError_t launch_groupnorm_apply(int dtype, const void* x, void* y, int64_t nb
 // ---- plain-ALU (SIMT) kernels: any shape, fp32 or bf16, fp32 accumulation -------------------------
 // Y[M, N] = program(A[M, K] @ W); W is [K, N] row-major, or [N, K] when w_transposed.
 // swiglu: W has 2N logical columns [gate | up] and Y = program(silu(A Wg) * (A Wu)).
-cudaError_t launch_gemm_simt(int dtype, const void* a, const void* w, bool w_transposed, void* y,
+cudaError_t launch_gemm_simt(int dtype, int out_dtype, const void* a, const void* w, bool w_transposed, void* y,
                              int64_t m, int64_t n, int64_t k, bool swiglu, const EpiProgram& p,
                              cudaStream_t s);
 // Small-shape fused chain: one CTA owns whole rows, so the row norm follows the GEMM in-kernel.

@@ -11,9 +11,9 @@ namespace mk {
 // =====================================================================================================
 // tiled GEMM, 64x64 tile, 16x16 threads, 4x4 micro-tile
 // =====================================================================================================
-template <typename T, bool SWIGLU>
+template <typename T, typename TO, bool SWIGLU>
 __global__ void __launch_bounds__(256) gemm_simt_kernel(const T* __restrict__ a, const T* __restrict__ w, bool wt,
-                                                        T* __restrict__ y, int64_t M, int64_t N, int64_t K,
+                                                        TO* __restrict__ y, int64_t M, int64_t N, int64_t K,
                                                         const __grid_constant__ EpiProgram p) {
   constexpr int BM = 64, BN = 64, BK = 16;
   __shared__ float As[BK][BM + 1];
@@ -66,25 +66,26 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const T* __restrict__ a,
       if (gm < M && gn < N) {
         float v = acc[i][j];
         if (SWIGLU) v = silu_f(v) * acc2[i][j];
-        Elem<T>::st(y + gm * N + gn, epi_apply(p, v, gm, gn, N));
+        Elem<TO>::st(y + gm * N + gn, epi_apply(p, v, gm, gn, N));
       }
     }
 }
 
-template <typename T>
+template <typename T, typename TO>
 static cudaError_t gemm_simt_dispatch(const void* a, const void* w, bool wt, void* y, int64_t m, int64_t n, int64_t k, bool swiglu,
                                       const EpiProgram& p, cudaStream_t s) {
   if (m == 0 || n == 0) return cudaSuccess;
   dim3 grid((unsigned)((n + 63) / 64), (unsigned)((m + 63) / 64));
-  if (swiglu) gemm_simt_kernel<T, true><<<grid, 256, 0, s>>>((const T*)a, (const T*)w, wt, (T*)y, m, n, k, p);
-  else gemm_simt_kernel<T, false><<<grid, 256, 0, s>>>((const T*)a, (const T*)w, wt, (T*)y, m, n, k, p);
+  if (swiglu) gemm_simt_kernel<T, TO, true><<<grid, 256, 0, s>>>((const T*)a, (const T*)w, wt, (TO*)y, m, n, k, p);
+  else gemm_simt_kernel<T, TO, false><<<grid, 256, 0, s>>>((const T*)a, (const T*)w, wt, (TO*)y, m, n, k, p);
   return cudaGetLastError();
 }
 
-cudaError_t launch_gemm_simt(int dtype, const void* a, const void* w, bool w_transposed, void* y, int64_t m, int64_t n, int64_t k,
-                             bool swiglu, const EpiProgram& p, cudaStream_t s) {
-  return dtype == DT_F32 ? gemm_simt_dispatch<float>(a, w, w_transposed, y, m, n, k, swiglu, p, s)
-                         : gemm_simt_dispatch<__nv_bfloat16>(a, w, w_transposed, y, m, n, k, swiglu, p, s);
+cudaError_t launch_gemm_simt(int dtype, int out_dtype, const void* a, const void* w, bool w_transposed, void* y, int64_t m, int64_t n,
+                             int64_t k, bool swiglu, const EpiProgram& p, cudaStream_t s) {
+  if (dtype == DT_F32) return out_dtype == DT_F32 ? gemm_simt_dispatch<float, float>(a, w, w_transposed, y, m, n, k, swiglu, p, s) : cudaErrorInvalidValue;
+  return out_dtype == DT_F32 ? gemm_simt_dispatch<__nv_bfloat16, float>(a, w, w_transposed, y, m, n, k, swiglu, p, s)
+                             : gemm_simt_dispatch<__nv_bfloat16, __nv_bfloat16>(a, w, w_transposed, y, m, n, k, swiglu, p, s);
 }
 
 // =====================================================================================================

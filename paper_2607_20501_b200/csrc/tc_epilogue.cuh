@@ -5,12 +5,16 @@
 //   * no dependent global load inside a chunk: the tile's bias slice is copied to shared memory when
 //     the warp starts the tile (before it waits for the accumulator), and a residual chunk is
 //     fetched into registers one chunk ahead (a global load under TMA traffic costs ~1 us of
-//     latency, and with one warp per scheduler nothing else would hide it);
-//   * coalesced global access: a lane's own 64 bytes sit 2*N bytes from its neighbour's, so stores
-//     (and residual loads) go through a shared-memory transpose and each instruction moves
-//     8 rows x 64 contiguous bytes instead of 32 half-filled sectors;
-//   * hardware-approximate tanh / exp2 (the output is bf16, whose half-ulp of 2^-9 dwarfs their 2^-11
-//     relative error).
+//     latency, and with one or two warps per scheduler nothing else would hide it);
+//   * coalesced global access: a lane's own bytes sit a whole output row from its neighbour's, so
+//     stores (and residual loads) go through a shared-memory transpose, one 32-row x 64-byte slab at
+//     a time, and each instruction moves 8 rows x 64 contiguous bytes instead of 32 half-filled
+//     sectors;
+//   * hardware-approximate tanh / exp2 (relative error ~2^-11, below bf16's half-ulp of 2^-9).
+// The residual operand and the output may each be bf16 or fp32 (an fp32 residual stream next to
+// bf16 activations): an fp32 chunk is two slabs.
+// Everything indexes the accumulator array with compile-time constants: one run-time index would
+// move the whole array, for its whole lifetime, from registers to local memory.
 #pragma once
 
 #include "device_common.cuh"
@@ -29,10 +33,11 @@ __device__ __forceinline__ float gelu_fast(float x) {
 }
 __device__ __forceinline__ float silu_fast(float x) { return __fdividef(x, 1.0f + tc::ex2_fast(-1.4426950408889634f * x)); }
 
-// Elementwise program on 32 consecutive columns of one row.  bias32 / res_row: the 64 bytes of bias /
-// residual for these columns in shared memory (null: read them from global memory).
+// Elementwise program on 32 consecutive columns of one row.  bias32: the 64 bytes of bias for these
+// columns in shared memory (null: read them from global memory).  resf: the residual values, already
+// in registers, when have_res; otherwise a residual op reads global memory.
 __device__ __forceinline__ void epi32(const EpiProgram& p, float (&v)[32], int64_t row, int64_t col0, int64_t ld, const uint8_t* bias32,
-                                      const uint8_t* res_row) {
+                                      bool have_res, const float (&resf)[32]) {
 #pragma unroll 1
   for (int i = 0; i < p.n; ++i) {
     const EpiOp& o = p.op[i];
@@ -49,14 +54,27 @@ __device__ __forceinline__ void epi32(const EpiProgram& p, float (&v)[32], int64
         break;
       }
       case EPI_RESIDUAL: {
-        const __nv_bfloat16* r = res_row ? reinterpret_cast<const __nv_bfloat16*>(res_row)
-                                         : reinterpret_cast<const __nv_bfloat16*>(o.ptr) + row * ld + col0;
+        if (have_res) {
 #pragma unroll
-        for (int j = 0; j < 32; j += 8) {
-          float t[8];
-          ld_vec(r + j, t);
+          for (int j = 0; j < 32; ++j) v[j] += resf[j];
+        } else if (o.ptr_dtype == DT_F32) {
+          const float* r = reinterpret_cast<const float*>(o.ptr) + row * ld + col0;
 #pragma unroll
-          for (int q = 0; q < 8; ++q) v[j + q] += t[q];
+          for (int j = 0; j < 32; j += 4) {
+            float t[4];
+            ld_vec(r + j, t);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) v[j + q] += t[q];
+          }
+        } else {
+          const __nv_bfloat16* r = reinterpret_cast<const __nv_bfloat16*>(o.ptr) + row * ld + col0;
+#pragma unroll
+          for (int j = 0; j < 32; j += 8) {
+            float t[8];
+            ld_vec(r + j, t);
+#pragma unroll
+            for (int q = 0; q < 8; ++q) v[j + q] += t[q];
+          }
         }
         break;
       }
@@ -98,12 +116,15 @@ struct EpiWarp {
   uint8_t* stage;  // EPI_WARP_STAGE bytes, this warp's transpose buffer
   uint8_t* bias;   // EPI_WARP_BIAS bytes, this warp's copy of the tile's bias slice
   int bias_idx, res_idx;
+  bool res_f32, out_f32;
   int lane;
-  __device__ __forceinline__ void init(uint8_t* warp_smem, const EpiProgram& p, int lane_) {
+  __device__ __forceinline__ void init(uint8_t* warp_smem, const EpiProgram& p, int lane_, bool out_f32_) {
     stage = warp_smem;
     bias = warp_smem + EPI_WARP_STAGE;
     bias_idx = epi_single_index(p, EPI_BIAS);
     res_idx = epi_single_index(p, EPI_RESIDUAL);
+    res_f32 = res_idx >= 0 && p.op[res_idx].ptr_dtype == DT_F32;
+    out_f32 = out_f32_;
     lane = lane_;
   }
   // Copy bias[col_base, col_base + width) (width <= 256) into shared memory; call before waiting for
@@ -117,66 +138,123 @@ struct EpiWarp {
     __syncwarp();
   }
   // Fetch the residual chunk [32 rows x 32 columns at col0] into registers, coalesced (8 rows x 64 B
-  // per instruction).  A chunk that is ragged in N is left to the element-wise path.
+  // per instruction; an fp32 chunk is two 64-byte slabs per row).  A chunk that is ragged in N is left
+  // to the element-wise path.
   template <typename RowMap>
-  __device__ __forceinline__ void prefetch_res(const EpiProgram& p, RowMap rowmap, int64_t col0, int64_t n_cols, uint4 (&regs)[4]) {
+  __device__ __forceinline__ void prefetch_res(const EpiProgram& p, RowMap rowmap, int64_t col0, int64_t n_cols, uint4 (&regs)[8]) {
     if (res_idx < 0 || col0 + 32 > n_cols) return;
-    const __nv_bfloat16* res = reinterpret_cast<const __nv_bfloat16*>(p.op[res_idx].ptr);
+    const uint8_t* res = reinterpret_cast<const uint8_t*>(p.op[res_idx].ptr);
     const int sub_row = lane >> 2, seg = lane & 3;
+    const int esz = res_f32 ? 4 : 2;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const int64_t gr = rowmap(sub_row + 8 * i);
-      regs[i] = gr >= 0 ? *reinterpret_cast<const uint4*>(res + gr * n_cols + col0 + seg * 8) : make_uint4(0, 0, 0, 0);
+      const uint8_t* src = res + (gr * n_cols + col0) * esz + seg * 16;
+      regs[i] = gr >= 0 ? *reinterpret_cast<const uint4*>(src) : make_uint4(0, 0, 0, 0);
+      if (res_f32) regs[4 + i] = gr >= 0 ? *reinterpret_cast<const uint4*>(src + 64) : make_uint4(0, 0, 0, 0);
     }
   }
-  // One chunk: program, bf16 pack, transposed coalesced store.
+  // registers (transposed role) -> staging -> this lane's own 64 bytes
+  __device__ __forceinline__ void slab_to_own_row(const uint4& r0, const uint4& r1, const uint4& r2, const uint4& r3, uint4 (&mine)[4]) {
+    const int sub_row = lane >> 2, seg = lane & 3;
+    *reinterpret_cast<uint4*>(stage + (sub_row + 0) * EPI_ROW_PITCH + seg * 16) = r0;
+    *reinterpret_cast<uint4*>(stage + (sub_row + 8) * EPI_ROW_PITCH + seg * 16) = r1;
+    *reinterpret_cast<uint4*>(stage + (sub_row + 16) * EPI_ROW_PITCH + seg * 16) = r2;
+    *reinterpret_cast<uint4*>(stage + (sub_row + 24) * EPI_ROW_PITCH + seg * 16) = r3;
+    __syncwarp();
+#pragma unroll
+    for (int i = 0; i < 4; ++i) mine[i] = *reinterpret_cast<const uint4*>(stage + lane * EPI_ROW_PITCH + i * 16);
+    __syncwarp();
+  }
+  // this lane's own 64 bytes -> staging -> coalesced global store at byte offset `byte_off` of each row
+  template <typename RowMap>
+  __device__ __forceinline__ void own_row_to_global(const uint4 (&mine)[4], RowMap rowmap, uint8_t* out, int64_t row_bytes, int64_t byte_off) {
+    const int sub_row = lane >> 2, seg = lane & 3;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) *reinterpret_cast<uint4*>(stage + lane * EPI_ROW_PITCH + i * 16) = mine[i];
+    __syncwarp();
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int r = sub_row + 8 * i;
+      const int64_t gr = rowmap(r);
+      if (gr >= 0) *reinterpret_cast<uint4*>(out + gr * row_bytes + byte_off + seg * 16) = *reinterpret_cast<const uint4*>(stage + r * EPI_ROW_PITCH + seg * 16);
+    }
+    __syncwarp();
+  }
+  // One chunk: program, pack, transposed coalesced store.
   //   v            the lane's fp32 values for columns [col0, col0 + 32) of its row
-  //   bias_off     offset of col0 inside the bias slice loaded by load_bias
+  //   bias_off     offset (elements) of col0 inside the bias slice loaded by load_bias
   //   rowmap(r)    global row of warp-local row r in [0, 32), or -1 if that row is not stored
   //   res_regs     this chunk's residual (from prefetch_res); on return the next chunk's, if next_col0 >= 0
   template <typename RowMap>
-  __device__ __forceinline__ void chunk_out(const EpiProgram& epi, float (&v)[32], RowMap rowmap, __nv_bfloat16* __restrict__ out,
-                                            int64_t col0, int bias_off, int64_t n_cols, uint4 (&res_regs)[4], int64_t next_col0) {
+  __device__ __forceinline__ void chunk_out(const EpiProgram& epi, float (&v)[32], RowMap rowmap, void* __restrict__ out_v, int64_t col0,
+                                            int bias_off, int64_t n_cols, uint4 (&res_regs)[8], int64_t next_col0) {
     if (col0 >= n_cols) return;  // warp-uniform
     const int64_t my_row = rowmap(lane);
-    const int sub_row = lane >> 2, seg = lane & 3;  // transposed role: 8 rows x 4 segments of 16 B per pass
+    uint8_t* out = reinterpret_cast<uint8_t*>(out_v);
     if (col0 + 32 <= n_cols) {
-      const uint8_t* res_row = nullptr;
-      if (res_idx >= 0) {
+      float resf[32];
+      const bool have_res = res_idx >= 0;
+      if (have_res) {
+        uint4 mine[4];
+        slab_to_own_row(res_regs[0], res_regs[1], res_regs[2], res_regs[3], mine);
+        if (res_f32) {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) *reinterpret_cast<uint4*>(stage + (sub_row + 8 * i) * EPI_ROW_PITCH + seg * 16) = res_regs[i];
-        __syncwarp();
-        res_row = stage + lane * EPI_ROW_PITCH;  // only this lane reads, then overwrites, its own row
+          for (int i = 0; i < 4; ++i) {
+            resf[4 * i] = __uint_as_float(mine[i].x); resf[4 * i + 1] = __uint_as_float(mine[i].y);
+            resf[4 * i + 2] = __uint_as_float(mine[i].z); resf[4 * i + 3] = __uint_as_float(mine[i].w);
+          }
+          slab_to_own_row(res_regs[4], res_regs[5], res_regs[6], res_regs[7], mine);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            resf[16 + 4 * i] = __uint_as_float(mine[i].x); resf[16 + 4 * i + 1] = __uint_as_float(mine[i].y);
+            resf[16 + 4 * i + 2] = __uint_as_float(mine[i].z); resf[16 + 4 * i + 3] = __uint_as_float(mine[i].w);
+          }
+        } else {
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const uint32_t w[4] = {mine[i].x, mine[i].y, mine[i].z, mine[i].w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              resf[8 * i + 2 * k] = __uint_as_float(w[k] << 16);
+              resf[8 * i + 2 * k + 1] = __uint_as_float(w[k] & 0xffff0000u);
+            }
+          }
+        }
         if (next_col0 >= 0) prefetch_res(epi, rowmap, next_col0, n_cols, res_regs);
       }
-      if (my_row >= 0) epi32(epi, v, my_row, col0, n_cols, bias_idx >= 0 ? bias + bias_off * 2 : nullptr, res_row);
-      uint4* dst = reinterpret_cast<uint4*>(stage + lane * EPI_ROW_PITCH);
+      if (my_row >= 0) epi32(epi, v, my_row, col0, n_cols, bias_idx >= 0 ? bias + bias_off * 2 : nullptr, have_res, resf);
+      uint4 mine[4];
+      if (!out_f32) {
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        uint4 pk;
-        pk.x = pack_bf16x2(v[8 * j + 0], v[8 * j + 1]);
-        pk.y = pack_bf16x2(v[8 * j + 2], v[8 * j + 3]);
-        pk.z = pack_bf16x2(v[8 * j + 4], v[8 * j + 5]);
-        pk.w = pack_bf16x2(v[8 * j + 6], v[8 * j + 7]);
-        dst[j] = pk;
-      }
-      __syncwarp();
+        for (int j = 0; j < 4; ++j) {
+          mine[j].x = pack_bf16x2(v[8 * j + 0], v[8 * j + 1]);
+          mine[j].y = pack_bf16x2(v[8 * j + 2], v[8 * j + 3]);
+          mine[j].z = pack_bf16x2(v[8 * j + 4], v[8 * j + 5]);
+          mine[j].w = pack_bf16x2(v[8 * j + 6], v[8 * j + 7]);
+        }
+        own_row_to_global(mine, rowmap, out, n_cols * 2, col0 * 2);
+      } else {
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const int r = sub_row + 8 * i;
-        const int64_t gr = rowmap(r);
-        if (gr >= 0)
-          *reinterpret_cast<uint4*>(out + gr * n_cols + col0 + seg * 8) = *reinterpret_cast<const uint4*>(stage + r * EPI_ROW_PITCH + seg * 16);
+        for (int j = 0; j < 4; ++j)
+          mine[j] = make_uint4(__float_as_uint(v[4 * j]), __float_as_uint(v[4 * j + 1]), __float_as_uint(v[4 * j + 2]), __float_as_uint(v[4 * j + 3]));
+        own_row_to_global(mine, rowmap, out, n_cols * 4, col0 * 4);
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          mine[j] = make_uint4(__float_as_uint(v[16 + 4 * j]), __float_as_uint(v[16 + 4 * j + 1]), __float_as_uint(v[16 + 4 * j + 2]),
+                               __float_as_uint(v[16 + 4 * j + 3]));
+        own_row_to_global(mine, rowmap, out, n_cols * 4, col0 * 4 + 64);
       }
-      __syncwarp();
     } else {
       // ragged last chunk of the row: element by element, operands from global memory
-      // (fully unrolled with a predicate: a run-time index into v[] would push the whole array, for its
-      // whole lifetime, out of registers into local memory)
       if (my_row >= 0) {
 #pragma unroll
         for (int j = 0; j < 32; ++j)
-          if (col0 + j < n_cols) out[my_row * n_cols + col0 + j] = __float2bfloat16_rn(epi_apply(epi, v[j], my_row, col0 + j, n_cols));
+          if (col0 + j < n_cols) {
+            const float r = epi_apply(epi, v[j], my_row, col0 + j, n_cols);
+            if (out_f32) reinterpret_cast<float*>(out)[my_row * n_cols + col0 + j] = r;
+            else reinterpret_cast<__nv_bfloat16*>(out)[my_row * n_cols + col0 + j] = __float2bfloat16_rn(r);
+          }
       }
       if (res_idx >= 0 && next_col0 >= 0) prefetch_res(epi, rowmap, next_col0, n_cols, res_regs);
     }

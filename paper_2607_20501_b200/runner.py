@@ -41,8 +41,8 @@ class DeviceWorkload:
         self.module = B.Module(ctx, w.ops, {k: (w.dtype, t.shape) for k, t in w.inputs.items()},
                                weight_layout)
         self.module.set_params(self.params, w.dtype)
-        _, out_shape, _ = self.module.value_spec(w.ops[-1]["out"])
-        self.out = torch.empty(out_shape, dtype=_TORCH[w.dtype], device=device)
+        out_dt, out_shape, _ = self.module.value_spec(w.ops[-1]["out"])
+        self.out = torch.empty(out_shape, dtype=torch.float32 if out_dt == B.MK_F32 else torch.bfloat16, device=device)
         self.ws = None
         self.ws_bytes = 0
 

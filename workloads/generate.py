@@ -221,7 +221,11 @@ def c4(seed=0, B=16, H=16, S=2048, D=128, dtype="bf16") -> Workload:
 # --------------------------------------------------------------------------
 # C5: bf16 4-layer pre-norm decoder (RMSNorm, causal MHA, SwiGLU FFN)
 # --------------------------------------------------------------------------
-def c5(seed=0, B=8, S=1024, E=2048, H=16, F=8192, L=4, dtype="bf16") -> Workload:
+def c5(seed=0, B=8, S=1024, E=2048, H=16, F=8192, L=4, dtype="bf16", stream="f32") -> Workload:
+    """`stream`: storage type of the residual stream (the running sum x).  fp32 by default: with a
+    bf16 stream the four layers' rounding errors, amplified layer over layer, put a few hundred of
+    the 16.8 M outputs outside rtol/atol 2e-2 even for exact kernels; every other activation and all
+    weights are `dtype`."""
     w = Workload("c5", dtype)
     D = E // H
     w.inputs["x"] = make("x", dtype, _normal(seed, 0, (B * S, E)))
@@ -243,12 +247,12 @@ def c5(seed=0, B=8, S=1024, E=2048, H=16, F=8192, L=4, dtype="bf16") -> Workload
             _op("attention_causal", f"att_{l}", [f"qkv_{l}"], layout="packed_qkv", heads=H,
                 head_dim=D, batch=B, seq=S),
             _op("linear", f"o_{l}", [f"att_{l}"], {"w": f"Wo{l}"}, n=E),
-            _op("residual_add", f"x1_{l}", [f"o_{l}", cur]),
+            _op("residual_add", f"x1_{l}", [f"o_{l}", cur], store=stream),
             _op("rmsnorm", f"n2_{l}", [f"x1_{l}"], {"gamma": "ones"}, eps=1e-6),
             _op("linear", f"gu_{l}", [f"n2_{l}"], {"w": f"Wgu{l}"}, n=2 * F),
             _op("swiglu", f"hid_{l}", [f"gu_{l}"]),
             _op("linear", f"d_{l}", [f"hid_{l}"], {"w": f"Wd{l}"}, n=E),
-            _op("residual_add", f"x2_{l}", [f"d_{l}", f"x1_{l}"]),
+            _op("residual_add", f"x2_{l}", [f"d_{l}", f"x1_{l}"], store=stream),
         ]
         cur = f"x2_{l}"
     w.ops.append(_op("rmsnorm", "y", [cur], {"gamma": "ones"}, eps=1e-6))
