@@ -78,6 +78,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   const int b = bh / H, h = bh - b * H;
   const int T = qt + 1;                               // key tiles 0 .. diagonal
   volatile int* abort_flag = &sh->abort_flag;
+  MK_TR_DECL
+  MK_TR_INIT;
 
   if (threadIdx.x == 0) {
     tc::mbar_init(&sh->q_full, 1);
@@ -174,6 +176,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
           umma_ts_lohi(d, p_tmem + k * 8, v_lo + (uint32_t)(k * ((16 * 128) >> 4)), v_hi, idesc_pv, k > 0 ? 1u : 0u);
         tc::umma_commit(&sh->v_empty[st]);
         tc::umma_commit(&sh->o_full[buf]);
+        if (j < 11) MK_TR(5 + j * 8);                        // P_j V_j issued
       }
     }
     __syncwarp();
@@ -193,6 +196,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       ok = tc::mbar_wait(&sh->s_full[buf], use, abort_flag, status, tc::WAIT_TMEM_FULL);
       ok = __all_sync(0xffffffffu, ok ? 1 : 0) != 0;
       if (!ok) break;
+      if (threadIdx.x == 64 && j < 11) MK_TR(1 + j * 8);   // S_j ready
       tc::tc_fence_after();
       const uint32_t s_addr = tmem_s + buf * 128 + lane_off;
       const bool diag = j == T - 1;
@@ -210,6 +214,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
           mx = fmaxf(mx, s);
         }
       }
+      if (threadIdx.x == 64 && j < 11) MK_TR(2 + j * 8);   // pass 1 done
       const float m_new = fmaxf(m, mx);
       const float alpha = tc::ex2_fast(m - m_new);     // 0 on the first tile (m = -inf)
       // pass 2: probabilities, row sum, P -> TMEM as packed bf16 over consumed S columns
@@ -237,6 +242,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       m = m_new;
       tc::tc_fence_before();
       tc::mbar_arrive(&sh->p_ready[buf]);
+      if (threadIdx.x == 64 && j < 11) MK_TR(3 + j * 8);   // P_j written
       // fold the previous tile's P V into the register accumulator
       if (j >= 1) {
         const int pb = (j - 1) & 1;
@@ -255,6 +261,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         }
         tc::tc_fence_before();
         tc::mbar_arrive(&sh->o_free[pb]);
+        if (threadIdx.x == 64 && j < 11) MK_TR(4 + j * 8);   // O_{j-1} folded in
       }
       alpha_prev = alpha;
     }
@@ -295,6 +302,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     }
   }
 
+  MK_TR_PRINT("attn");
   if (*abort_flag) {
     const long long t0 = clock64();
     while (clock64() - t0 < 4000000LL) {}

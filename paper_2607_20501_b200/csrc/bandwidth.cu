@@ -118,8 +118,11 @@ __global__ void __launch_bounds__(256) rowop_warp_kernel(const TI* __restrict__ 
   const int nvec = n / VE;
   const int64_t wstride = (int64_t)gridDim.x * (blockDim.x >> 5);
   const int64_t row_first = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  RawVec<TI, VE> raw[VPL];   // the NEXT row, in flight while the current one is reduced
-  if (row_first < rows) {
+  // the NEXT row is kept in flight while the current one is reduced, unless that would double an already
+  // large register footprint (fp32 input next to bf16 output: 32 raw bytes per 8 elements)
+  constexpr bool PREFETCH = sizeof(TI) == sizeof(T);
+  RawVec<TI, VE> raw[VPL];
+  if (PREFETCH && row_first < rows) {
 #pragma unroll
     for (int i = 0; i < VPL; ++i)
       if (lane + 32 * i < nvec) raw[i].load(x + row_first * n + (lane + 32 * i) * VE);
@@ -130,6 +133,7 @@ __global__ void __launch_bounds__(256) rowop_warp_kernel(const TI* __restrict__ 
   for (int i = 0; i < VPL; ++i) {
     const int vi = lane + 32 * i;
     if (vi < nvec) {
+      if (!PREFETCH) raw[i].load(x + row * n + vi * VE);
       raw[i].unpack(v[i]);
       epi_apply_vec<T, VE>(pre, v[i], row, (int64_t)vi * VE, n);
     } else {
@@ -137,7 +141,7 @@ __global__ void __launch_bounds__(256) rowop_warp_kernel(const TI* __restrict__ 
       for (int e = 0; e < VE; ++e) v[i][e] = (MODE == ROW_SOFTMAX) ? -INFINITY : 0.0f;
     }
   }
-  if (row + wstride < rows) {
+  if (PREFETCH && row + wstride < rows) {
 #pragma unroll
     for (int i = 0; i < VPL; ++i)
       if (lane + 32 * i < nvec) raw[i].load(x + (row + wstride) * n + (lane + 32 * i) * VE);

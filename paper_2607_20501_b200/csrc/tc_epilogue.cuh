@@ -34,10 +34,11 @@ __device__ __forceinline__ float gelu_fast(float x) {
 __device__ __forceinline__ float silu_fast(float x) { return __fdividef(x, 1.0f + tc::ex2_fast(-1.4426950408889634f * x)); }
 
 // Elementwise program on 32 consecutive columns of one row.  bias32: the 64 bytes of bias for these
-// columns in shared memory (null: read them from global memory).  resf: the residual values, already
-// in registers, when have_res; otherwise a residual op reads global memory.
+// columns in shared memory (null: read them from global memory).  res_mode 1: the row's 32 residual
+// values as bf16 in ra; 2: as fp32 in ra (columns 0..15) and rb (16..31); 0: a residual op reads
+// global memory.
 __device__ __forceinline__ void epi32(const EpiProgram& p, float (&v)[32], int64_t row, int64_t col0, int64_t ld, const uint8_t* bias32,
-                                      bool have_res, const float (&resf)[32]) {
+                                      int res_mode, const uint4 (&ra)[4], const uint4 (&rb)[4]) {
 #pragma unroll 1
   for (int i = 0; i < p.n; ++i) {
     const EpiOp& o = p.op[i];
@@ -54,9 +55,24 @@ __device__ __forceinline__ void epi32(const EpiProgram& p, float (&v)[32], int64
         break;
       }
       case EPI_RESIDUAL: {
-        if (have_res) {
+        if (res_mode == 1) {
 #pragma unroll
-          for (int j = 0; j < 32; ++j) v[j] += resf[j];
+          for (int i = 0; i < 4; ++i) {
+            const uint32_t w[4] = {ra[i].x, ra[i].y, ra[i].z, ra[i].w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              v[8 * i + 2 * k] += __uint_as_float(w[k] << 16);
+              v[8 * i + 2 * k + 1] += __uint_as_float(w[k] & 0xffff0000u);
+            }
+          }
+        } else if (res_mode == 2) {
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            v[4 * i] += __uint_as_float(ra[i].x); v[4 * i + 1] += __uint_as_float(ra[i].y);
+            v[4 * i + 2] += __uint_as_float(ra[i].z); v[4 * i + 3] += __uint_as_float(ra[i].w);
+            v[16 + 4 * i] += __uint_as_float(rb[i].x); v[16 + 4 * i + 1] += __uint_as_float(rb[i].y);
+            v[16 + 4 * i + 2] += __uint_as_float(rb[i].z); v[16 + 4 * i + 3] += __uint_as_float(rb[i].w);
+          }
         } else if (o.ptr_dtype == DT_F32) {
           const float* r = reinterpret_cast<const float*>(o.ptr) + row * ld + col0;
 #pragma unroll
@@ -154,9 +170,12 @@ struct EpiWarp {
       if (res_f32) regs[4 + i] = gr >= 0 ? *reinterpret_cast<const uint4*>(src + 64) : make_uint4(0, 0, 0, 0);
     }
   }
-  // registers (transposed role) -> staging -> this lane's own 64 bytes
-  __device__ __forceinline__ void slab_to_own_row(const uint4& r0, const uint4& r1, const uint4& r2, const uint4& r3, uint4 (&mine)[4]) {
+  // registers (transposed role) -> staging -> this lane's own 64 bytes.  No barrier after the own-row
+  // reads: whatever follows either touches only the lane's own row or starts with its own barrier.
+  __device__ __forceinline__ void slab_to_own_row(const uint4& r0, const uint4& r1, const uint4& r2, const uint4& r3, uint4 (&mine)[4],
+                                                  bool sync_first) {
     const int sub_row = lane >> 2, seg = lane & 3;
+    if (sync_first) __syncwarp();
     *reinterpret_cast<uint4*>(stage + (sub_row + 0) * EPI_ROW_PITCH + seg * 16) = r0;
     *reinterpret_cast<uint4*>(stage + (sub_row + 8) * EPI_ROW_PITCH + seg * 16) = r1;
     *reinterpret_cast<uint4*>(stage + (sub_row + 16) * EPI_ROW_PITCH + seg * 16) = r2;
@@ -164,7 +183,6 @@ struct EpiWarp {
     __syncwarp();
 #pragma unroll
     for (int i = 0; i < 4; ++i) mine[i] = *reinterpret_cast<const uint4*>(stage + lane * EPI_ROW_PITCH + i * 16);
-    __syncwarp();
   }
   // this lane's own 64 bytes -> staging -> coalesced global store at byte offset `byte_off` of each row
   template <typename RowMap>
@@ -193,37 +211,18 @@ struct EpiWarp {
     const int64_t my_row = rowmap(lane);
     uint8_t* out = reinterpret_cast<uint8_t*>(out_v);
     if (col0 + 32 <= n_cols) {
-      float resf[32];
-      const bool have_res = res_idx >= 0;
-      if (have_res) {
-        uint4 mine[4];
-        slab_to_own_row(res_regs[0], res_regs[1], res_regs[2], res_regs[3], mine);
+      uint4 ra[4], rb[4];
+      int res_mode = 0;
+      if (res_idx >= 0) {
+        slab_to_own_row(res_regs[0], res_regs[1], res_regs[2], res_regs[3], ra, false);
+        res_mode = 1;
         if (res_f32) {
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            resf[4 * i] = __uint_as_float(mine[i].x); resf[4 * i + 1] = __uint_as_float(mine[i].y);
-            resf[4 * i + 2] = __uint_as_float(mine[i].z); resf[4 * i + 3] = __uint_as_float(mine[i].w);
-          }
-          slab_to_own_row(res_regs[4], res_regs[5], res_regs[6], res_regs[7], mine);
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            resf[16 + 4 * i] = __uint_as_float(mine[i].x); resf[16 + 4 * i + 1] = __uint_as_float(mine[i].y);
-            resf[16 + 4 * i + 2] = __uint_as_float(mine[i].z); resf[16 + 4 * i + 3] = __uint_as_float(mine[i].w);
-          }
-        } else {
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const uint32_t w[4] = {mine[i].x, mine[i].y, mine[i].z, mine[i].w};
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-              resf[8 * i + 2 * k] = __uint_as_float(w[k] << 16);
-              resf[8 * i + 2 * k + 1] = __uint_as_float(w[k] & 0xffff0000u);
-            }
-          }
+          slab_to_own_row(res_regs[4], res_regs[5], res_regs[6], res_regs[7], rb, true);
+          res_mode = 2;
         }
         if (next_col0 >= 0) prefetch_res(epi, rowmap, next_col0, n_cols, res_regs);
       }
-      if (my_row >= 0) epi32(epi, v, my_row, col0, n_cols, bias_idx >= 0 ? bias + bias_off * 2 : nullptr, have_res, resf);
+      if (my_row >= 0) epi32(epi, v, my_row, col0, n_cols, bias_idx >= 0 ? bias + bias_off * 2 : nullptr, res_mode, ra, rb);
       uint4 mine[4];
       if (!out_f32) {
 #pragma unroll
