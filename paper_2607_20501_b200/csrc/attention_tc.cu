@@ -7,7 +7,7 @@
 //   warp 1      TMEM allocation; one lane issues   S_j = Q K_j^T   (SS form, 128x128x16 x 8)
 //                                           and   O_j = P_j V_j   (TS form: P is read from TMEM,
 //                                                                   V from shared memory, MN-major)
-//   warps 2..5  one query row per thread: two passes over S_j in TMEM (row max; then
+//   warps 2..9  two threads per query row, each owning half of the row's columns: two passes over S_j in TMEM (row max; then
 //               p = exp2(s * scale*log2e - m), row sum), P_j written back into TMEM as packed bf16
 //               OVER the columns of S_j that are already consumed; then O_{j-1} is read from TMEM and
 //               folded into a register accumulator  o = o * alpha + O_{j-1}  (alpha = exp2(m_old - m_new)).
@@ -15,7 +15,8 @@
 // TMEM (512 columns): S/P double buffer (2 x 128) + O_j double buffer (2 x 128), so S_{j+1} is being
 // computed while the softmax of tile j runs, and P_j V_j runs while the softmax of tile j+1 runs.
 // The diagonal tile is masked (key > query -> -inf, diagonal kept); tiles left of it need no mask;
-// tiles right of it are never visited.  Heavy query tiles (many key tiles) are launched first.
+// tiles right of it are never visited.  CTAs are ordered head by head (L2 reuse of K/V), heavy query
+// tiles first within a head.
 // Output rows go through the shared-memory transpose of the common epilogue (coalesced stores) to the
 // [B*S, H*D] matrix.  Every mbarrier wait is bounded.
 #include "device_common.cuh"
@@ -31,8 +32,9 @@ constexpr int BQ = 128, BKV = 128, HD = 128;
 constexpr int TILE_BYTES = 128 * HD * 2;   // 32 KB: two 128 x 64 sub-tiles of 16 KB
 constexpr int SUB_BYTES = TILE_BYTES / 2;
 constexpr int KV_STAGES = 2;
-constexpr int THREADS = 192;
-constexpr size_t ATTN_SMEM = (size_t)TILE_BYTES * (1 + 2 * KV_STAGES) + 4 * EPI_WARP_BYTES + 1024 + 256;
+constexpr int SOFTMAX_WARPS = 8;
+constexpr int THREADS = 64 + 32 * SOFTMAX_WARPS;
+constexpr size_t ATTN_SMEM = (size_t)TILE_BYTES * (1 + 2 * KV_STAGES) + SOFTMAX_WARPS * EPI_WARP_BYTES + 1024 + 256 + 2048;
 
 struct Shared {
   uint64_t q_full;
@@ -41,6 +43,7 @@ struct Shared {
   uint64_t s_full[2], p_ready[2], o_full[2], o_free[2];
   uint32_t tmem_base;
   int abort_flag;
+  float xch[2][128][2];   // row maximum / row sum exchange between the two threads of a row
 };
 
 // D[tmem] (+)= A[tmem] * B[smem], descriptor given as low word + constant high word
@@ -70,11 +73,14 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   uint8_t* k_tiles = base + TILE_BYTES;
   uint8_t* v_tiles = k_tiles + KV_STAGES * TILE_BYTES;
   uint8_t* staging = v_tiles + KV_STAGES * TILE_BYTES;
-  Shared* sh = reinterpret_cast<Shared*>(staging + 4 * EPI_WARP_BYTES);
+  Shared* sh = reinterpret_cast<Shared*>(staging + SOFTMAX_WARPS * EPI_WARP_BYTES);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int num_q = (S + BQ - 1) / BQ;
-  const int bh = blockIdx.x % (B * H);
-  const int qt = num_q - 1 - blockIdx.x / (B * H);   // heavy tiles first
+  // consecutive CTAs = the query tiles of ONE (batch, head), heaviest first: the CTAs resident at any
+  // time then share a handful of K/V tensors, which stay in L2, instead of each streaming its own
+  // head's K/V from HBM
+  const int bh = blockIdx.x / num_q;
+  const int qt = num_q - 1 - blockIdx.x % num_q;
   const int b = bh / H, h = bh - b * H;
   const int T = qt + 1;                               // key tiles 0 .. diagonal
   volatile int* abort_flag = &sh->abort_flag;
@@ -88,8 +94,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       tc::mbar_init(&sh->v_full[s], 1); tc::mbar_init(&sh->v_empty[s], 1);
     }
     for (int i = 0; i < 2; ++i) {
-      tc::mbar_init(&sh->s_full[i], 1); tc::mbar_init(&sh->p_ready[i], 128);
-      tc::mbar_init(&sh->o_full[i], 1); tc::mbar_init(&sh->o_free[i], 128);
+      tc::mbar_init(&sh->s_full[i], 1); tc::mbar_init(&sh->p_ready[i], 32 * SOFTMAX_WARPS);
+      tc::mbar_init(&sh->o_full[i], 1); tc::mbar_init(&sh->o_free[i], 32 * SOFTMAX_WARPS);
     }
     sh->abort_flag = 0;
     tc::fence_barrier_init();
@@ -112,21 +118,32 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       tc::tma_load_4d(q_tile, &tmQ, &sh->q_full, 0, qt * BQ, h, b);
       tc::tma_load_4d(q_tile + SUB_BYTES, &tmQ, &sh->q_full, 64, qt * BQ, h, b);
       bool ok = true;
-      for (int j = 0; j < T && ok; ++j) {
+      auto load_k = [&](int j) {
         const int st = j % KV_STAGES;
-        const uint32_t ph = ((j / KV_STAGES) & 1) ^ 1;
-        ok = tc::mbar_wait(&sh->k_empty[st], ph, abort_flag, status, tc::WAIT_SMEM_EMPTY);
-        if (!ok) break;
+        ok = tc::mbar_wait(&sh->k_empty[st], ((j / KV_STAGES) & 1) ^ 1, abort_flag, status, tc::WAIT_SMEM_EMPTY);
+        if (!ok) return;
         uint8_t* kd = k_tiles + (size_t)st * TILE_BYTES;
         tc::mbar_expect_tx(&sh->k_full[st], TILE_BYTES);
         tc::tma_load_4d(kd, &tmK, &sh->k_full[st], 0, j * BKV, h, b);
         tc::tma_load_4d(kd + SUB_BYTES, &tmK, &sh->k_full[st], 64, j * BKV, h, b);
-        ok = tc::mbar_wait(&sh->v_empty[st], ph, abort_flag, status, tc::WAIT_SMEM_EMPTY);
-        if (!ok) break;
+      };
+      auto load_v = [&](int j) {
+        const int st = j % KV_STAGES;
+        ok = tc::mbar_wait(&sh->v_empty[st], ((j / KV_STAGES) & 1) ^ 1, abort_flag, status, tc::WAIT_SMEM_EMPTY);
+        if (!ok) return;
         uint8_t* vd = v_tiles + (size_t)st * TILE_BYTES;
         tc::mbar_expect_tx(&sh->v_full[st], TILE_BYTES);
         tc::tma_load_4d(vd, &tmV, &sh->v_full[st], 0, j * BKV, h, b);
         tc::tma_load_4d(vd + SUB_BYTES, &tmV, &sh->v_full[st], 64, j * BKV, h, b);
+      };
+      // Loads are issued in the order their ring slots come free, which is the order the MMAs retire:
+      // QK(0) QK(1) PV(0) QK(2) PV(1) QK(3) ...  (a K load queued behind a V slot that frees later would
+      // stall the next Q K^T)
+      load_k(0);
+      if (ok && T > 1) load_k(1);
+      for (int j = 0; j < T && ok; ++j) {
+        load_v(j);
+        if (ok && j + 2 < T) load_k(j + 2);
       }
     }
     __syncwarp();
@@ -163,17 +180,22 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         if (!ok) break;
         const int st = j % KV_STAGES, buf = j & 1;
         const uint32_t use = (j >> 1) & 1;
+        if (j < 11) MK_TR(6 + j * 8);                        // QK(j+1) issued, now waiting for P_j
         ok = tc::mbar_wait(&sh->p_ready[buf], use, abort_flag, status, tc::WAIT_ATTN);
+        if (j < 11) MK_TR(7 + j * 8);                        // P_j seen
         if (ok) ok = tc::mbar_wait(&sh->v_full[st], (j / KV_STAGES) & 1, abort_flag, status, tc::WAIT_SMEM_FULL);
+        if (j < 10) MK_TR(8 + j * 8);                        // V_j seen
         if (ok) ok = tc::mbar_wait(&sh->o_free[buf], use ^ 1, abort_flag, status, tc::WAIT_TMEM_EMPTY);
         if (!ok) break;
         tc::tc_fence_after();
         const uint32_t v_lo = v_lo0 + (uint32_t)st * (TILE_BYTES >> 4);
-        const uint32_t p_tmem = tmem_s + buf * 128;      // packed bf16: 16 keys = 8 columns
+        // P_j: packed bf16, 16 keys = 8 columns; keys 0..63 sit in columns [0,32) of the S/P buffer, keys
+        // 64..127 in columns [64,96) (each softmax thread overwrites only S columns it has consumed itself)
+        const uint32_t p_tmem = tmem_s + buf * 128;
         const uint32_t d = tmem_o + buf * 128;
 #pragma unroll
         for (int k = 0; k < BKV / 16; ++k)
-          umma_ts_lohi(d, p_tmem + k * 8, v_lo + (uint32_t)(k * ((16 * 128) >> 4)), v_hi, idesc_pv, k > 0 ? 1u : 0u);
+          umma_ts_lohi(d, p_tmem + (k < 4 ? k * 8 : 64 + (k - 4) * 8), v_lo + (uint32_t)(k * ((16 * 128) >> 4)), v_hi, idesc_pv, k > 0 ? 1u : 0u);
         tc::umma_commit(&sh->v_empty[st]);
         tc::umma_commit(&sh->o_full[buf]);
         if (j < 11) MK_TR(5 + j * 8);                        // P_j V_j issued
@@ -181,13 +203,17 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     }
     __syncwarp();
   } else {
-    // ------------------------------------------------------------ softmax + O accumulation, one row per thread
-    const int q = warp & 3;
+    // ------------------------------------------------------------ softmax + O accumulation
+    // Eight warps: warps w and w + 4 share TMEM lane quarter w % 4, i.e. the same 32 query rows; each
+    // thread owns one row and one half of its columns (64 keys of S_j, 64 head-dim columns of O).  The
+    // two threads of a row meet once per tile to agree on the row maximum (shared memory + a 64-thread
+    // named barrier) and once at the end to add their row sums.
+    const int q = warp & 3, hf = (warp - 2) >> 2;
     const uint32_t lane_off = (uint32_t)(q * 32) << 16;
     const int row_in_tile = q * 32 + lane;
-    float o[HD];
+    float o[64];
 #pragma unroll
-    for (int i = 0; i < HD; ++i) o[i] = 0.0f;
+    for (int i = 0; i < 64; ++i) o[i] = 0.0f;
     float m = -INFINITY, l = 0.0f, alpha_prev = 0.0f;
     bool ok = true;
     for (int j = 0; j < T; ++j) {
@@ -198,47 +224,56 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       if (!ok) break;
       if (threadIdx.x == 64 && j < 11) MK_TR(1 + j * 8);   // S_j ready
       tc::tc_fence_after();
-      const uint32_t s_addr = tmem_s + buf * 128 + lane_off;
+      const uint32_t s_addr = tmem_s + buf * 128 + lane_off + hf * 64;
       const bool diag = j == T - 1;
-      // pass 1: row maximum (in log2 units)
-      float mx = -INFINITY;
-#pragma unroll 1
-      for (int c = 0; c < 4; ++c) {
+      const int col_base = hf * 64;                          // key index (inside the tile) of this thread's first column
+      // pass 1: maximum of the raw scores (four independent chains), then into log2 units
+      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
         uint32_t r[32];
         tc::tmem_ld32(s_addr + c * 32, r);
         tc::tmem_ld_wait();
+        if (!diag) {
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          float s = __uint_as_float(r[i]) * scale_log2;
-          if (diag && c * 32 + i > row_in_tile) s = -INFINITY;
-          mx = fmaxf(mx, s);
+          for (int i = 0; i < 32; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(r[i]));
+        } else {
+#pragma unroll
+          for (int i = 0; i < 32; ++i)
+            if (col_base + c * 32 + i <= row_in_tile) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(r[i]));
         }
       }
+      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * scale_log2;
+      sh->xch[j & 1][row_in_tile][hf] = mx;
+      asm volatile("bar.sync %0, %1;" ::"r"(1 + q), "r"(64) : "memory");
+      const float mx_other = sh->xch[j & 1][row_in_tile][hf ^ 1];
       if (threadIdx.x == 64 && j < 11) MK_TR(2 + j * 8);   // pass 1 done
-      const float m_new = fmaxf(m, mx);
-      const float alpha = tc::ex2_fast(m - m_new);     // 0 on the first tile (m = -inf)
-      // pass 2: probabilities, row sum, P -> TMEM as packed bf16 over consumed S columns
-      float sum = 0.0f;
-#pragma unroll 1
-      for (int c = 0; c < 4; ++c) {
+      const float m_new = fmaxf(m, fmaxf(mx, mx_other));
+      const float alpha = tc::ex2_fast(m - m_new);           // 0 on the first tile (m = -inf)
+      const float neg_m = -m_new;
+      // pass 2: probabilities, row sum, P -> TMEM as packed bf16 over S columns this thread has consumed
+      float sum4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
         uint32_t r[32];
         uint32_t pk[16];
         tc::tmem_ld32(s_addr + c * 32, r);
         tc::tmem_ld_wait();
 #pragma unroll
         for (int i = 0; i < 32; i += 2) {
-          float s0 = __uint_as_float(r[i]) * scale_log2 - m_new;
-          float s1 = __uint_as_float(r[i + 1]) * scale_log2 - m_new;
-          if (diag && c * 32 + i > row_in_tile) s0 = -INFINITY;
-          if (diag && c * 32 + i + 1 > row_in_tile) s1 = -INFINITY;
-          const float p0 = tc::ex2_fast(s0), p1 = tc::ex2_fast(s1);
-          sum += p0 + p1;
+          float p0 = tc::ex2_fast(fmaf(__uint_as_float(r[i]), scale_log2, neg_m));
+          float p1 = tc::ex2_fast(fmaf(__uint_as_float(r[i + 1]), scale_log2, neg_m));
+          if (diag) {
+            if (col_base + c * 32 + i > row_in_tile) p0 = 0.0f;
+            if (col_base + c * 32 + i + 1 > row_in_tile) p1 = 0.0f;
+          }
+          sum4[(i >> 1) & 3] += p0 + p1;
           pk[i >> 1] = pack_bf16x2(p0, p1);
         }
         tmem_st16(s_addr + c * 16, pk);
       }
       tc::tmem_st_wait();
-      l = l * alpha + sum;
+      l = l * alpha + ((sum4[0] + sum4[1]) + (sum4[2] + sum4[3]));
       m = m_new;
       tc::tc_fence_before();
       tc::mbar_arrive(&sh->p_ready[buf]);
@@ -250,14 +285,14 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         ok = __all_sync(0xffffffffu, ok ? 1 : 0) != 0;
         if (!ok) break;
         tc::tc_fence_after();
-        const uint32_t o_addr = tmem_o + pb * 128 + lane_off;
+        const uint32_t o_addr = tmem_o + pb * 128 + lane_off + hf * 64;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
+        for (int c = 0; c < 2; ++c) {
           uint32_t r[32];
           tc::tmem_ld32(o_addr + c * 32, r);
           tc::tmem_ld_wait();
 #pragma unroll
-          for (int i = 0; i < 32; ++i) o[c * 32 + i] = o[c * 32 + i] * alpha_prev + __uint_as_float(r[i]);
+          for (int i = 0; i < 32; ++i) o[c * 32 + i] = fmaf(o[c * 32 + i], alpha_prev, __uint_as_float(r[i]));
         }
         tc::tc_fence_before();
         tc::mbar_arrive(&sh->o_free[pb]);
@@ -272,32 +307,35 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     }
     if (ok) {
       tc::tc_fence_after();
-      const uint32_t o_addr = tmem_o + ((T - 1) & 1) * 128 + lane_off;
-      const float inv_l = 1.0f / l;
+      // the row sum is the sum of the two halves' sums (both are in units of the same final maximum)
+      sh->xch[T & 1][row_in_tile][hf] = l;
+      asm volatile("bar.sync %0, %1;" ::"r"(1 + q), "r"(64) : "memory");
+      const float inv_l = 1.0f / (l + sh->xch[T & 1][row_in_tile][hf ^ 1]);
+      const uint32_t o_addr = tmem_o + ((T - 1) & 1) * 128 + lane_off + hf * 64;
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
+      for (int c = 0; c < 2; ++c) {
         uint32_t r[32];
         tc::tmem_ld32(o_addr + c * 32, r);
         tc::tmem_ld_wait();
 #pragma unroll
-        for (int i = 0; i < 32; ++i) o[c * 32 + i] = (o[c * 32 + i] * alpha_prev + __uint_as_float(r[i])) * inv_l;
+        for (int i = 0; i < 32; ++i) o[c * 32 + i] = fmaf(o[c * 32 + i], alpha_prev, __uint_as_float(r[i])) * inv_l;
       }
-      // store: rows (b*S + query), columns h*D .. h*D + 127 of the [B*S, H*D] matrix
+      // store: rows (b*S + query), this thread's 64 of the columns h*D .. h*D + 127 of the [B*S, H*D] matrix
       EpiProgram none;
       none.n = 0;
       EpiWarp ew;
-      ew.init(staging + q * EPI_WARP_BYTES, none, lane, false);
+      ew.init(staging + (warp - 2) * EPI_WARP_BYTES, none, lane, false);
       const int64_t row0 = (int64_t)b * S + (int64_t)qt * BQ + q * 32;
       const int64_t row_end = (int64_t)b * S + S;
       auto rowmap = [&](int r) -> int64_t { const int64_t g = row0 + r; return g < row_end ? g : -1; };
       uint4 none_regs[8];
       const int64_t n_cols = (int64_t)H * HD;
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
+      for (int c = 0; c < 2; ++c) {
         float v[32];
 #pragma unroll
         for (int i = 0; i < 32; ++i) v[i] = o[c * 32 + i];
-        ew.chunk_out(none, v, rowmap, out, (int64_t)h * HD + c * 32, 0, n_cols, none_regs, -1);
+        ew.chunk_out(none, v, rowmap, out, (int64_t)h * HD + hf * 64 + c * 32, 0, n_cols, none_regs, -1);
       }
     }
   }
