@@ -33,7 +33,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ (null until a capture of that workload exists)
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {"c2": 105.7e6}   # profiles/gemm_tc2_c2.md
 
 DEFAULT_STEPS = {"c1": 2000, "c2": 1000, "c3": 1000, "c4": 200, "c5": 50}
 
