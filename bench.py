@@ -253,15 +253,13 @@ def roofline_of(name, launches_per_step, dominant, achieved, peak, pk, kernel_ms
 def run_ours(args):
     import torch
     import torch.distributed as dist
+    from paper_2607_20501_b200 import dist as D
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, local, world = D.env_world()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback for the product path")
     torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    D.init("nccl", torch.device("cuda", local))
 
     from paper_2607_20501_b200 import Context
     from paper_2607_20501_b200.runner import DeviceWorkload
@@ -282,8 +280,7 @@ def run_ours(args):
     stream = torch.cuda.current_stream()
 
     def barrier():
-        if world > 1:
-            dist.barrier()
+        D.barrier()
         torch.cuda.synchronize()
 
     for i in range(max(args.warmup, 3)):
@@ -369,10 +366,7 @@ def run_ours(args):
         dominant = (dk, agg[dk])
 
     # ---- max over ranks
-    t = torch.tensor([total_ms, kernel_ms, e2e_ms], dtype=torch.float64, device=f"cuda:{local}")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms, kernel_ms, e2e_ms = (float(v) for v in t.tolist())
+    total_ms, kernel_ms, e2e_ms = D.max_over_ranks([total_ms, kernel_ms, e2e_ms], device=f"cuda:{local}")
 
     if rank == 0:
         pk = peaks()
