@@ -1,0 +1,584 @@
+// K7, two-query-tile form: fused causal attention on tcgen05 / TMEM, head_dim 128, bf16 in, fp32 softmax
+// and accumulation.
+//
+//   O = softmax(mask_{j<=i}(Q K^T / sqrt(D))) V        online softmax, the S x S matrix never leaves the SM
+//
+// Persistent CTAs.  A work item is (batch, head, 256 consecutive queries) = two 128-query tiles ("streams"
+// 0 and 1) that share every K/V tile they both need; items are handed out as complementary pairs (the
+// heaviest query block of a head with its lightest), so every CTA gets the same number of key tiles.
+//
+//   warps 0-3    softmax of stream 0: one thread per query row.  S_j (128 fp32 columns of TMEM) -> registers,
+//                row maximum, p = exp2(s * scale*log2e - m), row sum, P_j back into TMEM as packed bf16 over
+//                the columns of S_j.
+//   warps 4-7    the same for stream 1.
+//   warps 8-11   correction and output: when a row maximum has grown by more than 2^8 the softmax thread
+//                publishes the factor and these warps rescale the running O in TMEM before the next P V
+//                is issued (smaller growth is left in place: the reference maximum only has to be the same
+//                in numerator and denominator, and 2^8 more headroom is nothing in fp32 / bf16); at the end of
+//                an item they read O, divide by the row sum and store it.
+//   warp 12      TMA: Q tiles per item, K and V tiles through two-stage rings (128-byte swizzle).
+//   warp 13      TMEM allocation; one lane issues every MMA, the two streams interleaved:
+//                   S_t = Q_t K_j^T (SS form, 128x128x16 x 8),   O_t (+)= P_t V_j (TS form: P from TMEM,
+//                   V from shared memory, MN-major).  While one stream's softmax runs, the tensor pipe
+//                   works for the other.
+// TMEM (512 columns): S/P of stream 0 and 1 (2 x 128), O of stream 0 and 1 (2 x 128); O accumulates in TMEM.
+// The diagonal tile is masked (key > query -> -inf, diagonal kept); tiles right of it are never visited.
+// Every mbarrier wait is bounded.
+#include "device_common.cuh"
+#include "tc_common.cuh"
+#include "tc_epilogue.cuh"
+#include "tc_plans.h"
+
+namespace mk {
+
+namespace {
+
+constexpr int BQ = 128, BKV = 128, HD = 128;
+constexpr int TILE_BYTES = 128 * HD * 2;   // 32 KB: two 128 x 64 sub-tiles of 16 KB
+constexpr int SUB_BYTES = TILE_BYTES / 2;
+constexpr int KV_STAGES = 2;
+constexpr int THREADS = 512;
+constexpr float RESCALE_THRESHOLD = 8.0f;             // log2 units
+
+#ifdef MK_TRACE
+__shared__ unsigned long long mk_tr[96];
+#endif
+#define TR2(cond, slot) do { if (cond) MK_TR(slot); } while (0)
+
+struct Shared {
+  uint64_t q_full[2], q_free[2];
+  uint64_t k_full[KV_STAGES], k_empty[KV_STAGES];
+  uint64_t v_full[KV_STAGES], v_empty[KV_STAGES];
+  uint64_t s_full[2], p_ready[2], alpha_ready[2], o_corr[2], o_final[2], l_ready[2], o_free[2];
+  uint32_t tmem_base;
+  int abort_flag;
+  float alpha[2][128];
+  float l[2][128];
+};
+constexpr size_t ATTN2_SMEM = (size_t)TILE_BYTES * (2 + 2 * KV_STAGES) + 4 * EPI_WARP_BYTES + 1024 + ((sizeof(Shared) + 255) / 256) * 256;
+
+// One work item: two query tiles of one (batch, head).  n0, n1 = number of key tiles stream 0, 1 visits
+// (0: the stream has no queries in this item), nk = key tiles loaded for the item.
+struct Item {
+  int b, h, q0;
+  int n0, n1;
+  int nk;
+};
+
+// Every role walks the same list: super-items blockIdx.x, + gridDim.x, ...; super-item s of a head is the
+// query block P-1-s followed by block s.
+struct ItemIter {
+  int sidx, half, n_super, SP, P, num_q, H;
+  __device__ __forceinline__ void init(int S, int B, int H_) {
+    num_q = (S + BQ - 1) / BQ;
+    P = (num_q + 1) / 2;
+    SP = (P + 1) / 2;
+    H = H_;
+    n_super = B * H * SP;
+    sidx = blockIdx.x;
+    half = 0;
+  }
+  __device__ __forceinline__ bool next(Item& it) {
+    while (sidx < n_super) {
+      const int bh = sidx / SP, s = sidx - bh * SP;
+      const int hi = P - 1 - s;
+      int p;
+      if (half == 0) {
+        p = hi;
+        half = 1;
+      } else {
+        half = 0;
+        sidx += gridDim.x;
+        if (s == hi) continue;
+        p = s;
+      }
+      it.b = bh / H;
+      it.h = bh - it.b * H;
+      it.q0 = p * 2 * BQ;
+      it.n0 = 2 * p + 1;
+      it.n1 = (2 * p + 1 < num_q) ? 2 * p + 2 : 0;
+      it.nk = it.n1 ? it.n1 : it.n0;
+      return true;
+    }
+    return false;
+  }
+};
+
+struct Ctx {
+  Shared* sh;
+  volatile int* abort_flag;
+  unsigned int* status;
+  __device__ __forceinline__ bool wait(uint64_t* bar, uint32_t parity, unsigned code) const {
+    return tc::mbar_wait(bar, parity, abort_flag, status, code);
+  }
+  // the same for a whole warp (its next instruction is warp-collective)
+  __device__ __forceinline__ bool wait_warp(uint64_t* bar, uint32_t parity, unsigned code) const {
+    const bool ok = tc::mbar_wait(bar, parity, abort_flag, status, code);
+    return __all_sync(0xffffffffu, ok ? 1 : 0) != 0;
+  }
+};
+
+// D[tmem] (+)= A[tmem] * B[smem], descriptor given as low word + constant high word
+__device__ __forceinline__ void umma_ts_lohi(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "mov.b64 db, {%2, %3};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}" ::"r"(d_tmem),
+      "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};" ::"r"(taddr),
+      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]),
+      "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+
+// ------------------------------------------------------------------------------------------ TMA producer
+// Order per item: Q0, K0, Q1, V0, K1, V1, ... : the order in which the slots come free (the MMAs retire
+// as QK(j) of both streams, PV(j) of both, QK(j+1) ...), so no load queues behind a slot that frees later.
+__device__ __forceinline__ void role_loader(const Ctx& cx, const CUtensorMap* tmQ, const CUtensorMap* tmK, const CUtensorMap* tmV,
+                                            uint8_t* q_tiles, uint8_t* k_tiles, uint8_t* v_tiles, int B, int H, int S) {
+  Shared* sh = cx.sh;
+  ItemIter iter;
+  iter.init(S, B, H);
+  Item it;
+  uint32_t n_items[2] = {0, 0};
+  uint32_t g = 0;   // key tiles loaded so far by this CTA (ring position)
+  while (iter.next(it)) {
+    auto load_q = [&](int t) -> bool {
+      if (!cx.wait(&sh->q_free[t], (n_items[t] & 1) ^ 1, tc::WAIT_SMEM_EMPTY)) return false;
+      ++n_items[t];
+      uint8_t* qd = q_tiles + (size_t)t * TILE_BYTES;
+      tc::mbar_expect_tx(&sh->q_full[t], TILE_BYTES);
+      tc::tma_load_4d(qd, tmQ, &sh->q_full[t], 0, it.q0 + t * BQ, it.h, it.b);
+      tc::tma_load_4d(qd + SUB_BYTES, tmQ, &sh->q_full[t], 64, it.q0 + t * BQ, it.h, it.b);
+      return true;
+    };
+    auto load_kv = [&](int j, bool is_v) -> bool {
+      const uint32_t gg = g + (uint32_t)j;
+      const int st = gg % KV_STAGES;
+      uint64_t* empty = is_v ? &sh->v_empty[st] : &sh->k_empty[st];
+      uint64_t* full = is_v ? &sh->v_full[st] : &sh->k_full[st];
+      if (!cx.wait(empty, ((gg / KV_STAGES) & 1) ^ 1, tc::WAIT_SMEM_EMPTY)) return false;
+      uint8_t* dst = (is_v ? v_tiles : k_tiles) + (size_t)st * TILE_BYTES;
+      const CUtensorMap* tm = is_v ? tmV : tmK;
+      tc::mbar_expect_tx(full, TILE_BYTES);
+      tc::tma_load_4d(dst, tm, full, 0, j * BKV, it.h, it.b);
+      tc::tma_load_4d(dst + SUB_BYTES, tm, full, 64, j * BKV, it.h, it.b);
+      return true;
+    };
+    if (!load_q(0)) return;
+    if (!load_kv(0, false)) return;
+    if (it.n1 && !load_q(1)) return;
+    if (!load_kv(0, true)) return;
+    for (int j = 1; j < it.nk; ++j) {
+      if (!load_kv(j, false)) return;
+      if (!load_kv(j, true)) return;
+    }
+    g += (uint32_t)it.nk;
+  }
+}
+
+// ------------------------------------------------------------------------------------------ MMA issuer
+// Issue order inside an item with J key tiles (iteration j = 0 .. J-1, stream t = 0, 1):
+//     PV_t(j)  if stream t has a tile j;   then QK_t(j+1) if it has a tile j+1,
+//     else, in the item's last iteration, QK_t(0) of the NEXT item.
+// QK_t(0) of the first item is issued before the loop.  P_t aliases S_t, so QK_t(j+1) must follow PV_t(j);
+// the other stream's MMAs fill the tensor pipe while stream t's softmax runs.
+// The stream index is a run-time value on purpose: one copy of the issue code, so that the roles of a
+// CTA (which all run different code) fit the instruction cache together.  Barrier parities of the two
+// streams are bits t of a mask.
+__device__ __forceinline__ void role_mma(const Ctx& cx, uint32_t tmem_base, uint8_t* q_tiles, uint8_t* k_tiles, uint8_t* v_tiles, int B, int H,
+                                         int S) {
+  Shared* sh = cx.sh;
+  constexpr uint32_t idesc_qk = tc::idesc_bf16_f32(BQ, BKV, 0, 0);   // A, B K-major
+  constexpr uint32_t idesc_pv = tc::idesc_bf16_f32(BQ, HD, 0, 1);    // B (= V) MN-major
+  // V, MN-major with 128-byte swizzle: 64 head-dim elements are contiguous (one 128-byte row per key),
+  // 8-key groups are 1024 B apart (SBO), the second 64 head-dim elements sit SUB_BYTES on (LBO)
+  constexpr uint32_t v_hi = ((1024u >> 4) & 0x3FFF) | (1u << 14) | (2u << 29);
+  const uint32_t q_lo0 = tc::desc_lo_sw128(tc::smem_u32(q_tiles));
+  const uint32_t k_lo0 = tc::desc_lo_sw128(tc::smem_u32(k_tiles));
+  const uint32_t v_lo0 = ((tc::smem_u32(v_tiles) & 0x3FFFF) >> 4) | ((uint32_t)(SUB_BYTES >> 4) << 16);
+  uint32_t par_qfull = 0;     // bit t: parity of the next q_full[t] phase to wait for
+  uint32_t par_ofree = 3;     // bit t: parity to wait for on o_free[t] (starts "already free")
+  uint32_t par_pv = 0, par_corr = 0;
+
+  // S_t = Q_t K^T for key tile j of the item whose tiles start at ring position gbase
+  auto issue_qk = [&](int n0, int n1, int t, int j, uint32_t gbase) -> bool {
+    if (j == 0) {
+      if (!cx.wait(&sh->q_full[t], (par_qfull >> t) & 1, tc::WAIT_SMEM_FULL)) return false;
+      par_qfull ^= 1u << t;
+    }
+    const uint32_t gg = gbase + (uint32_t)j;
+    const int st = gg % KV_STAGES;
+    if (!cx.wait(&sh->k_full[st], (gg / KV_STAGES) & 1, tc::WAIT_SMEM_FULL)) return false;
+    tc::tc_fence_after();
+    const uint32_t q_lo = q_lo0 + (uint32_t)t * (TILE_BYTES >> 4);
+    const uint32_t k_lo = k_lo0 + (uint32_t)st * (TILE_BYTES >> 4);
+    const uint32_t d = tmem_base + (uint32_t)t * 128;
+#pragma unroll
+    for (int k = 0; k < HD / 16; ++k) {
+      const uint32_t off = (uint32_t)((k >> 2) * (SUB_BYTES >> 4) + (k & 3) * 2);
+      tc::umma_ss_lohi(d, q_lo + off, k_lo + off, idesc_qk, k > 0 ? 1u : 0u);
+    }
+    // the slot is released by two arrivals: one per stream, or both from the only stream that reads it
+    tc::umma_commit(&sh->k_empty[st]);
+    if (!(j < n0 && j < n1)) tc::umma_commit(&sh->k_empty[st]);
+    tc::umma_commit(&sh->s_full[t]);
+    if (j == (t ? n1 : n0) - 1) tc::umma_commit(&sh->q_free[t]);
+    return true;
+  };
+  // O_t (+)= P_t V for key tile j
+  auto issue_pv = [&](int n0, int n1, int t, int j, uint32_t gbase) -> bool {
+    if (!cx.wait(&sh->p_ready[t], (par_pv >> t) & 1, tc::WAIT_ATTN)) return false;
+    par_pv ^= 1u << t;
+    if (j >= 1) {
+      if (!cx.wait(&sh->o_corr[t], (par_corr >> t) & 1, tc::WAIT_ATTN)) return false;
+      par_corr ^= 1u << t;
+    } else {
+      // the previous item's O of this stream has been read out
+      if (!cx.wait(&sh->o_free[t], (par_ofree >> t) & 1, tc::WAIT_TMEM_EMPTY)) return false;
+      par_ofree ^= 1u << t;
+    }
+    const uint32_t gg = gbase + (uint32_t)j;
+    const int st = gg % KV_STAGES;
+    if (!cx.wait(&sh->v_full[st], (gg / KV_STAGES) & 1, tc::WAIT_SMEM_FULL)) return false;
+    tc::tc_fence_after();
+    const uint32_t v_lo = v_lo0 + (uint32_t)st * (TILE_BYTES >> 4);
+    const uint32_t p_tmem = tmem_base + (uint32_t)t * 128;          // packed bf16: 16 keys = 8 columns
+    const uint32_t d = tmem_base + 256 + (uint32_t)t * 128;
+    const uint32_t acc0 = j > 0 ? 1u : 0u;
+#pragma unroll
+    for (int k = 0; k < BKV / 16; ++k)
+      umma_ts_lohi(d, p_tmem + k * 8, v_lo + (uint32_t)(k * ((16 * 128) >> 4)), v_hi, idesc_pv, k > 0 ? 1u : acc0);
+    tc::umma_commit(&sh->v_empty[st]);
+    if (!(j < n0 && j < n1)) tc::umma_commit(&sh->v_empty[st]);
+    if (j == (t ? n1 : n0) - 1) tc::umma_commit(&sh->o_final[t]);
+    return true;
+  };
+
+  ItemIter iter;
+  iter.init(S, B, H);
+  Item cur, nxt;
+  bool have = iter.next(cur);
+  uint32_t g = 0;
+  if (have) {
+#pragma unroll 1
+    for (int t = 0; t < 2; ++t)
+      if ((t ? cur.n1 : cur.n0) > 0 && !issue_qk(cur.n0, cur.n1, t, 0, g)) return;
+  }
+  while (have) {
+    const bool have_next = iter.next(nxt);
+    const int J = cur.nk;
+#pragma unroll 1
+    for (int j = 0; j < J; ++j) {
+#pragma unroll 1
+      for (int t = 0; t < 2; ++t) {
+        const int nt = t ? cur.n1 : cur.n0;
+        if (j < nt && !issue_pv(cur.n0, cur.n1, t, j, g)) return;
+        // what this stream computes next: its tile j + 1, or the next item's tile 0
+        int qn0, qn1, qj;
+        uint32_t qg;
+        if (j + 1 < nt) {
+          qn0 = cur.n0; qn1 = cur.n1; qj = j + 1; qg = g;
+        } else if (j == J - 1 && have_next && (t ? nxt.n1 : nxt.n0) > 0) {
+          qn0 = nxt.n0; qn1 = nxt.n1; qj = 0; qg = g + (uint32_t)J;
+        } else {
+          continue;
+        }
+        if (!issue_qk(qn0, qn1, t, qj, qg)) return;
+      }
+    }
+    g += (uint32_t)J;
+    cur = nxt;
+    have = have_next;
+  }
+}
+
+// ------------------------------------------------------------------------------------------ softmax
+// One thread per query row of stream T.  m is the reference maximum in log2 units (scores times
+// scale * log2 e); it follows the running row maximum only when that has grown by more than
+// RESCALE_THRESHOLD, and only then O and l are rescaled.  Two passes over S in TMEM, 32 columns at a
+// time (a TMEM load costs next to nothing; a loop body that fits the instruction cache matters more).
+__device__ __forceinline__ void role_softmax(const Ctx& cx, uint32_t tmem_base, int T, int warp, int lane, int B, int H, int S,
+                                             float scale_log2) {
+  Shared* sh = cx.sh;
+  const int q = warp & 3;
+  const int row = q * 32 + lane;
+  const uint32_t s_addr = tmem_base + (uint32_t)T * 128 + ((uint32_t)(q * 32) << 16);
+  ItemIter iter;
+  iter.init(S, B, H);
+  Item it;
+  uint32_t n_tiles = 0, n_items = 0;
+  while (iter.next(it)) {
+    const int nt = T ? it.n1 : it.n0;
+    if (nt == 0) continue;
+    float m = -INFINITY, l = 0.0f;
+#pragma unroll 1
+    for (int j = 0; j < nt; ++j) {
+      if (!cx.wait_warp(&sh->s_full[T], n_tiles & 1, tc::WAIT_TMEM_FULL)) return;
+      ++n_tiles;
+      tc::tc_fence_after();
+      TR2(T == 0 && threadIdx.x == 0 && n_items == 0 && j < 11, 1 + j * 8);
+      // last visible key of this row inside the tile: the diagonal tile masks key (column) > query (row)
+      const int last = (j == nt - 1) ? row : 127;
+      // pass 1: row maximum of the raw scores
+      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll 1
+      for (int c = 0; c < 4; ++c) {
+        uint32_t r[32];
+        tc::tmem_ld32(s_addr + c * 32, r);
+        tc::tmem_ld_wait();
+        const int lim = last - c * 32;
+        if (lim >= 31) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(r[i]));
+        } else {
+#pragma unroll
+          for (int i = 0; i < 32; ++i)
+            if (i <= lim) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(r[i]));
+        }
+      }
+      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * scale_log2;
+      if (j == 0) {
+        m = mx;
+      } else {
+        float alpha = 1.0f;
+        if (mx > m + RESCALE_THRESHOLD) {
+          alpha = tc::ex2_fast(m - mx);
+          m = mx;
+        }
+        sh->alpha[T][row] = alpha;
+        tc::mbar_arrive(&sh->alpha_ready[T]);
+        l *= alpha;
+      }
+      TR2(T == 0 && threadIdx.x == 0 && n_items == 0 && j < 11, 2 + j * 8);
+      // pass 2: probabilities and row sum; P (packed bf16, 16 columns per 32 keys) goes over columns of
+      // S that this thread has already consumed
+      const float neg_m = -m;
+      float sum4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll 1
+      for (int c = 0; c < 4; ++c) {
+        uint32_t r[32];
+        uint32_t pk[16];
+        tc::tmem_ld32(s_addr + c * 32, r);
+        tc::tmem_ld_wait();
+        const int lim = last - c * 32;
+        if (lim >= 31) {
+#pragma unroll
+          for (int i = 0; i < 32; i += 2) {
+            const float p0 = tc::ex2_fast(fmaf(__uint_as_float(r[i]), scale_log2, neg_m));
+            const float p1 = tc::ex2_fast(fmaf(__uint_as_float(r[i + 1]), scale_log2, neg_m));
+            sum4[(i >> 1) & 3] += p0 + p1;
+            pk[i >> 1] = pack_bf16x2(p0, p1);
+          }
+        } else {
+#pragma unroll
+          for (int i = 0; i < 32; i += 2) {
+            float p0 = tc::ex2_fast(fmaf(__uint_as_float(r[i]), scale_log2, neg_m));
+            float p1 = tc::ex2_fast(fmaf(__uint_as_float(r[i + 1]), scale_log2, neg_m));
+            if (i > lim) p0 = 0.0f;
+            if (i + 1 > lim) p1 = 0.0f;
+            sum4[(i >> 1) & 3] += p0 + p1;
+            pk[i >> 1] = pack_bf16x2(p0, p1);
+          }
+        }
+        tmem_st16(s_addr + c * 16, pk);
+      }
+      tc::tmem_st_wait();
+      tc::tc_fence_before();
+      tc::mbar_arrive(&sh->p_ready[T]);
+      TR2(T == 0 && threadIdx.x == 0 && n_items == 0 && j < 11, 3 + j * 8);
+      l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+    }
+    // the previous item's row sums have been read (a stream whose items are one tile long can otherwise
+    // finish two items before the output warps have finished one)
+    if (!cx.wait_warp(&sh->o_free[T], (n_items & 1) ^ 1, tc::WAIT_TMEM_EMPTY)) return;
+    ++n_items;
+    sh->l[T][row] = l;
+    tc::mbar_arrive(&sh->l_ready[T]);
+  }
+}
+
+// ------------------------------------------------------------------------------------------ correction + output
+__device__ __forceinline__ void role_correction(const Ctx& cx, uint32_t tmem_base, uint8_t* staging, int warp, int lane,
+                                                __nv_bfloat16* __restrict__ out, int B, int H, int S) {
+  Shared* sh = cx.sh;
+  const int q = warp & 3;
+  const int row = q * 32 + lane;
+  const uint32_t lane_off = (uint32_t)(q * 32) << 16;
+  EpiProgram none;
+  none.n = 0;
+  EpiWarp ew;
+  ew.init(staging + q * EPI_WARP_BYTES, none, lane, false);
+  ItemIter iter;
+  iter.init(S, B, H);
+  Item it;
+  uint32_t par_corr = 0, par_item = 0;   // bit t: parity of stream t's next phase
+  const int64_t row_bytes = (int64_t)H * HD * 2;
+  while (iter.next(it)) {
+#pragma unroll 1
+    for (int j = 1; j < it.nk; ++j) {
+#pragma unroll 1
+      for (int t = 0; t < 2; ++t) {
+        if (j >= (t ? it.n1 : it.n0)) continue;
+        if (!cx.wait_warp(&sh->alpha_ready[t], (par_corr >> t) & 1, tc::WAIT_ATTN)) return;
+        par_corr ^= 1u << t;
+        const float a = sh->alpha[t][row];
+        if (__any_sync(0xffffffffu, a != 1.0f)) {
+          tc::tc_fence_after();
+          const uint32_t o_addr = tmem_base + 256 + (uint32_t)t * 128 + lane_off;
+#pragma unroll 1
+          for (int c = 0; c < 4; ++c) {
+            uint32_t r[32];
+            tc::tmem_ld32(o_addr + c * 32, r);
+            tc::tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * a);
+            tc::tmem_st32(o_addr + c * 32, r);
+          }
+          tc::tmem_st_wait();
+        }
+        tc::tc_fence_before();
+        tc::mbar_arrive(&sh->o_corr[t]);
+      }
+    }
+#pragma unroll 1
+    for (int t = 0; t < 2; ++t) {
+      if ((t ? it.n1 : it.n0) == 0) continue;
+      if (!cx.wait_warp(&sh->l_ready[t], (par_item >> t) & 1, tc::WAIT_ATTN)) return;
+      if (!cx.wait_warp(&sh->o_final[t], (par_item >> t) & 1, tc::WAIT_TMEM_FULL)) return;
+      par_item ^= 1u << t;
+      tc::tc_fence_after();
+      const float inv_l = 1.0f / sh->l[t][row];
+      const uint32_t o_addr = tmem_base + 256 + (uint32_t)t * 128 + lane_off;
+      const int q_row0 = it.q0 + t * BQ + q * 32;                       // query index of this warp's first row
+      const int64_t g_row0 = (int64_t)it.b * S + q_row0;
+      auto rowmap = [&](int r) -> int64_t { return q_row0 + r < S ? g_row0 + r : -1; };
+#pragma unroll 1
+      for (int c = 0; c < 4; ++c) {
+        uint32_t r[32];
+        tc::tmem_ld32(o_addr + c * 32, r);
+        tc::tmem_ld_wait();
+        if (c == 3) {
+          // O has left TMEM: the next item's first P V of this stream may overwrite it
+          tc::tc_fence_before();
+          tc::mbar_arrive(&sh->o_free[t]);
+        }
+        uint4 mine[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          mine[k].x = pack_bf16x2(__uint_as_float(r[8 * k + 0]) * inv_l, __uint_as_float(r[8 * k + 1]) * inv_l);
+          mine[k].y = pack_bf16x2(__uint_as_float(r[8 * k + 2]) * inv_l, __uint_as_float(r[8 * k + 3]) * inv_l);
+          mine[k].z = pack_bf16x2(__uint_as_float(r[8 * k + 4]) * inv_l, __uint_as_float(r[8 * k + 5]) * inv_l);
+          mine[k].w = pack_bf16x2(__uint_as_float(r[8 * k + 6]) * inv_l, __uint_as_float(r[8 * k + 7]) * inv_l);
+        }
+        ew.own_row_to_global(mine, rowmap, reinterpret_cast<uint8_t*>(out), row_bytes, ((int64_t)it.h * HD + c * 32) * 2);
+      }
+    }
+  }
+}
+
+__global__ void __launch_bounds__(THREADS, 1)
+attention_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                     __nv_bfloat16* __restrict__ out, int B, int H, int S, float scale_log2, unsigned int* status) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* q_tiles = base;
+  uint8_t* k_tiles = q_tiles + 2 * TILE_BYTES;
+  uint8_t* v_tiles = k_tiles + KV_STAGES * TILE_BYTES;
+  uint8_t* staging = v_tiles + KV_STAGES * TILE_BYTES;
+  Shared* sh = reinterpret_cast<Shared*>(staging + 4 * EPI_WARP_BYTES);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  MK_TR_INIT;
+
+  if (threadIdx.x == 0) {
+    for (int t = 0; t < 2; ++t) {
+      tc::mbar_init(&sh->q_full[t], 1); tc::mbar_init(&sh->q_free[t], 1);
+      tc::mbar_init(&sh->s_full[t], 1); tc::mbar_init(&sh->p_ready[t], 128);
+      tc::mbar_init(&sh->alpha_ready[t], 128); tc::mbar_init(&sh->o_corr[t], 128);
+      tc::mbar_init(&sh->o_final[t], 1); tc::mbar_init(&sh->l_ready[t], 128); tc::mbar_init(&sh->o_free[t], 128);
+    }
+    for (int s = 0; s < KV_STAGES; ++s) {
+      tc::mbar_init(&sh->k_full[s], 1); tc::mbar_init(&sh->k_empty[s], 2);
+      tc::mbar_init(&sh->v_full[s], 1); tc::mbar_init(&sh->v_empty[s], 2);
+    }
+    sh->abort_flag = 0;
+    tc::fence_barrier_init();
+    tc::tma_prefetch_desc(&tmQ);
+    tc::tma_prefetch_desc(&tmK);
+    tc::tma_prefetch_desc(&tmV);
+  }
+  if (warp == 13) { tc::tmem_alloc(&sh->tmem_base, 512); tc::tmem_relinquish(); }
+  tc::tc_fence_before();
+  __syncthreads();
+  tc::tc_fence_after();
+  const uint32_t tmem_base = sh->tmem_base;
+  Ctx cx{sh, &sh->abort_flag, status};
+
+  if (warp < 8) {
+    role_softmax(cx, tmem_base, warp >> 2, warp, lane, B, H, S, scale_log2);
+  } else if (warp < 12) {
+    role_correction(cx, tmem_base, staging, warp, lane, out, B, H, S);
+  } else {
+    if (warp == 12 && lane == 0) role_loader(cx, &tmQ, &tmK, &tmV, q_tiles, k_tiles, v_tiles, B, H, S);
+    if (warp == 13 && lane == 0) role_mma(cx, tmem_base, q_tiles, k_tiles, v_tiles, B, H, S);
+    __syncwarp();
+  }
+
+  MK_TR_PRINT("attn2");
+  if (sh->abort_flag) {
+    // give copies in flight time to land before shared memory and TMEM are handed back
+    const long long t0 = clock64();
+    while (clock64() - t0 < 4000000LL) {}
+  }
+  tc::tc_fence_before();
+  __syncthreads();
+  if (warp == 13) {
+    tc::tc_fence_after();
+    tc::tmem_dealloc(tmem_base, 512);
+  }
+}
+
+}  // namespace
+
+bool attention_tc2_supported(const AttnView& a) {
+  if (a.D != HD || a.B < 1 || a.H < 1 || a.S < 1) return false;
+  if ((a.ss * 2) % 16 || (a.sh * 2) % 16 || (a.sb * 2) % 16) return false;
+  if (a.B * a.H * ((a.S + BQ - 1) / BQ) > INT32_MAX / 4) return false;
+  return true;
+}
+
+cudaError_t attention_tc2_plan(AttnTcPlan* p, const AttnView& a, void* o, int sm_count) {
+  if (!attention_tc2_supported(a)) return cudaErrorInvalidValue;
+  const uint64_t dims[4] = {(uint64_t)a.D, (uint64_t)a.S, (uint64_t)a.H, (uint64_t)a.B};
+  const uint64_t strides[3] = {(uint64_t)a.ss * 2, (uint64_t)a.sh * 2, (uint64_t)a.sb * 2};
+  const uint32_t box[4] = {64, 128, 1, 1};
+  cudaError_t e = encode_tmap_bf16(&p->tm_q, a.q, 4, dims, strides, box, true);
+  if (e == cudaSuccess) e = encode_tmap_bf16(&p->tm_k, a.k, 4, dims, strides, box, true);
+  if (e == cudaSuccess) e = encode_tmap_bf16(&p->tm_v, a.v, 4, dims, strides, box, true);
+  if (e != cudaSuccess) return e;
+  p->out = o;
+  p->B = (int)a.B; p->H = (int)a.H; p->S = (int)a.S;
+  p->scale_log2 = (float)(1.4426950408889634 / sqrt((double)a.D));
+  const int64_t num_q = (a.S + BQ - 1) / BQ, pairs = (num_q + 1) / 2, n_super = a.B * a.H * ((pairs + 1) / 2);
+  p->grid = (int)(n_super < sm_count ? n_super : sm_count);
+  return cudaSuccess;
+}
+
+cudaError_t launch_attention_tc2(const AttnTcPlan& p, cudaStream_t s) {
+  static bool attr_done = false;
+  if (!attr_done) {
+    cudaError_t e = cudaFuncSetAttribute(attention_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ATTN2_SMEM);
+    if (e != cudaSuccess) return e;
+    attr_done = true;
+  }
+  attention_tc2_kernel<<<p.grid, THREADS, ATTN2_SMEM, s>>>(p.tm_q, p.tm_k, p.tm_v, (__nv_bfloat16*)p.out, p.B, p.H, p.S, p.scale_log2,
+                                                           kernel_status_ptr());
+  return cudaGetLastError();
+}
+
+}  // namespace mk

@@ -299,6 +299,20 @@ mk_status attn_tc_emit(const Module& m, int lo, int, const Resolved& r, std::vec
   out.push_back([plan](cudaStream_t s) { return launch_attention_tc(*plan, s); });
   return MK_OK;
 }
+bool attn_tc2_match(const Module& m, int lo, int hi) {
+  if (hi - lo != 1 || m.ops[lo].d.kind != MK_OP_ATTENTION_CAUSAL || m.values[0].spec.dtype != MK_BF16) return false;
+  Resolved none;
+  none.value_ptr.assign(m.values.size(), nullptr);
+  return attention_tc2_supported(attn_view(m, m.ops[lo], none));
+}
+mk_status attn_tc2_emit(const Module& m, int lo, int, const Resolved& r, std::vector<Launch>& out, std::string& err) {
+  const Op& op = m.ops[lo];
+  auto plan = std::make_shared<AttnTcPlan>();
+  cudaError_t e = attention_tc2_plan(plan.get(), attn_view(m, op, r), r.value_ptr[op.out_id], m.ctx->sm_count);
+  if (e != cudaSuccess) { err = std::string("attention_tc2 plan: ") + cudaGetErrorString(e); return MK_ERR_CUDA; }
+  out.push_back([plan](cudaStream_t s) { return launch_attention_tc2(*plan, s); });
+  return MK_OK;
+}
 bool attn_simt_match(const Module& m, int lo, int hi) {
   return hi - lo == 1 && m.ops[lo].d.kind == MK_OP_ATTENTION_CAUSAL && m.ops[lo].d.i[1] <= 256;
 }
@@ -321,6 +335,7 @@ const std::vector<Impl>& registry() {
       {"gemm_simt", gemm_simt_match, no_scratch, gemm_simt_emit},
       {"conv3x3_tc2", conv_tc2_match, no_scratch, conv_tc2_emit},
       {"conv3x3_simt", conv_simt_match, no_scratch, conv_simt_emit},
+      {"attention_tc2", attn_tc2_match, no_scratch, attn_tc2_emit},
       {"attention_tc", attn_tc_match, no_scratch, attn_tc_emit},
       {"attention_simt", attn_simt_match, no_scratch, attn_simt_emit},
       {"rowop", rowop_match, no_scratch, rowop_emit},

@@ -63,4 +63,8 @@ struct AttnTcPlan {
 bool attention_tc_supported(const AttnView& a);
 cudaError_t attention_tc_plan(AttnTcPlan* p, const AttnView& a, void* o);
 cudaError_t launch_attention_tc(const AttnTcPlan& p, cudaStream_t s);
+// Two-query-tile persistent form (256 queries per work item, O accumulated in TMEM); same contract.
+bool attention_tc2_supported(const AttnView& a);
+cudaError_t attention_tc2_plan(AttnTcPlan* p, const AttnView& a, void* o, int sm_count);
+cudaError_t launch_attention_tc2(const AttnTcPlan& p, cudaStream_t s);
 }  // namespace mk

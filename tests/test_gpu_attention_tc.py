@@ -22,15 +22,29 @@ def _attn_only(w):
     return w
 
 
+TC_IMPLS = ("attention_tc2", "attention_tc")
+
+
+@pytest.mark.parametrize("impl", TC_IMPLS)
 @pytest.mark.parametrize("b,h,s", [(1, 1, 128), (1, 2, 256), (2, 3, 384), (1, 2, 200), (1, 1, 1000), (2, 2, 64), (1, 1, 1),
-                                   (1, 4, 2048)])
-def test_attention_matches_the_oracle(ctx, b, h, s):
+                                   (1, 4, 2048), (3, 5, 640)])
+def test_attention_matches_the_oracle(ctx, impl, b, h, s):
     for seed in range(2 if s <= 512 else 1):
         w = _attn_only(W.c4(seed, B=b, H=h, S=s, D=128))
         ref, _ = oracle(w, [0])
-        dw, out = run_gpu(ctx, w, [0], binds={0: "attention_tc"})
-        assert dw.module.bound_impl(0) == "attention_tc"
-        assert_parity(out, ref, "bf16", f"B{b} H{h} S{s} seed{seed}")
+        dw, out = run_gpu(ctx, w, [0], binds={0: impl})
+        assert dw.module.bound_impl(0) == impl
+        assert_parity(out, ref, "bf16", f"{impl} B{b} H{h} S{s} seed{seed}")
+
+
+@pytest.mark.parametrize("b,h,s", [(4, 48, 256), (2, 80, 512), (1, 150, 384)])
+def test_persistent_ctas_walk_several_items(ctx, b, h, s):
+    """More work items than SMs: a CTA of the two-tile kernel then runs several (batch, head, query
+    block) items back to back, with the next item's loads and first MMA issued under the current one."""
+    w = _attn_only(W.c4(3, B=b, H=h, S=s, D=128))
+    ref, _ = oracle(w, [0])
+    dw, out = run_gpu(ctx, w, [0], binds={0: "attention_tc2"})
+    assert_parity(out, ref, "bf16", f"B{b} H{h} S{s}")
 
 
 def test_closed_forms(ctx):
@@ -38,12 +52,13 @@ def test_closed_forms(ctx):
     w = _attn_only(W.c4(0, B=b, H=h, S=s, D=d))
     k = w.inputs["k"].store
     w.inputs["k"] = G.Tensor("k", "bf16", np.broadcast_to(k[:, :, :1], k.shape).copy())   # identical keys
-    dw, out = run_gpu(ctx, w, [0], binds={0: "attention_tc"})
     v = w.inputs["v"].f64()
     pm = np.cumsum(v, axis=2) / np.arange(1, s + 1)[None, None, :, None]     # prefix means of V
-    assert_parity(out, pm.transpose(0, 2, 1, 3).reshape(b * s, h * d), "bf16", "uniform weights")
-    # first query sees only the first key (the diagonal is kept)
-    assert np.array_equal(out[0].reshape(h, d), v[0, :, 0, :])
+    for impl in TC_IMPLS:
+        dw, out = run_gpu(ctx, w, [0], binds={0: impl})
+        assert_parity(out, pm.transpose(0, 2, 1, 3).reshape(b * s, h * d), "bf16", f"{impl} uniform weights")
+        # first query sees only the first key (the diagonal is kept)
+        assert np.array_equal(out[0].reshape(h, d), v[0, :, 0, :])
 
 
 def test_packed_qkv_view_and_swap(ctx):
@@ -51,12 +66,13 @@ def test_packed_qkv_view_and_swap(ctx):
     w.ops = w.ops[:3]            # rmsnorm -> qkv linear -> attention on the packed tensor
     ref, _ = oracle(w, [0])
     outs = {}
-    for impl in ("attention_tc", "attention_simt"):
+    for impl in ("attention_tc2", "attention_tc", "attention_simt"):
         dw, out = run_gpu(ctx, w, [0, 1, 2], binds={2: impl})
         assert dw.module.bound_impl(2) == impl
         assert_parity(out, ref, "bf16", impl)
         outs[impl] = out
     assert np.abs(outs["attention_tc"] - outs["attention_simt"]).max() <= 4e-2
+    assert np.abs(outs["attention_tc2"] - outs["attention_simt"]).max() <= 4e-2
 
 
 def test_c4_block_at_reduced_size(ctx):
@@ -66,3 +82,18 @@ def test_c4_block_at_reduced_size(ctx):
         dw, out = run_gpu(ctx, w, w.partitions[part])
         assert "attention_tc" in dw.module.bound_impl(0)
         assert_parity(out, ref, "bf16", part)
+
+
+@pytest.mark.parametrize("impl", TC_IMPLS)
+def test_row_maximum_growing_from_key_tile_to_key_tile(ctx, impl):
+    """Keys whose magnitude grows by a large factor every 128 positions: the running row maximum jumps
+    by more than 2^8 at most tile boundaries, so the running output and row sum are rescaled each time
+    (the two-tile kernel skips the rescale for smaller jumps; both branches must agree with the oracle)."""
+    b, h, s, d = 1, 2, 640, 128
+    w = _attn_only(W.c4(5, B=b, H=h, S=s, D=d))
+    k = w.inputs["k"].f64()
+    gain = 1.0 + 3.0 * (np.arange(s) // 128)
+    w.inputs["k"] = G.make("k", "bf16", (k * gain[None, None, :, None]).astype(np.float32))
+    ref, _ = oracle(w, [0])
+    dw, out = run_gpu(ctx, w, [0], binds={0: impl})
+    assert_parity(out, ref, "bf16", impl)
