@@ -44,6 +44,7 @@ constexpr float RESCALE_THRESHOLD = 8.0f;             // log2 units
 __shared__ unsigned long long mk_tr[96];
 #endif
 #define TR2(cond, slot) do { if (cond) MK_TR(slot); } while (0)
+#define TRM(jj, k) TR2(gbase == 0 && (jj) >= 2 && (jj) < 7, 1 + ((jj) - 2) * 16 + (k))
 
 struct Shared {
   uint64_t q_full[2], q_free[2];
@@ -128,6 +129,47 @@ __device__ __forceinline__ void umma_ts_lohi(uint32_t d_tmem, uint32_t a_tmem, u
       "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// Eight MMAs (one 128-wide K or key tile) from operands that are already in registers: the issuing
+// thread spends one instruction per MMA once the data it waits for has arrived.
+__device__ __forceinline__ void umma_ss_x8(uint32_t d, const uint64_t (&a)[8], const uint64_t (&b)[8], uint32_t idesc) {
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.b32 p, %1, %1;\n\t"
+      "setp.eq.b32 q, %1, %1;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %2, %10, %1, p;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %3, %11, %1, q;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %4, %12, %1, q;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %5, %13, %1, q;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %6, %14, %1, q;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %7, %15, %1, q;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %8, %16, %1, q;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %9, %17, %1, q;\n\t}" ::"r"(d),
+      "r"(idesc), "l"(a[0]), "l"(a[1]), "l"(a[2]), "l"(a[3]), "l"(a[4]), "l"(a[5]), "l"(a[6]), "l"(a[7]), "l"(b[0]), "l"(b[1]), "l"(b[2]),
+      "l"(b[3]), "l"(b[4]), "l"(b[5]), "l"(b[6]), "l"(b[7])
+      : "memory");
+}
+// D (+)= A[tmem] B[smem]; the first MMA accumulates only if acc0 != 0
+__device__ __forceinline__ void umma_ts_x8(uint32_t d, const uint32_t (&a)[8], const uint64_t (&b)[8], uint32_t idesc, uint32_t acc0) {
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.b32 p, %2, 0;\n\t"
+      "setp.eq.b32 q, %1, %1;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%3], %11, %1, p;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%4], %12, %1, q;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%5], %13, %1, q;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%6], %14, %1, q;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%7], %15, %1, q;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%8], %16, %1, q;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%9], %17, %1, q;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%10], %18, %1, q;\n\t}" ::"r"(d),
+      "r"(idesc), "r"(acc0), "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(a[4]), "r"(a[5]), "r"(a[6]), "r"(a[7]), "l"(b[0]), "l"(b[1]),
+      "l"(b[2]), "l"(b[3]), "l"(b[4]), "l"(b[5]), "l"(b[6]), "l"(b[7])
+      : "memory");
+}
+// keep a value computed before a wait in a register across it
+__device__ __forceinline__ void pin(uint32_t& x) { asm volatile("" : "+r"(x)); }
+__device__ __forceinline__ void pin(uint64_t& x) { asm volatile("" : "+l"(x)); }
+
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};" ::"r"(taddr),
@@ -183,16 +225,16 @@ __device__ __forceinline__ void role_loader(const Ctx& cx, const CUtensorMap* tm
 }
 
 // ------------------------------------------------------------------------------------------ MMA issuer
-// Issue order inside an item with J key tiles (iteration j = 0 .. J-1, stream t = 0, 1):
-//     PV_t(j)  if stream t has a tile j;   then QK_t(j+1) if it has a tile j+1,
-//     else, in the item's last iteration, QK_t(0) of the NEXT item.
-// QK_t(0) of the first item is issued before the loop.  P_t aliases S_t, so QK_t(j+1) must follow PV_t(j);
-// the other stream's MMAs fill the tensor pipe while stream t's softmax runs.
-// The stream index is a run-time value on purpose: one copy of the issue code, so that the roles of a
-// CTA (which all run different code) fit the instruction cache together.  Barrier parities of the two
-// streams are bits t of a mask.
-__device__ __forceinline__ void role_mma(const Ctx& cx, uint32_t tmem_base, uint8_t* q_tiles, uint8_t* k_tiles, uint8_t* v_tiles, int B, int H,
-                                         int S) {
+// One issuing thread per stream (warps 13 and 14).  Stream t's order is S_t(0), O_t(0), S_t(1), O_t(1), ...
+// straight across items: P_t aliases S_t, so QK_t(j+1) has to follow PV_t(j) anyway, and PV_t(j) waits
+// for the stream's softmax; during that wait the other thread keeps the tensor pipe busy.  Two threads
+// because the pipe accepts an MMA only about when it can start it: the issuing thread is blocked for
+// the whole run of its eight MMAs, and its waits, commits and bookkeeping (about as long again) would
+// otherwise leave the pipe idle.  The streams synchronise only through the K/V ring: a slot is
+// released by two commit arrivals, one per stream (both from the same thread for a tile only it reads).
+// The stream index is a run-time value on purpose: one copy of the code for both warps.
+__device__ __forceinline__ void role_mma(const Ctx& cx, uint32_t tmem_base, int t, uint8_t* q_tiles, uint8_t* k_tiles, uint8_t* v_tiles, int B,
+                                         int H, int S) {
   Shared* sh = cx.sh;
   constexpr uint32_t idesc_qk = tc::idesc_bf16_f32(BQ, BKV, 0, 0);   // A, B K-major
   constexpr uint32_t idesc_pv = tc::idesc_bf16_f32(BQ, HD, 0, 1);    // B (= V) MN-major
@@ -202,99 +244,99 @@ __device__ __forceinline__ void role_mma(const Ctx& cx, uint32_t tmem_base, uint
   const uint32_t q_lo0 = tc::desc_lo_sw128(tc::smem_u32(q_tiles));
   const uint32_t k_lo0 = tc::desc_lo_sw128(tc::smem_u32(k_tiles));
   const uint32_t v_lo0 = ((tc::smem_u32(v_tiles) & 0x3FFFF) >> 4) | ((uint32_t)(SUB_BYTES >> 4) << 16);
-  uint32_t par_qfull = 0;     // bit t: parity of the next q_full[t] phase to wait for
-  uint32_t par_ofree = 3;     // bit t: parity to wait for on o_free[t] (starts "already free")
+  uint32_t par_qfull = 0;     // parity of the next q_full[t] phase to wait for
+  uint32_t par_ofree = 1;     // parity to wait for on o_free[t] (starts "already free")
   uint32_t par_pv = 0, par_corr = 0;
 
   // S_t = Q_t K^T for key tile j of the item whose tiles start at ring position gbase
-  auto issue_qk = [&](int n0, int n1, int t, int j, uint32_t gbase) -> bool {
-    if (j == 0) {
-      if (!cx.wait(&sh->q_full[t], (par_qfull >> t) & 1, tc::WAIT_SMEM_FULL)) return false;
-      par_qfull ^= 1u << t;
-    }
+  auto issue_qk = [&](int n0, int n1, int j, uint32_t gbase) -> bool {
     const uint32_t gg = gbase + (uint32_t)j;
     const int st = gg % KV_STAGES;
-    if (!cx.wait(&sh->k_full[st], (gg / KV_STAGES) & 1, tc::WAIT_SMEM_FULL)) return false;
-    tc::tc_fence_after();
     const uint32_t q_lo = q_lo0 + (uint32_t)t * (TILE_BYTES >> 4);
     const uint32_t k_lo = k_lo0 + (uint32_t)st * (TILE_BYTES >> 4);
-    const uint32_t d = tmem_base + (uint32_t)t * 128;
+    uint32_t d = tmem_base + (uint32_t)t * 128;
+    uint64_t a[8], b[8];
 #pragma unroll
     for (int k = 0; k < HD / 16; ++k) {
       const uint32_t off = (uint32_t)((k >> 2) * (SUB_BYTES >> 4) + (k & 3) * 2);
-      tc::umma_ss_lohi(d, q_lo + off, k_lo + off, idesc_qk, k > 0 ? 1u : 0u);
+      a[k] = ((uint64_t)tc::kDescHiSw128 << 32) | (q_lo + off);
+      b[k] = ((uint64_t)tc::kDescHiSw128 << 32) | (k_lo + off);
+      pin(a[k]);
+      pin(b[k]);
     }
+    pin(d);
+    if (j == 0) {
+      if (!cx.wait(&sh->q_full[t], par_qfull, tc::WAIT_SMEM_FULL)) return false;
+      par_qfull ^= 1u;
+    }
+    if (!cx.wait(&sh->k_full[st], (gg / KV_STAGES) & 1, tc::WAIT_SMEM_FULL)) return false;
+    tc::tc_fence_after();
+    TRM(j - 1, t * 8 + 5);
+    umma_ss_x8(d, a, b, idesc_qk);
+    TRM(j - 1, t * 8 + 6);
     // the slot is released by two arrivals: one per stream, or both from the only stream that reads it
+    tc::umma_commit(&sh->s_full[t]);
     tc::umma_commit(&sh->k_empty[st]);
     if (!(j < n0 && j < n1)) tc::umma_commit(&sh->k_empty[st]);
-    tc::umma_commit(&sh->s_full[t]);
     if (j == (t ? n1 : n0) - 1) tc::umma_commit(&sh->q_free[t]);
+    TRM(j - 1, t * 8 + 7);
     return true;
   };
-  // O_t (+)= P_t V for key tile j
-  auto issue_pv = [&](int n0, int n1, int t, int j, uint32_t gbase) -> bool {
-    if (!cx.wait(&sh->p_ready[t], (par_pv >> t) & 1, tc::WAIT_ATTN)) return false;
-    par_pv ^= 1u << t;
-    if (j >= 1) {
-      if (!cx.wait(&sh->o_corr[t], (par_corr >> t) & 1, tc::WAIT_ATTN)) return false;
-      par_corr ^= 1u << t;
-    } else {
-      // the previous item's O of this stream has been read out
-      if (!cx.wait(&sh->o_free[t], (par_ofree >> t) & 1, tc::WAIT_TMEM_EMPTY)) return false;
-      par_ofree ^= 1u << t;
-    }
+  // O_t (+)= P_t V for key tile j.  Everything that is ready early is waited for first; P, which arrives
+  // last, is polled for, and then only the eight MMAs remain.
+  auto issue_pv = [&](int n0, int n1, int j, uint32_t gbase) -> bool {
     const uint32_t gg = gbase + (uint32_t)j;
     const int st = gg % KV_STAGES;
-    if (!cx.wait(&sh->v_full[st], (gg / KV_STAGES) & 1, tc::WAIT_SMEM_FULL)) return false;
-    tc::tc_fence_after();
     const uint32_t v_lo = v_lo0 + (uint32_t)st * (TILE_BYTES >> 4);
     const uint32_t p_tmem = tmem_base + (uint32_t)t * 128;          // packed bf16: 16 keys = 8 columns
-    const uint32_t d = tmem_base + 256 + (uint32_t)t * 128;
-    const uint32_t acc0 = j > 0 ? 1u : 0u;
+    uint32_t d = tmem_base + 256 + (uint32_t)t * 128;
+    uint32_t a[8];
+    uint64_t b[8];
+    TRM(j, t * 8 + 0);
 #pragma unroll
-    for (int k = 0; k < BKV / 16; ++k)
-      umma_ts_lohi(d, p_tmem + k * 8, v_lo + (uint32_t)(k * ((16 * 128) >> 4)), v_hi, idesc_pv, k > 0 ? 1u : acc0);
+    for (int k = 0; k < BKV / 16; ++k) {
+      a[k] = p_tmem + k * 8;
+      b[k] = ((uint64_t)v_hi << 32) | (v_lo + (uint32_t)(k * ((16 * 128) >> 4)));
+      pin(a[k]);
+      pin(b[k]);
+    }
+    pin(d);
+    if (j >= 1) {
+      if (!cx.wait(&sh->o_corr[t], par_corr, tc::WAIT_ATTN)) return false;
+      par_corr ^= 1u;
+    } else {
+      // the previous item's O of this stream has been read out
+      if (!cx.wait(&sh->o_free[t], par_ofree, tc::WAIT_TMEM_EMPTY)) return false;
+      par_ofree ^= 1u;
+    }
+    if (!cx.wait(&sh->v_full[st], (gg / KV_STAGES) & 1, tc::WAIT_SMEM_FULL)) return false;
+    TRM(j, t * 8 + 1);
+    if (!tc::mbar_wait_spin(&sh->p_ready[t], par_pv, cx.abort_flag, cx.status, tc::WAIT_ATTN)) return false;
+    par_pv ^= 1u;
+    TRM(j, t * 8 + 2);
+    tc::tc_fence_after();
+    umma_ts_x8(d, a, b, idesc_pv, j > 0 ? 1u : 0u);
+    TRM(j, t * 8 + 3);
+    if (j == (t ? n1 : n0) - 1) tc::umma_commit(&sh->o_final[t]);
     tc::umma_commit(&sh->v_empty[st]);
     if (!(j < n0 && j < n1)) tc::umma_commit(&sh->v_empty[st]);
-    if (j == (t ? n1 : n0) - 1) tc::umma_commit(&sh->o_final[t]);
+    TRM(j, t * 8 + 4);
     return true;
   };
 
+  // this stream's tiles in order: S(0), O(0), S(1), O(1), ... across items
   ItemIter iter;
   iter.init(S, B, H);
-  Item cur, nxt;
-  bool have = iter.next(cur);
+  Item it;
   uint32_t g = 0;
-  if (have) {
+  while (iter.next(it)) {
+    const int nt = t ? it.n1 : it.n0;
 #pragma unroll 1
-    for (int t = 0; t < 2; ++t)
-      if ((t ? cur.n1 : cur.n0) > 0 && !issue_qk(cur.n0, cur.n1, t, 0, g)) return;
-  }
-  while (have) {
-    const bool have_next = iter.next(nxt);
-    const int J = cur.nk;
-#pragma unroll 1
-    for (int j = 0; j < J; ++j) {
-#pragma unroll 1
-      for (int t = 0; t < 2; ++t) {
-        const int nt = t ? cur.n1 : cur.n0;
-        if (j < nt && !issue_pv(cur.n0, cur.n1, t, j, g)) return;
-        // what this stream computes next: its tile j + 1, or the next item's tile 0
-        int qn0, qn1, qj;
-        uint32_t qg;
-        if (j + 1 < nt) {
-          qn0 = cur.n0; qn1 = cur.n1; qj = j + 1; qg = g;
-        } else if (j == J - 1 && have_next && (t ? nxt.n1 : nxt.n0) > 0) {
-          qn0 = nxt.n0; qn1 = nxt.n1; qj = 0; qg = g + (uint32_t)J;
-        } else {
-          continue;
-        }
-        if (!issue_qk(qn0, qn1, t, qj, qg)) return;
-      }
+    for (int j = 0; j < nt; ++j) {
+      if (!issue_qk(it.n0, it.n1, j, g)) return;
+      if (!issue_pv(it.n0, it.n1, j, g)) return;
     }
-    g += (uint32_t)J;
-    cur = nxt;
-    have = have_next;
+    g += (uint32_t)it.nk;
   }
 }
 
@@ -319,10 +361,12 @@ __device__ __forceinline__ void role_softmax(const Ctx& cx, uint32_t tmem_base, 
     float m = -INFINITY, l = 0.0f;
 #pragma unroll 1
     for (int j = 0; j < nt; ++j) {
-      if (!cx.wait_warp(&sh->s_full[T], n_tiles & 1, tc::WAIT_TMEM_FULL)) return;
+      {
+        const bool ok = tc::mbar_wait_spin(&sh->s_full[T], n_tiles & 1, cx.abort_flag, cx.status, tc::WAIT_TMEM_FULL);
+        if (!__all_sync(0xffffffffu, ok ? 1 : 0)) return;
+      }
       ++n_tiles;
       tc::tc_fence_after();
-      TR2(T == 0 && threadIdx.x == 0 && n_items == 0 && j < 11, 1 + j * 8);
       // last visible key of this row inside the tile: the diagonal tile masks key (column) > query (row)
       const int last = (j == nt - 1) ? row : 127;
       // pass 1: row maximum of the raw scores
@@ -355,7 +399,6 @@ __device__ __forceinline__ void role_softmax(const Ctx& cx, uint32_t tmem_base, 
         tc::mbar_arrive(&sh->alpha_ready[T]);
         l *= alpha;
       }
-      TR2(T == 0 && threadIdx.x == 0 && n_items == 0 && j < 11, 2 + j * 8);
       // pass 2: probabilities and row sum; P (packed bf16, 16 columns per 32 keys) goes over columns of
       // S that this thread has already consumed
       const float neg_m = -m;
@@ -391,7 +434,6 @@ __device__ __forceinline__ void role_softmax(const Ctx& cx, uint32_t tmem_base, 
       tc::tmem_st_wait();
       tc::tc_fence_before();
       tc::mbar_arrive(&sh->p_ready[T]);
-      TR2(T == 0 && threadIdx.x == 0 && n_items == 0 && j < 11, 3 + j * 8);
       l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
     }
     // the previous item's row sums have been read (a stream whose items are one tile long can otherwise
@@ -525,7 +567,7 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     role_correction(cx, tmem_base, staging, warp, lane, out, B, H, S);
   } else {
     if (warp == 12 && lane == 0) role_loader(cx, &tmQ, &tmK, &tmV, q_tiles, k_tiles, v_tiles, B, H, S);
-    if (warp == 13 && lane == 0) role_mma(cx, tmem_base, q_tiles, k_tiles, v_tiles, B, H, S);
+    if ((warp == 13 || warp == 14) && lane == 0) role_mma(cx, tmem_base, warp - 13, q_tiles, k_tiles, v_tiles, B, H, S);
     __syncwarp();
   }
 

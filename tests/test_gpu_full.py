@@ -46,7 +46,7 @@ def test_c4_full_sampled_batch_elements(ctx):
     w = W.c4(0)
     B, H, S, D = w.inputs["q"].shape
     dw, out = run_gpu(ctx, w, w.partitions["fused"])
-    assert dw.module.bound_impl(0) == "attention_tc+gemm_tc2+rowop"
+    assert dw.module.bound_impl(0) == "attention_tc2+gemm_tc2+rowop"
     assert np.isfinite(out).all()
     assert np.abs((out * out).mean(axis=1) - 1).max() < 2e-2          # RMSNorm, gamma = 1, holds at any size
     for b in (0, B - 1):
@@ -64,7 +64,7 @@ def test_c5_full_sampled_batch_elements(ctx):
     B, S = attn["batch"], attn["seq"]
     dw, out = run_gpu(ctx, w, w.partitions["fused_tails"])
     impls = {dw.module.bound_impl(s) for s in range(dw.module.n_sub())}
-    assert impls == {"rowop", "gemm_tc2", "attention_tc"}
+    assert impls == {"rowop", "gemm_tc2", "attention_tc2"}
     assert np.isfinite(out).all()
     assert np.abs((out * out).mean(axis=1) - 1).max() < 2e-2
     ops1 = [dict(o, attrs=dict(o["attrs"])) for o in w.ops]
