@@ -8,14 +8,11 @@
 // heaviest query block of a head with its lightest), so every CTA gets the same number of key tiles.
 //
 //   warps 0-3    softmax of stream 0: one thread per query row.  S_j (128 fp32 columns of TMEM) -> registers,
-//                row maximum, p = exp2(s * scale*log2e - m), row sum, P_j back into TMEM as packed bf16 over
-//                the columns of S_j.
+//                p = exp2(s * scale*log2e - m), row sum, P_j back into TMEM as packed bf16 over the columns
+//                of S_j.  The reference m is raised (and the running O and l rescaled) only on an item's first
+//                and diagonal tiles or when a row sum would leave a safe range: see role_softmax.
 //   warps 4-7    the same for stream 1.
-//   warps 8-11   correction and output: when a row maximum has grown by more than 2^8 the softmax thread
-//                publishes the factor and these warps rescale the running O in TMEM before the next P V
-//                is issued (smaller growth is left in place: the reference maximum only has to be the same
-//                in numerator and denominator, and 2^8 more headroom is nothing in fp32 / bf16); at the end of
-//                an item they read O, divide by the row sum and store it.
+//   warps 8-11   output: at the end of an item they read O from TMEM, divide by the row sum and store it.
 //   warp 12      TMA: Q tiles per item, K and V tiles through two-stage rings (128-byte swizzle).
 //   warp 13      TMEM allocation; one lane issues every MMA, the two streams interleaved:
 //                   S_t = Q_t K_j^T (SS form, 128x128x16 x 8),   O_t (+)= P_t V_j (TS form: P from TMEM,
@@ -38,7 +35,6 @@ constexpr int TILE_BYTES = 128 * HD * 2;   // 32 KB: two 128 x 64 sub-tiles of 1
 constexpr int SUB_BYTES = TILE_BYTES / 2;
 constexpr int KV_STAGES = 2;
 constexpr int THREADS = 512;
-constexpr float RESCALE_THRESHOLD = 8.0f;             // log2 units
 
 #ifdef MK_TRACE
 __shared__ unsigned long long mk_tr[96];
@@ -50,10 +46,10 @@ struct Shared {
   uint64_t q_full[2], q_free[2];
   uint64_t k_full[KV_STAGES], k_empty[KV_STAGES];
   uint64_t v_full[KV_STAGES], v_empty[KV_STAGES];
-  uint64_t s_full[2], p_ready[2], alpha_ready[2], o_corr[2], o_final[2], l_ready[2], o_free[2];
+  uint64_t s_full[2], p_ready[2], o_final[2], l_ready[2], o_free[2];
   uint32_t tmem_base;
   int abort_flag;
-  float alpha[2][128];
+  int pipe_lock;   // held by the stream whose run of MMAs is being issued
   float l[2][128];
 };
 constexpr size_t ATTN2_SMEM = (size_t)TILE_BYTES * (2 + 2 * KV_STAGES) + 4 * EPI_WARP_BYTES + 1024 + ((sizeof(Shared) + 255) / 256) * 256;
@@ -111,6 +107,26 @@ struct Ctx {
   unsigned int* status;
   __device__ __forceinline__ bool wait(uint64_t* bar, uint32_t parity, unsigned code) const {
     return tc::mbar_wait(bar, parity, abort_flag, status, code);
+  }
+  // The two issuing threads take turns: a run of MMAs of one stream is issued whole, so that stream's next
+  // S is ready half a step before the other's and the two softmaxes stay out of phase (one stream's
+  // exponentials overlap the other's MMAs).  Left alone, the runs interleave and both streams end up
+  // doing softmax at the same time and MMAs at the same time.  The holder only issues MMAs, it never waits.
+  __device__ __forceinline__ bool lock_pipe() const {
+    const long long t0 = clock64();
+    while (atomicCAS(&sh->pipe_lock, 0, 1) != 0) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > tc::kWaitLimitCycles) {
+        *abort_flag = 1;
+        if (status) atomicExch(status, (unsigned)tc::WAIT_ATTN);
+        return false;
+      }
+    }
+    return true;
+  }
+  __device__ __forceinline__ void unlock_pipe() const {
+    __threadfence_block();
+    atomicExch(&sh->pipe_lock, 0);
   }
   // the same for a whole warp (its next instruction is warp-collective)
   __device__ __forceinline__ bool wait_warp(uint64_t* bar, uint32_t parity, unsigned code) const {
@@ -225,9 +241,11 @@ __device__ __forceinline__ void role_loader(const Ctx& cx, const CUtensorMap* tm
 }
 
 // ------------------------------------------------------------------------------------------ MMA issuer
-// One issuing thread per stream (warps 13 and 14).  Stream t's order is S_t(0), O_t(0), S_t(1), O_t(1), ...
+// One issuing thread per stream (warps 13 and 14).  Stream t's order is S_t(0), [O_t(0), S_t(1)], [O_t(1), S_t(2)], ...
 // straight across items: P_t aliases S_t, so QK_t(j+1) has to follow PV_t(j) anyway, and PV_t(j) waits
-// for the stream's softmax; during that wait the other thread keeps the tensor pipe busy.  Two threads
+// for the stream's softmax; the pair in brackets is issued as one run of sixteen MMAs, so the path from
+// "P is ready" to "the next S is ready" holds no waits, descriptor arithmetic or bookkeeping.  During the
+// wait for P the other thread keeps the tensor pipe busy.  Two threads
 // because the pipe accepts an MMA only about when it can start it: the issuing thread is blocked for
 // the whole run of its eight MMAs, and its waits, commits and bookkeeping (about as long again) would
 // otherwise leave the pipe idle.  The streams synchronise only through the K/V ring: a slot is
@@ -246,111 +264,141 @@ __device__ __forceinline__ void role_mma(const Ctx& cx, uint32_t tmem_base, int 
   const uint32_t v_lo0 = ((tc::smem_u32(v_tiles) & 0x3FFFF) >> 4) | ((uint32_t)(SUB_BYTES >> 4) << 16);
   uint32_t par_qfull = 0;     // parity of the next q_full[t] phase to wait for
   uint32_t par_ofree = 1;     // parity to wait for on o_free[t] (starts "already free")
-  uint32_t par_pv = 0, par_corr = 0;
+  uint32_t par_pv = 0;
+  const uint32_t q_lo = q_lo0 + (uint32_t)t * (TILE_BYTES >> 4);
+  const uint32_t s_tmem = tmem_base + (uint32_t)t * 128;          // S, and P over it (packed bf16: 16 keys = 8 columns)
+  const uint32_t o_tmem = tmem_base + 256 + (uint32_t)t * 128;
 
-  // S_t = Q_t K^T for key tile j of the item whose tiles start at ring position gbase
-  auto issue_qk = [&](int n0, int n1, int j, uint32_t gbase) -> bool {
-    const uint32_t gg = gbase + (uint32_t)j;
-    const int st = gg % KV_STAGES;
-    const uint32_t q_lo = q_lo0 + (uint32_t)t * (TILE_BYTES >> 4);
-    const uint32_t k_lo = k_lo0 + (uint32_t)st * (TILE_BYTES >> 4);
-    uint32_t d = tmem_base + (uint32_t)t * 128;
-    uint64_t a[8], b[8];
-#pragma unroll
-    for (int k = 0; k < HD / 16; ++k) {
-      const uint32_t off = (uint32_t)((k >> 2) * (SUB_BYTES >> 4) + (k & 3) * 2);
-      a[k] = ((uint64_t)tc::kDescHiSw128 << 32) | (q_lo + off);
-      b[k] = ((uint64_t)tc::kDescHiSw128 << 32) | (k_lo + off);
-      pin(a[k]);
-      pin(b[k]);
-    }
-    pin(d);
-    if (j == 0) {
-      if (!cx.wait(&sh->q_full[t], par_qfull, tc::WAIT_SMEM_FULL)) return false;
-      par_qfull ^= 1u;
-    }
-    if (!cx.wait(&sh->k_full[st], (gg / KV_STAGES) & 1, tc::WAIT_SMEM_FULL)) return false;
-    tc::tc_fence_after();
-    TRM(j - 1, t * 8 + 5);
-    umma_ss_x8(d, a, b, idesc_qk);
-    TRM(j - 1, t * 8 + 6);
-    // the slot is released by two arrivals: one per stream, or both from the only stream that reads it
-    tc::umma_commit(&sh->s_full[t]);
-    tc::umma_commit(&sh->k_empty[st]);
-    if (!(j < n0 && j < n1)) tc::umma_commit(&sh->k_empty[st]);
-    if (j == (t ? n1 : n0) - 1) tc::umma_commit(&sh->q_free[t]);
-    TRM(j - 1, t * 8 + 7);
-    return true;
+  // one key tile of this stream: j-th of nt in an item whose tiles start at ring position g
+  struct Pos {
+    int n0, n1, nt, j;
+    uint32_t g;
+    bool valid;
   };
-  // O_t (+)= P_t V for key tile j.  Everything that is ready early is waited for first; P, which arrives
-  // last, is polled for, and then only the eight MMAs remain.
-  auto issue_pv = [&](int n0, int n1, int j, uint32_t gbase) -> bool {
-    const uint32_t gg = gbase + (uint32_t)j;
-    const int st = gg % KV_STAGES;
-    const uint32_t v_lo = v_lo0 + (uint32_t)st * (TILE_BYTES >> 4);
-    const uint32_t p_tmem = tmem_base + (uint32_t)t * 128;          // packed bf16: 16 keys = 8 columns
-    uint32_t d = tmem_base + 256 + (uint32_t)t * 128;
-    uint32_t a[8];
-    uint64_t b[8];
-    TRM(j, t * 8 + 0);
-#pragma unroll
-    for (int k = 0; k < BKV / 16; ++k) {
-      a[k] = p_tmem + k * 8;
-      b[k] = ((uint64_t)v_hi << 32) | (v_lo + (uint32_t)(k * ((16 * 128) >> 4)));
-      pin(a[k]);
-      pin(b[k]);
-    }
-    pin(d);
-    if (j >= 1) {
-      if (!cx.wait(&sh->o_corr[t], par_corr, tc::WAIT_ATTN)) return false;
-      par_corr ^= 1u;
-    } else {
-      // the previous item's O of this stream has been read out
-      if (!cx.wait(&sh->o_free[t], par_ofree, tc::WAIT_TMEM_EMPTY)) return false;
-      par_ofree ^= 1u;
-    }
-    if (!cx.wait(&sh->v_full[st], (gg / KV_STAGES) & 1, tc::WAIT_SMEM_FULL)) return false;
-    TRM(j, t * 8 + 1);
-    if (!tc::mbar_wait_spin(&sh->p_ready[t], par_pv, cx.abort_flag, cx.status, tc::WAIT_ATTN)) return false;
-    par_pv ^= 1u;
-    TRM(j, t * 8 + 2);
-    tc::tc_fence_after();
-    umma_ts_x8(d, a, b, idesc_pv, j > 0 ? 1u : 0u);
-    TRM(j, t * 8 + 3);
-    if (j == (t ? n1 : n0) - 1) tc::umma_commit(&sh->o_final[t]);
-    tc::umma_commit(&sh->v_empty[st]);
-    if (!(j < n0 && j < n1)) tc::umma_commit(&sh->v_empty[st]);
-    TRM(j, t * 8 + 4);
-    return true;
-  };
-
-  // this stream's tiles in order: S(0), O(0), S(1), O(1), ... across items
   ItemIter iter;
   iter.init(S, B, H);
-  Item it;
-  uint32_t g = 0;
-  while (iter.next(it)) {
-    const int nt = t ? it.n1 : it.n0;
-#pragma unroll 1
-    for (int j = 0; j < nt; ++j) {
-      if (!issue_qk(it.n0, it.n1, j, g)) return;
-      if (!issue_pv(it.n0, it.n1, j, g)) return;
+  uint32_t g_next = 0;
+  auto next_item = [&](Pos& p) {
+    Item it;
+    p.valid = false;
+    while (iter.next(it)) {
+      const int nt = t ? it.n1 : it.n0;
+      const uint32_t g = g_next;
+      g_next += (uint32_t)it.nk;
+      if (nt > 0) {
+        p.n0 = it.n0; p.n1 = it.n1; p.nt = nt; p.j = 0; p.g = g; p.valid = true;
+        return;
+      }
     }
-    g += (uint32_t)it.nk;
+  };
+  // S_t = Q_t K^T for tile b (if do_qk), preceded by O_t (+)= P_t V for tile a (if do_pv).  The two are issued
+  // back to back: everything that is ready early is waited for first, P (which arrives last) is polled
+  // for, and from then on the thread only issues the sixteen MMAs and the commit that publishes S.
+  auto issue = [&](const Pos& a, bool do_pv, const Pos& b, bool do_qk) -> bool {
+    const uint32_t ga = a.g + (uint32_t)a.j, gb = b.g + (uint32_t)b.j;
+    const int sta = ga % KV_STAGES, stb = gb % KV_STAGES;
+    uint32_t pa[8];
+    uint64_t vb[8], qa[8], kb[8];
+    bool fused = false;
+    if (do_pv) {
+      const uint32_t v_lo = v_lo0 + (uint32_t)sta * (TILE_BYTES >> 4);
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        pa[k] = s_tmem + k * 8;
+        vb[k] = ((uint64_t)v_hi << 32) | (v_lo + (uint32_t)(k * ((16 * 128) >> 4)));
+        pin(pa[k]);
+        pin(vb[k]);
+      }
+    }
+    if (do_qk) {
+      const uint32_t k_lo = k_lo0 + (uint32_t)stb * (TILE_BYTES >> 4);
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const uint32_t off = (uint32_t)((k >> 2) * (SUB_BYTES >> 4) + (k & 3) * 2);
+        qa[k] = ((uint64_t)tc::kDescHiSw128 << 32) | (q_lo + off);
+        kb[k] = ((uint64_t)tc::kDescHiSw128 << 32) | (k_lo + off);
+        pin(qa[k]);
+        pin(kb[k]);
+      }
+      // Fuse only if the operands of the next S are already there: waiting for them here, before this
+      // tile's P V is issued, could wait for a load that is queued behind a slot this very P V releases.
+      fused = (b.j != 0 || tc::mbar_test_wait(&sh->q_full[t], par_qfull)) && tc::mbar_test_wait(&sh->k_full[stb], (gb / KV_STAGES) & 1);
+    }
+    if (do_pv) {
+      if (a.j == 0) {
+        // the previous item's O of this stream has been read out
+        if (!cx.wait(&sh->o_free[t], par_ofree, tc::WAIT_TMEM_EMPTY)) return false;
+        par_ofree ^= 1u;
+      }
+      if (!cx.wait(&sh->v_full[sta], (ga / KV_STAGES) & 1, tc::WAIT_SMEM_FULL)) return false;
+      if (!tc::mbar_wait_spin(&sh->p_ready[t], par_pv, cx.abort_flag, cx.status, tc::WAIT_ATTN)) return false;
+      par_pv ^= 1u;
+      TR2(a.g == 0 && a.j < 11, (t ? 8 : 4) + a.j * 8);
+      tc::tc_fence_after();
+      if (!cx.lock_pipe()) return false;
+      umma_ts_x8(o_tmem, pa, vb, idesc_pv, a.j > 0 ? 1u : 0u);
+      if (fused) {
+        umma_ss_x8(s_tmem, qa, kb, idesc_qk);
+        tc::umma_commit(&sh->s_full[t]);
+      }
+      cx.unlock_pipe();
+      // a K/V slot is released by two arrivals: one per stream, or both from the only stream that reads it
+      if (a.j == a.nt - 1) tc::umma_commit(&sh->o_final[t]);
+      tc::umma_commit(&sh->v_empty[sta]);
+      if (!(a.j < a.n0 && a.j < a.n1)) tc::umma_commit(&sh->v_empty[sta]);
+    }
+    if (do_qk) {
+      if (!fused || !do_pv) {
+        if (b.j == 0 && !cx.wait(&sh->q_full[t], par_qfull, tc::WAIT_SMEM_FULL)) return false;
+        if (!cx.wait(&sh->k_full[stb], (gb / KV_STAGES) & 1, tc::WAIT_SMEM_FULL)) return false;
+        tc::tc_fence_after();
+        if (!cx.lock_pipe()) return false;
+        umma_ss_x8(s_tmem, qa, kb, idesc_qk);
+        tc::umma_commit(&sh->s_full[t]);
+        cx.unlock_pipe();
+      }
+      if (b.j == 0) par_qfull ^= 1u;
+      tc::umma_commit(&sh->k_empty[stb]);
+      if (!(b.j < b.n0 && b.j < b.n1)) tc::umma_commit(&sh->k_empty[stb]);
+      if (b.j == b.nt - 1) tc::umma_commit(&sh->q_free[t]);
+    }
+    return true;
+  };
+
+  Pos a, b;
+  next_item(a);
+  if (!a.valid) return;
+  if (!issue(a, false, a, true)) return;
+  while (true) {
+    b = a;
+    if (b.j + 1 < b.nt) ++b.j;
+    else next_item(b);
+    if (!issue(a, true, b, b.valid)) return;
+    if (!b.valid) break;
+    a = b;
   }
 }
 
 // ------------------------------------------------------------------------------------------ softmax
 // One thread per query row of stream T.  m is the reference maximum in log2 units (scores times
-// scale * log2 e); it follows the running row maximum only when that has grown by more than
-// RESCALE_THRESHOLD, and only then O and l are rescaled.  Two passes over S in TMEM, 32 columns at a
-// time (a TMEM load costs next to nothing; a loop body that fits the instruction cache matters more).
+// scale * log2 e): p = exp2(s * scale*log2e - m).  Any m gives the same O / l as long as nothing
+// overflows, so m is NOT kept equal to the running row maximum:
+//   fast path (every tile but an item's first and its diagonal one): a single pass over S with the m
+//     the row already has; all of P stays in registers until the row sum has been checked;
+//   full path (first tile, diagonal tile, or a row sum above 2^60 somewhere in the warp): row maximum,
+//     m raised to it, the running O of this row (in TMEM) and l rescaled by exp2(m_old - m_new) by
+//     this very thread, then the probabilities.  S is still intact when the fast path gives up:
+//     it has stored nothing yet.
+// The previous P V of this stream is complete whenever S_j is visible (the tensor pipe runs in order),
+// so touching O here is safe, and the next P V is not issued before this thread's p_ready arrival.
 __device__ __forceinline__ void role_softmax(const Ctx& cx, uint32_t tmem_base, int T, int warp, int lane, int B, int H, int S,
                                              float scale_log2) {
   Shared* sh = cx.sh;
   const int q = warp & 3;
   const int row = q * 32 + lane;
-  const uint32_t s_addr = tmem_base + (uint32_t)T * 128 + ((uint32_t)(q * 32) << 16);
+  const uint32_t lane_off = (uint32_t)(q * 32) << 16;
+  const uint32_t s_addr = tmem_base + (uint32_t)T * 128 + lane_off;
+  const uint32_t o_addr = tmem_base + 256 + (uint32_t)T * 128 + lane_off;
   ItemIter iter;
   iter.init(S, B, H);
   Item it;
@@ -367,58 +415,80 @@ __device__ __forceinline__ void role_softmax(const Ctx& cx, uint32_t tmem_base, 
       }
       ++n_tiles;
       tc::tc_fence_after();
-      // last visible key of this row inside the tile: the diagonal tile masks key (column) > query (row)
-      const int last = (j == nt - 1) ? row : 127;
-      // pass 1: row maximum of the raw scores
-      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll 1
-      for (int c = 0; c < 4; ++c) {
-        uint32_t r[32];
-        tc::tmem_ld32(s_addr + c * 32, r);
-        tc::tmem_ld_wait();
-        const int lim = last - c * 32;
-        if (lim >= 31) {
+      TR2(T == 0 && threadIdx.x == 0 && n_items == 0 && j < 11, 1 + j * 8);
+      TR2(T == 1 && threadIdx.x == 128 && n_items == 0 && j < 11, 5 + j * 8);
+      bool full = j == 0 || j == nt - 1;
+      if (!full) {
+        const float neg_m = -m;
+        float sum4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+        uint32_t pk[64];
 #pragma unroll
-          for (int i = 0; i < 32; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(r[i]));
-        } else {
-#pragma unroll
-          for (int i = 0; i < 32; ++i)
-            if (i <= lim) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(r[i]));
-        }
-      }
-      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * scale_log2;
-      if (j == 0) {
-        m = mx;
-      } else {
-        float alpha = 1.0f;
-        if (mx > m + RESCALE_THRESHOLD) {
-          alpha = tc::ex2_fast(m - mx);
-          m = mx;
-        }
-        sh->alpha[T][row] = alpha;
-        tc::mbar_arrive(&sh->alpha_ready[T]);
-        l *= alpha;
-      }
-      // pass 2: probabilities and row sum; P (packed bf16, 16 columns per 32 keys) goes over columns of
-      // S that this thread has already consumed
-      const float neg_m = -m;
-      float sum4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-#pragma unroll 1
-      for (int c = 0; c < 4; ++c) {
-        uint32_t r[32];
-        uint32_t pk[16];
-        tc::tmem_ld32(s_addr + c * 32, r);
-        tc::tmem_ld_wait();
-        const int lim = last - c * 32;
-        if (lim >= 31) {
+        for (int c = 0; c < 4; ++c) {
+          uint32_t r[32];
+          tc::tmem_ld32(s_addr + c * 32, r);
+          tc::tmem_ld_wait();
 #pragma unroll
           for (int i = 0; i < 32; i += 2) {
             const float p0 = tc::ex2_fast(fmaf(__uint_as_float(r[i]), scale_log2, neg_m));
             const float p1 = tc::ex2_fast(fmaf(__uint_as_float(r[i + 1]), scale_log2, neg_m));
             sum4[(i >> 1) & 3] += p0 + p1;
-            pk[i >> 1] = pack_bf16x2(p0, p1);
+            pk[c * 16 + (i >> 1)] = pack_bf16x2(p0, p1);
           }
-        } else {
+        }
+        const float sum = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+        full = __any_sync(0xffffffffu, !(sum < 1.152921504606847e18f));   // 2^60; also true for inf / NaN
+        if (!full) {
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            uint32_t part[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) part[i] = pk[c * 16 + i];
+            tmem_st16(s_addr + c * 16, part);
+          }
+          l += sum;
+        }
+      }
+      if (full) {
+        // last visible key of this row inside the tile: the diagonal tile masks key (column) > query (row)
+        const int last = (j == nt - 1) ? row : 127;
+        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+          uint32_t r[32];
+          tc::tmem_ld32(s_addr + c * 32, r);
+          tc::tmem_ld_wait();
+          const int lim = last - c * 32;
+#pragma unroll
+          for (int i = 0; i < 32; ++i)
+            if (i <= lim) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(r[i]));
+        }
+        const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * scale_log2;
+        float alpha = 1.0f;
+        if (mx > m) {
+          alpha = tc::ex2_fast(m - mx);    // 0 on the first tile (m = -inf)
+          m = mx;
+        }
+        if (j > 0 && __any_sync(0xffffffffu, alpha != 1.0f)) {
+#pragma unroll 1
+          for (int c = 0; c < 4; ++c) {
+            uint32_t r[32];
+            tc::tmem_ld32(o_addr + c * 32, r);
+            tc::tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
+            tc::tmem_st32(o_addr + c * 32, r);
+          }
+        }
+        l *= alpha;
+        const float neg_m = -m;
+        float sum4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+          uint32_t r[32];
+          uint32_t pk[16];
+          tc::tmem_ld32(s_addr + c * 32, r);
+          tc::tmem_ld_wait();
+          const int lim = last - c * 32;
 #pragma unroll
           for (int i = 0; i < 32; i += 2) {
             float p0 = tc::ex2_fast(fmaf(__uint_as_float(r[i]), scale_log2, neg_m));
@@ -428,13 +498,15 @@ __device__ __forceinline__ void role_softmax(const Ctx& cx, uint32_t tmem_base, 
             sum4[(i >> 1) & 3] += p0 + p1;
             pk[i >> 1] = pack_bf16x2(p0, p1);
           }
+          tmem_st16(s_addr + c * 16, pk);
         }
-        tmem_st16(s_addr + c * 16, pk);
+        l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
       }
       tc::tmem_st_wait();
       tc::tc_fence_before();
       tc::mbar_arrive(&sh->p_ready[T]);
-      l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+      TR2(T == 0 && threadIdx.x == 0 && n_items == 0 && j < 11, 3 + j * 8);
+      TR2(T == 1 && threadIdx.x == 128 && n_items == 0 && j < 11, 7 + j * 8);
     }
     // the previous item's row sums have been read (a stream whose items are one tile long can otherwise
     // finish two items before the output warps have finished one)
@@ -445,9 +517,10 @@ __device__ __forceinline__ void role_softmax(const Ctx& cx, uint32_t tmem_base, 
   }
 }
 
-// ------------------------------------------------------------------------------------------ correction + output
-__device__ __forceinline__ void role_correction(const Ctx& cx, uint32_t tmem_base, uint8_t* staging, int warp, int lane,
-                                                __nv_bfloat16* __restrict__ out, int B, int H, int S) {
+// ------------------------------------------------------------------------------------------ output
+// At the end of an item: O / l, to bf16, through the shared-memory transpose to the [B*S, H*D] matrix.
+__device__ __forceinline__ void role_output(const Ctx& cx, uint32_t tmem_base, uint8_t* staging, int warp, int lane,
+                                            __nv_bfloat16* __restrict__ out, int B, int H, int S) {
   Shared* sh = cx.sh;
   const int q = warp & 3;
   const int row = q * 32 + lane;
@@ -459,35 +532,9 @@ __device__ __forceinline__ void role_correction(const Ctx& cx, uint32_t tmem_bas
   ItemIter iter;
   iter.init(S, B, H);
   Item it;
-  uint32_t par_corr = 0, par_item = 0;   // bit t: parity of stream t's next phase
+  uint32_t par_item = 0;   // bit t: parity of stream t's next phase
   const int64_t row_bytes = (int64_t)H * HD * 2;
   while (iter.next(it)) {
-#pragma unroll 1
-    for (int j = 1; j < it.nk; ++j) {
-#pragma unroll 1
-      for (int t = 0; t < 2; ++t) {
-        if (j >= (t ? it.n1 : it.n0)) continue;
-        if (!cx.wait_warp(&sh->alpha_ready[t], (par_corr >> t) & 1, tc::WAIT_ATTN)) return;
-        par_corr ^= 1u << t;
-        const float a = sh->alpha[t][row];
-        if (__any_sync(0xffffffffu, a != 1.0f)) {
-          tc::tc_fence_after();
-          const uint32_t o_addr = tmem_base + 256 + (uint32_t)t * 128 + lane_off;
-#pragma unroll 1
-          for (int c = 0; c < 4; ++c) {
-            uint32_t r[32];
-            tc::tmem_ld32(o_addr + c * 32, r);
-            tc::tmem_ld_wait();
-#pragma unroll
-            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * a);
-            tc::tmem_st32(o_addr + c * 32, r);
-          }
-          tc::tmem_st_wait();
-        }
-        tc::tc_fence_before();
-        tc::mbar_arrive(&sh->o_corr[t]);
-      }
-    }
 #pragma unroll 1
     for (int t = 0; t < 2; ++t) {
       if ((t ? it.n1 : it.n0) == 0) continue;
@@ -541,7 +588,6 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     for (int t = 0; t < 2; ++t) {
       tc::mbar_init(&sh->q_full[t], 1); tc::mbar_init(&sh->q_free[t], 1);
       tc::mbar_init(&sh->s_full[t], 1); tc::mbar_init(&sh->p_ready[t], 128);
-      tc::mbar_init(&sh->alpha_ready[t], 128); tc::mbar_init(&sh->o_corr[t], 128);
       tc::mbar_init(&sh->o_final[t], 1); tc::mbar_init(&sh->l_ready[t], 128); tc::mbar_init(&sh->o_free[t], 128);
     }
     for (int s = 0; s < KV_STAGES; ++s) {
@@ -549,6 +595,7 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
       tc::mbar_init(&sh->v_full[s], 1); tc::mbar_init(&sh->v_empty[s], 2);
     }
     sh->abort_flag = 0;
+    sh->pipe_lock = 0;
     tc::fence_barrier_init();
     tc::tma_prefetch_desc(&tmQ);
     tc::tma_prefetch_desc(&tmK);
@@ -564,7 +611,7 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
   if (warp < 8) {
     role_softmax(cx, tmem_base, warp >> 2, warp, lane, B, H, S, scale_log2);
   } else if (warp < 12) {
-    role_correction(cx, tmem_base, staging, warp, lane, out, B, H, S);
+    role_output(cx, tmem_base, staging, warp, lane, out, B, H, S);
   } else {
     if (warp == 12 && lane == 0) role_loader(cx, &tmQ, &tmK, &tmV, q_tiles, k_tiles, v_tiles, B, H, S);
     if ((warp == 13 || warp == 14) && lane == 0) role_mma(cx, tmem_base, warp - 13, q_tiles, k_tiles, v_tiles, B, H, S);

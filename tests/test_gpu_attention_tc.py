@@ -85,14 +85,16 @@ def test_c4_block_at_reduced_size(ctx):
 
 
 @pytest.mark.parametrize("impl", TC_IMPLS)
-def test_row_maximum_growing_from_key_tile_to_key_tile(ctx, impl):
-    """Keys whose magnitude grows by a large factor every 128 positions: the running row maximum jumps
-    by more than 2^8 at most tile boundaries, so the running output and row sum are rescaled each time
-    (the two-tile kernel skips the rescale for smaller jumps; both branches must agree with the oracle)."""
+@pytest.mark.parametrize("step", [3.0, 100.0])
+def test_row_maximum_growing_from_key_tile_to_key_tile(ctx, impl, step):
+    """Keys whose magnitude grows by a large factor every 128 positions, so the running row maximum
+    jumps at every tile boundary.  With step 3 the jumps are some tens of log2 units; with step 100 they
+    exceed the whole fp32 exponent range, so a kernel that keeps a stale reference maximum must notice
+    and rescale its running output and row sum (the two-tile kernel does so only then)."""
     b, h, s, d = 1, 2, 640, 128
     w = _attn_only(W.c4(5, B=b, H=h, S=s, D=d))
     k = w.inputs["k"].f64()
-    gain = 1.0 + 3.0 * (np.arange(s) // 128)
+    gain = 1.0 + step * (np.arange(s) // 128)
     w.inputs["k"] = G.make("k", "bf16", (k * gain[None, None, :, None]).astype(np.float32))
     ref, _ = oracle(w, [0])
     dw, out = run_gpu(ctx, w, [0], binds={0: impl})
