@@ -6,6 +6,8 @@ a row that share its built-in scratch array, and must refuse problems that array
 
 Collected last on purpose (file name), so a run that stops at the first failure has already run
 every other test."""
+import gc
+
 import numpy as np
 import pytest
 import torch
@@ -44,6 +46,8 @@ def test_noalloc_groupnorm_matches_the_workspace_path_twice_in_a_row(dtype):
         dw, ref = _module_groupnorm(ctx, x, gamma, beta, groups, 1e-5, dtype)
         y = torch.full_like(ref, float("nan"))
         g, b = dw.params["gamma"][0], dw.params["beta"][0]
+        gc.collect()            # tensors left over from earlier tests must not be freed between the two readings
+        torch.cuda.synchronize()
         before = torch.cuda.memory_allocated()
         st = B.mk_groupnorm_nhwc_noalloc(B.DTYPE[dtype], dw.inputs["x"].data_ptr(), y.data_ptr(), g.data_ptr(),
                                          b.data_ptr(), *shape, groups, 1e-5, stream)
