@@ -477,6 +477,89 @@ __global__ void __launch_bounds__(GN_THREADS) groupnorm_apply_generic(const T* _
   }
 }
 
+// Normalisation from partial sums that another kernel (the convolution's epilogue) has left behind:
+// float [nb][stat_slots][groups][2].  One CTA = one pixel chunk of one image; the partials of the image
+// are reduced by 2 * groups threads with independent loads, then every thread streams 16-byte vectors.
+template <typename T>
+__global__ void __launch_bounds__(GN_THREADS) groupnorm_apply_partials_kernel(const T* __restrict__ x, T* __restrict__ y, int64_t hw, int c,
+                                                                              int groups, const T* __restrict__ gamma,
+                                                                              const T* __restrict__ beta, float eps,
+                                                                              const float* __restrict__ stats, int stat_slots) {
+  constexpr int VE = Elem<T>::VEC;
+  __shared__ float sh_scale[GN_MAX_C];
+  __shared__ float sh_shift[GN_MAX_C];
+  __shared__ float sh_stat[2 * GN_MAX_C];
+  const int chunks = gridDim.x, chunk = blockIdx.x;
+  const int64_t img = blockIdx.y;
+  const int cg = c / groups;
+  const float* st = stats + img * stat_slots * groups * 2;
+  for (int idx = threadIdx.x; idx < 2 * groups; idx += GN_THREADS) {
+    float a0 = 0.0f, a1 = 0.0f, a2 = 0.0f, a3 = 0.0f;
+    int k = 0;
+    for (; k + 4 <= stat_slots; k += 4) {
+      a0 += st[(int64_t)(k + 0) * groups * 2 + idx];
+      a1 += st[(int64_t)(k + 1) * groups * 2 + idx];
+      a2 += st[(int64_t)(k + 2) * groups * 2 + idx];
+      a3 += st[(int64_t)(k + 3) * groups * 2 + idx];
+    }
+    for (; k < stat_slots; ++k) a0 += st[(int64_t)k * groups * 2 + idx];
+    sh_stat[idx] = (a0 + a1) + (a2 + a3);
+  }
+  __syncthreads();
+  const float inv_cnt = 1.0f / ((float)hw * (float)cg);
+  for (int ch = threadIdx.x; ch < c; ch += GN_THREADS) {
+    const int g = ch / cg;
+    const float mean = sh_stat[2 * g] * inv_cnt;
+    const float var = fmaxf(sh_stat[2 * g + 1] * inv_cnt - mean * mean, 0.0f);
+    const float rstd = rsqrtf(var + eps);
+    const float ga = gamma ? Elem<T>::ld(gamma + ch) : 1.0f;
+    const float be = beta ? Elem<T>::ld(beta + ch) : 0.0f;
+    sh_scale[ch] = rstd * ga;
+    sh_shift[ch] = be - mean * rstd * ga;
+  }
+  __syncthreads();
+  const int vpp = c / VE;
+  const int vcol = threadIdx.x % vpp, prow = threadIdx.x / vpp, pstride = GN_THREADS / vpp;
+  const int64_t p0 = hw * chunk / chunks, p1 = hw * (chunk + 1) / chunks;
+  float sc[VE], sf[VE];
+#pragma unroll
+  for (int e = 0; e < VE; ++e) { sc[e] = sh_scale[vcol * VE + e]; sf[e] = sh_shift[vcol * VE + e]; }
+#pragma unroll 4
+  for (int64_t pix = p0 + prow; pix < p1; pix += pstride) {
+    float v[VE];
+    const int64_t r = img * hw + pix;
+    ld_vec(x + r * c + vcol * VE, v);
+#pragma unroll
+    for (int e = 0; e < VE; ++e) v[e] = fmaf(v[e], sc[e], sf[e]);
+    st_vec(y + r * c + vcol * VE, v);
+  }
+}
+
+bool groupnorm_apply_partials_supported(int dtype, int64_t c, int groups) {
+  if (groups < 1 || c % groups) return false;
+  return dtype == DT_F32 ? gn_fast_ok<float>(c) : gn_fast_ok<__nv_bfloat16>(c);
+}
+cudaError_t launch_groupnorm_apply_partials(int dtype, const void* x, void* y, int64_t nb, int64_t hw, int64_t c, int groups,
+                                            const void* gamma, const void* beta, float eps, const float* stats, int stat_slots,
+                                            int sm_count, cudaStream_t s) {
+  if (nb == 0) return cudaSuccess;
+  if (!groupnorm_apply_partials_supported(dtype, c, groups)) return cudaErrorInvalidValue;
+  // about two CTAs per SM in all: few enough that the per-CTA reduction of the partials is amortised
+  int64_t chunks = (2 * (int64_t)sm_count + nb - 1) / nb;
+  const int64_t maxc = hw / 64 > 0 ? hw / 64 : 1;
+  if (chunks > maxc) chunks = maxc;
+  if (chunks < 1) chunks = 1;
+  dim3 grid((unsigned)chunks, (unsigned)nb);
+  if (dtype == DT_F32)
+    groupnorm_apply_partials_kernel<float><<<grid, GN_THREADS, 0, s>>>((const float*)x, (float*)y, hw, (int)c, groups, (const float*)gamma,
+                                                                       (const float*)beta, eps, stats, stat_slots);
+  else
+    groupnorm_apply_partials_kernel<__nv_bfloat16><<<grid, GN_THREADS, 0, s>>>((const __nv_bfloat16*)x, (__nv_bfloat16*)y, hw, (int)c, groups,
+                                                                               (const __nv_bfloat16*)gamma, (const __nv_bfloat16*)beta, eps,
+                                                                               stats, stat_slots);
+  return cudaGetLastError();
+}
+
 template <typename T>
 static cudaError_t gn_stats(const void* x, int64_t nb, int64_t hw, int64_t c, int groups, const EpiProgram& pre, float* scratch,
                             int chunks, cudaStream_t s) {

@@ -21,8 +21,8 @@
 //
 // Warp roles as in the GEMM: warp 0 TMA producer, warp 1 TMEM allocation + (leader) MMA issue with a
 // fully unrolled tap loop (a 256x128x16 MMA lasts 64 cycles, so the issuing thread may spend only a
-// handful of instructions per MMA), warps 2..5 epilogue with a double-buffered accumulator and
-// coalesced stores.  No TMA multicast.  Bounded waits.
+// handful of instructions per MMA), warps 2..9 epilogue (two per TMEM lane quarter) with a double-buffered
+// accumulator, coalesced stores and, on request, the GroupNorm partial sums of the stored values.  No TMA multicast.  Bounded waits.
 #include "device_common.cuh"
 #include "tc_common.cuh"
 #include "tc_epilogue.cuh"
@@ -37,7 +37,10 @@ constexpr int TILE_ROWS = 2;              // output rows per CTA
 constexpr int PATCH_ROWS = TILE_ROWS + 2; // input rows per CTA incl. halo
 constexpr int PATCH_BYTES = PATCH_ROWS * PITCH * 128;  // one 64-channel block: 32 KB
 constexpr int A_STAGES = 2;
-constexpr int THREADS = 192;
+constexpr int EPI_WARPS = 8;              // two per TMEM lane quarter, each taking half of the channel chunks
+constexpr int THREADS = 64 + 32 * EPI_WARPS;
+constexpr int STG_BYTES = 32 * 64;        // transpose buffer per epilogue warp: 32 rows x 64 bytes, XOR-swizzled
+constexpr int BIAS_BYTES = 512;           // one copy of the bias (C_out <= 256 bf16) per CTA
 
 struct Shared {
   uint64_t a_full[A_STAGES];
@@ -49,11 +52,75 @@ struct Shared {
   int abort_flag;
 };
 
+// 32 rows x 64 bytes from "one row per lane" to coalesced global stores (8 rows x 64 contiguous bytes per
+// instruction).  The 16-byte segment s of row r sits at segment s ^ ((r >> 1) & 3): both the row-wise
+// writes and the 8-lanes-per-two-rows reads then touch every bank group once.
+template <typename RowMap>
+__device__ __forceinline__ void store_rows64(uint8_t* stg, int lane, const uint4 (&mine)[4], RowMap rowmap, uint8_t* out, int64_t row_bytes,
+                                             int64_t byte_off) {
+  const int f = (lane >> 1) & 3;
+#pragma unroll
+  for (int sgm = 0; sgm < 4; ++sgm) *reinterpret_cast<uint4*>(stg + lane * 64 + ((sgm ^ f) * 16)) = mine[sgm];
+  __syncwarp();
+  const int sub_row = lane >> 2, seg = lane & 3;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int r = sub_row + 8 * i;
+    const int64_t gr = rowmap(r);
+    const uint4 val = *reinterpret_cast<const uint4*>(stg + r * 64 + ((seg ^ ((r >> 1) & 3)) * 16));
+    if (gr >= 0) *reinterpret_cast<uint4*>(out + gr * row_bytes + byte_off + seg * 16) = val;
+  }
+  __syncwarp();
+}
+
+// Sum over the warp's 32 rows of N per-lane values, N a power of two: each step halves the number of
+// values a lane carries (it keeps one half and receives the partner's other half), so N values cost N
+// shuffles instead of 5 N.  On return lane L holds, in a[0], the total of value L >> (5 - log2 N)
+// (every lane of that group of lanes holds the same total).
+template <int N>
+__device__ __forceinline__ void fold_rows(float* a, int lane, int m) {
+  if constexpr (N > 1) {
+    const bool up = (lane & m) != 0;
+#pragma unroll
+    for (int i = 0; i < N / 2; ++i) {
+      const float send = up ? a[i] : a[i + N / 2];
+      const float keep = up ? a[i + N / 2] : a[i];
+      a[i] = keep + __shfl_xor_sync(0xffffffffu, send, m);
+    }
+    fold_rows<N / 2>(a, lane, m >> 1);
+  } else {
+    for (; m >= 1; m >>= 1) a[0] += __shfl_xor_sync(0xffffffffu, a[0], m);
+  }
+}
+// GroupNorm partial sums of one 32-channel chunk over the warp's 32 pixels: groups of CPG adjacent
+// channels; dst = float[32 / CPG][2] = (sum, sum of squares) per group.  Rows that are not stored count 0.
+template <int CPG>
+__device__ __forceinline__ void chunk_stats(const float (&v)[32], bool valid, int lane, float* __restrict__ dst) {
+  constexpr int GPC = 32 / CPG, NV = 2 * GPC;
+  float a[NV];
+#pragma unroll
+  for (int g = 0; g < GPC; ++g) {
+    float sm = 0.0f, sq = 0.0f;
+#pragma unroll
+    for (int e = 0; e < CPG; ++e) {
+      const float x = valid ? v[g * CPG + e] : 0.0f;
+      sm += x;
+      sq = fmaf(x, x, sq);
+    }
+    a[2 * g] = sm;
+    a[2 * g + 1] = sq;
+  }
+  fold_rows<NV>(a, lane, 16);
+  constexpr int LOG = NV == 16 ? 4 : NV == 8 ? 3 : NV == 4 ? 2 : 1;
+  if ((lane & ((1 << (5 - LOG)) - 1)) == 0) dst[lane >> (5 - LOG)] = a[0];
+}
+
 // CB = C_in / 64 channel blocks
 template <int CB>
 __global__ void __launch_bounds__(THREADS, 1)
 conv3x3_tc2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW, __nv_bfloat16* __restrict__ y,
-                   int NB, int H, int W, int C_OUT, const __grid_constant__ EpiProgram epi, unsigned int* status) {
+                   int NB, int H, int W, int C_OUT, const __grid_constant__ EpiProgram epi, float* __restrict__ stats, int cpg,
+                   unsigned int* status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const int b_rows = C_OUT / 2;                       // weight rows held by this CTA
@@ -62,7 +129,7 @@ conv3x3_tc2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
   uint8_t* a_tiles = base;                            // A_STAGES patches (+ 1 KB the last tap's junk rows may touch)
   uint8_t* b_tiles = base + A_STAGES * PATCH_BYTES + 1024;
   uint8_t* staging = b_tiles + b_bytes;
-  Shared* sh = reinterpret_cast<Shared*>(staging + 4 * EPI_WARP_BYTES);
+  Shared* sh = reinterpret_cast<Shared*>(staging + EPI_WARPS * STG_BYTES + BIAS_BYTES);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = tc::cluster_ctarank();
   const bool leader = rank == 0;
@@ -76,7 +143,7 @@ conv3x3_tc2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
   if (threadIdx.x == 0) {
     for (int s = 0; s < A_STAGES; ++s) { tc::mbar_init(&sh->a_full[s], 1); tc::mbar_init(&sh->a_empty[s], 1); }
     tc::mbar_init(&sh->b_full, 1);
-    for (int b = 0; b < 2; ++b) { tc::mbar_init(&sh->tfull[b], 1); tc::mbar_init(&sh->tempty[b], 8); }
+    for (int b = 0; b < 2; ++b) { tc::mbar_init(&sh->tfull[b], 1); tc::mbar_init(&sh->tempty[b], 2 * EPI_WARPS); }
     sh->abort_flag = 0;
     tc::fence_barrier_init();
     tc::tma_prefetch_desc(&tmX);
@@ -163,11 +230,22 @@ conv3x3_tc2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     __syncwarp();
   } else {
     // ------------------------------------------------------------ epilogue: 128 tile rows = 2 output rows x 64 pitch
-    const int q = warp & 3;
-    EpiWarp ew;
-    ew.init(staging + q * EPI_WARP_BYTES, epi, lane, false);
-    ew.load_bias(epi, 0, C_OUT, C_OUT);          // the bias slice is the same for every tile: once
-    const int chunks = C_OUT / 32;
+    // Warps w and w + 4 share TMEM lane quarter q (tile rows [32q, 32q + 32)) and split its channel chunks.
+    const int ew = warp - 2, q = warp & 3, half = ew >> 2;
+    uint8_t* stg = staging + ew * STG_BYTES;
+    uint8_t* bias_sh = staging + EPI_WARPS * STG_BYTES;
+    const int bias_idx = epi_single_index(epi, EPI_BIAS);
+    if (bias_idx >= 0) {
+      // the bias slice is the same for every tile: one copy per CTA, once
+      for (int i = (int)threadIdx.x - 64; i < C_OUT / 8; i += 32 * EPI_WARPS)
+        reinterpret_cast<uint4*>(bias_sh)[i] = reinterpret_cast<const uint4*>(epi.op[bias_idx].ptr)[i];
+    }
+    asm volatile("bar.sync 1, %0;" ::"n"(32 * EPI_WARPS) : "memory");
+    const int chunks = C_OUT / 32, c_mid = (chunks + 1) / 2;
+    const int c_lo = half ? c_mid : 0, c_hi = half ? chunks : c_mid;
+    const int groups = stats ? C_OUT / cpg : 0;
+    const int stat_slots = quads * 2 * 4;          // partial sums per image: one per (pair-tile, CTA, lane quarter)
+    const uint4 no_res[4] = {};
     bool ok = true;
     int it = 0;
     for (int t = cluster_id; t < total_tiles && ok; t += num_clusters, ++it) {
@@ -179,23 +257,41 @@ conv3x3_tc2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
       const int64_t pix0 = ((int64_t)n * H + h) * W;
       const bool row_ok = h < H;
       auto rowmap = [&](int r) -> int64_t { return (row_ok && w0 + r < W) ? pix0 + w0 + r : -1; };
-      uint4 res_regs[8];
-      ew.prefetch_res(epi, rowmap, 0, C_OUT, res_regs);
+      const int64_t my_row = rowmap(lane);
       ok = tc::mbar_wait(&sh->tfull[acc], (it >> 1) & 1, abort_flag, status, tc::WAIT_TMEM_FULL);
       ok = __all_sync(0xffffffffu, ok ? 1 : 0) != 0;
       if (!ok) break;
       if (threadIdx.x == 64) MK_TR(4 + it * 8);  // epilogue: accumulator ready
       tc::tc_fence_after();
       const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + acc * 256;
+      float* stat_dst = stats ? stats + (((int64_t)n * stat_slots + (hq * 2 + (int)rank) * 4 + q) * groups) * 2 : nullptr;
 #pragma unroll 1
-      for (int c = 0; c < chunks; ++c) {
+      for (int c = c_lo; c < c_hi; ++c) {
         uint32_t rr[32];
         float v[32];
         tc::tmem_ld32(t_row + c * 32, rr);
         tc::tmem_ld_wait();
 #pragma unroll
         for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(rr[j]);
-        ew.chunk_out(epi, v, rowmap, y, (int64_t)c * 32, c * 32, (int64_t)C_OUT, res_regs, c + 1 < chunks ? (int64_t)(c + 1) * 32 : -1);
+        if (my_row >= 0) epi32(epi, v, my_row, (int64_t)c * 32, (int64_t)C_OUT, bias_idx >= 0 ? bias_sh + c * 64 : nullptr, 0, no_res, no_res);
+        if (stats) {
+          float* d = stat_dst + (c * 32 / cpg) * 2;
+          switch (cpg) {
+            case 4: chunk_stats<4>(v, my_row >= 0, lane, d); break;
+            case 8: chunk_stats<8>(v, my_row >= 0, lane, d); break;
+            case 16: chunk_stats<16>(v, my_row >= 0, lane, d); break;
+            default: chunk_stats<32>(v, my_row >= 0, lane, d); break;
+          }
+        }
+        uint4 mine[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          mine[k].x = pack_bf16x2(v[8 * k + 0], v[8 * k + 1]);
+          mine[k].y = pack_bf16x2(v[8 * k + 2], v[8 * k + 3]);
+          mine[k].z = pack_bf16x2(v[8 * k + 4], v[8 * k + 5]);
+          mine[k].w = pack_bf16x2(v[8 * k + 6], v[8 * k + 7]);
+        }
+        store_rows64(stg, lane, mine, rowmap, reinterpret_cast<uint8_t*>(y), (int64_t)C_OUT * 2, (int64_t)c * 64);
       }
       tc::tc_fence_before();
       __syncwarp();
@@ -219,10 +315,12 @@ conv3x3_tc2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
 }
 
 size_t conv_smem_bytes(int c_in, int c_out) {
-  return (size_t)A_STAGES * PATCH_BYTES + 1024 + (size_t)(c_out / 2) * 9 * c_in * 2 + 4 * EPI_WARP_BYTES + 1024 + 256;
+  return (size_t)A_STAGES * PATCH_BYTES + 1024 + (size_t)(c_out / 2) * 9 * c_in * 2 + EPI_WARPS * STG_BYTES + BIAS_BYTES + 1024 + 256;
 }
 
 }  // namespace
+
+int conv3x3_tc2_stat_slots(int64_t h) { return (int)((h + 2 * TILE_ROWS - 1) / (2 * TILE_ROWS)) * 2 * 4; }
 
 bool conv3x3_tc2_supported(int64_t nb, int64_t h, int64_t w, int64_t c_in, int64_t c_out) {
   if (nb < 1 || h < 1 || w < 1 || w > PITCH - 2) return false;
@@ -244,6 +342,8 @@ cudaError_t conv3x3_tc2_plan(ConvTcPlan* p, const void* x, const void* w, void* 
   cudaError_t e = encode_tmap_2d_bf16(&p->tm_w, w, (uint64_t)c_out, (uint64_t)(9 * c_in), (uint64_t)(9 * c_in), (uint32_t)(c_out / 2), 64);
   if (e != cudaSuccess) return e;
   p->y = y;
+  p->stats = nullptr;
+  p->cpg = 0;
   p->nb = (int)nb; p->h = (int)h; p->w = (int)wd; p->c_in = (int)c_in; p->c_out = (int)c_out;
   p->epi = epi;
   const int64_t tiles = nb * ((h + 2 * TILE_ROWS - 1) / (2 * TILE_ROWS));
@@ -275,8 +375,8 @@ cudaError_t launch_conv3x3_tc2(const ConvTcPlan& p, cudaStream_t s) {
   cfg.numAttrs = 1;
   unsigned int* status = kernel_status_ptr();
   __nv_bfloat16* y = (__nv_bfloat16*)p.y;
-  if (p.c_in == 64) return cudaLaunchKernelEx(&cfg, conv3x3_tc2_kernel<1>, p.tm_x, p.tm_w, y, p.nb, p.h, p.w, p.c_out, p.epi, status);
-  return cudaLaunchKernelEx(&cfg, conv3x3_tc2_kernel<2>, p.tm_x, p.tm_w, y, p.nb, p.h, p.w, p.c_out, p.epi, status);
+  if (p.c_in == 64) return cudaLaunchKernelEx(&cfg, conv3x3_tc2_kernel<1>, p.tm_x, p.tm_w, y, p.nb, p.h, p.w, p.c_out, p.epi, p.stats, p.cpg, status);
+  return cudaLaunchKernelEx(&cfg, conv3x3_tc2_kernel<2>, p.tm_x, p.tm_w, y, p.nb, p.h, p.w, p.c_out, p.epi, p.stats, p.cpg, status);
 }
 
 }  // namespace mk

@@ -262,6 +262,56 @@ mk_status conv_tc2_emit(const Module& m, int lo, int hi, const Resolved& r, std:
   return MK_OK;
 }
 
+// CONV2D_3x3 [elementwise]* GROUPNORM: the convolution's epilogue leaves the GroupNorm partial sums of
+// what it stores, so the statistics pass over the activation disappears; the activation itself sits in
+// scratch between the two launches (the normalisation needs the whole image's statistics first).
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+bool conv_gn_tc2_match(const Module& m, int lo, int hi) {
+  if (hi - lo < 2 || m.ops[hi - 1].d.kind != MK_OP_GROUPNORM || !is_chain(m, lo, hi)) return false;
+  if (!conv_tc2_match(m, lo, hi - 1)) return false;
+  const mk_tensor_spec& s = m.vspec(m.ops[hi - 1].out_id);
+  const int64_t c = s.shape[3];
+  const int groups = m.ops[hi - 1].d.i[0];
+  if (groups < 1 || c % groups) return false;
+  const int64_t cpg = c / groups;
+  if (cpg != 4 && cpg != 8 && cpg != 16 && cpg != 32) return false;
+  return groupnorm_apply_partials_supported(dt(m), c, groups);
+}
+size_t conv_gn_tc2_scratch(const Module& m, int, int hi) {
+  const mk_tensor_spec& s = m.vspec(m.ops[hi - 1].out_id);
+  const size_t act = (size_t)s.shape[0] * s.shape[1] * s.shape[2] * s.shape[3] * 2;
+  const size_t st = (size_t)s.shape[0] * conv3x3_tc2_stat_slots(s.shape[1]) * m.ops[hi - 1].d.i[0] * 2 * sizeof(float);
+  return align_up(act, 1024) + st;
+}
+mk_status conv_gn_tc2_emit(const Module& m, int lo, int hi, const Resolved& r, std::vector<Launch>& out, std::string& err) {
+  EpiProgram p;
+  mk_status st = build_epi(m, lo + 1, hi - 1, r, p, err);
+  if (st != MK_OK) return st;
+  const Op& op = m.ops[lo];
+  const Op& gn = m.ops[hi - 1];
+  const mk_tensor_spec& xs = m.vspec(op.in_id[0]);
+  const mk_tensor_spec& ys = m.vspec(gn.out_id);
+  const int64_t nb = ys.shape[0], hw = ys.shape[1] * ys.shape[2], c = ys.shape[3];
+  const int groups = gn.d.i[0];
+  char* act = (char*)r.scratch;
+  float* stats = (float*)(act + align_up((size_t)nb * hw * c * 2, 1024));
+  const int slots = conv3x3_tc2_stat_slots(ys.shape[1]);
+  auto plan = std::make_shared<ConvTcPlan>();
+  cudaError_t e = conv3x3_tc2_plan(plan.get(), r.value_ptr[op.in_id[0]], op.param[0].ptr, act, xs.shape[0], xs.shape[1], xs.shape[2],
+                                   xs.shape[3], op.d.i[0], p, m.ctx->sm_count);
+  if (e != cudaSuccess) { err = std::string("conv3x3_tc2 plan: ") + cudaGetErrorString(e); return MK_ERR_CUDA; }
+  plan->stats = stats;
+  plan->cpg = (int)(c / groups);
+  out.push_back([plan](cudaStream_t s) { return launch_conv3x3_tc2(*plan, s); });
+  void* y = r.value_ptr[gn.out_id];
+  const void* g = gn.param[0].set ? gn.param[0].ptr : nullptr;
+  const void* b = gn.param[1].set ? gn.param[1].ptr : nullptr;
+  const float eps = (float)gn.d.f[0];
+  const int d = dt(m), sms = m.ctx->sm_count;
+  out.push_back([=](cudaStream_t s_) { return launch_groupnorm_apply_partials(d, act, y, nb, hw, c, groups, g, b, eps, stats, slots, sms, s_); });
+  return MK_OK;
+}
+
 // ------------------------------------------------------------------ attention
 AttnView attn_view(const Module& m, const Op& op, const Resolved& r) {
   AttnView a{};
@@ -333,6 +383,7 @@ const std::vector<Impl>& registry() {
       {"gemm_tc2", gemm_tc2_match, no_scratch, gemm_tc2_emit},
       {"gemm_tc", gemm_tc_match, no_scratch, gemm_tc_emit},
       {"gemm_simt", gemm_simt_match, no_scratch, gemm_simt_emit},
+      {"conv3x3_gn_tc2", conv_gn_tc2_match, conv_gn_tc2_scratch, conv_gn_tc2_emit},
       {"conv3x3_tc2", conv_tc2_match, no_scratch, conv_tc2_emit},
       {"conv3x3_simt", conv_simt_match, no_scratch, conv_simt_emit},
       {"attention_tc2", attn_tc2_match, no_scratch, attn_tc2_emit},

@@ -65,6 +65,12 @@ cudaError_t launch_groupnorm_apply(int dtype, const void* x, void* y, int64_t nb
                                    int64_t c, int groups, const void* gamma, const void* beta,
                                    float eps, const EpiProgram& pre, const float* scratch, int chunks,
                                    cudaStream_t s);
+// Normalisation alone, from partial sums float [nb][stat_slots][groups][2] written by the producer of x
+// (the convolution's epilogue).  Needs c to be a multiple of the 16-byte vector and at most 2048.
+bool groupnorm_apply_partials_supported(int dtype, int64_t c, int groups);
+cudaError_t launch_groupnorm_apply_partials(int dtype, const void* x, void* y, int64_t nb, int64_t hw, int64_t c, int groups,
+                                            const void* gamma, const void* beta, float eps, const float* stats, int stat_slots,
+                                            int sm_count, cudaStream_t s);
 
 // ---- plain-ALU (SIMT) kernels: any shape, fp32 or bf16, fp32 accumulation -------------------------
 // Y[M, N] = program(A[M, K] @ W); W is [K, N] row-major, or [N, K] when w_transposed.

@@ -36,6 +36,10 @@ namespace mk {
 struct ConvTcPlan {
   CUtensorMap tm_x, tm_w;
   void* y = nullptr;
+  // optional GroupNorm partial sums of the stored output: float [nb][conv3x3_tc2_stat_slots(h)][c_out / cpg][2]
+  // = (sum, sum of squares) per group of cpg adjacent channels (cpg in {4, 8, 16, 32}); null: none
+  float* stats = nullptr;
+  int cpg = 0;
   int nb = 0, h = 0, w = 0, c_in = 0, c_out = 0;
   int grid = 0;
   size_t smem = 0;
@@ -45,6 +49,7 @@ struct ConvTcPlan {
 // Supported: C_in in {64, 128}, C_out multiple of 32 up to 256, W <= 62, and half the weights
 // plus two input patches must fit one SM's shared memory.
 bool conv3x3_tc2_supported(int64_t nb, int64_t h, int64_t w, int64_t c_in, int64_t c_out);
+int conv3x3_tc2_stat_slots(int64_t h);
 cudaError_t conv3x3_tc2_plan(ConvTcPlan* p, const void* x, const void* w, void* y, int64_t nb, int64_t h, int64_t wd, int64_t c_in,
                              int64_t c_out, const EpiProgram& epi, int sm_count);
 cudaError_t launch_conv3x3_tc2(const ConvTcPlan& p, cudaStream_t s);

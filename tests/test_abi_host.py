@@ -179,3 +179,27 @@ def test_host_only_context_cannot_launch(ctx):
     with pytest.raises(MkError) as e:
         m.forward([1 << 20], 1 << 21, None, 0, 0)
     assert e.value.status == B.MK_ERR_NO_DEVICE
+
+
+def test_fp32_residual_stream_dtypes(ctx):
+    """RESIDUAL_ADD with an fp32 store produces an fp32 value next to bf16 activations: the row norm that
+    reads it writes the module dtype again, the next residual may read the fp32 value as its second
+    operand, and a contraction refuses an fp32 operand in a bf16 module."""
+    w = W.c5(0, B=1, S=4, E=8, H=2, F=8, L=1)
+    m = _mod(ctx, w)
+    assert m.value_spec("x1_0")[0] == B.MK_F32 and m.value_spec("x2_0")[0] == B.MK_F32
+    assert m.value_spec("n2_0")[0] == B.MK_BF16 and m.value_spec("y")[0] == B.MK_BF16
+    assert m.value_spec("x1_0")[1] == (4, 8)
+    # the same module with a bf16 stream: every value is bf16
+    wb = W.c5(0, B=1, S=4, E=8, H=2, F=8, L=1, stream="bf16")
+    mb = _mod(ctx, wb)
+    assert mb.value_spec("x1_0")[0] == B.MK_BF16 and mb.value_spec("x2_0")[0] == B.MK_BF16
+    # a linear fed directly from the fp32 stream (no norm in between) is rejected
+    ops = [dict(o) for o in w.ops]
+    ops[6] = dict(ops[6], **{"in": ["x1_0"]})            # gu_0 = linear(x1_0) instead of linear(n2_0)
+    with pytest.raises(MkError):
+        Module(ctx, ops, {"x": ("bf16", (4, 8))})
+    # contracts carry the dtype across a split at the stream
+    m.set_decomposition([0, 5])
+    ins, outs = m.contract(1)
+    assert any(dt == B.MK_F32 for _, (dt, _, _) in ins)

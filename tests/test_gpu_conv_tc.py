@@ -45,8 +45,25 @@ def test_conv_chain_matches_the_oracle(ctx, nb, h, w, c, co):
         ref, _ = oracle(wl, [0])
         for part in ("fused", "split2", "split3"):
             dw, out = run_gpu(ctx, wl, wl.partitions[part])
-            assert dw.module.bound_impl(0).startswith("conv3x3_tc2"), dw.module.bound_impl(0)
+            want = "conv3x3_gn_tc2" if part == "fused" else "conv3x3_tc2"
+            assert dw.module.bound_impl(0).startswith(want), dw.module.bound_impl(0)
             assert_parity(out, ref, "bf16", f"{part} seed {seed}")
+
+
+@pytest.mark.parametrize("nb,h,w,c,co,g", [(2, 8, 8, 64, 64, 16), (3, 9, 7, 128, 128, 32), (2, 13, 62, 64, 96, 12), (1, 6, 10, 64, 256, 16),
+                                           (2, 5, 33, 64, 32, 1), (4, 56, 56, 128, 128, 32)])
+def test_groupnorm_statistics_from_the_conv_epilogue(ctx, nb, h, w, c, co, g):
+    """The fused form: the convolution's epilogue leaves per-(image, group) partial sums of what it stores
+    and the normalisation reads only those (4, 8, 16 and 32 channels per group; image heights that do not
+    fill the last tile; widths that leave junk rows in the tile).  Swapped against the two-pass GroupNorm."""
+    wl = W.c3(2, NB=nb, H=h, W=w, C=c, CO=co, G=g)
+    ref, _ = oracle(wl, [0])
+    dw, out = run_gpu(ctx, wl, wl.partitions["fused"])
+    assert dw.module.bound_impl(0) == "conv3x3_gn_tc2"
+    assert_parity(out, ref, "bf16", "fused")
+    dw2, out2 = run_gpu(ctx, wl, wl.partitions["split2"])
+    assert dw2.module.bound_impl(1) == "groupnorm_nhwc"
+    assert np.abs(out - out2).max() <= 4e-2
 
 
 def test_swap_conv_kernels(ctx):

@@ -34,7 +34,7 @@ def test_c3_full_every_element(ctx):
     ref, _ = OM.run_workload(w, [0])
     for part in ("fused", "split2"):
         dw, out = run_gpu(ctx, w, w.partitions[part])
-        assert dw.module.bound_impl(0).startswith("conv3x3_tc2")
+        assert dw.module.bound_impl(0) == ("conv3x3_gn_tc2" if part == "fused" else "conv3x3_tc2")
         assert_parity(out, ref, "bf16", f"c3 {part}")
     # per (image, group) statistics of the output before the affine: mean 0, variance 1
     g, b = w.params["gamma"].f64(), w.params["beta"].f64()
