@@ -307,6 +307,47 @@ def run_ours(args):
     step_ms = sorted(a.elapsed_time(b) for a, b in ev)
     kernel_ms = sum(step_ms) / len(step_ms)
 
+    # ---- launch-bound steps (a few microseconds of device work): the Python loop above times the host,
+    # not the GPU.  Replay the same K steps from a CUDA graph (one node per kernel launch, the
+    # rotation over input sets unrolled into it) and time that with events; a graph of as many
+    # one-element kernels gives the launch floor beside it.
+    graph_info = None
+    if kernel_ms < 0.1:
+        gstream = torch.cuda.Stream()
+        gstream.wait_stream(stream)
+        reps = max(1, args.steps // rot)
+        with torch.cuda.stream(gstream):
+            for dw in sets:
+                dw.forward()            # launch plans for this stream exist before capture
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=gstream):
+                for dw in sets:
+                    dw.forward()
+            tiny = torch.zeros(1, device=f"cuda:{local}")
+            gf = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(gf, stream=gstream):
+                for _ in range(rot * launches_per_step):
+                    tiny.add_(1.0)
+            for _ in range(3):
+                g.replay(); gf.replay()
+            torch.cuda.synchronize()
+            g0, g1, g2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+            g0.record(gstream)
+            for _ in range(reps):
+                g.replay()
+            g1.record(gstream)
+            for _ in range(reps):
+                gf.replay()
+            g2.record(gstream)
+            torch.cuda.synchronize()
+        ctx.check()
+        graph_info = {"ms_per_step": g0.elapsed_time(g1) / (reps * rot), "steps": reps * rot,
+                      "launch_floor_ms_per_step": g1.elapsed_time(g2) / (reps * rot),
+                      "eager_ms_per_step": total_ms / args.steps}
+        total_ms = graph_info["ms_per_step"] * args.steps
+        kernel_ms = graph_info["ms_per_step"]
+
     # ---- end to end: pinned host inputs in, result out, every step
     host_in = {k: torch.empty(t.shape, dtype=sets[0].inputs[k].dtype).pin_memory() for k, t in w.inputs.items()}
     for k in host_in:
@@ -383,7 +424,9 @@ def run_ours(args):
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
             "config": {"workload": name, "decomposition": part, "impls": impls,
-                       "l2": f"rotation over {rot} independent input/output sets ({rot * per_copy / 1e6:.0f} MB > L2)",
+                       "l2": (f"rotation over {rot} independent input/output sets ({rot * per_copy / 1e6:.0f} MB > L2)" if rot * per_copy > 126e6 else
+                              f"rotation over {rot} independent input/output sets ({rot * per_copy / 1e6:.1f} MB in all: the whole problem is "
+                              "smaller than L2 and bound by launch latency, so L2 residency is part of the measurement)"),
                        "shapes": {k: list(t.shape) for k, t in w.inputs.items()}},
             "roofline": roofline_of(name, launches_per_step, dominant, achieved, peak, pk, kernel_ms, t_roof_ms, ms_per_step, step_ms[0]),
             "e2e": {"value": world * w.flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
@@ -392,6 +435,9 @@ def run_ours(args):
             "clocks": clocks,
             "per_subkernel": breakdown,
         }
+        if graph_info:
+            line["config"]["timing"] = "CUDA graph replay (the step is launch-bound; eager Python-loop time kept beside it)"
+            line["graph"] = graph_info
         if not args.no_cpu and world == 1:
             f, s, what = oracle_sample(name, w, budget_s=args.cpu_seconds)
             line["cpu_baseline"] = {"value": f / s / 1e12, "unit": "TFLOP/s", "cores": os.cpu_count(), "kind": "oracle",

@@ -478,32 +478,76 @@ __global__ void __launch_bounds__(GN_THREADS) groupnorm_apply_generic(const T* _
 }
 
 // Normalisation from partial sums that another kernel (the convolution's epilogue) has left behind:
-// float [nb][stat_slots][groups][2].  One CTA = one pixel chunk of one image; the partials of the image
-// are reduced by 2 * groups threads with independent loads, then every thread streams 16-byte vectors.
+// float [nb][stat_slots][groups][2].  One CTA = one pixel chunk of one image.  The first batch of
+// activation loads is issued BEFORE the statistics are reduced (they do not depend on them), and the
+// main loop keeps a batch of 16-byte loads in flight while it normalises and stores the previous one.
 template <typename T>
-__global__ void __launch_bounds__(GN_THREADS) groupnorm_apply_partials_kernel(const T* __restrict__ x, T* __restrict__ y, int64_t hw, int c,
+__global__ void __launch_bounds__(GN_THREADS, 3) groupnorm_apply_partials_kernel(const T* __restrict__ x, T* __restrict__ y, int64_t hw, int c,
                                                                               int groups, const T* __restrict__ gamma,
                                                                               const T* __restrict__ beta, float eps,
                                                                               const float* __restrict__ stats, int stat_slots) {
   constexpr int VE = Elem<T>::VEC;
+  constexpr int UN = 4;
   __shared__ float sh_scale[GN_MAX_C];
   __shared__ float sh_shift[GN_MAX_C];
   __shared__ float sh_stat[2 * GN_MAX_C];
+  __shared__ float sh_part[8][2 * 64];
   const int chunks = gridDim.x, chunk = blockIdx.x;
   const int64_t img = blockIdx.y;
   const int cg = c / groups;
+  const int vpp = c / VE;
+  const int vcol = threadIdx.x % vpp, prow = threadIdx.x / vpp, pstride = GN_THREADS / vpp;
+  const int64_t p0 = hw * chunk / chunks, p1 = hw * (chunk + 1) / chunks;
+  const T* xin = x + (img * hw) * c + vcol * VE;
+  T* yout = y + (img * hw) * c + vcol * VE;
+  RawVec<T, VE> cur[UN];
+  int64_t pix = p0 + prow;
+#pragma unroll
+  for (int u = 0; u < UN; ++u)
+    if (pix + (int64_t)u * pstride < p1) cur[u].load(xin + (pix + (int64_t)u * pstride) * c);
+
+  // Reduction of the partials: 2 * groups columns, the slots of a column split over as many threads as
+  // the CTA can spare, sixteen independent loads in flight per thread.
   const float* st = stats + img * stat_slots * groups * 2;
-  for (int idx = threadIdx.x; idx < 2 * groups; idx += GN_THREADS) {
-    float a0 = 0.0f, a1 = 0.0f, a2 = 0.0f, a3 = 0.0f;
-    int k = 0;
-    for (; k + 4 <= stat_slots; k += 4) {
-      a0 += st[(int64_t)(k + 0) * groups * 2 + idx];
-      a1 += st[(int64_t)(k + 1) * groups * 2 + idx];
-      a2 += st[(int64_t)(k + 2) * groups * 2 + idx];
-      a3 += st[(int64_t)(k + 3) * groups * 2 + idx];
+  const int ncol = 2 * groups;
+  int parts = GN_THREADS / ncol;
+  if (parts < 1) parts = 1;
+  if (parts > 8) parts = 8;
+  const bool small = ncol <= 128 && parts > 1;
+  if (small) {
+    const int col = threadIdx.x % ncol, part = threadIdx.x / ncol;
+    if (part < parts) {
+      float acc = 0.0f;
+      for (int k0 = part; k0 < stat_slots; k0 += 16 * parts) {
+        float t[16];
+#pragma unroll
+        for (int u = 0; u < 16; ++u) {
+          const int k = k0 + u * parts;
+          t[u] = k < stat_slots ? st[(int64_t)k * ncol + col] : 0.0f;
+        }
+#pragma unroll
+        for (int u = 0; u < 16; ++u) acc += t[u];
+      }
+      sh_part[part][col] = acc;
     }
-    for (; k < stat_slots; ++k) a0 += st[(int64_t)k * groups * 2 + idx];
-    sh_stat[idx] = (a0 + a1) + (a2 + a3);
+    __syncthreads();
+    if ((int)threadIdx.x < ncol) {
+      float acc = 0.0f;
+      for (int p = 0; p < parts; ++p) acc += sh_part[p][threadIdx.x];
+      sh_stat[threadIdx.x] = acc;
+    }
+  } else {
+    for (int idx = threadIdx.x; idx < ncol; idx += GN_THREADS) {
+      float acc = 0.0f;
+      for (int k0 = 0; k0 < stat_slots; k0 += 16) {
+        float t[16];
+#pragma unroll
+        for (int u = 0; u < 16; ++u) t[u] = k0 + u < stat_slots ? st[(int64_t)(k0 + u) * ncol + idx] : 0.0f;
+#pragma unroll
+        for (int u = 0; u < 16; ++u) acc += t[u];
+      }
+      sh_stat[idx] = acc;
+    }
   }
   __syncthreads();
   const float inv_cnt = 1.0f / ((float)hw * (float)cg);
@@ -518,20 +562,28 @@ __global__ void __launch_bounds__(GN_THREADS) groupnorm_apply_partials_kernel(co
     sh_shift[ch] = be - mean * rstd * ga;
   }
   __syncthreads();
-  const int vpp = c / VE;
-  const int vcol = threadIdx.x % vpp, prow = threadIdx.x / vpp, pstride = GN_THREADS / vpp;
-  const int64_t p0 = hw * chunk / chunks, p1 = hw * (chunk + 1) / chunks;
   float sc[VE], sf[VE];
 #pragma unroll
   for (int e = 0; e < VE; ++e) { sc[e] = sh_scale[vcol * VE + e]; sf[e] = sh_shift[vcol * VE + e]; }
-#pragma unroll 4
-  for (int64_t pix = p0 + prow; pix < p1; pix += pstride) {
-    float v[VE];
-    const int64_t r = img * hw + pix;
-    ld_vec(x + r * c + vcol * VE, v);
+  for (; pix < p1; pix += (int64_t)UN * pstride) {
+    RawVec<T, VE> nxt[UN];
+    const int64_t npix = pix + (int64_t)UN * pstride;
 #pragma unroll
-    for (int e = 0; e < VE; ++e) v[e] = fmaf(v[e], sc[e], sf[e]);
-    st_vec(y + r * c + vcol * VE, v);
+    for (int u = 0; u < UN; ++u)
+      if (npix + (int64_t)u * pstride < p1) nxt[u].load(xin + (npix + (int64_t)u * pstride) * c);
+#pragma unroll
+    for (int u = 0; u < UN; ++u) {
+      const int64_t pp = pix + (int64_t)u * pstride;
+      if (pp < p1) {
+        float v[VE];
+        cur[u].unpack(v);
+#pragma unroll
+        for (int e = 0; e < VE; ++e) v[e] = fmaf(v[e], sc[e], sf[e]);
+        st_vec(yout + pp * c, v);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < UN; ++u) cur[u] = nxt[u];
   }
 }
 
@@ -544,8 +596,14 @@ cudaError_t launch_groupnorm_apply_partials(int dtype, const void* x, void* y, i
                                             int sm_count, cudaStream_t s) {
   if (nb == 0) return cudaSuccess;
   if (!groupnorm_apply_partials_supported(dtype, c, groups)) return cudaErrorInvalidValue;
-  // about two CTAs per SM in all: few enough that the per-CTA reduction of the partials is amortised
-  int64_t chunks = (2 * (int64_t)sm_count + nb - 1) / nb;
+  // exactly one wave: as many pixel chunks per image as the resident CTAs of the whole GPU allow
+  int occ = 0;
+  cudaError_t oe = dtype == DT_F32
+                       ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, groupnorm_apply_partials_kernel<float>, GN_THREADS, 0)
+                       : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, groupnorm_apply_partials_kernel<__nv_bfloat16>, GN_THREADS, 0);
+  if (oe != cudaSuccess) return oe;
+  if (occ < 1) occ = 1;
+  int64_t chunks = ((int64_t)occ * sm_count) / nb;
   const int64_t maxc = hw / 64 > 0 ? hw / 64 : 1;
   if (chunks > maxc) chunks = maxc;
   if (chunks < 1) chunks = 1;

@@ -45,7 +45,7 @@ constexpr int BIAS_BYTES = 512;           // one copy of the bias (C_out <= 256 
 struct Shared {
   uint64_t a_full[A_STAGES];
   uint64_t a_empty[A_STAGES];
-  uint64_t b_full;
+  uint64_t b_full[2];      // weights of channel block 0 / 1 (the MMAs start when the first has landed)
   uint64_t tfull[2];
   uint64_t tempty[2];
   uint32_t tmem_base;
@@ -115,6 +115,12 @@ __device__ __forceinline__ void chunk_stats(const float (&v)[32], bool valid, in
   if ((lane & ((1 << (5 - LOG)) - 1)) == 0) dst[lane >> (5 - LOG)] = a[0];
 }
 
+__device__ __forceinline__ void tma_prefetch_4d(const CUtensorMap* m, int32_t c, int32_t w, int32_t h, int32_t n) {
+  asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global.tile [%0, {%1, %2, %3, %4}];" ::"l"(reinterpret_cast<uint64_t>(m)), "r"(c), "r"(w),
+               "r"(h), "r"(n)
+               : "memory");
+}
+
 // CB = C_in / 64 channel blocks
 template <int CB>
 __global__ void __launch_bounds__(THREADS, 1)
@@ -142,7 +148,8 @@ conv3x3_tc2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < A_STAGES; ++s) { tc::mbar_init(&sh->a_full[s], 1); tc::mbar_init(&sh->a_empty[s], 1); }
-    tc::mbar_init(&sh->b_full, 1);
+    tc::mbar_init(&sh->b_full[0], 1);
+    tc::mbar_init(&sh->b_full[1], 1);
     for (int b = 0; b < 2; ++b) { tc::mbar_init(&sh->tfull[b], 1); tc::mbar_init(&sh->tempty[b], 2 * EPI_WARPS); }
     sh->abort_flag = 0;
     tc::fence_barrier_init();
@@ -159,17 +166,30 @@ conv3x3_tc2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
   if (warp == 0) {
     // ------------------------------------------------------------ producer
     if (lane == 0) {
-      // weights: this CTA's C_out half, every K block, once
-      const uint32_t bfull_leader = tc::map_to_cta(tc::smem_u32(&sh->b_full), 0);
-      if (leader) tc::mbar_expect_tx(&sh->b_full, 2u * (uint32_t)b_bytes);
-      for (int kb = 0; kb < 9 * CB; ++kb)
-        tc::tma_load_2d_pair(b_tiles + (size_t)kb * b_block_bytes, &tmW, bfull_leader, kb * 64, (int)rank * b_rows);
+      // weights: this CTA's C_out half, every K block, once; channel block by channel block, in the
+      // order the MMAs consume them (K block index = tap * CB + cb)
+      for (int cb = 0; cb < CB; ++cb) {
+        const uint32_t bfull_leader = tc::map_to_cta(tc::smem_u32(&sh->b_full[cb]), 0);
+        if (leader) tc::mbar_expect_tx(&sh->b_full[cb], 2u * 9u * (uint32_t)b_block_bytes);
+        for (int tap = 0; tap < 9; ++tap) {
+          const int kb = tap * CB + cb;
+          tc::tma_load_2d_pair(b_tiles + (size_t)kb * b_block_bytes, &tmW, bfull_leader, kb * 64, (int)rank * b_rows);
+        }
+      }
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
       for (int t = cluster_id; t < total_tiles && ok; t += num_clusters) {
         const int n = t / quads, hq = t - n * quads;
         const int h0 = hq * 2 * TILE_ROWS + (int)rank * TILE_ROWS;   // first output row of this CTA
+        {
+          // pull the patches of this CTA's next tile towards L2 a whole tile before they are asked for
+          const int tn = t + num_clusters;
+          if (tn < total_tiles) {
+            const int nn = tn / quads, hn = (tn - nn * quads) * 2 * TILE_ROWS + (int)rank * TILE_ROWS;
+            for (int cb = 0; cb < CB; ++cb) tma_prefetch_4d(&tmX, cb * 64, -1, hn - 1, nn);
+          }
+        }
         for (int cb = 0; cb < CB; ++cb) {
           ok = tc::mbar_wait(&sh->a_empty[stage], phase ^ 1, abort_flag, status, tc::WAIT_SMEM_EMPTY);
           if (!ok) break;
@@ -190,8 +210,7 @@ conv3x3_tc2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
       const uint32_t b_step = (uint32_t)b_block_bytes >> 4;
       int stage = 0;
       uint32_t phase = 0;
-      bool ok = tc::mbar_wait(&sh->b_full, 0, abort_flag, status, tc::WAIT_SMEM_FULL);
-      MK_TR(90);                                 // weights resident
+      bool ok = true;
       int it = 0;
       for (int t = cluster_id; t < total_tiles && ok; t += num_clusters, ++it) {
         const int acc = it & 1;
@@ -202,6 +221,10 @@ conv3x3_tc2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
         uint32_t accumulate = 0;
 #pragma unroll
         for (int cb = 0; cb < CB; ++cb) {
+          if (it == 0) {
+            ok = tc::mbar_wait(&sh->b_full[cb], 0, abort_flag, status, tc::WAIT_SMEM_FULL);
+            if (!ok) break;
+          }
           ok = tc::mbar_wait(&sh->a_full[stage], phase, abort_flag, status, tc::WAIT_SMEM_FULL);
           if (!ok) break;
           tc::tc_fence_after();

@@ -81,8 +81,20 @@ static cudaError_t gemm_simt_dispatch(const void* a, const void* w, bool wt, voi
   return cudaGetLastError();
 }
 
+template <typename T>
+static cudaError_t linear_rownorm_dispatch(const void* a, const void* w, bool wt, void* y, int64_t m, int64_t n, int64_t k,
+                                           const EpiProgram& p, int mode, const void* g, const void* b, float eps,
+                                           cudaStream_t s);
+
 cudaError_t launch_gemm_simt(int dtype, int out_dtype, const void* a, const void* w, bool w_transposed, void* y, int64_t m, int64_t n,
                              int64_t k, bool swiglu, const EpiProgram& p, cudaStream_t s) {
+  // A problem too small to fill the machine with 64 x 64 tiles runs faster row by row with K split inside
+  // the CTA (the small-shape kernel below without its norm).
+  if (!swiglu && dtype == out_dtype && m * n <= 64 * 1024 && n <= 1024 && k <= 8192) {
+    cudaError_t e = dtype == DT_F32 ? linear_rownorm_dispatch<float>(a, w, w_transposed, y, m, n, k, p, -1, nullptr, nullptr, 0.0f, s)
+                                    : linear_rownorm_dispatch<__nv_bfloat16>(a, w, w_transposed, y, m, n, k, p, -1, nullptr, nullptr, 0.0f, s);
+    if (e != cudaErrorInvalidValue) return e;
+  }
   if (dtype == DT_F32) return out_dtype == DT_F32 ? gemm_simt_dispatch<float, float>(a, w, w_transposed, y, m, n, k, swiglu, p, s) : cudaErrorInvalidValue;
   return out_dtype == DT_F32 ? gemm_simt_dispatch<__nv_bfloat16, float>(a, w, w_transposed, y, m, n, k, swiglu, p, s)
                              : gemm_simt_dispatch<__nv_bfloat16, __nv_bfloat16>(a, w, w_transposed, y, m, n, k, swiglu, p, s);
@@ -117,7 +129,34 @@ __global__ void __launch_bounds__(LR_THREADS) linear_rownorm_kernel(const T* __r
   const int kper = (K + KS - 1) / KS;
   const int kb = ks * kper, ke = min(K, kb + kper);
   float acc[LR_ROWS][LR_MAXC] = {};
-  if (ks < KS) {
+  constexpr int VE = Elem<T>::VEC;
+  const bool vec_k = wt && K % VE == 0 && kper % VE == 0;
+  if (ks < KS && vec_k) {
+    // W stored [N, K]: a column's K-slice is contiguous, so every thread streams 16-byte vectors of its own
+    // columns (a scalar load here would fetch a whole sector per lane for one element)
+#pragma unroll 4
+    for (int k = kb; k < ke; k += VE) {
+      float wv[LR_MAXC][VE];
+#pragma unroll
+      for (int j = 0; j < LR_MAXC; ++j) {
+        const int c = ct + j * NT;
+        if (c < N) {
+          ld_vec(w + (int64_t)c * K + k, wv[j]);
+        } else {
+#pragma unroll
+          for (int e = 0; e < VE; ++e) wv[j][e] = 0.0f;
+        }
+      }
+#pragma unroll
+      for (int r = 0; r < LR_ROWS; ++r)
+#pragma unroll
+        for (int e = 0; e < VE; ++e) {
+          const float xv = xs[r * K + k + e];
+#pragma unroll
+          for (int j = 0; j < LR_MAXC; ++j) acc[r][j] = fmaf(xv, wv[j][e], acc[r][j]);
+        }
+    }
+  } else if (ks < KS) {
 #pragma unroll 8
     for (int k = kb; k < ke; ++k) {
       float wv[LR_MAXC];
@@ -139,6 +178,15 @@ __global__ void __launch_bounds__(LR_THREADS) linear_rownorm_kernel(const T* __r
         if (c < N) part[(ks * LR_ROWS + r) * N + c] = acc[r][j];
       }
   }
+  if (ks < KS && vec_k) {
+#pragma unroll
+    for (int r = 0; r < LR_ROWS; ++r)
+#pragma unroll
+      for (int j = 0; j < LR_MAXC; ++j) {
+        const int c = ct + j * NT;
+        if (c < N) part[(ks * LR_ROWS + r) * N + c] = acc[r][j];
+      }
+  }
   __syncthreads();
   // sum the K-slices in a fixed order, apply the elementwise tail; result overwrites slice 0
   for (int i = threadIdx.x; i < LR_ROWS * N; i += LR_THREADS) {
@@ -148,6 +196,14 @@ __global__ void __launch_bounds__(LR_THREADS) linear_rownorm_kernel(const T* __r
     part[r * N + c] = epi_apply(p, v, m0 + r, c, N);
   }
   __syncthreads();
+  if (mode < 0) {
+    // no row norm: the fused linear + elementwise tail of a small problem
+    for (int i = threadIdx.x; i < LR_ROWS * N; i += LR_THREADS) {
+      const int r = i / N, c = i - r * N;
+      if (m0 + r < M) Elem<T>::st(y + (int64_t)(m0 + r) * N + c, part[r * N + c]);
+    }
+    return;
+  }
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (warp < LR_ROWS && m0 + warp < M) {
     const float* row = part + warp * N;
@@ -176,8 +232,10 @@ static cudaError_t linear_rownorm_dispatch(const void* a, const void* w, bool wt
                                            const EpiProgram& p, int mode, const void* g, const void* b, float eps,
                                            cudaStream_t s) {
   if (m == 0) return cudaSuccess;
+  // fewest column threads that cover N with LR_MAXC columns each: the rest of the CTA splits K, which
+  // shortens every thread's chain of loads
   int NT = 32;
-  while (NT < n && NT < 256) NT *= 2;
+  while ((int64_t)NT * LR_MAXC < n && NT < 256) NT *= 2;
   if ((int64_t)NT * LR_MAXC < n) return cudaErrorInvalidValue;
   const int KS = LR_THREADS / NT;
   const size_t smem = sizeof(float) * ((size_t)LR_ROWS * k + (size_t)KS * LR_ROWS * n);
