@@ -42,6 +42,19 @@ constexpr int THREADS = 64 + 32 * EPI_WARPS;
 constexpr int STG_BYTES = 32 * 64;        // transpose buffer per epilogue warp: 32 rows x 64 bytes, XOR-swizzled
 constexpr int BIAS_BYTES = 512;           // one copy of the bias (C_out <= 256 bf16) per CTA
 
+// The timeline of -DMK_TRACE builds lives in global memory here: this kernel leaves no shared memory for it.
+#ifdef MK_TRACE
+__device__ unsigned long long conv_tr[96];
+#define CTR_INIT do { if (blockIdx.x == 0 && threadIdx.x == 0) { for (int i_ = 0; i_ < 96; ++i_) conv_tr[i_] = 0; conv_tr[0] = tc::gtime(); } } while (0)
+#define CTR(slot) do { if (blockIdx.x == 0 && (slot) < 96) conv_tr[slot] = tc::gtime(); } while (0)
+#define CTR_PRINT do { __threadfence(); __syncthreads(); if (blockIdx.x == 0 && threadIdx.x == 0) { printf("conv end=%llu :", tc::gtime() - conv_tr[0]); \
+    for (int i_ = 1; i_ < 96; ++i_) if (conv_tr[i_]) printf(" [%d]%llu", i_, conv_tr[i_] - conv_tr[0]); printf("\n"); } } while (0)
+#else
+#define CTR_INIT do {} while (0)
+#define CTR(slot) do {} while (0)
+#define CTR_PRINT do {} while (0)
+#endif
+
 struct Shared {
   uint64_t a_full[A_STAGES];
   uint64_t a_empty[A_STAGES];
@@ -115,6 +128,27 @@ __device__ __forceinline__ void chunk_stats(const float (&v)[32], bool valid, in
   if ((lane & ((1 << (5 - LOG)) - 1)) == 0) dst[lane >> (5 - LOG)] = a[0];
 }
 
+// Four MMAs of one tap (K = 64 channels in steps of 16): the two descriptors advance by 32 bytes (2 in
+// the address field) per step, done on the low words inside the block, so the issuing thread spends three
+// instructions per 64-cycle MMA.  acc0 = 0 makes the first MMA overwrite the accumulator.
+__device__ __forceinline__ void umma_ss_pair_x4(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc0) {
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t.reg .b32 alo, ahi, blo, bhi;\n\t.reg .b64 da, db;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "setp.eq.b32 q, %3, %3;\n\t"
+      "mov.b64 {alo, ahi}, %1;\n\t"
+      "mov.b64 {blo, bhi}, %2;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t"
+      "add.u32 alo, alo, 2;\n\tadd.u32 blo, blo, 2;\n\tmov.b64 da, {alo, ahi};\n\tmov.b64 db, {blo, bhi};\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %3, q;\n\t"
+      "add.u32 alo, alo, 2;\n\tadd.u32 blo, blo, 2;\n\tmov.b64 da, {alo, ahi};\n\tmov.b64 db, {blo, bhi};\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %3, q;\n\t"
+      "add.u32 alo, alo, 2;\n\tadd.u32 blo, blo, 2;\n\tmov.b64 da, {alo, ahi};\n\tmov.b64 db, {blo, bhi};\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %3, q;\n\t}" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc0)
+      : "memory");
+}
+
 __device__ __forceinline__ void tma_prefetch_4d(const CUtensorMap* m, int32_t c, int32_t w, int32_t h, int32_t n) {
   asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global.tile [%0, {%1, %2, %3, %4}];" ::"l"(reinterpret_cast<uint64_t>(m)), "r"(c), "r"(w),
                "r"(h), "r"(n)
@@ -143,8 +177,7 @@ conv3x3_tc2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
   const int quads = (H + 2 * TILE_ROWS - 1) / (2 * TILE_ROWS);   // pair-tiles per image
   const int total_tiles = NB * quads;
   volatile int* abort_flag = &sh->abort_flag;
-  MK_TR_DECL
-  MK_TR_INIT;
+  CTR_INIT;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < A_STAGES; ++s) { tc::mbar_init(&sh->a_full[s], 1); tc::mbar_init(&sh->a_empty[s], 1); }
@@ -228,25 +261,22 @@ conv3x3_tc2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
           ok = tc::mbar_wait(&sh->a_full[stage], phase, abort_flag, status, tc::WAIT_SMEM_FULL);
           if (!ok) break;
           tc::tc_fence_after();
-          MK_TR(1 + it * 8 + cb);                // MMA: patch cb landed
-          const uint32_t patch_lo = patch_lo0 + (uint32_t)stage * (PATCH_BYTES >> 4);
-          uint32_t b_lo = b_lo0 + (uint32_t)cb * b_step;
+          CTR(1 + it * 8 + cb);                // MMA: patch cb landed
+          const uint64_t patch_desc = ((uint64_t)tc::kDescHiSw128 << 32) | (patch_lo0 + (uint32_t)stage * (PATCH_BYTES >> 4));
+          uint64_t b_desc = ((uint64_t)tc::kDescHiSw128 << 32) | (b_lo0 + (uint32_t)cb * b_step);
 #pragma unroll
           for (int tap = 0; tap < 9; ++tap) {
             const int kh = tap / 3, kw = tap % 3;                                   // compile-time after unrolling
-            const uint32_t a_lo = patch_lo + (uint32_t)(((kh * PITCH + kw) * 128) >> 4);
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-              tc::umma_ss_pair_lohi(d_tmem, a_lo + 2 * k, b_lo + 2 * k, idesc, accumulate);
-              accumulate = 1;
-            }
-            b_lo += (uint32_t)CB * b_step;
+            umma_ss_pair_x4(d_tmem, patch_desc + (uint64_t)(((kh * PITCH + kw) * 128) >> 4), b_desc, idesc, accumulate);
+            accumulate = 1;
+            b_desc += (uint64_t)((uint32_t)CB * b_step);
           }
+          CTR(6 + it * 8 + cb);                  // MMA: channel block issued
           tc::umma_commit_pair(&sh->a_empty[stage]);
           if (++stage == A_STAGES) { stage = 0; phase ^= 1; }
         }
         if (!ok) break;
-        MK_TR(3 + it * 8);                       // MMA: tile issued
+        CTR(3 + it * 8);                       // MMA: tile issued
         tc::umma_commit_pair(&sh->tfull[acc]);
       }
     }
@@ -284,7 +314,7 @@ conv3x3_tc2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
       ok = tc::mbar_wait(&sh->tfull[acc], (it >> 1) & 1, abort_flag, status, tc::WAIT_TMEM_FULL);
       ok = __all_sync(0xffffffffu, ok ? 1 : 0) != 0;
       if (!ok) break;
-      if (threadIdx.x == 64) MK_TR(4 + it * 8);  // epilogue: accumulator ready
+      if (threadIdx.x == 64) CTR(4 + it * 8);  // epilogue: accumulator ready
       tc::tc_fence_after();
       const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + acc * 256;
       float* stat_dst = stats ? stats + (((int64_t)n * stat_slots + (hq * 2 + (int)rank) * 4 + q) * groups) * 2 : nullptr;
@@ -318,12 +348,12 @@ conv3x3_tc2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
       }
       tc::tc_fence_before();
       __syncwarp();
-      if (threadIdx.x == 64) MK_TR(5 + it * 8);  // epilogue: tile stored
+      if (threadIdx.x == 64) CTR(5 + it * 8);  // epilogue: tile stored
       if (lane == 0) tc::mbar_arrive_cluster(tc::map_to_cta(tc::smem_u32(&sh->tempty[acc]), 0));
     }
   }
 
-  MK_TR_PRINT("conv");
+  CTR_PRINT;
   if (*abort_flag) {
     const long long t0 = clock64();
     while (clock64() - t0 < 4000000LL) {}
