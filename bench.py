@@ -38,9 +38,19 @@ NCU_TRAFFIC_BYTES = {"c2": 105.7e6}   # profiles/gemm_tc2_c2.md
 DEFAULT_STEPS = {"c1": 2000, "c2": 1000, "c3": 1000, "c4": 200, "c5": 50}
 
 
-def full_workload(name, seed=0):
+def full_workload(name, seed=0, batch=None, only_ops=None):
+    """The named workload at its full size.  `batch` (a smaller leading batch dimension) and `only_ops` (the
+    first N operators alone) cut out small cases of the same kernels for profiler captures."""
     import workloads as W
-    return W.generate.WORKLOADS[name](seed)
+    kw = {}
+    if batch is not None:
+        kw = {"c1": {"M": batch}, "c2": {"M": batch}, "c3": {"NB": batch}, "c4": {"B": batch}, "c5": {"B": batch}}[name]
+    w = W.generate.WORKLOADS[name](seed, **kw)
+    if only_ops is not None:
+        w.ops = w.ops[:only_ops]
+        w.partitions = {"fused": [0], "per_op": list(range(len(w.ops)))}
+        w.flops = None          # recomputed from the operators once the module exists
+    return w
 
 
 def peaks():
@@ -265,7 +275,7 @@ def run_ours(args):
     from paper_2607_20501_b200.runner import DeviceWorkload
 
     name = args.workload
-    w = full_workload(name)
+    w = full_workload(name, batch=args.batch, only_ops=args.only_ops)
     ctx = Context(local)
     # rotation: enough independent copies that a pass over all of them exceeds L2 (126 MB) twice over
     per_copy = sum(t.nbytes() for t in w.inputs.values()) + sum(t.nbytes() for t in w.params.values())
@@ -277,6 +287,10 @@ def run_ours(args):
             dw.module.set_decomposition(w.partitions[part])
         dw.ensure_workspace()
     impls = [sets[0].module.bound_impl(s) for s in range(sets[0].module.n_sub())]
+    if w.flops is None:
+        work = submodule_work(w, sets[0].module)
+        w.flops = sum(f for f, _ in work)
+        w.min_bytes = sum(b for _, b in work)
     stream = torch.cuda.current_stream()
 
     def barrier():
@@ -427,7 +441,8 @@ def run_ours(args):
                        "l2": (f"rotation over {rot} independent input/output sets ({rot * per_copy / 1e6:.0f} MB > L2)" if rot * per_copy > 126e6 else
                               f"rotation over {rot} independent input/output sets ({rot * per_copy / 1e6:.1f} MB in all: the whole problem is "
                               "smaller than L2 and bound by launch latency, so L2 residency is part of the measurement)"),
-                       "shapes": {k: list(t.shape) for k, t in w.inputs.items()}},
+                       "shapes": {k: list(t.shape) for k, t in w.inputs.items()},
+                       **({"cut": {"batch": args.batch, "only_ops": args.only_ops}} if (args.batch or args.only_ops) else {})},
             "roofline": roofline_of(name, launches_per_step, dominant, achieved, peak, pk, kernel_ms, t_roof_ms, ms_per_step, step_ms[0]),
             "e2e": {"value": world * w.flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
@@ -457,6 +472,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2", choices=["c1", "c2", "c3", "c4", "c5"])
     ap.add_argument("--decomposition", default=None)
+    ap.add_argument("--batch", type=int, default=None, help="smaller leading batch dimension (profiler captures)")
+    ap.add_argument("--only-ops", type=int, default=None, help="run the first N operators alone (profiler captures)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle leg")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     args = ap.parse_args()
