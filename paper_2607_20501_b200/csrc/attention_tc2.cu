@@ -46,10 +46,9 @@ struct Shared {
   uint64_t q_full[2], q_free[2];
   uint64_t k_full[KV_STAGES], k_empty[KV_STAGES];
   uint64_t v_full[KV_STAGES], v_empty[KV_STAGES];
-  uint64_t s_full[2], p_ready[2], o_final[2], l_ready[2], o_free[2];
+  uint64_t s_lo_full[2], s_hi_full[2], b_free[2], p_ready[2], o_final[2], l_ready[2], o_free[2];
   uint32_t tmem_base;
   int abort_flag;
-  int pipe_lock;   // held by the stream whose run of MMAs is being issued
   float l[2][128];
 };
 constexpr size_t ATTN2_SMEM = (size_t)TILE_BYTES * (2 + 2 * KV_STAGES) + 4 * EPI_WARP_BYTES + 1024 + ((sizeof(Shared) + 255) / 256) * 256;
@@ -107,26 +106,6 @@ struct Ctx {
   unsigned int* status;
   __device__ __forceinline__ bool wait(uint64_t* bar, uint32_t parity, unsigned code) const {
     return tc::mbar_wait(bar, parity, abort_flag, status, code);
-  }
-  // The two issuing threads take turns: a run of MMAs of one stream is issued whole, so that stream's next
-  // S is ready half a step before the other's and the two softmaxes stay out of phase (one stream's
-  // exponentials overlap the other's MMAs).  Left alone, the runs interleave and both streams end up
-  // doing softmax at the same time and MMAs at the same time.  The holder only issues MMAs, it never waits.
-  __device__ __forceinline__ bool lock_pipe() const {
-    const long long t0 = clock64();
-    while (atomicCAS(&sh->pipe_lock, 0, 1) != 0) {
-      if (*abort_flag) return false;
-      if (clock64() - t0 > tc::kWaitLimitCycles) {
-        *abort_flag = 1;
-        if (status) atomicExch(status, (unsigned)tc::WAIT_ATTN);
-        return false;
-      }
-    }
-    return true;
-  }
-  __device__ __forceinline__ void unlock_pipe() const {
-    __threadfence_block();
-    atomicExch(&sh->pipe_lock, 0);
   }
   // the same for a whole warp (its next instruction is warp-collective)
   __device__ __forceinline__ bool wait_warp(uint64_t* bar, uint32_t parity, unsigned code) const {
@@ -254,7 +233,7 @@ __device__ __forceinline__ void role_loader(const Ctx& cx, const CUtensorMap* tm
 __device__ __forceinline__ void role_mma(const Ctx& cx, uint32_t tmem_base, int t, uint8_t* q_tiles, uint8_t* k_tiles, uint8_t* v_tiles, int B,
                                          int H, int S) {
   Shared* sh = cx.sh;
-  constexpr uint32_t idesc_qk = tc::idesc_bf16_f32(BQ, BKV, 0, 0);   // A, B K-major
+  constexpr uint32_t idesc_qk64 = tc::idesc_bf16_f32(BQ, 64, 0, 0);  // A, B K-major, half a key tile
   constexpr uint32_t idesc_pv = tc::idesc_bf16_f32(BQ, HD, 0, 1);    // B (= V) MN-major
   // V, MN-major with 128-byte swizzle: 64 head-dim elements are contiguous (one 128-byte row per key),
   // 8-key groups are 1024 B apart (SBO), the second 64 head-dim elements sit SUB_BYTES on (LBO)
@@ -291,15 +270,23 @@ __device__ __forceinline__ void role_mma(const Ctx& cx, uint32_t tmem_base, int 
       }
     }
   };
-  // S_t = Q_t K^T for tile b (if do_qk), preceded by O_t (+)= P_t V for tile a (if do_pv).  The two are issued
-  // back to back: everything that is ready early is waited for first, P (which arrives last) is polled
-  // for, and from then on the thread only issues the sixteen MMAs and the commit that publishes S.
+  // One step: O_t (+)= P_t V for tile a (if do_pv) and S_t = Q_t K^T for the following tile b (if do_qk), S in two
+  // halves of 64 keys:
+  //   S_lo(b) (keys 0..63)   -> columns [64, 128) of the stream's S region ("region B"), as soon as the
+  //                             softmax has read S_lo(a) out of it: while softmax(a) is still busy with its second half;
+  //   P V(a), then S_hi(b)   -> columns [0, 64) ("region A", which also holds P(a)), once P(a) is there.
+  // So when softmax(a) ends, half of the next S is already waiting for it, and the other half arrives while it
+  // works on the first: the chain softmax -> P V -> Q K^T -> softmax no longer has the MMAs in it.
+  // Operands are precomputed before the waits.  The two issuing threads do not take turns: a lock around each
+  // run of MMAs (tried) makes the short early Q K^T wait for the other stream's whole run.
+  bool first_qk = true;
+  uint32_t par_bfree = 0;
   auto issue = [&](const Pos& a, bool do_pv, const Pos& b, bool do_qk) -> bool {
     const uint32_t ga = a.g + (uint32_t)a.j, gb = b.g + (uint32_t)b.j;
     const int sta = ga % KV_STAGES, stb = gb % KV_STAGES;
     uint32_t pa[8];
     uint64_t vb[8], qa[8], kb[8];
-    bool fused = false;
+    bool lo_done = false, hi_done = false;
     if (do_pv) {
       const uint32_t v_lo = v_lo0 + (uint32_t)sta * (TILE_BYTES >> 4);
 #pragma unroll
@@ -310,6 +297,17 @@ __device__ __forceinline__ void role_mma(const Ctx& cx, uint32_t tmem_base, int 
         pin(vb[k]);
       }
     }
+    auto issue_lo = [&]() {
+      umma_ss_x8(s_tmem + 64, qa, kb, idesc_qk64);
+      tc::umma_commit(&sh->s_lo_full[t]);
+    };
+    auto issue_hi = [&]() {
+      uint64_t kh[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) kh[k] = kb[k] + (uint64_t)((64 * 128) >> 4);   // key rows 64..127 of the K tile
+      umma_ss_x8(s_tmem, qa, kh, idesc_qk64);
+      tc::umma_commit(&sh->s_hi_full[t]);
+    };
     if (do_qk) {
       const uint32_t k_lo = k_lo0 + (uint32_t)stb * (TILE_BYTES >> 4);
 #pragma unroll
@@ -320,9 +318,27 @@ __device__ __forceinline__ void role_mma(const Ctx& cx, uint32_t tmem_base, int 
         pin(qa[k]);
         pin(kb[k]);
       }
-      // Fuse only if the operands of the next S are already there: waiting for them here, before this
-      // tile's P V is issued, could wait for a load that is queued behind a slot this very P V releases.
-      fused = (b.j != 0 || tc::mbar_test_wait(&sh->q_full[t], par_qfull)) && tc::mbar_test_wait(&sh->k_full[stb], (gb / KV_STAGES) & 1);
+      if (!first_qk) {
+        // region B has been read (the softmax signals it half-way through tile a)
+        if (!cx.wait(&sh->b_free[t], par_bfree, tc::WAIT_TMEM_EMPTY)) return false;
+        par_bfree ^= 1u;
+      }
+      first_qk = false;
+      // Early only if Q and K are already there: waiting for them here, before this tile's P V is issued, could
+      // wait for a load that is queued behind a slot this very P V releases.
+      bool ready = true;
+      if (do_pv) {
+        ready = (b.j != 0 || tc::mbar_test_wait(&sh->q_full[t], par_qfull)) && tc::mbar_test_wait(&sh->k_full[stb], (gb / KV_STAGES) & 1);
+      } else {
+        if (b.j == 0 && !cx.wait(&sh->q_full[t], par_qfull, tc::WAIT_SMEM_FULL)) return false;
+        if (!cx.wait(&sh->k_full[stb], (gb / KV_STAGES) & 1, tc::WAIT_SMEM_FULL)) return false;
+      }
+      if (ready) {
+        tc::tc_fence_after();
+        issue_lo();
+        if (!do_pv) { issue_hi(); hi_done = true; }
+        lo_done = true;
+      }
     }
     if (do_pv) {
       if (a.j == 0) {
@@ -335,27 +351,20 @@ __device__ __forceinline__ void role_mma(const Ctx& cx, uint32_t tmem_base, int 
       par_pv ^= 1u;
       TR2(a.g == 0 && a.j < 11, (t ? 8 : 4) + a.j * 8);
       tc::tc_fence_after();
-      if (!cx.lock_pipe()) return false;
       umma_ts_x8(o_tmem, pa, vb, idesc_pv, a.j > 0 ? 1u : 0u);
-      if (fused) {
-        umma_ss_x8(s_tmem, qa, kb, idesc_qk);
-        tc::umma_commit(&sh->s_full[t]);
-      }
-      cx.unlock_pipe();
+      if (do_qk && lo_done) { issue_hi(); hi_done = true; }
       // a K/V slot is released by two arrivals: one per stream, or both from the only stream that reads it
       if (a.j == a.nt - 1) tc::umma_commit(&sh->o_final[t]);
       tc::umma_commit(&sh->v_empty[sta]);
       if (!(a.j < a.n0 && a.j < a.n1)) tc::umma_commit(&sh->v_empty[sta]);
     }
     if (do_qk) {
-      if (!fused || !do_pv) {
+      if (!hi_done) {
         if (b.j == 0 && !cx.wait(&sh->q_full[t], par_qfull, tc::WAIT_SMEM_FULL)) return false;
         if (!cx.wait(&sh->k_full[stb], (gb / KV_STAGES) & 1, tc::WAIT_SMEM_FULL)) return false;
         tc::tc_fence_after();
-        if (!cx.lock_pipe()) return false;
-        umma_ss_x8(s_tmem, qa, kb, idesc_qk);
-        tc::umma_commit(&sh->s_full[t]);
-        cx.unlock_pipe();
+        if (!lo_done) issue_lo();
+        issue_hi();
       }
       if (b.j == 0) par_qfull ^= 1u;
       tc::umma_commit(&sh->k_empty[stb]);
@@ -382,22 +391,24 @@ __device__ __forceinline__ void role_mma(const Ctx& cx, uint32_t tmem_base, int 
 // ------------------------------------------------------------------------------------------ softmax
 // One thread per query row of stream T.  m is the reference maximum in log2 units (scores times
 // scale * log2 e): p = exp2(s * scale*log2e - m).  Any m gives the same O / l as long as nothing
-// overflows, so m is NOT kept equal to the running row maximum:
-//   fast path (every tile but an item's first and its diagonal one): a single pass over S with the m
-//     the row already has; all of P stays in registers until the row sum has been checked;
-//   full path (first tile, diagonal tile, or a row sum above 2^60 somewhere in the warp): row maximum,
-//     m raised to it, the running O of this row (in TMEM) and l rescaled by exp2(m_old - m_new) by
-//     this very thread, then the probabilities.  S is still intact when the fast path gives up:
-//     it has stored nothing yet.
-// The previous P V of this stream is complete whenever S_j is visible (the tensor pipe runs in order),
-// so touching O here is safe, and the next P V is not issued before this thread's p_ready arrival.
+// overflows, so m is NOT kept equal to the running row maximum; it is raised (and the running O in TMEM,
+// l, and whatever of this tile's P is already computed, rescaled by exp2(m_old - m_new)) only
+//   * on an item's first and diagonal tiles, after a pre-pass that also writes -inf over the masked
+//     scores in TMEM (key > query), so that the main pass needs no mask; and
+//   * when a half-row sum leaves the safe range (2^60) - then from that half's own maximum.
+// S arrives in two halves: keys 0..63 in columns [64, 128) of the stream's S region (B), keys 64..127 in
+// columns [0, 64) (A).  As soon as the first half has been turned into probabilities (kept in registers),
+// region B is handed back (b_free) and the tensor pipe computes the next tile's first half into it while this
+// thread works on the second half.  P (packed bf16, 64 columns) goes over region A at the end.
+// O may be touched only after S_hi of the same tile is visible: Q K^T_hi(j) is issued after P V(j-1), the
+// pipe runs in order, and the next P V is not issued before this thread's p_ready arrival.
 __device__ __forceinline__ void role_softmax(const Ctx& cx, uint32_t tmem_base, int T, int warp, int lane, int B, int H, int S,
                                              float scale_log2) {
   Shared* sh = cx.sh;
   const int q = warp & 3;
   const int row = q * 32 + lane;
   const uint32_t lane_off = (uint32_t)(q * 32) << 16;
-  const uint32_t s_addr = tmem_base + (uint32_t)T * 128 + lane_off;
+  const uint32_t s_addr = tmem_base + (uint32_t)T * 128 + lane_off;     // region A; region B = s_addr + 64
   const uint32_t o_addr = tmem_base + 256 + (uint32_t)T * 128 + lane_off;
   ItemIter iter;
   iter.init(S, B, H);
@@ -409,60 +420,16 @@ __device__ __forceinline__ void role_softmax(const Ctx& cx, uint32_t tmem_base, 
     float m = -INFINITY, l = 0.0f;
 #pragma unroll 1
     for (int j = 0; j < nt; ++j) {
-      {
-        const bool ok = tc::mbar_wait_spin(&sh->s_full[T], n_tiles & 1, cx.abort_flag, cx.status, tc::WAIT_TMEM_FULL);
-        if (!__all_sync(0xffffffffu, ok ? 1 : 0)) return;
-      }
+      const uint32_t par = n_tiles & 1;
       ++n_tiles;
-      tc::tc_fence_after();
-      TR2(T == 0 && threadIdx.x == 0 && n_items == 0 && j < 11, 1 + j * 8);
-      TR2(T == 1 && threadIdx.x == 128 && n_items == 0 && j < 11, 5 + j * 8);
-      bool full = j == 0 || j == nt - 1;
-      if (!full) {
-        const float neg_m = -m;
-        float sum4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-        uint32_t pk[64];
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          uint32_t r[32];
-          tc::tmem_ld32(s_addr + c * 32, r);
-          tc::tmem_ld_wait();
-#pragma unroll
-          for (int i = 0; i < 32; i += 2) {
-            const float p0 = tc::ex2_fast(fmaf(__uint_as_float(r[i]), scale_log2, neg_m));
-            const float p1 = tc::ex2_fast(fmaf(__uint_as_float(r[i + 1]), scale_log2, neg_m));
-            sum4[(i >> 1) & 3] += p0 + p1;
-            pk[c * 16 + (i >> 1)] = pack_bf16x2(p0, p1);
-          }
-        }
-        const float sum = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
-        full = __any_sync(0xffffffffu, !(sum < 1.152921504606847e18f));   // 2^60; also true for inf / NaN
-        if (!full) {
-#pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            uint32_t part[16];
-#pragma unroll
-            for (int i = 0; i < 16; ++i) part[i] = pk[c * 16 + i];
-            tmem_st16(s_addr + c * 16, part);
-          }
-          l += sum;
-        }
-      }
-      if (full) {
-        // last visible key of this row inside the tile: the diagonal tile masks key (column) > query (row)
-        const int last = (j == nt - 1) ? row : 127;
-        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
-          uint32_t r[32];
-          tc::tmem_ld32(s_addr + c * 32, r);
-          tc::tmem_ld_wait();
-          const int lim = last - c * 32;
-#pragma unroll
-          for (int i = 0; i < 32; ++i)
-            if (i <= lim) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(r[i]));
-        }
-        const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * scale_log2;
+      auto wait_half = [&](uint64_t* bar) -> bool {
+        const bool ok = tc::mbar_wait_spin(bar, par, cx.abort_flag, cx.status, tc::WAIT_TMEM_FULL);
+        const bool all = __all_sync(0xffffffffu, ok ? 1 : 0) != 0;
+        if (all) tc::tc_fence_after();
+        return all;
+      };
+      // m := max(m, mx); the running O (not on an item's first tile) and l follow
+      auto raise = [&](float mx) -> float {
         float alpha = 1.0f;
         if (mx > m) {
           alpha = tc::ex2_fast(m - mx);    // 0 on the first tile (m = -inf)
@@ -478,30 +445,124 @@ __device__ __forceinline__ void role_softmax(const Ctx& cx, uint32_t tmem_base, 
             for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
             tc::tmem_st32(o_addr + c * 32, r);
           }
+          tc::tmem_st_wait();
         }
         l *= alpha;
-        const float neg_m = -m;
-        float sum4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+        return alpha;
+      };
+      // maximum (log2 units) of 64 scores starting at TMEM address `base`
+      auto half_max = [&](uint32_t base) -> float {
+        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll 1
+        for (int c = 0; c < 2; ++c) {
+          uint32_t r[32];
+          tc::tmem_ld32(base + c * 32, r);
+          tc::tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(r[i]));
+        }
+        return fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * scale_log2;
+      };
+
+      if (j == 0 || j == nt - 1) {
+        // first / diagonal tile: both halves, masked scores replaced by -inf in place, m raised to the row maximum
+        if (!wait_half(&sh->s_lo_full[T])) return;
+        if (!wait_half(&sh->s_hi_full[T])) return;
+        const int last = (j == nt - 1) ? row : 127;     // last visible key of this row inside the tile
+        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll 1
         for (int c = 0; c < 4; ++c) {
+          const uint32_t addr = s_addr + (c < 2 ? 64 + c * 32 : (c - 2) * 32);
           uint32_t r[32];
-          uint32_t pk[16];
-          tc::tmem_ld32(s_addr + c * 32, r);
+          tc::tmem_ld32(addr, r);
           tc::tmem_ld_wait();
           const int lim = last - c * 32;
+          // the write-back is a warp-collective instruction: decide it for the whole warp (some lane of this
+          // warp, whose rows are q * 32 .. q * 32 + 31, has a masked key in this chunk)
+          if (j == nt - 1 && q * 32 - c * 32 < 31) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (i > lim) r[i] = 0xff800000u;
+            tc::tmem_st32(addr, r);
+          }
+#pragma unroll
+          for (int i = 0; i < 32; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(r[i]));
+        }
+        tc::tmem_st_wait();
+        raise(fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * scale_log2);
+      }
+
+      uint32_t pk[64];
+      float sum_lo = 0.0f, sum_hi = 0.0f;
+      // ---- first half: keys 0..63 from region B
+      if (!wait_half(&sh->s_lo_full[T])) return;
+      TR2(T == 0 && threadIdx.x == 0 && n_items == 0 && j < 11, 1 + j * 8);
+      TR2(T == 1 && threadIdx.x == 128 && n_items == 0 && j < 11, 5 + j * 8);
+#pragma unroll 1
+      for (int attempt = 0; attempt < 2; ++attempt) {
+        const float neg_m = -m;
+        float sum4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          uint32_t r[32];
+          tc::tmem_ld32(s_addr + 64 + c * 32, r);
+          tc::tmem_ld_wait();
 #pragma unroll
           for (int i = 0; i < 32; i += 2) {
-            float p0 = tc::ex2_fast(fmaf(__uint_as_float(r[i]), scale_log2, neg_m));
-            float p1 = tc::ex2_fast(fmaf(__uint_as_float(r[i + 1]), scale_log2, neg_m));
-            if (i > lim) p0 = 0.0f;
-            if (i + 1 > lim) p1 = 0.0f;
+            const float p0 = tc::ex2_fast(fmaf(__uint_as_float(r[i]), scale_log2, neg_m));
+            const float p1 = tc::ex2_fast(fmaf(__uint_as_float(r[i + 1]), scale_log2, neg_m));
             sum4[(i >> 1) & 3] += p0 + p1;
-            pk[i >> 1] = pack_bf16x2(p0, p1);
+            pk[c * 16 + (i >> 1)] = pack_bf16x2(p0, p1);
           }
-          tmem_st16(s_addr + c * 16, pk);
         }
-        l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+        sum_lo = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+        if (attempt == 1 || !__any_sync(0xffffffffu, !(sum_lo < 1.152921504606847e18f))) break;   // 2^60; also inf / NaN
+        // out of range: raise m to this half's maximum (O is safe to touch once S_hi is visible), then once more
+        if (!wait_half(&sh->s_hi_full[T])) return;
+        raise(half_max(s_addr + 64));
       }
+      tc::tc_fence_before();
+      tc::mbar_arrive(&sh->b_free[T]);
+      TR2(T == 0 && threadIdx.x == 0 && n_items == 0 && j < 11, 2 + j * 8);
+      // ---- second half: keys 64..127 from region A
+      if (!wait_half(&sh->s_hi_full[T])) return;
+      TR2(T == 0 && threadIdx.x == 0 && n_items == 0 && j < 11, 6 + j * 8);
+#pragma unroll 1
+      for (int attempt = 0; attempt < 2; ++attempt) {
+        const float neg_m = -m;
+        float sum4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          uint32_t r[32];
+          tc::tmem_ld32(s_addr + c * 32, r);
+          tc::tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 32; i += 2) {
+            const float p0 = tc::ex2_fast(fmaf(__uint_as_float(r[i]), scale_log2, neg_m));
+            const float p1 = tc::ex2_fast(fmaf(__uint_as_float(r[i + 1]), scale_log2, neg_m));
+            sum4[(i >> 1) & 3] += p0 + p1;
+            pk[32 + c * 16 + (i >> 1)] = pack_bf16x2(p0, p1);
+          }
+        }
+        sum_hi = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+        if (attempt == 1 || !__any_sync(0xffffffffu, !(sum_hi < 1.152921504606847e18f))) break;
+        // out of range: raise m to this half's maximum; the first half's probabilities and sum follow
+        const float alpha = raise(half_max(s_addr));
+        sum_lo *= alpha;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const float a0 = __uint_as_float(pk[i] << 16) * alpha, a1 = __uint_as_float(pk[i] & 0xffff0000u) * alpha;
+          pk[i] = pack_bf16x2(a0, a1);
+        }
+      }
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t part[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) part[i] = pk[c * 16 + i];
+        tmem_st16(s_addr + c * 16, part);
+      }
+      l += sum_lo + sum_hi;
       tc::tmem_st_wait();
       tc::tc_fence_before();
       tc::mbar_arrive(&sh->p_ready[T]);
@@ -587,7 +648,8 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
   if (threadIdx.x == 0) {
     for (int t = 0; t < 2; ++t) {
       tc::mbar_init(&sh->q_full[t], 1); tc::mbar_init(&sh->q_free[t], 1);
-      tc::mbar_init(&sh->s_full[t], 1); tc::mbar_init(&sh->p_ready[t], 128);
+      tc::mbar_init(&sh->s_lo_full[t], 1); tc::mbar_init(&sh->s_hi_full[t], 1); tc::mbar_init(&sh->b_free[t], 128);
+      tc::mbar_init(&sh->p_ready[t], 128);
       tc::mbar_init(&sh->o_final[t], 1); tc::mbar_init(&sh->l_ready[t], 128); tc::mbar_init(&sh->o_free[t], 128);
     }
     for (int s = 0; s < KV_STAGES; ++s) {
@@ -595,7 +657,6 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
       tc::mbar_init(&sh->v_full[s], 1); tc::mbar_init(&sh->v_empty[s], 2);
     }
     sh->abort_flag = 0;
-    sh->pipe_lock = 0;
     tc::fence_barrier_init();
     tc::tma_prefetch_desc(&tmQ);
     tc::tma_prefetch_desc(&tmK);
