@@ -63,6 +63,7 @@ struct Shared {
   uint64_t tempty[2];
   uint32_t tmem_base;
   int abort_flag;
+  EpiProgram epi;   // the kernel parameter, copied once (see epi_copy_to_smem)
 };
 
 // 32 rows x 64 bytes from "one row per lane" to coalesced global stores (8 rows x 64 contiguous bytes per
@@ -159,7 +160,7 @@ __device__ __forceinline__ void tma_prefetch_4d(const CUtensorMap* m, int32_t c,
 template <int CB>
 __global__ void __launch_bounds__(THREADS, 1)
 conv3x3_tc2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW, __nv_bfloat16* __restrict__ y,
-                   int NB, int H, int W, int C_OUT, const __grid_constant__ EpiProgram epi, float* __restrict__ stats, int cpg,
+                   int NB, int H, int W, int C_OUT, const __grid_constant__ EpiProgram epi_param, float* __restrict__ stats, int cpg,
                    unsigned int* status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -178,6 +179,9 @@ conv3x3_tc2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
   const int total_tiles = NB * quads;
   volatile int* abort_flag = &sh->abort_flag;
   CTR_INIT;
+  static_assert(sizeof(Shared) <= 512, "barrier block");
+  epi_copy_to_smem(&sh->epi, epi_param, threadIdx.x, THREADS);
+  const EpiProgram& epi = sh->epi;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < A_STAGES; ++s) { tc::mbar_init(&sh->a_full[s], 1); tc::mbar_init(&sh->a_empty[s], 1); }
@@ -368,7 +372,7 @@ conv3x3_tc2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
 }
 
 size_t conv_smem_bytes(int c_in, int c_out) {
-  return (size_t)A_STAGES * PATCH_BYTES + 1024 + (size_t)(c_out / 2) * 9 * c_in * 2 + EPI_WARPS * STG_BYTES + BIAS_BYTES + 1024 + 256;
+  return (size_t)A_STAGES * PATCH_BYTES + 1024 + (size_t)(c_out / 2) * 9 * c_in * 2 + EPI_WARPS * STG_BYTES + BIAS_BYTES + 1024 + 512;
 }
 
 }  // namespace

@@ -46,7 +46,7 @@ template <int CTAS> struct Cfg {
   static constexpr int A_BYTES = BM * BK * 2;
   static constexpr int B_BYTES = (BN / CTAS) * BK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  static constexpr size_t SMEM = (size_t)STAGES * STAGE_BYTES + EPI_WARPS * EPI_WARP_BYTES + 1024 /*alignment*/ + 256 /*barriers*/;
+  static constexpr size_t SMEM = (size_t)STAGES * STAGE_BYTES + EPI_WARPS * EPI_WARP_BYTES + 1024 /*alignment*/ + 512 /*barriers, program*/;
 };
 
 template <int STAGES> struct Shared {
@@ -56,6 +56,7 @@ template <int STAGES> struct Shared {
   uint64_t tempty[2];
   uint32_t tmem_base;
   int abort_flag;
+  EpiProgram epi;   // the kernel parameter, copied once (see epi_copy_to_smem)
 };
 
 __device__ __forceinline__ void tile_coords(int t, int num_m, int num_n, int& mi, int& ni) {
@@ -71,7 +72,7 @@ __device__ __forceinline__ void tile_coords(int t, int num_m, int num_n, int& mi
 template <int CTAS, bool SWIGLU>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, void* __restrict__ out, int out_f32, int M,
-               int N, int K, int up_row_offset, const __grid_constant__ EpiProgram epi, unsigned int* status) {
+               int N, int K, int up_row_offset, const __grid_constant__ EpiProgram epi_param, unsigned int* status) {
   using C = Cfg<CTAS>;
   constexpr int STAGES = C::STAGES;
   constexpr int OUT_N = SWIGLU ? BN / 2 : BN;  // output columns per tile
@@ -90,6 +91,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   MK_TR_DECL
   MK_TR_INIT;
 
+  static_assert(sizeof(Shared<STAGES>) <= 512, "barrier block");
+  epi_copy_to_smem(&sh->epi, epi_param, threadIdx.x, THREADS);
+  const EpiProgram& epi = sh->epi;
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { tc::mbar_init(&sh->full[s], 1); tc::mbar_init(&sh->empty[s], 1); }
     for (int b = 0; b < 2; ++b) { tc::mbar_init(&sh->tfull[b], 1); tc::mbar_init(&sh->tempty[b], EPI_WARPS * CTAS); }
@@ -255,6 +259,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   }
 
   MK_TR_PRINT("gemm");
+
   // common exit: on an aborted run give copies in flight time to land before the CTA retires
   if (*abort_flag) {
     const long long t0 = clock64();

@@ -119,6 +119,18 @@ __device__ __forceinline__ void epi32(const EpiProgram& p, float (&v)[32], int64
   }
 }
 
+// The elementwise program arrives as a kernel parameter and is interpreted per 32-column chunk through a
+// reference.  The tensor-core kernels copy it to shared memory once, before their first __syncthreads, so
+// the interpreter's run-time-indexed reads are shared-memory broadcasts whatever the compiler makes of a
+// reference to the parameter space.  (Measured: no change in kernel time; kept for the predictable latency.)
+__device__ __forceinline__ void epi_copy_to_smem(EpiProgram* dst, const EpiProgram& src, int tid, int nthreads) {
+  constexpr int WORDS = (int)(sizeof(EpiProgram) / 4);
+  static_assert(sizeof(EpiProgram) % 4 == 0, "EpiProgram is copied word by word");
+  const uint32_t* s = reinterpret_cast<const uint32_t*>(&src);
+  uint32_t* d = reinterpret_cast<uint32_t*>(dst);
+  for (int i = tid; i < WORDS; i += nthreads) d[i] = s[i];
+}
+
 // index of the op of kind `kind` if the program has exactly one, else -1 (then that kind is read
 // straight from global memory inside epi32)
 __device__ __forceinline__ int epi_single_index(const EpiProgram& p, int kind) {
