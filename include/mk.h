@@ -14,8 +14,9 @@
  *   4. run the composed forward                               mk_module_set_param,
  *                                                             mk_module_workspace_size,
  *                                                             mk_module_forward
- *   5. observe: per-subkernel time, boundary tensors          mk_module_profile,
- *                                                             mk_module_intermediate
+ *   5. observe: per-subkernel time, boundary tensors;         mk_module_profile,
+ *      swap what is slower than an alternative                mk_module_intermediate,
+ *                                                             mk_module_swap
  *
  * Conventions
  *   - Every pointer named dev_* / in_ptrs[i] / out_ptrs[i] / workspace is a DEVICE pointer
@@ -229,6 +230,21 @@ MK_API mk_status mk_module_forward(mk_module* m, const void* const* in_ptrs, voi
 MK_API mk_status mk_module_profile(mk_module* m, const void* const* in_ptrs, void* const* out_ptrs,
                             void* workspace, size_t workspace_bytes, void* cuda_stream,
                             int32_t iters, float* ms_per_sub);
+/* Swap (paper, Algorithm 1's Swap step and the "MKEvolve (Swap)" variant: a subkernel that is slower
+ * than an available alternative by more than a threshold is replaced, the rest of the composition is
+ * left alone).  For every submodule in turn: time every registered implementation that accepts the whole
+ * submodule (mk_module_profile's event pairs, on the caller's buffers: the tensors are overwritten
+ * with valid results of whichever binding ran last) and, if the bound one runs at less than `tau`
+ * (paper: 0.9; 0 < tau <= 1) of the fastest one's speed, rebind the submodule to the fastest; otherwise
+ * the original binding - a composer-chosen chain included - is restored.  Modules with fewer than two
+ * submodules are left alone, as in the paper.  An alternative that needs more workspace than
+ * workspace_bytes, or whose first run takes more than four times the best time so far, is skipped.
+ * n_swapped (optional): number of submodules rebound.  ms_before_after (optional): float
+ * [n_sub][2], each submodule's time with its old and with its final binding.  Synchronises the stream.
+ * Errors: as mk_module_profile; the bindings are valid (old or new) on every return. */
+MK_API mk_status mk_module_swap(mk_module* m, const void* const* in_ptrs, void* const* out_ptrs, void* workspace,
+                         size_t workspace_bytes, void* cuda_stream, int32_t iters, double tau,
+                         int32_t* n_swapped, float* ms_before_after);
 /* Device pointer and spec of the tensor produced by value `value_id` at a submodule boundary
  * during the last forward (requires keep_intermediates; MK_ERR_INVALID_ARG if the value is
  * internal to a submodule or no forward has run). */

@@ -87,6 +87,7 @@ _sig("mk_module_workspace_size", C.c_int32, _P, C.POINTER(C.c_size_t))
 _sig("mk_module_launch_count", C.c_int32, _P, _I32P)
 _sig("mk_module_forward", C.c_int32, _P, _PP, _PP, _P, C.c_size_t, _P)
 _sig("mk_module_profile", C.c_int32, _P, _PP, _PP, _P, C.c_size_t, _P, C.c_int32, C.POINTER(C.c_float))
+_sig("mk_module_swap", C.c_int32, _P, _PP, _PP, _P, C.c_size_t, _P, C.c_int32, C.c_double, C.POINTER(C.c_int32), C.POINTER(C.c_float))
 _sig("mk_module_intermediate", C.c_int32, _P, C.c_int32, _PP, _SPECP)
 _sig("mk_groupnorm_nhwc_noalloc", C.c_int32, C.c_int32, _P, _P, _P, _P, C.c_int64, C.c_int64, C.c_int64,
      C.c_int64, C.c_int32, C.c_double, _P)
@@ -334,6 +335,16 @@ class Module:
         ms = (C.c_float * self.n_sub())()
         self._ck(mk_module_profile(self.h, ins, outs, ws, workspace_bytes, stream, iters, ms))
         return list(ms)
+
+    def swap(self, inputs, output, workspace=None, workspace_bytes=0, stream=0, iters=5, tau=0.9):
+        """Rebind every submodule that runs at less than `tau` of its fastest alternative's speed.
+        Returns (number rebound, [(ms before, ms after)] per submodule)."""
+        ins, outs = self._marshal(inputs, output)
+        ws = _ptr(workspace) if workspace is not None else None
+        n = C.c_int32(0)
+        ms = (C.c_float * (2 * self.n_sub()))()
+        self._ck(mk_module_swap(self.h, ins, outs, ws, workspace_bytes, stream, iters, tau, C.byref(n), ms))
+        return n.value, [(ms[2 * i], ms[2 * i + 1]) for i in range(self.n_sub())]
 
     def intermediate(self, value):
         vid = self.value_id[value] if isinstance(value, str) else value

@@ -387,6 +387,54 @@ mk_status mk_module_profile(mk_module* m, const void* const* in_ptrs, void* cons
   return ret;
 }
 
+mk_status mk_module_swap(mk_module* m, const void* const* in_ptrs, void* const* out_ptrs, void* workspace, size_t workspace_bytes,
+                         void* cuda_stream, int32_t iters, double tau, int32_t* n_swapped, float* ms_before_after) {
+  if (!m || iters < 1 || !(tau > 0.0) || tau > 1.0) return MK_ERR_INVALID_ARG;
+  if (n_swapped) *n_swapped = 0;
+  const int ns = m->n_sub();
+  std::vector<float> base(ns, 0.f), ms(ns, 0.f);
+  mk_status st = mk_module_profile(m, in_ptrs, out_ptrs, workspace, workspace_bytes, cuda_stream, iters, base.data());
+  if (st != MK_OK) return st;
+  if (ms_before_after)
+    for (int s_ = 0; s_ < ns; ++s_) ms_before_after[2 * s_] = ms_before_after[2 * s_ + 1] = base[s_];
+  if (ns < 2) return MK_OK;
+  int swapped = 0;
+  for (int sub = 0; sub < ns; ++sub) {
+    const Binding original = m->bind[sub];
+    std::string best_name = original.name;
+    float best_ms = base[sub];
+    std::vector<const char*> cands;
+    for (const Impl& im : registry())
+      if (im.match(*m, m->sub_lo(sub), m->sub_hi(sub)) && original.name != im.name) cands.push_back(im.name);
+    for (const char* cand : cands) {
+      if (mk_module_bind(m, sub, cand) != MK_OK) continue;
+      size_t need = 0;
+      if (mk_module_workspace_size(m, &need) != MK_OK || need > workspace_bytes) continue;
+      // one run first: it builds the plan and shows whether the alternative is in the race at all
+      if (mk_module_profile(m, in_ptrs, out_ptrs, workspace, workspace_bytes, cuda_stream, 1, ms.data()) != MK_OK) continue;
+      if (ms[sub] > 4.0f * best_ms) continue;
+      if (mk_module_profile(m, in_ptrs, out_ptrs, workspace, workspace_bytes, cuda_stream, iters, ms.data()) != MK_OK) continue;
+      if (ms[sub] < best_ms) { best_ms = ms[sub]; best_name = cand; }
+    }
+    // the bound one keeps its place unless it reaches less than tau of the fastest one's speed
+    if (best_name != original.name && (double)best_ms < tau * (double)base[sub]) {
+      st = mk_module_bind(m, sub, best_name.c_str());
+      if (st != MK_OK) { m->bind[sub] = original; invalidate(*m); return st; }
+      ++swapped;
+      if (ms_before_after) ms_before_after[2 * sub + 1] = best_ms;
+    } else {
+      m->bind[sub] = original;
+      invalidate(*m);
+    }
+  }
+  if (n_swapped) *n_swapped = swapped;
+  // leave a valid result of the final composition in the caller's output
+  size_t need = 0;
+  st = mk_module_workspace_size(m, &need);
+  if (st != MK_OK) return st;
+  return mk_module_profile(m, in_ptrs, out_ptrs, workspace, workspace_bytes, cuda_stream, 1, ms.data());
+}
+
 mk_status mk_module_intermediate(const mk_module* m, int32_t value_id, const void** dev_ptr, mk_tensor_spec* spec) {
   if (!m || !dev_ptr) return MK_ERR_INVALID_ARG;
   if (value_id < 0 || value_id >= (int)m->values.size()) return fail(m->ctx, MK_ERR_INVALID_ARG, "value id out of range");

@@ -60,6 +60,15 @@ class DeviceWorkload:
                             self.ws_bytes, s)
         return self.out
 
+    def swap(self, iters=5, tau=0.9):
+        """Rebind submodules that run slower than tau x their fastest alternative (the output tensor is
+        overwritten with the result of the final composition)."""
+        self.ensure_workspace()
+        s = torch.cuda.current_stream().cuda_stream
+        r = self.module.swap([self.inputs[k] for k in self.module.input_names], self.out, self.ws, self.ws_bytes, s, iters, tau)
+        self.ensure_workspace()
+        return r
+
     def profile(self, iters=10):
         self.ensure_workspace()
         s = torch.cuda.current_stream().cuda_stream

@@ -203,3 +203,17 @@ def test_fp32_residual_stream_dtypes(ctx):
     m.set_decomposition([0, 5])
     ins, outs = m.contract(1)
     assert any(dt == B.MK_F32 for _, (dt, _, _) in ins)
+
+
+def test_swap_needs_a_device_and_sane_arguments(ctx):
+    w = W.c2(0, 16, 8, 8)
+    m = _mod(ctx, w)
+    m.set_decomposition(w.partitions["split"])
+    n = C.c_int32(7)
+    ins = (C.c_void_p * 1)(None)
+    outs = (C.c_void_p * 1)(None)
+    assert B.mk_module_swap(m.h, ins, outs, None, 0, None, 0, 0.9, C.byref(n), None) == B.MK_ERR_INVALID_ARG
+    assert B.mk_module_swap(m.h, ins, outs, None, 0, None, 3, 1.5, C.byref(n), None) == B.MK_ERR_INVALID_ARG
+    st = B.mk_module_swap(m.h, ins, outs, None, 0, None, 3, 0.9, C.byref(n), None)
+    assert st != B.MK_OK and n.value == 0          # a host-only context cannot time anything
+    assert m.n_sub() == 4 and m.bound_impl(1) == "eltwise"    # bindings untouched
