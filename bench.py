@@ -35,7 +35,10 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # capture summarised under profiles/ (null until a capture of that workload exists)
 NCU_TRAFFIC_BYTES = {"c2": 105.7e6}   # profiles/gemm_tc2_c2.md
 
-DEFAULT_STEPS = {"c1": 2000, "c2": 1000, "c3": 1000, "c4": 200, "c5": 50}
+# Timed regions of a few tens of milliseconds: long enough for stable event timing, short enough that the
+# 1 kW power cap has not yet pulled the clocks down (a 4096^3 GEMM step goes from 110 us at K = 200 to
+# 117 us at K = 1000 and 122 us at K = 3000); the burst peak is the matching denominator for one-kernel steps.
+DEFAULT_STEPS = {"c1": 2000, "c2": 200, "c3": 400, "c4": 100, "c5": 50}
 
 
 def full_workload(name, seed=0, batch=None, only_ops=None):
