@@ -32,12 +32,13 @@ METRIC = "composed-module fwd latency, TFLOP/s & GB/s as % of B200 roofline, per
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
-# capture summarised under profiles/ (null until a capture of that workload exists)
-NCU_TRAFFIC_BYTES = {"c2": 105.7e6}   # profiles/gemm_tc2_c2.md
+# captures summarised under profiles/ (null where no capture of that workload's dominant kernel exists).
+# c4: the attention kernel was captured on 2 of the 16 batch elements (52.2 MB; its traffic is
+# proportional to the batch) and is scaled by 8 here.
+NCU_TRAFFIC_BYTES = {"c2": 105.7e6,            # profiles/gemm_tc2_c2.md
+                     "c3": 26.25e6,            # profiles/conv3x3_tc2_groupnorm_c3.md (conv; its output stays in L2)
+                     "c4": 8 * 52.2e6}         # profiles/attention_tc2_c4.md
 
-# Timed regions of a few tens of milliseconds: long enough for stable event timing, short enough that the
-# 1 kW power cap has not yet pulled the clocks down (a 4096^3 GEMM step goes from 110 us at K = 200 to
-# 117 us at K = 1000 and 122 us at K = 3000); the burst peak is the matching denominator for one-kernel steps.
 DEFAULT_STEPS = {"c1": 2000, "c2": 200, "c3": 400, "c4": 100, "c5": 50}
 
 
