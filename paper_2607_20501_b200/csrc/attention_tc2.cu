@@ -393,9 +393,10 @@ __device__ __forceinline__ void role_mma(const Ctx& cx, uint32_t tmem_base, int 
 // scale * log2 e): p = exp2(s * scale*log2e - m).  Any m gives the same O / l as long as nothing
 // overflows, so m is NOT kept equal to the running row maximum; it is raised (and the running O in TMEM,
 // l, and whatever of this tile's P is already computed, rescaled by exp2(m_old - m_new)) only
-//   * on an item's first and diagonal tiles, after a pre-pass that also writes -inf over the masked
-//     scores in TMEM (key > query), so that the main pass needs no mask; and
-//   * when a half-row sum leaves the safe range (2^60) - then from that half's own maximum.
+//   * on an item's diagonal tile, after a pre-pass that also writes -inf over the masked scores in TMEM
+//     (key > query), so that the main pass needs no mask; and
+//   * when a half-row sum leaves the safe range (above 2^60; or, on an item's very first half, where m is
+//     a mere guess of 0, underflowed) - then from that half's own maximum.
 // S arrives in two halves: keys 0..63 in columns [64, 128) of the stream's S region (B), keys 64..127 in
 // columns [0, 64) (A).  As soon as the first half has been turned into probabilities (kept in registers),
 // region B is handed back (b_free) and the tensor pipe computes the next tile's first half into it while this
@@ -417,7 +418,10 @@ __device__ __forceinline__ void role_softmax(const Ctx& cx, uint32_t tmem_base, 
   while (iter.next(it)) {
     const int nt = T ? it.n1 : it.n0;
     if (nt == 0) continue;
-    float m = -INFINITY, l = 0.0f;
+    // m = 0 is the first guess of an item (scores of the usual size then need no maximum at all); `fresh`
+    // says that nothing of this item has been accumulated yet, so m may still be set freely
+    float m = 0.0f, l = 0.0f;
+    bool fresh = true;
 #pragma unroll 1
     for (int j = 0; j < nt; ++j) {
       const uint32_t par = n_tiles & 1;
@@ -430,9 +434,13 @@ __device__ __forceinline__ void role_softmax(const Ctx& cx, uint32_t tmem_base, 
       };
       // m := max(m, mx); the running O (not on an item's first tile) and l follow
       auto raise = [&](float mx) -> float {
+        if (fresh) {
+          m = mx;                          // nothing to rescale yet
+          return 1.0f;
+        }
         float alpha = 1.0f;
         if (mx > m) {
-          alpha = tc::ex2_fast(m - mx);    // 0 on the first tile (m = -inf)
+          alpha = tc::ex2_fast(m - mx);
           m = mx;
         }
         if (j > 0 && __any_sync(0xffffffffu, alpha != 1.0f)) {
@@ -464,11 +472,11 @@ __device__ __forceinline__ void role_softmax(const Ctx& cx, uint32_t tmem_base, 
         return fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * scale_log2;
       };
 
-      if (j == 0 || j == nt - 1) {
-        // first / diagonal tile: both halves, masked scores replaced by -inf in place, m raised to the row maximum
+      if (j == nt - 1) {
+        // diagonal tile: both halves, masked scores replaced by -inf in place, m raised to the row maximum
         if (!wait_half(&sh->s_lo_full[T])) return;
         if (!wait_half(&sh->s_hi_full[T])) return;
-        const int last = (j == nt - 1) ? row : 127;     // last visible key of this row inside the tile
+        const int last = row;                           // last visible key of this row inside the tile
         float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll 1
         for (int c = 0; c < 4; ++c) {
@@ -516,11 +524,14 @@ __device__ __forceinline__ void role_softmax(const Ctx& cx, uint32_t tmem_base, 
           }
         }
         sum_lo = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
-        if (attempt == 1 || !__any_sync(0xffffffffu, !(sum_lo < 1.152921504606847e18f))) break;   // 2^60; also inf / NaN
+        // safe range: below 2^60 (also false for inf / NaN) and, while m is still the first guess, not underflowed
+        const bool bad = !(sum_lo < 1.152921504606847e18f) || (fresh && !(sum_lo > 8.673617379884035e-19f));
+        if (attempt == 1 || !__any_sync(0xffffffffu, bad)) break;
         // out of range: raise m to this half's maximum (O is safe to touch once S_hi is visible), then once more
         if (!wait_half(&sh->s_hi_full[T])) return;
         raise(half_max(s_addr + 64));
       }
+      fresh = false;
       tc::tc_fence_before();
       tc::mbar_arrive(&sh->b_free[T]);
       TR2(T == 0 && threadIdx.x == 0 && n_items == 0 && j < 11, 2 + j * 8);

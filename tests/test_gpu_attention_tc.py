@@ -99,3 +99,21 @@ def test_row_maximum_growing_from_key_tile_to_key_tile(ctx, impl, step):
     ref, _ = oracle(w, [0])
     dw, out = run_gpu(ctx, w, [0], binds={0: impl})
     assert_parity(out, ref, "bf16", impl)
+
+
+@pytest.mark.parametrize("impl", TC_IMPLS)
+def test_scores_far_below_zero_at_the_start_of_a_row(ctx, impl):
+    """The first 64 keys score about -100 log2 units against every query: a kernel that starts from a guessed
+    reference maximum (0) sees its first partial row sum underflow and has to take the maximum from the data;
+    the early queries see ONLY those keys, so nothing later can hide a zero row sum."""
+    b, h, s, d = 1, 2, 512, 128
+    w = _attn_only(W.c4(9, B=b, H=h, S=s, D=d))
+    q = 2.5 + 0.25 * w.inputs["q"].f64()
+    k = w.inputs["k"].f64()
+    k[:, :, :64, :] = -2.5
+    w.inputs["q"] = G.make("q", "bf16", q.astype(np.float32))
+    w.inputs["k"] = G.make("k", "bf16", k.astype(np.float32))
+    ref, _ = oracle(w, [0])
+    dw, out = run_gpu(ctx, w, [0], binds={0: impl})
+    assert np.isfinite(out).all()
+    assert_parity(out, ref, "bf16", impl)
