@@ -393,10 +393,10 @@ __device__ __forceinline__ void role_mma(const Ctx& cx, uint32_t tmem_base, int 
 // scale * log2 e): p = exp2(s * scale*log2e - m).  Any m gives the same O / l as long as nothing
 // overflows, so m is NOT kept equal to the running row maximum; it is raised (and the running O in TMEM,
 // l, and whatever of this tile's P is already computed, rescaled by exp2(m_old - m_new)) only
-//   * on an item's diagonal tile, after a pre-pass that also writes -inf over the masked scores in TMEM
-//     (key > query), so that the main pass needs no mask; and
-//   * when a half-row sum leaves the safe range (above 2^60; or, on an item's very first half, where m is
-//     a mere guess of 0, underflowed) - then from that half's own maximum.
+// when a half-row sum leaves the safe range (above 2^60; or, on an item's very first half, where m is a
+// mere guess of 0, underflowed) - then from that half's own maximum.  The common tile is therefore one pass
+// over S with no maximum at all.  On the diagonal tile (an item's last) a warp masks the one 32-key chunk
+// that holds its own diagonal by writing -inf over the hidden scores in TMEM, and skips the chunks right of it.
 // S arrives in two halves: keys 0..63 in columns [64, 128) of the stream's S region (B), keys 64..127 in
 // columns [0, 64) (A).  As soon as the first half has been turned into probabilities (kept in registers),
 // region B is handed back (b_free) and the tensor pipe computes the next tile's first half into it while this
@@ -459,10 +459,10 @@ __device__ __forceinline__ void role_softmax(const Ctx& cx, uint32_t tmem_base, 
         return alpha;
       };
       // maximum (log2 units) of 64 scores starting at TMEM address `base`
-      auto half_max = [&](uint32_t base) -> float {
+      auto half_max = [&](uint32_t base, int nchunks) -> float {
         float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll 1
-        for (int c = 0; c < 2; ++c) {
+        for (int c = 0; c < nchunks; ++c) {
           uint32_t r[32];
           tc::tmem_ld32(base + c * 32, r);
           tc::tmem_ld_wait();
@@ -472,32 +472,24 @@ __device__ __forceinline__ void role_softmax(const Ctx& cx, uint32_t tmem_base, 
         return fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * scale_log2;
       };
 
-      if (j == nt - 1) {
-        // diagonal tile: both halves, masked scores replaced by -inf in place, m raised to the row maximum
+      // Chunks of 32 keys this warp's rows can see at all: every one off the diagonal; on the diagonal tile
+      // (the item's last) chunk q holds the warp's own diagonal (key i of it is visible to lane >= i) and the
+      // chunks right of it are skipped outright.
+      const bool diag = j == nt - 1;
+      const int vis = diag ? q + 1 : 4;
+      if (diag) {
+        // -inf over the masked scores of chunk q, in place, so that the main pass needs no mask code
         if (!wait_half(&sh->s_lo_full[T])) return;
         if (!wait_half(&sh->s_hi_full[T])) return;
-        const int last = row;                           // last visible key of this row inside the tile
-        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
-          const uint32_t addr = s_addr + (c < 2 ? 64 + c * 32 : (c - 2) * 32);
-          uint32_t r[32];
-          tc::tmem_ld32(addr, r);
-          tc::tmem_ld_wait();
-          const int lim = last - c * 32;
-          // the write-back is a warp-collective instruction: decide it for the whole warp (some lane of this
-          // warp, whose rows are q * 32 .. q * 32 + 31, has a masked key in this chunk)
-          if (j == nt - 1 && q * 32 - c * 32 < 31) {
+        const uint32_t addr = s_addr + (q < 2 ? 64 + q * 32 : (q - 2) * 32);
+        uint32_t r[32];
+        tc::tmem_ld32(addr, r);
+        tc::tmem_ld_wait();
 #pragma unroll
-            for (int i = 0; i < 32; ++i)
-              if (i > lim) r[i] = 0xff800000u;
-            tc::tmem_st32(addr, r);
-          }
-#pragma unroll
-          for (int i = 0; i < 32; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(r[i]));
-        }
+        for (int i = 0; i < 32; ++i)
+          if (i > lane) r[i] = 0xff800000u;
+        tc::tmem_st32(addr, r);
         tc::tmem_st_wait();
-        raise(fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * scale_log2);
       }
 
       uint32_t pk[64];
@@ -512,6 +504,11 @@ __device__ __forceinline__ void role_softmax(const Ctx& cx, uint32_t tmem_base, 
         float sum4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll
         for (int c = 0; c < 2; ++c) {
+          if (c >= vis) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) pk[c * 16 + i] = 0u;
+            continue;
+          }
           uint32_t r[32];
           tc::tmem_ld32(s_addr + 64 + c * 32, r);
           tc::tmem_ld_wait();
@@ -529,7 +526,7 @@ __device__ __forceinline__ void role_softmax(const Ctx& cx, uint32_t tmem_base, 
         if (attempt == 1 || !__any_sync(0xffffffffu, bad)) break;
         // out of range: raise m to this half's maximum (O is safe to touch once S_hi is visible), then once more
         if (!wait_half(&sh->s_hi_full[T])) return;
-        raise(half_max(s_addr + 64));
+        raise(half_max(s_addr + 64, vis < 2 ? vis : 2));
       }
       fresh = false;
       tc::tc_fence_before();
@@ -544,6 +541,11 @@ __device__ __forceinline__ void role_softmax(const Ctx& cx, uint32_t tmem_base, 
         float sum4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll
         for (int c = 0; c < 2; ++c) {
+          if (2 + c >= vis) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) pk[32 + c * 16 + i] = 0u;
+            continue;
+          }
           uint32_t r[32];
           tc::tmem_ld32(s_addr + c * 32, r);
           tc::tmem_ld_wait();
@@ -558,7 +560,7 @@ __device__ __forceinline__ void role_softmax(const Ctx& cx, uint32_t tmem_base, 
         sum_hi = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
         if (attempt == 1 || !__any_sync(0xffffffffu, !(sum_hi < 1.152921504606847e18f))) break;
         // out of range: raise m to this half's maximum; the first half's probabilities and sum follow
-        const float alpha = raise(half_max(s_addr));
+        const float alpha = raise(half_max(s_addr, vis - 2 > 0 ? vis - 2 : 0));
         sum_lo *= alpha;
 #pragma unroll
         for (int i = 0; i < 32; ++i) {

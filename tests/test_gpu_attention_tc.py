@@ -57,8 +57,9 @@ def test_closed_forms(ctx):
     for impl in TC_IMPLS:
         dw, out = run_gpu(ctx, w, [0], binds={0: impl})
         assert_parity(out, pm.transpose(0, 2, 1, 3).reshape(b * s, h * d), "bf16", f"{impl} uniform weights")
-        # first query sees only the first key (the diagonal is kept)
-        assert np.array_equal(out[0].reshape(h, d), v[0, :, 0, :])
+        # first query sees only the first key (the diagonal is kept): O = p V / p with p rounded to bf16 in the
+        # numerator only, so equal up to one bf16 rounding of a single probability
+        assert np.abs(out[0].reshape(h, d) - v[0, :, 0, :]).max() <= 2.0 ** -7 * np.abs(v[0, :, 0, :]).max()
 
 
 def test_packed_qkv_view_and_swap(ctx):
