@@ -71,8 +71,9 @@ __device__ __forceinline__ void tile_coords(int t, int num_m, int num_n, int& mi
 
 template <int CTAS, bool SWIGLU>
 __global__ void __launch_bounds__(THREADS, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, void* __restrict__ out, int out_f32, int M,
-               int N, int K, int up_row_offset, const __grid_constant__ EpiProgram epi_param, unsigned int* status) {
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmBh,
+               void* __restrict__ out, int out_f32, int M, int N, int K, int up_row_offset, int tail_first,
+               const __grid_constant__ EpiProgram epi_param, unsigned int* status) {
   using C = Cfg<CTAS>;
   constexpr int STAGES = C::STAGES;
   constexpr int OUT_N = SWIGLU ? BN / 2 : BN;  // output columns per tile
@@ -86,6 +87,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const int unit_id = blockIdx.x / CTAS, num_units = gridDim.x / CTAS;   // a unit = a CTA or a CTA pair
   const int num_m = (M + CTAS * BM - 1) / (CTAS * BM), num_n = (N + OUT_N - 1) / OUT_N;
   const int total_tiles = num_m * num_n;
+  // Work units: tiles [0, tail_first) whole; each tile from tail_first on as two units of half the columns
+  // (256 x 128, N = 128 MMAs), so that a last wave that would leave more than half of the machine idle is
+  // spread over twice as many CTA pairs.  tail_first = total_tiles: no split.
+  const int total_units = tail_first + 2 * (total_tiles - tail_first);
+  auto decode = [&](int u, int& tile, int& nhalf) {
+    if (u < tail_first) { tile = u; nhalf = -1; }
+    else { tile = tail_first + ((u - tail_first) >> 1); nhalf = (u - tail_first) & 1; }
+  };
   const int num_kb = (K + BK - 1) / BK;
   volatile int* abort_flag = &sh->abort_flag;
   MK_TR_DECL
@@ -118,7 +127,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int t = unit_id; t < total_tiles && ok; t += num_units) {
+      for (int u = unit_id; u < total_units && ok; u += num_units) {
+        int t, nhalf;
+        decode(u, t, nhalf);
         int mi, ni;
         tile_coords(t, num_m, num_n, mi, ni);
         const int m0 = (mi * CTAS + (int)rank) * BM;
@@ -133,17 +144,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           ok = tc::mbar_wait(&sh->empty[stage], phase ^ 1, abort_flag, status, tc::WAIT_SMEM_EMPTY);
 #ifdef MK_TRACE
           esum += tc::gtime() - w0_;
-          if (kb == num_kb - 1 && blockIdx.x == 0) mk_tr[70 + (t - unit_id) / num_units] = mk_tr[0] + esum;
+          if (kb == num_kb - 1 && blockIdx.x == 0) mk_tr[70 + (u - unit_id) / num_units] = mk_tr[0] + esum;
 #endif
           if (!ok) break;
           uint8_t* a_dst = tiles + (size_t)stage * C::STAGE_BYTES;
           uint8_t* b_dst = a_dst + C::A_BYTES;
           if (CTAS == 2) {
             const uint32_t full_leader = tc::map_to_cta(tc::smem_u32(&sh->full[stage]), 0);
-            if (leader) tc::mbar_expect_tx(&sh->full[stage], 2 * C::STAGE_BYTES);
-            const int b_row = SWIGLU ? (leader ? n0 : up_row_offset + n0) : n0 + (int)rank * (BN / 2);
             tc::tma_load_2d_pair(a_dst, &tmA, full_leader, kb * BK, m0);
-            tc::tma_load_2d_pair(b_dst, &tmB, full_leader, kb * BK, b_row);
+            if (nhalf < 0) {
+              if (leader) tc::mbar_expect_tx(&sh->full[stage], 2 * C::STAGE_BYTES);
+              const int b_row = SWIGLU ? (leader ? n0 : up_row_offset + n0) : n0 + (int)rank * (BN / 2);
+              tc::tma_load_2d_pair(b_dst, &tmB, full_leader, kb * BK, b_row);
+            } else {
+              // half the columns: 64 W rows per CTA
+              if (leader) tc::mbar_expect_tx(&sh->full[stage], 2 * (C::A_BYTES + C::B_BYTES / 2));
+              tc::tma_load_2d_pair(b_dst, &tmBh, full_leader, kb * BK, n0 + nhalf * (BN / 2) + (int)rank * (BN / 4));
+            }
           } else {
             tc::mbar_expect_tx(&sh->full[stage], C::STAGE_BYTES);
             tc::tma_load_2d(a_dst, &tmA, &sh->full[stage], kb * BK, m0);
@@ -158,13 +175,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer (one lane of the leader)
     if (leader && lane == 0) {
-      constexpr uint32_t idesc = tc::idesc_bf16_f32(CTAS * BM, BN, 0, 0);
+      constexpr uint32_t idesc_full = tc::idesc_bf16_f32(CTAS * BM, BN, 0, 0);
+      constexpr uint32_t idesc_half = tc::idesc_bf16_f32(CTAS * BM, BN / 2, 0, 0);
       const uint32_t a_lo0 = tc::desc_lo_sw128(tc::smem_u32(tiles));
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
       int it = 0;
-      for (int t = unit_id; t < total_tiles && ok; t += num_units, ++it) {
+      for (int u = unit_id; u < total_units && ok; u += num_units, ++it) {
+        const uint32_t idesc = u < tail_first ? idesc_full : idesc_half;
         const int acc = it & 1;
         const uint32_t d_tmem = tmem_base + acc * BN;
         ok = tc::mbar_wait(&sh->tempty[acc], ((it >> 1) & 1) ^ 1, abort_flag, status, tc::WAIT_TMEM_EMPTY);
@@ -216,15 +235,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     ew.init(staging + (warp - 2) * EPI_WARP_BYTES, epi, lane, out_f32 != 0);
     bool ok = true;
     int it = 0;
-    for (int t = unit_id; t < total_tiles && ok; t += num_units, ++it) {
+    for (int u = unit_id; u < total_units && ok; u += num_units, ++it) {
+      int t, nhalf;
+      decode(u, t, nhalf);
       int mi, ni;
       tile_coords(t, num_m, num_n, mi, ni);
       const int acc = it & 1;
       const int64_t row0 = (int64_t)(mi * CTAS + (int)rank) * BM + q * 32;
       auto rowmap = [&](int r) -> int64_t { const int64_t g = row0 + r; return g < M ? g : -1; };
-      const int64_t col_base = (int64_t)ni * OUT_N;
+      const int64_t col_base = (int64_t)ni * OUT_N + (nhalf > 0 ? BN / 2 : 0);
+      const int chunks_here = nhalf < 0 ? CHUNKS : CHUNKS / 2;
       uint4 res_regs[8];
-      ew.load_bias(epi, col_base, OUT_N, N);
+      ew.load_bias(epi, col_base, nhalf < 0 ? OUT_N : OUT_N / 2, N);
       ew.prefetch_res(epi, rowmap, col_base + half * 32, N, res_regs);
       ok = tc::mbar_wait(&sh->tfull[acc], (it >> 1) & 1, abort_flag, status, tc::WAIT_TMEM_FULL);
       ok = __all_sync(0xffffffffu, ok ? 1 : 0) != 0;
@@ -233,7 +255,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       tc::tc_fence_after();
       const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN;
 #pragma unroll 1
-      for (int c = half; c < CHUNKS; c += 2) {
+      for (int c = half; c < chunks_here; c += 2) {
         uint32_t r[32];
         float v[32];
         tc::tmem_ld32(t_row + c * 32, r);
@@ -246,7 +268,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
           for (int j = 0; j < 32; ++j) v[j] = silu_fast(v[j]) * __uint_as_float(r[j]);
         }
-        ew.chunk_out(epi, v, rowmap, out, col_base + c * 32, c * 32, (int64_t)N, res_regs, c + 2 < CHUNKS ? col_base + (c + 2) * 32 : -1);
+        ew.chunk_out(epi, v, rowmap, out, col_base + c * 32, c * 32, (int64_t)N, res_regs, c + 2 < chunks_here ? col_base + (c + 2) * 32 : -1);
       }
       tc::tc_fence_before();
       __syncwarp();
@@ -285,6 +307,8 @@ cudaError_t plan_impl(GemmTcPlan* p, const void* a, const void* w_nk, void* y, b
   if (e != cudaSuccess) return e;
   e = encode_tmap_2d_bf16(&p->tm_b, w_nk, (uint64_t)w_rows, (uint64_t)k, (uint64_t)k, BN / 2, BK);
   if (e != cudaSuccess) return e;
+  e = encode_tmap_2d_bf16(&p->tm_b_half, w_nk, (uint64_t)w_rows, (uint64_t)k, (uint64_t)k, BN / 4, BK);
+  if (e != cudaSuccess) return e;
   p->out = y;
   p->out_f32 = out_f32;
   p->m = (int)m; p->n = (int)n; p->k = (int)k;
@@ -294,6 +318,10 @@ cudaError_t plan_impl(GemmTcPlan* p, const void* a, const void* w_nk, void* y, b
   const int64_t tiles = ((m + CTAS * BM - 1) / (CTAS * BM)) * ((n + out_n - 1) / out_n);
   const int64_t units = tiles < sm_count / CTAS ? tiles : sm_count / CTAS;
   p->grid = (int)(CTAS * units);
+  // a last wave that fills at most half of the CTA pairs is run as half-width units (two-SM form only)
+  const int64_t tail = tiles % units;
+  p->tail_first = (int)tiles;
+  if (CTAS == 2 && !swiglu && tiles > units && tail > 0 && 2 * tail <= units) p->tail_first = (int)(tiles - tail);
   return cudaSuccess;
 }
 
@@ -320,8 +348,11 @@ cudaError_t launch_impl(const GemmTcPlan& p, cudaStream_t s) {
   cfg.numAttrs = 1;
   unsigned int* status = kernel_status_ptr();
   const int out_f32 = p.out_f32 ? 1 : 0;
-  if (p.swiglu) return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<CTAS, true>, p.tm_a, p.tm_b, p.out, out_f32, p.m, p.n, p.k, p.n, p.epi, status);
-  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<CTAS, false>, p.tm_a, p.tm_b, p.out, out_f32, p.m, p.n, p.k, 0, p.epi, status);
+  if (p.swiglu)
+    return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<CTAS, true>, p.tm_a, p.tm_b, p.tm_b_half, p.out, out_f32, p.m, p.n, p.k, p.n, p.tail_first, p.epi,
+                              status);
+  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<CTAS, false>, p.tm_a, p.tm_b, p.tm_b_half, p.out, out_f32, p.m, p.n, p.k, 0, p.tail_first, p.epi,
+                            status);
 }
 
 }  // namespace

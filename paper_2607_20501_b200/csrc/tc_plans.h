@@ -10,6 +10,8 @@ namespace mk {
 
 struct GemmTcPlan {
   CUtensorMap tm_a, tm_b;
+  CUtensorMap tm_b_half;    // W with a box of half as many rows, for the half-width units of the last wave
+  int tail_first = 0;       // tiles from this index on run as two half-width units (= tile count: none)
   void* out = nullptr;
   bool out_f32 = false;     // output stored as fp32 (an fp32 residual stream), else bf16
   int m = 0, n = 0, k = 0;  // n = output columns
