@@ -204,7 +204,7 @@ mk_status default_binding(const Module& m, int lo, int hi, Binding& out, std::st
     int best_end = p;
     for (int end = hi; end > p && !best; --end) {
       for (const Impl& im : registry()) {
-        if (im.match(m, p, end)) { best = &im; best_end = end; break; }
+        if (im.default_pick && im.match(m, p, end)) { best = &im; best_end = end; break; }
       }
     }
     if (!best) {

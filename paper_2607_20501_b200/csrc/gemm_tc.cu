@@ -57,6 +57,10 @@ template <int STAGES> struct Shared {
   uint32_t tmem_base;
   int abort_flag;
   EpiProgram epi;   // the kernel parameter, copied once (see epi_copy_to_smem)
+  // fused row norm: first row of the 32-row block each epilogue warp completed with its last tile (-1: none),
+  // double-buffered by tile parity
+  long long fix_row0[2][EPI_WARPS];
+  uint64_t fix_bar;   // the epilogue warps meet here once per tile (bounded wait, like every other)
 };
 
 __device__ __forceinline__ void tile_coords(int t, int num_m, int num_n, int& mi, int& ni) {
@@ -69,11 +73,72 @@ __device__ __forceinline__ void tile_coords(int t, int num_m, int num_n, int& mi
   ni = r / gsz;
 }
 
-template <int CTAS, bool SWIGLU>
+// Normalise rows [row0 + first, row0 + first + count) of the bf16 matrix out[M, N] in place, from the partial
+// sums every epilogue warp left behind.  One warp: lane l < count sums the partials of row l, then the whole
+// warp streams each row with all of a row's loads in flight at once (16 bytes per lane, read through L2:
+// other SMs wrote these bytes; a load-compute-store loop would pay one L2 round trip per 512 bytes).
+__device__ __forceinline__ void rownorm_fixup(const RowNormArgs& na, __nv_bfloat16* out, int64_t row0, int first, int count, int M, int N,
+                                              int slots, int lane) {
+  const int64_t my = row0 + first + lane;
+  float sm = 0.0f, sq = 0.0f;
+  if (lane < count && my < M) {
+    const float2* p = reinterpret_cast<const float2*>(na.partials) + my * slots;
+    for (int k = 0; k < slots; ++k) {
+      const float2 v = __ldcg(p + k);
+      sm += v.x;
+      sq += v.y;
+    }
+  }
+  const float inv_n = 1.0f / (float)N;
+  const float mean = na.mode == ROW_LAYERNORM ? sm * inv_n : 0.0f;
+  const float rstd = rsqrtf(fmaxf(sq * inv_n - mean * mean, 0.0f) + na.eps);
+  const __nv_bfloat16* gamma = reinterpret_cast<const __nv_bfloat16*>(na.gamma);
+  const __nv_bfloat16* beta = na.mode == ROW_LAYERNORM ? reinterpret_cast<const __nv_bfloat16*>(na.beta) : nullptr;
+#pragma unroll 1
+  for (int r = 0; r < count; ++r) {
+    const int64_t gr = row0 + first + r;
+    if (gr >= M) break;
+    const float mr = __shfl_sync(0xffffffffu, mean, r), rs = __shfl_sync(0xffffffffu, rstd, r);
+    __nv_bfloat16* rowp = out + gr * N;
+#pragma unroll 1
+    for (int base = 0; base < N; base += 8 * 256) {
+      uint4 raw[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int c0 = base + u * 256 + lane * 8;
+        if (c0 < N) raw[u] = __ldcg(reinterpret_cast<const uint4*>(rowp + c0));
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int c0 = base + u * 256 + lane * 8;
+        if (c0 >= N) continue;
+        const uint32_t w[4] = {raw[u].x, raw[u].y, raw[u].z, raw[u].w};
+        float x[8], g[8], b[8];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          x[2 * k] = __uint_as_float(w[k] << 16);
+          x[2 * k + 1] = __uint_as_float(w[k] & 0xffff0000u);
+        }
+        if (gamma) ld_vec(gamma + c0, g);
+        if (beta) ld_vec(beta + c0, b);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          float y = (x[k] - mr) * rs;
+          if (gamma) y *= g[k];
+          if (beta) y += b[k];
+          x[k] = y;
+        }
+        st_vec(rowp + c0, x);
+      }
+    }
+  }
+}
+
+template <int CTAS, bool SWIGLU, bool NORM = false>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmBh,
                void* __restrict__ out, int out_f32, int M, int N, int K, int up_row_offset, int tail_first,
-               const __grid_constant__ EpiProgram epi_param, unsigned int* status) {
+               const __grid_constant__ EpiProgram epi_param, const __grid_constant__ RowNormArgs na, unsigned int* status) {
   using C = Cfg<CTAS>;
   constexpr int STAGES = C::STAGES;
   constexpr int OUT_N = SWIGLU ? BN / 2 : BN;  // output columns per tile
@@ -106,6 +171,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { tc::mbar_init(&sh->full[s], 1); tc::mbar_init(&sh->empty[s], 1); }
     for (int b = 0; b < 2; ++b) { tc::mbar_init(&sh->tfull[b], 1); tc::mbar_init(&sh->tempty[b], EPI_WARPS * CTAS); }
+    tc::mbar_init(&sh->fix_bar, EPI_WARPS);
     sh->abort_flag = 0;
     tc::fence_barrier_init();
     tc::tma_prefetch_desc(&tmA);
@@ -254,6 +320,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       if (threadIdx.x == 64) MK_TR(3 + it * 8);  // epilogue: accumulator ready
       tc::tc_fence_after();
       const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN;
+      float rsum = 0.0f, rsq = 0.0f;   // NORM: this lane's row, over the columns this warp stores
 #pragma unroll 1
       for (int c = half; c < chunks_here; c += 2) {
         uint32_t r[32];
@@ -269,6 +336,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           for (int j = 0; j < 32; ++j) v[j] = silu_fast(v[j]) * __uint_as_float(r[j]);
         }
         ew.chunk_out(epi, v, rowmap, out, col_base + c * 32, c * 32, (int64_t)N, res_regs, c + 2 < chunks_here ? col_base + (c + 2) * 32 : -1);
+        if (NORM) {
+          // v now holds the values after the elementwise tail (what was just stored, before its bf16 rounding)
+          const int64_t c0 = col_base + c * 32;
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (c0 + j < N) { rsum += v[j]; rsq = fmaf(v[j], v[j], rsq); }
+        }
       }
       tc::tc_fence_before();
       __syncwarp();
@@ -276,6 +350,35 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       if (lane == 0) {
         if (CTAS == 2) tc::mbar_arrive_cluster(tc::map_to_cta(tc::smem_u32(&sh->tempty[acc]), 0));
         else tc::mbar_arrive(&sh->tempty[acc]);
+      }
+      if (NORM) {
+        // partial sums of this warp's share of the rows, then count this warp in; the warp that completes the
+        // block of 32 rows (2 * column tiles arrivals: both column halves of every tile) normalises it
+        const int slots = 2 * num_n;
+        const int64_t my = row0 + lane;
+        if (my < M) reinterpret_cast<float2*>(na.partials)[my * slots + ni * 2 + half] = make_float2(rsum, rsq);
+        __threadfence();
+        __syncwarp();
+        int old = 0;
+        if (lane == 0) old = atomicAdd(na.counters + ((mi * CTAS + (int)rank) * 4 + q), 1);
+        old = __shfl_sync(0xffffffffu, old, 0);
+        // A completed block is normalised by all eight epilogue warps of this CTA together (four rows each): one
+        // warp alone would spend tens of microseconds on it.  Every warp posts what it completed, the warps
+        // meet, and each takes its rows of every posted block.
+        const int ew_id = warp - 2;
+        if (lane == 0) sh->fix_row0[it & 1][ew_id] = old == slots - 1 ? (long long)row0 : -1LL;
+        __syncwarp();
+        if (lane == 0) tc::mbar_arrive(&sh->fix_bar);
+        ok = tc::mbar_wait(&sh->fix_bar, it & 1, abort_flag, status, tc::WAIT_TMEM_FULL);
+        ok = __all_sync(0xffffffffu, ok ? 1 : 0) != 0;
+        if (!ok) break;
+#pragma unroll 1
+        for (int w_ = 0; w_ < EPI_WARPS; ++w_) {
+          const long long fr = sh->fix_row0[it & 1][w_];
+          if (fr < 0) continue;
+          __threadfence();
+          rownorm_fixup(na, reinterpret_cast<__nv_bfloat16*>(out), fr, ew_id * (32 / EPI_WARPS), 32 / EPI_WARPS, M, N, slots, lane);
+        }
       }
     }
   }
@@ -350,12 +453,61 @@ cudaError_t launch_impl(const GemmTcPlan& p, cudaStream_t s) {
   const int out_f32 = p.out_f32 ? 1 : 0;
   if (p.swiglu)
     return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<CTAS, true>, p.tm_a, p.tm_b, p.tm_b_half, p.out, out_f32, p.m, p.n, p.k, p.n, p.tail_first, p.epi,
-                              status);
+                              p.norm, status);
   return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<CTAS, false>, p.tm_a, p.tm_b, p.tm_b_half, p.out, out_f32, p.m, p.n, p.k, 0, p.tail_first, p.epi,
-                            status);
+                            p.norm, status);
+}
+
+cudaError_t launch_norm_impl(const GemmTcPlan& p, cudaStream_t s) {
+  static bool attr_done = false;
+  if (!attr_done) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<2, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<2>::SMEM);
+    if (e != cudaSuccess) return e;
+    attr_done = true;
+  }
+  const int64_t row_blocks = ((p.m + 2 * BM - 1) / (2 * BM)) * 2 * 4;
+  cudaError_t e = cudaMemsetAsync(p.norm.counters, 0, (size_t)row_blocks * sizeof(int), s);
+  if (e != cudaSuccess) return e;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)p.grid);
+  cfg.blockDim = dim3(THREADS);
+  cfg.dynamicSmemBytes = Cfg<2>::SMEM;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<2, false, true>, p.tm_a, p.tm_b, p.tm_b_half, p.out, 0, p.m, p.n, p.k, 0, p.tail_first, p.epi, p.norm,
+                            kernel_status_ptr());
 }
 
 }  // namespace
+
+size_t gemm_rownorm_tc2_scratch(int64_t m, int64_t n) {
+  const int64_t num_n = (n + BN - 1) / BN, num_m = (m + 2 * BM - 1) / (2 * BM);
+  const size_t partials = (size_t)m * (size_t)(2 * num_n) * sizeof(float2);
+  return (partials + 255) / 256 * 256 + (size_t)num_m * 2 * 4 * sizeof(int);
+}
+cudaError_t gemm_rownorm_tc2_plan(GemmTcPlan* p, const void* a, const void* w_nk, void* y, int64_t m, int64_t n, int64_t k,
+                                  const EpiProgram& epi, int mode, const void* gamma, const void* beta, float eps, void* scratch,
+                                  int sm_count) {
+  cudaError_t e = plan_impl<2>(p, a, w_nk, y, false, m, n, k, false, epi, sm_count);
+  if (e != cudaSuccess) return e;
+  p->tail_first = (int)(((m + 2 * BM - 1) / (2 * BM)) * ((n + BN - 1) / BN));   // whole tiles only: the arrival count assumes it
+  const int64_t num_n = (n + BN - 1) / BN;
+  const size_t partials = (size_t)m * (size_t)(2 * num_n) * sizeof(float2);
+  p->norm.partials = reinterpret_cast<float*>(scratch);
+  p->norm.counters = reinterpret_cast<int*>(reinterpret_cast<char*>(scratch) + (partials + 255) / 256 * 256);
+  p->norm.gamma = gamma;
+  p->norm.beta = beta;
+  p->norm.eps = eps;
+  p->norm.mode = mode;
+  return cudaSuccess;
+}
+cudaError_t launch_gemm_rownorm_tc2(const GemmTcPlan& p, cudaStream_t s) { return launch_norm_impl(p, s); }
 
 cudaError_t gemm_tc_plan(GemmTcPlan* p, const void* a, const void* w_nk, void* y, bool out_f32, int64_t m, int64_t n, int64_t k, bool swiglu,
                          const EpiProgram& epi, int sm_count) {

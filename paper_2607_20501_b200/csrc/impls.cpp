@@ -194,6 +194,45 @@ mk_status gemm_tc2_emit(const Module& m, int lo, int hi, const Resolved& r, std:
   return gemm_tc_emit_impl(m, lo, hi, r, out, err, true);
 }
 
+// LINEAR [elementwise]* (LAYERNORM | RMSNORM) on the tensor cores: the norm's statistics come out of the GEMM's
+// epilogue and the warp that completes a block of rows normalises it in place - the paper's projection +
+// residual + norm fusion at tensor-core shape, without a pass of its own over the activation.
+bool gemm_rownorm_tc2_match(const Module& m, int lo, int hi) {
+  if (hi - lo < 2 || !is_chain(m, lo, hi)) return false;
+  const int32_t k = m.ops[hi - 1].d.kind;
+  if (k != MK_OP_LAYERNORM && k != MK_OP_RMSNORM) return false;
+  if (!gemm_tc2_match(m, lo, hi - 1)) return false;
+  bool sw; int t;
+  if (!gemm_shape(m, lo, hi - 1, &sw, &t) || sw) return false;
+  // the value handed to the norm and the norm's result are both bf16 (the row is normalised in place)
+  if (m.vspec(m.ops[hi - 2].out_id).dtype != MK_BF16 || m.vspec(m.ops[hi - 1].out_id).dtype != MK_BF16) return false;
+  const int64_t N = last_dim(m.vspec(m.ops[hi - 1].out_id));
+  return N <= 16384;
+}
+size_t gemm_rownorm_tc2_scratch_fn(const Module& m, int lo, int hi) {
+  const mk_tensor_spec& xs = m.vspec(m.ops[lo].in_id[0]);
+  return gemm_rownorm_tc2_scratch(xs.shape[0], last_dim(m.vspec(m.ops[hi - 1].out_id)));
+}
+mk_status gemm_rownorm_tc2_emit(const Module& m, int lo, int hi, const Resolved& r, std::vector<Launch>& out, std::string& err) {
+  bool sw; int t;
+  gemm_shape(m, lo, hi - 1, &sw, &t);
+  EpiProgram p;
+  mk_status st = build_epi(m, t, hi - 1, r, p, err);
+  if (st != MK_OK) return st;
+  const Op& op = m.ops[lo];
+  const Op& nop = m.ops[hi - 1];
+  const mk_tensor_spec& xs = m.vspec(op.in_id[0]);
+  const int64_t M = xs.shape[0], K = xs.shape[1], N = last_dim(m.vspec(nop.out_id));
+  const void* g = nop.param[0].set ? nop.param[0].ptr : nullptr;
+  const void* b = nop.param[1].set ? nop.param[1].ptr : nullptr;
+  auto plan = std::make_shared<GemmTcPlan>();
+  cudaError_t e = gemm_rownorm_tc2_plan(plan.get(), r.value_ptr[op.in_id[0]], op.param[0].ptr, r.value_ptr[nop.out_id], M, N, K, p,
+                                        row_mode(nop.d.kind), g, b, (float)nop.d.f[0], r.scratch, m.ctx->sm_count);
+  if (e != cudaSuccess) { err = std::string("gemm_rownorm_tc2 plan: ") + cudaGetErrorString(e); return MK_ERR_CUDA; }
+  out.push_back([plan](cudaStream_t s) { return launch_gemm_rownorm_tc2(*plan, s); });
+  return MK_OK;
+}
+
 // LINEAR [elementwise]* (LAYERNORM | RMSNORM), fp32, one CTA owns whole rows
 bool linear_rownorm_match(const Module& m, int lo, int hi) {
   if (hi - lo < 2 || !is_chain(m, lo, hi) || m.ops[lo].d.kind != MK_OP_LINEAR) return false;
@@ -380,6 +419,7 @@ mk_status attn_simt_emit(const Module& m, int lo, int, const Resolved& r, std::v
 const std::vector<Impl>& registry() {
   static const std::vector<Impl> reg = {
       {"linear_rownorm_simt", linear_rownorm_match, no_scratch, linear_rownorm_emit},
+      {"gemm_rownorm_tc2", gemm_rownorm_tc2_match, gemm_rownorm_tc2_scratch_fn, gemm_rownorm_tc2_emit, false},
       {"gemm_tc2", gemm_tc2_match, no_scratch, gemm_tc2_emit},
       {"gemm_tc", gemm_tc_match, no_scratch, gemm_tc_emit},
       {"gemm_simt", gemm_simt_match, no_scratch, gemm_simt_emit},

@@ -59,6 +59,9 @@ struct Impl {
   // Append the piece's kernel launches.
   mk_status (*emit)(const Module& m, int lo, int hi, const Resolved& r, std::vector<Launch>& out,
                     std::string& err);
+  // false: legal and bindable by name (and a candidate for Swap, which decides by measured time), but the
+  // composer's default cover does not pick it - for variants that are not (yet) faster than what they replace
+  bool default_pick = true;
 };
 const std::vector<Impl>& registry();
 

@@ -263,6 +263,7 @@ struct EpiWarp {
         for (int j = 0; j < 32; ++j)
           if (col0 + j < n_cols) {
             const float r = epi_apply(epi, v[j], my_row, col0 + j, n_cols);
+            v[j] = r;   // callers that go on with the chunk (row statistics) see the values after the tail
             if (out_f32) reinterpret_cast<float*>(out)[my_row * n_cols + col0 + j] = r;
             else reinterpret_cast<__nv_bfloat16*>(out)[my_row * n_cols + col0 + j] = __float2bfloat16_rn(r);
           }

@@ -8,8 +8,21 @@
 
 namespace mk {
 
+// Row norm fused behind the GEMM's tail (LayerNorm or RMSNorm over the whole output row, which spans
+// several tiles): every epilogue warp leaves per-row partial sums of what it stores and counts itself
+// in; the warp that completes a block of 32 rows normalises those rows in place.
+struct RowNormArgs {
+  float* partials = nullptr;   // [m][2 * column tiles][2] = (sum, sum of squares) per row and epilogue-warp slot
+  int* counters = nullptr;     // [row blocks of 32]; zeroed before every launch
+  const void* gamma = nullptr; // bf16 [n] or null
+  const void* beta = nullptr;  // bf16 [n] or null (LayerNorm only)
+  float eps = 0.f;
+  int mode = 0;                // RowMode
+};
+
 struct GemmTcPlan {
   CUtensorMap tm_a, tm_b;
+  RowNormArgs norm;         // used by the fused GEMM + row norm form only
   CUtensorMap tm_b_half;    // W with a box of half as many rows, for the half-width units of the last wave
   int tail_first = 0;       // tiles from this index on run as two half-width units (= tile count: none)
   void* out = nullptr;
@@ -32,6 +45,12 @@ namespace mk {
 cudaError_t gemm_tc2_plan(GemmTcPlan* p, const void* a, const void* w_nk, void* y, bool out_f32, int64_t m, int64_t n, int64_t k, bool swiglu,
                           const EpiProgram& epi, int sm_count);
 cudaError_t launch_gemm_tc2(const GemmTcPlan& p, cudaStream_t s);
+// Fused GEMM + tail + row norm (bf16 out).  Scratch: gemm_rownorm_tc2_scratch(m, n) bytes, laid out by the plan.
+size_t gemm_rownorm_tc2_scratch(int64_t m, int64_t n);
+cudaError_t gemm_rownorm_tc2_plan(GemmTcPlan* p, const void* a, const void* w_nk, void* y, int64_t m, int64_t n, int64_t k,
+                                  const EpiProgram& epi, int mode, const void* gamma, const void* beta, float eps, void* scratch,
+                                  int sm_count);
+cudaError_t launch_gemm_rownorm_tc2(const GemmTcPlan& p, cudaStream_t s);
 }  // namespace mk
 
 namespace mk {
