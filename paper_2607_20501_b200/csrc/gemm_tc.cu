@@ -137,7 +137,7 @@ __device__ __forceinline__ void rownorm_fixup(const RowNormArgs& na, __nv_bfloat
 template <int CTAS, bool SWIGLU, bool NORM = false>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmBh,
-               void* __restrict__ out, int out_f32, int M, int N, int K, int up_row_offset, int tail_first,
+               const __grid_constant__ CUtensorMap tmOut, int bulk_store, void* __restrict__ out, int out_f32, int M, int N, int K, int up_row_offset, int tail_first,
                const __grid_constant__ EpiProgram epi_param, const __grid_constant__ RowNormArgs na, unsigned int* status) {
   using C = Cfg<CTAS>;
   constexpr int STAGES = C::STAGES;
@@ -335,7 +335,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
           for (int j = 0; j < 32; ++j) v[j] = silu_fast(v[j]) * __uint_as_float(r[j]);
         }
-        ew.chunk_out(epi, v, rowmap, out, col_base + c * 32, c * 32, (int64_t)N, res_regs, c + 2 < chunks_here ? col_base + (c + 2) * 32 : -1);
+        ew.chunk_out(epi, v, rowmap, out, col_base + c * 32, c * 32, (int64_t)N, res_regs, c + 2 < chunks_here ? col_base + (c + 2) * 32 : -1,
+                     (!NORM && bulk_store) ? &tmOut : nullptr, row0);
         if (NORM) {
           // v now holds the values after the elementwise tail (what was just stored, before its bf16 rounding)
           const int64_t c0 = col_base + c * 32;
@@ -381,6 +382,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
       }
     }
+    if (lane == 0) tc::tma_store_wait_all();   // bulk stores of this warp are complete before the CTA retires
   }
 
   MK_TR_PRINT("gemm");
@@ -414,6 +416,14 @@ cudaError_t plan_impl(GemmTcPlan* p, const void* a, const void* w_nk, void* y, b
   if (e != cudaSuccess) return e;
   p->out = y;
   p->out_f32 = out_f32;
+  p->use_tm_out = false;
+  if (!out_f32) {
+    e = encode_tmap_2d_bf16_store(&p->tm_out, y, (uint64_t)m, (uint64_t)n, (uint64_t)n);
+    if (e != cudaSuccess) return e;
+    p->use_tm_out = true;
+  } else {
+    p->tm_out = p->tm_a;   // never read
+  }
   p->m = (int)m; p->n = (int)n; p->k = (int)k;
   p->swiglu = swiglu;
   p->epi = epi;
@@ -452,9 +462,9 @@ cudaError_t launch_impl(const GemmTcPlan& p, cudaStream_t s) {
   unsigned int* status = kernel_status_ptr();
   const int out_f32 = p.out_f32 ? 1 : 0;
   if (p.swiglu)
-    return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<CTAS, true>, p.tm_a, p.tm_b, p.tm_b_half, p.out, out_f32, p.m, p.n, p.k, p.n, p.tail_first, p.epi,
+    return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<CTAS, true>, p.tm_a, p.tm_b, p.tm_b_half, p.tm_out, p.use_tm_out ? 1 : 0, p.out, out_f32, p.m, p.n, p.k, p.n, p.tail_first, p.epi,
                               p.norm, status);
-  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<CTAS, false>, p.tm_a, p.tm_b, p.tm_b_half, p.out, out_f32, p.m, p.n, p.k, 0, p.tail_first, p.epi,
+  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<CTAS, false>, p.tm_a, p.tm_b, p.tm_b_half, p.tm_out, p.use_tm_out ? 1 : 0, p.out, out_f32, p.m, p.n, p.k, 0, p.tail_first, p.epi,
                             p.norm, status);
 }
 
@@ -480,7 +490,7 @@ cudaError_t launch_norm_impl(const GemmTcPlan& p, cudaStream_t s) {
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<2, false, true>, p.tm_a, p.tm_b, p.tm_b_half, p.out, 0, p.m, p.n, p.k, 0, p.tail_first, p.epi, p.norm,
+  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<2, false, true>, p.tm_a, p.tm_b, p.tm_b_half, p.tm_out, 0, p.out, 0, p.m, p.n, p.k, 0, p.tail_first, p.epi, p.norm,
                             kernel_status_ptr());
 }
 

@@ -123,6 +123,18 @@ __device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* m, uin
       : "memory");
 }
 
+// Bulk tensor store shared -> global (asynchronous; rows and columns outside the tensor are clipped).  The
+// issuing thread tracks its stores in bulk groups: wait_read = the source buffer may be rewritten,
+// wait_all = the stores are complete.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* m, const void* src, int32_t x, int32_t y) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(reinterpret_cast<uint64_t>(m)),
+               "r"(smem_u32(src)), "r"(x), "r"(y)
+               : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
 // ---------------------------------------------------------------- TMEM
 __device__ __forceinline__ void tmem_alloc(uint32_t* smem_slot, uint32_t ncols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_slot)), "r"(ncols) : "memory");
@@ -343,5 +355,7 @@ cudaError_t encode_tmap_2d_bf16(CUtensorMap* out, const void* base, uint64_t row
 // General bf16 map: dims/strides innermost first (strides in bytes for dims 1..rank-1).
 cudaError_t encode_tmap_bf16(CUtensorMap* out, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
                              const uint32_t* box, bool swizzle128);
+// bf16 [rows, cols] output map for the epilogue's bulk stores: box 32 x 32, 64-byte swizzle
+cudaError_t encode_tmap_2d_bf16_store(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint64_t ld);
 
 }  // namespace mk

@@ -211,15 +211,37 @@ struct EpiWarp {
     }
     __syncwarp();
   }
+  // this lane's own 64 bytes -> staging (64-byte rows, the bulk store's 64-byte swizzle) -> one asynchronous
+  // bulk tensor store of the 32 x 64-byte block at column x (elements), row y; lane 0 issues and tracks it.
+  // Rows and columns beyond the tensor are clipped by the copy engine.
+  __device__ __forceinline__ void own_row_to_global_bulk(const uint4 (&mine)[4], const CUtensorMap* tm, int32_t x, int32_t y) {
+    const int f = (lane >> 1) & 3;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) *reinterpret_cast<uint4*>(stage + lane * 64 + ((i ^ f) * 16)) = mine[i];
+    tc::fence_proxy_async();
+    __syncwarp();
+    if (lane == 0) {
+      tc::tma_store_2d(tm, stage, x, y);
+      tc::tma_store_commit();
+    }
+  }
   // One chunk: program, pack, transposed coalesced store.
   //   v            the lane's fp32 values for columns [col0, col0 + 32) of its row
   //   bias_off     offset (elements) of col0 inside the bias slice loaded by load_bias
   //   rowmap(r)    global row of warp-local row r in [0, 32), or -1 if that row is not stored
   //   res_regs     this chunk's residual (from prefetch_res); on return the next chunk's, if next_col0 >= 0
   template <typename RowMap>
+  //   tm_store     if not null (bf16 output, rows of the warp consecutive from global row y0): the block leaves by a
+  //                bulk tensor store instead of 16-byte stores
   __device__ __forceinline__ void chunk_out(const EpiProgram& epi, float (&v)[32], RowMap rowmap, void* __restrict__ out_v, int64_t col0,
-                                            int bias_off, int64_t n_cols, uint4 (&res_regs)[8], int64_t next_col0) {
+                                            int bias_off, int64_t n_cols, uint4 (&res_regs)[8], int64_t next_col0,
+                                            const CUtensorMap* tm_store = nullptr, int64_t y0 = 0) {
     if (col0 >= n_cols) return;  // warp-uniform
+    if (tm_store) {
+      // the previous chunk's bulk store has finished reading the staging buffer (the residual slabs go through it too)
+      if (lane == 0) tc::tma_store_wait_read();
+      __syncwarp();
+    }
     const int64_t my_row = rowmap(lane);
     uint8_t* out = reinterpret_cast<uint8_t*>(out_v);
     if (col0 + 32 <= n_cols) {
@@ -244,7 +266,8 @@ struct EpiWarp {
           mine[j].z = pack_bf16x2(v[8 * j + 4], v[8 * j + 5]);
           mine[j].w = pack_bf16x2(v[8 * j + 6], v[8 * j + 7]);
         }
-        own_row_to_global(mine, rowmap, out, n_cols * 2, col0 * 2);
+        if (tm_store) own_row_to_global_bulk(mine, tm_store, (int32_t)col0, (int32_t)y0);
+        else own_row_to_global(mine, rowmap, out, n_cols * 2, col0 * 2);
       } else {
 #pragma unroll
         for (int j = 0; j < 4; ++j)

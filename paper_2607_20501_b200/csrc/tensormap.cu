@@ -56,4 +56,19 @@ cudaError_t encode_tmap_2d_bf16(CUtensorMap* out, const void* base, uint64_t row
   return encode_tmap_bf16(out, base, 2, dims, strides, box, true);
 }
 
+// Output map for the epilogue's bulk stores: bf16 [rows, cols] row-major, box 32 rows x 32 columns (64 bytes),
+// 64-byte swizzle (the 16-byte segment s of row r sits at segment s ^ ((r >> 1) & 3) in shared memory).
+cudaError_t encode_tmap_2d_bf16_store(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint64_t ld) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return cudaErrorNotSupported;
+  if (((uintptr_t)base & 15) != 0 || (ld * 2) % 16) return cudaErrorInvalidValue;
+  cuuint64_t gdim[2] = {cols, rows};
+  cuuint64_t gstr[1] = {ld * 2};
+  cuuint32_t bdim[2] = {32, 32};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstr, bdim, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
 }  // namespace mk
