@@ -388,6 +388,25 @@ __device__ __forceinline__ void role_mma(const Ctx& cx, uint32_t tmem_base, int 
   }
 }
 
+// Two fp32 multiply-adds / adds in one instruction (sm_100 packed fp32): the softmax's issue slots are as
+// scarce as its special-function slots.
+__device__ __forceinline__ void fma2(float& d0, float& d1, float a0, float a1, float b, float c) {
+  asm("{\n\t.reg .b64 ra, rb, rc, rd;\n\t"
+      "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %4};\n\tmov.b64 rc, {%5, %5};\n\t"
+      "fma.rn.f32x2 rd, ra, rb, rc;\n\t"
+      "mov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(d0), "=f"(d1)
+      : "f"(a0), "f"(a1), "f"(b), "f"(c));
+}
+__device__ __forceinline__ void add2(float& s0, float& s1, float a0, float a1) {
+  asm("{\n\t.reg .b64 ra, rs;\n\t"
+      "mov.b64 ra, {%2, %3};\n\tmov.b64 rs, {%0, %1};\n\t"
+      "add.rn.f32x2 rs, rs, ra;\n\t"
+      "mov.b64 {%0, %1}, rs;\n\t}"
+      : "+f"(s0), "+f"(s1)
+      : "f"(a0), "f"(a1));
+}
+
 // ------------------------------------------------------------------------------------------ softmax
 // One thread per query row of stream T.  m is the reference maximum in log2 units (scores times
 // scale * log2 e): p = exp2(s * scale*log2e - m).  Any m gives the same O / l as long as nothing
@@ -514,9 +533,10 @@ __device__ __forceinline__ void role_softmax(const Ctx& cx, uint32_t tmem_base, 
           tc::tmem_ld_wait();
 #pragma unroll
           for (int i = 0; i < 32; i += 2) {
-            const float p0 = tc::ex2_fast(fmaf(__uint_as_float(r[i]), scale_log2, neg_m));
-            const float p1 = tc::ex2_fast(fmaf(__uint_as_float(r[i + 1]), scale_log2, neg_m));
-            sum4[(i >> 1) & 3] += p0 + p1;
+            float x0, x1;
+            fma2(x0, x1, __uint_as_float(r[i]), __uint_as_float(r[i + 1]), scale_log2, neg_m);
+            const float p0 = tc::ex2_fast(x0), p1 = tc::ex2_fast(x1);
+            add2(sum4[(i >> 1) & 1 ? 2 : 0], sum4[(i >> 1) & 1 ? 3 : 1], p0, p1);
             pk[c * 16 + (i >> 1)] = pack_bf16x2(p0, p1);
           }
         }
@@ -551,9 +571,10 @@ __device__ __forceinline__ void role_softmax(const Ctx& cx, uint32_t tmem_base, 
           tc::tmem_ld_wait();
 #pragma unroll
           for (int i = 0; i < 32; i += 2) {
-            const float p0 = tc::ex2_fast(fmaf(__uint_as_float(r[i]), scale_log2, neg_m));
-            const float p1 = tc::ex2_fast(fmaf(__uint_as_float(r[i + 1]), scale_log2, neg_m));
-            sum4[(i >> 1) & 3] += p0 + p1;
+            float x0, x1;
+            fma2(x0, x1, __uint_as_float(r[i]), __uint_as_float(r[i + 1]), scale_log2, neg_m);
+            const float p0 = tc::ex2_fast(x0), p1 = tc::ex2_fast(x1);
+            add2(sum4[(i >> 1) & 1 ? 2 : 0], sum4[(i >> 1) & 1 ? 3 : 1], p0, p1);
             pk[32 + c * 16 + (i >> 1)] = pack_bf16x2(p0, p1);
           }
         }
