@@ -39,7 +39,7 @@ NCU_TRAFFIC_BYTES = {"c2": 105.7e6,            # profiles/gemm_tc2_c2.md
                      "c3": 26.25e6,            # profiles/conv3x3_tc2_groupnorm_c3.md (conv; its output stays in L2)
                      "c4": 8 * 52.2e6}         # profiles/attention_tc2_c4.md
 
-DEFAULT_STEPS = {"c1": 2000, "c2": 200, "c3": 400, "c4": 100, "c5": 50}
+DEFAULT_STEPS = {"c1": 2000, "c2": 200, "c3": 400, "c4": 100, "c5": 50, "c6": 100}
 
 
 def full_workload(name, seed=0, batch=None, only_ops=None):
@@ -48,7 +48,8 @@ def full_workload(name, seed=0, batch=None, only_ops=None):
     import workloads as W
     kw = {}
     if batch is not None:
-        kw = {"c1": {"M": batch}, "c2": {"M": batch}, "c3": {"NB": batch}, "c4": {"B": batch}, "c5": {"B": batch}}[name]
+        kw = {"c1": {"M": batch}, "c2": {"M": batch}, "c3": {"NB": batch}, "c4": {"B": batch}, "c5": {"B": batch},
+              "c6": {"B": batch}}[name]
     w = W.generate.WORKLOADS[name](seed, **kw)
     if only_ops is not None:
         w.ops = w.ops[:only_ops]
@@ -154,16 +155,16 @@ def oracle_sample(name, w, budget_s=12.0):
             total = b_total
             what = f"first {frac_units} of {total} batch elements"
         else:
-            attn = [o for o in w.ops if o["kind"] == "attention_causal"][0]["attrs"]
+            attn = [o for o in w.ops if o["kind"] in ("attention_causal", "attention")][0]["attrs"]
             sq, total = attn["seq"], attn["batch"]
             s.inputs["x"] = Tensor("x", w.dtype, w.inputs["x"].store[: frac_units * sq])
             for o in s.ops:
-                if o["kind"] == "attention_causal":
+                if o["kind"] in ("attention_causal", "attention"):
                     o["attrs"]["batch"] = frac_units
             what = f"first {frac_units} of {total} batch elements"
         return s, total, what
 
-    probe_units = {"c1": 64, "c2": 64, "c3": 1, "c4": 1, "c5": 1}[name]
+    probe_units = {"c1": 64, "c2": 64, "c3": 1, "c4": 1, "c5": 1, "c6": 1}[name]
     s, total, _ = sub(probe_units)
     t0 = time.perf_counter()
     OM.run_workload(s, [0])
@@ -205,13 +206,14 @@ def submodule_work(w, module):
                 fl += 2.0 * xs[0] * xs[1] * op["attrs"]["n"]
             elif op["kind"] == "conv2d_3x3":
                 fl += 2.0 * xs[0] * xs[1] * xs[2] * 9 * xs[3] * op["attrs"]["c_out"]
-            elif op["kind"] == "attention_causal":
+            elif op["kind"] in ("attention_causal", "attention"):
                 a = op["attrs"]
                 if a["layout"] == "bhsd":
                     b_, h_, sq, d_ = xs
                 else:
                     b_, sq, h_, d_ = a["batch"], a["seq"], a["heads"], a["head_dim"]
-                fl += 4.0 * b_ * h_ * d_ * (sq * (sq + 1) / 2)
+                # causal: the exact j <= i triangle; unmasked: every (query, key) pair
+                fl += 4.0 * b_ * h_ * d_ * (sq * (sq + 1) / 2 if op["kind"] == "attention_causal" else sq * sq)
         out.append((fl, by))
     return out
 
@@ -395,7 +397,7 @@ def run_ours(args):
     # (time, share, algorithmic work, roofline fraction of that subkernel)
     breakdown = None
     dominant = None
-    split_name = {"c1": "split", "c2": "split", "c3": "split2", "c4": "split3", "c5": "fused_tails"}.get(name)
+    split_name = {"c1": "split", "c2": "split", "c3": "split2", "c4": "split3", "c5": "fused_tails", "c6": "fused_tails"}.get(name)
     if rank == 0 and split_name in w.partitions:
         pk_ = peaks()
         dw = sets[0]
@@ -474,7 +476,7 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c2", choices=["c1", "c2", "c3", "c4", "c5"])
+    ap.add_argument("--workload", default="c2", choices=["c1", "c2", "c3", "c4", "c5", "c6"])
     ap.add_argument("--decomposition", default=None)
     ap.add_argument("--batch", type=int, default=None, help="smaller leading batch dimension (profiler captures)")
     ap.add_argument("--only-ops", type=int, default=None, help="run the first N operators alone (profiler captures)")

@@ -104,6 +104,8 @@ typedef struct mk_tensor_spec {
  *                   i[2] = B > 0: one input, packed [B*S, 3*H*D] with columns [Q | K | V],
  *                                 each head-major, and i[3] = S.
  *                   Output is the logical [B*S, H*D] matrix (head-major columns).
+ *   ATTENTION       the same without the mask: softmax(Q K^T / sqrt(D)) V over every key (the encoder
+ *                   attention of the paper's transformer-block example); attributes and layouts as above.
  * Definitions: the paper's subkernel listings (linear with W stored [K, N]; LayerNorm; online-
  * softmax attention) and its correctness appendix (safe softmax, tril(diagonal=0) mask, fp32
  * accumulation); RMSNorm, GroupNorm, SwiGLU, tanh-GELU and the 3x3 convolution follow the
@@ -124,7 +126,8 @@ typedef enum {
   MK_OP_RMSNORM = 12,
   MK_OP_GROUPNORM = 13,
   MK_OP_SOFTMAX = 14,
-  MK_OP_ATTENTION_CAUSAL = 15
+  MK_OP_ATTENTION_CAUSAL = 15,
+  MK_OP_ATTENTION = 16
 } mk_op_kind;
 
 /* Value numbering: module input k has id k; operator j produces id n_inputs + j.

@@ -53,6 +53,10 @@ def apply_op(op, vals, params):
         if a["layout"] == "bhsd":
             return O.attention_causal_bhsd(ins[0], ins[1], ins[2])
         return O.attention_causal_packed(ins[0], a["batch"], a["seq"], a["heads"], a["head_dim"])
+    if kind == "attention":
+        if a["layout"] == "bhsd":
+            return O.attention_bhsd(ins[0], ins[1], ins[2])
+        return O.attention_packed(ins[0], a["batch"], a["seq"], a["heads"], a["head_dim"])
     raise ValueError(f"unknown operator kind {kind!r}")
 
 

@@ -203,3 +203,32 @@ def attention_causal_packed(qkv, batch, seq, heads, head_dim):
     k = np.ascontiguousarray(t[:, :, 1].transpose(0, 2, 1, 3))
     v = np.ascontiguousarray(t[:, :, 2].transpose(0, 2, 1, 3))
     return attention_causal_bhsd(q, k, v)
+
+
+def attention_bhsd(q, k, v):
+    """Unmasked (encoder) attention: q, k, v [B, H, S, D]; S_ij = (q_i . k_j)/sqrt(D) for every
+    pair; P = softmax over keys; O = P V.  This is the paper's transformer-block attention
+    (its ConvolutionalVisionTransformer example): scale, softmax over all keys, weighted sum.
+    Returns the logical [B*S, H*D] matrix, head-major columns."""
+    q, k, v = _f64(q), _f64(k), _f64(v)
+    b, h, s, d = q.shape
+    out = np.empty((b, s, h, d), F64)
+    for bi in range(b):
+        for hi in range(h):
+            sc = (q[bi, hi] @ k[bi, hi].T) / np.sqrt(F64(d))
+            out[bi, :, hi, :] = softmax(sc) @ v[bi, hi]
+    return out.reshape(b * s, h * d)
+
+
+def attention_packed(qkv, batch, seq, heads, head_dim):
+    """qkv [B*S, 3*H*D] with columns [Q | K | V], each head-major.
+    Same computation as attention_bhsd; returns [B*S, H*D]."""
+    qkv = _f64(qkv)
+    e = heads * head_dim
+    if qkv.shape != (batch * seq, 3 * e):
+        raise ValueError("attention_packed: bad shape")
+    t = qkv.reshape(batch, seq, 3, heads, head_dim)
+    q = np.ascontiguousarray(t[:, :, 0].transpose(0, 2, 1, 3))
+    k = np.ascontiguousarray(t[:, :, 1].transpose(0, 2, 1, 3))
+    v = np.ascontiguousarray(t[:, :, 2].transpose(0, 2, 1, 3))
+    return attention_bhsd(q, k, v)

@@ -356,6 +356,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 }  // namespace
 
 bool attention_tc_supported(const AttnView& a) {
+  if (!a.causal) return false;
   if (a.D != HD || a.B < 1 || a.H < 1 || a.S < 1) return false;
   if ((a.ss * 2) % 16 || (a.sh * 2) % 16 || (a.sb * 2) % 16) return false;
   if (a.B * a.H * ((a.S + BQ - 1) / BQ) > INT32_MAX) return false;

@@ -1,4 +1,4 @@
-// K7, two-query-tile form: fused causal attention on tcgen05 / TMEM, head_dim 128, bf16 in, fp32 softmax
+// K7, two-query-tile form: fused attention (causal, or unmasked with a run-time flag) on tcgen05 / TMEM, head_dim 128, bf16 in, fp32 softmax
 // and accumulation.
 //
 //   O = softmax(mask_{j<=i}(Q K^T / sqrt(D))) V        online softmax, the S x S matrix never leaves the SM
@@ -19,7 +19,8 @@
 //                   V from shared memory, MN-major).  While one stream's softmax runs, the tensor pipe
 //                   works for the other.
 // TMEM (512 columns): S/P of stream 0 and 1 (2 x 128), O of stream 0 and 1 (2 x 128); O accumulates in TMEM.
-// The diagonal tile is masked (key > query -> -inf, diagonal kept); tiles right of it are never visited.
+// Causal: the diagonal tile is masked (key > query -> -inf, diagonal kept); tiles right of it are never visited.
+// Unmasked: every stream visits every key tile; only the keys past S in a ragged last tile are hidden.
 // Every mbarrier wait is bounded.
 #include "device_common.cuh"
 #include "tc_common.cuh"
@@ -65,7 +66,9 @@ struct Item {
 // query block P-1-s followed by block s.
 struct ItemIter {
   int sidx, half, n_super, SP, P, num_q, H;
-  __device__ __forceinline__ void init(int S, int B, int H_) {
+  bool causal;
+  __device__ __forceinline__ void init(int S, int B, int H_, bool causal_) {
+    causal = causal_;
     num_q = (S + BQ - 1) / BQ;
     P = (num_q + 1) / 2;
     SP = (P + 1) / 2;
@@ -91,8 +94,9 @@ struct ItemIter {
       it.b = bh / H;
       it.h = bh - it.b * H;
       it.q0 = p * 2 * BQ;
-      it.n0 = 2 * p + 1;
-      it.n1 = (2 * p + 1 < num_q) ? 2 * p + 2 : 0;
+      // causal: the query tile at index i sees key tiles 0..i; unmasked: every stream sees all of them
+      it.n0 = causal ? 2 * p + 1 : num_q;
+      it.n1 = (2 * p + 1 < num_q) ? (causal ? 2 * p + 2 : num_q) : 0;
       it.nk = it.n1 ? it.n1 : it.n0;
       return true;
     }
@@ -177,10 +181,10 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16
 // Order per item: Q0, K0, Q1, V0, K1, V1, ... : the order in which the slots come free (the MMAs retire
 // as QK(j) of both streams, PV(j) of both, QK(j+1) ...), so no load queues behind a slot that frees later.
 __device__ __forceinline__ void role_loader(const Ctx& cx, const CUtensorMap* tmQ, const CUtensorMap* tmK, const CUtensorMap* tmV,
-                                            uint8_t* q_tiles, uint8_t* k_tiles, uint8_t* v_tiles, int B, int H, int S) {
+                                            uint8_t* q_tiles, uint8_t* k_tiles, uint8_t* v_tiles, int B, int H, int S, bool causal) {
   Shared* sh = cx.sh;
   ItemIter iter;
-  iter.init(S, B, H);
+  iter.init(S, B, H, causal);
   Item it;
   uint32_t n_items[2] = {0, 0};
   uint32_t g = 0;   // key tiles loaded so far by this CTA (ring position)
@@ -231,7 +235,7 @@ __device__ __forceinline__ void role_loader(const Ctx& cx, const CUtensorMap* tm
 // released by two commit arrivals, one per stream (both from the same thread for a tile only it reads).
 // The stream index is a run-time value on purpose: one copy of the code for both warps.
 __device__ __forceinline__ void role_mma(const Ctx& cx, uint32_t tmem_base, int t, uint8_t* q_tiles, uint8_t* k_tiles, uint8_t* v_tiles, int B,
-                                         int H, int S) {
+                                         int H, int S, bool causal) {
   Shared* sh = cx.sh;
   constexpr uint32_t idesc_qk64 = tc::idesc_bf16_f32(BQ, 64, 0, 0);  // A, B K-major, half a key tile
   constexpr uint32_t idesc_pv = tc::idesc_bf16_f32(BQ, HD, 0, 1);    // B (= V) MN-major
@@ -255,7 +259,7 @@ __device__ __forceinline__ void role_mma(const Ctx& cx, uint32_t tmem_base, int 
     bool valid;
   };
   ItemIter iter;
-  iter.init(S, B, H);
+  iter.init(S, B, H, causal);
   uint32_t g_next = 0;
   auto next_item = [&](Pos& p) {
     Item it;
@@ -423,7 +427,7 @@ __device__ __forceinline__ void add2(float& s0, float& s1, float a0, float a1) {
 // O may be touched only after S_hi of the same tile is visible: Q K^T_hi(j) is issued after P V(j-1), the
 // pipe runs in order, and the next P V is not issued before this thread's p_ready arrival.
 __device__ __forceinline__ void role_softmax(const Ctx& cx, uint32_t tmem_base, int T, int warp, int lane, int B, int H, int S,
-                                             float scale_log2) {
+                                             bool causal, float scale_log2) {
   Shared* sh = cx.sh;
   const int q = warp & 3;
   const int row = q * 32 + lane;
@@ -431,7 +435,7 @@ __device__ __forceinline__ void role_softmax(const Ctx& cx, uint32_t tmem_base, 
   const uint32_t s_addr = tmem_base + (uint32_t)T * 128 + lane_off;     // region A; region B = s_addr + 64
   const uint32_t o_addr = tmem_base + 256 + (uint32_t)T * 128 + lane_off;
   ItemIter iter;
-  iter.init(S, B, H);
+  iter.init(S, B, H, causal);
   Item it;
   uint32_t n_tiles = 0, n_items = 0;
   while (iter.next(it)) {
@@ -494,21 +498,29 @@ __device__ __forceinline__ void role_softmax(const Ctx& cx, uint32_t tmem_base, 
       // Chunks of 32 keys this warp's rows can see at all: every one off the diagonal; on the diagonal tile
       // (the item's last) chunk q holds the warp's own diagonal (key i of it is visible to lane >= i) and the
       // chunks right of it are skipped outright.
-      const bool diag = j == nt - 1;
-      const int vis = diag ? q + 1 : 4;
+      // Without the causal mask only a ragged last key tile has anything hidden: keys from `rem` on, the same
+      // for every row.  All of these conditions are the same for the whole warp.
+      const int rem = S - (nt - 1) * BKV;                       // keys of the item's last tile that exist
+      const bool diag = j == nt - 1 && (causal || rem < BKV);
+      const int vis = !diag ? 4 : causal ? q + 1 : (rem + 31) >> 5;
       if (diag) {
-        // -inf over the masked scores of chunk q, in place, so that the main pass needs no mask code
         if (!wait_half(&sh->s_lo_full[T])) return;
         if (!wait_half(&sh->s_hi_full[T])) return;
-        const uint32_t addr = s_addr + (q < 2 ? 64 + q * 32 : (q - 2) * 32);
-        uint32_t r[32];
-        tc::tmem_ld32(addr, r);
-        tc::tmem_ld_wait();
+        // -inf over the hidden scores of the one partly visible chunk, in place, so that the main pass needs no
+        // mask code: chunk mc, elements above `lim`
+        const int mc = causal ? q : ((rem & 31) ? rem >> 5 : -1);
+        const int lim = causal ? lane : (rem & 31) - 1;
+        if (mc >= 0) {
+          const uint32_t addr = s_addr + (mc < 2 ? 64 + mc * 32 : (mc - 2) * 32);
+          uint32_t r[32];
+          tc::tmem_ld32(addr, r);
+          tc::tmem_ld_wait();
 #pragma unroll
-        for (int i = 0; i < 32; ++i)
-          if (i > lane) r[i] = 0xff800000u;
-        tc::tmem_st32(addr, r);
-        tc::tmem_st_wait();
+          for (int i = 0; i < 32; ++i)
+            if (i > lim) r[i] = 0xff800000u;
+          tc::tmem_st32(addr, r);
+          tc::tmem_st_wait();
+        }
       }
 
       uint32_t pk[64];
@@ -615,7 +627,7 @@ __device__ __forceinline__ void role_softmax(const Ctx& cx, uint32_t tmem_base, 
 // ------------------------------------------------------------------------------------------ output
 // At the end of an item: O / l, to bf16, through the shared-memory transpose to the [B*S, H*D] matrix.
 __device__ __forceinline__ void role_output(const Ctx& cx, uint32_t tmem_base, uint8_t* staging, int warp, int lane,
-                                            __nv_bfloat16* __restrict__ out, int B, int H, int S) {
+                                            __nv_bfloat16* __restrict__ out, int B, int H, int S, bool causal) {
   Shared* sh = cx.sh;
   const int q = warp & 3;
   const int row = q * 32 + lane;
@@ -625,7 +637,7 @@ __device__ __forceinline__ void role_output(const Ctx& cx, uint32_t tmem_base, u
   EpiWarp ew;
   ew.init(staging + q * EPI_WARP_BYTES, none, lane, false);
   ItemIter iter;
-  iter.init(S, B, H);
+  iter.init(S, B, H, causal);
   Item it;
   uint32_t par_item = 0;   // bit t: parity of stream t's next phase
   const int64_t row_bytes = (int64_t)H * HD * 2;
@@ -668,7 +680,8 @@ __device__ __forceinline__ void role_output(const Ctx& cx, uint32_t tmem_base, u
 
 __global__ void __launch_bounds__(THREADS, 1)
 attention_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
-                     __nv_bfloat16* __restrict__ out, int B, int H, int S, float scale_log2, unsigned int* status) {
+                     __nv_bfloat16* __restrict__ out, int B, int H, int S, int causal_i, float scale_log2, unsigned int* status) {
+  const bool causal = causal_i != 0;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* q_tiles = base;
@@ -704,12 +717,12 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
   Ctx cx{sh, &sh->abort_flag, status};
 
   if (warp < 8) {
-    role_softmax(cx, tmem_base, warp >> 2, warp, lane, B, H, S, scale_log2);
+    role_softmax(cx, tmem_base, warp >> 2, warp, lane, B, H, S, causal, scale_log2);
   } else if (warp < 12) {
-    role_output(cx, tmem_base, staging, warp, lane, out, B, H, S);
+    role_output(cx, tmem_base, staging, warp, lane, out, B, H, S, causal);
   } else {
-    if (warp == 12 && lane == 0) role_loader(cx, &tmQ, &tmK, &tmV, q_tiles, k_tiles, v_tiles, B, H, S);
-    if ((warp == 13 || warp == 14) && lane == 0) role_mma(cx, tmem_base, warp - 13, q_tiles, k_tiles, v_tiles, B, H, S);
+    if (warp == 12 && lane == 0) role_loader(cx, &tmQ, &tmK, &tmV, q_tiles, k_tiles, v_tiles, B, H, S, causal);
+    if ((warp == 13 || warp == 14) && lane == 0) role_mma(cx, tmem_base, warp - 13, q_tiles, k_tiles, v_tiles, B, H, S, causal);
     __syncwarp();
   }
 
@@ -747,6 +760,7 @@ cudaError_t attention_tc2_plan(AttnTcPlan* p, const AttnView& a, void* o, int sm
   if (e != cudaSuccess) return e;
   p->out = o;
   p->B = (int)a.B; p->H = (int)a.H; p->S = (int)a.S;
+  p->causal = a.causal;
   p->scale_log2 = (float)(1.4426950408889634 / sqrt((double)a.D));
   const int64_t num_q = (a.S + BQ - 1) / BQ, pairs = (num_q + 1) / 2, n_super = a.B * a.H * ((pairs + 1) / 2);
   p->grid = (int)(n_super < sm_count ? n_super : sm_count);
@@ -760,7 +774,7 @@ cudaError_t launch_attention_tc2(const AttnTcPlan& p, cudaStream_t s) {
     if (e != cudaSuccess) return e;
     attr_done = true;
   }
-  attention_tc2_kernel<<<p.grid, THREADS, ATTN2_SMEM, s>>>(p.tm_q, p.tm_k, p.tm_v, (__nv_bfloat16*)p.out, p.B, p.H, p.S, p.scale_log2,
+  attention_tc2_kernel<<<p.grid, THREADS, ATTN2_SMEM, s>>>(p.tm_q, p.tm_k, p.tm_v, (__nv_bfloat16*)p.out, p.B, p.H, p.S, p.causal ? 1 : 0, p.scale_log2,
                                                            kernel_status_ptr());
   return cudaGetLastError();
 }

@@ -56,7 +56,7 @@ static mk_tensor_spec make_spec(int32_t dtype, std::initializer_list<int64_t> sh
 
 static int n_inputs_of(const mk_op_desc& d) {
   if (d.kind == MK_OP_RESIDUAL_ADD) return 2;
-  if (d.kind == MK_OP_ATTENTION_CAUSAL) return d.i[2] == 0 ? 3 : 1;
+  if (d.kind == MK_OP_ATTENTION_CAUSAL || d.kind == MK_OP_ATTENTION) return d.i[2] == 0 ? 3 : 1;
   return 1;
 }
 
@@ -137,9 +137,10 @@ mk_status infer_shapes(Module& m, std::string& err) {
         if (d.i[0] < 1 || last % d.i[0]) { err = at + "GROUPNORM: channels must be divisible by groups"; return MK_ERR_SHAPE_MISMATCH; }
         if (!(d.f[0] >= 0.0)) { err = at + "eps must be >= 0"; return MK_ERR_INVALID_ARG; }
         break;
-      case MK_OP_ATTENTION_CAUSAL: {
+      case MK_OP_ATTENTION_CAUSAL:
+      case MK_OP_ATTENTION: {
         const int64_t H = d.i[0], D = d.i[1];
-        if (H < 1 || D < 1) { err = at + "ATTENTION_CAUSAL needs i[0] = heads, i[1] = head_dim"; return MK_ERR_INVALID_ARG; }
+        if (H < 1 || D < 1) { err = at + "attention needs i[0] = heads, i[1] = head_dim"; return MK_ERR_INVALID_ARG; }
         if (d.i[2] == 0) {
           if (x.rank != 4 || x.shape[1] != H || x.shape[3] != D) { err = at + "q must be [B, H, S, D]"; return MK_ERR_SHAPE_MISMATCH; }
           if (!same_spec(x, m.values[op.in_id[1]].spec) || !same_spec(x, m.values[op.in_id[2]].spec)) { err = at + "q, k, v differ in shape"; return MK_ERR_SHAPE_MISMATCH; }
@@ -190,8 +191,8 @@ void contract_of(const Module& m, int lo, int hi, std::vector<int>& in_ids, std:
 
 static std::string kind_name(int32_t k) {
   static const char* names[] = {"?", "LINEAR", "CONV2D_3X3", "BIAS_ADD", "RELU", "GELU_TANH", "SILU", "SCALE", "CLAMP",
-                                "RESIDUAL_ADD", "SWIGLU", "LAYERNORM", "RMSNORM", "GROUPNORM", "SOFTMAX", "ATTENTION_CAUSAL"};
-  return (k >= 1 && k <= 15) ? names[k] : "?";
+                                "RESIDUAL_ADD", "SWIGLU", "LAYERNORM", "RMSNORM", "GROUPNORM", "SOFTMAX", "ATTENTION_CAUSAL", "ATTENTION"};
+  return (k >= 1 && k <= 16) ? names[k] : "?";
 }
 
 mk_status default_binding(const Module& m, int lo, int hi, Binding& out, std::string& err) {

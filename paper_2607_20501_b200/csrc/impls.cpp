@@ -354,6 +354,7 @@ mk_status conv_gn_tc2_emit(const Module& m, int lo, int hi, const Resolved& r, s
 // ------------------------------------------------------------------ attention
 AttnView attn_view(const Module& m, const Op& op, const Resolved& r) {
   AttnView a{};
+  a.causal = op.d.kind == MK_OP_ATTENTION_CAUSAL;
   const int64_t H = op.d.i[0], D = op.d.i[1];
   const size_t es = dtype_size(m.values[0].spec.dtype);
   if (op.d.i[2] == 0) {
@@ -388,8 +389,9 @@ mk_status attn_tc_emit(const Module& m, int lo, int, const Resolved& r, std::vec
   out.push_back([plan](cudaStream_t s) { return launch_attention_tc(*plan, s); });
   return MK_OK;
 }
+bool is_attention(int32_t k) { return k == MK_OP_ATTENTION_CAUSAL || k == MK_OP_ATTENTION; }
 bool attn_tc2_match(const Module& m, int lo, int hi) {
-  if (hi - lo != 1 || m.ops[lo].d.kind != MK_OP_ATTENTION_CAUSAL || m.values[0].spec.dtype != MK_BF16) return false;
+  if (hi - lo != 1 || !is_attention(m.ops[lo].d.kind) || m.values[0].spec.dtype != MK_BF16) return false;
   Resolved none;
   none.value_ptr.assign(m.values.size(), nullptr);
   return attention_tc2_supported(attn_view(m, m.ops[lo], none));
@@ -403,7 +405,7 @@ mk_status attn_tc2_emit(const Module& m, int lo, int, const Resolved& r, std::ve
   return MK_OK;
 }
 bool attn_simt_match(const Module& m, int lo, int hi) {
-  return hi - lo == 1 && m.ops[lo].d.kind == MK_OP_ATTENTION_CAUSAL && m.ops[lo].d.i[1] <= 256;
+  return hi - lo == 1 && (m.ops[lo].d.kind == MK_OP_ATTENTION_CAUSAL || m.ops[lo].d.kind == MK_OP_ATTENTION) && m.ops[lo].d.i[1] <= 256;
 }
 mk_status attn_simt_emit(const Module& m, int lo, int, const Resolved& r, std::vector<Launch>& out, std::string&) {
   const Op& op = m.ops[lo];

@@ -94,6 +94,7 @@ struct AttnView {
   const void* v;
   int64_t sb, sh, ss;
   int64_t B, H, S, D;
+  bool causal;   // mask keys after the query (diagonal kept); false: every key is visible
 };
 // O is the dense [B*S, H*D] matrix.
 cudaError_t launch_attention_simt(int dtype, const AttnView& a, void* o, cudaStream_t s);

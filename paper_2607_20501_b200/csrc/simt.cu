@@ -310,7 +310,7 @@ cudaError_t launch_conv3x3_simt(int dtype, const void* x, const void* w, void* y
 template <typename T>
 __global__ void __launch_bounds__(128) attention_simt_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
                                                              T* __restrict__ o, int64_t sb, int64_t sh, int64_t ss, int64_t B, int H,
-                                                             int S, int D) {
+                                                             int S, int D, int causal) {
   constexpr int MAXE = 8;  // D <= 256
   const int lane = threadIdx.x & 31;
   const int64_t wid = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -328,7 +328,8 @@ __global__ void __launch_bounds__(128) attention_simt_kernel(const T* __restrict
   }
   const float scale = rsqrtf((float)D);
   float m = -INFINITY, l = 0.0f;
-  for (int j = 0; j <= i; ++j) {
+  const int last = causal ? i : S - 1;
+  for (int j = 0; j <= last; ++j) {
     float dot = 0.0f;
 #pragma unroll
     for (int e = 0; e < MAXE; ++e) {
@@ -361,10 +362,11 @@ cudaError_t launch_attention_simt(int dtype, const AttnView& a, void* o, cudaStr
   const unsigned grid = (unsigned)((warps + 3) / 4);
   if (dtype == DT_F32)
     attention_simt_kernel<float><<<grid, 128, 0, s>>>((const float*)a.q, (const float*)a.k, (const float*)a.v, (float*)o, a.sb, a.sh, a.ss, a.B,
-                                                      (int)a.H, (int)a.S, (int)a.D);
+                                                      (int)a.H, (int)a.S, (int)a.D, a.causal ? 1 : 0);
   else
     attention_simt_kernel<__nv_bfloat16><<<grid, 128, 0, s>>>((const __nv_bfloat16*)a.q, (const __nv_bfloat16*)a.k, (const __nv_bfloat16*)a.v,
-                                                              (__nv_bfloat16*)o, a.sb, a.sh, a.ss, a.B, (int)a.H, (int)a.S, (int)a.D);
+                                                              (__nv_bfloat16*)o, a.sb, a.sh, a.ss, a.B, (int)a.H, (int)a.S, (int)a.D,
+                                                              a.causal ? 1 : 0);
   return cudaGetLastError();
 }
 

@@ -83,6 +83,7 @@ struct AttnTcPlan {
   CUtensorMap tm_q, tm_k, tm_v;
   void* out = nullptr;
   int B = 0, H = 0, S = 0;
+  bool causal = true;
   float scale_log2 = 0.f;
   int grid = 0;
 };
@@ -91,7 +92,8 @@ struct AttnTcPlan {
 bool attention_tc_supported(const AttnView& a);
 cudaError_t attention_tc_plan(AttnTcPlan* p, const AttnView& a, void* o);
 cudaError_t launch_attention_tc(const AttnTcPlan& p, cudaStream_t s);
-// Two-query-tile persistent form (256 queries per work item, O accumulated in TMEM); same contract.
+// Two-query-tile persistent form (256 queries per work item, O accumulated in TMEM); same contract, and also
+// the unmasked operator (AttnView::causal false).
 bool attention_tc2_supported(const AttnView& a);
 cudaError_t attention_tc2_plan(AttnTcPlan* p, const AttnView& a, void* o, int sm_count);
 cudaError_t launch_attention_tc2(const AttnTcPlan& p, cudaStream_t s);

@@ -313,3 +313,70 @@ def test_attention_closed_forms():
     full = np.einsum("bhid,bhjd->bhij", q, k) / math.sqrt(d)
     nomask = (O.softmax(full) @ v).transpose(0, 2, 1, 3)
     assert np.abs(nomask - o).max() > 1e-2
+
+
+# ------------------------------------------------------------------ unmasked (encoder) attention
+def _attn_full_brute(q, k, v):
+    b, h, s, d = q.shape
+    out = np.zeros((b * s, h * d))
+    for bi in range(b):
+        for hi in range(h):
+            for i in range(s):
+                sc = [sum(float(q[bi, hi, i, t]) * float(k[bi, hi, j, t]) for t in range(d)) / math.sqrt(d)
+                      for j in range(s)]
+                m = max(sc)
+                e = [math.exp(v_ - m) for v_ in sc]
+                z = sum(e)
+                for t in range(d):
+                    out[bi * s + i, hi * d + t] = sum(e[j] / z * float(v[bi, hi, j, t]) for j in range(s))
+    return out
+
+
+def test_full_attention_brute_force_and_layout():
+    b, h, s, d = 2, 3, 7, 4
+    q, k, v = rnd(b, h, s, d), rnd(b, h, s, d), rnd(b, h, s, d)
+    o = O.attention_bhsd(q, k, v)
+    assert o.shape == (b * s, h * d)
+    assert np.allclose(o, _attn_full_brute(q, k, v), atol=1e-13)
+    packed = np.concatenate([t.transpose(0, 2, 1, 3).reshape(b * s, h * d) for t in (q, k, v)], axis=1)
+    assert np.allclose(O.attention_packed(packed, b, s, h, d), o, atol=1e-14)
+
+
+def test_full_attention_closed_forms_and_invariants():
+    b, h, s, d = 1, 2, 16, 8
+    q, k, v = rnd(b, h, s, d), rnd(b, h, s, d), rnd(b, h, s, d)
+    o = O.attention_bhsd(q, k, v).reshape(b, s, h, d)
+    # library special case
+    t = torch.nn.functional.scaled_dot_product_attention(
+        torch.from_numpy(q), torch.from_numpy(k), torch.from_numpy(v), is_causal=False)
+    assert np.allclose(o, t.permute(0, 2, 1, 3).numpy(), atol=1e-12)
+    # identical keys (or zero queries) -> uniform weights -> every query gets the mean of V
+    kk = np.broadcast_to(k[:, :, :1], k.shape).copy()
+    mean_v = np.broadcast_to(v.mean(axis=2, keepdims=True), v.shape).transpose(0, 2, 1, 3)
+    assert np.allclose(O.attention_bhsd(q, kk, v).reshape(b, s, h, d), mean_v, atol=1e-13)
+    assert np.allclose(O.attention_bhsd(np.zeros_like(q), k, v).reshape(b, s, h, d), mean_v, atol=1e-13)
+    # keys and values permuted together leave the output unchanged (no mask, no position);
+    # the causal operator does not have this invariance
+    perm = np.random.default_rng(5).permutation(s)
+    assert np.allclose(O.attention_bhsd(q, k[:, :, perm], v[:, :, perm]).reshape(b, s, h, d), o, atol=1e-13)
+    oc = O.attention_causal_bhsd(q, k, v).reshape(b, s, h, d)
+    assert np.abs(O.attention_causal_bhsd(q, k[:, :, perm], v[:, :, perm]).reshape(b, s, h, d) - oc).max() > 1e-2
+    # permuting the queries permutes the output rows
+    assert np.allclose(O.attention_bhsd(q[:, :, perm], k, v).reshape(b, s, h, d), o[:, perm], atol=1e-13)
+    # the last query of the causal operator sees every key: the two operators agree there and only there
+    assert np.allclose(o[:, -1], oc[:, -1], atol=1e-13)
+    assert np.abs(o[:, :-1] - oc[:, :-1]).max() > 1e-2
+    # one key far ahead of the others takes all the weight: output = its value row
+    k2 = k.copy()
+    q2 = np.ones_like(q)
+    k2[:, :, :, :] = 0.0
+    k2[:, :, 5, :] = 100.0
+    assert np.allclose(O.attention_bhsd(q2, k2, v).reshape(b, s, h, d), np.broadcast_to(v[:, :, 5][:, None], (b, s, h, d)), atol=1e-12)
+    # a shift of every score of a row by a constant (k -> k + c along q's direction is not that; use q . (k + u) with u
+    # orthogonal to nothing in particular) changes nothing when the shift is the same for all keys: add a vector to all keys
+    u = rnd(d)
+    assert np.allclose(O.attention_bhsd(q, k + u, v).reshape(b, s, h, d), o, atol=1e-12)
+    # linear in V
+    v2 = rnd(b, h, s, d)
+    lin = O.attention_bhsd(q, k, 2.0 * v - 3.0 * v2) - (2.0 * O.attention_bhsd(q, k, v) - 3.0 * O.attention_bhsd(q, k, v2))
+    assert np.abs(lin).max() < 1e-12

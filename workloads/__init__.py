@@ -13,6 +13,7 @@ from .generate import (  # noqa: F401
     c3,
     c4,
     c5,
+    c6,
     f32_to_bf16_bits,
     int_valued,
     make,

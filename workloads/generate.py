@@ -271,4 +271,56 @@ def c5(seed=0, B=8, S=1024, E=2048, H=16, F=8192, L=4, dtype="bf16", stream="f32
     return w
 
 
-WORKLOADS = {"c1": c1, "c2": c2, "c3": c3, "c4": c4, "c5": c5}
+# --------------------------------------------------------------------------
+# C6: bf16 post-norm encoder layers (unmasked MHA with biases, LayerNorm, ReLU FFN): the shape of
+# the transformer block in the paper's ConvolutionalVisionTransformer example, at a head_dim the
+# tensor-core attention kernel takes
+# --------------------------------------------------------------------------
+def c6(seed=0, B=16, S=512, E=1024, H=8, F=4096, L=2, dtype="bf16") -> Workload:
+    w = Workload("c6", dtype)
+    D = E // H
+    w.inputs["x"] = make("x", dtype, _normal(seed, 0, (B * S, E)))
+    cur = "x"
+    tid = 1
+    layer_starts = []
+    for l in range(L):
+        layer_starts.append(len(w.ops))
+        shapes = {"Wqkv": (E, 3 * E), "Wo": (E, E), "W1": (E, F), "W2": (F, E)}
+        for i, (nm, shp) in enumerate(shapes.items()):
+            w.params[f"{nm}{l}"] = make(f"{nm}{l}", dtype, _normal(seed, tid + i, shp, std=0.02))
+            w.params[f"b{nm[1:]}{l}"] = make(f"b{nm[1:]}{l}", dtype, _normal(seed, tid + 4 + i, (shp[1],), std=0.02))
+        for i, nm in enumerate(("g1", "g2")):
+            w.params[f"{nm}_{l}"] = make(f"{nm}_{l}", dtype, 1.0 + _normal(seed, tid + 8 + i, (E,), std=0.02))
+            w.params[f"{nm}b_{l}"] = make(f"{nm}b_{l}", dtype, _normal(seed, tid + 10 + i, (E,), std=0.02))
+        tid += 12
+        w.ops += [
+            _op("linear", f"qkv0_{l}", [cur], {"w": f"Wqkv{l}"}, n=3 * E),
+            _op("bias_add", f"qkv_{l}", [f"qkv0_{l}"], {"b": f"bqkv{l}"}),
+            _op("attention", f"att_{l}", [f"qkv_{l}"], layout="packed_qkv", heads=H, head_dim=D, batch=B, seq=S),
+            _op("linear", f"o0_{l}", [f"att_{l}"], {"w": f"Wo{l}"}, n=E),
+            _op("bias_add", f"o1_{l}", [f"o0_{l}"], {"b": f"bo{l}"}),
+            _op("residual_add", f"r1_{l}", [f"o1_{l}", cur]),
+            _op("layernorm", f"x1_{l}", [f"r1_{l}"], {"gamma": f"g1_{l}", "beta": f"g1b_{l}"}, eps=1e-5),
+            _op("linear", f"h0_{l}", [f"x1_{l}"], {"w": f"W1{l}"}, n=F),
+            _op("bias_add", f"h1_{l}", [f"h0_{l}"], {"b": f"b1{l}"}),
+            _op("relu", f"h_{l}", [f"h1_{l}"]),
+            _op("linear", f"d0_{l}", [f"h_{l}"], {"w": f"W2{l}"}, n=E),
+            _op("bias_add", f"d1_{l}", [f"d0_{l}"], {"b": f"b2{l}"}),
+            _op("residual_add", f"r2_{l}", [f"d1_{l}", f"x1_{l}"]),
+            _op("layernorm", f"x2_{l}", [f"r2_{l}"], {"gamma": f"g2_{l}", "beta": f"g2b_{l}"}, eps=1e-5),
+        ]
+        cur = f"x2_{l}"
+    n_ops = len(w.ops)
+    # default decomposition: GEMMs carry bias, activation and residual; attention and the norms stand alone
+    fused_cuts = []
+    for s in layer_starts:
+        fused_cuts += [s + 0, s + 2, s + 3, s + 6, s + 7, s + 10, s + 13]
+    w.partitions = {"fused_tails": fused_cuts, "per_op": list(range(n_ops)), "fused": [0]}
+    T = B * S
+    per_layer = 2.0 * T * E * 3 * E + 4.0 * B * H * D * S * S + 2.0 * T * E * E + 4.0 * T * E * F
+    w.flops = L * per_layer
+    w.min_bytes = 2 * (2 * T * E + L * (4 * E * E + 2 * E * F))
+    return w
+
+
+WORKLOADS = {"c1": c1, "c2": c2, "c3": c3, "c4": c4, "c5": c5, "c6": c6}
