@@ -134,18 +134,26 @@ __device__ __forceinline__ void rownorm_fixup(const RowNormArgs& na, __nv_bfloat
   }
 }
 
-template <int CTAS, bool SWIGLU, bool NORM = false>
+// RING (two-SM form): one pipeline stage less, and its shared memory holds, per epilogue warp, two 32-row x 64-byte
+// slots into which a bf16 residual is copied asynchronously two chunks ahead of its use (RES_RING_BYTES in all).
+constexpr int RES_SLOT_BYTES = 32 * 64;
+constexpr int RES_RING_BYTES = EPI_WARPS * 2 * RES_SLOT_BYTES;
+static_assert(RES_RING_BYTES <= Cfg<2>::STAGE_BYTES, "the residual ring takes the place of one pipeline stage");
+
+template <int CTAS, bool SWIGLU, bool NORM = false, bool RING = false>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmBh,
                const __grid_constant__ CUtensorMap tmOut, int bulk_store, void* __restrict__ out, int out_f32, int M, int N, int K, int up_row_offset, int tail_first,
                const __grid_constant__ EpiProgram epi_param, const __grid_constant__ RowNormArgs na, unsigned int* status) {
   using C = Cfg<CTAS>;
-  constexpr int STAGES = C::STAGES;
+  static_assert(!RING || (CTAS == 2 && !SWIGLU && !NORM), "the residual ring exists in the plain two-SM form only");
+  constexpr int STAGES = C::STAGES - (RING ? 1 : 0);
   constexpr int OUT_N = SWIGLU ? BN / 2 : BN;  // output columns per tile
   extern __shared__ uint8_t smem_raw[];
   uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  uint8_t* staging = tiles + (size_t)STAGES * C::STAGE_BYTES;
-  Shared<STAGES>* sh = reinterpret_cast<Shared<STAGES>*>(staging + EPI_WARPS * EPI_WARP_BYTES);
+  uint8_t* res_ring = tiles + (size_t)STAGES * C::STAGE_BYTES;       // RING only: the space of the stage given up
+  uint8_t* staging = tiles + (size_t)C::STAGES * C::STAGE_BYTES;
+  Shared<C::STAGES>* sh = reinterpret_cast<Shared<C::STAGES>*>(staging + EPI_WARPS * EPI_WARP_BYTES);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = CTAS == 2 ? tc::cluster_ctarank() : 0;
   const bool leader = rank == 0;
@@ -165,7 +173,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   MK_TR_DECL
   MK_TR_INIT;
 
-  static_assert(sizeof(Shared<STAGES>) <= 512, "barrier block");
+  static_assert(sizeof(Shared<C::STAGES>) <= 512, "barrier block");
   epi_copy_to_smem(&sh->epi, epi_param, threadIdx.x, THREADS);
   const EpiProgram& epi = sh->epi;
   if (threadIdx.x == 0) {
@@ -301,6 +309,57 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     ew.init(staging + (warp - 2) * EPI_WARP_BYTES, epi, lane, out_f32 != 0);
     bool ok = true;
     int it = 0;
+    // RING: the warp's chunks form one sequence across its tiles (unit u, chunk c = half, half + 2, ...).  A cursor
+    // runs two chunks ahead of the one being stored; every chunk, once its residual has been read out of its slot,
+    // starts the copy of the chunk at the cursor into that slot (16 bytes per lane and row, swizzled like the store
+    // staging so that the lane's read of its own 64-byte row is free of bank conflicts), one commit group per chunk.
+    uint8_t* my_ring = res_ring + (warp - 2) * 2 * RES_SLOT_BYTES;
+    int pf_u = unit_id, pf_c = half, res_slot = 0;
+    auto ring_issue = [&](int slot) {
+      if (pf_u < total_units) {
+        int t, nhalf;
+        decode(pf_u, t, nhalf);
+        int mi, ni;
+        tile_coords(t, num_m, num_n, mi, ni);
+        const int64_t r0 = (int64_t)(mi * CTAS + (int)rank) * BM + q * 32;
+        const int64_t c0 = (int64_t)ni * OUT_N + (nhalf > 0 ? BN / 2 : 0) + pf_c * 32;
+        if (c0 + 32 <= N) {
+          const uint8_t* res = reinterpret_cast<const uint8_t*>(epi.op[ew.res_idx].ptr);
+          const int sub_row = lane >> 2, seg = lane & 3;
+          const uint32_t dst0 = tc::smem_u32(my_ring + slot * RES_SLOT_BYTES);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int r = sub_row + 8 * i;
+            if (r0 + r < M) tc::cp_async16(dst0 + r * 64 + ((seg ^ ((r >> 1) & 3)) * 16), res + ((r0 + r) * (int64_t)N + c0) * 2 + seg * 16);
+          }
+        }
+        pf_c += 2;
+        if (pf_c >= (nhalf < 0 ? CHUNKS : CHUNKS / 2)) { pf_u += num_units; pf_c = half; }
+      }
+      tc::cp_async_commit();
+    };
+    auto ring_get = [&](uint4 (&ra)[4], uint4 (&)[4]) -> int {
+      tc::cp_async_wait<1>();      // this chunk's group (the older of the two in flight) has landed
+      __syncwarp();                // ... for every lane
+      const uint8_t* src = my_ring + res_slot * RES_SLOT_BYTES + lane * 64;
+      const int f = (lane >> 1) & 3;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) ra[i] = *reinterpret_cast<const uint4*>(src + ((i ^ f) * 16));
+      __syncwarp();                // every lane has read its row: the slot may be refilled
+      ring_issue(res_slot);
+      res_slot ^= 1;
+      return 1;
+    };
+    auto ring_skip = [&]() {
+      tc::cp_async_wait<1>();
+      __syncwarp();
+      ring_issue(res_slot);
+      res_slot ^= 1;
+    };
+    if (RING) {
+      ring_issue(0);
+      ring_issue(1);
+    }
     for (int u = unit_id; u < total_units && ok; u += num_units, ++it) {
       int t, nhalf;
       decode(u, t, nhalf);
@@ -313,7 +372,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int chunks_here = nhalf < 0 ? CHUNKS : CHUNKS / 2;
       uint4 res_regs[8];
       ew.load_bias(epi, col_base, nhalf < 0 ? OUT_N : OUT_N / 2, N);
-      ew.prefetch_res(epi, rowmap, col_base + half * 32, N, res_regs);
+      if (!RING) ew.prefetch_res(epi, rowmap, col_base + half * 32, N, res_regs);
       ok = tc::mbar_wait(&sh->tfull[acc], (it >> 1) & 1, abort_flag, status, tc::WAIT_TMEM_FULL);
       ok = __all_sync(0xffffffffu, ok ? 1 : 0) != 0;
       if (!ok) break;
@@ -327,6 +386,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         float v[32];
         tc::tmem_ld32(t_row + c * 32, r);
         tc::tmem_ld_wait();
+        if (threadIdx.x == 64 && c == half + 2) MK_TR(5 + it * 8);  // epilogue: second chunk in registers
 #pragma unroll
         for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
         if (SWIGLU) {
@@ -335,8 +395,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
           for (int j = 0; j < 32; ++j) v[j] = silu_fast(v[j]) * __uint_as_float(r[j]);
         }
-        ew.chunk_out(epi, v, rowmap, out, col_base + c * 32, c * 32, (int64_t)N, res_regs, c + 2 < chunks_here ? col_base + (c + 2) * 32 : -1,
-                     (!NORM && bulk_store) ? &tmOut : nullptr, row0);
+        if (RING)
+          ew.chunk_out_from(epi, v, rowmap, out, col_base + c * 32, c * 32, (int64_t)N, ring_get, ring_skip, bulk_store ? &tmOut : nullptr, row0);
+        else
+          ew.chunk_out(epi, v, rowmap, out, col_base + c * 32, c * 32, (int64_t)N, res_regs, c + 2 < chunks_here ? col_base + (c + 2) * 32 : -1,
+                       (!NORM && bulk_store) ? &tmOut : nullptr, row0);
+        if (threadIdx.x == 64 && c == half + 2) MK_TR(6 + it * 8);  // epilogue: second chunk handed to the store
         if (NORM) {
           // v now holds the values after the elementwise tail (what was just stored, before its bf16 rounding)
           const int64_t c0 = col_base + c * 32;
@@ -382,6 +446,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
       }
     }
+    if (RING) tc::cp_async_wait<0>();           // no copy into shared memory is in flight when the CTA retires
     if (lane == 0) tc::tma_store_wait_all();   // bulk stores of this warp are complete before the CTA retires
   }
 
@@ -432,6 +497,14 @@ cudaError_t plan_impl(GemmTcPlan* p, const void* a, const void* w_nk, void* y, b
   const int64_t units = tiles < sm_count / CTAS ? tiles : sm_count / CTAS;
   p->grid = (int)(CTAS * units);
   // a last wave that fills at most half of the CTA pairs is run as half-width units (two-SM form only)
+  // a bf16 residual of the plain two-SM form travels through the shared-memory ring
+  p->res_ring = false;
+  if (CTAS == 2 && !swiglu) {
+    int idx = -1, cnt = 0;
+    for (int i = 0; i < epi.n; ++i)
+      if (epi.op[i].kind == EPI_RESIDUAL) { idx = i; ++cnt; }
+    p->res_ring = cnt == 1 && epi.op[idx].ptr_dtype == DT_BF16;
+  }
   const int64_t tail = tiles % units;
   p->tail_first = (int)tiles;
   if (CTAS == 2 && !swiglu && tiles > units && tail > 0 && 2 * tail <= units) p->tail_first = (int)(tiles - tail);
@@ -444,6 +517,8 @@ cudaError_t launch_impl(const GemmTcPlan& p, cudaStream_t s) {
   if (!attr_done) {
     cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<CTAS, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<CTAS>::SMEM);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<CTAS, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<CTAS>::SMEM);
+    if (e == cudaSuccess && CTAS == 2)
+      e = cudaFuncSetAttribute(gemm_tc_kernel<2, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<2>::SMEM);
     if (e != cudaSuccess) return e;
     attr_done = true;
   }
@@ -464,6 +539,9 @@ cudaError_t launch_impl(const GemmTcPlan& p, cudaStream_t s) {
   if (p.swiglu)
     return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<CTAS, true>, p.tm_a, p.tm_b, p.tm_b_half, p.tm_out, p.use_tm_out ? 1 : 0, p.out, out_f32, p.m, p.n, p.k, p.n, p.tail_first, p.epi,
                               p.norm, status);
+  if (CTAS == 2 && p.res_ring)
+    return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<2, false, false, true>, p.tm_a, p.tm_b, p.tm_b_half, p.tm_out, p.use_tm_out ? 1 : 0, p.out, out_f32, p.m, p.n, p.k, 0,
+                              p.tail_first, p.epi, p.norm, status);
   return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<CTAS, false>, p.tm_a, p.tm_b, p.tm_b_half, p.tm_out, p.use_tm_out ? 1 : 0, p.out, out_f32, p.m, p.n, p.k, 0, p.tail_first, p.epi,
                             p.norm, status);
 }

@@ -264,6 +264,18 @@ __device__ __forceinline__ unsigned long long gtime() {
 #define MK_TR_PRINT(tag) do {} while (0)
 #endif
 
+// ---------------------------------------------------------------- asynchronous 16-byte copies (global -> shared)
+// Per-thread copies that need no register for the data in flight; completion is tracked per thread in commit
+// groups, so other lanes see the bytes only after the issuing lane's wait and a warp barrier.
+__device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void* gsrc) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_dst), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
 // ---------------------------------------------------------------- lean issue path
 // One thread issues every MMA of a CTA (pair), a few dependent instructions at a time, so the
 // issue loop itself can starve the tensor pipe: a 256x256x16 MMA lasts 128 cycles, a 256x128x16

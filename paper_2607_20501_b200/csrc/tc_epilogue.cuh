@@ -230,13 +230,39 @@ struct EpiWarp {
   //   bias_off     offset (elements) of col0 inside the bias slice loaded by load_bias
   //   rowmap(r)    global row of warp-local row r in [0, 32), or -1 if that row is not stored
   //   res_regs     this chunk's residual (from prefetch_res); on return the next chunk's, if next_col0 >= 0
-  template <typename RowMap>
   //   tm_store     if not null (bf16 output, rows of the warp consecutive from global row y0): the block leaves by a
   //                bulk tensor store instead of 16-byte stores
+  template <typename RowMap>
   __device__ __forceinline__ void chunk_out(const EpiProgram& epi, float (&v)[32], RowMap rowmap, void* __restrict__ out_v, int64_t col0,
                                             int bias_off, int64_t n_cols, uint4 (&res_regs)[8], int64_t next_col0,
                                             const CUtensorMap* tm_store = nullptr, int64_t y0 = 0) {
     if (col0 >= n_cols) return;  // warp-uniform
+    // the residual through registers: this chunk's values were fetched one chunk ago, the next chunk's are fetched now
+    auto get = [&](uint4 (&ra)[4], uint4 (&rb)[4]) -> int {
+      if (res_idx < 0) return 0;
+      slab_to_own_row(res_regs[0], res_regs[1], res_regs[2], res_regs[3], ra, false);
+      if (res_f32) slab_to_own_row(res_regs[4], res_regs[5], res_regs[6], res_regs[7], rb, true);
+      if (next_col0 >= 0) prefetch_res(epi, rowmap, next_col0, n_cols, res_regs);
+      return res_f32 ? 2 : 1;
+    };
+    auto skip = [&]() {
+      if (res_idx >= 0 && next_col0 >= 0) prefetch_res(epi, rowmap, next_col0, n_cols, res_regs);
+    };
+    chunk_out_from(epi, v, rowmap, out_v, col0, bias_off, n_cols, get, skip, tm_store, y0);
+  }
+  // The same with the residual supplied by the caller:
+  //   get(ra, rb)  called once for a chunk that is stored whole: fills the lane's own 32 residual values (bf16 in ra:
+  //                returns 1; fp32 in ra, rb: returns 2; no residual operand prepared: returns 0) and may start the
+  //                fetch of a later chunk
+  //   skip()       called instead for a chunk that is ragged in N (its residual is read element by element)
+  template <typename RowMap, typename Get, typename Skip>
+  __device__ __forceinline__ void chunk_out_from(const EpiProgram& epi, float (&v)[32], RowMap rowmap, void* __restrict__ out_v, int64_t col0,
+                                                 int bias_off, int64_t n_cols, Get get, Skip skip, const CUtensorMap* tm_store = nullptr,
+                                                 int64_t y0 = 0) {
+    if (col0 >= n_cols) {  // warp-uniform
+      skip();
+      return;
+    }
     if (tm_store) {
       // the previous chunk's bulk store has finished reading the staging buffer (the residual slabs go through it too)
       if (lane == 0) tc::tma_store_wait_read();
@@ -246,16 +272,7 @@ struct EpiWarp {
     uint8_t* out = reinterpret_cast<uint8_t*>(out_v);
     if (col0 + 32 <= n_cols) {
       uint4 ra[4], rb[4];
-      int res_mode = 0;
-      if (res_idx >= 0) {
-        slab_to_own_row(res_regs[0], res_regs[1], res_regs[2], res_regs[3], ra, false);
-        res_mode = 1;
-        if (res_f32) {
-          slab_to_own_row(res_regs[4], res_regs[5], res_regs[6], res_regs[7], rb, true);
-          res_mode = 2;
-        }
-        if (next_col0 >= 0) prefetch_res(epi, rowmap, next_col0, n_cols, res_regs);
-      }
+      const int res_mode = get(ra, rb);
       if (my_row >= 0) epi32(epi, v, my_row, col0, n_cols, bias_idx >= 0 ? bias + bias_off * 2 : nullptr, res_mode, ra, rb);
       uint4 mine[4];
       if (!out_f32) {
@@ -291,7 +308,7 @@ struct EpiWarp {
             else reinterpret_cast<__nv_bfloat16*>(out)[my_row * n_cols + col0 + j] = __float2bfloat16_rn(r);
           }
       }
-      if (res_idx >= 0 && next_col0 >= 0) prefetch_res(epi, rowmap, next_col0, n_cols, res_regs);
+      skip();
     }
   }
 };
