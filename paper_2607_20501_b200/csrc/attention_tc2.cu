@@ -715,6 +715,8 @@ attention_tc2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
   tc::tc_fence_after();
   const uint32_t tmem_base = sh->tmem_base;
   Ctx cx{sh, &sh->abort_flag, status};
+  pdl_launch_dependents();
+  pdl_wait();   // Q, K, V may come from the kernel before this one
 
   if (warp < 8) {
     role_softmax(cx, tmem_base, warp >> 2, warp, lane, B, H, S, causal, scale_log2);
@@ -774,9 +776,9 @@ cudaError_t launch_attention_tc2(const AttnTcPlan& p, cudaStream_t s) {
     if (e != cudaSuccess) return e;
     attr_done = true;
   }
-  attention_tc2_kernel<<<p.grid, THREADS, ATTN2_SMEM, s>>>(p.tm_q, p.tm_k, p.tm_v, (__nv_bfloat16*)p.out, p.B, p.H, p.S, p.causal ? 1 : 0, p.scale_log2,
-                                                           kernel_status_ptr());
-  return cudaGetLastError();
+  LaunchCfg lc(PDL_ATTENTION, dim3((unsigned)p.grid), dim3(THREADS), ATTN2_SMEM, s);
+  return cudaLaunchKernelEx(&lc.cfg, attention_tc2_kernel, p.tm_q, p.tm_k, p.tm_v, (__nv_bfloat16*)p.out, p.B, p.H, p.S, p.causal ? 1 : 0, p.scale_log2,
+                            kernel_status_ptr());
 }
 
 }  // namespace mk

@@ -20,6 +20,8 @@ __global__ void __launch_bounds__(256) eltwise_vec_kernel(const T* __restrict__ 
                                                           int64_t cols, int tx, const __grid_constant__ EpiProgram p) {
   constexpr int VE = Elem<T>::VEC;
   constexpr int UNROLL = 4;
+  pdl_launch_dependents();
+  pdl_wait();
   const int vpr = (int)(cols / VE);
   const int cx = threadIdx.x & (tx - 1), ry = threadIdx.x / tx, rpb = 256 / tx;
   const int vc = blockIdx.x * tx + cx;
@@ -87,8 +89,9 @@ static cudaError_t eltwise_dispatch(const void* x, void* y, int64_t rows, int64_
     if (gy < 1) gy = 1;
     if (gy > 65535) gy = 65535;
     dim3 grid((unsigned)gx, (unsigned)gy);
-    if (swiglu) eltwise_vec_kernel<T, TO, true><<<grid, 256, 0, s>>>(xp, yp, rows, cols, tx, p);
-    else eltwise_vec_kernel<T, TO, false><<<grid, 256, 0, s>>>(xp, yp, rows, cols, tx, p);
+    LaunchCfg lc(PDL_ELTWISE, grid, dim3(256), 0, s);
+    if (swiglu) return cudaLaunchKernelEx(&lc.cfg, eltwise_vec_kernel<T, TO, true>, xp, yp, rows, cols, tx, p);
+    return cudaLaunchKernelEx(&lc.cfg, eltwise_vec_kernel<T, TO, false>, xp, yp, rows, cols, tx, p);
   } else {
     int grid = ceil_div_i64(rows * cols, 256);
     grid = grid > sm_count * 8 ? sm_count * 8 : grid;
@@ -114,6 +117,8 @@ __global__ void __launch_bounds__(256) rowop_warp_kernel(const TI* __restrict__ 
                                                          const T* __restrict__ gamma, const T* __restrict__ beta, float eps,
                                                          const __grid_constant__ EpiProgram pre) {
   constexpr int VE = Elem<T>::VEC;
+  pdl_launch_dependents();
+  pdl_wait();
   const int lane = threadIdx.x & 31;
   const int nvec = n / VE;
   const int64_t wstride = (int64_t)gridDim.x * (blockDim.x >> 5);
@@ -279,11 +284,12 @@ static cudaError_t rowop_mode(const TI* x, T* y, int64_t rows, int64_t n, const 
     int grid = ceil_div_i64(rows, 8);
     if (grid > 148 * 8) grid = 148 * 8;
     const int ni = (int)n;
-    if (nvec <= 32) rowop_warp_kernel<TI, T, 1, MODE><<<grid, 256, 0, s>>>(x, y, rows, ni, g, b, eps, pre);
-    else if (nvec <= 64) rowop_warp_kernel<TI, T, 2, MODE><<<grid, 256, 0, s>>>(x, y, rows, ni, g, b, eps, pre);
-    else if (nvec <= 128) rowop_warp_kernel<TI, T, 4, MODE><<<grid, 256, 0, s>>>(x, y, rows, ni, g, b, eps, pre);
-    else if (nvec <= 256) rowop_warp_kernel<TI, T, 8, MODE><<<grid, 256, 0, s>>>(x, y, rows, ni, g, b, eps, pre);
-    else rowop_warp_kernel<TI, T, 16, MODE><<<grid, 256, 0, s>>>(x, y, rows, ni, g, b, eps, pre);
+    LaunchCfg lc(PDL_ROWOP, dim3((unsigned)grid), dim3(256), 0, s);
+    if (nvec <= 32) return cudaLaunchKernelEx(&lc.cfg, rowop_warp_kernel<TI, T, 1, MODE>, x, y, rows, ni, g, b, eps, pre);
+    if (nvec <= 64) return cudaLaunchKernelEx(&lc.cfg, rowop_warp_kernel<TI, T, 2, MODE>, x, y, rows, ni, g, b, eps, pre);
+    if (nvec <= 128) return cudaLaunchKernelEx(&lc.cfg, rowop_warp_kernel<TI, T, 4, MODE>, x, y, rows, ni, g, b, eps, pre);
+    if (nvec <= 256) return cudaLaunchKernelEx(&lc.cfg, rowop_warp_kernel<TI, T, 8, MODE>, x, y, rows, ni, g, b, eps, pre);
+    return cudaLaunchKernelEx(&lc.cfg, rowop_warp_kernel<TI, T, 16, MODE>, x, y, rows, ni, g, b, eps, pre);
   } else {
     rowop_block_kernel<TI, T, MODE><<<(unsigned)rows, 256, 0, s>>>(x, y, rows, n, g, b, eps, pre);
   }
@@ -500,6 +506,8 @@ __global__ void __launch_bounds__(GN_THREADS, 3) groupnorm_apply_partials_kernel
   const int64_t p0 = hw * chunk / chunks, p1 = hw * (chunk + 1) / chunks;
   const T* xin = x + (img * hw) * c + vcol * VE;
   T* yout = y + (img * hw) * c + vcol * VE;
+  pdl_launch_dependents();
+  pdl_wait();   // x and the partial sums come from the kernel before this one
   RawVec<T, VE> cur[UN];
   int64_t pix = p0 + prow;
 #pragma unroll
@@ -608,14 +616,12 @@ cudaError_t launch_groupnorm_apply_partials(int dtype, const void* x, void* y, i
   if (chunks > maxc) chunks = maxc;
   if (chunks < 1) chunks = 1;
   dim3 grid((unsigned)chunks, (unsigned)nb);
+  LaunchCfg lc(PDL_GROUPNORM, grid, dim3(GN_THREADS), 0, s);
   if (dtype == DT_F32)
-    groupnorm_apply_partials_kernel<float><<<grid, GN_THREADS, 0, s>>>((const float*)x, (float*)y, hw, (int)c, groups, (const float*)gamma,
-                                                                       (const float*)beta, eps, stats, stat_slots);
-  else
-    groupnorm_apply_partials_kernel<__nv_bfloat16><<<grid, GN_THREADS, 0, s>>>((const __nv_bfloat16*)x, (__nv_bfloat16*)y, hw, (int)c, groups,
-                                                                               (const __nv_bfloat16*)gamma, (const __nv_bfloat16*)beta, eps,
-                                                                               stats, stat_slots);
-  return cudaGetLastError();
+    return cudaLaunchKernelEx(&lc.cfg, groupnorm_apply_partials_kernel<float>, (const float*)x, (float*)y, hw, (int)c, groups, (const float*)gamma,
+                              (const float*)beta, eps, stats, stat_slots);
+  return cudaLaunchKernelEx(&lc.cfg, groupnorm_apply_partials_kernel<__nv_bfloat16>, (const __nv_bfloat16*)x, (__nv_bfloat16*)y, hw, (int)c, groups,
+                            (const __nv_bfloat16*)gamma, (const __nv_bfloat16*)beta, eps, stats, stat_slots);
 }
 
 template <typename T>

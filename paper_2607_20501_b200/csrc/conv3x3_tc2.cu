@@ -199,6 +199,8 @@ conv3x3_tc2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
   tc::cluster_sync();
   tc::tc_fence_after();
   const uint32_t tmem_base = sh->tmem_base;
+  pdl_launch_dependents();
+  pdl_wait();   // X may come from the kernel before this one
 
   if (warp == 0) {
     // ------------------------------------------------------------ producer
@@ -418,18 +420,8 @@ cudaError_t launch_conv3x3_tc2(const ConvTcPlan& p, cudaStream_t s) {
     if (e != cudaSuccess) return e;
     attr_bytes = p.smem;
   }
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)p.grid);
-  cfg.blockDim = dim3(THREADS);
-  cfg.dynamicSmemBytes = p.smem;
-  cfg.stream = s;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = 2;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  LaunchCfg lc(PDL_CONV, dim3((unsigned)p.grid), dim3(THREADS), p.smem, s, 2);
+  cudaLaunchConfig_t& cfg = lc.cfg;
   unsigned int* status = kernel_status_ptr();
   __nv_bfloat16* y = (__nv_bfloat16*)p.y;
   if (p.c_in == 64) return cudaLaunchKernelEx(&cfg, conv3x3_tc2_kernel<1>, p.tm_x, p.tm_w, y, p.nb, p.h, p.w, p.c_out, p.epi, p.stats, p.cpg, status);

@@ -10,6 +10,13 @@
 
 namespace mk {
 
+// Programmatic dependent launch, device side.  pdl_launch_dependents(): the next kernel on the stream (if it was
+// launched as a dependent) may start being scheduled once every CTA of this grid has said so or retired.
+// pdl_wait(): block until every kernel this grid depends on has completed and its writes are visible; a no-op
+// for a grid launched in plain stream order.  Nothing produced by an earlier kernel may be read before it.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 template <typename T> struct Elem;
 template <> struct Elem<float> {
   static constexpr int VEC = 4;  // elements per 128-bit access

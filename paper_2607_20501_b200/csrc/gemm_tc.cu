@@ -194,6 +194,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   if (CTAS == 2) tc::cluster_sync();  // both CTAs' barriers exist before anything remote touches them
   tc::tc_fence_after();
   const uint32_t tmem_base = sh->tmem_base;
+  // set-up done: the next kernel may be scheduled as this grid drains; nothing of the previous kernel's
+  // output (A, a residual) is read before it has completed
+  pdl_launch_dependents();
+  pdl_wait();
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
@@ -522,18 +526,8 @@ cudaError_t launch_impl(const GemmTcPlan& p, cudaStream_t s) {
     if (e != cudaSuccess) return e;
     attr_done = true;
   }
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)p.grid);
-  cfg.blockDim = dim3(THREADS);
-  cfg.dynamicSmemBytes = Cfg<CTAS>::SMEM;
-  cfg.stream = s;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = CTAS;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  LaunchCfg lc(PDL_GEMM, dim3((unsigned)p.grid), dim3(THREADS), Cfg<CTAS>::SMEM, s, CTAS == 2 ? 2 : 0);
+  cudaLaunchConfig_t& cfg = lc.cfg;
   unsigned int* status = kernel_status_ptr();
   const int out_f32 = p.out_f32 ? 1 : 0;
   if (p.swiglu)

@@ -41,6 +41,42 @@ struct EpiProgram {
 unsigned int* kernel_status_ptr();   // device address, nullptr without a device
 cudaError_t kernel_status_fetch_and_clear(unsigned int* out);
 
+// ---- programmatic dependent launch ----------------------------------------------------------------------
+// A kernel launched through LaunchCfg may be scheduled while the kernel before it on the stream is still
+// draining: its CTAs become resident as the predecessor's CTAs retire, run their set-up, and block in
+// pdl_wait() (device_common.cuh) until the predecessor has completed and its writes are visible.  Only
+// kernels that execute pdl_wait() before their first read of global data may be launched this way.
+// MK_NO_PDL=1 in the environment turns the attribute off (plain stream order); MK_PDL_MASK=<bits> sets which
+// kernel families (PDL_* below) are launched as dependents (default: GEMM, attention, convolution, GroupNorm pass).
+enum PdlFamily : unsigned { PDL_GEMM = 1, PDL_ATTENTION = 2, PDL_CONV = 4, PDL_ROWOP = 8, PDL_ELTWISE = 16, PDL_GROUPNORM = 32 };
+bool pdl_enabled(unsigned family);
+struct LaunchCfg {
+  cudaLaunchConfig_t cfg;
+  cudaLaunchAttribute attr[2];
+  LaunchCfg(unsigned family, dim3 grid, dim3 block, size_t smem, cudaStream_t s, int cluster = 1) {
+    cfg = cudaLaunchConfig_t{};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    int n = 0;
+    if (cluster > 1) {
+      attr[n].id = cudaLaunchAttributeClusterDimension;
+      attr[n].val.clusterDim.x = (unsigned)cluster;
+      attr[n].val.clusterDim.y = 1;
+      attr[n].val.clusterDim.z = 1;
+      ++n;
+    }
+    if (pdl_enabled(family)) {
+      attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+      attr[n].val.programmaticStreamSerializationAllowed = 1;
+      ++n;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = (unsigned)n;
+  }
+};
+
 // ---- HBM-bound kernels ------------------------------------------------------------------------------
 // y[rows, cols] = program(x).  swiglu: x is [rows, 2*cols] = [gate | up] and the program runs on
 // silu(gate) * up.  x has the module dtype; y has out_dtype (fp32 for an fp32 residual stream).

@@ -1,5 +1,6 @@
 // Device status word: a kernel whose bounded wait (mbarrier, flag) runs out records a code here and
 // leaves through its normal exit path instead of spinning forever; the host reads it after a sync.
+#include <stdlib.h>
 #include "kernels.h"
 
 namespace mk {
@@ -14,6 +15,19 @@ unsigned int* kernel_status_ptr() {
     p = (unsigned int*)a;
   }
   return p;
+}
+
+bool pdl_enabled(unsigned family) {
+  static const unsigned mask = [] {
+    const char* v = getenv("MK_NO_PDL");
+    if (v && v[0] && v[0] != '0') return 0u;
+    const char* m = getenv("MK_PDL_MASK");
+    // Default: the kernels that fill an SM by themselves (shared memory) and the GroupNorm pass that follows the
+    // convolution.  The row and elementwise kernels are small enough to become resident BESIDE a running GEMM; as
+    // dependents they did (blocked in their wait) and slowed it by 3 % (measured), so they keep plain stream order.
+    return m && m[0] ? (unsigned)strtoul(m, nullptr, 0) : (unsigned)(PDL_GEMM | PDL_ATTENTION | PDL_CONV | PDL_GROUPNORM);
+  }();
+  return (mask & family) != 0;
 }
 
 cudaError_t kernel_status_fetch_and_clear(unsigned int* out) {
