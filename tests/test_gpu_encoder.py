@@ -1,7 +1,7 @@
 """Unmasked (encoder) attention and the post-norm encoder block against the fp64 oracle: every key
-visible, ragged last key tiles at every 32-key chunk boundary and inside a chunk, the packed-QKV
-view, invariances that only the unmasked operator has, Swap against the plain-ALU kernel, and the
-composed block at a reduced size."""
+visible, ragged last key tiles at every 32-key chunk boundary and inside a chunk, invariances that
+only the unmasked operator has, the plain-ALU kernel beside the tensor-core one, and the composed
+block (packed-QKV view, residual GEMMs, LayerNorm) at a reduced size and at the benchmark's size."""
 import numpy as np
 import pytest
 
