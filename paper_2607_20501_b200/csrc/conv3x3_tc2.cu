@@ -150,11 +150,6 @@ __device__ __forceinline__ void umma_ss_pair_x4(uint32_t d_tmem, uint64_t a_desc
       : "memory");
 }
 
-__device__ __forceinline__ void tma_prefetch_4d(const CUtensorMap* m, int32_t c, int32_t w, int32_t h, int32_t n) {
-  asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global.tile [%0, {%1, %2, %3, %4}];" ::"l"(reinterpret_cast<uint64_t>(m)), "r"(c), "r"(w),
-               "r"(h), "r"(n)
-               : "memory");
-}
 
 // CB = C_in / 64 channel blocks
 template <int CB>
@@ -226,7 +221,7 @@ conv3x3_tc2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
           const int tn = t + num_clusters;
           if (tn < total_tiles) {
             const int nn = tn / quads, hn = (tn - nn * quads) * 2 * TILE_ROWS + (int)rank * TILE_ROWS;
-            for (int cb = 0; cb < CB; ++cb) tma_prefetch_4d(&tmX, cb * 64, -1, hn - 1, nn);
+            for (int cb = 0; cb < CB; ++cb) tc::tma_prefetch_4d(&tmX, cb * 64, -1, hn - 1, nn);
           }
         }
         for (int cb = 0; cb < CB; ++cb) {

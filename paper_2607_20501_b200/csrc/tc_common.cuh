@@ -264,6 +264,13 @@ __device__ __forceinline__ unsigned long long gtime() {
 #define MK_TR_PRINT(tag) do {} while (0)
 #endif
 
+// L2 prefetch of a 4-D tensor-map box: no shared memory, no barrier; a later load of the same box hits L2.
+__device__ __forceinline__ void tma_prefetch_4d(const CUtensorMap* m, int32_t c0, int32_t c1, int32_t c2, int32_t c3) {
+  asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global.tile [%0, {%1, %2, %3, %4}];" ::"l"(reinterpret_cast<uint64_t>(m)), "r"(c0), "r"(c1),
+               "r"(c2), "r"(c3)
+               : "memory");
+}
+
 // ---------------------------------------------------------------- asynchronous 16-byte copies (global -> shared)
 // Per-thread copies that need no register for the data in flight; completion is tracked per thread in commit
 // groups, so other lanes see the bytes only after the issuing lane's wait and a warp barrier.
