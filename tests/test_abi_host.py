@@ -217,3 +217,35 @@ def test_swap_needs_a_device_and_sane_arguments(ctx):
     st = B.mk_module_swap(m.h, ins, outs, None, 0, None, 3, 0.9, C.byref(n), None)
     assert st != B.MK_OK and n.value == 0          # a host-only context cannot time anything
     assert m.n_sub() == 4 and m.bound_impl(1) == "eltwise"    # bindings untouched
+
+
+def test_unmasked_attention_and_the_encoder_block_on_the_host(ctx):
+    """Shape inference, contracts and implementation legality of MK_OP_ATTENTION and of workload C6."""
+    w = W.c6(0, B=2, S=24, E=256, H=2, F=64, L=2)
+    m = _mod(ctx, w)
+    assert m.n_ops() == 28
+    assert m.value_spec("qkv_0") == (B.MK_BF16, (48, 768), 0)
+    assert m.value_spec("att_1") == (B.MK_BF16, (48, 256), 0)
+    assert m.value_spec("x2_1") == (B.MK_BF16, (48, 256), 0)
+    m.set_decomposition(w.partitions["fused_tails"])
+    assert m.n_sub() == 14
+    # the attention submodule: both kernels that know the unmasked operator, not the one-tile causal kernel
+    assert m.impls(1) == ["attention_tc2", "attention_simt"]
+    ins, outs = m.contract(1)
+    vid = m.value_id
+    assert [n for n, _ in ins] == [vid["qkv_0"]] and [n for n, _ in outs] == [vid["att_0"]]
+    # projection + bias + residual is one GEMM with its tail; the residual's source is a contract input
+    ins, outs = m.contract(2)
+    assert sorted(n for n, _ in ins) == sorted([vid["att_0"], vid["x"]]) and [n for n, _ in outs] == [vid["r1_0"]]
+    assert m.bound_impl(2) == "gemm_tc" and m.bound_impl(3) == "rowop"      # 48 rows: the one-SM form
+    # head_dim 64: only the plain-ALU kernel is legal
+    w64 = W.c6(0, B=1, S=8, E=128, H=2, F=32, L=1)
+    m64 = _mod(ctx, w64)
+    m64.set_decomposition(w64.partitions["fused_tails"])
+    assert m64.impls(1) == ["attention_simt"]
+    # a packed tensor of the wrong width is rejected at creation
+    ops = [dict(o, attrs=dict(o["attrs"])) for o in w.ops]
+    ops[2]["attrs"]["heads"] = 3
+    with pytest.raises(MkError) as e:
+        Module(ctx, ops, {k: (w.dtype, t.shape) for k, t in w.inputs.items()})
+    assert e.value.status == B.MK_ERR_SHAPE_MISMATCH
