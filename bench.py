@@ -39,7 +39,7 @@ NCU_TRAFFIC_BYTES = {"c2": 105.7e6,            # profiles/gemm_tc2_c2.md
                      "c3": 26.25e6,            # profiles/conv3x3_tc2_groupnorm_c3.md (conv; its output stays in L2)
                      "c4": 8 * 52.2e6}         # profiles/attention_tc2_c4.md
 
-DEFAULT_STEPS = {"c1": 2000, "c2": 200, "c3": 400, "c4": 100, "c5": 50, "c6": 100}
+DEFAULT_STEPS = {"c1": 2000, "c2": 200, "c3": 400, "c4": 100, "c5": 50, "c6": 100, "c7": 400}
 
 
 def full_workload(name, seed=0, batch=None, only_ops=None):
@@ -49,7 +49,7 @@ def full_workload(name, seed=0, batch=None, only_ops=None):
     kw = {}
     if batch is not None:
         kw = {"c1": {"M": batch}, "c2": {"M": batch}, "c3": {"NB": batch}, "c4": {"B": batch}, "c5": {"B": batch},
-              "c6": {"B": batch}}[name]
+              "c6": {"B": batch}, "c7": {"NB": batch}}[name]
     w = W.generate.WORKLOADS[name](seed, **kw)
     if only_ops is not None:
         w.ops = w.ops[:only_ops]
@@ -143,7 +143,7 @@ def oracle_sample(name, w, budget_s=12.0):
             s.inputs["x"] = Tensor("x", w.dtype, w.inputs["x"].store[:rows])
             total = w.inputs["x"].shape[0]
             what = f"first {rows} of {total} rows of X"
-        elif name == "c3":
+        elif name in ("c3", "c7"):
             s.inputs["x"] = Tensor("x", w.dtype, w.inputs["x"].store[:frac_units])
             total = w.inputs["x"].shape[0]
             what = f"first {frac_units} of {total} images"
@@ -164,7 +164,7 @@ def oracle_sample(name, w, budget_s=12.0):
             what = f"first {frac_units} of {total} batch elements"
         return s, total, what
 
-    probe_units = {"c1": 64, "c2": 64, "c3": 1, "c4": 1, "c5": 1, "c6": 1}[name]
+    probe_units = {"c1": 64, "c2": 64, "c3": 1, "c4": 1, "c5": 1, "c6": 1, "c7": 1}[name]
     s, total, _ = sub(probe_units)
     t0 = time.perf_counter()
     OM.run_workload(s, [0])
@@ -397,7 +397,7 @@ def run_ours(args):
     # (time, share, algorithmic work, roofline fraction of that subkernel)
     breakdown = None
     dominant = None
-    split_name = {"c1": "split", "c2": "split", "c3": "split2", "c4": "split3", "c5": "fused_tails", "c6": "fused_tails"}.get(name)
+    split_name = {"c1": "split", "c2": "split", "c3": "split2", "c4": "split3", "c5": "fused_tails", "c6": "fused_tails", "c7": "split2"}.get(name)
     if rank == 0 and split_name in w.partitions:
         pk_ = peaks()
         dw = sets[0]
@@ -476,7 +476,7 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c2", choices=["c1", "c2", "c3", "c4", "c5", "c6"])
+    ap.add_argument("--workload", default="c2", choices=["c1", "c2", "c3", "c4", "c5", "c6", "c7"])
     ap.add_argument("--decomposition", default=None)
     ap.add_argument("--batch", type=int, default=None, help="smaller leading batch dimension (profiler captures)")
     ap.add_argument("--only-ops", type=int, default=None, help="run the first N operators alone (profiler captures)")

@@ -106,6 +106,10 @@ typedef struct mk_tensor_spec {
  *                   Output is the logical [B*S, H*D] matrix (head-major columns).
  *   ATTENTION       the same without the mask: softmax(Q K^T / sqrt(D)) V over every key (the encoder
  *                   attention of the paper's transformer-block example); attributes and layouts as above.
+ *   AVGPOOL2D, MAXPOOL2D, LPPOOL2D   NHWC, square window i[0] = k, stride i[1], no padding, output
+ *                   [N, (H - k) / stride + 1, (W - k) / stride + 1, C] (whole windows only).  Mean, maximum, and
+ *                   the p-norm (sum |x|^p)^(1/p) with p = f[0] >= 1 of each window: the pooling subkernel of the
+ *                   paper's MobileNetV1 example and the two variants of its transfer study.
  * Definitions: the paper's subkernel listings (linear with W stored [K, N]; LayerNorm; online-
  * softmax attention) and its correctness appendix (safe softmax, tril(diagonal=0) mask, fp32
  * accumulation); RMSNorm, GroupNorm, SwiGLU, tanh-GELU and the 3x3 convolution follow the
@@ -127,7 +131,10 @@ typedef enum {
   MK_OP_GROUPNORM = 13,
   MK_OP_SOFTMAX = 14,
   MK_OP_ATTENTION_CAUSAL = 15,
-  MK_OP_ATTENTION = 16
+  MK_OP_ATTENTION = 16,
+  MK_OP_AVGPOOL2D = 17,
+  MK_OP_MAXPOOL2D = 18,
+  MK_OP_LPPOOL2D = 19
 } mk_op_kind;
 
 /* Value numbering: module input k has id k; operator j produces id n_inputs + j.

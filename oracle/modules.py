@@ -53,6 +53,12 @@ def apply_op(op, vals, params):
         if a["layout"] == "bhsd":
             return O.attention_causal_bhsd(ins[0], ins[1], ins[2])
         return O.attention_causal_packed(ins[0], a["batch"], a["seq"], a["heads"], a["head_dim"])
+    if kind == "avgpool":
+        return O.avgpool_nhwc(ins[0], a["k"], a["stride"])
+    if kind == "maxpool":
+        return O.maxpool_nhwc(ins[0], a["k"], a["stride"])
+    if kind == "lppool":
+        return O.lppool_nhwc(ins[0], a["k"], a["stride"], a["p"])
     if kind == "attention":
         if a["layout"] == "bhsd":
             return O.attention_bhsd(ins[0], ins[1], ins[2])

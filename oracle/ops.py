@@ -174,6 +174,38 @@ def groupnorm_nhwc(x, gamma, beta, groups, eps):
     return y
 
 
+# ---------------------------------------------------------------- pooling (NHWC, square window, no padding)
+def _windows(x, k, stride):
+    """x [N, H, W, C] -> [N, OH, OW, k*k, C]: every window written out, OH = (H - k)//stride + 1."""
+    x = _f64(x)
+    n, h, w, c = x.shape
+    if k < 1 or stride < 1 or k > h or k > w:
+        raise ValueError("pooling: bad window")
+    oh, ow = (h - k) // stride + 1, (w - k) // stride + 1
+    out = np.empty((n, oh, ow, k * k, c), F64)
+    for i in range(oh):
+        for j in range(ow):
+            out[:, i, j] = x[:, i * stride:i * stride + k, j * stride:j * stride + k, :].reshape(n, k * k, c)
+    return out
+
+
+def avgpool_nhwc(x, k, stride):
+    """Mean over each k x k window (the pooling of the paper's MobileNetV1 example)."""
+    return _windows(x, k, stride).mean(axis=3)
+
+
+def maxpool_nhwc(x, k, stride):
+    """Maximum over each window (first variant of the paper's transfer study)."""
+    return _windows(x, k, stride).max(axis=3)
+
+
+def lppool_nhwc(x, k, stride, p):
+    """p-norm of each window, (sum |x|^p)^(1/p) (second variant of the transfer study)."""
+    if not p >= 1.0:
+        raise ValueError("lppool: p must be >= 1")
+    return (np.abs(_windows(x, k, stride)) ** F64(p)).sum(axis=3) ** (1.0 / F64(p))
+
+
 # ---------------------------------------------------------------- attention
 def attention_causal_bhsd(q, k, v):
     """q, k, v [B, H, S, D].  S_ij = (q_i . k_j)/sqrt(D) for j <= i, masked

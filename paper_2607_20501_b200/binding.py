@@ -33,7 +33,7 @@ MK_PREV, MK_NONE = -1, -2
 OP = {
     "linear": 1, "conv2d_3x3": 2, "bias_add": 3, "relu": 4, "gelu_tanh": 5, "silu": 6, "scale": 7,
     "clamp": 8, "residual_add": 9, "swiglu": 10, "layernorm": 11, "rmsnorm": 12, "groupnorm": 13,
-    "softmax": 14, "attention_causal": 15, "attention": 16,
+    "softmax": 14, "attention_causal": 15, "attention": 16, "avgpool": 17, "maxpool": 18, "lppool": 19,
 }
 DTYPE = {"f32": MK_F32, "bf16": MK_BF16}
 
@@ -192,6 +192,10 @@ class Module:
                 d.i[1] = weight_layout
             elif kind == "conv2d_3x3":
                 d.i[0] = int(a["c_out"])
+            elif kind in ("avgpool", "maxpool", "lppool"):
+                d.i[0], d.i[1] = int(a["k"]), int(a["stride"])
+                if kind == "lppool":
+                    d.f[0] = float(a["p"])
             elif kind in ("attention_causal", "attention"):
                 d.i[0], d.i[1] = a["heads"], a["head_dim"]
                 if a["layout"] == "packed_qkv":

@@ -137,6 +137,17 @@ mk_status infer_shapes(Module& m, std::string& err) {
         if (d.i[0] < 1 || last % d.i[0]) { err = at + "GROUPNORM: channels must be divisible by groups"; return MK_ERR_SHAPE_MISMATCH; }
         if (!(d.f[0] >= 0.0)) { err = at + "eps must be >= 0"; return MK_ERR_INVALID_ARG; }
         break;
+      case MK_OP_AVGPOOL2D:
+      case MK_OP_MAXPOOL2D:
+      case MK_OP_LPPOOL2D: {
+        const int64_t k = d.i[0], st = d.i[1];
+        if (x.rank != 4) { err = at + "pooling takes an NHWC rank-4 input"; return MK_ERR_SHAPE_MISMATCH; }
+        if (k < 1 || st < 1) { err = at + "pooling needs i[0] = window >= 1 and i[1] = stride >= 1"; return MK_ERR_INVALID_ARG; }
+        if (k > x.shape[1] || k > x.shape[2]) { err = at + "pooling window larger than the image"; return MK_ERR_SHAPE_MISMATCH; }
+        if (d.kind == MK_OP_LPPOOL2D && !(d.f[0] >= 1.0)) { err = at + "LPPOOL2D needs f[0] = p >= 1"; return MK_ERR_INVALID_ARG; }
+        y = make_spec(dtype, {x.shape[0], (x.shape[1] - k) / st + 1, (x.shape[2] - k) / st + 1, x.shape[3]});
+        break;
+      }
       case MK_OP_ATTENTION_CAUSAL:
       case MK_OP_ATTENTION: {
         const int64_t H = d.i[0], D = d.i[1];
@@ -191,8 +202,9 @@ void contract_of(const Module& m, int lo, int hi, std::vector<int>& in_ids, std:
 
 static std::string kind_name(int32_t k) {
   static const char* names[] = {"?", "LINEAR", "CONV2D_3X3", "BIAS_ADD", "RELU", "GELU_TANH", "SILU", "SCALE", "CLAMP",
-                                "RESIDUAL_ADD", "SWIGLU", "LAYERNORM", "RMSNORM", "GROUPNORM", "SOFTMAX", "ATTENTION_CAUSAL", "ATTENTION"};
-  return (k >= 1 && k <= 16) ? names[k] : "?";
+                                "RESIDUAL_ADD", "SWIGLU", "LAYERNORM", "RMSNORM", "GROUPNORM", "SOFTMAX", "ATTENTION_CAUSAL", "ATTENTION",
+                                "AVGPOOL2D", "MAXPOOL2D", "LPPOOL2D"};
+  return (k >= 1 && k <= 19) ? names[k] : "?";
 }
 
 mk_status default_binding(const Module& m, int lo, int hi, Binding& out, std::string& err) {

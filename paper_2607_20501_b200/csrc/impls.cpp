@@ -65,6 +65,23 @@ mk_status eltwise_emit(const Module& m, int lo, int hi, const Resolved& r, std::
   return MK_OK;
 }
 
+// ------------------------------------------------------------------ pooling
+bool is_pool(int32_t k) { return k == MK_OP_AVGPOOL2D || k == MK_OP_MAXPOOL2D || k == MK_OP_LPPOOL2D; }
+bool pool_match(const Module& m, int lo, int hi) { return hi - lo == 1 && is_pool(m.ops[lo].d.kind) && in_is_module_dtype(m, lo); }
+mk_status pool_emit(const Module& m, int lo, int, const Resolved& r, std::vector<Launch>& out, std::string&) {
+  const Op& op = m.ops[lo];
+  const mk_tensor_spec& xs = m.vspec(op.in_id[0]);
+  const void* x = r.value_ptr[op.in_id[0]];
+  void* y = r.value_ptr[op.out_id];
+  const int d = dt(m), sms = m.ctx->sm_count;
+  const int mode = op.d.kind == MK_OP_AVGPOOL2D ? POOL_AVG : op.d.kind == MK_OP_MAXPOOL2D ? POOL_MAX : POOL_LP;
+  const int64_t nb = xs.shape[0], h = xs.shape[1], w = xs.shape[2], c = xs.shape[3];
+  const int k = (int)op.d.i[0], st = (int)op.d.i[1];
+  const float p = (float)op.d.f[0];
+  out.push_back([=](cudaStream_t s) { return launch_pool_nhwc(d, mode, x, y, nb, h, w, c, k, st, p, sms, s); });
+  return MK_OK;
+}
+
 // ------------------------------------------------------------------ row reductions
 bool is_rowop(int32_t k) { return k == MK_OP_LAYERNORM || k == MK_OP_RMSNORM || k == MK_OP_SOFTMAX; }
 int row_mode(int32_t k) { return k == MK_OP_LAYERNORM ? ROW_LAYERNORM : k == MK_OP_RMSNORM ? ROW_RMSNORM : ROW_SOFTMAX; }
@@ -434,6 +451,7 @@ const std::vector<Impl>& registry() {
       {"rowop", rowop_match, no_scratch, rowop_emit},
       {"groupnorm_nhwc", groupnorm_match, groupnorm_scratch, groupnorm_emit},
       {"eltwise", eltwise_match, no_scratch, eltwise_emit},
+      {"pool_nhwc", pool_match, no_scratch, pool_emit},
   };
   return reg;
 }

@@ -108,6 +108,11 @@ cudaError_t launch_groupnorm_apply_partials(int dtype, const void* x, void* y, i
                                             const void* gamma, const void* beta, float eps, const float* stats, int stat_slots,
                                             int sm_count, cudaStream_t s);
 
+// Pooling over NHWC [nb, h, w, c], square window k, stride, no padding: mode 0 mean, 1 maximum, 2 p-norm.
+enum PoolMode : int32_t { POOL_AVG = 0, POOL_MAX = 1, POOL_LP = 2 };
+cudaError_t launch_pool_nhwc(int dtype, int mode, const void* x, void* y, int64_t nb, int64_t h, int64_t w, int64_t c, int k,
+                             int stride, float p, int sm_count, cudaStream_t s);
+
 // ---- plain-ALU (SIMT) kernels: any shape, fp32 or bf16, fp32 accumulation -------------------------
 // Y[M, N] = program(A[M, K] @ W); W is [K, N] row-major, or [N, K] when w_transposed.
 // swiglu: W has 2N logical columns [gate | up] and Y = program(silu(A Wg) * (A Wu)).

@@ -249,3 +249,22 @@ def test_unmasked_attention_and_the_encoder_block_on_the_host(ctx):
     with pytest.raises(MkError) as e:
         Module(ctx, ops, {k: (w.dtype, t.shape) for k, t in w.inputs.items()})
     assert e.value.status == B.MK_ERR_SHAPE_MISMATCH
+
+
+def test_pooling_operators_on_the_host(ctx):
+    for pool in ("avg", "max", "lp"):
+        w = W.c7(0, NB=2, H=20, W=17, C=8, CO=16, pool=pool, k=3, stride=2)
+        m = _mod(ctx, w)
+        assert m.value_spec("y3") == (B.MK_BF16, (2, 9, 8, 16), 0)      # floor((20 - 3) / 2) + 1, floor((17 - 3) / 2) + 1
+        m.set_decomposition(w.partitions["split2"])
+        assert m.impls(1) == ["pool_nhwc"]
+        m.total_fuse()
+        assert m.bound_impl(0).endswith("+pool_nhwc")                   # no kernel fuses a pooling window into a producer
+    bad = W.c7(0, NB=1, H=6, W=6, C=8, CO=8, pool="avg", k=7, stride=7)   # window larger than the image
+    with pytest.raises(MkError) as e:
+        _mod(ctx, bad)
+    assert e.value.status == B.MK_ERR_SHAPE_MISMATCH
+    bad = W.c7(0, NB=1, H=8, W=8, C=8, CO=8, pool="lp", k=2, stride=2, p=0.5)
+    with pytest.raises(MkError) as e:
+        _mod(ctx, bad)
+    assert e.value.status == B.MK_ERR_INVALID_ARG

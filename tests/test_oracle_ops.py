@@ -380,3 +380,47 @@ def test_full_attention_closed_forms_and_invariants():
     v2 = rnd(b, h, s, d)
     lin = O.attention_bhsd(q, k, 2.0 * v - 3.0 * v2) - (2.0 * O.attention_bhsd(q, k, v) - 3.0 * O.attention_bhsd(q, k, v2))
     assert np.abs(lin).max() < 1e-12
+
+
+# ------------------------------------------------------------------ pooling
+def test_pooling_brute_force_library_and_invariants():
+    n, h, w, c = 2, 7, 9, 3
+    x = rnd(n, h, w, c)
+    for k, st in ((2, 2), (3, 2), (3, 1), (7, 7), (1, 1)):
+        oh, ow = (h - k) // st + 1, (w - k) // st + 1
+        avg = O.avgpool_nhwc(x, k, st)
+        mx = O.maxpool_nhwc(x, k, st)
+        l2 = O.lppool_nhwc(x, k, st, 2.0)
+        l3 = O.lppool_nhwc(x, k, st, 3.0)
+        assert avg.shape == mx.shape == l2.shape == (n, oh, ow, c)
+        # brute force, one output at a time
+        for ni in range(n):
+            for i in range(oh):
+                for j in range(ow):
+                    for ci in range(c):
+                        win = [float(x[ni, i * st + a, j * st + b, ci]) for a in range(k) for b in range(k)]
+                        assert abs(avg[ni, i, j, ci] - sum(win) / len(win)) < 1e-13
+                        assert mx[ni, i, j, ci] == max(win)
+                        assert abs(l2[ni, i, j, ci] - math.sqrt(sum(v * v for v in win))) < 1e-13
+                        assert abs(l3[ni, i, j, ci] - sum(abs(v) ** 3 for v in win) ** (1 / 3)) < 1e-13
+        # library routines (NCHW)
+        t = torch.from_numpy(x).permute(0, 3, 1, 2)
+        assert np.allclose(avg, torch.nn.functional.avg_pool2d(t, k, st).permute(0, 2, 3, 1).numpy(), atol=1e-14)
+        assert np.array_equal(mx, torch.nn.functional.max_pool2d(t, k, st).permute(0, 2, 3, 1).numpy())
+        assert np.allclose(l2, torch.nn.functional.lp_pool2d(t, 2.0, k, st).permute(0, 2, 3, 1).numpy(), atol=1e-13)
+        # invariants: max >= mean; p-norms decrease in p and are bounded below by the largest magnitude
+        assert (mx >= avg - 1e-15).all()
+        amax = O.maxpool_nhwc(np.abs(x), k, st)
+        l1 = O.lppool_nhwc(x, k, st, 1.0)
+        assert (l1 >= l2 - 1e-12).all() and (l2 >= l3 - 1e-12).all() and (l3 >= amax - 1e-12).all()
+        assert np.allclose(l1, k * k * O.avgpool_nhwc(np.abs(x), k, st), atol=1e-13)
+        l20 = O.lppool_nhwc(x, k, st, 20.0)                                            # p -> infinity tends to the maximum:
+        assert (l20 >= amax * (1 - 1e-12)).all() and (l20 <= amax * (k * k) ** (1 / 20.0) * (1 + 1e-12)).all()
+    # a constant image: mean and max return the constant, the p-norm k^(2/p) times it
+    cst = np.full((1, 6, 6, 2), 1.5)
+    assert np.allclose(O.avgpool_nhwc(cst, 3, 3), 1.5) and np.allclose(O.maxpool_nhwc(cst, 3, 3), 1.5)
+    assert np.allclose(O.lppool_nhwc(cst, 3, 3, 2.0), 1.5 * 3.0)
+    # the rows and columns that no whole window covers are dropped (floor), not padded
+    assert O.avgpool_nhwc(rnd(1, 8, 8, 1), 3, 2).shape == (1, 3, 3, 1)
+    with pytest.raises(ValueError):
+        O.avgpool_nhwc(rnd(1, 2, 2, 1), 3, 1)

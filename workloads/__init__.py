@@ -14,6 +14,7 @@ from .generate import (  # noqa: F401
     c4,
     c5,
     c6,
+    c7,
     f32_to_bf16_bits,
     int_valued,
     make,

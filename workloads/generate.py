@@ -323,4 +323,29 @@ def c6(seed=0, B=16, S=512, E=1024, H=8, F=4096, L=2, dtype="bf16") -> Workload:
     return w
 
 
-WORKLOADS = {"c1": c1, "c2": c2, "c3": c3, "c4": c4, "c5": c5, "c6": c6}
+# --------------------------------------------------------------------------
+# C7: bf16 conv3x3 -> +bias -> ReLU -> pooling (mean / maximum / p-norm): the convolution stage and the
+# swappable pooling subkernel of the paper's MobileNetV1 transfer study, at C3's convolution shape
+# --------------------------------------------------------------------------
+def c7(seed=0, NB=32, H=56, W=56, C=128, CO=128, pool="avg", k=7, stride=7, p=2.0, dtype="bf16") -> Workload:
+    w = Workload("c7", dtype)
+    w.inputs["x"] = make("x", dtype, _normal(seed, 0, (NB, H, W, C)))
+    w.params["Wc"] = make("Wc", dtype, _normal(seed, 1, (CO, 3, 3, C), std=(1.0 / (9 * C)) ** 0.5))
+    w.params["bias"] = make("bias", dtype, _normal(seed, 2, (CO,), std=0.02))
+    attrs = {"k": k, "stride": stride}
+    if pool == "lp":
+        attrs["p"] = p
+    w.ops = [
+        _op("conv2d_3x3", "y0", ["x"], {"w": "Wc"}, c_out=CO),
+        _op("bias_add", "y1", ["y0"], {"b": "bias"}),
+        _op("relu", "y2", ["y1"]),
+        _op(pool + "pool", "y3", ["y2"], **attrs),
+    ]
+    w.partitions = {"fused": [0], "split2": [0, 3], "per_op": [0, 1, 2, 3]}
+    oh, ow = (H - k) // stride + 1, (W - k) // stride + 1
+    w.flops = 2.0 * NB * H * W * CO * 9 * C
+    w.min_bytes = 2 * (NB * H * W * C + CO * 9 * C + CO + NB * oh * ow * CO)
+    return w
+
+
+WORKLOADS = {"c1": c1, "c2": c2, "c3": c3, "c4": c4, "c5": c5, "c6": c6, "c7": c7}
