@@ -249,13 +249,19 @@ def run_reference(args):
 # ----------------------------------------------------------------------------------------------------
 # GPU arm
 # ----------------------------------------------------------------------------------------------------
-def roofline_of(name, launches_per_step, dominant, achieved, peak, pk, kernel_ms, t_roof_ms, ms_per_step, min_step_ms):
+# nominal B200 figures, for the second column the metric asks for (context, not the denominator of `frac`)
+NOMINAL = {"bf16_tflops": 2250.0, "hbm_gbs": 8000.0}
+
+
+def roofline_of(name, launches_per_step, dominant, achieved, peak, pk, kernel_ms, t_roof_ms, ms_per_step, min_step_ms,
+                median_step_ms=None, t_roof_nominal_ms=None):
     """Roofline object of the dominant kernel.  A one-launch step is timed directly by the per-step
     event pairs; in a multi-kernel step the dominant kernel's duration comes from the per-submodule
     event pairs of mk_module_profile (mean over its launches)."""
     r = {"bound": "tensor" if peak > 100 else "alu", "unit": "TFLOP/s", "peak": peak, "peak_source": pk["_source"] if peak > 100 else "derived",
          "traffic": NCU_TRAFFIC_BYTES.get(name), "module_t_roof_ms": t_roof_ms, "module_frac": t_roof_ms / ms_per_step,
-         "min_step_ms": min_step_ms}
+         "min_step_ms": min_step_ms, "median_step_ms": median_step_ms,
+         "module_frac_of_nominal": (t_roof_nominal_ms / ms_per_step) if t_roof_nominal_ms else None}
     if launches_per_step == 1 or dominant is None:
         r.update({"kernel": "whole step (one launch)", "achieved": achieved, "frac": achieved / peak, "kernel_ms": kernel_ms})
     else:
@@ -449,7 +455,10 @@ def run_ours(args):
                               "smaller than L2 and bound by launch latency, so L2 residency is part of the measurement)"),
                        "shapes": {k: list(t.shape) for k, t in w.inputs.items()},
                        **({"cut": {"batch": args.batch, "only_ops": args.only_ops}} if (args.batch or args.only_ops) else {})},
-            "roofline": roofline_of(name, launches_per_step, dominant, achieved, peak, pk, kernel_ms, t_roof_ms, ms_per_step, step_ms[0]),
+            "roofline": roofline_of(name, launches_per_step, dominant, achieved, peak, pk, kernel_ms, t_roof_ms, ms_per_step, step_ms[0],
+                                    median_step_ms=step_ms[len(step_ms) // 2],
+                                    t_roof_nominal_ms=(None if w.dtype == "f32" else
+                                                       max(w.flops / (NOMINAL["bf16_tflops"] * 1e12), w.min_bytes / (NOMINAL["hbm_gbs"] * 1e9)) * 1e3)),
             "e2e": {"value": world * w.flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
             "gpu_launches": launches_per_step * args.steps,
