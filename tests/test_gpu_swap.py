@@ -55,3 +55,19 @@ def test_composer_chosen_chains_survive(ctx):
     n, _ = dw.swap(iters=2)
     assert n == 0 and dw.module.bound_impl(0) == chain
     assert_parity(to_host_f64(dw.forward()), ref, "bf16", "chain kept")
+
+
+def test_swap_on_the_encoder_block(ctx):
+    """The unmasked attention bound to the plain-ALU kernel and two residual GEMMs bound to the plain-ALU GEMM are
+    found and rebound; the pooling-free, single-implementation submodules (LayerNorm) are left as they are."""
+    w = W.c6(0, B=2, S=256, E=256, H=2, F=512, L=1)
+    ref, _ = oracle(w, None)
+    cuts = w.partitions["fused_tails"]
+    dw, out = run_gpu(ctx, w, cuts, binds={1: "attention_simt", 2: "gemm_simt", 5: "gemm_simt"})
+    before = [dw.module.bound_impl(s) for s in range(7)]
+    assert before[1] == "attention_simt" and before[2] == "gemm_simt" and before[5] == "gemm_simt"
+    n, times = dw.swap(iters=3, tau=0.9)
+    after = [dw.module.bound_impl(s) for s in range(7)]
+    assert n >= 3 and after[1] == "attention_tc2" and not any("simt" in a for a in after)
+    assert after[3] == before[3] == "rowop" and after[6] == before[6] == "rowop"
+    assert_parity(to_host_f64(dw.forward()), ref, "bf16", "encoder block after swap")
