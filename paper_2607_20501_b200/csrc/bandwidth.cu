@@ -649,7 +649,30 @@ __global__ void __launch_bounds__(GN_THREADS, 3) groupnorm_apply_partials_kernel
   if (parts < 1) parts = 1;
   if (parts > 8) parts = 8;
   const bool small = ncol <= 128 && parts > 1;
-  if (small) {
+  const int quads = ncol / 4;                         // 16-byte pieces per slot
+  if (ncol % 4 == 0 && quads <= 16 && GN_THREADS / quads <= 16 && stat_slots <= 8 * (GN_THREADS / quads)) {
+    // a slot is a few hundred contiguous bytes: 16-byte loads, every thread's (at most eight) in flight at once,
+    // so the whole reduction costs one round trip to L2 instead of two or more
+    const int lanes = GN_THREADS / quads;             // slots read side by side
+    const int qd = threadIdx.x % quads, sl = threadIdx.x / quads;
+    float4 t[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int k = sl + u * lanes;
+      t[u] = (sl < lanes && k < stat_slots) ? *reinterpret_cast<const float4*>(st + (int64_t)k * ncol + qd * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    float4 a = t[0];
+#pragma unroll
+    for (int u = 1; u < 8; ++u) { a.x += t[u].x; a.y += t[u].y; a.z += t[u].z; a.w += t[u].w; }
+    float* pp = &sh_part[0][0];                        // [lanes <= 16][ncol <= 64] floats: 8 x 128 are enough
+    if (sl < lanes) *reinterpret_cast<float4*>(pp + sl * ncol + qd * 4) = a;
+    __syncthreads();
+    if ((int)threadIdx.x < ncol) {
+      float acc = 0.0f;
+      for (int p = 0; p < lanes; ++p) acc += pp[p * ncol + threadIdx.x];
+      sh_stat[threadIdx.x] = acc;
+    }
+  } else if (small) {
     const int col = threadIdx.x % ncol, part = threadIdx.x / ncol;
     if (part < parts) {
       float acc = 0.0f;
