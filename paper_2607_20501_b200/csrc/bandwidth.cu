@@ -345,16 +345,24 @@ __global__ void __launch_bounds__(256) pool_nhwc_kernel(const T* __restrict__ x,
       const int64_t n = q / oh;
       const T* base = x + ((n * h + (int64_t)oy * stride) * w + (int64_t)ox * stride) * c + vc * VE;
       for (int a = r; a < k; a += R) {
-#pragma unroll 4
-        for (int b = 0; b < k; ++b) {
-          float v[VE];
-          ld_vec(base + ((int64_t)a * w + b) * c, v);
+        // a window row in pieces of up to eight pixels: all of a piece's loads are issued before any is used
+        for (int b0 = 0; b0 < k; b0 += 8) {
+          RawVec<T, VE> raw[8];
 #pragma unroll
-          for (int e = 0; e < VE; ++e) {
-            if (MODE == POOL_AVG) acc[e] += v[e];
-            else if (MODE == POOL_MAX) acc[e] = fmaxf(acc[e], v[e]);
-            else acc[e] += p == 2.0f ? v[e] * v[e] : __powf(fabsf(v[e]), p);
-          }
+          for (int u = 0; u < 8; ++u)
+            if (b0 + u < k) raw[u].load(base + ((int64_t)a * w + b0 + u) * c);
+#pragma unroll
+          for (int u = 0; u < 8; ++u)
+            if (b0 + u < k) {
+              float v[VE];
+              raw[u].unpack(v);
+#pragma unroll
+              for (int e = 0; e < VE; ++e) {
+                if (MODE == POOL_AVG) acc[e] += v[e];
+                else if (MODE == POOL_MAX) acc[e] = fmaxf(acc[e], v[e]);
+                else acc[e] += p == 2.0f ? v[e] * v[e] : __powf(fabsf(v[e]), p);
+              }
+            }
         }
       }
     }
