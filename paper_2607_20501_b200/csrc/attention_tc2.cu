@@ -128,43 +128,44 @@ __device__ __forceinline__ void umma_ts_lohi(uint32_t d_tmem, uint32_t a_tmem, u
       "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
       : "memory");
 }
-// Eight MMAs (one 128-wide K or key tile) from operands that are already in registers: the issuing
-// thread spends one instruction per MMA once the data it waits for has arrived.
-__device__ __forceinline__ void umma_ss_x8(uint32_t d, const uint64_t (&a)[8], const uint64_t (&b)[8], uint32_t idesc) {
+// Eight MMAs (one 128-wide K or key tile).  The descriptors are formed inside the block from two base words and
+// compile-time offsets (two adds and two moves per MMA, which run while the MMA before executes): the issuing
+// thread keeps four words in registers across its waits instead of thirty-two.
+// a_lo / b_lo: low descriptor words (address >> 4 | ...) of the first K slice; slice k sits OFF(k) further, where
+// OFF(k) = (k / 4) * (SUB_BYTES >> 4) + (k % 4) * 2 (two 64-element sub-tiles of four 16-element slices each).
+#define MK_SS_STEP(OFF, PRED)                                   \
+  "add.u32 la, %2, " #OFF ";\n\tadd.u32 lb, %3, " #OFF ";\n\t" \
+  "mov.b64 da, {la, %4};\n\tmov.b64 db, {lb, %4};\n\t"         \
+  "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %1, " #PRED ";\n\t"
+__device__ __forceinline__ void umma_ss_x8(uint32_t d, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc) {
+  static_assert((SUB_BYTES >> 4) == 1024, "offsets below");
   asm volatile(
-      "{\n\t.reg .pred p, q;\n\t"
+      "{\n\t.reg .pred p, q;\n\t.reg .b32 la, lb;\n\t.reg .b64 da, db;\n\t"
       "setp.ne.b32 p, %1, %1;\n\t"
       "setp.eq.b32 q, %1, %1;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %2, %10, %1, p;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %3, %11, %1, q;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %4, %12, %1, q;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %5, %13, %1, q;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %6, %14, %1, q;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %7, %15, %1, q;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %8, %16, %1, q;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %9, %17, %1, q;\n\t}" ::"r"(d),
-      "r"(idesc), "l"(a[0]), "l"(a[1]), "l"(a[2]), "l"(a[3]), "l"(a[4]), "l"(a[5]), "l"(a[6]), "l"(a[7]), "l"(b[0]), "l"(b[1]), "l"(b[2]),
-      "l"(b[3]), "l"(b[4]), "l"(b[5]), "l"(b[6]), "l"(b[7])
+      MK_SS_STEP(0, p) MK_SS_STEP(2, q) MK_SS_STEP(4, q) MK_SS_STEP(6, q)
+      MK_SS_STEP(1024, q) MK_SS_STEP(1026, q) MK_SS_STEP(1028, q) MK_SS_STEP(1030, q)
+      "}" ::"r"(d), "r"(idesc), "r"(a_lo), "r"(b_lo), "r"(desc_hi)
       : "memory");
 }
-// D (+)= A[tmem] B[smem]; the first MMA accumulates only if acc0 != 0
-__device__ __forceinline__ void umma_ts_x8(uint32_t d, const uint32_t (&a)[8], const uint64_t (&b)[8], uint32_t idesc, uint32_t acc0) {
+#undef MK_SS_STEP
+// D (+)= A[tmem] B[smem]; the first MMA accumulates only if acc0 != 0.  A: 8 TMEM columns per 16-key slice;
+// B (= V, MN-major): 16 keys = 16 rows of 128 bytes = 128 descriptor units per slice.
+#define MK_TS_STEP(K, PRED)                                             \
+  "add.u32 ta, %3, " #K "*8;\n\tadd.u32 lb, %4, " #K "*128;\n\t"       \
+  "mov.b64 db, {lb, %5};\n\t"                                          \
+  "tcgen05.mma.cta_group::1.kind::f16 [%0], [ta], db, %1, " #PRED ";\n\t"
+__device__ __forceinline__ void umma_ts_x8(uint32_t d, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi, uint32_t idesc, uint32_t acc0) {
   asm volatile(
-      "{\n\t.reg .pred p, q;\n\t"
+      "{\n\t.reg .pred p, q;\n\t.reg .b32 ta, lb;\n\t.reg .b64 db;\n\t"
       "setp.ne.b32 p, %2, 0;\n\t"
       "setp.eq.b32 q, %1, %1;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%3], %11, %1, p;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%4], %12, %1, q;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%5], %13, %1, q;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%6], %14, %1, q;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%7], %15, %1, q;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%8], %16, %1, q;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%9], %17, %1, q;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%10], %18, %1, q;\n\t}" ::"r"(d),
-      "r"(idesc), "r"(acc0), "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(a[4]), "r"(a[5]), "r"(a[6]), "r"(a[7]), "l"(b[0]), "l"(b[1]),
-      "l"(b[2]), "l"(b[3]), "l"(b[4]), "l"(b[5]), "l"(b[6]), "l"(b[7])
+      MK_TS_STEP(0, p) MK_TS_STEP(1, q) MK_TS_STEP(2, q) MK_TS_STEP(3, q)
+      MK_TS_STEP(4, q) MK_TS_STEP(5, q) MK_TS_STEP(6, q) MK_TS_STEP(7, q)
+      "}" ::"r"(d), "r"(idesc), "r"(acc0), "r"(a_tmem), "r"(b_lo), "r"(b_hi)
       : "memory");
 }
+#undef MK_TS_STEP
 // keep a value computed before a wait in a register across it
 __device__ __forceinline__ void pin(uint32_t& x) { asm volatile("" : "+r"(x)); }
 __device__ __forceinline__ void pin(uint64_t& x) { asm volatile("" : "+l"(x)); }
@@ -288,40 +289,20 @@ __device__ __forceinline__ void role_mma(const Ctx& cx, uint32_t tmem_base, int 
   auto issue = [&](const Pos& a, bool do_pv, const Pos& b, bool do_qk) -> bool {
     const uint32_t ga = a.g + (uint32_t)a.j, gb = b.g + (uint32_t)b.j;
     const int sta = ga % KV_STAGES, stb = gb % KV_STAGES;
-    uint32_t pa[8];
-    uint64_t vb[8], qa[8], kb[8];
     bool lo_done = false, hi_done = false;
-    if (do_pv) {
-      const uint32_t v_lo = v_lo0 + (uint32_t)sta * (TILE_BYTES >> 4);
-#pragma unroll
-      for (int k = 0; k < 8; ++k) {
-        pa[k] = s_tmem + k * 8;
-        vb[k] = ((uint64_t)v_hi << 32) | (v_lo + (uint32_t)(k * ((16 * 128) >> 4)));
-        pin(pa[k]);
-        pin(vb[k]);
-      }
-    }
+    uint32_t v_lo = v_lo0 + (uint32_t)sta * (TILE_BYTES >> 4);
+    uint32_t k_lo = k_lo0 + (uint32_t)stb * (TILE_BYTES >> 4);
+    pin(v_lo);
+    pin(k_lo);
     auto issue_lo = [&]() {
-      umma_ss_x8(s_tmem + 64, qa, kb, idesc_qk64);
+      umma_ss_x8(s_tmem + 64, q_lo, k_lo, tc::kDescHiSw128, idesc_qk64);
       tc::umma_commit(&sh->s_lo_full[t]);
     };
     auto issue_hi = [&]() {
-      uint64_t kh[8];
-#pragma unroll
-      for (int k = 0; k < 8; ++k) kh[k] = kb[k] + (uint64_t)((64 * 128) >> 4);   // key rows 64..127 of the K tile
-      umma_ss_x8(s_tmem, qa, kh, idesc_qk64);
+      umma_ss_x8(s_tmem, q_lo, k_lo + (uint32_t)((64 * 128) >> 4), tc::kDescHiSw128, idesc_qk64);   // key rows 64..127 of the K tile
       tc::umma_commit(&sh->s_hi_full[t]);
     };
     if (do_qk) {
-      const uint32_t k_lo = k_lo0 + (uint32_t)stb * (TILE_BYTES >> 4);
-#pragma unroll
-      for (int k = 0; k < 8; ++k) {
-        const uint32_t off = (uint32_t)((k >> 2) * (SUB_BYTES >> 4) + (k & 3) * 2);
-        qa[k] = ((uint64_t)tc::kDescHiSw128 << 32) | (q_lo + off);
-        kb[k] = ((uint64_t)tc::kDescHiSw128 << 32) | (k_lo + off);
-        pin(qa[k]);
-        pin(kb[k]);
-      }
       if (!first_qk) {
         // region B has been read (the softmax signals it half-way through tile a)
         if (!cx.wait(&sh->b_free[t], par_bfree, tc::WAIT_TMEM_EMPTY)) return false;
@@ -355,7 +336,7 @@ __device__ __forceinline__ void role_mma(const Ctx& cx, uint32_t tmem_base, int 
       par_pv ^= 1u;
       TR2(a.g == 0 && a.j < 11, (t ? 8 : 4) + a.j * 8);
       tc::tc_fence_after();
-      umma_ts_x8(o_tmem, pa, vb, idesc_pv, a.j > 0 ? 1u : 0u);
+      umma_ts_x8(o_tmem, s_tmem, v_lo, v_hi, idesc_pv, a.j > 0 ? 1u : 0u);
       if (do_qk && lo_done) { issue_hi(); hi_done = true; }
       // a K/V slot is released by two arrivals: one per stream, or both from the only stream that reads it
       if (a.j == a.nt - 1) tc::umma_commit(&sh->o_final[t]);
