@@ -5,6 +5,7 @@
 // fused single-launch kernel in which one CTA owns whole rows so the row norm needs no second pass
 // over memory.
 #include "device_common.cuh"
+#include "tc_common.cuh"
 
 namespace mk {
 
@@ -79,6 +80,194 @@ static cudaError_t gemm_simt_dispatch(const void* a, const void* w, bool wt, voi
   if (swiglu) gemm_simt_kernel<T, TO, true><<<grid, 256, 0, s>>>((const T*)a, (const T*)w, wt, (TO*)y, m, n, k, p);
   else gemm_simt_kernel<T, TO, false><<<grid, 256, 0, s>>>((const T*)a, (const T*)w, wt, (TO*)y, m, n, k, p);
   return cudaGetLastError();
+}
+
+// =====================================================================================================
+// The same fused chain on a thread-block cluster, for the small problems whose whole time is latency (N <= 256):
+// a cluster of eight CTAs owns eight rows, each CTA a slice of the columns, so a CTA loads an eighth of W
+// instead of all of it; the row statistics meet through distributed shared memory (every CTA writes its
+// partial sums into all eight CTAs' slots, one cluster barrier per statistic).  Two-pass LayerNorm
+// (mean, then centred squares), as in the single-CTA form.
+// =====================================================================================================
+constexpr int LC_CL = 8;         // CTAs per cluster
+constexpr int LC_RB = 8;         // rows per cluster
+constexpr int LC_THREADS = 256;
+constexpr int LC_MAXNC = 32;     // columns per CTA: N <= LC_CL * LC_MAXNC
+
+__device__ __forceinline__ void st_cluster_f32(uint32_t cluster_addr, float v) {
+  asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(cluster_addr), "f"(v) : "memory");
+}
+
+template <typename T>
+__global__ void __launch_bounds__(LC_THREADS) linear_rownorm_cluster_kernel(const T* __restrict__ a, const T* __restrict__ w, bool wt,
+                                                                            T* __restrict__ y, int M, int N, int K, int NC,
+                                                                            const __grid_constant__ EpiProgram p, int mode,
+                                                                            const T* __restrict__ gamma, const T* __restrict__ beta,
+                                                                            float eps) {
+  extern __shared__ float smem[];
+  const int KP = K + 1;                                    // odd pitch: threads of different columns hit different banks
+  float* xs = smem;                                        // [LC_RB][K]
+  float* ws = xs + LC_RB * K;                              // [NC][KP]: this CTA's columns of W, K contiguous
+  float* part = ws + NC * KP;                              // [KS][LC_RB * NC]
+  __shared__ float val[LC_RB][LC_MAXNC];                   // this CTA's outputs after the elementwise tail
+  __shared__ float slot[2][LC_CL][LC_RB];                  // row partial sums of every CTA of the cluster (two statistics)
+  __shared__ float stat[2][LC_RB];
+  pdl_launch_dependents();
+  pdl_wait();
+  const uint32_t rank = tc::cluster_ctarank();
+  const int m0 = (int)(blockIdx.x / LC_CL) * LC_RB, c0 = (int)rank * NC;
+  const int nc = min(NC, N - c0) > 0 ? min(NC, N - c0) : 0;   // columns of this CTA that exist
+  // Everything that is read late - the norm's scale and shift, a bias vector inside the elementwise tail - is asked
+  // for now: a dependent global load at the end of this kernel would be a tenth of its whole duration.
+  float ga = 1.0f, be = 0.0f;
+  {
+    const int rj = threadIdx.x, j = rj % NC;
+    if (rj < LC_RB * NC && j < nc) {
+      if (gamma) ga = Elem<T>::ld(gamma + c0 + j);
+      if (mode == ROW_LAYERNORM && beta) be = Elem<T>::ld(beta + c0 + j);
+      for (int i = 0; i < p.n; ++i)
+        if (p.op[i].kind == EPI_BIAS && p.op[i].ptr)
+          asm volatile("prefetch.global.L1 [%0];" ::"l"(reinterpret_cast<const char*>(p.op[i].ptr) + (size_t)(c0 + j) * sizeof(T)));
+    }
+  }
+  constexpr int VE = Elem<T>::VEC;
+  if (K % VE == 0) {
+    // 16-byte loads, all of a thread's in flight together: the whole kernel is a few round trips to L2 long
+    const int kv = K / VE;
+    for (int i = threadIdx.x; i < LC_RB * kv; i += LC_THREADS) {
+      const int r = i / kv, k = (i - r * kv) * VE;
+      float v[VE];
+      if (m0 + r < M) {
+        ld_vec(a + (int64_t)(m0 + r) * K + k, v);
+      } else {
+#pragma unroll
+        for (int e = 0; e < VE; ++e) v[e] = 0.0f;
+      }
+#pragma unroll
+      for (int e = 0; e < VE; ++e) xs[r * K + k + e] = v[e];
+    }
+  } else {
+    for (int i = threadIdx.x; i < LC_RB * K; i += LC_THREADS) {
+      const int r = i / K, k = i - r * K;
+      xs[i] = (m0 + r < M) ? Elem<T>::ld(a + (int64_t)(m0 + r) * K + k) : 0.0f;
+    }
+  }
+  if (wt && K % VE == 0) {
+    const int kv = K / VE;
+    for (int i = threadIdx.x; i < nc * kv; i += LC_THREADS) {
+      const int j = i / kv, k = (i - j * kv) * VE;
+      float v[VE];
+      ld_vec(w + (int64_t)(c0 + j) * K + k, v);
+#pragma unroll
+      for (int e = 0; e < VE; ++e) ws[j * KP + k + e] = v[e];
+    }
+  } else if (wt) {
+    for (int i = threadIdx.x; i < nc * K; i += LC_THREADS) {
+      const int j = i / K, k = i - j * K;                   // consecutive threads walk K: contiguous in memory
+      ws[j * KP + k] = Elem<T>::ld(w + (int64_t)(c0 + j) * K + k);
+    }
+  } else {
+    for (int i = threadIdx.x; i < nc * K; i += LC_THREADS) {
+      const int k = i / nc, j = i - k * nc;                 // consecutive threads walk the columns: contiguous in memory
+      ws[j * KP + k] = Elem<T>::ld(w + (int64_t)k * N + c0 + j);
+    }
+  }
+  __syncthreads();
+  // outputs r * NC + j; the threads beyond them split K
+  const int outs = LC_RB * NC;
+  const int KS = LC_THREADS / outs > 0 ? LC_THREADS / outs : 1;
+  for (int o = threadIdx.x; o < outs * KS; o += LC_THREADS) {
+    const int ks = o / outs, rj = o - ks * outs, r = rj / NC, j = rj - r * NC;
+    const int kper = (K + KS - 1) / KS, kb = ks * kper, ke = min(K, kb + kper);
+    float acc = 0.0f;
+    if (j < nc) {
+      const float* xr = xs + r * K;
+      const float* wr = ws + j * KP;
+#pragma unroll 8
+      for (int k = kb; k < ke; ++k) acc = fmaf(xr[k], wr[k], acc);
+    }
+    part[ks * outs + rj] = acc;
+  }
+  __syncthreads();
+  for (int rj = threadIdx.x; rj < outs; rj += LC_THREADS) {
+    const int r = rj / NC, j = rj - r * NC;
+    float v = 0.0f;
+    for (int q = 0; q < KS; ++q) v += part[q * outs + rj];       // fixed order
+    val[r][j] = j < nc ? epi_apply(p, v, m0 + r, c0 + j, N) : 0.0f;
+  }
+  __syncthreads();
+  const float inv_n = 1.0f / (float)N;
+  // statistic 0: the row sums (LayerNorm) -> mean
+  if (mode == ROW_LAYERNORM) {
+    if (threadIdx.x < LC_RB) {
+      float sm = 0.0f;
+      for (int j = 0; j < nc; ++j) sm += val[threadIdx.x][j];
+      const uint32_t local = tc::smem_u32(&slot[0][rank][threadIdx.x]);
+      for (uint32_t c = 0; c < LC_CL; ++c) st_cluster_f32(tc::map_to_cta(local, c), sm);
+    }
+    tc::cluster_sync();
+    if (threadIdx.x < LC_RB) {
+      float sm = 0.0f;
+      for (int c = 0; c < LC_CL; ++c) sm += slot[0][c][threadIdx.x];   // the same order in every CTA
+      stat[0][threadIdx.x] = sm * inv_n;
+    }
+  } else if (threadIdx.x < LC_RB) {
+    stat[0][threadIdx.x] = 0.0f;
+  }
+  __syncthreads();
+  // statistic 1: centred squares -> 1 / sqrt(var + eps)  (RMSNorm: squares about zero)
+  if (threadIdx.x < LC_RB) {
+    const float mean = stat[0][threadIdx.x];
+    float q = 0.0f;
+    for (int j = 0; j < nc; ++j) { const float d = val[threadIdx.x][j] - mean; q += d * d; }
+    const uint32_t local = tc::smem_u32(&slot[1][rank][threadIdx.x]);
+    for (uint32_t c = 0; c < LC_CL; ++c) st_cluster_f32(tc::map_to_cta(local, c), q);
+  }
+  tc::cluster_sync();
+  if (threadIdx.x < LC_RB) {
+    float q = 0.0f;
+    for (int c = 0; c < LC_CL; ++c) q += slot[1][c][threadIdx.x];
+    stat[1][threadIdx.x] = rsqrtf(q * inv_n + eps);
+  }
+  __syncthreads();
+  for (int rj = threadIdx.x; rj < outs; rj += LC_THREADS) {
+    const int r = rj / NC, j = rj - r * NC;
+    if (j < nc && m0 + r < M) {
+      const int c = c0 + j;
+      const float o = (val[r][j] - stat[0][r]) * stat[1][r] * ga + be;
+      Elem<T>::st(y + (int64_t)(m0 + r) * N + c, o);
+    }
+  }
+  // nobody writes into a peer's shared memory after the second cluster barrier: a CTA may retire here
+}
+
+template <typename T>
+static cudaError_t linear_rownorm_cluster_launch(const void* a, const void* w, bool wt, void* y, int64_t m, int64_t n, int64_t k,
+                                                 const EpiProgram& p, int mode, const void* g, const void* b, float eps, cudaStream_t s) {
+  int NC = (int)((n + LC_CL - 1) / LC_CL);
+  // a power of two keeps LC_RB * NC a divisor of the CTA size, so the idle threads split K evenly
+  int pw = 1;
+  while (pw < NC) pw *= 2;
+  NC = pw;
+  const int outs = LC_RB * NC, KS = LC_THREADS / outs > 0 ? LC_THREADS / outs : 1;
+  const size_t smem = sizeof(float) * ((size_t)LC_RB * k + (size_t)NC * (k + 1) + (size_t)KS * outs);
+  static size_t attr_bytes[2] = {0, 0};
+  size_t& have = attr_bytes[sizeof(T) == 4 ? 0 : 1];
+  if (smem > 48 * 1024 && smem > have) {
+    cudaError_t e = cudaFuncSetAttribute(linear_rownorm_cluster_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    have = smem;
+  }
+  const unsigned grid = (unsigned)((m + LC_RB - 1) / LC_RB) * LC_CL;
+  LaunchCfg lc(PDL_ELTWISE, dim3(grid), dim3(LC_THREADS), smem, s, LC_CL);
+  return cudaLaunchKernelEx(&lc.cfg, linear_rownorm_cluster_kernel<T>, (const T*)a, (const T*)w, wt, (T*)y, (int)m, (int)n, (int)k, NC, p, mode,
+                            (const T*)g, (const T*)b, eps);
+}
+// what the cluster form takes: a row norm with two statistics at most, few columns, operands that fit
+static bool linear_rownorm_cluster_ok(int64_t m, int64_t n, int64_t k, int mode) {
+  if (mode != ROW_LAYERNORM && mode != ROW_RMSNORM) return false;
+  if (n > LC_CL * LC_MAXNC || n < LC_CL || k > 2048 || m > (1 << 20)) return false;
+  return sizeof(float) * ((size_t)(LC_RB + LC_MAXNC) * (k + 1) + LC_THREADS) <= 160 * 1024;
 }
 
 template <typename T>
@@ -232,6 +421,7 @@ static cudaError_t linear_rownorm_dispatch(const void* a, const void* w, bool wt
                                            const EpiProgram& p, int mode, const void* g, const void* b, float eps,
                                            cudaStream_t s) {
   if (m == 0) return cudaSuccess;
+  if (linear_rownorm_cluster_ok(m, n, k, mode)) return linear_rownorm_cluster_launch<T>(a, w, wt, y, m, n, k, p, mode, g, b, eps, s);
   // fewest column threads that cover N with LR_MAXC columns each: the rest of the CTA splits K, which
   // shortens every thread's chain of loads
   int NT = 32;
