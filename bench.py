@@ -431,6 +431,30 @@ def run_ours(args):
                      "submodules": rows if len(rows) <= 12 else rows[:12]}
         dk = max(agg, key=lambda k: agg[k]["ms"])
         dominant = (dk, agg[dk])
+        if graph_info:
+            # launch-bound module: the split decomposition's step by graph replay too (the fused / split comparison)
+            gs = torch.cuda.Stream()
+            gs.wait_stream(stream)
+            with torch.cuda.stream(gs):
+                dw.forward()
+                torch.cuda.synchronize()
+                gsp = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(gsp, stream=gs):
+                    for _ in range(8):
+                        dw.forward()
+                for _ in range(3):
+                    gsp.replay()
+                torch.cuda.synchronize()
+                s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                nrep = max(1, args.steps // 8)
+                s0.record(gs)
+                for _ in range(nrep):
+                    gsp.replay()
+                s1.record(gs)
+                torch.cuda.synchronize()
+            ctx.check()
+            breakdown["graph_ms_per_step"] = s0.elapsed_time(s1) / (nrep * 8)
+            breakdown["launches_per_step"] = dw.module.launch_count()
 
     # ---- max over ranks
     total_ms, kernel_ms, e2e_ms = D.max_over_ranks([total_ms, kernel_ms, e2e_ms], device=f"cuda:{local}")
