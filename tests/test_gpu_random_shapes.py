@@ -87,3 +87,22 @@ def test_pooling_with_random_shape(ctx, i):
     ref, _ = oracle(w, [0])
     _, out = run_gpu(ctx, w, [0])
     assert_parity(out, ref, "bf16", f"{pool} {nb}x{h}x{wd}x{c} k{k} s{st}")
+
+
+FUSED = _cases(5, 36, lambda r: (int(r.integers(1, 200)), int(r.integers(1, 700)), int(r.choice([8, 9, 16, 40, 100, 128, 200, 256, 257, 300, 640, 1024])),
+                                 "f32", str(r.choice(["layernorm", "rmsnorm"])), bool(r.integers(0, 2))))
+
+
+@pytest.mark.parametrize("i", range(len(FUSED)))
+def test_small_fused_chain_with_random_shape(ctx, i):
+    """linear -> +bias -> ReLU -> row norm in one launch: the cluster form (rows up to 256 wide, any K, either weight
+    layout, ragged row and column counts) and the single-CTA form beyond it; fp32, the type this kernel serves."""
+    from paper_2607_20501_b200 import binding as B
+    m, k, n, dtype, norm, row_major = FUSED[i]
+    w = W.c1(400 + i, M=m, K=k, N=n, dtype=dtype)
+    if norm == "rmsnorm":
+        w.ops[-1] = dict(w.ops[-1], kind="rmsnorm", params={"gamma": "gamma"}, attrs={"eps": 1e-6})
+    ref, _ = oracle(w, [0])
+    dw, out = run_gpu(ctx, w, [0], weight_layout=B.MK_LAYOUT_ROW_MAJOR if row_major else None)
+    assert dw.module.bound_impl(0) == "linear_rownorm_simt"
+    assert_parity(out, ref, dtype, f"M{m} K{k} N{n} {dtype} {norm} row_major={row_major}")
