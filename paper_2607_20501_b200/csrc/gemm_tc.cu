@@ -39,7 +39,7 @@ constexpr int BN = 256;   // accumulator columns
 constexpr int BK = 64, UMMA_K = 16;
 constexpr int EPI_WARPS = 8;
 constexpr int THREADS = 64 + 32 * EPI_WARPS;
-constexpr int GROUP_M = 8;  // tile rows walked together for L2 reuse
+constexpr int GROUP_M = 16;  // tile rows walked together for L2 reuse
 
 template <int CTAS> struct Cfg {
   static constexpr int STAGES = CTAS == 2 ? 6 : 4;
