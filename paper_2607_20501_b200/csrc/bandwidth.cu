@@ -320,7 +320,7 @@ cudaError_t launch_rowop(int dtype, int in_dtype, int mode, const void* x, void*
 // channels, so a warp reads contiguous runs of every window pixel; fp32 accumulation.
 // =====================================================================================================
 template <typename T, int MODE>
-__global__ void __launch_bounds__(256) pool_nhwc_kernel(const T* __restrict__ x, T* __restrict__ y, int64_t nb, int h, int w, int c, int oh,
+__global__ void __launch_bounds__(256, 4) pool_nhwc_kernel(const T* __restrict__ x, T* __restrict__ y, int64_t nb, int h, int w, int c, int oh,
                                                         int ow, int k, int stride, float p, float inv_p) {
   // A block = 32 consecutive output vectors (lane) x R window-row slots (warp): warp r takes window rows r, r + R, ...,
   // so a 7 x 7 window is 7 loads per thread instead of 49 in a row, and the grid has R times as many threads.
