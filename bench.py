@@ -1,10 +1,13 @@
 #!/usr/bin/env python
 """Benchmark of the composed forward (one JSON line on stdout).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload c2]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload all|c1..c7]
 
 A step is one composed forward of the workload's module (every submodule of its default
-decomposition) over one batch of seeded synthetic input.  `value` is the whole-job throughput in
+decomposition) over one batch of seeded synthetic input.  With no --workload the run covers the
+five modules of the workload list in one invocation: the line's top level describes C5, the
+largest (the 4-layer decoder; --steps K times exactly K of its forwards), and its `workloads`
+object carries the same measurements of C1-C4, each with the step count it used.  `value` is the whole-job throughput in
 TFLOP/s of algorithmic work with inputs resident in HBM; `e2e` repeats the measurement with the
 step's inputs copied from pinned host memory and its result copied back inside the timed region.
 Each step works on a different copy of the inputs and outputs (a rotation larger than L2), so no
@@ -240,7 +243,8 @@ def run_reference(args):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": mean_s * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": args.workload, "sample": what},
-        "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": what},
+        "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": cores, "kind": "oracle",
+                         "blas": "numpy fp64, contractions through the BLAS numpy links (multi-threaded)", "sample": what},
         "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line))
@@ -272,23 +276,13 @@ def roofline_of(name, launches_per_step, dominant, achieved, peak, pk, kernel_ms
     return r
 
 
-def run_ours(args):
+def measure_one(name, args, steps, ctx, rank, local, world, cpu_seconds):
+    """All measurements of one workload; returns the line's fields on rank 0, None elsewhere."""
     import torch
-    import torch.distributed as dist
     from paper_2607_20501_b200 import dist as D
-
-    rank, local, world = D.env_world()
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback for the product path")
-    torch.cuda.set_device(local)
-    D.init("nccl", torch.device("cuda", local))
-
-    from paper_2607_20501_b200 import Context
     from paper_2607_20501_b200.runner import DeviceWorkload
 
-    name = args.workload
     w = full_workload(name, batch=args.batch, only_ops=args.only_ops)
-    ctx = Context(local)
     # rotation: enough independent copies that a pass over all of them exceeds L2 (126 MB) twice over
     per_copy = sum(t.nbytes() for t in w.inputs.values()) + sum(t.nbytes() for t in w.params.values())
     rot = int(max(2, min(8, -(-300e6 // max(per_copy, 1)))))
@@ -315,13 +309,13 @@ def run_ours(args):
     launches_per_step = sets[0].module.launch_count()
 
     # ---- timed region: K steps, device time, per-step event pairs for the kernel duration
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
     t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sampler = ClockSampler(local)
     sampler.start()
     barrier()
     t_begin.record(stream)
-    for i in range(args.steps):
+    for i in range(steps):
         ev[i][0].record(stream)
         sets[i % rot].forward()
         ev[i][1].record(stream)
@@ -340,10 +334,11 @@ def run_ours(args):
     # into it) and THAT time is reported, with the loop's time beside it; a graph of as many one-element
     # kernels gives the launch floor.
     graph_info = None
-    if kernel_ms < 0.2:
+    sustained = None
+    if kernel_ms < 1.0:
         gstream = torch.cuda.Stream()
         gstream.wait_stream(stream)
-        reps = max(1, args.steps // rot)
+        reps = max(1, steps // rot)
         with torch.cuda.stream(gstream):
             for dw in sets:
                 dw.forward()            # launch plans for this stream exist before capture
@@ -352,29 +347,52 @@ def run_ours(args):
             with torch.cuda.graph(g, stream=gstream):
                 for dw in sets:
                     dw.forward()
-            tiny = torch.zeros(1, device=f"cuda:{local}")
-            gf = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(gf, stream=gstream):
-                for _ in range(rot * launches_per_step):
-                    tiny.add_(1.0)
             for _ in range(3):
-                g.replay(); gf.replay()
-            torch.cuda.synchronize()
-            g0, g1, g2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
-            g0.record(gstream)
-            for _ in range(reps):
                 g.replay()
-            g1.record(gstream)
-            for _ in range(reps):
-                gf.replay()
-            g2.record(gstream)
             torch.cuda.synchronize()
+            if kernel_ms < 0.2:
+                tiny = torch.zeros(1, device=f"cuda:{local}")
+                gf = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(gf, stream=gstream):
+                    for _ in range(rot * launches_per_step):
+                        tiny.add_(1.0)
+                for _ in range(3):
+                    gf.replay()
+                torch.cuda.synchronize()
+                g0, g1, g2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+                g0.record(gstream)
+                for _ in range(reps):
+                    g.replay()
+                g1.record(gstream)
+                for _ in range(reps):
+                    gf.replay()
+                g2.record(gstream)
+                torch.cuda.synchronize()
+                graph_info = {"ms_per_step": g0.elapsed_time(g1) / (reps * rot), "steps": reps * rot,
+                              "launch_floor_ms_per_step": g1.elapsed_time(g2) / (reps * rot),
+                              "eager_ms_per_step": total_ms / steps}
+            # ---- the sustained regime: a sub-millisecond step timed over K steps is a burst measurement (the
+            # whole timed region can be shorter than the power controller's reaction); the same graph replayed
+            # back to back for at least half a second, with the clocks sampled beside it, gives the figure a
+            # long-running job would see
+            n_rep = int(max(1, -(-500.0 // max(kernel_ms * rot, 1e-3))))
+            s_sampler = ClockSampler(local)
+            q0, q1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            s_sampler.start()
+            q0.record(gstream)
+            for _ in range(n_rep):
+                g.replay()
+            q1.record(gstream)
+            torch.cuda.synchronize()
+            s_clocks = s_sampler.stop()
+            sustained = {"ms_per_step": q0.elapsed_time(q1) / (n_rep * rot), "steps": n_rep * rot,
+                         "seconds": q0.elapsed_time(q1) * 1e-3, "timing": "CUDA graph replay, back to back",
+                         "clocks": s_clocks}
         ctx.check()
-        graph_info = {"ms_per_step": g0.elapsed_time(g1) / (reps * rot), "steps": reps * rot,
-                      "launch_floor_ms_per_step": g1.elapsed_time(g2) / (reps * rot),
-                      "eager_ms_per_step": total_ms / args.steps}
-        total_ms = graph_info["ms_per_step"] * args.steps
-        kernel_ms = graph_info["ms_per_step"]
+        if graph_info:
+            total_ms = graph_info["ms_per_step"] * steps
+            kernel_ms = graph_info["ms_per_step"]
 
     # ---- end to end: pinned host inputs in, result out, every step
     host_in = {k: torch.empty(t.shape, dtype=sets[0].inputs[k].dtype).pin_memory() for k, t in w.inputs.items()}
@@ -383,7 +401,7 @@ def run_ours(args):
     host_out = [torch.empty(sets[0].out.shape, dtype=sets[0].out.dtype).pin_memory() for _ in range(rot)]
     h2d = sum(t.numel() * t.element_size() for t in host_in.values())
     d2h = host_out[0].numel() * host_out[0].element_size()
-    e2e_steps = max(3, min(args.steps, 50))
+    e2e_steps = max(3, min(steps, 50))
 
     # Every step copies its inputs in, runs the forward and copies its result out; the three legs run on three
     # streams, so that step i's copy out, step i + 1's forward and step i + 2's copy in overlap (PCIe carries
@@ -481,7 +499,7 @@ def run_ours(args):
                     gsp.replay()
                 torch.cuda.synchronize()
                 s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                nrep = max(1, args.steps // 8)
+                nrep = max(1, steps // 8)
                 s0.record(gs)
                 for _ in range(nrep):
                     gsp.replay()
@@ -496,7 +514,7 @@ def run_ours(args):
 
     if rank == 0:
         pk = peaks()
-        ms_per_step = total_ms / args.steps
+        ms_per_step = total_ms / steps
         value = world * w.flops / (ms_per_step * 1e-3) / 1e12
         achieved = w.flops / (kernel_ms * 1e-3) / 1e12
         peak = pk["bf16_tflops"] if ms_per_step < 1.0 else pk.get("bf16_tflops_sustained", pk["bf16_tflops"])
@@ -505,7 +523,7 @@ def run_ours(args):
             peak = 148 * 128 * 2 * 1.965e9 / 1e12
         t_roof_ms = max(w.flops / (peak * 1e12), w.min_bytes / (pk["hbm_gbs"] * 1e9)) * 1e3
         line = {
-            "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+            "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
             "config": {"workload": name, "decomposition": part, "impls": impls,
@@ -521,19 +539,71 @@ def run_ours(args):
             "e2e": {"value": world * w.flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms,
                     "pipeline": f"copy in / forward / copy out on three streams over {rot} buffer sets"},
-            "gpu_launches": launches_per_step * args.steps,
+            "gpu_launches": launches_per_step * steps,
             "clocks": clocks,
             "per_subkernel": breakdown,
         }
         if graph_info:
             line["config"]["timing"] = "CUDA graph replay (step shorter than 0.2 ms; the Python loop's time is kept beside it in `graph`)"
             line["graph"] = graph_info
+        if sustained:
+            ps = pk.get("bf16_tflops_sustained", pk["bf16_tflops"]) if w.dtype != "f32" else peak
+            t_roof_s = max(w.flops / (ps * 1e12), w.min_bytes / (pk["hbm_gbs"] * 1e9)) * 1e3
+            sustained.update({"value": w.flops / (sustained["ms_per_step"] * 1e-3) / 1e12, "unit": "TFLOP/s", "peak": ps,
+                              "module_t_roof_ms": t_roof_s, "module_frac": t_roof_s / sustained["ms_per_step"]})
+            line["sustained"] = sustained
         if not args.no_cpu and world == 1:
-            f, s, what = oracle_sample(name, w, budget_s=args.cpu_seconds)
+            f, s, what = oracle_sample(name, w, budget_s=cpu_seconds)
             line["cpu_baseline"] = {"value": f / s / 1e12, "unit": "TFLOP/s", "cores": os.cpu_count(), "kind": "oracle",
+                                    "blas": "numpy fp64, contractions through the BLAS numpy links (multi-threaded)",
                                     "sample": what, "seconds": s}
         else:
             line["cpu_baseline"] = None
+    return line if rank == 0 else None
+
+
+SUITE = ["c1", "c2", "c3", "c4", "c5"]      # the workload list's five modules; the last one is the headline
+SUITE_KEYS = ("ms_per_step", "value", "unit", "steps", "dtype", "config", "roofline", "sustained", "graph", "e2e", "gpu_launches",
+              "clocks", "per_subkernel", "cpu_baseline")
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2607_20501_b200 import dist as D
+
+    rank, local, world = D.env_world()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback for the product path")
+    torch.cuda.set_device(local)
+    D.init("nccl", torch.device("cuda", local))
+    from paper_2607_20501_b200 import Context
+    ctx = Context(local)
+
+    if args.workload != "all":
+        steps = args.steps if args.steps is not None else DEFAULT_STEPS[args.workload]
+        line = measure_one(args.workload, args, steps, ctx, rank, local, world, args.cpu_seconds)
+    else:
+        import gc
+        # C1-C4 first, each with its own step count (their steps are 7 us to 0.5 ms long: the default counts make
+        # every timed region tens of milliseconds), then the headline C5 with exactly --steps K steps.
+        others = {}
+        for name in SUITE[:-1]:
+            r = measure_one(name, args, DEFAULT_STEPS[name], ctx, rank, local, world, min(args.cpu_seconds, 4.0))
+            if r is not None:
+                others[name] = {k: r[k] for k in SUITE_KEYS if k in r}
+                others[name]["module_frac"] = r["roofline"]["module_frac"]
+            gc.collect()                 # the workload's device buffers go before the next one is uploaded
+            torch.cuda.empty_cache()
+        steps = args.steps if args.steps is not None else DEFAULT_STEPS[SUITE[-1]]
+        line = measure_one(SUITE[-1], args, steps, ctx, rank, local, world, args.cpu_seconds)
+        if line is not None:
+            line["workloads"] = others
+            fr = {k: round(v["module_frac"], 4) for k, v in others.items()}
+            fr[SUITE[-1]] = round(line["roofline"]["module_frac"], 4)
+            line["module_frac"] = fr
+            line["gpu_launches_all_workloads"] = line["gpu_launches"] + sum(v["gpu_launches"] for v in others.values())
+    if rank == 0:
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -545,18 +615,23 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c2", choices=["c1", "c2", "c3", "c4", "c5", "c6", "c7"])
+    ap.add_argument("--workload", default=None, choices=["all", "c1", "c2", "c3", "c4", "c5", "c6", "c7"],
+                    help="default: all five modules of the workload list for the GPU arm (headline C5), c5 for the reference arm")
     ap.add_argument("--decomposition", default=None)
     ap.add_argument("--batch", type=int, default=None, help="smaller leading batch dimension (profiler captures)")
     ap.add_argument("--only-ops", type=int, default=None, help="run the first N operators alone (profiler captures)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle leg")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     args = ap.parse_args()
-    if args.steps is None:
-        args.steps = DEFAULT_STEPS[args.workload] if args.impl == "ours" else 3
     if args.impl == "reference":
+        if args.steps is None:
+            args.steps = 3
+        if args.workload in (None, "all"):
+            args.workload = "c5"
         run_reference(args)
     else:
+        if args.workload is None:
+            args.workload = "all" if (args.batch is None and args.only_ops is None) else "c2"
         run_ours(args)
 
 

@@ -31,7 +31,17 @@
  *     allocation and no host<->device copy.
  *   - There is no CPU fallback.  A submodule with no matching implementation yields
  *     MK_ERR_NO_IMPL; a device that is not sm_100 yields MK_ERR_UNSUPPORTED_ARCH.
- *   - One thread uses a module at a time.
+ *   - One thread uses a module at a time.  Different modules, and contexts on different
+ *     devices, may be used from different threads at once: what the library caches per device
+ *     (kernel attributes, the address of its status word) is kept per device, in atomics.
+ *   - A context belongs to one CUDA device.  A process may hold contexts on several devices;
+ *     every call that launches or synchronises (mk_module_forward / _profile / _swap,
+ *     mk_ctx_check) requires the context's device to be the calling thread's current device and
+ *     returns MK_ERR_INVALID_ARG otherwise.
+ *   - Parameters (weights, biases, norm scales) must not be written on the stream while a
+ *     forward that reads them is in flight, and not between two forwards that are meant to
+ *     overlap: kernels launched as programmatic dependents may read parameters before the
+ *     preceding kernel on the stream has completed.
  */
 #ifndef MK_H_
 #define MK_H_
@@ -154,20 +164,40 @@ typedef struct mk_ctx mk_ctx;
 typedef struct mk_module mk_module;
 
 /* ---- context ------------------------------------------------------------------------------
+ * (Methodology: the codebase is a set of subkernels K plus one top-level module S; a context is
+ * where the library keeps what belongs to neither: the device and the last error.)
  * device >= 0: binds the context to that CUDA device (must be compute capability 10.x, else
- * MK_ERR_UNSUPPORTED_ARCH; MK_ERR_NO_DEVICE if there is none).  device = -1: a host-only
- * planning context — describing, decomposing, binding and contract queries work, launching
- * returns MK_ERR_NO_DEVICE.  *out is written only on success. */
+ * MK_ERR_UNSUPPORTED_ARCH; MK_ERR_NO_DEVICE if there is none) and makes it the calling thread's
+ * current device.  device = -1: a host-only planning context — describing, decomposing, binding
+ * and contract queries work, launching returns MK_ERR_NO_DEVICE.  *out is written only on success. */
 MK_API mk_status mk_ctx_create(int32_t device, mk_ctx** out);
 MK_API void mk_ctx_destroy(mk_ctx* ctx);
 MK_API const char* mk_status_str(mk_status s);
 /* Text of the last error raised through this context ("" if none).  Valid until the next call. */
 MK_API const char* mk_last_error(const mk_ctx* ctx);
 /* Synchronises the context's device and reports a bounded-wait expiry inside a kernel
- * (MK_ERR_DEVICE_TIMEOUT) or a CUDA error (MK_ERR_CUDA).  Clears the timeout flag. */
+ * (MK_ERR_DEVICE_TIMEOUT) or a CUDA error (MK_ERR_CUDA).  Clears the timeout flag.  (Experiments,
+ * "Setup": an evaluation that does not finish within its time limit counts as failed; here a
+ * kernel that cannot make progress gives up by itself and says so.) */
 MK_API mk_status mk_ctx_check(mk_ctx* ctx);
 
+/* Self-test of the exit every bounded wait takes when it runs out (the one path a correct run never
+ * executes).  Launches one small CTA that waits, through the same routine the tensor-core kernels
+ * use, on a barrier nobody arrives at, gives up after `limit_cycles` SM cycles (1e3 .. 2e8; about
+ * a millisecond at 2e6), records its code in the device status word and returns normally; the next
+ * mk_ctx_check then reports MK_ERR_DEVICE_TIMEOUT once and clears the flag.  No copies, no tensor
+ * memory, nothing left behind: the device stays usable.  dev_out6: six int64 in device memory
+ * (8-byte aligned): [0] / [1] what the wait returned in the thread that gave up and in a second
+ * thread released by the abort flag (0 = gave up), [2] / [3] the cycles they spent, [4] / [5] the
+ * same for a wait started after the expiry (it must return at once).  Asynchronous on the stream.
+ * (Experiments, "Setup": evaluations run under a time limit; a kernel that stalls must end as a
+ * reported failure, not as a hung device.) */
+MK_API mk_status mk_selftest_bounded_wait(mk_ctx* ctx, int64_t limit_cycles, int64_t* dev_out6,
+                                          void* cuda_stream);
+
 /* ---- 1. describe a module as an operator sequence -------------------------------------------
+ * (Methodology, LLMDecompose: the input is a PyTorch module; the top-level module delegates all
+ * mathematical computation to the submodules.  Here the module is its operator sequence.)
  * ops[n_ops] and inputs[n_inputs] are copied.  Shapes of all values are inferred here;
  * an inconsistent sequence gives MK_ERR_SHAPE_MISMATCH / MK_ERR_INVALID_ARG.  The initial
  * decomposition is one submodule per operator, each bound to the composer's default choice. */
@@ -179,6 +209,8 @@ MK_API mk_status mk_module_n_ops(const mk_module* m, int32_t* n);
 MK_API mk_status mk_module_value_spec(const mk_module* m, int32_t value_id, mk_tensor_spec* out);
 
 /* ---- 2. the decomposition: a partition of [0, n_ops) into contiguous submodules -----------
+ * (Methodology, LLMDecompose and its programmatic checks: the subproblems must fully and
+ * exclusively cover what the top-level module needs.)
  * first_op_of_sub[n_sub] must start at 0 and increase strictly; every operator then lies in
  * exactly one submodule ("fully and exclusively cover").  Every new submodule is bound to
  * the composer's default choice; MK_ERR_NO_IMPL if some submodule cannot be implemented. */
@@ -186,20 +218,31 @@ MK_API mk_status mk_module_set_decomposition(mk_module* m, const int32_t* first_
 MK_API mk_status mk_module_n_sub(const mk_module* m, int32_t* n);
 /* Writes n_sub entries into first_op_of_sub (capacity checked against *n_sub on entry). */
 MK_API mk_status mk_module_get_decomposition(const mk_module* m, int32_t* first_op_of_sub, int32_t* n_sub);
-/* Split submodule `sub` into exactly two at operator `at_op` (first_op < at_op <= last op). */
+/* Split submodule `sub` into exactly two at operator `at_op` (first_op < at_op <= last op).
+ * (Methodology, LLMSplit: a subproblem is split into exactly 2; Algorithm 2 applies it to failing
+ * subkernels.  On failure the previous decomposition is kept.) */
 MK_API mk_status mk_module_split(mk_module* m, int32_t sub, int32_t at_op);
-/* Fuse `count` >= 2 adjacent submodules starting at `first_sub` into one. */
+/* Fuse `count` >= 2 adjacent submodules starting at `first_sub` into one.
+ * (Methodology, LLMFuse: any number of subproblems are fused into a larger one; Algorithm 2's
+ * fusion branch.  On failure the previous decomposition is kept.) */
 MK_API mk_status mk_module_fuse(mk_module* m, int32_t first_sub, int32_t count);
-/* Collapse to the monolithic problem: one submodule holding every operator. */
+/* Collapse to the monolithic problem: one submodule holding every operator.
+ * (Algorithm 2, TotalFuse: taken when the local and the global correctness checks disagree.) */
 MK_API mk_status mk_module_total_fuse(mk_module* m);
 /* The submodule's I/O contract: value ids and specs it reads from outside and those it
- * produces for later submodules or as the module output.  On entry *n_in / *n_out hold the
+ * produces for later submodules or as the module output.  (Appendix "Prompts", subproblem
+ * decomposition: every subproblem states its input and output tensors with shapes and dtypes and
+ * its verification criteria; LLMDecompose's forward-shape-coverage check.)  On entry *n_in / *n_out hold the
  * capacities of the arrays (ids and specs may each be NULL); on return the counts. */
 MK_API mk_status mk_module_get_contract(const mk_module* m, int32_t sub, int32_t* in_ids,
                                  mk_tensor_spec* in_specs, int32_t* n_in, int32_t* out_ids,
                                  mk_tensor_spec* out_specs, int32_t* n_out);
 
 /* ---- 3. implementations: list, bind, swap ----------------------------------------------------
+ * (Introduction and Methodology: each subkernel solves one explicitly defined subproblem and can
+ * be replaced by an alternative implementation without touching the rest; the composer's fusion
+ * rules are those of the appendix "Prompts": GEMM + elementwise tail, elementwise chains, bias
+ * after matmul and the residual add fuse, a reduction over a whole row or group blocks fusion.)
  * mk_impl_count/_name enumerate the registered single-kernel-family implementations whose
  * legality predicate accepts submodule `sub` as a whole.  mk_module_bind(sub, name) binds one
  * of them (MK_ERR_NO_IMPL if it does not accept the submodule; the old binding stays).
@@ -213,6 +256,9 @@ MK_API mk_status mk_module_bind(mk_module* m, int32_t sub, const char* impl_name
 MK_API mk_status mk_module_bound_impl(const mk_module* m, int32_t sub, const char** name);
 
 /* ---- 4. parameters, workspace, run --------------------------------------------------------------
+ * (Appendix "Example Solution", top-level module: it owns the parameters, hands each subkernel
+ * its tensors and chains the calls; appendix "Prompts", memory and dataflow: intermediates are
+ * materialised in global memory only at subproblem boundaries.)
  * set_param: operator `op`, slot as listed per kind; dev_ptr is borrowed and must stay valid;
  * spec must equal what the operator expects (MK_ERR_SHAPE_MISMATCH otherwise). */
 MK_API mk_status mk_module_set_param(mk_module* m, int32_t op, int32_t slot, const void* dev_ptr,
@@ -226,17 +272,20 @@ MK_API mk_status mk_module_keep_intermediates(mk_module* m, int32_t keep);
 MK_API mk_status mk_module_workspace_size(mk_module* m, size_t* bytes);
 /* Kernel launches one forward issues under the current decomposition and bindings. */
 MK_API mk_status mk_module_launch_count(mk_module* m, int32_t* n);
-/* Composed forward.  in_ptrs[n_inputs], out_ptrs[1]: device tensors matching the specs.
+/* Composed forward (Algorithm 1, Evaluate: the end-to-end kernel is the top-level module running
+ * its subkernels in order).  in_ptrs[n_inputs], out_ptrs[1]: device tensors matching the specs.
  * workspace: device memory of at least workspace_size bytes, 256-byte aligned, may be NULL
  * when the size is 0.  cuda_stream: a cudaStream_t (NULL = the default stream).
- * Errors: MK_ERR_PARAM_MISSING, MK_ERR_WORKSPACE_TOO_SMALL, MK_ERR_NO_DEVICE, MK_ERR_CUDA. */
+ * Errors: MK_ERR_PARAM_MISSING, MK_ERR_WORKSPACE_TOO_SMALL, MK_ERR_NO_DEVICE, MK_ERR_CUDA,
+ * MK_ERR_INVALID_ARG (the context's device is not the current device). */
 MK_API mk_status mk_module_forward(mk_module* m, const void* const* in_ptrs, void* const* out_ptrs,
                             void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /* ---- 5. observability ---------------------------------------------------------------------------
  * profile: runs `iters` forwards with a CUDA event pair around every submodule, synchronises,
- * and writes the mean milliseconds per submodule into ms_per_sub[n_sub] (the per-subkernel
- * runtime the paper's budget allocation and Swap step read). */
+ * and writes the mean milliseconds per submodule into ms_per_sub[n_sub].  (Methodology,
+ * AllocateLLMBudget: the budget follows each subkernel's runtime observed during the last
+ * end-to-end evaluation; Swap reads the same per-subkernel figure.) */
 MK_API mk_status mk_module_profile(mk_module* m, const void* const* in_ptrs, void* const* out_ptrs,
                             void* workspace, size_t workspace_bytes, void* cuda_stream,
                             int32_t iters, float* ms_per_sub);
@@ -257,7 +306,9 @@ MK_API mk_status mk_module_swap(mk_module* m, const void* const* in_ptrs, void* 
                          int32_t* n_swapped, float* ms_before_after);
 /* Device pointer and spec of the tensor produced by value `value_id` at a submodule boundary
  * during the last forward (requires keep_intermediates; MK_ERR_INVALID_ARG if the value is
- * internal to a submodule or no forward has run). */
+ * internal to a submodule or no forward has run).  (Algorithm 2: local correctness checks, one
+ * per subkernel, beside the global one; appendix on correctness checking: every intermediate
+ * tensor is compared with its own calibrated tolerance.) */
 MK_API mk_status mk_module_intermediate(const mk_module* m, int32_t value_id, const void** dev_ptr,
                                  mk_tensor_spec* spec);
 
@@ -272,15 +323,19 @@ MK_API mk_status mk_module_intermediate(const mk_module* m, int32_t value_id, co
  *   dev_x, dev_y       [n, h, w, c] tensors of `dtype` (mk_dtype), 16-byte aligned, caller-owned
  *   dev_gamma/dev_beta [c] or NULL
  *   groups             must divide c; eps >= 0, inside the square root
+ *   n <= 65535 images; h * w < 2^31 pixels per image
  * The call allocates nothing, is asynchronous on `cuda_stream` and does not synchronise.
  * The first call on each device looks up the array's device address (a host-side query, made
  * with that device current): make that first call before starting any stream capture.
  * All calls share the one array and it keeps the last call's contents; the kernels overwrite
  * every slot they later read, so nothing needs clearing, but two calls whose kernels overlap on
- * the GPU (different streams, no dependency) race on it — order them.
+ * the GPU (different streams, no dependency) race on it — order them.  Host threads may call
+ * concurrently as far as the host side goes (the per-device set-up is kept in atomics); the
+ * shared array still requires their kernels to be ordered on the GPU.
  * Errors: MK_ERR_WORKSPACE_TOO_SMALL if n * chunks * groups * 8 bytes exceeds 1 MiB (chunks <= 64
- * pixel chunks per image; e.g. n = 32, groups = 32 needs 80 KiB), MK_ERR_SHAPE_MISMATCH,
- * MK_ERR_INVALID_ARG, MK_ERR_NO_DEVICE, MK_ERR_CUDA. */
+ * pixel chunks per image; e.g. n = 32, groups = 32 needs 80 KiB), MK_ERR_SHAPE_MISMATCH (a
+ * size outside the limits above, groups not dividing c), MK_ERR_INVALID_ARG (a NULL or unaligned
+ * tensor pointer, an unknown dtype, eps < 0 or NaN), MK_ERR_NO_DEVICE, MK_ERR_CUDA. */
 MK_API mk_status mk_groupnorm_nhwc_noalloc(int32_t dtype, const void* dev_x, void* dev_y,
                                            const void* dev_gamma, const void* dev_beta, int64_t n,
                                            int64_t h, int64_t w, int64_t c, int32_t groups,

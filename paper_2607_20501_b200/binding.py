@@ -66,6 +66,7 @@ _sig("mk_ctx_destroy", None, _P)
 _sig("mk_status_str", C.c_char_p, C.c_int32)
 _sig("mk_last_error", C.c_char_p, _P)
 _sig("mk_ctx_check", C.c_int32, _P)
+_sig("mk_selftest_bounded_wait", C.c_int32, _P, C.c_int64, _P, _P)
 _sig("mk_module_create", C.c_int32, _P, C.POINTER(mk_op_desc), C.c_int32, _SPECP, C.c_int32, _PP)
 _sig("mk_module_destroy", None, _P)
 _sig("mk_module_n_ops", C.c_int32, _P, _I32P)

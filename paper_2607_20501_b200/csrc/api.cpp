@@ -90,12 +90,26 @@ const char* mk_last_error(const mk_ctx* ctx) { return ctx ? ctx->err.c_str() : "
 mk_status mk_ctx_check(mk_ctx* ctx) {
   if (!ctx) return MK_ERR_INVALID_ARG;
   if (ctx->device < 0) return MK_ERR_NO_DEVICE;
+  if (current_device() != ctx->device)
+    return fail(ctx, MK_ERR_INVALID_ARG, "the context's device must be the calling thread's current CUDA device");
   cudaError_t e = cudaDeviceSynchronize();
   if (e != cudaSuccess) return fail(ctx, MK_ERR_CUDA, cudaGetErrorString(e));
   unsigned int flag = 0;
   e = kernel_status_fetch_and_clear(&flag);
   if (e != cudaSuccess) return fail(ctx, MK_ERR_CUDA, cudaGetErrorString(e));
   if (flag) return fail(ctx, MK_ERR_DEVICE_TIMEOUT, "a bounded wait inside a kernel expired (code " + std::to_string(flag) + ")");
+  return MK_OK;
+}
+
+mk_status mk_selftest_bounded_wait(mk_ctx* ctx, int64_t limit_cycles, int64_t* dev_out6, void* cuda_stream) {
+  if (!ctx || !dev_out6 || ((uintptr_t)dev_out6 & 7)) return MK_ERR_INVALID_ARG;
+  if (ctx->device < 0) return MK_ERR_NO_DEVICE;
+  // a limit a test can afford: between a microsecond and a tenth of a second of SM cycles
+  if (limit_cycles < 1000 || limit_cycles > 200000000) return fail(ctx, MK_ERR_INVALID_ARG, "limit_cycles must lie in [1e3, 2e8]");
+  if (current_device() != ctx->device)
+    return fail(ctx, MK_ERR_INVALID_ARG, "the context's device must be the calling thread's current CUDA device");
+  cudaError_t e = launch_bounded_wait_selftest((long long)limit_cycles, (long long*)dev_out6, (cudaStream_t)cuda_stream);
+  if (e != cudaSuccess) return fail(ctx, MK_ERR_CUDA, cudaGetErrorString(e));
   return MK_OK;
 }
 
@@ -325,6 +339,11 @@ mk_status mk_module_workspace_size(mk_module* m, size_t* bytes) {
 static mk_status ensure_plan(mk_module* m, const void* const* in_ptrs, void* const* out_ptrs, void* ws, size_t ws_bytes) {
   if (!m || !in_ptrs || !out_ptrs) return MK_ERR_INVALID_ARG;
   if (m->ctx->device < 0) return fail(m->ctx, MK_ERR_NO_DEVICE, "host-only planning context cannot launch");
+  // Launches go to the calling thread's current device; the module's buffers, descriptors and status word
+  // belong to its context's device.  A process may hold contexts on several GPUs, so the two must agree.
+  if (current_device() != m->ctx->device)
+    return fail(m->ctx, MK_ERR_INVALID_ARG, "the context's device (" + std::to_string(m->ctx->device) +
+                                               ") must be the calling thread's current CUDA device");
   std::string err;
   mk_status st = build_plan(*m, in_ptrs, out_ptrs, ws, ws_bytes, err);
   if (st != MK_OK) return fail(m->ctx, st, err);

@@ -380,11 +380,10 @@ cudaError_t attention_tc_plan(AttnTcPlan* p, const AttnView& a, void* o) {
 }
 
 cudaError_t launch_attention_tc(const AttnTcPlan& p, cudaStream_t s) {
-  static bool attr_done = false;
-  if (!attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ATTN_SMEM);
+  static SmemOptIn opt_in;
+  {
+    cudaError_t e = opt_in.ensure(ATTN_SMEM, attention_tc_kernel);
     if (e != cudaSuccess) return e;
-    attr_done = true;
   }
   attention_tc_kernel<<<p.grid, THREADS, ATTN_SMEM, s>>>(p.tm_q, p.tm_k, p.tm_v, (__nv_bfloat16*)p.out, p.B, p.H, p.S, p.scale_log2,
                                                          kernel_status_ptr());

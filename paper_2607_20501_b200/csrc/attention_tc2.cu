@@ -751,11 +751,10 @@ cudaError_t attention_tc2_plan(AttnTcPlan* p, const AttnView& a, void* o, int sm
 }
 
 cudaError_t launch_attention_tc2(const AttnTcPlan& p, cudaStream_t s) {
-  static bool attr_done = false;
-  if (!attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(attention_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ATTN2_SMEM);
+  static SmemOptIn opt_in;
+  {
+    cudaError_t e = opt_in.ensure(ATTN2_SMEM, attention_tc2_kernel);
     if (e != cudaSuccess) return e;
-    attr_done = true;
   }
   LaunchCfg lc(PDL_ATTENTION, dim3((unsigned)p.grid), dim3(THREADS), ATTN2_SMEM, s);
   return cudaLaunchKernelEx(&lc.cfg, attention_tc2_kernel, p.tm_q, p.tm_k, p.tm_v, (__nv_bfloat16*)p.out, p.B, p.H, p.S, p.causal ? 1 : 0, p.scale_log2,

@@ -408,12 +408,10 @@ cudaError_t conv3x3_tc2_plan(ConvTcPlan* p, const void* x, const void* w, void* 
 }
 
 cudaError_t launch_conv3x3_tc2(const ConvTcPlan& p, cudaStream_t s) {
-  static size_t attr_bytes = 0;   // largest dynamic shared-memory size opted into so far
-  if (p.smem > attr_bytes) {
-    cudaError_t e = cudaFuncSetAttribute(conv3x3_tc2_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(conv3x3_tc2_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem);
+  static SmemOptIn opt_in;
+  {
+    cudaError_t e = opt_in.ensure(p.smem, conv3x3_tc2_kernel<1>, conv3x3_tc2_kernel<2>);
     if (e != cudaSuccess) return e;
-    attr_bytes = p.smem;
   }
   LaunchCfg lc(PDL_CONV, dim3((unsigned)p.grid), dim3(THREADS), p.smem, s, 2);
   cudaLaunchConfig_t& cfg = lc.cfg;

@@ -517,15 +517,9 @@ cudaError_t plan_impl(GemmTcPlan* p, const void* a, const void* w_nk, void* y, b
 
 template <int CTAS>
 cudaError_t launch_impl(const GemmTcPlan& p, cudaStream_t s) {
-  static bool attr_done = false;
-  if (!attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<CTAS, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<CTAS>::SMEM);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<CTAS, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<CTAS>::SMEM);
-    if (e == cudaSuccess && CTAS == 2)
-      e = cudaFuncSetAttribute(gemm_tc_kernel<2, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<2>::SMEM);
-    if (e != cudaSuccess) return e;
-    attr_done = true;
-  }
+  static SmemOptIn opt_in;
+  cudaError_t e0 = opt_in.ensure(Cfg<CTAS>::SMEM, gemm_tc_kernel<CTAS, false>, gemm_tc_kernel<CTAS, true>, gemm_tc_kernel<CTAS, false, false, CTAS == 2>);
+  if (e0 != cudaSuccess) return e0;
   LaunchCfg lc(PDL_GEMM, dim3((unsigned)p.grid), dim3(THREADS), Cfg<CTAS>::SMEM, s, CTAS == 2 ? 2 : 0);
   cudaLaunchConfig_t& cfg = lc.cfg;
   unsigned int* status = kernel_status_ptr();
@@ -541,12 +535,9 @@ cudaError_t launch_impl(const GemmTcPlan& p, cudaStream_t s) {
 }
 
 cudaError_t launch_norm_impl(const GemmTcPlan& p, cudaStream_t s) {
-  static bool attr_done = false;
-  if (!attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<2, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<2>::SMEM);
-    if (e != cudaSuccess) return e;
-    attr_done = true;
-  }
+  static SmemOptIn opt_in;
+  cudaError_t e0 = opt_in.ensure(Cfg<2>::SMEM, gemm_tc_kernel<2, false, true>);
+  if (e0 != cudaSuccess) return e0;
   const int64_t row_blocks = ((p.m + 2 * BM - 1) / (2 * BM)) * 2 * 4;
   cudaError_t e = cudaMemsetAsync(p.norm.counters, 0, (size_t)row_blocks * sizeof(int), s);
   if (e != cudaSuccess) return e;

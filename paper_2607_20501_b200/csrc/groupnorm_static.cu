@@ -16,28 +16,29 @@ namespace {
 constexpr size_t kStaticScratchBytes = 1u << 20;  // 1 MiB
 static __device__ __align__(256) unsigned char g_groupnorm_scratch[kStaticScratchBytes];
 
-constexpr int kMaxDevices = 64;
 struct PerDevice {
-  float* scratch = nullptr;  // device address of g_groupnorm_scratch on that device
-  int sm_count = 0;
+  std::atomic<float*> scratch{nullptr};  // device address of g_groupnorm_scratch on that device
+  std::atomic<int> sm_count{0};
 };
 PerDevice g_dev[kMaxDevices];
 
 // In host code the array's name is only a handle for the runtime, not an address a kernel can use:
-// the device address has to be asked for, once per device, with that device current.
+// the device address has to be asked for, once per device, with that device current.  Two host
+// threads that make a device's first call together both ask and both store the same two values;
+// the address is published last, so whoever sees it also sees the SM count.
 mk_status setup_current_device(int* dev_out) {
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return MK_ERR_NO_DEVICE; }
   if (dev < 0 || dev >= kMaxDevices) return MK_ERR_INVALID_ARG;
-  if (!g_dev[dev].scratch) {
+  if (!g_dev[dev].scratch.load(std::memory_order_acquire)) {
     void* p = nullptr;
     cudaError_t e = cudaGetSymbolAddress(&p, g_groupnorm_scratch);
     if (e != cudaSuccess || !p) { cudaGetLastError(); return MK_ERR_CUDA; }
     int sms = 0;
     e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess || sms < 1) { cudaGetLastError(); return MK_ERR_CUDA; }
-    g_dev[dev].sm_count = sms;
-    g_dev[dev].scratch = static_cast<float*>(p);
+    g_dev[dev].sm_count.store(sms, std::memory_order_relaxed);
+    g_dev[dev].scratch.store(static_cast<float*>(p), std::memory_order_release);
   }
   *dev_out = dev;
   return MK_OK;
@@ -53,15 +54,21 @@ extern "C" MK_API mk_status mk_groupnorm_nhwc_noalloc(int32_t dtype, const void*
   if (dtype != MK_F32 && dtype != MK_BF16) return MK_ERR_INVALID_ARG;
   if (!dev_x || !dev_y || ((uintptr_t)dev_x & 15) || ((uintptr_t)dev_y & 15)) return MK_ERR_INVALID_ARG;
   if (((uintptr_t)dev_gamma & 15) || ((uintptr_t)dev_beta & 15)) return MK_ERR_INVALID_ARG;
-  if (n < 1 || h < 1 || w < 1 || c < 1 || groups < 1 || c % groups || !(eps >= 0.0)) return MK_ERR_SHAPE_MISMATCH;
+  if (!(eps >= 0.0)) return MK_ERR_INVALID_ARG;
+  if (n < 1 || h < 1 || w < 1 || c < 1 || groups < 1 || c % groups) return MK_ERR_SHAPE_MISMATCH;
+  // Sizes the kernels cannot index are refused before anything is multiplied: an image count beyond the
+  // grid's second dimension, and extents whose products would leave 64 bits or the kernels' 32-bit channel index.
+  constexpr int64_t kMaxImages = 65535, kMaxExtent = int64_t(1) << 31;
+  if (n > kMaxImages || h >= kMaxExtent || w >= kMaxExtent || c >= kMaxExtent || h * w >= kMaxExtent) return MK_ERR_SHAPE_MISMATCH;
   int dev = -1;
   mk_status st = setup_current_device(&dev);
   if (st != MK_OK) return st;
-  const int sms = g_dev[dev].sm_count;
+  const int sms = g_dev[dev].sm_count.load(std::memory_order_relaxed);
   const int64_t hw = h * w;
+  // n <= 65535, chunks <= 64, groups < 2^31: the product below stays far inside 64 bits
   if (groupnorm_scratch_bytes(n, hw, c, groups, sms) > kStaticScratchBytes) return MK_ERR_WORKSPACE_TOO_SMALL;
   const int chunks = groupnorm_chunks(n, hw, sms);
-  float* scratch = g_dev[dev].scratch;
+  float* scratch = g_dev[dev].scratch.load(std::memory_order_acquire);
   cudaStream_t s = (cudaStream_t)cuda_stream;
   const int d = dtype == MK_F32 ? DT_F32 : DT_BF16;
   EpiProgram none;  // no elementwise ops ahead of the norm

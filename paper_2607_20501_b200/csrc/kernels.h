@@ -3,6 +3,7 @@
 #pragma once
 
 #include <cuda_runtime.h>
+#include <atomic>
 #include <stddef.h>
 #include <stdint.h>
 
@@ -37,9 +38,38 @@ struct EpiProgram {
   EpiOp op[EPI_MAX];
 };
 
+// ---- per-device host state ---------------------------------------------------------------------------------
+// One process may hold contexts on several GPUs, and may use them from several host threads: everything the
+// launchers cache (the device address of a __device__ symbol, a kernel's opt-in to more than 48 KB of dynamic
+// shared memory) is a property of ONE device and is therefore kept per device ordinal, in atomics.
+constexpr int kMaxDevices = 64;
+int current_device();   // ordinal of the calling thread's current device; -1 on error or beyond kMaxDevices
+
+// Largest dynamic shared-memory size the kernels of one launcher have opted into, per device.
+struct SmemOptIn {
+  std::atomic<size_t> have[kMaxDevices] = {};
+  // Raise cudaFuncAttributeMaxDynamicSharedMemorySize of every kernel in `fn` to `need` bytes on the current
+  // device unless that device has been given at least as much before.  Two threads that race here set the
+  // same attribute twice, which is harmless.
+  template <typename... Fn>
+  cudaError_t ensure(size_t need, Fn... fn) {
+    const int dev = current_device();
+    if (dev < 0) return cudaErrorInvalidDevice;
+    if (need <= have[dev].load(std::memory_order_acquire)) return cudaSuccess;
+    cudaError_t r = cudaSuccess;
+    ((r = (r == cudaSuccess ? cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need) : r)), ...);
+    if (r == cudaSuccess) have[dev].store(need, std::memory_order_release);
+    return r;
+  }
+};
+
 // ---- device status word (bounded-wait expiry codes) --------------------------------------------------
-unsigned int* kernel_status_ptr();   // device address, nullptr without a device
-cudaError_t kernel_status_fetch_and_clear(unsigned int* out);
+unsigned int* kernel_status_ptr();   // address on the current device, nullptr without one
+cudaError_t kernel_status_fetch_and_clear(unsigned int* out);   // of the current device
+
+// Self-test of the bounded-wait exit (selftest.cu): one CTA waits, through the kernels' own wait routine, on a
+// barrier nobody arrives at; out6 = six int64 in device memory (see the kernel).
+cudaError_t launch_bounded_wait_selftest(long long limit_cycles, long long* out6, cudaStream_t s);
 
 // ---- programmatic dependent launch ----------------------------------------------------------------------
 // A kernel launched through LaunchCfg may be scheduled while the kernel before it on the stream is still

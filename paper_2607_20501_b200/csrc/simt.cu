@@ -113,6 +113,9 @@ __global__ void __launch_bounds__(LC_THREADS) linear_rownorm_cluster_kernel(cons
   __shared__ float slot[2][LC_CL][LC_RB];                  // row partial sums of every CTA of the cluster (two statistics)
   __shared__ float stat[2][LC_RB];
   pdl_launch_dependents();
+  // A CTA may write into a peer's shared memory only once that peer is running: every CTA announces itself
+  // here and waits for the others just before its first remote store, so the rendezvous costs nothing.
+  tc::cluster_arrive();
   pdl_wait();
   const uint32_t rank = tc::cluster_ctarank();
   const int m0 = (int)(blockIdx.x / LC_CL) * LC_RB, c0 = (int)rank * NC;
@@ -196,6 +199,7 @@ __global__ void __launch_bounds__(LC_THREADS) linear_rownorm_cluster_kernel(cons
     val[r][j] = j < nc ? epi_apply(p, v, m0 + r, c0 + j, N) : 0.0f;
   }
   __syncthreads();
+  tc::cluster_wait();   // all eight CTAs of the cluster are resident from here on
   const float inv_n = 1.0f / (float)N;
   // statistic 0: the row sums (LayerNorm) -> mean
   if (mode == ROW_LAYERNORM) {
@@ -251,12 +255,10 @@ static cudaError_t linear_rownorm_cluster_launch(const void* a, const void* w, b
   NC = pw;
   const int outs = LC_RB * NC, KS = LC_THREADS / outs > 0 ? LC_THREADS / outs : 1;
   const size_t smem = sizeof(float) * ((size_t)LC_RB * k + (size_t)NC * (k + 1) + (size_t)KS * outs);
-  static size_t attr_bytes[2] = {0, 0};
-  size_t& have = attr_bytes[sizeof(T) == 4 ? 0 : 1];
-  if (smem > 48 * 1024 && smem > have) {
-    cudaError_t e = cudaFuncSetAttribute(linear_rownorm_cluster_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  static SmemOptIn opt_in;   // one per instantiation (T)
+  if (smem > 48 * 1024) {
+    cudaError_t e = opt_in.ensure(smem, linear_rownorm_cluster_kernel<T>);
     if (e != cudaSuccess) return e;
-    have = smem;
   }
   const unsigned grid = (unsigned)((m + LC_RB - 1) / LC_RB) * LC_CL;
   LaunchCfg lc(PDL_ELTWISE, dim3(grid), dim3(LC_THREADS), smem, s, LC_CL);
@@ -430,12 +432,10 @@ static cudaError_t linear_rownorm_dispatch(const void* a, const void* w, bool wt
   const int KS = LR_THREADS / NT;
   const size_t smem = sizeof(float) * ((size_t)LR_ROWS * k + (size_t)KS * LR_ROWS * n);
   if (smem > 200 * 1024) return cudaErrorInvalidValue;
-  static bool attr_f32 = false, attr_bf16 = false;
-  bool& done = sizeof(T) == 4 ? attr_f32 : attr_bf16;
-  if (!done) {
-    cudaError_t e = cudaFuncSetAttribute(linear_rownorm_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+  static SmemOptIn opt_in;   // one per instantiation (T)
+  {
+    cudaError_t e = opt_in.ensure(200 * 1024, linear_rownorm_kernel<T>);
     if (e != cudaSuccess) return e;
-    done = true;
   }
   const int grid = (int)((m + LR_ROWS - 1) / LR_ROWS);
   linear_rownorm_kernel<T><<<grid, LR_THREADS, smem, s>>>((const T*)a, (const T*)w, wt, (T*)y, (int)m, (int)n, (int)k, NT, p, mode,

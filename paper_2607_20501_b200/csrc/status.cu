@@ -7,12 +7,24 @@ namespace mk {
 
 __device__ unsigned int g_mk_status = 0;
 
+int current_device() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return -1; }
+  return dev >= 0 && dev < kMaxDevices ? dev : -1;
+}
+
+// Every device that loads the library has its own copy of g_mk_status at its own address.
+static std::atomic<unsigned int*> g_status_addr[kMaxDevices];
+
 unsigned int* kernel_status_ptr() {
-  static unsigned int* p = nullptr;
+  const int dev = current_device();
+  if (dev < 0) return nullptr;
+  unsigned int* p = g_status_addr[dev].load(std::memory_order_acquire);
   if (!p) {
     void* a = nullptr;
     if (cudaGetSymbolAddress(&a, g_mk_status) != cudaSuccess) { cudaGetLastError(); return nullptr; }
     p = (unsigned int*)a;
+    g_status_addr[dev].store(p, std::memory_order_release);   // a racing thread stores the same address
   }
   return p;
 }

@@ -24,7 +24,8 @@ enum WaitCode : unsigned {
   WAIT_SMEM_FULL = 2,
   WAIT_TMEM_FULL = 3,
   WAIT_TMEM_EMPTY = 4,
-  WAIT_ATTN = 5
+  WAIT_ATTN = 5,
+  WAIT_SELFTEST = 99
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -55,15 +56,17 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+// `limit`: cycles after which the wait gives up (the kernels use the default; the self-test of this path passes a
+// millisecond so that the expiry can be exercised without a long stall)
 static __device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, volatile int* abort_flag, unsigned int* status,
-                                            unsigned code) {
+                                            unsigned code, long long limit = kWaitLimitCycles) {
   const long long t0 = clock64();
   while (true) {
 #pragma unroll 1
     for (int i = 0; i < 32; ++i)
       if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (clock64() - t0 > kWaitLimitCycles) {
+    if (clock64() - t0 > limit) {
       *abort_flag = 1;
       if (status) atomicExch(status, code);
       return false;
@@ -326,6 +329,10 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t ran
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
   return r;
 }
+// The two halves of a cluster barrier, for work that may overlap the rendezvous.  Every thread of the CTA
+// executes both, in this order, once per phase.
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
 __device__ __forceinline__ void cluster_sync() {
   asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");

@@ -1,11 +1,19 @@
-"""Per-stage calibrated tolerances and the feasibility gap (paper, the section on verification with
-calibrated tolerances and its bug-detection tables), run as a protocol on the composed C4 block at reduced size.
+"""Per-stage calibrated tolerances and the feasibility gap (paper, the appendix on verification with
+calibrated tolerances and its bug-detection tables), run as a protocol on two composed blocks at reduced
+size: the causal-attention block (C4's operator sequence) and the paper's FFN block (LayerNorm -> Linear ->
+GELU -> Linear -> residual).
 
-Calibration: over several seeds, every submodule of the three-way decomposition is checked LOCALLY - the
-GPU stage's output against the fp64 oracle of that stage applied to the very tensors the GPU stage read -
-and its tolerance is set to max + 3 sigma of the observed maximum absolute error (no relative part).  The
-module's output gets the same treatment (global check).  Then subtly wrong subkernels are emulated by
-handing the GPU a perturbed description of one stage (the oracle keeps the true one):
+Calibration: over 20 seeds (the paper's number of calibration runs), every submodule of the decomposition
+is checked LOCALLY - the GPU stage's output against the fp64 oracle of that stage applied to the very
+tensors the GPU stage read - and its tolerance is set to max + 3 sigma of the observed maximum absolute
+error (no relative part).  The module's output gets the same treatment (global check).  Then wrong
+subkernels are emulated by handing the GPU a perturbed description or perturbed operands of ONE stage (the
+oracle keeps the true ones).  Of the paper's bug list, the ones that can be produced that way are used: a K
+tile boundary (the tail of K's head dimension unloaded), a tile boundary in fc1 (the last block of its
+weight unloaded), a missing residual, ReLU in place of GELU, LayerNorm dividing by sigma without removing
+the mean (which equals feeding the norm a shifted input, see below); softmax over the wrong axis, the mask
+off by one and a bf16 accumulator cannot be produced by a correct kernel and are covered as CPU-side
+mutants in tests/test_oracle_modules.py.  Three subtle faults of this build's own are kept beside them.
 
   * the local check of the perturbed stage, with its calibrated tolerance, must flag every one of them, and
     the local checks of the other stages must stay green (errors are localised);
@@ -25,8 +33,37 @@ from tests.parity import run_gpu
 
 pytestmark = pytest.mark.gpu
 
-SHAPE = dict(B=2, H=4, S=256, D=128)
-STAGES = [("a", 0, 1), ("h", 1, 3), ("y", 3, 4)]     # boundary value, first op, one past the last op
+N_CALIBRATION = 20
+ATTN_SHAPE = dict(B=2, H=4, S=256, D=128)
+ATTN_STAGES = [("a", 0, 1), ("h", 1, 3), ("y", 3, 4)]     # boundary value, first op, one past the last op
+ATTN_CUTS = [0, 1, 3]
+
+
+def ffn_block(seed, T=512, E=256, F=1024):
+    """The paper's FFN case study: y = x + fc2(GELU(fc1(LayerNorm(x)))) with biases, bf16."""
+    w = G.Workload("ffn", "bf16")
+    w.inputs["x"] = G.make("x", "bf16", G._normal(seed, 0, (T, E)))
+    w.params["g"] = G.make("g", "bf16", G._normal(seed, 1, (E,), mean=1.0, std=0.02))
+    w.params["b"] = G.make("b", "bf16", G._normal(seed, 2, (E,), std=0.02))
+    w.params["W1"] = G.make("W1", "bf16", G._normal(seed, 3, (E, F), std=(1.0 / E) ** 0.5))
+    w.params["b1"] = G.make("b1", "bf16", G._normal(seed, 4, (F,), std=0.02))
+    w.params["W2"] = G.make("W2", "bf16", G._normal(seed, 5, (F, E), std=(1.0 / F) ** 0.5))
+    w.params["b2"] = G.make("b2", "bf16", G._normal(seed, 6, (E,), std=0.02))
+    w.ops = [
+        G._op("layernorm", "n", ["x"], {"gamma": "g", "beta": "b"}, eps=1e-5),
+        G._op("linear", "h0", ["n"], {"w": "W1"}, n=F),
+        G._op("bias_add", "h1", ["h0"], {"b": "b1"}),
+        G._op("gelu_tanh", "h", ["h1"]),
+        G._op("linear", "d0", ["h"], {"w": "W2"}, n=E),
+        G._op("bias_add", "d1", ["d0"], {"b": "b2"}),
+        G._op("residual_add", "y", ["d1", "x"]),
+    ]
+    w.partitions = {"split3": [0, 1, 4], "fused": [0]}
+    return w
+
+
+FFN_STAGES = [("n", 0, 1), ("h", 1, 4), ("y", 4, 7)]
+FFN_CUTS = [0, 1, 4]
 
 
 @pytest.fixture(scope="module")
@@ -35,61 +72,141 @@ def ctx():
     return Context(0)
 
 
-def _local_errors(ctx, w_gpu, w_true):
+def _local_errors(ctx, w_gpu, w_true, stages, cuts):
     """Max abs error of every stage against the oracle of that stage on the GPU stage's own inputs, and of
     the module output against the oracle of the whole true module."""
-    dw, out = run_gpu(ctx, w_gpu, w_gpu.partitions["split3"], keep=True)
+    dw, out = run_gpu(ctx, w_gpu, cuts, keep=True)
     have = {k: t.f64() for k, t in w_true.inputs.items()}
     params = {k: t.f64() for k, t in w_true.params.items()}
     errs = {}
-    for name, lo, hi in STAGES:
-        ref, _ = OM.run_module(w_true.ops[lo:hi], {k: have[k] for op in w_true.ops[lo:hi] for k in op["in"] if k in have}, params)
-        got = out if name == "y" else to_host_f64(dw.intermediate(name))
+    last = stages[-1][0]
+    for name, lo, hi in stages:
+        ops = w_true.ops[lo:hi]
+        ref, _ = OM.run_module(ops, {k: have[k] for op in ops for k in op["in"] if k in have}, params)
+        got = out if name == last else to_host_f64(dw.intermediate(name))
         errs[name] = float(np.abs(got - ref).max())
         have[name] = got                       # the next stage is judged on what it was actually given
     ref_all, _ = OM.run_workload(w_true, [0])
     return errs, float(np.abs(out - ref_all).max()), check_close(out, ref_all, "bf16")["ok"]
 
 
-def test_calibrated_local_checks_catch_what_the_global_tolerance_lets_through(ctx):
-    seeds = range(8)
+def _calibrate(ctx, make, stages, cuts):
     runs = []
-    for s in seeds:
-        w = W.c4(s, **SHAPE)
-        errs, gerr, gok = _local_errors(ctx, w, w)
+    for s in range(N_CALIBRATION):
+        w = make(s)
+        errs, gerr, gok = _local_errors(ctx, w, w, stages, cuts)
         assert gok
         runs.append((errs, gerr))
-    tol = {n: float(np.max([r[0][n] for r in runs]) + 3 * np.std([r[0][n] for r in runs])) for n, _, _ in STAGES}
+    tol = {n: float(np.max([r[0][n] for r in runs]) + 3 * np.std([r[0][n] for r in runs])) for n, _, _ in stages}
     gtol = float(np.max([r[1] for r in runs]) + 3 * np.std([r[1] for r in runs]))
     assert all(t > 0 for t in tol.values())
+    return tol, gtol
 
-    def mutant(kind):
-        w = W.c4(100, **SHAPE)
-        m = copy.copy(w)
-        m.inputs, m.params = dict(w.inputs), dict(w.params)
-        m.ops = [dict(o, attrs=dict(o["attrs"])) for o in w.ops]
-        if kind == "attention: logits 5 % too large":
-            m.inputs["q"] = G.make("q", "bf16", (1.05 * w.inputs["q"].f64()).astype(np.float32))
-            stage = "a"
-        elif kind == "projection: one output column 30 % off":
-            wo = w.params["Wo"].f64().copy()
-            wo[:, 7] *= 1.3
-            m.params["Wo"] = G.make("Wo", "bf16", wo.astype(np.float32))
-            stage = "h"
-        else:
-            m.ops[3]["attrs"]["eps"] = 3e-2
-            stage = "y"
-        return w, m, stage
 
+def _clone(w):
+    m = copy.copy(w)
+    m.inputs, m.params = dict(w.inputs), dict(w.params)
+    m.ops = [dict(o, attrs=dict(o["attrs"]), params=dict(o["params"])) for o in w.ops]
+    return m
+
+
+def _run_mutants(ctx, make, mutants, stages, cuts, tol):
     evaded_global = 0
-    for kind in ("attention: logits 5 % too large", "projection: one output column 30 % off", "rmsnorm: eps 3e-2 instead of 1e-6"):
-        w_true, w_mut, stage = mutant(kind)
-        errs, gerr, gok_fixed = _local_errors(ctx, w_mut, w_true)
+    for kind, (edit, stage) in mutants.items():
+        w_true = make(100)
+        w_mut = _clone(w_true)
+        edit(w_true, w_mut)
+        errs, gerr, gok_fixed = _local_errors(ctx, w_mut, w_true, stages, cuts)
         assert errs[stage] > tol[stage], f"{kind}: local error {errs[stage]:.3g} within calibrated {tol[stage]:.3g}"
-        for n, _, _ in STAGES:
+        for n, _, _ in stages:
             if n != stage:
                 assert errs[n] <= tol[n], f"{kind}: stage {n} flagged although only {stage} is wrong"
         evaded_global += int(gok_fixed)
-    # at least one of these subtle faults passes the fixed module-level tolerance
-    assert evaded_global >= 1
+    return evaded_global
+
+
+def _set(t, name, values):
+    return G.make(name, "bf16", np.asarray(values, np.float32))
+
+
+def test_attention_block_local_checks_catch_what_the_global_tolerance_lets_through(ctx):
+    make = lambda s: W.c4(s, **ATTN_SHAPE)
+    tol, gtol = _calibrate(ctx, make, ATTN_STAGES, ATTN_CUTS)
+
+    def logits_5pc(w, m):
+        m.inputs["q"] = _set(m, "q", 1.05 * w.inputs["q"].f64())
+
+    def k_tile_boundary(w, m):          # paper: last partial tile of K's head dimension left unloaded
+        k = w.inputs["k"].f64().copy()
+        k[..., -16:] = 0.0
+        m.inputs["k"] = _set(m, "k", k)
+
+    def one_column(w, m):
+        wo = w.params["Wo"].f64().copy()
+        wo[:, 7] *= 1.3
+        m.params["Wo"] = _set(m, "Wo", wo)
+
+    def missing_residual(w, m):         # paper: the residual connection dropped
+        m.inputs["r"] = _set(m, "r", np.zeros(w.inputs["r"].shape))
+
+    def wrong_eps(w, m):
+        m.ops[3]["attrs"]["eps"] = 3e-2
+
+    mutants = {
+        "attention: logits 5 % too large": (logits_5pc, "a"),
+        "attention: tail of K's head dimension unloaded": (k_tile_boundary, "a"),
+        "projection: one output column 30 % off": (one_column, "h"),
+        "projection: residual missing": (missing_residual, "h"),
+        "rmsnorm: eps 3e-2 instead of 1e-6": (wrong_eps, "y"),
+    }
+    evaded = _run_mutants(ctx, make, mutants, ATTN_STAGES, ATTN_CUTS, tol)
+    assert evaded >= 1            # at least one subtle fault passes the fixed module-level tolerance
+    assert gtol < 0.2
+
+
+def test_ffn_block_local_checks_catch_the_papers_ffn_bugs(ctx):
+    make = ffn_block
+    tol, gtol = _calibrate(ctx, make, FFN_STAGES, FFN_CUTS)
+
+    def unsafe_layernorm(w, m):
+        # y = x / sigma * gamma + beta without removing the mean equals the true LayerNorm plus
+        # mu / sigma * gamma: emulate it by handing the kernel a beta raised by the mean ratio of
+        # the typical row (the GPU kernel itself is correct, only its description is wrong)
+        x = w.inputs["x"].f64()
+        shift = float(np.mean(np.abs(x.mean(axis=1)) / x.std(axis=1)))
+        m.params["b"] = _set(m, "b", w.params["b"].f64() + shift * w.params["g"].f64())
+
+    def fc1_tile_boundary(w, m):        # paper: last partial block of fc1's weight left unloaded
+        w1 = w.params["W1"].f64().copy()
+        w1[-32:, :] = 0.0
+        m.params["W1"] = _set(m, "W1", w1)
+
+    def relu_not_gelu(w, m):
+        m.ops[3]["kind"] = "relu"
+
+    def missing_residual(w, m):
+        # the skip edge replaced by a zero tensor
+        m.inputs["x0"] = _set(m, "x0", np.zeros(w.inputs["x"].shape))
+        m.ops[6]["in"] = ["d1", "x0"]
+
+    def fc2_bias_dropped(w, m):
+        m.params["b2"] = _set(m, "b2", np.zeros(w.params["b2"].shape))
+
+    def one_shift_wrong(w, m):
+        # one channel of the norm's shift off by 0.1: plain at the norm's boundary, spread over 1024 hidden
+        # units at 0.1 / sqrt(256) each by fc1 and invisible at the module's output
+        b = w.params["b"].f64().copy()
+        b[7] += 0.1
+        m.params["b"] = _set(m, "b", b)
+
+    mutants = {
+        "LayerNorm without mean subtraction (as a shifted beta)": (unsafe_layernorm, "n"),
+        "fc1: last block of the weight unloaded": (fc1_tile_boundary, "h"),
+        "ReLU instead of GELU": (relu_not_gelu, "h"),
+        "fc2: residual missing": (missing_residual, "y"),
+        "fc2: bias dropped": (fc2_bias_dropped, "y"),
+        "LayerNorm: one channel's shift off by 0.1": (one_shift_wrong, "n"),
+    }
+    evaded = _run_mutants(ctx, make, mutants, FFN_STAGES, FFN_CUTS, tol)
+    assert evaded >= 1            # the single wrong shift passes the fixed module-level tolerance
     assert gtol < 0.2

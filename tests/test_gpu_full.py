@@ -1,7 +1,9 @@
 """Parity at the full workload sizes, in the launch configuration bench.py times (default
 decomposition, default bindings, tensor-core kernels): every element where the fp64 oracle
-finishes in seconds (C2, C3), and on whole batch elements — which are independent through every
-operator — where it does not (C4, C5)."""
+finishes in seconds (C2, C3), and batch element by batch element — they are independent through
+every operator, so the oracle of one element is exact for its rows — for C4 and C5, where the
+oracle of the whole tensor at once would need tens of GB.  Every batch element is compared, i.e.
+every element of every output."""
 import numpy as np
 import pytest
 
@@ -42,14 +44,14 @@ def test_c3_full_every_element(ctx):
     assert np.abs(z.mean(axis=(1, 3))).max() < 2e-2 and np.abs(z.var(axis=(1, 3)) - 1).max() < 5e-2
 
 
-def test_c4_full_sampled_batch_elements(ctx):
+def test_c4_full_every_element(ctx):
     w = W.c4(0)
     B, H, S, D = w.inputs["q"].shape
     dw, out = run_gpu(ctx, w, w.partitions["fused"])
     assert dw.module.bound_impl(0) == "attention_tc2+gemm_tc2+rowop"
     assert np.isfinite(out).all()
     assert np.abs((out * out).mean(axis=1) - 1).max() < 2e-2          # RMSNorm, gamma = 1, holds at any size
-    for b in (0, B - 1):
+    for b in range(B):
         sub = W.c4(0, B=1, H=1, S=1, D=D)                              # a shell to carry the slices
         sub.ops, sub.params = w.ops, w.params
         sub.inputs = {k: Tensor(k, "bf16", w.inputs[k].store[b:b + 1]) for k in ("q", "k", "v")}
@@ -58,7 +60,7 @@ def test_c4_full_sampled_batch_elements(ctx):
         assert_parity(out[b * S:(b + 1) * S], ref, "bf16", f"c4 batch element {b}")
 
 
-def test_c5_full_sampled_batch_elements(ctx):
+def test_c5_full_every_element(ctx):
     w = W.c5(0)
     attn = [o for o in w.ops if o["kind"] == "attention_causal"][0]["attrs"]
     B, S = attn["batch"], attn["seq"]
@@ -72,7 +74,7 @@ def test_c5_full_sampled_batch_elements(ctx):
         if o["kind"] == "attention_causal":
             o["attrs"]["batch"] = 1
     params = {k: t.f64() for k, t in w.params.items()}
-    for b in (B - 1,):
+    for b in range(B):
         x = {"x": w.inputs["x"].f64()[b * S:(b + 1) * S]}
         ref, _ = OM.run_module(ops1, x, params, [0])
         assert_parity(out[b * S:(b + 1) * S], ref, "bf16", f"c5 batch element {b}")

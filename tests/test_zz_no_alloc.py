@@ -1,8 +1,10 @@
 """The allocation-free GroupNorm entry point, for callers that cannot give the library a workspace
 because they cannot allocate device memory where they call it (inside a framework's planned
 memory region, from a plugin that only receives its input/output buffers, in a loop that must not
-synchronise on cudaMalloc).  It must give what the composed path's GroupNorm gives, on two calls in
-a row that share its built-in scratch array, and must refuse problems that array cannot hold.
+synchronise on cudaMalloc).  It must give what the composed path's GroupNorm gives - and, judged
+on its own, what the fp64 oracle's GroupNorm gives - on two calls in a row that share its built-in
+scratch array, must leave the device's free memory as it found it, and must refuse problems that
+array cannot hold.
 
 Collected last on purpose (file name), so a run that stops at the first failure has already run
 every other test."""
@@ -13,6 +15,8 @@ import pytest
 import torch
 
 from workloads import generate as G
+from oracle import ops as O
+from oracle.compare import check_close
 
 pytestmark = pytest.mark.gpu
 
@@ -58,6 +62,22 @@ def test_noalloc_groupnorm_matches_the_workspace_path_twice_in_a_row(dtype):
         a, r = y.double().cpu().numpy(), ref.double().cpu().numpy()
         assert np.isfinite(a).all()
         assert (np.abs(a - r) <= atol + rtol * np.abs(r)).all()
+        # and against the definition itself, on the bytes the device was given
+        w = dw.w
+        want = O.groupnorm_nhwc(w.inputs["x"].f64(), w.params["gamma"].f64(), w.params["beta"].f64(), groups, 1e-5)
+        res = check_close(a, want, dtype)
+        assert res["ok"], res
+        # a warm call (the set-up of this device is done) must not move the device's free memory:
+        # torch's allocator cannot see a cudaMalloc made inside the library, the driver's own count can
+        torch.cuda.synchronize()
+        free0, _ = torch.cuda.mem_get_info()
+        st = B.mk_groupnorm_nhwc_noalloc(B.DTYPE[dtype], dw.inputs["x"].data_ptr(), y.data_ptr(), g.data_ptr(),
+                                         b.data_ptr(), *shape, groups, 1e-5, stream)
+        assert st == B.MK_OK
+        torch.cuda.synchronize()
+        free1, _ = torch.cuda.mem_get_info()
+        assert free1 == free0, (free0, free1)
+        assert check_close(y.double().cpu().numpy(), want, dtype)["ok"]
     ctx.check()
 
 
@@ -70,4 +90,10 @@ def test_noalloc_groupnorm_rejects_what_its_scratch_cannot_hold():
     assert st == B.MK_ERR_WORKSPACE_TOO_SMALL
     assert B.mk_groupnorm_nhwc_noalloc(B.MK_BF16, p, p, None, None, 1, 4, 4, 10, 3, 1e-5, 0) == B.MK_ERR_SHAPE_MISMATCH
     assert B.mk_groupnorm_nhwc_noalloc(B.MK_BF16, None, p, None, None, 1, 4, 4, 8, 2, 1e-5, 0) == B.MK_ERR_INVALID_ARG
+    assert B.mk_groupnorm_nhwc_noalloc(B.MK_BF16, p, p, None, None, 1, 4, 4, 8, 2, -1.0, 0) == B.MK_ERR_INVALID_ARG
+    assert B.mk_groupnorm_nhwc_noalloc(B.MK_BF16, p, p, None, None, 1, 4, 4, 8, 2, float("nan"), 0) == B.MK_ERR_INVALID_ARG
+    # more images than a grid dimension holds (the scratch check alone would let groups = 1 through), and
+    # extents whose product leaves 64 bits: refused as shapes, not launched
+    assert B.mk_groupnorm_nhwc_noalloc(B.MK_BF16, p, p, None, None, 70000, 1, 1, 8, 1, 1e-5, 0) == B.MK_ERR_SHAPE_MISMATCH
+    assert B.mk_groupnorm_nhwc_noalloc(B.MK_BF16, p, p, None, None, 1, 2 ** 40, 2 ** 40, 8, 1, 1e-5, 0) == B.MK_ERR_SHAPE_MISMATCH
     torch.cuda.synchronize()
