@@ -26,6 +26,7 @@
 // Ragged M / N / K: TMA zero-fills out-of-range rows and K columns; stores are guarded.
 // Every mbarrier wait is bounded (tc_common.cuh); a CTA pair leaves through a cluster barrier.
 #include "device_common.cuh"
+#include <stdlib.h>
 #include "tc_common.cuh"
 #include "tc_epilogue.cuh"
 #include "tc_plans.h"
@@ -39,7 +40,7 @@ constexpr int BN = 256;   // accumulator columns
 constexpr int BK = 64, UMMA_K = 16;
 constexpr int EPI_WARPS = 8;
 constexpr int THREADS = 64 + 32 * EPI_WARPS;
-constexpr int GROUP_M = 16;  // tile rows walked together for L2 reuse
+constexpr int GROUP_M_MAX = 16;  // most tile rows walked together for L2 reuse (the plan picks fewer for a long K)
 
 template <int CTAS> struct Cfg {
   static constexpr int STAGES = CTAS == 2 ? 6 : 4;
@@ -63,11 +64,11 @@ template <int STAGES> struct Shared {
   uint64_t fix_bar;   // the epilogue warps meet here once per tile (bounded wait, like every other)
 };
 
-__device__ __forceinline__ void tile_coords(int t, int num_m, int num_n, int& mi, int& ni) {
-  const int per_group = GROUP_M * num_n;
+__device__ __forceinline__ void tile_coords(int t, int num_m, int num_n, int group_m, int& mi, int& ni) {
+  const int per_group = group_m * num_n;
   const int g = t / per_group;
-  const int first_m = g * GROUP_M;
-  const int gsz = min(num_m - first_m, GROUP_M);
+  const int first_m = g * group_m;
+  const int gsz = min(num_m - first_m, group_m);
   const int r = t - g * per_group;
   mi = first_m + r % gsz;
   ni = r / gsz;
@@ -143,7 +144,7 @@ static_assert(RES_RING_BYTES <= Cfg<2>::STAGE_BYTES, "the residual ring takes th
 template <int CTAS, bool SWIGLU, bool NORM = false, bool RING = false>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmBh,
-               const __grid_constant__ CUtensorMap tmOut, int bulk_store, void* __restrict__ out, int out_f32, int M, int N, int K, int up_row_offset, int tail_first,
+               const __grid_constant__ CUtensorMap tmOut, int bulk_store, void* __restrict__ out, int out_f32, int M, int N, int K, int up_row_offset, int tail_first, int group_m,
                const __grid_constant__ EpiProgram epi_param, const __grid_constant__ RowNormArgs na, unsigned int* status) {
   using C = Cfg<CTAS>;
   static_assert(!RING || (CTAS == 2 && !SWIGLU && !NORM), "the residual ring exists in the plain two-SM form only");
@@ -209,7 +210,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         int t, nhalf;
         decode(u, t, nhalf);
         int mi, ni;
-        tile_coords(t, num_m, num_n, mi, ni);
+        tile_coords(t, num_m, num_n, group_m, mi, ni);
         const int m0 = (mi * CTAS + (int)rank) * BM;
         const int n0 = ni * OUT_N;
 #ifdef MK_TRACE
@@ -324,7 +325,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         int t, nhalf;
         decode(pf_u, t, nhalf);
         int mi, ni;
-        tile_coords(t, num_m, num_n, mi, ni);
+        tile_coords(t, num_m, num_n, group_m, mi, ni);
         const int64_t r0 = (int64_t)(mi * CTAS + (int)rank) * BM + q * 32;
         const int64_t c0 = (int64_t)ni * OUT_N + (nhalf > 0 ? BN / 2 : 0) + pf_c * 32;
         if (c0 + 32 <= N) {
@@ -368,7 +369,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       int t, nhalf;
       decode(u, t, nhalf);
       int mi, ni;
-      tile_coords(t, num_m, num_n, mi, ni);
+      tile_coords(t, num_m, num_n, group_m, mi, ni);
       const int acc = it & 1;
       const int64_t row0 = (int64_t)(mi * CTAS + (int)rank) * BM + q * 32;
       auto rowmap = [&](int r) -> int64_t { const int64_t g = row0 + r; return g < M ? g : -1; };
@@ -509,6 +510,16 @@ cudaError_t plan_impl(GemmTcPlan* p, const void* a, const void* w_nk, void* y, b
       if (epi.op[i].kind == EPI_RESIDUAL) { idx = i; ++cnt; }
     p->res_ring = cnt == 1 && epi.op[idx].ptr_dtype == DT_BF16;
   }
+  // Tile rows walked together: their A rows (group_m x CTAS x 128 rows of K) plus the W slabs in flight should stay
+  // in L2 for the walk across the columns.  With K = 8192 sixteen tile rows are 67 MB of A and the DRAM traffic
+  // doubles (measured: 541 MB for 302 MB algorithmic); the budget below keeps a group's A rows under ~36 MB.
+  {
+    int g = GROUP_M_MAX;
+    const char* ov = getenv("MK_GEMM_GROUP_M");
+    if (ov && ov[0]) g = atoi(ov);
+    else while (g > 2 && (int64_t)g * CTAS * BM * k * 2 > (int64_t)36 << 20) g /= 2;
+    p->group_m = g < 1 ? 1 : g;
+  }
   const int64_t tail = tiles % units;
   p->tail_first = (int)tiles;
   if (CTAS == 2 && !swiglu && tiles > units && tail > 0 && 2 * tail <= units) p->tail_first = (int)(tiles - tail);
@@ -525,12 +536,12 @@ cudaError_t launch_impl(const GemmTcPlan& p, cudaStream_t s) {
   unsigned int* status = kernel_status_ptr();
   const int out_f32 = p.out_f32 ? 1 : 0;
   if (p.swiglu)
-    return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<CTAS, true>, p.tm_a, p.tm_b, p.tm_b_half, p.tm_out, p.use_tm_out ? 1 : 0, p.out, out_f32, p.m, p.n, p.k, p.n, p.tail_first, p.epi,
+    return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<CTAS, true>, p.tm_a, p.tm_b, p.tm_b_half, p.tm_out, p.use_tm_out ? 1 : 0, p.out, out_f32, p.m, p.n, p.k, p.n, p.tail_first, p.group_m, p.epi,
                               p.norm, status);
   if (CTAS == 2 && p.res_ring)
     return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<2, false, false, true>, p.tm_a, p.tm_b, p.tm_b_half, p.tm_out, p.use_tm_out ? 1 : 0, p.out, out_f32, p.m, p.n, p.k, 0,
-                              p.tail_first, p.epi, p.norm, status);
-  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<CTAS, false>, p.tm_a, p.tm_b, p.tm_b_half, p.tm_out, p.use_tm_out ? 1 : 0, p.out, out_f32, p.m, p.n, p.k, 0, p.tail_first, p.epi,
+                              p.tail_first, p.group_m, p.epi, p.norm, status);
+  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<CTAS, false>, p.tm_a, p.tm_b, p.tm_b_half, p.tm_out, p.use_tm_out ? 1 : 0, p.out, out_f32, p.m, p.n, p.k, 0, p.tail_first, p.group_m, p.epi,
                             p.norm, status);
 }
 
@@ -553,7 +564,7 @@ cudaError_t launch_norm_impl(const GemmTcPlan& p, cudaStream_t s) {
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<2, false, true>, p.tm_a, p.tm_b, p.tm_b_half, p.tm_out, 0, p.out, 0, p.m, p.n, p.k, 0, p.tail_first, p.epi, p.norm,
+  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<2, false, true>, p.tm_a, p.tm_b, p.tm_b_half, p.tm_out, 0, p.out, 0, p.m, p.n, p.k, 0, p.tail_first, p.group_m, p.epi, p.norm,
                             kernel_status_ptr());
 }
 

@@ -250,6 +250,54 @@ mk_status gemm_rownorm_tc2_emit(const Module& m, int lo, int hi, const Resolved&
   return MK_OK;
 }
 
+// The same operator range with the rows kept in tensor memory until their statistics are known (a cluster of CTA
+// pairs covers whole rows): one store of the normalised row, nothing read back.  The value handed to the norm may
+// itself be needed later (a residual stream): it is then written as well, from the same pass.
+bool chain_with_open_prenorm(const Module& m, int lo, int hi) {
+  if (hi - lo < 2) return false;
+  for (int j = lo + 1; j < hi; ++j)
+    if (m.ops[j].in_id[0] != m.ops[j - 1].out_id) return false;
+  for (int j = lo; j < hi - 2; ++j)
+    if (m.escapes(j, lo, hi)) return false;
+  for (int j = lo; j < hi; ++j)
+    if (m.ops[j].d.kind == MK_OP_RESIDUAL_ADD) {
+      const int prod = m.values[m.ops[j].in_id[1]].producer;
+      if (prod >= lo && prod < hi) return false;
+    }
+  return true;
+}
+bool gemm_rownorm_cl_match(const Module& m, int lo, int hi) {
+  if (!chain_with_open_prenorm(m, lo, hi)) return false;
+  const int32_t k = m.ops[hi - 1].d.kind;
+  if (k != MK_OP_LAYERNORM && k != MK_OP_RMSNORM) return false;
+  const Op& op = m.ops[lo];
+  if (op.d.kind != MK_OP_LINEAR || !in_is_module_dtype(m, lo) || m.values[0].spec.dtype != MK_BF16) return false;
+  if (op.d.i[1] != MK_LAYOUT_TRANSPOSED || !all_eltwise(m, lo + 1, hi - 1)) return false;
+  if (m.vspec(m.ops[hi - 1].out_id).dtype != MK_BF16) return false;
+  const mk_tensor_spec& xs = m.vspec(op.in_id[0]);
+  return gemm_rownorm_cl_supported(xs.shape[0], last_dim(m.vspec(m.ops[hi - 1].out_id)), xs.shape[1]);
+}
+mk_status gemm_rownorm_cl_emit(const Module& m, int lo, int hi, const Resolved& r, std::vector<Launch>& out, std::string& err) {
+  EpiProgram p;
+  mk_status st = build_epi(m, lo + 1, hi - 1, r, p, err);
+  if (st != MK_OK) return st;
+  const Op& op = m.ops[lo];
+  const Op& nop = m.ops[hi - 1];
+  const mk_tensor_spec& xs = m.vspec(op.in_id[0]);
+  const int64_t M = xs.shape[0], K = xs.shape[1], N = last_dim(m.vspec(nop.out_id));
+  const void* g = nop.param[0].set ? nop.param[0].ptr : nullptr;
+  const void* b = nop.param[1].set ? nop.param[1].ptr : nullptr;
+  const int pre = m.ops[hi - 2].out_id;
+  void* mid = m.escapes(hi - 2, lo, hi) ? r.value_ptr[pre] : nullptr;
+  const bool mid_f32 = m.vspec(pre).dtype == MK_F32;
+  auto plan = std::make_shared<GemmRowNormClPlan>();
+  cudaError_t e = gemm_rownorm_cl_plan(plan.get(), r.value_ptr[op.in_id[0]], op.param[0].ptr, r.value_ptr[nop.out_id], mid, mid_f32, M, N, K, p,
+                                       row_mode(nop.d.kind), g, b, (float)nop.d.f[0], m.ctx->sm_count);
+  if (e != cudaSuccess) { err = std::string("gemm_rownorm_cl plan: ") + cudaGetErrorString(e); return MK_ERR_CUDA; }
+  out.push_back([plan](cudaStream_t s) { return launch_gemm_rownorm_cl(*plan, s); });
+  return MK_OK;
+}
+
 // LINEAR [elementwise]* (LAYERNORM | RMSNORM), fp32, one CTA owns whole rows
 bool linear_rownorm_match(const Module& m, int lo, int hi) {
   if (hi - lo < 2 || !is_chain(m, lo, hi) || m.ops[lo].d.kind != MK_OP_LINEAR) return false;
@@ -438,6 +486,7 @@ mk_status attn_simt_emit(const Module& m, int lo, int, const Resolved& r, std::v
 const std::vector<Impl>& registry() {
   static const std::vector<Impl> reg = {
       {"linear_rownorm_simt", linear_rownorm_match, no_scratch, linear_rownorm_emit},
+      {"gemm_rownorm_cl", gemm_rownorm_cl_match, no_scratch, gemm_rownorm_cl_emit, false},
       {"gemm_rownorm_tc2", gemm_rownorm_tc2_match, gemm_rownorm_tc2_scratch_fn, gemm_rownorm_tc2_emit, false},
       {"gemm_tc2", gemm_tc2_match, no_scratch, gemm_tc2_emit},
       {"gemm_tc", gemm_tc_match, no_scratch, gemm_tc_emit},

@@ -25,6 +25,7 @@ enum WaitCode : unsigned {
   WAIT_TMEM_FULL = 3,
   WAIT_TMEM_EMPTY = 4,
   WAIT_ATTN = 5,
+  WAIT_ROW_STATS = 6,
   WAIT_SELFTEST = 99
 };
 
@@ -62,10 +63,13 @@ static __device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parit
                                             unsigned code, long long limit = kWaitLimitCycles) {
   const long long t0 = clock64();
   while (true) {
+    // checked first: after an expiry anywhere in the CTA, a role that still has a chain of waits ahead of it
+    // (a producer with a tile's worth of stages to go) must fall through each of them at once, not after
+    // another round of parked probes
+    if (*abort_flag) return false;
 #pragma unroll 1
     for (int i = 0; i < 32; ++i)
       if (mbar_try_wait(bar, parity)) return true;
-    if (*abort_flag) return false;
     if (clock64() - t0 > limit) {
       *abort_flag = 1;
       if (status) atomicExch(status, code);
@@ -336,6 +340,45 @@ __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.w
 __device__ __forceinline__ void cluster_sync() {
   asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Cluster-scope forms for data handed between CTAs through distributed shared memory: the writer stores into the
+// peer's shared memory, fences, and arrives (release) on the peer's barrier; the reader waits with acquire at
+// cluster scope before it reads.
+__device__ __forceinline__ void st_cluster_f32x2(uint32_t cluster_addr, float a, float b) {
+  asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(cluster_addr), "f"(a), "f"(b) : "memory");
+}
+__device__ __forceinline__ void fence_acq_rel_cluster() { asm volatile("fence.acq_rel.cluster;" ::: "memory"); }
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(20000u)
+      : "memory");
+  return ok != 0;
+}
+static __device__ __noinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity, volatile int* abort_flag, unsigned int* status,
+                                                      unsigned code, long long limit = kWaitLimitCycles) {
+  const long long t0 = clock64();
+  while (true) {
+    if (*abort_flag) return false;
+#pragma unroll 1
+    for (int i = 0; i < 32; ++i)
+      if (mbar_try_wait_cluster(bar, parity)) return true;
+    if (clock64() - t0 > limit) {
+      *abort_flag = 1;
+      if (status) atomicExch(status, code);
+      return false;
+    }
+  }
+}
+// one arrival on the barrier at this offset in the two CTAs of the pair whose leader has cluster rank `leader_rank`
+__device__ __forceinline__ void umma_commit_pair_at(uint64_t* bar, uint32_t leader_rank) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(smem_u32(bar)),
+               "h"((uint16_t)(3u << leader_rank))
+               : "memory");
 }
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");

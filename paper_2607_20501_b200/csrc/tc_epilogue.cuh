@@ -145,6 +145,7 @@ struct EpiWarp {
   uint8_t* bias;   // EPI_WARP_BIAS bytes, this warp's copy of the tile's bias slice
   int bias_idx, res_idx;
   bool res_f32, out_f32;
+  bool store = true;   // false: chunk_out applies the program to v and stores nothing (the caller goes on with v)
   int lane;
   __device__ __forceinline__ void init(uint8_t* warp_smem, const EpiProgram& p, int lane_, bool out_f32_) {
     stage = warp_smem;
@@ -275,7 +276,9 @@ struct EpiWarp {
       const int res_mode = get(ra, rb);
       if (my_row >= 0) epi32(epi, v, my_row, col0, n_cols, bias_idx >= 0 ? bias + bias_off * 2 : nullptr, res_mode, ra, rb);
       uint4 mine[4];
-      if (!out_f32) {
+      if (!store) {
+        // program only
+      } else if (!out_f32) {
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           mine[j].x = pack_bf16x2(v[8 * j + 0], v[8 * j + 1]);
@@ -304,6 +307,7 @@ struct EpiWarp {
           if (col0 + j < n_cols) {
             const float r = epi_apply(epi, v[j], my_row, col0 + j, n_cols);
             v[j] = r;   // callers that go on with the chunk (row statistics) see the values after the tail
+            if (!store) continue;
             if (out_f32) reinterpret_cast<float*>(out)[my_row * n_cols + col0 + j] = r;
             else reinterpret_cast<__nv_bfloat16*>(out)[my_row * n_cols + col0 + j] = __float2bfloat16_rn(r);
           }

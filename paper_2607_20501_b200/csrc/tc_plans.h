@@ -28,6 +28,7 @@ struct GemmTcPlan {
   bool use_tm_out = false;
   bool res_ring = false;    // a bf16 residual is staged through shared memory two chunks ahead (one pipeline stage less)
   int tail_first = 0;       // tiles from this index on run as two half-width units (= tile count: none)
+  int group_m = 16;         // tile rows walked together, column by column, so that their A rows and the W slabs stay in L2
   void* out = nullptr;
   bool out_f32 = false;     // output stored as fp32 (an fp32 residual stream), else bf16
   int m = 0, n = 0, k = 0;  // n = output columns
@@ -54,6 +55,30 @@ cudaError_t gemm_rownorm_tc2_plan(GemmTcPlan* p, const void* a, const void* w_nk
                                   const EpiProgram& epi, int mode, const void* gamma, const void* beta, float eps, void* scratch,
                                   int sm_count);
 cudaError_t launch_gemm_rownorm_tc2(const GemmTcPlan& p, cudaStream_t s);
+
+// GEMM + tail + row norm with the rows held in tensor memory until their statistics are known (a cluster of CTA
+// pairs covers whole rows and exchanges partial sums through distributed shared memory): y = norm(tail(A W)),
+// bf16; mid_out (optional, bf16 or fp32) also receives tail(A W), the value before the norm.
+struct GemmRowNormClPlan {
+  CUtensorMap tm_a, tm_b, tm_out;
+  void* out = nullptr;
+  void* mid_out = nullptr;
+  bool mid_f32 = false;
+  int m = 0, n = 0, k = 0;
+  int pairs = 1, nt = 1;     // CTA pairs per cluster; 256-column tiles per pair and row block
+  int grid = 0;
+  EpiProgram epi;
+  const void* gamma = nullptr;
+  const void* beta = nullptr;
+  float eps = 0.f;
+  int mode = 0;
+};
+// m > 128, k % 8 == 0, n % 8 == 0, n <= 2048
+bool gemm_rownorm_cl_supported(int64_t m, int64_t n, int64_t k);
+cudaError_t gemm_rownorm_cl_plan(GemmRowNormClPlan* p, const void* a, const void* w_nk, void* y, void* mid_out, bool mid_f32, int64_t m,
+                                 int64_t n, int64_t k, const EpiProgram& epi, int mode, const void* gamma, const void* beta, float eps,
+                                 int sm_count);
+cudaError_t launch_gemm_rownorm_cl(const GemmRowNormClPlan& p, cudaStream_t s);
 }  // namespace mk
 
 namespace mk {
