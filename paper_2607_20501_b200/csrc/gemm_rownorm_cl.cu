@@ -9,16 +9,20 @@
 // The rows stay in TMEM until their statistics are known:
 //   pass 1   an epilogue warp reads its accumulator chunks, applies the elementwise tail (bias, residual, ...),
 //            writes the result back to TMEM - and to global memory too when the value before the norm is needed
-//            later (a residual stream) - and sums it;
-//   pass 2   (LayerNorm) squares about the warp's own mean, again out of TMEM;
-//   exchange every warp leaves (mean, M2) or the sum of squares of its 32 rows in the shared memory of the P CTAs
-//            that hold the other columns of those rows (st.shared::cluster), fences, and arrives on their barrier;
-//   pass 3   after the barrier each lane combines the 2P partials of its own row (Chan's formula: no
-//            cancellation between a large mean and a small variance), normalises straight out of TMEM and the
-//            block leaves by a bulk tensor store.
+//            later (a residual stream) - and accumulates, per row, the sum and the sum of squares of the
+//            differences from a pivot (the row's first value in this warp's columns: sums about a value of
+//            the row itself lose nothing to cancellation when the mean is far from zero);
+//   exchange every lane sends (mean, M2) of its row over the warp's columns - for RMSNorm the sum of squares - to
+//            the P CTAs that hold the other columns of that row, as asynchronous stores into their shared memory
+//            that complete a transaction on their barrier (data and signal travel together);
+//   pass 2   after the barrier each lane combines the 2P partials of its own row (Chan's formula), normalises
+//            straight out of TMEM and the block leaves by a bulk tensor store.
+// A bf16 residual is copied into shared memory (cp.async, all of the tile's chunks for this warp) while the MMAs of
+// the row block run, so pass 1 never waits for global memory.
 // Nothing un-normalised is written and read back: against GEMM + row kernel this saves one write and one read of
 // the activation and a launch.  No TMA multicast: every CTA loads its own operands.
 #include <stdlib.h>
+#include <cstdio>
 
 #include "device_common.cuh"
 #include "tc_common.cuh"
@@ -31,11 +35,15 @@ namespace {
 constexpr int BM = 128, BN = 256, BK = 64, UMMA_K = 16;
 constexpr int EPI_WARPS = 8;
 constexpr int THREADS = 64 + 32 * EPI_WARPS;
-constexpr int STAGES = 5;
+constexpr int STAGES = 4;
 constexpr int A_BYTES = BM * BK * 2, B_BYTES = (BN / 2) * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int MAX_PAIRS = 4, MAX_NT = 2;
 constexpr int COLVEC_BYTES = 2 * MAX_NT * BN * 4;                  // gamma and beta of this pair's columns, fp32
 constexpr int PART_BYTES = 2 * MAX_PAIRS * 2 * BM * 8;             // [buffer][source pair][column half][row] float2
+constexpr int RES_SLOT_BYTES = 32 * 64;                           // one 32-row x 32-column bf16 residual chunk
+constexpr int RES_EXTRA_SLOTS = 3;                                // per epilogue warp, beside its staging buffer
+constexpr int RES_BYTES = EPI_WARPS * RES_EXTRA_SLOTS * RES_SLOT_BYTES;
+static_assert(RES_SLOT_BYTES <= EPI_WARP_STAGE, "the staging buffer serves as the first residual slot");
 
 struct SharedCl {
   uint64_t full[STAGES];
@@ -45,9 +53,10 @@ struct SharedCl {
   uint64_t stat_bar[2];
   uint32_t tmem_base;
   int abort_flag;
+  float ncols[MAX_PAIRS * 2];   // valid columns of every (pair, column half) warp: the weights of the partial means
   EpiProgram epi;
 };
-constexpr size_t SMEM_CL = (size_t)STAGES * STAGE_BYTES + EPI_WARPS * EPI_WARP_BYTES + COLVEC_BYTES + PART_BYTES + 1024 + 512;
+constexpr size_t SMEM_CL = (size_t)STAGES * STAGE_BYTES + EPI_WARPS * EPI_WARP_BYTES + COLVEC_BYTES + PART_BYTES + RES_BYTES + 1024 + 512;
 static_assert(sizeof(SharedCl) <= 512, "barrier block");
 static_assert(SMEM_CL <= 227 * 1024, "shared memory of one SM");
 
@@ -73,7 +82,8 @@ gemm_rownorm_cl_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
   float* gvec = reinterpret_cast<float*>(staging + EPI_WARPS * EPI_WARP_BYTES);   // [NT * 256]
   float* bvec = gvec + MAX_NT * BN;
   float2* part = reinterpret_cast<float2*>(reinterpret_cast<uint8_t*>(gvec) + COLVEC_BYTES);
-  SharedCl* sh = reinterpret_cast<SharedCl*>(reinterpret_cast<uint8_t*>(part) + PART_BYTES);
+  uint8_t* res_slots = reinterpret_cast<uint8_t*>(part) + PART_BYTES;
+  SharedCl* sh = reinterpret_cast<SharedCl*>(res_slots + RES_BYTES);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t crank = tc::cluster_ctarank();
   const uint32_t r = crank & 1u, leader_rank = crank & ~1u;
@@ -92,8 +102,9 @@ gemm_rownorm_cl_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
     for (int b = 0; b < 2; ++b) {
       tc::mbar_init(&sh->tfull[b], 1);
       tc::mbar_init(&sh->tempty[b], EPI_WARPS * 2);
-      tc::mbar_init(&sh->stat_bar[b], EPI_WARPS * P);     // every epilogue warp of the P CTAs that share these rows
+      tc::mbar_init(&sh->stat_bar[b], 1);     // one local arrival that announces the bytes the P CTAs sharing these rows will send
     }
+    for (int i = 0; i < MAX_PAIRS * 2; ++i) sh->ncols[i] = (float)warp_cols(i >> 1, i & 1, NT, N);
     sh->abort_flag = 0;
     tc::fence_barrier_init();
     tc::tma_prefetch_desc(&tmA);
@@ -189,32 +200,72 @@ gemm_rownorm_cl_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
     bool ok = true;
     int use = 0, it = 0;
     const float inv_n = 1.0f / (float)N;
-    const int n_w = warp_cols(pi, half, NT, N);
-    const float inv_nw = n_w > 0 ? 1.0f / (float)n_w : 0.0f;
+    const float n_w = sh->ncols[pi * 2 + half];
+    const float inv_nw = n_w > 0.0f ? 1.0f / n_w : 0.0f;
     const uint32_t part_local = tc::smem_u32(part);
     const uint32_t stat_local = tc::smem_u32(&sh->stat_bar[0]);
+    // A bf16 residual, when nothing else needs the staging buffer during pass 1 (no second output), is staged in
+    // shared memory: this warp's four chunks of a tile land in four slots (the staging buffer and three more) while
+    // the tile's MMAs run.  Slot layout as the bulk store's: a lane reads its own 64-byte row without conflicts.
+    const bool res_ring = ew.res_idx >= 0 && !ew.res_f32 && mid_out == nullptr && NT == 1;
+    uint8_t* my_slots = res_slots + (warp - 2) * RES_EXTRA_SLOTS * RES_SLOT_BYTES;
+    auto slot_ptr = [&](int i) -> uint8_t* { return i == 0 ? ew.stage : my_slots + (i - 1) * RES_SLOT_BYTES; };
+    auto ring_fill = [&](int64_t r0, int64_t col_base) {
+      const uint8_t* res = reinterpret_cast<const uint8_t*>(epi.op[ew.res_idx].ptr);
+      const int sub_row = lane >> 2, seg = lane & 3;
+      int i = 0;
+      for (int c = half; c < CHUNKS; c += 2, ++i) {
+        const int64_t c0 = col_base + c * 32;
+        if (c0 + 32 > N) break;
+        const uint32_t dst0 = tc::smem_u32(slot_ptr(i));
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const int rr = sub_row + 8 * k;
+          if (r0 + rr < M) tc::cp_async16(dst0 + rr * 64 + ((seg ^ ((rr >> 1) & 3)) * 16), res + ((r0 + rr) * (int64_t)N + c0) * 2 + seg * 16);
+        }
+      }
+      tc::cp_async_commit();
+    };
     for (int rb = cluster_id; rb < num_rb && ok; rb += num_clusters, ++it) {
       const int64_t row0 = (int64_t)(rb * 2 + (int)r) * BM + q * 32;
       auto rowmap = [&](int rr) -> int64_t { const int64_t g = row0 + rr; return g < M ? g : -1; };
       const int use0 = use;
+      const int buf = it & 1;
+#ifdef MK_TRACE_RN
+      long long tr[8];
+      tr[0] = clock64();
+#endif
       // the last bulk store of the row block before has finished reading the staging buffer, which pass 1 reuses
       if (lane == 0) tc::tma_store_wait_read();
       __syncwarp();
-      float s1 = 0.0f, s2 = 0.0f;   // this lane's row over the warp's columns: sum, then sum of squares (about the warp's mean for LayerNorm)
+      // announce what this row block's partials will bring to this CTA's barrier (one thread per CTA)
+      if (warp == 2 && lane == 0) tc::mbar_expect_tx(&sh->stat_bar[buf], (uint32_t)(P * EPI_WARPS * 32 * 8));
+      if (res_ring) ring_fill(row0, (int64_t)pi * BN);
+      // this lane's row over the warp's columns: for LayerNorm sums of (x - pivot) and (x - pivot)^2, for RMSNorm the sum of squares
+      float s1 = 0.0f, s2 = 0.0f, pivot = 0.0f;
+      bool have_pivot = false;
       // ---- pass 1: tail, write-back, sums
       for (int j = 0; j < NT && ok; ++j, ++use) {
         const int slot = use & 1;
         const int64_t col_base = (int64_t)(pi * NT + j) * BN;
         uint4 res_regs[8];
         ew.load_bias(epi, col_base, BN, N);
-        ew.prefetch_res(epi, rowmap, col_base + half * 32, N, res_regs);
+        if (!res_ring) ew.prefetch_res(epi, rowmap, col_base + half * 32, N, res_regs);
         ok = tc::mbar_wait(&sh->tfull[slot], (use >> 1) & 1, abort_flag, status, tc::WAIT_TMEM_FULL);
         ok = __all_sync(0xffffffffu, ok ? 1 : 0) != 0;
         if (!ok) break;
         tc::tc_fence_after();
+#ifdef MK_TRACE_RN
+        if (j == 0) tr[1] = clock64();
+#endif
+        if (res_ring) {
+          tc::cp_async_wait<0>();
+          __syncwarp();
+        }
         const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + slot * BN;
+        int ci = 0;
 #pragma unroll 1
-        for (int c = half; c < CHUNKS; c += 2) {
+        for (int c = half; c < CHUNKS; c += 2, ++ci) {
           const int64_t c0 = col_base + c * 32;
           if (c0 >= N) break;            // warp-uniform; nothing of this tile is left
           uint32_t rg[32];
@@ -223,7 +274,20 @@ gemm_rownorm_cl_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
           tc::tmem_ld_wait();
 #pragma unroll
           for (int k = 0; k < 32; ++k) v[k] = __uint_as_float(rg[k]);
-          ew.chunk_out(epi, v, rowmap, mid_out, c0, c * 32, (int64_t)N, res_regs, c + 2 < CHUNKS ? col_base + (c + 2) * 32 : -1);
+          if (res_ring) {
+            const uint8_t* src = slot_ptr(ci) + lane * 64;
+            const int f = (lane >> 1) & 3;
+            auto get = [&](uint4 (&ra)[4], uint4 (&)[4]) -> int {
+#pragma unroll
+              for (int k = 0; k < 4; ++k) ra[k] = *reinterpret_cast<const uint4*>(src + ((k ^ f) * 16));
+              return 1;
+            };
+            auto skip = [&]() {};
+            ew.chunk_out_from(epi, v, rowmap, mid_out, c0, c * 32, (int64_t)N, get, skip);
+          } else {
+            ew.chunk_out(epi, v, rowmap, mid_out, c0, c * 32, (int64_t)N, res_regs, c + 2 < CHUNKS ? col_base + (c + 2) * 32 : -1);
+          }
+          if (!have_pivot) { pivot = v[0]; have_pivot = true; }
 #pragma unroll
           for (int k = 0; k < 32; ++k) {
             if (c0 + k >= N) v[k] = 0.0f;
@@ -232,7 +296,10 @@ gemm_rownorm_cl_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
           tc::tmem_st32(t_row + c * 32, rg);
           if (mode == ROW_LAYERNORM) {
 #pragma unroll
-            for (int k = 0; k < 32; ++k) s1 += v[k];
+            for (int k = 0; k < 32; ++k) {
+              const float d = v[k] - pivot;
+              if (c0 + k < N) { s1 += d; s2 = fmaf(d, d, s2); }
+            }
           } else {
 #pragma unroll
             for (int k = 0; k < 32; ++k) s2 = fmaf(v[k], v[k], s2);
@@ -241,69 +308,54 @@ gemm_rownorm_cl_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
         tc::tmem_st_wait();
       }
       if (!ok) break;
-      // ---- pass 2 (LayerNorm): squares about this warp's own mean
-      float mean_w = 0.0f;
-      if (mode == ROW_LAYERNORM) {
-        mean_w = s1 * inv_nw;
-        for (int j = 0; j < NT; ++j) {
-          const int slot = (use0 + j) & 1;
-          const int64_t col_base = (int64_t)(pi * NT + j) * BN;
-          const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + slot * BN;
-#pragma unroll 1
-          for (int c = half; c < CHUNKS; c += 2) {
-            const int64_t c0 = col_base + c * 32;
-            if (c0 >= N) break;
-            uint32_t rg[32];
-            tc::tmem_ld32(t_row + c * 32, rg);
-            tc::tmem_ld_wait();
-#pragma unroll
-            for (int k = 0; k < 32; ++k) {
-              const float d = __uint_as_float(rg[k]) - mean_w;
-              if (c0 + k < N) s2 = fmaf(d, d, s2);
-            }
-          }
-        }
-      }
-      // ---- exchange: this warp's partial for its 32 rows goes to the P CTAs that hold the rest of those rows
+#ifdef MK_TRACE_RN
+      tr[2] = clock64();
+      tr[3] = tr[2];
+#endif
+      // ---- exchange: this lane's partial goes to the P CTAs that hold the rest of its row
       {
-        const int buf = it & 1;
+        float mean_w = 0.0f, m2_w = s2;
+        if (mode == ROW_LAYERNORM) {
+          mean_w = pivot + s1 * inv_nw;
+          m2_w = fmaxf(s2 - s1 * s1 * inv_nw, 0.0f);
+        }
         const uint32_t slot_off = (uint32_t)((((buf * MAX_PAIRS + pi) * 2 + half) * BM + q * 32 + lane) * 8);
-        for (int pj = 0; pj < P; ++pj)
-          tc::st_cluster_f32x2(tc::map_to_cta(part_local + slot_off, (uint32_t)(2 * pj) + r), mean_w, s2);
-        tc::fence_acq_rel_cluster();
-        __syncwarp();
-        if (lane == 0)
-          for (int pj = 0; pj < P; ++pj) tc::mbar_arrive_cluster(tc::map_to_cta(stat_local + (uint32_t)buf * 8u, (uint32_t)(2 * pj) + r));
-        ok = tc::mbar_wait_cluster(&sh->stat_bar[buf], (it >> 1) & 1, abort_flag, status, tc::WAIT_ROW_STATS);
+        for (int pj = 0; pj < P; ++pj) {
+          const uint32_t dst_rank = (uint32_t)(2 * pj) + r;
+          tc::st_async_f32x2(tc::map_to_cta(part_local + slot_off, dst_rank), mean_w, m2_w, tc::map_to_cta(stat_local + (uint32_t)buf * 8u, dst_rank));
+        }
+        ok = tc::mbar_wait(&sh->stat_bar[buf], (it >> 1) & 1, abort_flag, status, tc::WAIT_ROW_STATS);
         ok = __all_sync(0xffffffffu, ok ? 1 : 0) != 0;
         if (!ok) break;
       }
+#ifdef MK_TRACE_RN
+      tr[4] = clock64();
+#endif
       // ---- combine the 2P partials of this lane's row
       float mean = 0.0f, rstd;
       {
-        const int buf = it & 1;
         const float2* pp = part + (size_t)buf * MAX_PAIRS * 2 * BM + q * 32 + lane;
         if (mode == ROW_LAYERNORM) {
           float sm = 0.0f;
-          for (int pj = 0; pj < P; ++pj)
-            for (int h = 0; h < 2; ++h) sm += (float)warp_cols(pj, h, NT, N) * pp[(pj * 2 + h) * BM].x;
+          for (int i = 0; i < 2 * P; ++i) sm += sh->ncols[i] * pp[i * BM].x;
           mean = sm * inv_n;
           float m2 = 0.0f;
-          for (int pj = 0; pj < P; ++pj)
-            for (int h = 0; h < 2; ++h) {
-              const float2 t = pp[(pj * 2 + h) * BM];
-              const float d = t.x - mean;
-              m2 += t.y + (float)warp_cols(pj, h, NT, N) * d * d;
-            }
+          for (int i = 0; i < 2 * P; ++i) {
+            const float2 t = pp[i * BM];
+            const float d = t.x - mean;
+            m2 += t.y + sh->ncols[i] * d * d;
+          }
           rstd = rsqrtf(m2 * inv_n + eps);
         } else {
           float sq = 0.0f;
-          for (int pj = 0; pj < P; ++pj)
-            for (int h = 0; h < 2; ++h) sq += pp[(pj * 2 + h) * BM].y;
+          for (int i = 0; i < 2 * P; ++i) sq += pp[i * BM].y;
           rstd = rsqrtf(sq * inv_n + eps);
         }
       }
-      // ---- pass 3: normalise out of TMEM, store, hand the accumulator back
+#ifdef MK_TRACE_RN
+      tr[5] = clock64();
+#endif
+      // ---- pass 2: normalise out of TMEM, store, hand the accumulator back
       const float nm = -mean * rstd;
       for (int j = 0; j < NT; ++j) {
         const int slot = (use0 + j) & 1;
@@ -347,7 +399,14 @@ gemm_rownorm_cl_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
         __syncwarp();
         if (lane == 0) tc::mbar_arrive_cluster(tc::map_to_cta(tc::smem_u32(&sh->tempty[slot]), leader_rank));
       }
+#ifdef MK_TRACE_RN
+      tr[6] = clock64();
+      if (blockIdx.x == 0 && lane == 0 && (warp == 2 || warp == 9))
+        printf("rn w%d it%d: wait_full %lld p1 %lld p2 %lld exch %lld comb %lld p3 %lld total %lld\n", warp, it, tr[1] - tr[0], tr[2] - tr[1],
+               tr[3] - tr[2], tr[4] - tr[3], tr[5] - tr[4], tr[6] - tr[5], tr[6] - tr[0]);
+#endif
     }
+    if (res_ring) tc::cp_async_wait<0>();
     if (lane == 0) tc::tma_store_wait_all();
   }
 
@@ -393,11 +452,27 @@ cudaError_t gemm_rownorm_cl_plan(GemmRowNormClPlan* p, const void* a, const void
   p->m = (int)m; p->n = (int)n; p->k = (int)k;
   p->epi = epi; p->gamma = gamma; p->beta = beta; p->eps = eps; p->mode = mode;
   const int64_t row_blocks = (m + 2 * BM - 1) / (2 * BM);
+  // A cluster lives inside one GPC, so fewer clusters of eight fit the machine than SMs / 8 (16 on a B200 whose
+  // GPCs have 18 or 20 SMs): a cluster beyond that number would only start when another has finished and
+  // double the kernel's time.  Ask the runtime how many can be resident at once.
   int64_t clusters = sm_count / (2 * P);
+  {
+    static SmemOptIn opt_in;
+    cudaError_t e2 = opt_in.ensure(SMEM_CL, gemm_rownorm_cl_kernel);
+    if (e2 != cudaSuccess) return e2;
+    LaunchCfg lc(0, dim3((unsigned)(clusters * 2 * P)), dim3(THREADS), SMEM_CL, nullptr, 2 * P);
+    int active = 0;
+    if (cudaOccupancyMaxActiveClusters(&active, gemm_rownorm_cl_kernel, &lc.cfg) == cudaSuccess && active > 0) {
+      if (active < clusters) clusters = active;
+    } else {
+      cudaGetLastError();
+    }
+  }
   const char* ov = getenv("MK_ROWNORM_CLUSTERS");
   if (ov && ov[0]) clusters = atoi(ov);
   if (clusters > row_blocks) clusters = row_blocks;
   if (clusters < 1) clusters = 1;
+  if (getenv("MK_DEBUG_PLAN")) fprintf(stderr, "gemm_rownorm_cl plan: m %d n %d k %d pairs %d nt %d clusters %d\n", (int)m, (int)n, (int)k, P, NT, (int)clusters);
   p->grid = (int)(clusters * 2 * P);
   return cudaSuccess;
 }
