@@ -21,8 +21,10 @@ def _bf16_round(x):
     return W.bf16_bits_to_f64(W.f32_to_bf16_bits(np.asarray(x, np.float32)))
 
 
+# the last two: more tiles than CTA pairs with a last wave of at most half the pairs, which runs as units of half the
+# output channels each (320 and 150 tiles on 74 pairs; C_out 128 and 256)
 SHAPES = [(1, 4, 4, 64, 32), (2, 8, 8, 64, 64), (3, 9, 7, 128, 128), (2, 13, 62, 64, 96), (1, 56, 56, 128, 128),
-          (5, 6, 10, 64, 256)]
+          (5, 6, 10, 64, 256), (20, 64, 20, 64, 128), (25, 24, 9, 64, 256)]
 
 
 @pytest.mark.parametrize("nb,h,w,c,co", SHAPES)
@@ -51,7 +53,7 @@ def test_conv_chain_matches_the_oracle(ctx, nb, h, w, c, co):
 
 
 @pytest.mark.parametrize("nb,h,w,c,co,g", [(2, 8, 8, 64, 64, 16), (3, 9, 7, 128, 128, 32), (2, 13, 62, 64, 128, 16), (1, 6, 10, 64, 256, 16),
-                                           (2, 5, 33, 64, 32, 1), (4, 56, 56, 128, 128, 32)])
+                                           (2, 5, 33, 64, 32, 1), (4, 56, 56, 128, 128, 32), (20, 64, 20, 64, 128, 32), (25, 24, 9, 64, 256, 8)])
 def test_groupnorm_statistics_from_the_conv_epilogue(ctx, nb, h, w, c, co, g):
     """The fused form: the convolution's epilogue leaves per-(image, group) partial sums of what it stores
     and the normalisation reads only those (4, 8, 16 and 32 channels per group; image heights that do not
