@@ -63,6 +63,28 @@ struct SmemOptIn {
   }
 };
 
+// Blocks of one kernel that can be resident on the current device at once (SM count x blocks per SM at the kernel's
+// register and shared-memory footprint), asked once per device: the grid size of a persistent launch.
+struct ResidentBlocks {
+  std::atomic<int> n[kMaxDevices] = {};
+  template <typename K>
+  int get(K kernel, int block_threads, size_t dyn_smem = 0) {
+    const int dev = current_device();
+    if (dev < 0) return 0;
+    int v = n[dev].load(std::memory_order_acquire);
+    if (v > 0) return v;
+    int per_sm = 0, sms = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, block_threads, dyn_smem) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || per_sm < 1 || sms < 1) {
+      cudaGetLastError();
+      return 0;
+    }
+    v = per_sm * sms;
+    n[dev].store(v, std::memory_order_release);
+    return v;
+  }
+};
+
 // ---- device status word (bounded-wait expiry codes) --------------------------------------------------
 unsigned int* kernel_status_ptr();   // address on the current device, nullptr without one
 cudaError_t kernel_status_fetch_and_clear(unsigned int* out);   // of the current device
