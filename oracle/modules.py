@@ -23,6 +23,8 @@ def apply_op(op, vals, params):
     a = op["attrs"]
     if kind == "linear":
         return O.linear(ins[0], p["w"])
+    if kind == "linear_fp8":
+        return O.linear_fp8_block(ins[0], ins[1], p["w"], p["sw"])
     if kind == "conv2d_3x3":
         return O.conv2d_3x3_nhwc(ins[0], p["w"])
     if kind == "bias_add":

@@ -46,6 +46,21 @@ def linear(x, w):
     return x @ w
 
 
+def linear_fp8_block(xq, sx, wq, sw, block=128):
+    """Block-scaled fp8 contraction (the paper's FP8 MoE inference task; blocks as in that task: activations one
+    scale per row and 128-wide K block, weights one per 128 x 128 block):
+        Y[m, n] = sum_kb sx[m, kb] * sw[n // 128, kb] * sum_{k in block kb} xq[m, k] * wq[k, n]
+    xq [M, K] and wq [K, N] hold the decoded fp8 values (exact in fp64), sx [M, K/128], sw [ceil(N/128), K/128].
+    Written as the definition: dequantise, then the plain contraction."""
+    xq, sx, wq, sw = _f64(xq), _f64(sx), _f64(wq), _f64(sw)
+    M, K = xq.shape
+    N = wq.shape[1]
+    assert K % block == 0 and sx.shape == (M, K // block) and sw.shape == (-(-N // block), K // block)
+    x = xq * np.repeat(sx, block, axis=1)
+    wscale = np.repeat(np.repeat(sw.T, block, axis=0), block, axis=1)[:K, :N]      # [K, N]
+    return x @ (wq * wscale)
+
+
 def conv2d_3x3_nhwc(x, w):
     """Y[n,h,w,co] = sum_{kh,kw,ci} Xpad[n, h+kh-1, w+kw-1, ci] * W[co,kh,kw,ci]
 

@@ -185,7 +185,17 @@ def _hand_c7(w, pool):
     return v, "y3"
 
 
+def _hand_c8(w):
+    i, p = _widen(w)
+    v = {}
+    v["y0"] = O.linear_fp8_block(i["xq"], i["sx"], p["Wq"], p["sw"])
+    v["y1"] = O.bias_add(v["y0"], p["bias"])
+    v["y2"] = O.silu(v["y1"])
+    return v, "y2"
+
+
 HAND = {
+    "c8": (lambda s: W.c8(s, M=24, K=256, N=136, bias=True), _hand_c8),
     "c1": (lambda s: W.c1(s), _hand_c1),
     "c2": (lambda s: W.c2(s, M=48, K=64, N=40), _hand_c2),
     "c3": (lambda s: W.c3(s, NB=2, H=6, W=5, C=8, CO=8, G=4), _hand_c3),

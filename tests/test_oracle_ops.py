@@ -424,3 +424,59 @@ def test_pooling_brute_force_library_and_invariants():
     assert O.avgpool_nhwc(rnd(1, 8, 8, 1), 3, 2).shape == (1, 3, 3, 1)
     with pytest.raises(ValueError):
         O.avgpool_nhwc(rnd(1, 2, 2, 1), 3, 1)
+
+
+def test_linear_fp8_block_scaled():
+    """Block-scaled fp8 contraction: brute force with the scale looked up per element, the special case of unit
+    scales (the plain linear), a single non-zero activation (pins which scale multiplies which block, and the
+    [N-block, K-block] orientation of the weight scales), homogeneity in every scale, exact integers."""
+    rng = np.random.default_rng(5)
+    blk = 4
+    M, K, N = 5, 12, 10                       # 3 K blocks, 3 N blocks (the last one partial)
+    xq = rng.integers(-8, 9, (M, K)).astype(np.float64) / 4
+    wq = rng.integers(-8, 9, (K, N)).astype(np.float64) / 8
+    sx = rng.uniform(0.5, 2.0, (M, K // blk))
+    sw = rng.uniform(0.5, 2.0, (-(-N // blk), K // blk))
+    y = O.linear_fp8_block(xq, sx, wq, sw, block=blk)
+    assert y.shape == (M, N)
+    for m in range(M):
+        for n in range(N):
+            acc = 0.0
+            for k in range(K):
+                acc += (xq[m, k] * sx[m, k // blk]) * (wq[k, n] * sw[n // blk, k // blk])
+            assert abs(y[m, n] - acc) < 1e-12
+    # unit scales: the plain contraction
+    one_x, one_w = np.ones_like(sx), np.ones_like(sw)
+    assert np.array_equal(O.linear_fp8_block(xq, one_x, wq, one_w, block=blk), O.linear(xq, wq))
+    # one non-zero activation: row m0 of the result is a * sx[m0, kb0] * sw[:, kb0] (per column block) * wq[k0, :]
+    m0, k0 = 3, 6
+    e = np.zeros_like(xq)
+    e[m0, k0] = 1.5
+    y1 = O.linear_fp8_block(e, sx, wq, sw, block=blk)
+    want = 1.5 * sx[m0, k0 // blk] * np.repeat(sw[:, k0 // blk], blk)[:N] * wq[k0]
+    assert np.allclose(y1[m0], want, rtol=0, atol=1e-14) and not y1[np.arange(M) != m0].any()
+    # a transposed scale table would change the answer (the two block counts differ only when N != K; here they are equal: use values)
+    assert not np.allclose(O.linear_fp8_block(xq, sx, wq, sw.T.copy(), block=blk), y)
+    # homogeneity: doubling one activation scale doubles that (row, K block)'s contribution only
+    sx2 = sx.copy()
+    sx2[1, 2] *= 2
+    d = O.linear_fp8_block(xq, sx2, wq, sw, block=blk) - y
+    contrib = (xq[1, 8:12] * sx[1, 2]) @ (wq[8:12] * np.repeat(sw[:, 2], blk)[:N])
+    assert np.allclose(d[1], contrib, atol=1e-13) and not d[np.arange(M) != 1].any()
+    # integers with power-of-two scales: exact
+    xi = rng.integers(-4, 5, (M, K)).astype(np.float64)
+    wi = rng.integers(-4, 5, (K, N)).astype(np.float64)
+    s2 = 2.0 ** rng.integers(-2, 3, sx.shape)
+    w2 = 2.0 ** rng.integers(-2, 3, sw.shape)
+    yi = O.linear_fp8_block(xi, s2, wi, w2, block=blk)
+    brute = np.zeros((M, N))
+    for kb in range(K // blk):
+        part = xi[:, kb * blk:(kb + 1) * blk] @ wi[kb * blk:(kb + 1) * blk]
+        brute += part * s2[:, kb:kb + 1] * np.repeat(w2[:, kb], blk)[:N][None, :]
+    assert np.array_equal(yi, brute)
+    # the default block is the task's 128
+    big = O.linear_fp8_block(np.ones((2, 256)), np.array([[1.0, 3.0], [2.0, 1.0]]), np.ones((256, 130)),
+                             np.array([[1.0, 1.0], [1.0, 10.0]]))
+    assert np.array_equal(big[:, 0], [128 + 384, 256 + 128]) and np.array_equal(big[:, 129], [128 + 3840, 256 + 1280])
+    with pytest.raises(AssertionError):
+        O.linear_fp8_block(np.ones((2, 100)), np.ones((2, 1)), np.ones((100, 4)), np.ones((1, 1)))

@@ -15,6 +15,9 @@ from .generate import (  # noqa: F401
     c5,
     c6,
     c7,
+    c8,
+    e4m3_bits_to_f64,
+    f32_to_e4m3_bits,
     f32_to_bf16_bits,
     int_valued,
     make,

@@ -36,12 +36,55 @@ def bf16_bits_to_f64(b: np.ndarray) -> np.ndarray:
     return bf16_bits_to_f32(b).astype(np.float64)
 
 
+# fp8 e4m3 ("fn" variant: bias 7, no infinities, 0x7f / 0xff NaN, largest finite 448, subnormals of 2^-9)
+def _e4m3_table() -> np.ndarray:
+    t = np.empty(256, np.float64)
+    for b in range(256):
+        e, m = (b >> 3) & 0xF, b & 7
+        if e == 15 and m == 7:
+            v = np.nan
+        elif e == 0:
+            v = m * 2.0 ** -9
+        else:
+            v = (1.0 + m / 8.0) * 2.0 ** (e - 7)
+        t[b] = -v if b & 0x80 else v
+    return t
+
+
+E4M3_VALUES = _e4m3_table()
+E4M3_MAX = 448.0
+
+
+def f32_to_e4m3_bits(x: np.ndarray) -> np.ndarray:
+    """fp32 -> e4m3 codes (uint8), round-to-nearest-even, magnitudes beyond 448 saturate to 448."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    sign = (np.signbit(x)).astype(np.uint8) << 7
+    a = np.minimum(np.abs(x).astype(np.float64), E4M3_MAX)
+    f, ex = np.frexp(a)                      # a = f * 2^ex, f in [0.5, 1)
+    e = ex - 1                               # a = (2 f) * 2^e, 2 f in [1, 2)
+    normal = a >= 2.0 ** -6
+    mant = np.rint((2.0 * f - 1.0) * 8.0)    # ties to even
+    carry = mant == 8
+    e = np.where(carry, e + 1, e)
+    mant = np.where(carry, 0, mant)
+    nb = ((e + 7).astype(np.int64) << 3) | mant.astype(np.int64)
+    sb = np.rint(a * 2.0 ** 9).astype(np.int64)   # subnormals: multiples of 2^-9; 8 is the smallest normal's code
+    bits = np.where(normal, nb, sb)
+    bits = np.minimum(bits, 0x7E)
+    return (bits.astype(np.uint8) | sign).astype(np.uint8)
+
+
+def e4m3_bits_to_f64(b: np.ndarray) -> np.ndarray:
+    return E4M3_VALUES[b]
+
+
 @dataclass
 class Tensor:
     """One named tensor in its storage format.
 
     dtype "f32": `store` is float32.  dtype "bf16": `store` is uint16 holding
-    bf16 bit patterns.  Shapes are logical, row-major, innermost last.
+    bf16 bit patterns.  dtype "fp8": `store` is uint8 holding e4m3 codes.
+    Shapes are logical, row-major, innermost last.
     """
 
     name: str
@@ -55,6 +98,8 @@ class Tensor:
     def f64(self) -> np.ndarray:
         if self.dtype == "bf16":
             return bf16_bits_to_f64(self.store)
+        if self.dtype == "fp8":
+            return e4m3_bits_to_f64(self.store)
         return self.store.astype(np.float64)
 
     def nbytes(self) -> int:
@@ -68,7 +113,26 @@ def make(name: str, dtype: str, values_f32: np.ndarray) -> Tensor:
         return Tensor(name, "bf16", f32_to_bf16_bits(v))
     if dtype == "f32":
         return Tensor(name, "f32", v)
+    if dtype == "fp8":
+        return Tensor(name, "fp8", f32_to_e4m3_bits(v))
     raise ValueError(f"unknown dtype {dtype!r}")
+
+
+def quantize_blocks(name: str, values_f32: np.ndarray, block_rows: int, block_cols: int):
+    """Synthesis of a block-scaled fp8 tensor from fp32 values: one fp32 scale per block_rows x block_cols block,
+    scale = amax / 448, codes = e4m3(value / scale).  Returns (codes Tensor [R, C], scales Tensor
+    [ceil(R / block_rows), ceil(C / block_cols)]).  This only MAKES inputs; what a consumer computes from
+    codes and scales is defined where it is computed."""
+    v = np.ascontiguousarray(values_f32, dtype=np.float32)
+    R, Cc = v.shape
+    nr, nc = -(-R // block_rows), -(-Cc // block_cols)
+    pad = np.zeros((nr * block_rows, nc * block_cols), np.float32)
+    pad[:R, :Cc] = v
+    blk = pad.reshape(nr, block_rows, nc, block_cols)
+    amax = np.abs(blk).max(axis=(1, 3))
+    scale = (np.maximum(amax, np.float32(1e-10)) / np.float32(E4M3_MAX)).astype(np.float32)
+    q = (blk / scale[:, None, :, None]).astype(np.float32).reshape(nr * block_rows, nc * block_cols)[:R, :Cc]
+    return Tensor(name, "fp8", f32_to_e4m3_bits(q)), Tensor(name + "_scale", "f32", scale)
 
 
 # --------------------------------------------------------------------------
@@ -348,4 +412,25 @@ def c7(seed=0, NB=32, H=56, W=56, C=128, CO=128, pool="avg", k=7, stride=7, p=2.
     return w
 
 
-WORKLOADS = {"c1": c1, "c2": c2, "c3": c3, "c4": c4, "c5": c5, "c6": c6, "c7": c7}
+# --------------------------------------------------------------------------
+# C8: block-scaled fp8 GEMM, the contraction of the paper's FP8 MoE inference task: activations quantised per
+# token and 128-channel block, weights per 128 x 128 block, fp32 scales, bf16 result (the expert projection
+# shape hidden 7168 -> 4096 by default)
+# --------------------------------------------------------------------------
+def c8(seed=0, M=4096, K=7168, N=4096, bias=False) -> Workload:
+    w = Workload("c8", "bf16")
+    xq, sx = quantize_blocks("xq", _normal(seed, 0, (M, K)), 1, 128)
+    wq, sw = quantize_blocks("Wq", _normal(seed, 1, (K, N), std=(1.0 / K) ** 0.5), 128, 128)
+    w.inputs["xq"], w.inputs["sx"] = xq, Tensor("sx", "f32", sx.store)
+    w.params["Wq"], w.params["sw"] = wq, Tensor("sw", "f32", np.ascontiguousarray(sw.store.T))   # [N / 128, K / 128]
+    w.ops = [_op("linear_fp8", "y0", ["xq", "sx"], {"w": "Wq", "sw": "sw"}, n=N)]
+    if bias:
+        w.params["bias"] = make("bias", "bf16", _normal(seed, 2, (N,), std=0.02))
+        w.ops += [_op("bias_add", "y1", ["y0"], {"b": "bias"}), _op("silu", "y2", ["y1"])]
+    w.partitions = {"fused": [0], "per_op": list(range(len(w.ops)))}
+    w.flops = 2.0 * M * K * N
+    w.min_bytes = M * K + K * N + 4 * (sx.store.size + sw.store.size) + 2 * M * N
+    return w
+
+
+WORKLOADS = {"c1": c1, "c2": c2, "c3": c3, "c4": c4, "c5": c5, "c6": c6, "c7": c7, "c8": c8}
