@@ -22,6 +22,9 @@
  *   - Every pointer named dev_* / in_ptrs[i] / out_ptrs[i] / workspace is a DEVICE pointer
  *     owned by the caller; the library borrows it and never allocates, frees or copies
  *     device memory.  All other pointers are HOST pointers.
+ *   - A module's activations have ONE storage type, MK_F32 or MK_BF16: that of its inputs.  A module that has
+ *     an MK_FP8_E4M3 input is a bf16 module; beside its fp8 inputs it may have MK_F32 inputs (the block scales)
+ *     and MK_BF16 ones.  fp8 and scale tensors may only feed LINEAR_FP8.
  *   - Tensors are dense, row-major, innermost dimension last.  Device pointers must be
  *     16-byte aligned.
  *   - Every function returns an mk_status (0 = MK_OK, negative = error) and never throws or
@@ -74,7 +77,9 @@ enum {
   MK_ERR_PARAM_MISSING = -10
 };
 
-typedef enum { MK_F32 = 0, MK_BF16 = 1 } mk_dtype;
+/* MK_FP8_E4M3: 8-bit float, 4 exponent bits (bias 7), 3 mantissa bits, no infinities, 0x7f / 0xff are NaN, largest
+ * finite value 448 (the "fn" variant).  Only LINEAR_FP8 reads it. */
+typedef enum { MK_F32 = 0, MK_BF16 = 1, MK_FP8_E4M3 = 2 } mk_dtype;
 
 /* Physical layout of a rank-2 tensor.  MK_LAYOUT_TRANSPOSED stores the logical [R, C] matrix
  * as its transpose, i.e. a dense row-major [C, R] array (a linear weight kept [out, in]). */
@@ -120,6 +125,14 @@ typedef struct mk_tensor_spec {
  *                   [N, (H - k) / stride + 1, (W - k) / stride + 1, C] (whole windows only).  Mean, maximum, and
  *                   the p-norm (sum |x|^p)^(1/p) with p = f[0] >= 1 of each window: the pooling subkernel of the
  *                   paper's MobileNetV1 example and the two variants of its transfer study.
+ *   LINEAR_FP8      block-scaled fp8 GEMM, the contraction of the paper's FP8 MoE inference task:
+ *                   y[M,N] = sum over K blocks kb of sx[m,kb] * sw[n/128,kb] * sum_{k in block kb} xq[m,k] * wq[k,n]
+ *                   with blocks of 128 along K (activations: one scale per row and block; weights: one per
+ *                   128 x 128 block).  in[0] = xq [M,K] MK_FP8_E4M3, in[1] = sx [M, K/128] MK_F32;
+ *                   param 0 = wq (logical [K,N], MK_FP8_E4M3; i[1] = mk_layout of its storage),
+ *                   param 1 = sw [ceil(N/128), K/128] MK_F32; i[0] = N; K must be a multiple of 128.
+ *                   The result has the module's activation type (bf16 in a module that has fp8 inputs); the
+ *                   products are accumulated in fp32 and every block's partial sum is scaled in fp32.
  * Definitions: the paper's subkernel listings (linear with W stored [K, N]; LayerNorm; online-
  * softmax attention) and its correctness appendix (safe softmax, tril(diagonal=0) mask, fp32
  * accumulation); RMSNorm, GroupNorm, SwiGLU, tanh-GELU and the 3x3 convolution follow the
@@ -144,7 +157,8 @@ typedef enum {
   MK_OP_ATTENTION = 16,
   MK_OP_AVGPOOL2D = 17,
   MK_OP_MAXPOOL2D = 18,
-  MK_OP_LPPOOL2D = 19
+  MK_OP_LPPOOL2D = 19,
+  MK_OP_LINEAR_FP8 = 20
 } mk_op_kind;
 
 /* Value numbering: module input k has id k; operator j produces id n_inputs + j.

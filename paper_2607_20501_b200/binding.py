@@ -26,7 +26,7 @@ STATUS = {
 }
 for _code, _name in STATUS.items():
     globals()[_name] = _code
-MK_F32, MK_BF16 = 0, 1
+MK_F32, MK_BF16, MK_FP8_E4M3 = 0, 1, 2
 MK_LAYOUT_ROW_MAJOR, MK_LAYOUT_TRANSPOSED = 0, 1
 MK_MAX_RANK = 4
 MK_PREV, MK_NONE = -1, -2
@@ -34,8 +34,9 @@ OP = {
     "linear": 1, "conv2d_3x3": 2, "bias_add": 3, "relu": 4, "gelu_tanh": 5, "silu": 6, "scale": 7,
     "clamp": 8, "residual_add": 9, "swiglu": 10, "layernorm": 11, "rmsnorm": 12, "groupnorm": 13,
     "softmax": 14, "attention_causal": 15, "attention": 16, "avgpool": 17, "maxpool": 18, "lppool": 19,
+    "linear_fp8": 20,
 }
-DTYPE = {"f32": MK_F32, "bf16": MK_BF16}
+DTYPE = {"f32": MK_F32, "bf16": MK_BF16, "fp8": MK_FP8_E4M3}
 
 
 class mk_tensor_spec(C.Structure):
@@ -158,7 +159,7 @@ class Module:
     weight_layout picks how LINEAR weights are stored (MK_LAYOUT_*).
     """
 
-    PARAM_SLOTS = {"linear": ("w",), "conv2d_3x3": ("w",), "bias_add": ("b",), "rmsnorm": ("gamma",),
+    PARAM_SLOTS = {"linear": ("w",), "linear_fp8": ("w", "sw"), "conv2d_3x3": ("w",), "bias_add": ("b",), "rmsnorm": ("gamma",),
                    "layernorm": ("gamma", "beta"), "groupnorm": ("gamma", "beta")}
 
     def __init__(self, ctx: Context, ops, inputs, weight_layout=MK_LAYOUT_TRANSPOSED):
@@ -188,7 +189,7 @@ class Module:
                 d.i[0] = a["groups"]
             elif kind == "residual_add":
                 d.i[0] = 1 if a.get("store") == "f32" else 0
-            elif kind == "linear":
+            elif kind in ("linear", "linear_fp8"):
                 d.i[0] = int(a["n"])
                 d.i[1] = weight_layout
             elif kind == "conv2d_3x3":
@@ -299,17 +300,18 @@ class Module:
         self._ck(mk_module_set_param(self.h, op_index, slot, _ptr(tensor), C.byref(spec)))
         self._keep.append(tensor)
 
-    def set_params(self, device_params, dtype):
+    def set_params(self, device_params, dtype, param_dtypes=None):
         """device_params: name -> (tensor on the device, logical shape).  LINEAR weights must
-        already be stored in this module's weight_layout."""
+        already be stored in this module's weight_layout.  param_dtypes: name -> storage type of the
+        parameters that do not have the module's (fp8 weights and their fp32 block scales)."""
         for j, op in enumerate(self.ops):
             for slot, key in enumerate(self.PARAM_SLOTS.get(op["kind"], ())):
                 name = op["params"].get(key)
                 if name is None:
                     continue
                 t, shape = device_params[name]
-                layout = self.weight_layout if op["kind"] == "linear" else MK_LAYOUT_ROW_MAJOR
-                self.set_param(j, slot, t, dtype, shape, layout)
+                layout = self.weight_layout if (op["kind"] in ("linear", "linear_fp8") and slot == 0) else MK_LAYOUT_ROW_MAJOR
+                self.set_param(j, slot, t, (param_dtypes or {}).get(name, dtype), shape, layout)
 
     def keep_intermediates(self, keep=True):
         self._ck(mk_module_keep_intermediates(self.h, 1 if keep else 0))

@@ -289,11 +289,15 @@ mk_status mk_module_set_param(mk_module* m, int32_t op, int32_t slot, const void
   const mk_tensor_spec& x = m->values[o.in_id[0]].spec;
   const int64_t last = x.shape[x.rank - 1];
   mk_tensor_spec want{};
-  want.dtype = m->values[0].spec.dtype;   // parameters always have the module's storage type
+  want.dtype = m->dtype;   // parameters always have the module's storage type
   bool ok = false;
   switch (o.d.kind) {
     case MK_OP_LINEAR:
       if (slot == 0) { want.rank = 2; want.shape[0] = last; want.shape[1] = o.d.i[0]; want.layout = o.d.i[1]; ok = true; }
+      break;
+    case MK_OP_LINEAR_FP8:
+      if (slot == 0) { want.dtype = MK_FP8_E4M3; want.rank = 2; want.shape[0] = last; want.shape[1] = o.d.i[0]; want.layout = o.d.i[1]; ok = true; }
+      else { want.dtype = MK_F32; want.rank = 2; want.shape[0] = (o.d.i[0] + 127) / 128; want.shape[1] = last / 128; ok = true; }
       break;
     case MK_OP_CONV2D_3X3:
       if (slot == 0) { want.rank = 4; want.shape[0] = o.d.i[0]; want.shape[1] = 3; want.shape[2] = 3; want.shape[3] = last; ok = true; }

@@ -15,7 +15,7 @@ int64_t numel(const mk_tensor_spec& s) {
   for (int i = 0; i < s.rank; ++i) n *= s.shape[i];
   return n;
 }
-size_t dtype_size(int32_t dtype) { return dtype == MK_F32 ? 4 : 2; }
+size_t dtype_size(int32_t dtype) { return dtype == MK_F32 ? 4 : dtype == MK_FP8_E4M3 ? 1 : 2; }
 size_t spec_bytes(const mk_tensor_spec& s) { return (size_t)numel(s) * dtype_size(s.dtype); }
 bool same_spec(const mk_tensor_spec& a, const mk_tensor_spec& b) {
   if (a.dtype != b.dtype || a.rank != b.rank || a.layout != b.layout) return false;
@@ -55,7 +55,7 @@ static mk_tensor_spec make_spec(int32_t dtype, std::initializer_list<int64_t> sh
 }
 
 static int n_inputs_of(const mk_op_desc& d) {
-  if (d.kind == MK_OP_RESIDUAL_ADD) return 2;
+  if (d.kind == MK_OP_RESIDUAL_ADD || d.kind == MK_OP_LINEAR_FP8) return 2;
   if (d.kind == MK_OP_ATTENTION_CAUSAL || d.kind == MK_OP_ATTENTION) return d.i[2] == 0 ? 3 : 1;
   return 1;
 }
@@ -63,11 +63,16 @@ static int n_inputs_of(const mk_op_desc& d) {
 mk_status infer_shapes(Module& m, std::string& err) {
   const int n_in = m.n_inputs;
   if (n_in < 1) { err = "a module needs at least one input"; return MK_ERR_INVALID_ARG; }
-  const int32_t dtype = m.values[0].spec.dtype;
+  // the activations' storage type: that of the inputs; a module with an fp8 input is a bf16 module whose other
+  // inputs may be fp32 (block scales) or bf16
+  bool has_fp8 = false;
+  for (int k = 0; k < n_in; ++k) has_fp8 = has_fp8 || m.values[k].spec.dtype == MK_FP8_E4M3;
+  m.dtype = has_fp8 ? MK_BF16 : m.values[0].spec.dtype;
+  const int32_t dtype = m.dtype;
   for (int k = 0; k < n_in; ++k) {
     const mk_tensor_spec& s = m.values[k].spec;
-    if (s.dtype != MK_F32 && s.dtype != MK_BF16) { err = "input dtype must be MK_F32 or MK_BF16"; return MK_ERR_INVALID_ARG; }
-    if (s.dtype != dtype) { err = "all module inputs must share one dtype"; return MK_ERR_INVALID_ARG; }
+    if (s.dtype != MK_F32 && s.dtype != MK_BF16 && s.dtype != MK_FP8_E4M3) { err = "input dtype must be MK_F32, MK_BF16 or MK_FP8_E4M3"; return MK_ERR_INVALID_ARG; }
+    if (s.dtype != dtype && !has_fp8) { err = "all module inputs must share one dtype"; return MK_ERR_INVALID_ARG; }
     if (s.rank < 1 || s.rank > MK_MAX_RANK) { err = "input rank out of range"; return MK_ERR_INVALID_ARG; }
     if (s.layout != MK_LAYOUT_ROW_MAJOR) { err = "module inputs must be row-major"; return MK_ERR_INVALID_ARG; }
     for (int i = 0; i < s.rank; ++i)
@@ -92,9 +97,22 @@ mk_status infer_shapes(Module& m, std::string& err) {
     y.dtype = dtype;
     // an fp32 value inside a bf16 module (an fp32 residual stream) may only feed a residual add or a row norm
     const bool takes_f32 = d.kind == MK_OP_RESIDUAL_ADD || d.kind == MK_OP_RMSNORM || d.kind == MK_OP_LAYERNORM;
-    for (int k = 0; k < op.n_in; ++k)
-      if (m.values[op.in_id[k]].spec.dtype != dtype && !takes_f32) { err = at + "this operator does not take an fp32 residual-stream value"; return MK_ERR_SHAPE_MISMATCH; }
+    for (int k = 0; k < op.n_in && d.kind != MK_OP_LINEAR_FP8; ++k) {
+      const int32_t vd = m.values[op.in_id[k]].spec.dtype;
+      if (vd == MK_FP8_E4M3) { err = at + "an fp8 value may only feed LINEAR_FP8"; return MK_ERR_SHAPE_MISMATCH; }
+      if (vd != dtype && !takes_f32) { err = at + "this operator does not take an fp32 residual-stream value"; return MK_ERR_SHAPE_MISMATCH; }
+    }
     switch (d.kind) {
+      case MK_OP_LINEAR_FP8: {
+        const mk_tensor_spec& sx = m.values[op.in_id[1]].spec;
+        if (x.rank != 2 || x.dtype != MK_FP8_E4M3) { err = at + "LINEAR_FP8 takes a rank-2 MK_FP8_E4M3 input"; return MK_ERR_SHAPE_MISMATCH; }
+        if (x.shape[1] % 128) { err = at + "LINEAR_FP8 needs K to be a multiple of the 128-element scale block"; return MK_ERR_SHAPE_MISMATCH; }
+        if (sx.rank != 2 || sx.dtype != MK_F32 || sx.shape[0] != x.shape[0] || sx.shape[1] != x.shape[1] / 128) { err = at + "LINEAR_FP8 scales must be MK_F32 [M, K / 128]"; return MK_ERR_SHAPE_MISMATCH; }
+        if (d.i[0] < 1) { err = at + "LINEAR_FP8 needs i[0] = N >= 1"; return MK_ERR_INVALID_ARG; }
+        if (d.i[1] != MK_LAYOUT_ROW_MAJOR && d.i[1] != MK_LAYOUT_TRANSPOSED) { err = at + "LINEAR_FP8 i[1] must be an mk_layout"; return MK_ERR_INVALID_ARG; }
+        y = make_spec(dtype, {x.shape[0], d.i[0]});
+        break;
+      }
       case MK_OP_LINEAR: {
         if (x.rank != 2) { err = at + "LINEAR takes a rank-2 input"; return MK_ERR_SHAPE_MISMATCH; }
         if (d.i[0] < 1) { err = at + "LINEAR needs i[0] = N >= 1"; return MK_ERR_INVALID_ARG; }
@@ -333,9 +351,13 @@ mk_status build_plan(Module& m, const void* const* in_ptrs, void* const* out_ptr
 
   for (int j = 0; j < (int)m.ops.size(); ++j) {
     const Op& op = m.ops[j];
-    const bool need0 = op.d.kind == MK_OP_LINEAR || op.d.kind == MK_OP_CONV2D_3X3 || op.d.kind == MK_OP_BIAS_ADD;
+    const bool need0 = op.d.kind == MK_OP_LINEAR || op.d.kind == MK_OP_CONV2D_3X3 || op.d.kind == MK_OP_BIAS_ADD || op.d.kind == MK_OP_LINEAR_FP8;
     if (need0 && !op.param[0].set) {
       err = "op " + std::to_string(j) + ": parameter 0 has not been set";
+      return MK_ERR_PARAM_MISSING;
+    }
+    if (op.d.kind == MK_OP_LINEAR_FP8 && !op.param[1].set) {
+      err = "op " + std::to_string(j) + ": parameter 1 (the weight scales) has not been set";
       return MK_ERR_PARAM_MISSING;
     }
   }
@@ -374,7 +396,7 @@ mk_status build_plan(Module& m, const void* const* in_ptrs, void* const* out_ptr
 
 mk_status build_epi(const Module& m, int lo, int hi, const Resolved& r, EpiProgram& p, std::string& err) {
   p.n = 0;
-  p.dtype = m.values[0].spec.dtype == MK_F32 ? DT_F32 : DT_BF16;
+  p.dtype = m.dtype == MK_F32 ? DT_F32 : DT_BF16;
   for (int j = lo; j < hi; ++j) {
     const Op& op = m.ops[j];
     if (p.n >= EPI_MAX) { err = "elementwise tail longer than the kernel's program"; return MK_ERR_NO_IMPL; }

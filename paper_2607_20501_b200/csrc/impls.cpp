@@ -13,11 +13,11 @@
 namespace mk {
 namespace {
 
-int dt(const Module& m) { return m.values[0].spec.dtype == MK_F32 ? DT_F32 : DT_BF16; }
+int dt(const Module& m) { return m.dtype == MK_F32 ? DT_F32 : DT_BF16; }
 int dt_of(const mk_tensor_spec& s) { return s.dtype == MK_F32 ? DT_F32 : DT_BF16; }
 // the piece's first input / its output stored in the module's dtype (not an fp32 residual stream)
-bool in_is_module_dtype(const Module& m, int lo) { return m.vspec(m.ops[lo].in_id[0]).dtype == m.values[0].spec.dtype; }
-bool out_is_module_dtype(const Module& m, int hi) { return m.vspec(m.ops[hi - 1].out_id).dtype == m.values[0].spec.dtype; }
+bool in_is_module_dtype(const Module& m, int lo) { return m.vspec(m.ops[lo].in_id[0]).dtype == m.dtype; }
+bool out_is_module_dtype(const Module& m, int hi) { return m.vspec(m.ops[hi - 1].out_id).dtype == m.dtype; }
 
 // ops lo+1.. read their predecessor as first input; nothing but the last value leaves the piece;
 // residual operands come from outside the piece.
@@ -173,7 +173,7 @@ mk_status gemm_simt_emit(const Module& m, int lo, int hi, const Resolved& r, std
 bool gemm_tc_match(const Module& m, int lo, int hi) {
   bool sw; int t;
   if (!gemm_shape(m, lo, hi, &sw, &t)) return false;
-  if (m.values[0].spec.dtype != MK_BF16) return false;
+  if (m.dtype != MK_BF16) return false;
   const Op& op = m.ops[lo];
   if (op.d.i[1] != MK_LAYOUT_TRANSPOSED) return false;
   const int64_t K = m.vspec(op.in_id[0]).shape[1];
@@ -209,6 +209,46 @@ bool gemm_tc2_match(const Module& m, int lo, int hi) {
 }
 mk_status gemm_tc2_emit(const Module& m, int lo, int hi, const Resolved& r, std::vector<Launch>& out, std::string& err) {
   return gemm_tc_emit_impl(m, lo, hi, r, out, err, true);
+}
+
+// LINEAR_FP8 [elementwise]*: block-scaled fp8 contraction (the paper's FP8 MoE inference task), bf16 out
+bool gemm_fp8_shape(const Module& m, int lo, int hi) {
+  return is_chain(m, lo, hi) && m.ops[lo].d.kind == MK_OP_LINEAR_FP8 && all_eltwise(m, lo + 1, hi) && out_is_module_dtype(m, hi) && m.dtype == MK_BF16;
+}
+bool gemm_fp8_simt_match(const Module& m, int lo, int hi) { return gemm_fp8_shape(m, lo, hi); }
+bool gemm_fp8_tc2_match(const Module& m, int lo, int hi) {
+  if (!gemm_fp8_shape(m, lo, hi) || m.ops[lo].d.i[1] != MK_LAYOUT_TRANSPOSED) return false;
+  const mk_tensor_spec& xs = m.vspec(m.ops[lo].in_id[0]);
+  return gemm_fp8_tc2_supported(xs.shape[0], m.ops[lo].d.i[0], xs.shape[1]);
+}
+mk_status gemm_fp8_emit_impl(const Module& m, int lo, int hi, const Resolved& r, std::vector<Launch>& out, std::string& err, bool tc) {
+  EpiProgram p;
+  mk_status st = build_epi(m, lo + 1, hi, r, p, err);
+  if (st != MK_OK) return st;
+  const Op& op = m.ops[lo];
+  const mk_tensor_spec& xs = m.vspec(op.in_id[0]);
+  const int64_t M = xs.shape[0], K = xs.shape[1], N = op.d.i[0];
+  const void* xq = r.value_ptr[op.in_id[0]];
+  const float* sx = (const float*)r.value_ptr[op.in_id[1]];
+  const void* wq = op.param[0].ptr;
+  const float* sw = (const float*)op.param[1].ptr;
+  void* y = r.value_ptr[m.ops[hi - 1].out_id];
+  if (tc) {
+    auto plan = std::make_shared<GemmFp8Plan>();
+    cudaError_t e = gemm_fp8_tc2_plan(plan.get(), xq, sx, wq, sw, y, M, N, K, p, m.ctx->sm_count);
+    if (e != cudaSuccess) { err = std::string("gemm_fp8_tc2 plan: ") + cudaGetErrorString(e); return MK_ERR_CUDA; }
+    out.push_back([plan](cudaStream_t s) { return launch_gemm_fp8_tc2(*plan, s); });
+  } else {
+    const bool wt = op.d.i[1] == MK_LAYOUT_TRANSPOSED;
+    out.push_back([=](cudaStream_t s) { return launch_gemm_fp8_simt(xq, sx, wq, wt, sw, y, M, N, K, p, s); });
+  }
+  return MK_OK;
+}
+mk_status gemm_fp8_tc2_emit(const Module& m, int lo, int hi, const Resolved& r, std::vector<Launch>& out, std::string& err) {
+  return gemm_fp8_emit_impl(m, lo, hi, r, out, err, true);
+}
+mk_status gemm_fp8_simt_emit(const Module& m, int lo, int hi, const Resolved& r, std::vector<Launch>& out, std::string& err) {
+  return gemm_fp8_emit_impl(m, lo, hi, r, out, err, false);
 }
 
 // LINEAR [elementwise]* (LAYERNORM | RMSNORM) on the tensor cores: the norm's statistics come out of the GEMM's
@@ -271,7 +311,7 @@ bool gemm_rownorm_cl_match(const Module& m, int lo, int hi) {
   const int32_t k = m.ops[hi - 1].d.kind;
   if (k != MK_OP_LAYERNORM && k != MK_OP_RMSNORM) return false;
   const Op& op = m.ops[lo];
-  if (op.d.kind != MK_OP_LINEAR || !in_is_module_dtype(m, lo) || m.values[0].spec.dtype != MK_BF16) return false;
+  if (op.d.kind != MK_OP_LINEAR || !in_is_module_dtype(m, lo) || m.dtype != MK_BF16) return false;
   if (op.d.i[1] != MK_LAYOUT_TRANSPOSED || !all_eltwise(m, lo + 1, hi - 1)) return false;
   if (m.vspec(m.ops[hi - 1].out_id).dtype != MK_BF16) return false;
   const mk_tensor_spec& xs = m.vspec(op.in_id[0]);
@@ -304,7 +344,7 @@ bool linear_rownorm_match(const Module& m, int lo, int hi) {
   const int32_t k = m.ops[hi - 1].d.kind;
   if (k != MK_OP_LAYERNORM && k != MK_OP_RMSNORM) return false;
   if (!all_eltwise(m, lo + 1, hi - 1)) return false;
-  if (m.values[0].spec.dtype != MK_F32) return false;
+  if (m.dtype != MK_F32) return false;
   return m.ops[lo].d.i[0] <= 1024;
 }
 mk_status linear_rownorm_emit(const Module& m, int lo, int hi, const Resolved& r, std::vector<Launch>& out, std::string& err) {
@@ -348,7 +388,7 @@ mk_status conv_simt_emit(const Module& m, int lo, int hi, const Resolved& r, std
 
 // tcgen05 implicit GEMM, weights resident in shared memory
 bool conv_tc2_match(const Module& m, int lo, int hi) {
-  if (!conv_simt_match(m, lo, hi) || m.values[0].spec.dtype != MK_BF16) return false;
+  if (!conv_simt_match(m, lo, hi) || m.dtype != MK_BF16) return false;
   const mk_tensor_spec& xs = m.vspec(m.ops[lo].in_id[0]);
   return conv3x3_tc2_supported(xs.shape[0], xs.shape[1], xs.shape[2], xs.shape[3], m.ops[lo].d.i[0]);
 }
@@ -421,7 +461,7 @@ AttnView attn_view(const Module& m, const Op& op, const Resolved& r) {
   AttnView a{};
   a.causal = op.d.kind == MK_OP_ATTENTION_CAUSAL;
   const int64_t H = op.d.i[0], D = op.d.i[1];
-  const size_t es = dtype_size(m.values[0].spec.dtype);
+  const size_t es = dtype_size(m.dtype);
   if (op.d.i[2] == 0) {
     const mk_tensor_spec& q = m.vspec(op.in_id[0]);
     a.q = r.value_ptr[op.in_id[0]];
@@ -441,7 +481,7 @@ AttnView attn_view(const Module& m, const Op& op, const Resolved& r) {
   return a;
 }
 bool attn_tc_match(const Module& m, int lo, int hi) {
-  if (hi - lo != 1 || m.ops[lo].d.kind != MK_OP_ATTENTION_CAUSAL || m.values[0].spec.dtype != MK_BF16) return false;
+  if (hi - lo != 1 || m.ops[lo].d.kind != MK_OP_ATTENTION_CAUSAL || m.dtype != MK_BF16) return false;
   Resolved none;
   none.value_ptr.assign(m.values.size(), nullptr);
   return attention_tc_supported(attn_view(m, m.ops[lo], none));
@@ -456,7 +496,7 @@ mk_status attn_tc_emit(const Module& m, int lo, int, const Resolved& r, std::vec
 }
 bool is_attention(int32_t k) { return k == MK_OP_ATTENTION_CAUSAL || k == MK_OP_ATTENTION; }
 bool attn_tc2_match(const Module& m, int lo, int hi) {
-  if (hi - lo != 1 || !is_attention(m.ops[lo].d.kind) || m.values[0].spec.dtype != MK_BF16) return false;
+  if (hi - lo != 1 || !is_attention(m.ops[lo].d.kind) || m.dtype != MK_BF16) return false;
   Resolved none;
   none.value_ptr.assign(m.values.size(), nullptr);
   return attention_tc2_supported(attn_view(m, m.ops[lo], none));
@@ -491,6 +531,8 @@ const std::vector<Impl>& registry() {
       {"gemm_tc2", gemm_tc2_match, no_scratch, gemm_tc2_emit},
       {"gemm_tc", gemm_tc_match, no_scratch, gemm_tc_emit},
       {"gemm_simt", gemm_simt_match, no_scratch, gemm_simt_emit},
+      {"gemm_fp8_tc2", gemm_fp8_tc2_match, no_scratch, gemm_fp8_tc2_emit},
+      {"gemm_fp8_simt", gemm_fp8_simt_match, no_scratch, gemm_fp8_simt_emit},
       {"conv3x3_gn_tc2", conv_gn_tc2_match, conv_gn_tc2_scratch, conv_gn_tc2_emit},
       {"conv3x3_tc2", conv_tc2_match, no_scratch, conv_tc2_emit},
       {"conv3x3_simt", conv_simt_match, no_scratch, conv_simt_emit},

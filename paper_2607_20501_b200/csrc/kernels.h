@@ -171,6 +171,10 @@ cudaError_t launch_pool_nhwc(int dtype, int mode, const void* x, void* y, int64_
 cudaError_t launch_gemm_simt(int dtype, int out_dtype, const void* a, const void* w, bool w_transposed, void* y,
                              int64_t m, int64_t n, int64_t k, bool swiglu, const EpiProgram& p,
                              cudaStream_t s);
+// Block-scaled fp8 GEMM on the plain ALUs (any m, n; k a multiple of 128): xq [m, k] e4m3, sx [m, k / 128], wq [k, n] or
+// [n, k] when w_transposed, sw [ceil(n / 128), k / 128]; y = program(...) in `dtype` (bf16).
+cudaError_t launch_gemm_fp8_simt(const void* xq, const float* sx, const void* wq, bool w_transposed, const float* sw, void* y, int64_t m,
+                                 int64_t n, int64_t k, const EpiProgram& p, cudaStream_t s);
 // Small-shape fused chain: one CTA owns whole rows, so the row norm follows the GEMM in-kernel.
 // Y = rownorm(program(A @ W)); n <= 1024.
 cudaError_t launch_linear_rownorm_simt(int dtype, const void* a, const void* w, bool w_transposed,

@@ -86,6 +86,7 @@ struct Ctx {
 struct Module {
   Ctx* ctx = nullptr;
   int n_inputs = 0;
+  int32_t dtype = MK_BF16;       // storage type of the activations (MK_F32 or MK_BF16), set by infer_shapes
   std::vector<Op> ops;
   std::vector<Value> values;
   std::vector<int> cuts;         // first op of each submodule

@@ -321,6 +321,21 @@ __device__ __forceinline__ void umma_ss_pair_lohi(uint32_t d_tmem, uint32_t a_lo
       : "memory");
 }
 
+// fp8 (e4m3 x e4m3 -> fp32): kind::f8f6f4, K = 32 per instruction; the instruction descriptor's operand formats are 0 = E4M3
+__host__ __device__ constexpr uint32_t idesc_e4m3_f32(int m, int n) {
+  return (1u << 4) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+__device__ __forceinline__ void umma_fp8_pair_lohi(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "mov.b64 da, {%1, %3};\n\t"
+      "mov.b64 db, {%2, %3};\n\t"
+      "tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], da, db, %4, p;\n\t}" ::"r"(d_tmem),
+      "r"(a_lo), "r"(b_lo), "r"(kDescHiSw128), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
 // ---------------------------------------------------------------- CTA pairs (cluster of 2, cta_group::2)
 __device__ __forceinline__ uint32_t cluster_ctarank() {
   uint32_t r;
@@ -432,6 +447,8 @@ cudaError_t encode_tmap_2d_bf16(CUtensorMap* out, const void* base, uint64_t row
 // General bf16 map: dims/strides innermost first (strides in bytes for dims 1..rank-1).
 cudaError_t encode_tmap_bf16(CUtensorMap* out, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
                              const uint32_t* box, bool swizzle128);
+// 8-bit [rows, cols] tensor (fp8 operands), box [box_rows, 128 bytes], 128-byte swizzle, zero fill out of bounds
+cudaError_t encode_tmap_2d_u8(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows);
 // bf16 [rows, cols] output map for the epilogue's bulk stores: box 32 x 32, 64-byte swizzle
 cudaError_t encode_tmap_2d_bf16_store(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint64_t ld);
 

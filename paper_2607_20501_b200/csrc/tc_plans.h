@@ -82,6 +82,24 @@ cudaError_t launch_gemm_rownorm_cl(const GemmRowNormClPlan& p, cudaStream_t s);
 }  // namespace mk
 
 namespace mk {
+// Block-scaled fp8 GEMM (LINEAR_FP8): y = tail( sum_kb sx[m, kb] * sw[n / 128, kb] * (xq[m, kb-th block] . wq[kb-th block, n]) ), bf16 out.
+struct GemmFp8Plan {
+  CUtensorMap tm_a, tm_b, tm_out;
+  const float* sx = nullptr;   // [m, k / 128]
+  const float* sw = nullptr;   // [ceil(n / 128), k / 128]
+  void* out = nullptr;
+  int m = 0, n = 0, k = 0;
+  int grid = 0;
+  EpiProgram epi;
+};
+// xq [m, k] and wq stored [n, k], both e4m3 bytes; k % 128 == 0, k <= 8192, n % 8 == 0
+bool gemm_fp8_tc2_supported(int64_t m, int64_t n, int64_t k);
+cudaError_t gemm_fp8_tc2_plan(GemmFp8Plan* p, const void* xq, const float* sx, const void* wq_nk, const float* sw, void* y, int64_t m,
+                              int64_t n, int64_t k, const EpiProgram& epi, int sm_count);
+cudaError_t launch_gemm_fp8_tc2(const GemmFp8Plan& p, cudaStream_t s);
+}  // namespace mk
+
+namespace mk {
 struct ConvTcPlan {
   CUtensorMap tm_x, tm_w;
   void* y = nullptr;

@@ -56,6 +56,20 @@ cudaError_t encode_tmap_2d_bf16(CUtensorMap* out, const void* base, uint64_t row
   return encode_tmap_bf16(out, base, 2, dims, strides, box, true);
 }
 
+// 8-bit elements (fp8 operands): [rows, cols] row-major bytes, box [box_rows, 128 bytes], 128-byte swizzle, zero fill.
+cudaError_t encode_tmap_2d_u8(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return cudaErrorNotSupported;
+  if (((uintptr_t)base & 15) != 0 || ld % 16) return cudaErrorInvalidValue;
+  cuuint64_t gdim[2] = {cols, rows};
+  cuuint64_t gstr[1] = {ld};
+  cuuint32_t bdim[2] = {128, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), gdim, gstr, bdim, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
 // Output map for the epilogue's bulk stores: bf16 [rows, cols] row-major, box 32 rows x 32 columns (64 bytes),
 // 64-byte swizzle (the 16-byte segment s of row r sits at segment s ^ ((r >> 1) & 3) in shared memory).
 cudaError_t encode_tmap_2d_bf16_store(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint64_t ld) {

@@ -14,7 +14,7 @@ def to_device(t, device="cuda"):
     """workload Tensor (store = float32 or bf16 bit patterns) -> torch tensor on the device."""
     if t.dtype == "bf16":
         return torch.from_numpy(t.store.view(np.int16)).to(device).view(torch.bfloat16)
-    return torch.from_numpy(t.store).to(device)
+    return torch.from_numpy(t.store).to(device)        # fp32 as float32, fp8 as its bytes (uint8)
 
 
 def to_host_f64(x: torch.Tensor) -> np.ndarray:
@@ -32,15 +32,15 @@ class DeviceWorkload:
         self.dtype = w.dtype
         self.inputs = {k: to_device(t, device) for k, t in w.inputs.items()}
         self.params = {}
-        linear_weights = {op["params"]["w"] for op in w.ops if op["kind"] == "linear"}
+        linear_weights = {op["params"]["w"] for op in w.ops if op["kind"] in ("linear", "linear_fp8")}
         for k, t in w.params.items():
             d = to_device(t, device)
             if k in linear_weights and weight_layout == B.MK_LAYOUT_TRANSPOSED:
                 d = d.t().contiguous()          # storage layout only: [N, K] row-major
             self.params[k] = (d, t.shape)
-        self.module = B.Module(ctx, w.ops, {k: (w.dtype, t.shape) for k, t in w.inputs.items()},
+        self.module = B.Module(ctx, w.ops, {k: (t.dtype, t.shape) for k, t in w.inputs.items()},
                                weight_layout)
-        self.module.set_params(self.params, w.dtype)
+        self.module.set_params(self.params, w.dtype, {k: t.dtype for k, t in w.params.items()})
         out_dt, out_shape, _ = self.module.value_spec(w.ops[-1]["out"])
         self.out = torch.empty(out_shape, dtype=torch.float32 if out_dt == B.MK_F32 else torch.bfloat16, device=device)
         self.ws = None
