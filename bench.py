@@ -42,7 +42,7 @@ NCU_TRAFFIC_BYTES = {"c2": 89.9e6,            # profiles/gemm_tc2_c2.md
                      "c3": 26.25e6,            # profiles/conv3x3_tc2_groupnorm_c3.md (conv; its output stays in L2)
                      "c4": 8 * 52.2e6}         # profiles/attention_tc2_c4.md
 
-DEFAULT_STEPS = {"c1": 2000, "c2": 200, "c3": 400, "c4": 100, "c5": 50, "c6": 100, "c7": 400}
+DEFAULT_STEPS = {"c1": 2000, "c2": 200, "c3": 400, "c4": 100, "c5": 50, "c6": 100, "c7": 400, "c8": 200}
 
 
 def full_workload(name, seed=0, batch=None, only_ops=None):
@@ -52,7 +52,7 @@ def full_workload(name, seed=0, batch=None, only_ops=None):
     kw = {}
     if batch is not None:
         kw = {"c1": {"M": batch}, "c2": {"M": batch}, "c3": {"NB": batch}, "c4": {"B": batch}, "c5": {"B": batch},
-              "c6": {"B": batch}, "c7": {"NB": batch}}[name]
+              "c6": {"B": batch}, "c7": {"NB": batch}, "c8": {"M": batch}}[name]
     w = W.generate.WORKLOADS[name](seed, **kw)
     if only_ops is not None:
         w.ops = w.ops[:only_ops]
@@ -146,6 +146,12 @@ def oracle_sample(name, w, budget_s=12.0):
             s.inputs["x"] = Tensor("x", w.dtype, w.inputs["x"].store[:rows])
             total = w.inputs["x"].shape[0]
             what = f"first {rows} of {total} rows of X"
+        elif name == "c8":
+            rows = frac_units
+            for k in ("xq", "sx"):
+                s.inputs[k] = Tensor(k, w.inputs[k].dtype, w.inputs[k].store[:rows])
+            total = w.inputs["xq"].shape[0]
+            what = f"first {rows} of {total} rows of X"
         elif name in ("c3", "c7"):
             s.inputs["x"] = Tensor("x", w.dtype, w.inputs["x"].store[:frac_units])
             total = w.inputs["x"].shape[0]
@@ -167,7 +173,7 @@ def oracle_sample(name, w, budget_s=12.0):
             what = f"first {frac_units} of {total} batch elements"
         return s, total, what
 
-    probe_units = {"c1": 64, "c2": 64, "c3": 1, "c4": 1, "c5": 1, "c6": 1, "c7": 1}[name]
+    probe_units = {"c1": 64, "c2": 64, "c3": 1, "c4": 1, "c5": 1, "c6": 1, "c7": 1, "c8": 64}[name]
     s, total, _ = sub(probe_units)
     t0 = time.perf_counter()
     OM.run_workload(s, [0])
@@ -205,7 +211,7 @@ def submodule_work(w, module):
                     by += w.params[pn].nbytes()
             _, xs, _ = module.value_spec(op["in"][0])
             _, ys, _ = module.value_spec(op["out"])
-            if op["kind"] == "linear":
+            if op["kind"] in ("linear", "linear_fp8"):
                 fl += 2.0 * xs[0] * xs[1] * op["attrs"]["n"]
             elif op["kind"] == "conv2d_3x3":
                 fl += 2.0 * xs[0] * xs[1] * xs[2] * 9 * xs[3] * op["attrs"]["c_out"]
@@ -258,7 +264,7 @@ NOMINAL = {"bf16_tflops": 2250.0, "hbm_gbs": 8000.0}
 
 
 def roofline_of(name, launches_per_step, dominant, achieved, peak, pk, kernel_ms, t_roof_ms, ms_per_step, min_step_ms,
-                median_step_ms=None, t_roof_nominal_ms=None):
+                median_step_ms=None, t_roof_nominal_ms=None, peak_scale=1.0):
     """Roofline object of the dominant kernel.  A one-launch step is timed directly by the per-step
     event pairs; in a multi-kernel step the dominant kernel's duration comes from the per-submodule
     event pairs of mk_module_profile (mean over its launches)."""
@@ -272,7 +278,7 @@ def roofline_of(name, launches_per_step, dominant, achieved, peak, pk, kernel_ms
         fl = t_roof_ms * 1e-3 * peak      # algorithmic TFLOP of the module when it is tensor-bound
         for key in ("bf16_tflops", "bf16_tflops_sustained"):
             if key in pk:
-                r["module_frac_of_" + ("burst" if key == "bf16_tflops" else "sustained") + "_peak"] = (fl / pk[key]) / (ms_per_step * 1e-3)
+                r["module_frac_of_" + ("burst" if key == "bf16_tflops" else "sustained") + "_peak"] = (fl / (pk[key] * peak_scale)) / (ms_per_step * 1e-3)
     if launches_per_step == 1 or dominant is None:
         r.update({"kernel": "whole step (one launch)", "achieved": achieved, "frac": achieved / peak, "kernel_ms": kernel_ms})
     else:
@@ -548,6 +554,10 @@ def measure_one(name, args, steps, ctx, rank, local, world, cpu_seconds):
         value = world * w.flops / (ms_per_step * 1e-3) / 1e12
         achieved = w.flops / (kernel_ms * 1e-3) / 1e12
         peak = pk["bf16_tflops"] if ms_per_step < 1.0 else pk.get("bf16_tflops_sustained", pk["bf16_tflops"])
+        fp8 = any(t.dtype == "fp8" for t in w.inputs.values())
+        if fp8:
+            # the contraction's own peak: the measured bf16 figure times the nominal fp8 : bf16 ratio of the tensor cores (2)
+            peak *= 2.0
         if w.dtype == "f32":
             # plain fp32 FMA units: 148 SMs x 128 lanes x 2 flop x 1.965 GHz (no fp32 tensor path at this tolerance)
             peak = 148 * 128 * 2 * 1.965e9 / 1e12
@@ -555,7 +565,7 @@ def measure_one(name, args, steps, ctx, rank, local, world, cpu_seconds):
         line = {
             "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
+            "vs_baseline": None, "dtype": "fp8" if fp8 else ("bf16" if w.dtype == "bf16" else "f32"), "data": "synthetic",
             "config": {"workload": name, "decomposition": part, "impls": impls,
                        "l2": (f"rotation over {rot} independent input/output sets ({rot * per_copy / 1e6:.0f} MB > L2)" if rot * per_copy > 126e6 else
                               f"rotation over {rot} independent input/output sets ({rot * per_copy / 1e6:.1f} MB in all: the whole problem is "
@@ -563,9 +573,9 @@ def measure_one(name, args, steps, ctx, rank, local, world, cpu_seconds):
                        "shapes": {k: list(t.shape) for k, t in w.inputs.items()},
                        **({"cut": {"batch": args.batch, "only_ops": args.only_ops}} if (args.batch or args.only_ops) else {})},
             "roofline": roofline_of(name, launches_per_step, dominant, achieved, peak, pk, kernel_ms, t_roof_ms, ms_per_step, step_ms[0],
-                                    median_step_ms=step_ms[len(step_ms) // 2],
+                                    median_step_ms=step_ms[len(step_ms) // 2], peak_scale=2.0 if fp8 else 1.0,
                                     t_roof_nominal_ms=(None if w.dtype == "f32" else
-                                                       max(w.flops / (NOMINAL["bf16_tflops"] * 1e12), w.min_bytes / (NOMINAL["hbm_gbs"] * 1e9)) * 1e3)),
+                                                       max(w.flops / (NOMINAL["bf16_tflops"] * (2 if fp8 else 1) * 1e12), w.min_bytes / (NOMINAL["hbm_gbs"] * 1e9)) * 1e3)),
             "e2e": {"value": world * w.flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms,
                     "pipeline": f"copy in / forward / copy out on three streams over {rot} buffer sets"},
@@ -577,7 +587,7 @@ def measure_one(name, args, steps, ctx, rank, local, world, cpu_seconds):
             line["config"]["timing"] = "CUDA graph replay (step shorter than 0.2 ms; the Python loop's time is kept beside it in `graph`)"
             line["graph"] = graph_info
         if sustained:
-            ps = pk.get("bf16_tflops_sustained", pk["bf16_tflops"]) if w.dtype != "f32" else peak
+            ps = pk.get("bf16_tflops_sustained", pk["bf16_tflops"]) * (2.0 if fp8 else 1.0) if w.dtype != "f32" else peak
             t_roof_s = max(w.flops / (ps * 1e12), w.min_bytes / (pk["hbm_gbs"] * 1e9)) * 1e3
             sustained.update({"value": w.flops / (sustained["ms_per_step"] * 1e-3) / 1e12, "unit": "TFLOP/s", "peak": ps,
                               "module_t_roof_ms": t_roof_s, "module_frac": t_roof_s / sustained["ms_per_step"]})
@@ -645,7 +655,7 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default=None, choices=["all", "c1", "c2", "c3", "c4", "c5", "c6", "c7"],
+    ap.add_argument("--workload", default=None, choices=["all", "c1", "c2", "c3", "c4", "c5", "c6", "c7", "c8"],
                     help="default: all five modules of the workload list for the GPU arm (headline C5), c5 for the reference arm")
     ap.add_argument("--decomposition", default=None)
     ap.add_argument("--batch", type=int, default=None, help="smaller leading batch dimension (profiler captures)")

@@ -197,14 +197,9 @@ gemm_fp8_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         tc::tc_fence_after();
         const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + b * BN + half * 64;
         {
-          uint32_t r0[32];
+          // both chunks in flight at once: a tensor-memory load takes several hundred cycles beside running MMAs
+          uint32_t r0[32], r1[32];
           tc::tmem_ld32(t_row, r0);
-          tc::tmem_ld_wait();
-#pragma unroll
-          for (int j = 0; j < 32; ++j) acc[0][j] = fmaf(__uint_as_float(r0[j]), f, acc[0][j]);
-        }
-        {
-          uint32_t r1[32];
           tc::tmem_ld32(t_row + 32, r1);
           tc::tmem_ld_wait();
           // the buffer is free as soon as its values are in registers
@@ -212,7 +207,10 @@ gemm_fp8_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           __syncwarp();
           if (lane == 0) tc::mbar_arrive_cluster(tc::map_to_cta(tc::smem_u32(&sh->tempty[b]), 0));
 #pragma unroll
-          for (int j = 0; j < 32; ++j) acc[1][j] = fmaf(__uint_as_float(r1[j]), f, acc[1][j]);
+          for (int j = 0; j < 32; ++j) {
+            acc[0][j] = fmaf(__uint_as_float(r0[j]), f, acc[0][j]);
+            acc[1][j] = fmaf(__uint_as_float(r1[j]), f, acc[1][j]);
+          }
         }
       }
       if (!ok) break;
