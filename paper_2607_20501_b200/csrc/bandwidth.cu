@@ -491,6 +491,17 @@ __host__ __device__ inline bool gn_fast_ok(int64_t c) {
   return c % Elem<T>::VEC == 0 && vpp >= 1 && vpp <= GN_THREADS && (GN_THREADS % vpp) == 0 && c <= GN_MAX_C;
 }
 
+// The statistics are sums of differences from a pivot, not of the values themselves: with E[x^2] - mean^2 taken about
+// zero, a group whose mean is fifty standard deviations from zero loses the variance to cancellation in fp32.  The
+// pivot of (image, group) is the group's own first element (first pixel, first channel, after the elementwise
+// prefix): a sample of the data, so (mean - pivot)^2 is of the order of the variance.  Both passes read it from the
+// same address; the partial sums keep their layout.
+template <typename T>
+__device__ __forceinline__ float gn_pivot(const T* __restrict__ x, int64_t img, int64_t hw, int64_t c, int64_t g, int64_t cg, const EpiProgram& pre) {
+  const int64_t r = img * hw, ch = g * cg;
+  return epi_apply(pre, Elem<T>::ld(x + r * c + ch), r, ch, c);
+}
+
 template <typename T>
 __global__ void __launch_bounds__(GN_THREADS) groupnorm_stats_kernel(const T* __restrict__ x, int64_t hw, int c, int groups,
                                                                      const __grid_constant__ EpiProgram pre,
@@ -503,16 +514,17 @@ __global__ void __launch_bounds__(GN_THREADS) groupnorm_stats_kernel(const T* __
   const int vpp = c / VE;
   const int vcol = threadIdx.x % vpp, prow = threadIdx.x / vpp, pstride = GN_THREADS / vpp;
   const int64_t p0 = hw * chunk / chunks, p1 = hw * (chunk + 1) / chunks;
-  float s[VE], q[VE];
+  float s[VE], q[VE], piv[VE];
+  const int cg_ = c / groups;
 #pragma unroll
-  for (int e = 0; e < VE; ++e) { s[e] = 0.0f; q[e] = 0.0f; }
+  for (int e = 0; e < VE; ++e) { s[e] = 0.0f; q[e] = 0.0f; piv[e] = gn_pivot(x, img, hw, c, (vcol * VE + e) / cg_, cg_, pre); }
   for (int64_t pix = p0 + prow; pix < p1; pix += pstride) {
     float v[VE];
     const int64_t r = img * hw + pix;
     ld_vec(x + r * c + vcol * VE, v);
     epi_apply_vec<T, VE>(pre, v, r, (int64_t)vcol * VE, c);
 #pragma unroll
-    for (int e = 0; e < VE; ++e) { s[e] += v[e]; q[e] += v[e] * v[e]; }
+    for (int e = 0; e < VE; ++e) { const float d = v[e] - piv[e]; s[e] += d; q[e] = fmaf(d, d, q[e]); }
   }
 #pragma unroll
   for (int e = 0; e < VE; ++e) {
@@ -552,8 +564,9 @@ __global__ void __launch_bounds__(GN_THREADS) groupnorm_apply_kernel(const T* __
       ts += o[0];
       tq += o[1];
     }
-    const float mean = ts * inv_cnt;
-    const float var = fmaxf(tq * inv_cnt - mean * mean, 0.0f);
+    const float md = ts * inv_cnt;                                   // mean - pivot
+    const float mean = gn_pivot(x, img, hw, c, g, cg, pre) + md;
+    const float var = fmaxf(tq * inv_cnt - md * md, 0.0f);
     const float rstd = rsqrtf(var + eps);
     const float ga = gamma ? Elem<T>::ld(gamma + ch) : 1.0f;
     const float be = beta ? Elem<T>::ld(beta + ch) : 0.0f;
@@ -589,12 +602,13 @@ __global__ void __launch_bounds__(GN_THREADS) groupnorm_stats_generic(const T* _
     __shared__ float sh[32];
     float s = 0.0f, q = 0.0f;
     const int64_t cnt = (p1 - p0) * cg;
+    const float piv = gn_pivot(x, img, hw, c, g, cg, pre);
     for (int64_t i = threadIdx.x; i < cnt; i += GN_THREADS) {
       const int64_t pix = p0 + i / cg, ch = g * cg + i % cg;
       const int64_t r = img * hw + pix;
-      const float v = epi_apply(pre, Elem<T>::ld(x + r * c + ch), r, ch, c);
-      s += v;
-      q += v * v;
+      const float d = epi_apply(pre, Elem<T>::ld(x + r * c + ch), r, ch, c) - piv;
+      s += d;
+      q = fmaf(d, d, q);
     }
     s = block_reduce<0>(s, sh);
     q = block_reduce<0>(q, sh);
@@ -622,8 +636,9 @@ __global__ void __launch_bounds__(GN_THREADS) groupnorm_apply_generic(const T* _
       ts += o[0];
       tq += o[1];
     }
-    const float mean = ts * inv_cnt;
-    const float rstd = rsqrtf(fmaxf(tq * inv_cnt - mean * mean, 0.0f) + eps);
+    const float md = ts * inv_cnt;                                   // mean - pivot
+    const float mean = gn_pivot(x, img, hw, c, g, cg, pre) + md;
+    const float rstd = rsqrtf(fmaxf(tq * inv_cnt - md * md, 0.0f) + eps);
     const int64_t r = img * hw + pix;
     float v = (epi_apply(pre, Elem<T>::ld(x + r * c + ch), r, ch, c) - mean) * rstd;
     if (gamma) v *= Elem<T>::ld(gamma + ch);

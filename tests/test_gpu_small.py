@@ -135,6 +135,27 @@ def test_groupnorm_shapes(ctx, dtype, shape, groups):
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("shape,groups", [((2, 14, 14, 128), 32), ((3, 9, 7, 24), 3), ((1, 30, 30, 64), 8)])
+def test_groupnorm_far_from_zero_mean(ctx, dtype, shape, groups):
+    """Groups whose mean is fifty standard deviations from zero (and of either sign): sums of squares about zero
+    would lose the variance to cancellation in fp32; the kernels sum about a pivot taken from the group itself."""
+    rng = np.random.default_rng(11)
+    c = shape[-1]
+    offs = np.repeat(rng.choice([-50.0, 50.0, 37.5], groups), c // groups)
+    x = (rng.standard_normal(shape) + offs).astype(np.float32)
+    w = _single("groupnorm", x, dtype, {"gamma": 1 + 0.1 * rng.standard_normal(c).astype(np.float32),
+                                        "beta": 0.1 * rng.standard_normal(c).astype(np.float32)},
+                groups=groups, eps=1e-5)
+    ref, _ = oracle(w, [0])
+    _, out = run_gpu(ctx, w, [0])
+    if dtype == "f32":
+        assert_parity(out, ref, dtype)
+    else:
+        # bf16 input: the stored values near 50 carry steps of 0.25, which the oracle sees too; the output tolerance applies
+        assert_parity(out, ref, dtype)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_elementwise_ragged_and_swiglu(ctx, dtype):
     rng = np.random.default_rng(3)
     for rows, cols in ((1, 1), (7, 13), (33, 64), (129, 1000)):
