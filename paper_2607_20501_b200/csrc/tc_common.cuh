@@ -403,6 +403,13 @@ __device__ __forceinline__ void umma_commit_pair_at(uint64_t* bar, uint32_t lead
                "h"((uint16_t)(3u << leader_rank))
                : "memory");
 }
+// The same without release semantics, for hand-backs of TENSOR memory: the reads that must be over are tcgen05.ld
+// (complete after tcgen05.wait::ld, ordered by tcgen05.fence::before_thread_sync), not writes to memory, so the
+// arrival has nothing to publish.  A release at cluster scope costs several hundred cycles; a kernel that hands a
+// buffer back once per K block cannot afford it.
+__device__ __forceinline__ void mbar_arrive_cluster_relaxed(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
