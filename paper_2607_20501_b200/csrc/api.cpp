@@ -366,9 +366,13 @@ mk_status mk_module_forward(mk_module* m, const void* const* in_ptrs, void* cons
   mk_status st = ensure_plan(m, in_ptrs, out_ptrs, workspace, workspace_bytes);
   if (st != MK_OK) return st;
   cudaStream_t s = (cudaStream_t)cuda_stream;
-  for (const Launch& l : m->launches) {
-    cudaError_t e = l(s);
-    if (e != cudaSuccess) return fail(m->ctx, MK_ERR_CUDA, cudaGetErrorString(e));
+  for (size_t q = 0; q < m->launches.size(); ++q) {
+    cudaError_t e = m->launches[q](s);
+    if (e != cudaSuccess) {
+      const int sub = q < m->launch_sub.size() ? m->launch_sub[q] : -1;
+      return fail(m->ctx, MK_ERR_CUDA, "launch " + std::to_string(q) + " (submodule " + std::to_string(sub) + ", " +
+                                           (sub >= 0 && sub < (int)m->bind.size() ? m->bind[sub].name : std::string("?")) + "): " + cudaGetErrorString(e));
+    }
   }
   return MK_OK;
 }

@@ -290,7 +290,7 @@ static cudaError_t rowop_mode(const TI* x, T* y, int64_t rows, int64_t n, const 
     // Measured at 2048-element rows: 8192 rows 18.4 -> 16.4 us with one wave; 32768 rows 47 us with three, 50 with one.
     auto go = [&](auto kernel, ResidentBlocks& rb) -> cudaError_t {
       const int resident = rb.get(kernel, 256);
-      if (resident <= 0) return cudaErrorInvalidDevice;
+      if (resident <= 0) return rb.last_error != cudaSuccess ? rb.last_error : cudaErrorInvalidDevice;
       const int64_t want = ceil_div_i64(rows, 24);
       int64_t grid = 2 * want <= 3 * (int64_t)resident ? resident : (want < 3 * (int64_t)resident ? want : 3 * (int64_t)resident);
       if (sizeof(TI) != sizeof(T)) grid = 148 * 8;   // no prefetch (fp32 in, bf16 out): a row per warp, the block scheduler does the rest

@@ -189,6 +189,13 @@ mk_status infer_shapes(Module& m, std::string& err) {
     m.values[op.out_id].spec = y;
     m.values[op.out_id].producer = j;
   }
+  // Every operator's result must be read by a later operator, except the last one's, which is the module's output:
+  // a value nobody reads would get no buffer, and the kernel that produces it nowhere to write.
+  std::vector<char> used(m.values.size(), 0);
+  for (const Op& op : m.ops)
+    for (int k = 0; k < op.n_in; ++k) used[op.in_id[k]] = 1;
+  for (int j = 0; j + 1 < (int)m.ops.size(); ++j)
+    if (!used[m.ops[j].out_id]) { err = "op " + std::to_string(j) + ": its result is never read and is not the module's output"; return MK_ERR_INVALID_ARG; }
   return MK_OK;
 }
 

@@ -141,13 +141,15 @@ constexpr int RES_SLOT_BYTES = 32 * 64;
 constexpr int RES_RING_BYTES = EPI_WARPS * 2 * RES_SLOT_BYTES;
 static_assert(RES_RING_BYTES <= Cfg<2>::STAGE_BYTES, "the residual ring takes the place of one pipeline stage");
 
-template <int CTAS, bool SWIGLU, bool NORM = false, bool RING = false>
+template <int CTAS, bool SWIGLU, bool NORM = false, bool RING = false, bool PRE = false>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmBh,
                const __grid_constant__ CUtensorMap tmOut, int bulk_store, void* __restrict__ out, int out_f32, int M, int N, int K, int up_row_offset, int tail_first, int group_m,
-               const __grid_constant__ EpiProgram epi_param, const __grid_constant__ RowNormArgs na, unsigned int* status) {
+               const __grid_constant__ EpiProgram epi_param, const __grid_constant__ RowNormArgs na, unsigned int* status,
+               const __grid_constant__ CUtensorMap tmAux, const __grid_constant__ PreNormArgs pn) {
   using C = Cfg<CTAS>;
   static_assert(!RING || (CTAS == 2 && !SWIGLU && !NORM), "the residual ring exists in the plain two-SM form only");
+  static_assert(!PRE || (CTAS == 2 && !NORM && !RING), "the folded pre-norm exists in the plain two-SM form only");
   constexpr int STAGES = C::STAGES - (RING ? 1 : 0);
   constexpr int OUT_N = SWIGLU ? BN / 2 : BN;  // output columns per tile
   extern __shared__ uint8_t smem_raw[];
@@ -378,27 +380,63 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       uint4 res_regs[8];
       ew.load_bias(epi, col_base, nhalf < 0 ? OUT_N : OUT_N / 2, N);
       if (!RING) ew.prefetch_res(epi, rowmap, col_base + half * 32, N, res_regs);
+      float pre_rstd = 1.0f;
+      if (PRE && pn.part_in) {
+        // this lane's row: the partial sums of squares its producer left, read while the accumulator is still filling
+        const int64_t my = row0 + lane;
+        float sq = 0.0f;
+        if (my < M) {
+          const float* pp = pn.part_in + my * pn.slots_in;
+          if ((pn.slots_in & 3) == 0) {
+            for (int k = 0; k < pn.slots_in; k += 4) {
+              const float4 t4 = *reinterpret_cast<const float4*>(pp + k);
+              sq += (t4.x + t4.y) + (t4.z + t4.w);
+            }
+          } else {
+            for (int k = 0; k < pn.slots_in; ++k) sq += pp[k];
+          }
+        }
+        pre_rstd = rsqrtf(sq * pn.inv_n_in + pn.eps_in);
+      }
       ok = tc::mbar_wait(&sh->tfull[acc], (it >> 1) & 1, abort_flag, status, tc::WAIT_TMEM_FULL);
       ok = __all_sync(0xffffffffu, ok ? 1 : 0) != 0;
       if (!ok) break;
       if (threadIdx.x == 64) MK_TR(3 + it * 8);  // epilogue: accumulator ready
       tc::tc_fence_after();
       const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN;
-      float rsum = 0.0f, rsq = 0.0f;   // NORM: this lane's row, over the columns this warp stores
+      float rsum = 0.0f, rsq = 0.0f;   // NORM: this lane's row, over the columns this warp stores (PRE producer: rsq alone)
 #pragma unroll 1
       for (int c = half; c < chunks_here; c += 2) {
         uint32_t r[32];
         float v[32];
+        float gl = 1.0f;               // PRE producer: gamma of column c0 + lane, asked for before the accumulator is read
+        if (PRE && pn.part_out) {
+          const int64_t gc = col_base + c * 32 + lane;
+          if (pn.gamma && gc < N) gl = __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(pn.gamma)[gc]);
+          // the previous chunk's bulk store of xg has finished reading the staging buffer
+          if (lane == 0) tc::tma_store_wait_read();
+          __syncwarp();
+        }
         tc::tmem_ld32(t_row + c * 32, r);
         tc::tmem_ld_wait();
         if (threadIdx.x == 64 && c == half + 2) MK_TR(5 + it * 8);  // epilogue: second chunk in registers
 #pragma unroll
         for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+        if (PRE && pn.part_in) {
+          // consumer of a folded RMSNorm: the row's 1 / rms multiplies the accumulator before anything else
+#pragma unroll
+          for (int j = 0; j < 32; ++j) v[j] *= pre_rstd;
+        }
         if (SWIGLU) {
           tc::tmem_ld32(t_row + BN / 2 + c * 32, r);
           tc::tmem_ld_wait();
+          if (PRE && pn.part_in) {
 #pragma unroll
-          for (int j = 0; j < 32; ++j) v[j] = silu_fast(v[j]) * __uint_as_float(r[j]);
+            for (int j = 0; j < 32; ++j) v[j] = silu_fast(v[j]) * (__uint_as_float(r[j]) * pre_rstd);
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] = silu_fast(v[j]) * __uint_as_float(r[j]);
+          }
         }
         if (RING)
           ew.chunk_out_from(epi, v, rowmap, out, col_base + c * 32, c * 32, (int64_t)N, ring_get, ring_skip, bulk_store ? &tmOut : nullptr, row0);
@@ -413,6 +451,42 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           for (int j = 0; j < 32; ++j)
             if (c0 + j < N) { rsum += v[j]; rsq = fmaf(v[j], v[j], rsq); }
         }
+        if (PRE && pn.part_out) {
+          // producer of a folded RMSNorm: v is the norm's input (after this GEMM's tail).  Its squares go to the row's
+          // partial sum, and xg = bf16(v * gamma) leaves beside the main output, as a bulk tensor store.
+          const int64_t c0 = col_base + c * 32;
+          if (c0 < N) {
+            const int64_t my_row = rowmap(lane);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              if (c0 + j < N) rsq = fmaf(v[j], v[j], rsq);
+              v[j] *= __shfl_sync(0xffffffffu, gl, j);
+            }
+            if (c0 + 32 <= N) {
+              uint4 mine[4];
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {
+                mine[k].x = pack_bf16x2(v[8 * k + 0], v[8 * k + 1]);
+                mine[k].y = pack_bf16x2(v[8 * k + 2], v[8 * k + 3]);
+                mine[k].z = pack_bf16x2(v[8 * k + 4], v[8 * k + 5]);
+                mine[k].w = pack_bf16x2(v[8 * k + 6], v[8 * k + 7]);
+              }
+              // a bf16 main output has just left through the same staging buffer
+              if (lane == 0) tc::tma_store_wait_read();
+              __syncwarp();
+              ew.own_row_to_global_bulk(mine, &tmAux, (int32_t)c0, (int32_t)row0);
+            } else if (my_row >= 0) {
+              __nv_bfloat16* xg = reinterpret_cast<__nv_bfloat16*>(pn.xg);
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (c0 + j < N) xg[my_row * N + c0 + j] = __float2bfloat16_rn(v[j]);
+            }
+          }
+        }
+      }
+      if (PRE && pn.part_out) {
+        const int64_t my = row0 + lane;
+        if (my < M) pn.part_out[my * (2 * num_n) + ni * 2 + half] = rsq;
       }
       tc::tc_fence_before();
       __syncwarp();
@@ -497,6 +571,9 @@ cudaError_t plan_impl(GemmTcPlan* p, const void* a, const void* w_nk, void* y, b
   p->m = (int)m; p->n = (int)n; p->k = (int)k;
   p->swiglu = swiglu;
   p->epi = epi;
+  p->tm_aux = p->tm_a;   // never read unless a folded pre-norm replaces it
+  p->pre = PreNormArgs{};
+  p->use_pre = false;
   const int out_n = swiglu ? BN / 2 : BN;
   const int64_t tiles = ((m + CTAS * BM - 1) / (CTAS * BM)) * ((n + out_n - 1) / out_n);
   const int64_t units = tiles < sm_count / CTAS ? tiles : sm_count / CTAS;
@@ -535,14 +612,26 @@ cudaError_t launch_impl(const GemmTcPlan& p, cudaStream_t s) {
   cudaLaunchConfig_t& cfg = lc.cfg;
   unsigned int* status = kernel_status_ptr();
   const int out_f32 = p.out_f32 ? 1 : 0;
+  if constexpr (CTAS == 2) {
+    if (p.use_pre) {
+      static SmemOptIn opt_in_pre;
+      cudaError_t e1 = opt_in_pre.ensure(Cfg<2>::SMEM, gemm_tc_kernel<2, false, false, false, true>, gemm_tc_kernel<2, true, false, false, true>);
+      if (e1 != cudaSuccess) return e1;
+      if (p.swiglu)
+        return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<2, true, false, false, true>, p.tm_a, p.tm_b, p.tm_b_half, p.tm_out, p.use_tm_out ? 1 : 0, p.out, out_f32, p.m, p.n,
+                                  p.k, p.n, p.tail_first, p.group_m, p.epi, p.norm, status, p.tm_aux, p.pre);
+      return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<2, false, false, false, true>, p.tm_a, p.tm_b, p.tm_b_half, p.tm_out, p.use_tm_out ? 1 : 0, p.out, out_f32, p.m,
+                                p.n, p.k, 0, p.tail_first, p.group_m, p.epi, p.norm, status, p.tm_aux, p.pre);
+    }
+  }
   if (p.swiglu)
     return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<CTAS, true>, p.tm_a, p.tm_b, p.tm_b_half, p.tm_out, p.use_tm_out ? 1 : 0, p.out, out_f32, p.m, p.n, p.k, p.n, p.tail_first, p.group_m, p.epi,
-                              p.norm, status);
+                              p.norm, status, p.tm_aux, p.pre);
   if (CTAS == 2 && p.res_ring)
     return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<2, false, false, true>, p.tm_a, p.tm_b, p.tm_b_half, p.tm_out, p.use_tm_out ? 1 : 0, p.out, out_f32, p.m, p.n, p.k, 0,
-                              p.tail_first, p.group_m, p.epi, p.norm, status);
+                              p.tail_first, p.group_m, p.epi, p.norm, status, p.tm_aux, p.pre);
   return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<CTAS, false>, p.tm_a, p.tm_b, p.tm_b_half, p.tm_out, p.use_tm_out ? 1 : 0, p.out, out_f32, p.m, p.n, p.k, 0, p.tail_first, p.group_m, p.epi,
-                            p.norm, status);
+                            p.norm, status, p.tm_aux, p.pre);
 }
 
 cudaError_t launch_norm_impl(const GemmTcPlan& p, cudaStream_t s) {
@@ -565,7 +654,7 @@ cudaError_t launch_norm_impl(const GemmTcPlan& p, cudaStream_t s) {
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<2, false, true>, p.tm_a, p.tm_b, p.tm_b_half, p.tm_out, 0, p.out, 0, p.m, p.n, p.k, 0, p.tail_first, p.group_m, p.epi, p.norm,
-                            kernel_status_ptr());
+                            kernel_status_ptr(), p.tm_aux, p.pre);
 }
 
 }  // namespace
@@ -592,6 +681,40 @@ cudaError_t gemm_rownorm_tc2_plan(GemmTcPlan* p, const void* a, const void* w_nk
   return cudaSuccess;
 }
 cudaError_t launch_gemm_rownorm_tc2(const GemmTcPlan& p, cudaStream_t s) { return launch_norm_impl(p, s); }
+
+size_t gemm_prenorm_scratch(int64_t m, int64_t n1) {
+  const int64_t num_n = (n1 + BN - 1) / BN;
+  const size_t xg = ((size_t)m * (size_t)n1 * 2 + 255) / 256 * 256;
+  return xg + (size_t)m * (size_t)(2 * num_n) * sizeof(float);
+}
+cudaError_t gemm_prenorm_pair_plan(GemmTcPlan* p1, GemmTcPlan* p2, const void* a, const void* w1_nk, void* y1, bool y1_f32, int64_t m, int64_t n1,
+                                   int64_t k1, const EpiProgram& epi1, const void* gamma, float eps, const void* w2_nk, void* y2, int64_t n2,
+                                   bool swiglu2, const EpiProgram& epi2, void* scratch, int sm_count) {
+  if (!scratch || ((uintptr_t)scratch & 255)) return cudaErrorInvalidValue;
+  cudaError_t e = plan_impl<2>(p1, a, w1_nk, y1, y1_f32, m, n1, k1, false, epi1, sm_count);
+  if (e != cudaSuccess) return e;
+  const int64_t num_n1 = (n1 + BN - 1) / BN;
+  void* xg = scratch;
+  float* part = reinterpret_cast<float*>(reinterpret_cast<char*>(scratch) + ((size_t)m * (size_t)n1 * 2 + 255) / 256 * 256);
+  e = encode_tmap_2d_bf16_store(&p1->tm_aux, xg, (uint64_t)m, (uint64_t)n1, (uint64_t)n1);
+  if (e != cudaSuccess) return e;
+  p1->tail_first = (int)(((m + 2 * BM - 1) / (2 * BM)) * num_n1);   // whole tiles only: one partial-sum slot per (tile column, epilogue half)
+  p1->res_ring = false;
+  p1->use_pre = true;
+  p1->pre.part_out = part;
+  p1->pre.xg = xg;
+  p1->pre.gamma = gamma;
+  e = plan_impl<2>(p2, xg, w2_nk, y2, false, m, n2, n1, swiglu2, epi2, sm_count);
+  if (e != cudaSuccess) return e;
+  p2->tail_first = (int)(((m + 2 * BM - 1) / (2 * BM)) * ((n2 + (swiglu2 ? BN / 2 : BN) - 1) / (swiglu2 ? BN / 2 : BN)));
+  p2->res_ring = false;
+  p2->use_pre = true;
+  p2->pre.part_in = part;
+  p2->pre.slots_in = (int)(2 * num_n1);
+  p2->pre.inv_n_in = 1.0f / (float)n1;
+  p2->pre.eps_in = eps;
+  return cudaSuccess;
+}
 
 cudaError_t gemm_tc_plan(GemmTcPlan* p, const void* a, const void* w_nk, void* y, bool out_f32, int64_t m, int64_t n, int64_t k, bool swiglu,
                          const EpiProgram& epi, int sm_count) {

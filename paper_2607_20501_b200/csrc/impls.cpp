@@ -338,6 +338,75 @@ mk_status gemm_rownorm_cl_emit(const Module& m, int lo, int hi, const Resolved& 
   return MK_OK;
 }
 
+// LINEAR [elementwise]* RMSNORM LINEAR [SWIGLU] [elementwise]* as TWO tensor-core GEMMs and no pass over the
+// activation in between: the paper's fusion across a norm boundary in the form that survives a reduction over the
+// whole row.  The norm's scale 1 / rms is one scalar per row, so it commutes with the second contraction: the first
+// GEMM's epilogue also leaves xg = bf16(x * gamma) and per-row partial sums of x^2, the second takes xg as its A
+// operand and multiplies its accumulator rows by 1 / rms before its own tail.  The value handed to the norm must be
+// needed later anyway (a residual stream): it is the first GEMM's ordinary output.
+bool gemm_prenorm_find(const Module& m, int lo, int hi, int* norm_at, bool* swiglu2, int* tail2_lo) {
+  if (hi - lo < 3 || m.dtype != MK_BF16) return false;
+  int r = -1;
+  for (int j = lo + 1; j < hi; ++j)
+    if (m.ops[j].d.kind == MK_OP_RMSNORM) { r = j; break; }
+  if (r < 0 || r + 1 >= hi) return false;
+  // structure: a chain; only the norm's input may leave the piece early, and it must; the norm's output feeds the second GEMM alone
+  for (int j = lo + 1; j < hi; ++j)
+    if (m.ops[j].in_id[0] != m.ops[j - 1].out_id) return false;
+  for (int j = lo; j < hi - 1; ++j)
+    if (m.escapes(j, lo, hi) != (j == r - 1)) return false;
+  for (int j = lo; j < hi; ++j)
+    if (m.ops[j].d.kind == MK_OP_RESIDUAL_ADD) {
+      const int prod = m.values[m.ops[j].in_id[1]].producer;
+      if (prod >= lo && prod < hi) return false;
+    }
+  const Op& l1 = m.ops[lo];
+  const Op& l2 = m.ops[r + 1];
+  if (l1.d.kind != MK_OP_LINEAR || l2.d.kind != MK_OP_LINEAR || !in_is_module_dtype(m, lo)) return false;
+  if (l1.d.i[1] != MK_LAYOUT_TRANSPOSED || l2.d.i[1] != MK_LAYOUT_TRANSPOSED) return false;
+  if (!all_eltwise(m, lo + 1, r)) return false;
+  int t = r + 2;
+  *swiglu2 = t < hi && m.ops[t].d.kind == MK_OP_SWIGLU;
+  if (*swiglu2) ++t;
+  if (!all_eltwise(m, t, hi) || !out_is_module_dtype(m, hi)) return false;
+  const mk_tensor_spec& xs = m.vspec(l1.in_id[0]);
+  const int64_t M = xs.shape[0], K1 = xs.shape[1], N1 = l1.d.i[0], N2 = last_dim(m.vspec(m.ops[hi - 1].out_id));
+  if (M <= 128 || K1 % 8 || N1 % 8 || N2 % 8) return false;
+  *norm_at = r;
+  *tail2_lo = t;
+  return true;
+}
+bool gemm_prenorm_match(const Module& m, int lo, int hi) {
+  int r, t; bool sw;
+  return gemm_prenorm_find(m, lo, hi, &r, &sw, &t);
+}
+size_t gemm_prenorm_scratch_fn(const Module& m, int lo, int) {
+  return gemm_prenorm_scratch(m.vspec(m.ops[lo].in_id[0]).shape[0], m.ops[lo].d.i[0]);
+}
+mk_status gemm_prenorm_emit(const Module& m, int lo, int hi, const Resolved& r, std::vector<Launch>& out, std::string& err) {
+  int nr, t2; bool sw2;
+  gemm_prenorm_find(m, lo, hi, &nr, &sw2, &t2);
+  EpiProgram p1, p2;
+  mk_status st = build_epi(m, lo + 1, nr, r, p1, err);
+  if (st == MK_OK) st = build_epi(m, t2, hi, r, p2, err);
+  if (st != MK_OK) return st;
+  const Op& l1 = m.ops[lo];
+  const Op& nop = m.ops[nr];
+  const Op& l2 = m.ops[nr + 1];
+  const mk_tensor_spec& xs = m.vspec(l1.in_id[0]);
+  const int64_t M = xs.shape[0], K1 = xs.shape[1], N1 = l1.d.i[0], N2 = last_dim(m.vspec(m.ops[hi - 1].out_id));
+  const int pre = m.ops[nr - 1].out_id;
+  auto plan1 = std::make_shared<GemmTcPlan>();
+  auto plan2 = std::make_shared<GemmTcPlan>();
+  cudaError_t e = gemm_prenorm_pair_plan(plan1.get(), plan2.get(), r.value_ptr[l1.in_id[0]], l1.param[0].ptr, r.value_ptr[pre], m.vspec(pre).dtype == MK_F32,
+                                         M, N1, K1, p1, nop.param[0].set ? nop.param[0].ptr : nullptr, (float)nop.d.f[0], l2.param[0].ptr,
+                                         r.value_ptr[m.ops[hi - 1].out_id], N2, sw2, p2, r.scratch, m.ctx->sm_count);
+  if (e != cudaSuccess) { err = std::string("gemm_prenorm_gemm_tc2 plan: ") + cudaGetErrorString(e); return MK_ERR_CUDA; }
+  out.push_back([plan1](cudaStream_t s) { return launch_gemm_tc2(*plan1, s); });
+  out.push_back([plan2](cudaStream_t s) { return launch_gemm_tc2(*plan2, s); });
+  return MK_OK;
+}
+
 // LINEAR [elementwise]* (LAYERNORM | RMSNORM), fp32, one CTA owns whole rows
 bool linear_rownorm_match(const Module& m, int lo, int hi) {
   if (hi - lo < 2 || !is_chain(m, lo, hi) || m.ops[lo].d.kind != MK_OP_LINEAR) return false;
@@ -526,6 +595,7 @@ mk_status attn_simt_emit(const Module& m, int lo, int, const Resolved& r, std::v
 const std::vector<Impl>& registry() {
   static const std::vector<Impl> reg = {
       {"linear_rownorm_simt", linear_rownorm_match, no_scratch, linear_rownorm_emit},
+      {"gemm_prenorm_gemm_tc2", gemm_prenorm_match, gemm_prenorm_scratch_fn, gemm_prenorm_emit, false},
       {"gemm_rownorm_cl", gemm_rownorm_cl_match, no_scratch, gemm_rownorm_cl_emit, false},
       {"gemm_rownorm_tc2", gemm_rownorm_tc2_match, gemm_rownorm_tc2_scratch_fn, gemm_rownorm_tc2_emit, false},
       {"gemm_tc2", gemm_tc2_match, no_scratch, gemm_tc2_emit},

@@ -67,6 +67,7 @@ struct SmemOptIn {
 // register and shared-memory footprint), asked once per device: the grid size of a persistent launch.
 struct ResidentBlocks {
   std::atomic<int> n[kMaxDevices] = {};
+  cudaError_t last_error = cudaSuccess;   // why get() returned 0
   template <typename K>
   int get(K kernel, int block_threads, size_t dyn_smem = 0) {
     const int dev = current_device();
@@ -74,8 +75,10 @@ struct ResidentBlocks {
     int v = n[dev].load(std::memory_order_acquire);
     if (v > 0) return v;
     int per_sm = 0, sms = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, block_threads, dyn_smem) != cudaSuccess ||
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || per_sm < 1 || sms < 1) {
+    const cudaError_t e1 = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, block_threads, dyn_smem);
+    const cudaError_t e2 = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e1 != cudaSuccess || e2 != cudaSuccess || per_sm < 1 || sms < 1) {
+      last_error = e1 != cudaSuccess ? e1 : e2 != cudaSuccess ? e2 : cudaErrorInvalidConfiguration;
       cudaGetLastError();
       return 0;
     }

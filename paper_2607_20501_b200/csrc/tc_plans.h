@@ -20,8 +20,28 @@ struct RowNormArgs {
   int mode = 0;                // RowMode
 };
 
+// RMSNorm folded across two GEMMs (the norm's reduction blocks fusion into ONE kernel, but not its arithmetic:
+// rstd is a scalar per row, so (rstd x * gamma) W = rstd ((x * gamma) W)).  The GEMM that PRODUCES the norm's input
+// also writes xg = bf16(x * gamma) and, per row and epilogue-warp slot, the sum of x^2 over the columns that warp
+// stored; the GEMM that CONSUMES the norm's output takes xg as its A operand and multiplies every accumulator row
+// by rstd = 1 / sqrt(sum of the row's partials / n + eps) before its own tail.  No pass over the activation is left.
+struct PreNormArgs {
+  // producer side (null: none)
+  float* part_out = nullptr;      // [m][2 * column tiles] sums of squares
+  void* xg = nullptr;             // bf16 [m, n]
+  const void* gamma = nullptr;    // bf16 [n] or null
+  // consumer side (null: none)
+  const float* part_in = nullptr; // [m][slots_in]
+  int slots_in = 0;
+  float inv_n_in = 0.f;           // 1 / (row length of the normalised tensor)
+  float eps_in = 0.f;
+};
+
 struct GemmTcPlan {
   CUtensorMap tm_a, tm_b;
+  CUtensorMap tm_aux;       // producer of a folded pre-norm: store map of xg (never read otherwise)
+  PreNormArgs pre;
+  bool use_pre = false;
   RowNormArgs norm;         // used by the fused GEMM + row norm form only
   CUtensorMap tm_b_half;    // W with a box of half as many rows, for the half-width units of the last wave
   CUtensorMap tm_out;       // bf16 output, for the epilogue's bulk stores (use_tm_out)
@@ -49,6 +69,13 @@ namespace mk {
 cudaError_t gemm_tc2_plan(GemmTcPlan* p, const void* a, const void* w_nk, void* y, bool out_f32, int64_t m, int64_t n, int64_t k, bool swiglu,
                           const EpiProgram& epi, int sm_count);
 cudaError_t launch_gemm_tc2(const GemmTcPlan& p, cudaStream_t s);
+// The pair of GEMMs around a folded RMSNorm (see PreNormArgs).  Scratch: gemm_prenorm_scratch(m, n1) bytes =
+// xg [m, n1] bf16 followed by the partial sums.  First plan: y1 = tail1(A W1) (bf16 or fp32), n1 columns; second:
+// y2 = tail2(swiglu?(rmsnorm(y1; gamma, eps) W2)).
+size_t gemm_prenorm_scratch(int64_t m, int64_t n1);
+cudaError_t gemm_prenorm_pair_plan(GemmTcPlan* p1, GemmTcPlan* p2, const void* a, const void* w1_nk, void* y1, bool y1_f32, int64_t m, int64_t n1,
+                                   int64_t k1, const EpiProgram& epi1, const void* gamma, float eps, const void* w2_nk, void* y2, int64_t n2,
+                                   bool swiglu2, const EpiProgram& epi2, void* scratch, int sm_count);
 // Fused GEMM + tail + row norm (bf16 out).  Scratch: gemm_rownorm_tc2_scratch(m, n) bytes, laid out by the plan.
 size_t gemm_rownorm_tc2_scratch(int64_t m, int64_t n);
 cudaError_t gemm_rownorm_tc2_plan(GemmTcPlan* p, const void* a, const void* w_nk, void* y, int64_t m, int64_t n, int64_t k,

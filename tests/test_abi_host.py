@@ -34,6 +34,14 @@ def test_library_exports_every_declared_symbol():
     assert B.mk_status_str(0) == b"MK_OK" and B.mk_status_str(-3) == b"MK_ERR_NO_IMPL"
 
 
+def test_a_result_nobody_reads_is_rejected(ctx):
+    w = W.c2(0, 16, 8, 8)
+    ops = [dict(o) for o in w.ops]
+    ops[3] = dict(ops[3], **{"in": ["y1"]})              # the scale now skips the GELU: y2 is dead
+    with pytest.raises(MkError):
+        Module(ctx, ops, {k: (w.dtype, t.shape) for k, t in w.inputs.items()})
+
+
 def test_struct_layouts_match_the_header():
     assert C.sizeof(B.mk_tensor_spec) == 4 + 4 + 8 * 4 + 4 + 4
     assert C.sizeof(B.mk_op_desc) == 4 + 12 + 16 + 16
