@@ -500,26 +500,68 @@ def measure_one(name, args, steps, ctx, rank, local, world, cpu_seconds):
         dw.ensure_workspace()
         dw.forward()
         torch.cuda.synchronize()
-        ms = dw.profile(iters=20)
+        ev_ms = dw.profile(iters=20)
+        # The event pairs of mk_module_profile include the gap between two kernels in a stream (several microseconds:
+        # a third of a 20 us row kernel).  Each submodule is therefore also timed ALONE: mk_module_forward_sub of that
+        # submodule, over the rotating buffer sets (their boundary tensors kept from one whole forward each), replayed
+        # back to back from a CUDA graph.  `ms` is that device time; `event_ms` the event-pair figure.
+        n_sub = dw.module.n_sub()
+        for d_ in sets:
+            d_.module.set_decomposition(w.partitions[split_name])
+            d_.module.keep_intermediates(True)
+            d_.ensure_workspace()
+            d_.forward()
+        torch.cuda.synchronize()
+        ms = []
+        bs = torch.cuda.Stream()
+        bs.wait_stream(stream)
+        with torch.cuda.stream(bs):
+            for s_ in range(n_sub):
+                reps_in = max(1, 8 // rot)
+                for d_ in sets:
+                    d_.forward_sub(s_)
+                torch.cuda.synchronize()
+                gsub = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(gsub, stream=bs):
+                    for _ in range(reps_in):
+                        for d_ in sets:
+                            d_.forward_sub(s_)
+                gsub.replay()
+                torch.cuda.synchronize()
+                n_rep = int(max(2, min(50, 2.0 // max(ev_ms[s_] * reps_in * rot, 1e-3))))     # about 2 ms per submodule
+                b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                b0.record(bs)
+                for _ in range(n_rep):
+                    gsub.replay()
+                b1.record(bs)
+                torch.cuda.synchronize()
+                ms.append(b0.elapsed_time(b1) / (n_rep * reps_in * rot))
+                del gsub
+        ctx.check()
         tot = sum(ms)
         work = submodule_work(w, dw.module)
-        rows, agg = [], {}
+        rows, agg, agg_ev = [], {}, {}
         for s_, (t_, (fl, by)) in enumerate(zip(ms, work)):
             impl = dw.module.bound_impl(s_)
+            ae = agg_ev.setdefault(impl, {"ms": 0.0, "flops": 0.0, "bytes": 0.0, "launches": 0})
+            ae["ms"] += ev_ms[s_]; ae["flops"] += fl; ae["bytes"] += by; ae["launches"] += 1
             t_roof = max(fl / (pk_["bf16_tflops"] * 1e12), by / (pk_["hbm_gbs"] * 1e9)) * 1e3
-            rows.append({"sub": s_, "impl": impl, "ms": round(t_, 5), "tflops": round(fl / (t_ * 1e-3) / 1e12, 1),
+            rows.append({"sub": s_, "impl": impl, "ms": round(t_, 5), "event_ms": round(ev_ms[s_], 5), "tflops": round(fl / (t_ * 1e-3) / 1e12, 1),
                          "gbs": round(by / (t_ * 1e-3) / 1e9, 1), "roof_frac": round(t_roof / t_, 3),
                          "bound": "tensor" if fl / (pk_["bf16_tflops"] * 1e12) >= by / (pk_["hbm_gbs"] * 1e9) else "hbm"})
             a = agg.setdefault(impl, {"ms": 0.0, "flops": 0.0, "bytes": 0.0, "launches": 0})
             a["ms"] += t_; a["flops"] += fl; a["bytes"] += by; a["launches"] += 1
-        breakdown = {"decomposition": split_name, "ms_total": tot,
+        breakdown = {"decomposition": split_name, "ms_total": tot, "event_ms_total": sum(ev_ms),
+                     "timing": "each submodule alone (mk_module_forward_sub) by CUDA graph replay over the rotating buffer sets; event_ms: mk_module_profile's event pairs",
                      "share": {k: round(v["ms"] / tot, 4) for k, v in agg.items()},
                      "per_kernel": {k: {"ms": round(v["ms"], 5), "launches": v["launches"],
                                         "tflops": round(v["flops"] / (v["ms"] * 1e-3) / 1e12, 1),
                                         "gbs": round(v["bytes"] / (v["ms"] * 1e-3) / 1e9, 1)} for k, v in agg.items()},
                      "submodules": rows if len(rows) <= 12 else rows[:12]}
-        dk = max(agg, key=lambda k: agg[k]["ms"])
-        dominant = (dk, agg[dk])
+        # the roofline object describes the dominant kernel as it ran INSIDE whole forwards (the event-pair figures, taken
+        # at the clocks of a long step); the per-submodule device times above are short bursts of one kernel alone
+        dk = max(agg_ev, key=lambda k: agg_ev[k]["ms"])
+        dominant = (dk, agg_ev[dk])
         if graph_info:
             # launch-bound module: the split decomposition's step by graph replay too (the fused / split comparison)
             gs = torch.cuda.Stream()

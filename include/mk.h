@@ -295,6 +295,16 @@ MK_API mk_status mk_module_launch_count(mk_module* m, int32_t* n);
 MK_API mk_status mk_module_forward(mk_module* m, const void* const* in_ptrs, void* const* out_ptrs,
                             void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* The same for submodules [first_sub, first_sub + count) alone: their launches of the cached plan, nothing else.
+ * What they read from earlier submodules must already be in the workspace (run a whole forward first, with
+ * mk_module_keep_intermediates on so that no later submodule has reused those ranges).  This is how one subkernel
+ * is evaluated or timed in isolation on the inputs the composition gives it (Methodology, LLMEvolveKernel: every
+ * subkernel is verified and profiled on its own subproblem; Algorithm 2: local checks beside the global one).
+ * Errors: as mk_module_forward; MK_ERR_INVALID_ARG for a range outside the decomposition. */
+MK_API mk_status mk_module_forward_sub(mk_module* m, const void* const* in_ptrs, void* const* out_ptrs,
+                                void* workspace, size_t workspace_bytes, void* cuda_stream,
+                                int32_t first_sub, int32_t count);
+
 /* ---- 5. observability ---------------------------------------------------------------------------
  * profile: runs `iters` forwards with a CUDA event pair around every submodule, synchronises,
  * and writes the mean milliseconds per submodule into ms_per_sub[n_sub].  (Methodology,

@@ -88,6 +88,7 @@ _sig("mk_module_keep_intermediates", C.c_int32, _P, C.c_int32)
 _sig("mk_module_workspace_size", C.c_int32, _P, C.POINTER(C.c_size_t))
 _sig("mk_module_launch_count", C.c_int32, _P, _I32P)
 _sig("mk_module_forward", C.c_int32, _P, _PP, _PP, _P, C.c_size_t, _P)
+_sig("mk_module_forward_sub", C.c_int32, _P, _PP, _PP, _P, C.c_size_t, _P, C.c_int32, C.c_int32)
 _sig("mk_module_profile", C.c_int32, _P, _PP, _PP, _P, C.c_size_t, _P, C.c_int32, C.POINTER(C.c_float))
 _sig("mk_module_swap", C.c_int32, _P, _PP, _PP, _P, C.c_size_t, _P, C.c_int32, C.c_double, C.POINTER(C.c_int32), C.POINTER(C.c_float))
 _sig("mk_module_intermediate", C.c_int32, _P, C.c_int32, _PP, _SPECP)
@@ -335,6 +336,11 @@ class Module:
         ins, outs = self._marshal(inputs, output)
         ws = _ptr(workspace) if workspace is not None else None
         self._ck(mk_module_forward(self.h, ins, outs, ws, workspace_bytes, stream))
+
+    def forward_sub(self, inputs, output, first_sub, count=1, workspace=None, workspace_bytes=0, stream=0):
+        ins, outs = self._marshal(inputs, output)
+        ws = _ptr(workspace) if workspace is not None else None
+        self._ck(mk_module_forward_sub(self.h, ins, outs, ws, workspace_bytes, stream, first_sub, count))
 
     def profile(self, inputs, output, workspace=None, workspace_bytes=0, stream=0, iters=10):
         ins, outs = self._marshal(inputs, output)

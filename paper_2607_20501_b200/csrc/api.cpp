@@ -377,6 +377,22 @@ mk_status mk_module_forward(mk_module* m, const void* const* in_ptrs, void* cons
   return MK_OK;
 }
 
+mk_status mk_module_forward_sub(mk_module* m, const void* const* in_ptrs, void* const* out_ptrs, void* workspace,
+                                size_t workspace_bytes, void* cuda_stream, int32_t first_sub, int32_t count) {
+  mk_status st = ensure_plan(m, in_ptrs, out_ptrs, workspace, workspace_bytes);
+  if (st != MK_OK) return st;
+  if (first_sub < 0 || count < 1 || first_sub + count > m->n_sub()) return fail(m->ctx, MK_ERR_INVALID_ARG, "submodule range outside the decomposition");
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  for (size_t q = 0; q < m->launches.size(); ++q) {
+    const int sub = m->launch_sub[q];
+    if (sub < first_sub || sub >= first_sub + count) continue;
+    cudaError_t e = m->launches[q](s);
+    if (e != cudaSuccess)
+      return fail(m->ctx, MK_ERR_CUDA, "launch " + std::to_string(q) + " (submodule " + std::to_string(sub) + ", " + m->bind[sub].name + "): " + cudaGetErrorString(e));
+  }
+  return MK_OK;
+}
+
 mk_status mk_module_profile(mk_module* m, const void* const* in_ptrs, void* const* out_ptrs, void* workspace,
                             size_t workspace_bytes, void* cuda_stream, int32_t iters, float* ms_per_sub) {
   if (!ms_per_sub || iters < 1) return MK_ERR_INVALID_ARG;

@@ -60,6 +60,14 @@ class DeviceWorkload:
                             self.ws_bytes, s)
         return self.out
 
+    def forward_sub(self, first_sub, count=1, stream=None):
+        """Submodules [first_sub, first_sub + count) alone, on what an earlier whole forward left in the workspace."""
+        self.ensure_workspace()
+        s = torch.cuda.current_stream().cuda_stream if stream is None else stream
+        self.module.forward_sub([self.inputs[k] for k in self.module.input_names], self.out, first_sub, count, self.ws,
+                                self.ws_bytes, s)
+        return self.out
+
     def swap(self, iters=5, tau=0.9):
         """Rebind submodules that run slower than tau x their fastest alternative (the output tensor is
         overwritten with the result of the final composition)."""

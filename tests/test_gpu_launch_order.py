@@ -55,3 +55,4 @@ def test_dependent_launch_and_plain_stream_order_agree_bit_for_bit():
     b = _run(no_pdl=True)
     assert set(a) == {"c3", "c4", "c6"}
     assert a == b
+
