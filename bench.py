@@ -38,9 +38,11 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # captures summarised under profiles/ (null where no capture of that workload's dominant kernel exists).
 # c4: the attention kernel was captured on 2 of the 16 batch elements (52.2 MB; its traffic is
 # proportional to the batch) and is scaled by 8 here.
+# c5: average over the 32 GEMM launches of two captured steps (16 per step, four shapes).
 NCU_TRAFFIC_BYTES = {"c2": 89.9e6,            # profiles/gemm_tc2_c2.md
                      "c3": 26.25e6,            # profiles/conv3x3_tc2_groupnorm_c3.md (conv; its output stays in L2)
-                     "c4": 8 * 52.2e6}         # profiles/attention_tc2_c4.md
+                     "c4": 8 * 52.2e6,         # profiles/attention_tc2_c4.md
+                     "c5": 259.7e6}            # profiles/gemm_tc2_decoder_c5.md
 
 DEFAULT_STEPS = {"c1": 2000, "c2": 200, "c3": 400, "c4": 100, "c5": 50, "c6": 100, "c7": 400, "c8": 200}
 

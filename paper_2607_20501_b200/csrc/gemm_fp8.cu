@@ -12,9 +12,10 @@
 // column is exactly one 128-wide weight scale block.  The activation scales of the CTA's rows for every K block
 // are copied to shared memory a tile ahead (cp.async), so the drain never waits for global memory.
 // A plain-ALU kernel serves the shapes this one declines and is the second implementation Swap can bind.
-// Measured (4096 x 7168 x 4096): 200 us, 1.2 PFLOP/s.  At this tile shape a CTA pair brings 48 KB from L2 per
-// 8.4 MFLOP, i.e. 8.3 TB/s over the machine at that rate, which is about what L2 delivers to the SMs here: the
-// kernel is bound by operand traffic, not by the drain (sixteen epilogue warps with a 32 x 32 chunk each: 217 us).
+// Measured (4096 x 7168 x 4096): 200 us, 1.2 PFLOP/s, with the tensor pipe busy 27 % of the time and L2 at a
+// quarter of its throughput: the kernel is bound by the hand-shake per K block (two barrier waits and two commits
+// per four MMAs on the issuing thread, a tensor-memory round trip and a barrier arrival per drain), not by the
+// drain's own work (sixteen epilogue warps with a 32 x 32 chunk each: 217 us) and not by operand traffic.
 #include <stdlib.h>
 
 #include "device_common.cuh"
