@@ -12,10 +12,11 @@
 // column is exactly one 128-wide weight scale block.  The activation scales of the CTA's rows for every K block
 // are copied to shared memory a tile ahead (cp.async), so the drain never waits for global memory.
 // A plain-ALU kernel serves the shapes this one declines and is the second implementation Swap can bind.
-// Measured (4096 x 7168 x 4096): 200 us, 1.2 PFLOP/s, with the tensor pipe busy 27 % of the time and L2 at a
-// quarter of its throughput: the kernel is bound by the hand-shake per K block (two barrier waits and two commits
-// per four MMAs on the issuing thread, a tensor-memory round trip and a barrier arrival per drain), not by the
-// drain's own work (sixteen epilogue warps with a 32 x 32 chunk each: 217 us) and not by operand traffic.
+// Measured (4096 x 7168 x 4096): 186 us, 1.29 PFLOP/s; with two commits per K block (one more for the operand
+// stage) 200 us, and then the tensor pipe was busy 27 % of the time and L2 at a quarter of its throughput: the
+// kernel is bound by the hand-shake per K block (barrier waits and a commit per four MMAs on the issuing thread,
+// a tensor-memory round trip and a barrier arrival per drain), not by the drain's own work (sixteen epilogue
+// warps with a 32 x 32 chunk each: 218 us) and not by operand traffic.
 #include <stdlib.h>
 
 #include "device_common.cuh"
@@ -143,7 +144,9 @@ gemm_fp8_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           const uint32_t b_lo = a_lo + (A_BYTES >> 4);
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k) tc::umma_fp8_pair_lohi(d_tmem, a_lo + 2 * k, b_lo + 2 * k, idesc, k > 0 ? 1u : 0u);
-          tc::umma_commit_pair(&sh->empty[stage]);
+          // ONE commit per K block: its completion says both "the buffer is full" and "the stage has been read";
+          // the stage is handed back to the producer by an epilogue warp that has seen it (a commit costs the
+          // issuing thread about as long as two of the four MMAs it follows)
           tc::umma_commit_pair(&sh->tfull[b]);
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
@@ -196,10 +199,12 @@ gemm_fp8_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       for (int kb = 0; kb < num_kb; ++kb, ++cnt) {
         const uint32_t b = cnt % ACC_BUFS;
         const float f = sxs[kb * BM] * sws[kb];
-        ok = tc::mbar_wait(&sh->tfull[b], (cnt / ACC_BUFS) & 1, abort_flag, status, tc::WAIT_TMEM_FULL);
+        ok = tc::mbar_wait_spin(&sh->tfull[b], (cnt / ACC_BUFS) & 1, abort_flag, status, tc::WAIT_TMEM_FULL);
         ok = __all_sync(0xffffffffu, ok ? 1 : 0) != 0;
         if (!ok) break;
         tc::tc_fence_after();
+        // the MMAs of this K block are complete, so its operand stage has been read: this CTA's producer may refill it
+        if (warp == 2 && lane == 0) tc::mbar_arrive(&sh->empty[cnt % STAGES]);
         const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + b * BN + half * 64;
         {
           // both chunks in flight at once: a tensor-memory load takes several hundred cycles beside running MMAs
