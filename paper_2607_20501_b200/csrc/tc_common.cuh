@@ -271,13 +271,6 @@ __device__ __forceinline__ unsigned long long gtime() {
 #define MK_TR_PRINT(tag) do {} while (0)
 #endif
 
-// L2 prefetch of a 4-D tensor-map box: no shared memory, no barrier; a later load of the same box hits L2.
-__device__ __forceinline__ void tma_prefetch_4d(const CUtensorMap* m, int32_t c0, int32_t c1, int32_t c2, int32_t c3) {
-  asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global.tile [%0, {%1, %2, %3, %4}];" ::"l"(reinterpret_cast<uint64_t>(m)), "r"(c0), "r"(c1),
-               "r"(c2), "r"(c3)
-               : "memory");
-}
-
 // ---------------------------------------------------------------- asynchronous 16-byte copies (global -> shared)
 // Per-thread copies that need no register for the data in flight; completion is tracked per thread in commit
 // groups, so other lanes see the bytes only after the issuing lane's wait and a warp barrier.
@@ -458,5 +451,6 @@ cudaError_t encode_tmap_bf16(CUtensorMap* out, const void* base, int rank, const
 cudaError_t encode_tmap_2d_u8(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows);
 // bf16 [rows, cols] output map for the epilogue's bulk stores: box 32 x 32, 64-byte swizzle
 cudaError_t encode_tmap_2d_bf16_store(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint64_t ld);
+cudaError_t encode_tmap_2d_f32_store(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint64_t ld);
 
 }  // namespace mk

@@ -231,8 +231,8 @@ struct EpiWarp {
   //   bias_off     offset (elements) of col0 inside the bias slice loaded by load_bias
   //   rowmap(r)    global row of warp-local row r in [0, 32), or -1 if that row is not stored
   //   res_regs     this chunk's residual (from prefetch_res); on return the next chunk's, if next_col0 >= 0
-  //   tm_store     if not null (bf16 output, rows of the warp consecutive from global row y0): the block leaves by a
-  //                bulk tensor store instead of 16-byte stores
+  //   tm_store     if not null (a map of the output in its own type, rows of the warp consecutive from global row y0):
+  //                the block leaves by bulk tensor stores (one for bf16, two for fp32) instead of 16-byte stores
   template <typename RowMap>
   __device__ __forceinline__ void chunk_out(const EpiProgram& epi, float (&v)[32], RowMap rowmap, void* __restrict__ out_v, int64_t col0,
                                             int bias_off, int64_t n_cols, uint4 (&res_regs)[8], int64_t next_col0,
@@ -289,15 +289,23 @@ struct EpiWarp {
         if (tm_store) own_row_to_global_bulk(mine, tm_store, (int32_t)col0, (int32_t)y0);
         else own_row_to_global(mine, rowmap, out, n_cols * 2, col0 * 2);
       } else {
+        // an fp32 chunk is two 64-byte slabs per row
 #pragma unroll
         for (int j = 0; j < 4; ++j)
           mine[j] = make_uint4(__float_as_uint(v[4 * j]), __float_as_uint(v[4 * j + 1]), __float_as_uint(v[4 * j + 2]), __float_as_uint(v[4 * j + 3]));
-        own_row_to_global(mine, rowmap, out, n_cols * 4, col0 * 4);
+        if (tm_store) own_row_to_global_bulk(mine, tm_store, (int32_t)col0, (int32_t)y0);
+        else own_row_to_global(mine, rowmap, out, n_cols * 4, col0 * 4);
 #pragma unroll
         for (int j = 0; j < 4; ++j)
           mine[j] = make_uint4(__float_as_uint(v[16 + 4 * j]), __float_as_uint(v[16 + 4 * j + 1]), __float_as_uint(v[16 + 4 * j + 2]),
                                __float_as_uint(v[16 + 4 * j + 3]));
-        own_row_to_global(mine, rowmap, out, n_cols * 4, col0 * 4 + 64);
+        if (tm_store) {
+          if (lane == 0) tc::tma_store_wait_read();   // the first slab has left the staging buffer
+          __syncwarp();
+          own_row_to_global_bulk(mine, tm_store, (int32_t)col0 + 16, (int32_t)y0);
+        } else {
+          own_row_to_global(mine, rowmap, out, n_cols * 4, col0 * 4 + 64);
+        }
       }
     } else {
       // ragged last chunk of the row: element by element, operands from global memory

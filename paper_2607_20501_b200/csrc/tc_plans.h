@@ -44,7 +44,7 @@ struct GemmTcPlan {
   bool use_pre = false;
   RowNormArgs norm;         // used by the fused GEMM + row norm form only
   CUtensorMap tm_b_half;    // W with a box of half as many rows, for the half-width units of the last wave
-  CUtensorMap tm_out;       // bf16 output, for the epilogue's bulk stores (use_tm_out)
+  CUtensorMap tm_out;       // the output in its own type (bf16 or fp32), for the epilogue's bulk stores (use_tm_out)
   bool use_tm_out = false;
   bool res_ring = false;    // a bf16 residual is staged through shared memory two chunks ahead (one pipeline stage less)
   int tail_first = 0;       // tiles from this index on run as two half-width units (= tile count: none)
