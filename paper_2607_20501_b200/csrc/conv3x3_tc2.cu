@@ -45,9 +45,10 @@ constexpr int BIAS_BYTES = 512;           // one copy of the bias (C_out <= 256 
 // The timeline of -DMK_TRACE builds lives in global memory here: this kernel leaves no shared memory for it.
 #ifdef MK_TRACE
 __device__ unsigned long long conv_tr[96];
-#define CTR_INIT do { if (blockIdx.x == 0 && threadIdx.x == 0) { for (int i_ = 0; i_ < 96; ++i_) conv_tr[i_] = 0; conv_tr[0] = tc::gtime(); } } while (0)
+__device__ long long conv_clk0;
+#define CTR_INIT do { if (blockIdx.x == 0 && threadIdx.x == 0) { for (int i_ = 0; i_ < 96; ++i_) conv_tr[i_] = 0; conv_tr[0] = tc::gtime(); conv_clk0 = clock64(); } } while (0)
 #define CTR(slot) do { if (blockIdx.x == 0 && (slot) < 96) conv_tr[slot] = tc::gtime(); } while (0)
-#define CTR_PRINT do { __threadfence(); __syncthreads(); if (blockIdx.x == 0 && threadIdx.x == 0) { printf("conv end=%llu :", tc::gtime() - conv_tr[0]); \
+#define CTR_PRINT do { __threadfence(); __syncthreads(); if (blockIdx.x == 0 && threadIdx.x == 0) { printf("conv end=%llu cycles=%lld :", tc::gtime() - conv_tr[0], clock64() - conv_clk0); \
     for (int i_ = 1; i_ < 96; ++i_) if (conv_tr[i_]) printf(" [%d]%llu", i_, conv_tr[i_] - conv_tr[0]); printf("\n"); } } while (0)
 #else
 #define CTR_INIT do {} while (0)
@@ -65,27 +66,6 @@ struct Shared {
   int abort_flag;
   EpiProgram epi;   // the kernel parameter, copied once (see epi_copy_to_smem)
 };
-
-// 32 rows x 64 bytes from "one row per lane" to coalesced global stores (8 rows x 64 contiguous bytes per
-// instruction).  The 16-byte segment s of row r sits at segment s ^ ((r >> 1) & 3): both the row-wise
-// writes and the 8-lanes-per-two-rows reads then touch every bank group once.
-template <typename RowMap>
-__device__ __forceinline__ void store_rows64(uint8_t* stg, int lane, const uint4 (&mine)[4], RowMap rowmap, uint8_t* out, int64_t row_bytes,
-                                             int64_t byte_off) {
-  const int f = (lane >> 1) & 3;
-#pragma unroll
-  for (int sgm = 0; sgm < 4; ++sgm) *reinterpret_cast<uint4*>(stg + lane * 64 + ((sgm ^ f) * 16)) = mine[sgm];
-  __syncwarp();
-  const int sub_row = lane >> 2, seg = lane & 3;
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const int r = sub_row + 8 * i;
-    const int64_t gr = rowmap(r);
-    const uint4 val = *reinterpret_cast<const uint4*>(stg + r * 64 + ((seg ^ ((r >> 1) & 3)) * 16));
-    if (gr >= 0) *reinterpret_cast<uint4*>(out + gr * row_bytes + byte_off + seg * 16) = val;
-  }
-  __syncwarp();
-}
 
 // Sum over the warp's 32 rows of N per-lane values, N a power of two: each step halves the number of
 // values a lane carries (it keeps one half and receives the partner's other half), so N values cost N
@@ -154,7 +134,7 @@ __device__ __forceinline__ void umma_ss_pair_x4(uint32_t d_tmem, uint64_t a_desc
 // CB = C_in / 64 channel blocks
 template <int CB>
 __global__ void __launch_bounds__(THREADS, 1)
-conv3x3_tc2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW, __nv_bfloat16* __restrict__ y,
+conv3x3_tc2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmY,
                    int NB, int H, int W, int C_OUT, const __grid_constant__ EpiProgram epi_param, float* __restrict__ stats, int cpg,
                    unsigned int* status) {
   extern __shared__ uint8_t smem_raw[];
@@ -187,6 +167,7 @@ conv3x3_tc2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     tc::fence_barrier_init();
     tc::tma_prefetch_desc(&tmX);
     tc::tma_prefetch_desc(&tmW);
+    tc::tma_prefetch_desc(&tmY);
   }
   if (warp == 1) tc::tmem_alloc_pair(&sh->tmem_base, 512);
   tc::tc_fence_before();
@@ -254,6 +235,7 @@ conv3x3_tc2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
         ok = tc::mbar_wait(&sh->tempty[acc], ((it >> 1) & 1) ^ 1, abort_flag, status, tc::WAIT_TMEM_EMPTY);
         if (!ok) break;
         tc::tc_fence_after();
+        if (it > 0) CTR(it * 8);               // MMA: accumulator free
         uint32_t accumulate = 0;
 #pragma unroll
         for (int cb = 0; cb < CB; ++cb) {
@@ -347,7 +329,21 @@ conv3x3_tc2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
           mine[k].z = pack_bf16x2(v[8 * k + 4], v[8 * k + 5]);
           mine[k].w = pack_bf16x2(v[8 * k + 6], v[8 * k + 7]);
         }
-        store_rows64(stg, lane, mine, rowmap, reinterpret_cast<uint8_t*>(y), (int64_t)C_OUT * 2, (int64_t)c * 64);
+        // the lane's own 64 bytes into the staging buffer (64-byte swizzle), then one bulk tensor store of the
+        // 32 pixels x 32 channels; pixels past the end of the image row are clipped by the copy engine
+        if (lane == 0) tc::tma_store_wait_read();   // the previous chunk's store has finished reading the buffer
+        __syncwarp();
+        {
+          const int f = (lane >> 1) & 3;
+#pragma unroll
+          for (int sgm = 0; sgm < 4; ++sgm) *reinterpret_cast<uint4*>(stg + lane * 64 + ((sgm ^ f) * 16)) = mine[sgm];
+        }
+        tc::fence_proxy_async();
+        __syncwarp();
+        if (lane == 0 && row_ok && w0 < W) {
+          tc::tma_store_4d(&tmY, stg, c * 32, w0, h, n);
+          tc::tma_store_commit();
+        }
       }
       tc::tc_fence_before();
       __syncwarp();
@@ -356,6 +352,7 @@ conv3x3_tc2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     }
   }
 
+  if (warp >= 2 && lane == 0) tc::tma_store_wait_all();   // this warp's bulk stores are complete before the CTA retires
   CTR_PRINT;
   if (*abort_flag) {
     const long long t0 = clock64();
@@ -397,6 +394,8 @@ cudaError_t conv3x3_tc2_plan(ConvTcPlan* p, const void* x, const void* w, void* 
   }
   cudaError_t e = encode_tmap_2d_bf16(&p->tm_w, w, (uint64_t)c_out, (uint64_t)(9 * c_in), (uint64_t)(9 * c_in), (uint32_t)(c_out / 2), 64);
   if (e != cudaSuccess) return e;
+  e = encode_tmap_nhwc_bf16_store(&p->tm_y, y, (uint64_t)nb, (uint64_t)h, (uint64_t)wd, (uint64_t)c_out);
+  if (e != cudaSuccess) return e;
   p->y = y;
   p->stats = nullptr;
   p->cpg = 0;
@@ -418,9 +417,8 @@ cudaError_t launch_conv3x3_tc2(const ConvTcPlan& p, cudaStream_t s) {
   LaunchCfg lc(PDL_CONV, dim3((unsigned)p.grid), dim3(THREADS), p.smem, s, 2);
   cudaLaunchConfig_t& cfg = lc.cfg;
   unsigned int* status = kernel_status_ptr();
-  __nv_bfloat16* y = (__nv_bfloat16*)p.y;
-  if (p.c_in == 64) return cudaLaunchKernelEx(&cfg, conv3x3_tc2_kernel<1>, p.tm_x, p.tm_w, y, p.nb, p.h, p.w, p.c_out, p.epi, p.stats, p.cpg, status);
-  return cudaLaunchKernelEx(&cfg, conv3x3_tc2_kernel<2>, p.tm_x, p.tm_w, y, p.nb, p.h, p.w, p.c_out, p.epi, p.stats, p.cpg, status);
+  if (p.c_in == 64) return cudaLaunchKernelEx(&cfg, conv3x3_tc2_kernel<1>, p.tm_x, p.tm_w, p.tm_y, p.nb, p.h, p.w, p.c_out, p.epi, p.stats, p.cpg, status);
+  return cudaLaunchKernelEx(&cfg, conv3x3_tc2_kernel<2>, p.tm_x, p.tm_w, p.tm_y, p.nb, p.h, p.w, p.c_out, p.epi, p.stats, p.cpg, status);
 }
 
 }  // namespace mk

@@ -138,6 +138,11 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* m, const void* s
                "r"(smem_u32(src)), "r"(x), "r"(y)
                : "memory");
 }
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap* m, const void* src, int32_t c0, int32_t c1, int32_t c2, int32_t c3) {
+  asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];" ::"l"(reinterpret_cast<uint64_t>(m)),
+               "r"(smem_u32(src)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+               : "memory");
+}
 __device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
@@ -451,6 +456,7 @@ cudaError_t encode_tmap_bf16(CUtensorMap* out, const void* base, int rank, const
 cudaError_t encode_tmap_2d_u8(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows);
 // bf16 [rows, cols] output map for the epilogue's bulk stores: box 32 x 32, 64-byte swizzle
 cudaError_t encode_tmap_2d_bf16_store(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint64_t ld);
+cudaError_t encode_tmap_nhwc_bf16_store(CUtensorMap* out, const void* base, uint64_t nb, uint64_t h, uint64_t w, uint64_t c);
 cudaError_t encode_tmap_2d_f32_store(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint64_t ld);
 
 }  // namespace mk

@@ -129,6 +129,7 @@ cudaError_t launch_gemm_fp8_tc2(const GemmFp8Plan& p, cudaStream_t s);
 namespace mk {
 struct ConvTcPlan {
   CUtensorMap tm_x, tm_w;
+  CUtensorMap tm_y;         // the output, for the epilogue's bulk stores
   void* y = nullptr;
   // optional GroupNorm partial sums of the stored output: float [nb][conv3x3_tc2_stat_slots(h)][c_out / cpg][2]
   // = (sum, sum of squares) per group of cpg adjacent channels (cpg in {4, 8, 16, 32}); null: none
