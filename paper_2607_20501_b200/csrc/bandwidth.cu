@@ -2,6 +2,7 @@
 // NHWC GroupNorm.  All global traffic is 128-bit wide on the vector paths; statistics are fp32;
 // rows stay in registers between the reduction and the normalising pass, so each element is read
 // once and written once.
+#include <stdlib.h>
 #include "device_common.cuh"
 
 namespace mk {
@@ -469,9 +470,22 @@ cudaError_t launch_pool_nhwc(int dtype, int mode, const void* x, void* y, int64_
 // pass that reduces the partials (a few dozen values) and normalises.
 // scratch layout: float [nb][chunks][groups][2] = (sum, sum of squares)
 // =====================================================================================================
+constexpr int GN_THREADS = 256;
+constexpr int GN_MAX_C = 2048;
+#ifndef MK_GN_RESIDENT
+#define MK_GN_RESIDENT 2
+#endif
+constexpr int GN_RESIDENT = MK_GN_RESIDENT;
+#ifndef MK_GN_UN
+#define MK_GN_UN 8
+#endif
+constexpr int GN_UN = MK_GN_UN;               // independent 16-byte loads per thread and batch   // CTAs per SM the two-pass kernels are compiled for
+
 int groupnorm_chunks(int64_t nb, int64_t hw, int sm_count) {
-  // enough CTAs to fill the machine twice over, at least 32 pixels each
-  int64_t want = (2 * (int64_t)sm_count + nb - 1) / nb;
+  // as many CTAs as are resident at once (GN_RESIDENT per SM: both kernels are built for it), never one more: a
+  // CTA walks its pixels in a few dependent batches, so a second, nearly empty wave would double the kernel's time;
+  // at least 32 pixels each
+  int64_t want = (GN_RESIDENT * (int64_t)sm_count) / nb;
   int64_t maxc = hw / 32 > 0 ? hw / 32 : 1;
   int64_t c = want < 1 ? 1 : want;
   if (c > maxc) c = maxc;
@@ -482,8 +496,6 @@ size_t groupnorm_scratch_bytes(int64_t nb, int64_t hw, int64_t, int groups, int 
   return (size_t)nb * groupnorm_chunks(nb, hw, sm_count) * groups * 2 * sizeof(float);
 }
 
-constexpr int GN_THREADS = 256;
-constexpr int GN_MAX_C = 2048;
 
 template <typename T>
 __host__ __device__ inline bool gn_fast_ok(int64_t c) {
@@ -502,8 +514,59 @@ __device__ __forceinline__ float gn_pivot(const T* __restrict__ x, int64_t img, 
   return epi_apply(pre, Elem<T>::ld(x + r * c + ch), r, ch, c);
 }
 
+// A thread's walk over its 16-byte vectors (one per pixel row of the thread grid): batches of UN independent loads,
+// the next batch asked for before the current one is used, pointers advanced by a fixed stride, no per-load
+// bounds test.  f(raw, i) receives the i-th vector of the walk.  These kernels are issue-bound before they are
+// bandwidth-bound (a profile of the first form showed 94 warp instructions per vector, a third of all issue slots
+// taken, 1.7 TB/s), so the loop carries nothing but the loads and the arithmetic.
+template <int UN, typename F>
+__device__ __forceinline__ void walk16(const uint4* __restrict__ ptr, size_t step, int n, F f) {
+  int i = 0;
+  uint4 cur[UN];
+  if (n >= UN) {
+#pragma unroll
+    for (int u = 0; u < UN; ++u) cur[u] = ptr[u * step];
+  }
+  for (; i + UN <= n; i += UN) {
+    uint4 nxt[UN];
+    const bool more = i + 2 * UN <= n;
+    if (more) {
+#pragma unroll
+      for (int u = 0; u < UN; ++u) nxt[u] = ptr[(UN + u) * step];
+    }
+    ptr += UN * step;
+#pragma unroll
+    for (int u = 0; u < UN; ++u) f(cur[u], i + u);
+    if (more) {
+#pragma unroll
+      for (int u = 0; u < UN; ++u) cur[u] = nxt[u];
+    }
+  }
+  for (; i < n; ++i) {
+    const uint4 t = *ptr;
+    ptr += step;
+    f(t, i);
+  }
+}
+template <typename T> __device__ __forceinline__ void unpack16(const uint4& r, float (&v)[Elem<T>::VEC]) {
+  if constexpr (sizeof(T) == 4) {
+    v[0] = __uint_as_float(r.x); v[1] = __uint_as_float(r.y); v[2] = __uint_as_float(r.z); v[3] = __uint_as_float(r.w);
+  } else {
+    const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) { v[2 * k] = __uint_as_float(w[k] << 16); v[2 * k + 1] = __uint_as_float(w[k] & 0xffff0000u); }
+  }
+}
+template <typename T> __device__ __forceinline__ uint4 pack16(const float (&v)[Elem<T>::VEC]) {
+  if constexpr (sizeof(T) == 4) {
+    return make_uint4(__float_as_uint(v[0]), __float_as_uint(v[1]), __float_as_uint(v[2]), __float_as_uint(v[3]));
+  } else {
+    return make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]), pack_bf16x2(v[6], v[7]));
+  }
+}
+
 template <typename T>
-__global__ void __launch_bounds__(GN_THREADS) groupnorm_stats_kernel(const T* __restrict__ x, int64_t hw, int c, int groups,
+__global__ void __launch_bounds__(GN_THREADS, GN_RESIDENT) groupnorm_stats_kernel(const T* __restrict__ x, int64_t hw, int c, int groups,
                                                                      const __grid_constant__ EpiProgram pre,
                                                                      float* __restrict__ scratch) {
   constexpr int VE = Elem<T>::VEC;
@@ -518,13 +581,27 @@ __global__ void __launch_bounds__(GN_THREADS) groupnorm_stats_kernel(const T* __
   const int cg_ = c / groups;
 #pragma unroll
   for (int e = 0; e < VE; ++e) { s[e] = 0.0f; q[e] = 0.0f; piv[e] = gn_pivot(x, img, hw, c, (vcol * VE + e) / cg_, cg_, pre); }
-  for (int64_t pix = p0 + prow; pix < p1; pix += pstride) {
-    float v[VE];
-    const int64_t r = img * hw + pix;
-    ld_vec(x + r * c + vcol * VE, v);
-    epi_apply_vec<T, VE>(pre, v, r, (int64_t)vcol * VE, c);
+  {
+    const int64_t first = p0 + prow;
+    const int n_my = first < p1 ? (int)((p1 - first + pstride - 1) / pstride) : 0;
+    const uint4* ptr = reinterpret_cast<const uint4*>(x + (img * hw + first) * c + vcol * VE);
+    const size_t step = (size_t)pstride * c / VE;             // 16-byte vectors between two pixels of this thread
+    if (pre.n == 0) {
+      walk16<GN_UN>(ptr, step, n_my, [&](const uint4& raw, int) {
+        float v[VE];
+        unpack16<T>(raw, v);
 #pragma unroll
-    for (int e = 0; e < VE; ++e) { const float d = v[e] - piv[e]; s[e] += d; q[e] = fmaf(d, d, q[e]); }
+        for (int e = 0; e < VE; ++e) { const float d = v[e] - piv[e]; s[e] += d; q[e] = fmaf(d, d, q[e]); }
+      });
+    } else {
+      walk16<GN_UN>(ptr, step, n_my, [&](const uint4& raw, int i) {
+        float v[VE];
+        unpack16<T>(raw, v);
+        epi_apply_vec<T, VE>(pre, v, img * hw + first + (int64_t)i * pstride, (int64_t)vcol * VE, c);
+#pragma unroll
+        for (int e = 0; e < VE; ++e) { const float d = v[e] - piv[e]; s[e] += d; q[e] = fmaf(d, d, q[e]); }
+      });
+    }
   }
 #pragma unroll
   for (int e = 0; e < VE; ++e) {
@@ -543,8 +620,77 @@ __global__ void __launch_bounds__(GN_THREADS) groupnorm_stats_kernel(const T* __
   }
 }
 
+// Column sums of float [stat_slots][ncol] (ncol = 2 * groups <= 2 * GN_MAX_C partial sums per slot) into sh_stat[ncol],
+// by the whole CTA; the caller synchronises before reading sh_stat.
+__device__ __forceinline__ void gn_reduce_slots(const float* __restrict__ st, int stat_slots, int ncol, float* sh_stat, float (*sh_part)[2 * 64]) {
+  // Reduction of the partials: 2 * groups columns, the slots of a column split over as many threads as
+  // the CTA can spare, sixteen independent loads in flight per thread.
+  int parts = GN_THREADS / ncol;
+  if (parts < 1) parts = 1;
+  if (parts > 8) parts = 8;
+  const bool small = ncol <= 128 && parts > 1;
+  const int quads = ncol / 4;                         // 16-byte pieces per slot
+  if (ncol % 4 == 0 && quads <= 16 && GN_THREADS / quads <= 16 && stat_slots <= 8 * (GN_THREADS / quads)) {
+    // a slot is a few hundred contiguous bytes: 16-byte loads, every thread's (at most eight) in flight at once,
+    // so the whole reduction costs one round trip to L2 instead of two or more
+    const int lanes = GN_THREADS / quads;             // slots read side by side
+    const int qd = threadIdx.x % quads, sl = threadIdx.x / quads;
+    float4 t[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int k = sl + u * lanes;
+      t[u] = (sl < lanes && k < stat_slots) ? *reinterpret_cast<const float4*>(st + (int64_t)k * ncol + qd * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    float4 a = t[0];
+#pragma unroll
+    for (int u = 1; u < 8; ++u) { a.x += t[u].x; a.y += t[u].y; a.z += t[u].z; a.w += t[u].w; }
+    float* pp = &sh_part[0][0];                        // [lanes <= 16][ncol <= 64] floats: 8 x 128 are enough
+    if (sl < lanes) *reinterpret_cast<float4*>(pp + sl * ncol + qd * 4) = a;
+    __syncthreads();
+    if ((int)threadIdx.x < ncol) {
+      float acc = 0.0f;
+      for (int p = 0; p < lanes; ++p) acc += pp[p * ncol + threadIdx.x];
+      sh_stat[threadIdx.x] = acc;
+    }
+  } else if (small) {
+    const int col = threadIdx.x % ncol, part = threadIdx.x / ncol;
+    if (part < parts) {
+      float acc = 0.0f;
+      for (int k0 = part; k0 < stat_slots; k0 += 16 * parts) {
+        float t[16];
+#pragma unroll
+        for (int u = 0; u < 16; ++u) {
+          const int k = k0 + u * parts;
+          t[u] = k < stat_slots ? st[(int64_t)k * ncol + col] : 0.0f;
+        }
+#pragma unroll
+        for (int u = 0; u < 16; ++u) acc += t[u];
+      }
+      sh_part[part][col] = acc;
+    }
+    __syncthreads();
+    if ((int)threadIdx.x < ncol) {
+      float acc = 0.0f;
+      for (int p = 0; p < parts; ++p) acc += sh_part[p][threadIdx.x];
+      sh_stat[threadIdx.x] = acc;
+    }
+  } else {
+    for (int idx = threadIdx.x; idx < ncol; idx += GN_THREADS) {
+      float acc = 0.0f;
+      for (int k0 = 0; k0 < stat_slots; k0 += 16) {
+        float t[16];
+#pragma unroll
+        for (int u = 0; u < 16; ++u) t[u] = k0 + u < stat_slots ? st[(int64_t)(k0 + u) * ncol + idx] : 0.0f;
+#pragma unroll
+        for (int u = 0; u < 16; ++u) acc += t[u];
+      }
+      sh_stat[idx] = acc;
+    }
+  }
+}
+
 template <typename T>
-__global__ void __launch_bounds__(GN_THREADS) groupnorm_apply_kernel(const T* __restrict__ x, T* __restrict__ y, int64_t hw,
+__global__ void __launch_bounds__(GN_THREADS, GN_RESIDENT) groupnorm_apply_kernel(const T* __restrict__ x, T* __restrict__ y, int64_t hw,
                                                                      int c, int groups, const T* __restrict__ gamma,
                                                                      const T* __restrict__ beta, float eps,
                                                                      const __grid_constant__ EpiProgram pre,
@@ -552,21 +698,24 @@ __global__ void __launch_bounds__(GN_THREADS) groupnorm_apply_kernel(const T* __
   constexpr int VE = Elem<T>::VEC;
   __shared__ float sh_scale[GN_MAX_C];
   __shared__ float sh_shift[GN_MAX_C];
+  __shared__ float sh_stat[2 * GN_MAX_C];
+  __shared__ float sh_part[8][2 * 64];
   const int chunks = gridDim.x, chunk = blockIdx.x;
   const int64_t img = blockIdx.y;
   const int cg = c / groups;
+  const int vpp = c / VE;
+  const int vcol = threadIdx.x % vpp, prow = threadIdx.x / vpp, pstride = GN_THREADS / vpp;
+  const int64_t p0 = hw * chunk / chunks, p1 = hw * (chunk + 1) / chunks;
+  const T* xin = x + (img * hw) * c + vcol * VE;
+  T* yout = y + (img * hw) * c + vcol * VE;
+  gn_reduce_slots(scratch + img * chunks * groups * 2, chunks, 2 * groups, sh_stat, sh_part);
+  __syncthreads();
   const float inv_cnt = 1.0f / ((float)hw * (float)cg);
   for (int ch = threadIdx.x; ch < c; ch += GN_THREADS) {
     const int g = ch / cg;
-    float ts = 0.0f, tq = 0.0f;
-    for (int k = 0; k < chunks; ++k) {
-      const float* o = scratch + ((img * chunks + k) * groups + g) * 2;
-      ts += o[0];
-      tq += o[1];
-    }
-    const float md = ts * inv_cnt;                                   // mean - pivot
+    const float md = sh_stat[2 * g] * inv_cnt;                       // mean - pivot
     const float mean = gn_pivot(x, img, hw, c, g, cg, pre) + md;
-    const float var = fmaxf(tq * inv_cnt - md * md, 0.0f);
+    const float var = fmaxf(sh_stat[2 * g + 1] * inv_cnt - md * md, 0.0f);
     const float rstd = rsqrtf(var + eps);
     const float ga = gamma ? Elem<T>::ld(gamma + ch) : 1.0f;
     const float be = beta ? Elem<T>::ld(beta + ch) : 0.0f;
@@ -574,17 +723,31 @@ __global__ void __launch_bounds__(GN_THREADS) groupnorm_apply_kernel(const T* __
     sh_shift[ch] = be - mean * rstd * ga;
   }
   __syncthreads();
-  const int vpp = c / VE;
-  const int vcol = threadIdx.x % vpp, prow = threadIdx.x / vpp, pstride = GN_THREADS / vpp;
-  const int64_t p0 = hw * chunk / chunks, p1 = hw * (chunk + 1) / chunks;
-  for (int64_t pix = p0 + prow; pix < p1; pix += pstride) {
-    float v[VE];
-    const int64_t r = img * hw + pix;
-    ld_vec(x + r * c + vcol * VE, v);
-    epi_apply_vec<T, VE>(pre, v, r, (int64_t)vcol * VE, c);
+  float sc[VE], sf[VE];
 #pragma unroll
-    for (int e = 0; e < VE; ++e) v[e] = v[e] * sh_scale[vcol * VE + e] + sh_shift[vcol * VE + e];
-    st_vec(y + r * c + vcol * VE, v);
+  for (int e = 0; e < VE; ++e) { sc[e] = sh_scale[vcol * VE + e]; sf[e] = sh_shift[vcol * VE + e]; }
+  const int64_t first = p0 + prow;
+  const int n_my = first < p1 ? (int)((p1 - first + pstride - 1) / pstride) : 0;
+  const size_t step = (size_t)pstride * c / VE;
+  const uint4* ptr = reinterpret_cast<const uint4*>(xin + first * c);
+  uint4* out = reinterpret_cast<uint4*>(yout + first * c);
+  if (pre.n == 0) {
+    walk16<GN_UN>(ptr, step, n_my, [&](const uint4& raw, int i) {
+      float v[VE];
+      unpack16<T>(raw, v);
+#pragma unroll
+      for (int e = 0; e < VE; ++e) v[e] = fmaf(v[e], sc[e], sf[e]);
+      out[(size_t)i * step] = pack16<T>(v);
+    });
+  } else {
+    walk16<GN_UN>(ptr, step, n_my, [&](const uint4& raw, int i) {
+      float v[VE];
+      unpack16<T>(raw, v);
+      epi_apply_vec<T, VE>(pre, v, img * hw + first + (int64_t)i * pstride, (int64_t)vcol * VE, c);
+#pragma unroll
+      for (int e = 0; e < VE; ++e) v[e] = fmaf(v[e], sc[e], sf[e]);
+      out[(size_t)i * step] = pack16<T>(v);
+    });
   }
 }
 
@@ -678,72 +841,7 @@ __global__ void __launch_bounds__(GN_THREADS, 3) groupnorm_apply_partials_kernel
   for (int u = 0; u < UN; ++u)
     if (pix + (int64_t)u * pstride < p1) cur[u].load(xin + (pix + (int64_t)u * pstride) * c);
 
-  // Reduction of the partials: 2 * groups columns, the slots of a column split over as many threads as
-  // the CTA can spare, sixteen independent loads in flight per thread.
-  const float* st = stats + img * stat_slots * groups * 2;
-  const int ncol = 2 * groups;
-  int parts = GN_THREADS / ncol;
-  if (parts < 1) parts = 1;
-  if (parts > 8) parts = 8;
-  const bool small = ncol <= 128 && parts > 1;
-  const int quads = ncol / 4;                         // 16-byte pieces per slot
-  if (ncol % 4 == 0 && quads <= 16 && GN_THREADS / quads <= 16 && stat_slots <= 8 * (GN_THREADS / quads)) {
-    // a slot is a few hundred contiguous bytes: 16-byte loads, every thread's (at most eight) in flight at once,
-    // so the whole reduction costs one round trip to L2 instead of two or more
-    const int lanes = GN_THREADS / quads;             // slots read side by side
-    const int qd = threadIdx.x % quads, sl = threadIdx.x / quads;
-    float4 t[8];
-#pragma unroll
-    for (int u = 0; u < 8; ++u) {
-      const int k = sl + u * lanes;
-      t[u] = (sl < lanes && k < stat_slots) ? *reinterpret_cast<const float4*>(st + (int64_t)k * ncol + qd * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
-    }
-    float4 a = t[0];
-#pragma unroll
-    for (int u = 1; u < 8; ++u) { a.x += t[u].x; a.y += t[u].y; a.z += t[u].z; a.w += t[u].w; }
-    float* pp = &sh_part[0][0];                        // [lanes <= 16][ncol <= 64] floats: 8 x 128 are enough
-    if (sl < lanes) *reinterpret_cast<float4*>(pp + sl * ncol + qd * 4) = a;
-    __syncthreads();
-    if ((int)threadIdx.x < ncol) {
-      float acc = 0.0f;
-      for (int p = 0; p < lanes; ++p) acc += pp[p * ncol + threadIdx.x];
-      sh_stat[threadIdx.x] = acc;
-    }
-  } else if (small) {
-    const int col = threadIdx.x % ncol, part = threadIdx.x / ncol;
-    if (part < parts) {
-      float acc = 0.0f;
-      for (int k0 = part; k0 < stat_slots; k0 += 16 * parts) {
-        float t[16];
-#pragma unroll
-        for (int u = 0; u < 16; ++u) {
-          const int k = k0 + u * parts;
-          t[u] = k < stat_slots ? st[(int64_t)k * ncol + col] : 0.0f;
-        }
-#pragma unroll
-        for (int u = 0; u < 16; ++u) acc += t[u];
-      }
-      sh_part[part][col] = acc;
-    }
-    __syncthreads();
-    if ((int)threadIdx.x < ncol) {
-      float acc = 0.0f;
-      for (int p = 0; p < parts; ++p) acc += sh_part[p][threadIdx.x];
-      sh_stat[threadIdx.x] = acc;
-    }
-  } else {
-    for (int idx = threadIdx.x; idx < ncol; idx += GN_THREADS) {
-      float acc = 0.0f;
-      for (int k0 = 0; k0 < stat_slots; k0 += 16) {
-        float t[16];
-#pragma unroll
-        for (int u = 0; u < 16; ++u) t[u] = k0 + u < stat_slots ? st[(int64_t)(k0 + u) * ncol + idx] : 0.0f;
-#pragma unroll
-        for (int u = 0; u < 16; ++u) acc += t[u];
-      }
-      sh_stat[idx] = acc;
-    }
-  }
+  gn_reduce_slots(stats + img * stat_slots * groups * 2, stat_slots, 2 * groups, sh_stat, sh_part);
   __syncthreads();
   const float inv_cnt = 1.0f / ((float)hw * (float)cg);
   for (int ch = threadIdx.x; ch < c; ch += GN_THREADS) {

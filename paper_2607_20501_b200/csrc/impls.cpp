@@ -5,6 +5,8 @@
 // used blocks fusion unless one CTA owns the whole row).
 //
 // Order = the composer's preference among implementations that accept the same range.
+#include <stdio.h>
+#include <stdlib.h>
 #include <memory>
 
 #include "mk_internal.h"
@@ -130,6 +132,15 @@ mk_status groupnorm_emit(const Module& m, int lo, int hi, const Resolved& r, std
   const void* b = op.param[1].set ? op.param[1].ptr : nullptr;
   const float eps = (float)op.d.f[0];
   const int d = dt(m);
+  const int sms = m.ctx->sm_count;
+  if (getenv("MK_DEBUG_PLAN"))
+    fprintf(stderr, "groupnorm_nhwc: nb %lld hw %lld c %lld groups %d -> %s\n", (long long)nb, (long long)hw, (long long)c, groups,
+            groupnorm_cluster_supported(d, x, y, nb, hw, c, groups, sms) ? "cluster form" : "two passes");
+  if (!getenv("MK_GN_TWO_PASS") && groupnorm_cluster_supported(d, x, y, nb, hw, c, groups, sms)) {
+    // the image fits a cluster's shared memory: one launch, the tensor read once
+    out.push_back([=](cudaStream_t st_) { return launch_groupnorm_cluster(d, x, y, nb, hw, c, groups, g, b, eps, p, sms, st_); });
+    return MK_OK;
+  }
   const int chunks = groupnorm_chunks(nb, hw, m.ctx->sm_count);
   float* scratch = (float*)r.scratch;
   out.push_back([=](cudaStream_t st_) { return launch_groupnorm_stats(d, x, nb, hw, c, groups, p, scratch, chunks, st_); });

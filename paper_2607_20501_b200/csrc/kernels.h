@@ -148,6 +148,11 @@ cudaError_t launch_rowop(int dtype, int in_dtype, int mode, const void* x, void*
 // GroupNorm over NHWC [nb, hw, c]: stats writes per-(image, chunk, group) partial sums into
 // scratch, apply reduces them and normalises.  scratch must hold groupnorm_scratch_bytes().
 int groupnorm_chunks(int64_t nb, int64_t hw, int sm_count);
+// One launch, one pass over HBM: a thread-block cluster holds an image in its shared memory (groupnorm_cluster.cu).
+// supported: the image fits a cluster of at most eight CTAs, 16-byte-aligned tensors, vectorisable channel count.
+bool groupnorm_cluster_supported(int dtype, const void* x, const void* y, int64_t nb, int64_t hw, int64_t c, int groups, int sm_count);
+cudaError_t launch_groupnorm_cluster(int dtype, const void* x, void* y, int64_t nb, int64_t hw, int64_t c, int groups, const void* gamma,
+                                     const void* beta, float eps, const EpiProgram& pre, int sm_count, cudaStream_t s);
 size_t groupnorm_scratch_bytes(int64_t nb, int64_t hw, int64_t c, int groups, int sm_count);
 cudaError_t launch_groupnorm_stats(int dtype, const void* x, int64_t nb, int64_t hw, int64_t c,
                                    int groups, const EpiProgram& pre, float* scratch, int chunks,

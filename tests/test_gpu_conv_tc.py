@@ -68,6 +68,32 @@ def test_groupnorm_statistics_from_the_conv_epilogue(ctx, nb, h, w, c, co, g):
     assert np.abs(out - out2).max() <= 4e-2
 
 
+@pytest.mark.parametrize("nb,h,w,c,co,g", [(2, 8, 8, 64, 64, 16), (3, 9, 7, 128, 128, 32), (2, 13, 62, 64, 128, 4)])
+def test_conv_epilogue_statistics_far_from_zero_mean(ctx, nb, h, w, c, co, g):
+    """Groups whose mean is some forty standard deviations from zero.  Inputs in {0, 1}, sparse weights in {-1, 0, 1}
+    and a bias of 40 to 56 per group make every value the convolution stores a small integer, exact in bf16, so the
+    only error left is that of the statistics: the epilogue's partial sums are taken about zero in fp32 (relative
+    error of the variance about 2^-24 * mean^2 / var), the two-pass form's about a pivot.  Both must meet the oracle."""
+    wl = W.c3(5, NB=nb, H=h, W=w, C=c, CO=co, G=g)
+    rng = np.random.default_rng(17)
+    wl.inputs["x"] = G.make("x", "bf16", (rng.random((nb, h, w, c)) < 0.5).astype(np.float32))
+    sparse = rng.random((co, 3, 3, c)) < 2.0 / (9 * c)
+    wl.params["Wc"] = G.make("Wc", "bf16", (sparse * rng.choice([-1.0, 1.0], (co, 3, 3, c))).astype(np.float32))
+    wl.params["bias"] = G.make("bias", "bf16", np.repeat(rng.choice([40.0, 48.0, 56.0], g), co // g).astype(np.float32))
+    ref, bnd = oracle(wl, list(range(len(wl.ops))))
+    y2 = bnd["y2"]
+    assert np.array_equal(y2, np.round(y2)) and y2.max() < 256 and y2.min() > 8     # exact in bf16, above the ReLU's cut
+    grp = y2.reshape(nb, h * w, g, co // g)
+    sd = grp.std(axis=(1, 3))
+    assert sd.min() > 0.3 and (np.abs(grp.mean(axis=(1, 3))) / sd).min() > 15.0
+    dw, out = run_gpu(ctx, wl, wl.partitions["fused"])
+    assert dw.module.bound_impl(0) == "conv3x3_gn_tc2"
+    assert_parity(out, ref, "bf16", "fused, far mean")
+    dw2, out2 = run_gpu(ctx, wl, wl.partitions["split2"])
+    assert dw2.module.bound_impl(1) == "groupnorm_nhwc"
+    assert_parity(out2, ref, "bf16", "two-pass, far mean")
+
+
 def test_swap_conv_kernels(ctx):
     wl = W.c3(0, NB=2, H=12, W=12, C=64, CO=64, G=8)
     ref, _ = oracle(wl, [0])
