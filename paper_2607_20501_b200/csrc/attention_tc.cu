@@ -28,13 +28,14 @@ namespace mk {
 
 namespace {
 
-constexpr int BQ = 128, BKV = 128, HD = 128;
-constexpr int TILE_BYTES = 128 * HD * 2;   // 32 KB: two 128 x 64 sub-tiles of 16 KB
-constexpr int SUB_BYTES = TILE_BYTES / 2;
+constexpr int BQ = 128, BKV = 128;
+constexpr int SUB_BYTES = 128 * 64 * 2;    // a 128 x 64 sub-tile (one 128-byte swizzle row per query / key): 16 KB
+// a Q / K / V tile: 128 rows x head_dim = one sub-tile (head_dim 64) or two (head_dim 128)
+constexpr int tile_bytes(int hd) { return 128 * hd * 2; }
 constexpr int KV_STAGES = 2;
 constexpr int SOFTMAX_WARPS = 8;
 constexpr int THREADS = 64 + 32 * SOFTMAX_WARPS;
-constexpr size_t ATTN_SMEM = (size_t)TILE_BYTES * (1 + 2 * KV_STAGES) + SOFTMAX_WARPS * EPI_WARP_BYTES + 1024 + 256 + 2048;
+constexpr size_t attn_smem(int hd) { return (size_t)tile_bytes(hd) * (1 + 2 * KV_STAGES) + SOFTMAX_WARPS * EPI_WARP_BYTES + 1024 + 256 + 2048; }
 
 struct Shared {
   uint64_t q_full;
@@ -64,9 +65,15 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16
       : "memory");
 }
 
+// HD: head dimension, 64 or 128.  causal != 0: query i sees keys 0..i; else every key (the last key tile may be
+// ragged: keys past S are hidden the way the diagonal hides them, with one limit for every row).
+template <int HD>
 __global__ void __launch_bounds__(THREADS, 1)
 attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
-                    __nv_bfloat16* __restrict__ out, int B, int H, int S, float scale_log2, unsigned int* status) {
+                    __nv_bfloat16* __restrict__ out, int B, int H, int S, int causal, float scale_log2, unsigned int* status) {
+  static_assert(HD == 64 || HD == 128, "head dimension");
+  constexpr int TILE_BYTES = tile_bytes(HD);
+  constexpr int OC = HD / 64;                    // 32-column chunks of O per softmax thread (it owns HD / 2 columns)
   extern __shared__ uint8_t smem_raw[];
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* q_tile = base;
@@ -82,7 +89,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   const int bh = blockIdx.x / num_q;
   const int qt = num_q - 1 - blockIdx.x % num_q;
   const int b = bh / H, h = bh - b * H;
-  const int T = qt + 1;                               // key tiles 0 .. diagonal
+  const int T = causal ? qt + 1 : num_q;              // key tiles 0 .. diagonal, or all of them
   volatile int* abort_flag = &sh->abort_flag;
   MK_TR_DECL
   MK_TR_INIT;
@@ -116,7 +123,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     if (lane == 0) {
       tc::mbar_expect_tx(&sh->q_full, TILE_BYTES);
       tc::tma_load_4d(q_tile, &tmQ, &sh->q_full, 0, qt * BQ, h, b);
-      tc::tma_load_4d(q_tile + SUB_BYTES, &tmQ, &sh->q_full, 64, qt * BQ, h, b);
+      if (HD == 128) tc::tma_load_4d(q_tile + SUB_BYTES, &tmQ, &sh->q_full, 64, qt * BQ, h, b);
       bool ok = true;
       auto load_k = [&](int j) {
         const int st = j % KV_STAGES;
@@ -125,7 +132,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         uint8_t* kd = k_tiles + (size_t)st * TILE_BYTES;
         tc::mbar_expect_tx(&sh->k_full[st], TILE_BYTES);
         tc::tma_load_4d(kd, &tmK, &sh->k_full[st], 0, j * BKV, h, b);
-        tc::tma_load_4d(kd + SUB_BYTES, &tmK, &sh->k_full[st], 64, j * BKV, h, b);
+        if (HD == 128) tc::tma_load_4d(kd + SUB_BYTES, &tmK, &sh->k_full[st], 64, j * BKV, h, b);
       };
       auto load_v = [&](int j) {
         const int st = j % KV_STAGES;
@@ -134,7 +141,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         uint8_t* vd = v_tiles + (size_t)st * TILE_BYTES;
         tc::mbar_expect_tx(&sh->v_full[st], TILE_BYTES);
         tc::tma_load_4d(vd, &tmV, &sh->v_full[st], 0, j * BKV, h, b);
-        tc::tma_load_4d(vd + SUB_BYTES, &tmV, &sh->v_full[st], 64, j * BKV, h, b);
+        if (HD == 128) tc::tma_load_4d(vd + SUB_BYTES, &tmV, &sh->v_full[st], 64, j * BKV, h, b);
       };
       // Loads are issued in the order their ring slots come free, which is the order the MMAs retire:
       // QK(0) QK(1) PV(0) QK(2) PV(1) QK(3) ...  (a K load queued behind a V slot that frees later would
@@ -205,15 +212,15 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   } else {
     // ------------------------------------------------------------ softmax + O accumulation
     // Eight warps: warps w and w + 4 share TMEM lane quarter w % 4, i.e. the same 32 query rows; each
-    // thread owns one row and one half of its columns (64 keys of S_j, 64 head-dim columns of O).  The
+    // thread owns one row and one half of its columns (64 keys of S_j, HD / 2 head-dim columns of O).  The
     // two threads of a row meet once per tile to agree on the row maximum (shared memory + a 64-thread
     // named barrier) and once at the end to add their row sums.
     const int q = warp & 3, hf = (warp - 2) >> 2;
     const uint32_t lane_off = (uint32_t)(q * 32) << 16;
     const int row_in_tile = q * 32 + lane;
-    float o[64];
+    float o[HD / 2];
 #pragma unroll
-    for (int i = 0; i < 64; ++i) o[i] = 0.0f;
+    for (int i = 0; i < HD / 2; ++i) o[i] = 0.0f;
     float m = -INFINITY, l = 0.0f, alpha_prev = 0.0f;
     bool ok = true;
     for (int j = 0; j < T; ++j) {
@@ -225,7 +232,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       if (threadIdx.x == 64 && j < 11) MK_TR(1 + j * 8);   // S_j ready
       tc::tc_fence_after();
       const uint32_t s_addr = tmem_s + buf * 128 + lane_off + hf * 64;
-      const bool diag = j == T - 1;
+      // the tile with hidden keys: the diagonal one (limit = the row's own index), or an unmasked head's ragged last
+      // tile (limit = the last real key, the same for every row)
+      const bool diag = j == T - 1 && (causal || (S & (BKV - 1)) != 0);
+      const int lim = causal ? row_in_tile : S - 1 - j * BKV;
       const int col_base = hf * 64;                          // key index (inside the tile) of this thread's first column
       // pass 1: maximum of the raw scores (four independent chains), then into log2 units
       float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
@@ -240,7 +250,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         } else {
 #pragma unroll
           for (int i = 0; i < 32; ++i)
-            if (col_base + c * 32 + i <= row_in_tile) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(r[i]));
+            if (col_base + c * 32 + i <= lim) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(r[i]));
         }
       }
       const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * scale_log2;
@@ -264,8 +274,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
           float p0 = tc::ex2_fast(fmaf(__uint_as_float(r[i]), scale_log2, neg_m));
           float p1 = tc::ex2_fast(fmaf(__uint_as_float(r[i + 1]), scale_log2, neg_m));
           if (diag) {
-            if (col_base + c * 32 + i > row_in_tile) p0 = 0.0f;
-            if (col_base + c * 32 + i + 1 > row_in_tile) p1 = 0.0f;
+            if (col_base + c * 32 + i > lim) p0 = 0.0f;
+            if (col_base + c * 32 + i + 1 > lim) p1 = 0.0f;
           }
           sum4[(i >> 1) & 3] += p0 + p1;
           pk[i >> 1] = pack_bf16x2(p0, p1);
@@ -285,9 +295,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         ok = __all_sync(0xffffffffu, ok ? 1 : 0) != 0;
         if (!ok) break;
         tc::tc_fence_after();
-        const uint32_t o_addr = tmem_o + pb * 128 + lane_off + hf * 64;
+        const uint32_t o_addr = tmem_o + pb * 128 + lane_off + hf * (HD / 2);
 #pragma unroll
-        for (int c = 0; c < 2; ++c) {
+        for (int c = 0; c < OC; ++c) {
           uint32_t r[32];
           tc::tmem_ld32(o_addr + c * 32, r);
           tc::tmem_ld_wait();
@@ -311,16 +321,16 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       sh->xch[T & 1][row_in_tile][hf] = l;
       asm volatile("bar.sync %0, %1;" ::"r"(1 + q), "r"(64) : "memory");
       const float inv_l = 1.0f / (l + sh->xch[T & 1][row_in_tile][hf ^ 1]);
-      const uint32_t o_addr = tmem_o + ((T - 1) & 1) * 128 + lane_off + hf * 64;
+      const uint32_t o_addr = tmem_o + ((T - 1) & 1) * 128 + lane_off + hf * (HD / 2);
 #pragma unroll
-      for (int c = 0; c < 2; ++c) {
+      for (int c = 0; c < OC; ++c) {
         uint32_t r[32];
         tc::tmem_ld32(o_addr + c * 32, r);
         tc::tmem_ld_wait();
 #pragma unroll
         for (int i = 0; i < 32; ++i) o[c * 32 + i] = fmaf(o[c * 32 + i], alpha_prev, __uint_as_float(r[i])) * inv_l;
       }
-      // store: rows (b*S + query), this thread's 64 of the columns h*D .. h*D + 127 of the [B*S, H*D] matrix
+      // store: rows (b*S + query), this thread's HD / 2 of the columns h*D .. h*D + HD - 1 of the [B*S, H*D] matrix
       EpiProgram none;
       none.n = 0;
       EpiWarp ew;
@@ -331,11 +341,11 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       uint4 none_regs[8];
       const int64_t n_cols = (int64_t)H * HD;
 #pragma unroll
-      for (int c = 0; c < 2; ++c) {
+      for (int c = 0; c < OC; ++c) {
         float v[32];
 #pragma unroll
         for (int i = 0; i < 32; ++i) v[i] = o[c * 32 + i];
-        ew.chunk_out(none, v, rowmap, out, (int64_t)h * HD + hf * 64 + c * 32, 0, n_cols, none_regs, -1);
+        ew.chunk_out(none, v, rowmap, out, (int64_t)h * HD + hf * (HD / 2) + c * 32, 0, n_cols, none_regs, -1);
       }
     }
   }
@@ -356,8 +366,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 }  // namespace
 
 bool attention_tc_supported(const AttnView& a) {
-  if (!a.causal) return false;
-  if (a.D != HD || a.B < 1 || a.H < 1 || a.S < 1) return false;
+  if ((a.D != 64 && a.D != 128) || a.B < 1 || a.H < 1 || a.S < 1) return false;
   if ((a.ss * 2) % 16 || (a.sh * 2) % 16 || (a.sb * 2) % 16) return false;
   if (a.B * a.H * ((a.S + BQ - 1) / BQ) > INT32_MAX) return false;
   return true;
@@ -373,7 +382,8 @@ cudaError_t attention_tc_plan(AttnTcPlan* p, const AttnView& a, void* o) {
   if (e == cudaSuccess) e = encode_tmap_bf16(&p->tm_v, a.v, 4, dims, strides, box, true);
   if (e != cudaSuccess) return e;
   p->out = o;
-  p->B = (int)a.B; p->H = (int)a.H; p->S = (int)a.S;
+  p->B = (int)a.B; p->H = (int)a.H; p->S = (int)a.S; p->D = (int)a.D;
+  p->causal = a.causal;
   p->scale_log2 = (float)(1.4426950408889634 / sqrt((double)a.D));
   p->grid = (int)(a.B * a.H * ((a.S + BQ - 1) / BQ));
   return cudaSuccess;
@@ -382,11 +392,15 @@ cudaError_t attention_tc_plan(AttnTcPlan* p, const AttnView& a, void* o) {
 cudaError_t launch_attention_tc(const AttnTcPlan& p, cudaStream_t s) {
   static SmemOptIn opt_in;
   {
-    cudaError_t e = opt_in.ensure(ATTN_SMEM, attention_tc_kernel);
+    cudaError_t e = opt_in.ensure(attn_smem(128), attention_tc_kernel<64>, attention_tc_kernel<128>);
     if (e != cudaSuccess) return e;
   }
-  attention_tc_kernel<<<p.grid, THREADS, ATTN_SMEM, s>>>(p.tm_q, p.tm_k, p.tm_v, (__nv_bfloat16*)p.out, p.B, p.H, p.S, p.scale_log2,
-                                                         kernel_status_ptr());
+  if (p.D == 64)
+    attention_tc_kernel<64><<<p.grid, THREADS, attn_smem(64), s>>>(p.tm_q, p.tm_k, p.tm_v, (__nv_bfloat16*)p.out, p.B, p.H, p.S, p.causal ? 1 : 0,
+                                                                  p.scale_log2, kernel_status_ptr());
+  else
+    attention_tc_kernel<128><<<p.grid, THREADS, attn_smem(128), s>>>(p.tm_q, p.tm_k, p.tm_v, (__nv_bfloat16*)p.out, p.B, p.H, p.S,
+                                                                    p.causal ? 1 : 0, p.scale_log2, kernel_status_ptr());
   return cudaGetLastError();
 }
 

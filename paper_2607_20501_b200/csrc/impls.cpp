@@ -560,8 +560,9 @@ AttnView attn_view(const Module& m, const Op& op, const Resolved& r) {
   }
   return a;
 }
+bool is_attention(int32_t k) { return k == MK_OP_ATTENTION_CAUSAL || k == MK_OP_ATTENTION; }
 bool attn_tc_match(const Module& m, int lo, int hi) {
-  if (hi - lo != 1 || m.ops[lo].d.kind != MK_OP_ATTENTION_CAUSAL || m.dtype != MK_BF16) return false;
+  if (hi - lo != 1 || !is_attention(m.ops[lo].d.kind) || m.dtype != MK_BF16) return false;
   Resolved none;
   none.value_ptr.assign(m.values.size(), nullptr);
   return attention_tc_supported(attn_view(m, m.ops[lo], none));
@@ -574,7 +575,6 @@ mk_status attn_tc_emit(const Module& m, int lo, int, const Resolved& r, std::vec
   out.push_back([plan](cudaStream_t s) { return launch_attention_tc(*plan, s); });
   return MK_OK;
 }
-bool is_attention(int32_t k) { return k == MK_OP_ATTENTION_CAUSAL || k == MK_OP_ATTENTION; }
 bool attn_tc2_match(const Module& m, int lo, int hi) {
   if (hi - lo != 1 || !is_attention(m.ops[lo].d.kind) || m.dtype != MK_BF16) return false;
   Resolved none;

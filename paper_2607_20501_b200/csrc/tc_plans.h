@@ -154,13 +154,13 @@ namespace mk {
 struct AttnTcPlan {
   CUtensorMap tm_q, tm_k, tm_v;
   void* out = nullptr;
-  int B = 0, H = 0, S = 0;
+  int B = 0, H = 0, S = 0, D = 128;
   bool causal = true;
   float scale_log2 = 0.f;
   int grid = 0;
 };
-// Causal attention, bf16, head_dim 128, any strided [B, H, S, D] view whose strides are multiples of
-// 16 bytes; output the dense [B*S, H*D] matrix.
+// Attention (causal or unmasked), bf16, head_dim 64 or 128, any strided [B, H, S, D] view whose strides are
+// multiples of 16 bytes; output the dense [B*S, H*D] matrix.  One 128-query tile per CTA.
 bool attention_tc_supported(const AttnView& a);
 cudaError_t attention_tc_plan(AttnTcPlan* p, const AttnView& a, void* o);
 cudaError_t launch_attention_tc(const AttnTcPlan& p, cudaStream_t s);

@@ -37,6 +37,50 @@ def test_attention_matches_the_oracle(ctx, impl, b, h, s):
         assert_parity(out, ref, "bf16", f"{impl} B{b} H{h} S{s} seed{seed}")
 
 
+def _unmasked(w):
+    w.ops[0]["kind"] = "attention"
+    return w
+
+
+@pytest.mark.parametrize("causal", [True, False])
+@pytest.mark.parametrize("b,h,s", [(1, 1, 128), (2, 3, 384), (1, 2, 200), (1, 1, 1000), (2, 2, 64), (1, 1, 1), (1, 6, 1024), (3, 5, 197)])
+def test_head_dim_64_on_the_tensor_cores(ctx, causal, b, h, s):
+    """Head dimension 64 (the Transformer block of the paper's ConvolutionalVisionTransformer example has 6 heads of
+    64): the composer's own pick must be the one-tile tensor-core kernel, masked and unmasked, ragged lengths
+    included (197 = 14 x 14 patches + a class token)."""
+    w = _attn_only(W.c4(1, B=b, H=h, S=s, D=64))
+    if not causal:
+        _unmasked(w)
+    ref, _ = oracle(w, [0])
+    dw, out = run_gpu(ctx, w, [0])
+    assert dw.module.bound_impl(0) == "attention_tc"
+    assert_parity(out, ref, "bf16", f"D64 causal={causal} B{b} H{h} S{s}")
+    dw2, out2 = run_gpu(ctx, w, [0], binds={0: "attention_simt"})
+    assert np.abs(out - out2).max() <= 4e-2
+
+
+@pytest.mark.parametrize("b,h,s", [(1, 2, 256), (2, 3, 200), (1, 1, 1000)])
+def test_unmasked_one_tile_kernel_at_head_dim_128(ctx, b, h, s):
+    w = _unmasked(_attn_only(W.c4(2, B=b, H=h, S=s, D=128)))
+    ref, _ = oracle(w, [0])
+    for impl in TC_IMPLS:
+        dw, out = run_gpu(ctx, w, [0], binds={0: impl})
+        assert dw.module.bound_impl(0) == impl
+        assert_parity(out, ref, "bf16", f"{impl} unmasked B{b} H{h} S{s}")
+
+
+def test_encoder_block_with_heads_of_64(ctx):
+    """The encoder block at the ConvolutionalVisionTransformer example's head shape: E = 384, 6 heads of 64, packed
+    QKV, unmasked attention; every attention of the default decomposition runs on the tensor cores."""
+    w = W.c6(0, B=2, S=197, E=384, H=6, F=1536, L=1)
+    part = w.partitions["fused_tails"]
+    ref, _ = oracle(w, part)
+    dw, out = run_gpu(ctx, w, part)
+    impls = [dw.module.bound_impl(i) for i in range(dw.module.n_sub())]
+    assert impls.count("attention_tc") == 1 and "attention_simt" not in impls, impls
+    assert_parity(out, ref, "bf16", "encoder block, heads of 64")
+
+
 @pytest.mark.parametrize("b,h,s", [(4, 48, 256), (2, 80, 512), (1, 150, 384)])
 def test_persistent_ctas_walk_several_items(ctx, b, h, s):
     """More work items than SMs: a CTA of the two-tile kernel then runs several (batch, head, query

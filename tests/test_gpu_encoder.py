@@ -39,11 +39,12 @@ def test_unmasked_attention_matches_the_oracle(ctx, impl, b, h, s):
     assert_parity(out, ref, "bf16", f"{impl} B{b} H{h} S{s}")
 
 
-def test_the_one_tile_kernel_declines_the_unmasked_operator(ctx):
-    from paper_2607_20501_b200 import MkError
+def test_the_one_tile_kernel_takes_the_unmasked_operator_too(ctx):
     w = _attn_only(1, 1, 128)
-    with pytest.raises(MkError):
-        run_gpu(ctx, w, [0], binds={0: "attention_tc"})
+    ref, _ = oracle(w, [0])
+    dw, out = run_gpu(ctx, w, [0], binds={0: "attention_tc"})
+    assert dw.module.bound_impl(0) == "attention_tc"
+    assert_parity(out, ref, "bf16", "one-tile kernel, unmasked")
     dw, _ = run_gpu(ctx, w, [0])
     assert dw.module.bound_impl(0) == "attention_tc2"          # the default cover takes the two-tile kernel
 
@@ -53,8 +54,9 @@ def test_ragged_key_tails(ctx, s):
     """Keys past S in the last key tile are hidden from every query: every remainder class modulo 32."""
     w = _attn_only(1, 2, s, seed=1)
     ref, _ = oracle(w, [0])
-    _, out = run_gpu(ctx, w, [0], binds={0: "attention_tc2"})
-    assert_parity(out, ref, "bf16", f"S{s}")
+    for impl in ("attention_tc2", "attention_tc"):
+        _, out = run_gpu(ctx, w, [0], binds={0: impl})
+        assert_parity(out, ref, "bf16", f"{impl} S{s}")
 
 
 def test_persistent_ctas_walk_several_items(ctx):
