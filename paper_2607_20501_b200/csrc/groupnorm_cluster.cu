@@ -159,7 +159,7 @@ groupnorm_cluster_kernel(const T* __restrict__ x, T* __restrict__ y, int64_t hw,
   for (int k = 0; k < GC_PIECES && ok; ++k) {
     const int a = piece_lo(k), b = piece_lo(k + 1);
     if (b <= a) continue;               // uniform over the CTA
-    // the same verdict in every thread: what follows has CTA-wide barriers in it
+    // the same answer in every thread: what follows has CTA-wide barriers in it
     ok = __syncthreads_and(tc::mbar_wait(&bars[k], 0, abort_flag, status, tc::WAIT_SMEM_FULL) ? 1 : 0) != 0;
     if (!ok) break;
     GCT(2 + k);
