@@ -68,6 +68,7 @@ def test_swap_on_the_encoder_block(ctx):
     assert before[1] == "attention_simt" and before[2] == "gemm_simt" and before[5] == "gemm_simt"
     n, times = dw.swap(iters=3, tau=0.9)
     after = [dw.module.bound_impl(s) for s in range(7)]
-    assert n >= 3 and after[1] == "attention_tc2" and not any("simt" in a for a in after)
+    # at this size either tensor-core attention kernel may measure fastest (four work items on 148 SMs)
+    assert n >= 3 and after[1] in ("attention_tc2", "attention_tc") and not any("simt" in a for a in after)
     assert after[3] == before[3] == "rowop" and after[6] == before[6] == "rowop"
     assert_parity(to_host_f64(dw.forward()), ref, "bf16", "encoder block after swap")
