@@ -16,7 +16,8 @@
 //    is therefore just another shared-memory descriptor with a shifted start address (the 128-byte
 //    swizzle follows absolute shared-memory address bits, so a row-shifted view stays consistent),
 //    and the 9 taps x 4 MMAs of a channel block re-read the same 32 KB.
-//    Rows with w >= W are junk and never stored (W <= 62; 56 of 64 useful at W = 56).
+//    The last two rows of each 64, and rows with w >= W, are junk and never stored (56 of 64 useful at W = 56).  An
+//    image row wider than 62 pixels is covered by several tiles of 62 pixels each (the box starts at w = 62 s - 1).
 //  * L2 -> SM traffic per tile and CTA is the patch alone; the kernel is bound by the tensor pipe.
 //
 // Warp roles as in the GEMM: warp 0 TMA producer, warp 1 TMEM allocation + (leader) MMA issue with a
@@ -32,7 +33,8 @@ namespace mk {
 
 namespace {
 
-constexpr int PITCH = 64;                 // pixel pitch of the patch (>= W + 2)
+constexpr int PITCH = 64;                 // pixel pitch of the patch
+constexpr int SEG = PITCH - 2;            // output pixels of one image row a tile covers; wider rows take several tiles
 constexpr int TILE_ROWS = 2;              // output rows per CTA
 constexpr int PATCH_ROWS = TILE_ROWS + 2; // input rows per CTA incl. halo
 constexpr int PATCH_BYTES = PATCH_ROWS * PITCH * 128;  // one 64-channel block: 32 KB
@@ -131,10 +133,11 @@ __device__ __forceinline__ void umma_ss_pair_x4(uint32_t d_tmem, uint64_t a_desc
 }
 
 
-// CB = C_in / 64 channel blocks
-template <int CB>
+// CB = C_in / 64 channel blocks; WIDE: image rows of more than SEG pixels (several tiles per row)
+template <int CB, bool WIDE>
 __global__ void __launch_bounds__(THREADS, 1)
 conv3x3_tc2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmY,
+                   const __grid_constant__ CUtensorMap tmY30,
                    int NB, int H, int W, int C_OUT, const __grid_constant__ EpiProgram epi_param, float* __restrict__ stats, int cpg,
                    unsigned int* status) {
   extern __shared__ uint8_t smem_raw[];
@@ -150,8 +153,9 @@ conv3x3_tc2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
   const uint32_t rank = tc::cluster_ctarank();
   const bool leader = rank == 0;
   const int cluster_id = blockIdx.x >> 1, num_clusters = gridDim.x >> 1;
-  const int quads = (H + 2 * TILE_ROWS - 1) / (2 * TILE_ROWS);   // pair-tiles per image
-  const int total_tiles = NB * quads;
+  const int quads = (H + 2 * TILE_ROWS - 1) / (2 * TILE_ROWS);   // row groups (four output rows per CTA pair) per image
+  const int nseg = WIDE ? (W + SEG - 1) / SEG : 1;               // SEG-pixel segments per image row
+  const int total_tiles = NB * quads * nseg;                     // tile t = ((n * quads + hq) * nseg + sg)
   volatile int* abort_flag = &sh->abort_flag;
   CTR_INIT;
   static_assert(sizeof(Shared) <= 512, "barrier block");
@@ -168,6 +172,7 @@ conv3x3_tc2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     tc::tma_prefetch_desc(&tmX);
     tc::tma_prefetch_desc(&tmW);
     tc::tma_prefetch_desc(&tmY);
+    if (nseg > 1) tc::tma_prefetch_desc(&tmY30);
   }
   if (warp == 1) tc::tmem_alloc_pair(&sh->tmem_base, 512);
   tc::tc_fence_before();
@@ -208,7 +213,8 @@ conv3x3_tc2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
       uint32_t phase = 0;
       bool ok = true;
       for (int t = cluster_id; t < total_tiles && ok; t += num_clusters) {
-        const int n = t / quads, hq = t - n * quads;
+        const int sg = nseg == 1 ? 0 : t % nseg, nq = nseg == 1 ? t : t / nseg;
+        const int n = nq / quads, hq = nq - n * quads;
         const int h0 = hq * 2 * TILE_ROWS + (int)rank * TILE_ROWS;   // first output row of this CTA
         // No L2 prefetch of the next tile's patches: with one issued here, a whole tile early, the step measured
         // 39.9 us against 39.4 us without (32 x 56 x 56 x 128, inputs rotated through more than L2).
@@ -217,7 +223,7 @@ conv3x3_tc2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
           if (!ok) break;
           const uint32_t full_leader = tc::map_to_cta(tc::smem_u32(&sh->a_full[stage]), 0);
           if (leader) tc::mbar_expect_tx(&sh->a_full[stage], 2 * PATCH_BYTES);
-          tc::tma_load_4d_pair(a_tiles + (size_t)stage * PATCH_BYTES, &tmX, full_leader, cb * 64, -1, h0 - 1, n);
+          tc::tma_load_4d_pair(a_tiles + (size_t)stage * PATCH_BYTES, &tmX, full_leader, cb * 64, sg * SEG - 1, h0 - 1, n);
           if (++stage == A_STAGES) { stage = 0; phase ^= 1; }
         }
       }
@@ -289,19 +295,22 @@ conv3x3_tc2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     const int chunks = C_OUT / 32, c_mid = (chunks + 1) / 2;
     const int c_lo = half ? c_mid : 0, c_hi = half ? chunks : c_mid;
     const int groups = stats ? C_OUT / cpg : 0;
-    const int stat_slots = quads * 2 * 4;          // partial sums per image: one per (pair-tile, CTA, lane quarter)
+    const int stat_slots = quads * nseg * 2 * 4;   // partial sums per image: one per (pair-tile, CTA, lane quarter)
     const uint4 no_res[4] = {};
     bool ok = true;
     int it = 0;
     for (int t = cluster_id; t < total_tiles && ok; t += num_clusters, ++it) {
-      const int n = t / quads, hq = t - n * quads;
+      const int sg = nseg == 1 ? 0 : t % nseg, nq = nseg == 1 ? t : t / nseg;
+      const int n = nq / quads, hq = nq - n * quads;
       const int acc = it & (nacc - 1);
-      // warp q covers tile rows [32q, 32q + 32): output row hl = q / 2, pixels w0 .. w0 + 31
-      const int hl = q >> 1, w0 = (q & 1) * 32;
+      // warp q covers tile rows [32q, 32q + 32): output row hl = q / 2, pixels w0 .. w0 + 31 of the image row, of
+      // which those inside the segment (the first SEG of the tile row's 64) and inside the image are real
+      const int hl = q >> 1, w0 = sg * SEG + (q & 1) * 32;
+      const int w_end = (sg + 1) * SEG < W ? (sg + 1) * SEG : W;
       const int h = hq * 2 * TILE_ROWS + (int)rank * TILE_ROWS + hl;
       const int64_t pix0 = ((int64_t)n * H + h) * W;
       const bool row_ok = h < H;
-      auto rowmap = [&](int r) -> int64_t { return (row_ok && w0 + r < W) ? pix0 + w0 + r : -1; };
+      auto rowmap = [&](int r) -> int64_t { return (row_ok && w0 + r < w_end) ? pix0 + w0 + r : -1; };
       const int64_t my_row = rowmap(lane);
       ok = tc::mbar_wait(&sh->tfull[acc], (it >> acc_shift) & 1, abort_flag, status, tc::WAIT_TMEM_FULL);
       ok = __all_sync(0xffffffffu, ok ? 1 : 0) != 0;
@@ -309,7 +318,7 @@ conv3x3_tc2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
       if (threadIdx.x == 64) CTR(4 + it * 8);  // epilogue: accumulator ready
       tc::tc_fence_after();
       const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + acc * acc_cols;
-      float* stat_dst = stats ? stats + (((int64_t)n * stat_slots + (hq * 2 + (int)rank) * 4 + q) * groups) * 2 : nullptr;
+      float* stat_dst = stats ? stats + (((int64_t)n * stat_slots + ((hq * nseg + sg) * 2 + (int)rank) * 4 + q) * groups) * 2 : nullptr;
 #pragma unroll 1
       for (int c = c_lo; c < c_hi; ++c) {
         uint32_t rr[32];
@@ -347,8 +356,10 @@ conv3x3_tc2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
         }
         tc::fence_proxy_async();
         __syncwarp();
+        // the second half of a tile row holds 30 pixels of the segment: where the image row goes on behind it, its box
+        // is 30 pixels long, so that the two junk rows are not written over the next segment's first pixels
         if (lane == 0 && row_ok && w0 < W) {
-          tc::tma_store_4d(&tmY, stg, c * 32, w0, h, n);
+          tc::tma_store_4d((nseg > 1 && (q & 1)) ? &tmY30 : &tmY, stg, c * 32, w0, h, n);
           tc::tma_store_commit();
         }
       }
@@ -380,10 +391,13 @@ size_t conv_smem_bytes(int c_in, int c_out) {
 
 }  // namespace
 
-int conv3x3_tc2_stat_slots(int64_t h) { return (int)((h + 2 * TILE_ROWS - 1) / (2 * TILE_ROWS)) * 2 * 4; }
+int conv3x3_tc2_stat_slots(int64_t h, int64_t w) {
+  return (int)(((h + 2 * TILE_ROWS - 1) / (2 * TILE_ROWS)) * ((w + SEG - 1) / SEG)) * 2 * 4;
+}
 
 bool conv3x3_tc2_supported(int64_t nb, int64_t h, int64_t w, int64_t c_in, int64_t c_out) {
-  if (nb < 1 || h < 1 || w < 1 || w > PITCH - 2) return false;
+  if (nb < 1 || h < 1 || w < 1) return false;
+  if (nb * ((h + 2 * TILE_ROWS - 1) / (2 * TILE_ROWS)) * ((w + SEG - 1) / SEG) > INT32_MAX) return false;
   if (c_in != 64 && c_in != 128) return false;
   if (c_out < 32 || c_out > 256 || c_out % 32) return false;
   return conv_smem_bytes((int)c_in, (int)c_out) <= 227 * 1024;
@@ -401,14 +415,16 @@ cudaError_t conv3x3_tc2_plan(ConvTcPlan* p, const void* x, const void* w, void* 
   }
   cudaError_t e = encode_tmap_2d_bf16(&p->tm_w, w, (uint64_t)c_out, (uint64_t)(9 * c_in), (uint64_t)(9 * c_in), (uint32_t)(c_out / 2), 64);
   if (e != cudaSuccess) return e;
-  e = encode_tmap_nhwc_bf16_store(&p->tm_y, y, (uint64_t)nb, (uint64_t)h, (uint64_t)wd, (uint64_t)c_out);
+  e = encode_tmap_nhwc_bf16_store(&p->tm_y, y, (uint64_t)nb, (uint64_t)h, (uint64_t)wd, (uint64_t)c_out, 32);
+  if (e != cudaSuccess) return e;
+  e = encode_tmap_nhwc_bf16_store(&p->tm_y30, y, (uint64_t)nb, (uint64_t)h, (uint64_t)wd, (uint64_t)c_out, 30);
   if (e != cudaSuccess) return e;
   p->y = y;
   p->stats = nullptr;
   p->cpg = 0;
   p->nb = (int)nb; p->h = (int)h; p->w = (int)wd; p->c_in = (int)c_in; p->c_out = (int)c_out;
   p->epi = epi;
-  const int64_t tiles = nb * ((h + 2 * TILE_ROWS - 1) / (2 * TILE_ROWS));
+  const int64_t tiles = nb * ((h + 2 * TILE_ROWS - 1) / (2 * TILE_ROWS)) * ((wd + SEG - 1) / SEG);
   const int64_t clusters = tiles < sm_count / 2 ? tiles : sm_count / 2;
   p->grid = (int)(2 * clusters);
   p->smem = conv_smem_bytes((int)c_in, (int)c_out);
@@ -418,14 +434,24 @@ cudaError_t conv3x3_tc2_plan(ConvTcPlan* p, const void* x, const void* w, void* 
 cudaError_t launch_conv3x3_tc2(const ConvTcPlan& p, cudaStream_t s) {
   static SmemOptIn opt_in;
   {
-    cudaError_t e = opt_in.ensure(p.smem, conv3x3_tc2_kernel<1>, conv3x3_tc2_kernel<2>);
+    cudaError_t e = opt_in.ensure(p.smem, conv3x3_tc2_kernel<1, false>, conv3x3_tc2_kernel<2, false>, conv3x3_tc2_kernel<1, true>,
+                                  conv3x3_tc2_kernel<2, true>);
     if (e != cudaSuccess) return e;
   }
   LaunchCfg lc(PDL_CONV, dim3((unsigned)p.grid), dim3(THREADS), p.smem, s, 2);
   cudaLaunchConfig_t& cfg = lc.cfg;
   unsigned int* status = kernel_status_ptr();
-  if (p.c_in == 64) return cudaLaunchKernelEx(&cfg, conv3x3_tc2_kernel<1>, p.tm_x, p.tm_w, p.tm_y, p.nb, p.h, p.w, p.c_out, p.epi, p.stats, p.cpg, status);
-  return cudaLaunchKernelEx(&cfg, conv3x3_tc2_kernel<2>, p.tm_x, p.tm_w, p.tm_y, p.nb, p.h, p.w, p.c_out, p.epi, p.stats, p.cpg, status);
+  const bool wide = p.w > SEG;
+#define MK_CONV_LAUNCH(CB_, WIDE_)                                                                                                          \
+  return cudaLaunchKernelEx(&cfg, conv3x3_tc2_kernel<CB_, WIDE_>, p.tm_x, p.tm_w, p.tm_y, p.tm_y30, p.nb, p.h, p.w, p.c_out, p.epi, p.stats, \
+                            p.cpg, status)
+  if (p.c_in == 64) {
+    if (wide) MK_CONV_LAUNCH(1, true);
+    MK_CONV_LAUNCH(1, false);
+  }
+  if (wide) MK_CONV_LAUNCH(2, true);
+  MK_CONV_LAUNCH(2, false);
+#undef MK_CONV_LAUNCH
 }
 
 }  // namespace mk

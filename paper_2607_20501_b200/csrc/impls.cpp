@@ -504,7 +504,7 @@ bool conv_gn_tc2_match(const Module& m, int lo, int hi) {
 size_t conv_gn_tc2_scratch(const Module& m, int, int hi) {
   const mk_tensor_spec& s = m.vspec(m.ops[hi - 1].out_id);
   const size_t act = (size_t)s.shape[0] * s.shape[1] * s.shape[2] * s.shape[3] * 2;
-  const size_t st = (size_t)s.shape[0] * conv3x3_tc2_stat_slots(s.shape[1]) * m.ops[hi - 1].d.i[0] * 2 * sizeof(float);
+  const size_t st = (size_t)s.shape[0] * conv3x3_tc2_stat_slots(s.shape[1], s.shape[2]) * m.ops[hi - 1].d.i[0] * 2 * sizeof(float);
   return align_up(act, 1024) + st;
 }
 mk_status conv_gn_tc2_emit(const Module& m, int lo, int hi, const Resolved& r, std::vector<Launch>& out, std::string& err) {
@@ -519,7 +519,7 @@ mk_status conv_gn_tc2_emit(const Module& m, int lo, int hi, const Resolved& r, s
   const int groups = gn.d.i[0];
   char* act = (char*)r.scratch;
   float* stats = (float*)(act + align_up((size_t)nb * hw * c * 2, 1024));
-  const int slots = conv3x3_tc2_stat_slots(ys.shape[1]);
+  const int slots = conv3x3_tc2_stat_slots(ys.shape[1], ys.shape[2]);
   auto plan = std::make_shared<ConvTcPlan>();
   cudaError_t e = conv3x3_tc2_plan(plan.get(), r.value_ptr[op.in_id[0]], op.param[0].ptr, act, xs.shape[0], xs.shape[1], xs.shape[2],
                                    xs.shape[3], op.d.i[0], p, m.ctx->sm_count);

@@ -456,7 +456,7 @@ cudaError_t encode_tmap_bf16(CUtensorMap* out, const void* base, int rank, const
 cudaError_t encode_tmap_2d_u8(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows);
 // bf16 [rows, cols] output map for the epilogue's bulk stores: box 32 x 32, 64-byte swizzle
 cudaError_t encode_tmap_2d_bf16_store(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint64_t ld);
-cudaError_t encode_tmap_nhwc_bf16_store(CUtensorMap* out, const void* base, uint64_t nb, uint64_t h, uint64_t w, uint64_t c);
+cudaError_t encode_tmap_nhwc_bf16_store(CUtensorMap* out, const void* base, uint64_t nb, uint64_t h, uint64_t w, uint64_t c, uint32_t box_pixels);
 cudaError_t encode_tmap_2d_f32_store(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint64_t ld);
 
 }  // namespace mk

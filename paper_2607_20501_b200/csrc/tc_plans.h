@@ -129,9 +129,9 @@ cudaError_t launch_gemm_fp8_tc2(const GemmFp8Plan& p, cudaStream_t s);
 namespace mk {
 struct ConvTcPlan {
   CUtensorMap tm_x, tm_w;
-  CUtensorMap tm_y;         // the output, for the epilogue's bulk stores
+  CUtensorMap tm_y, tm_y30; // the output, for the epilogue's bulk stores: boxes of 32 and of 30 pixels
   void* y = nullptr;
-  // optional GroupNorm partial sums of the stored output: float [nb][conv3x3_tc2_stat_slots(h)][c_out / cpg][2]
+  // optional GroupNorm partial sums of the stored output: float [nb][conv3x3_tc2_stat_slots(h, w)][c_out / cpg][2]
   // = (sum, sum of squares) per group of cpg adjacent channels (cpg in {4, 8, 16, 32}); null: none
   float* stats = nullptr;
   int cpg = 0;
@@ -141,10 +141,10 @@ struct ConvTcPlan {
   EpiProgram epi;
 };
 // NHWC bf16 3x3 conv (stride 1, pad 1) + elementwise tail; weights [C_out, 3, 3, C_in].
-// Supported: C_in in {64, 128}, C_out multiple of 32 up to 256, W <= 62, and half the weights
+// Supported: C_in in {64, 128}, C_out multiple of 32 up to 256, any H and W, and half the weights
 // plus two input patches must fit one SM's shared memory.
 bool conv3x3_tc2_supported(int64_t nb, int64_t h, int64_t w, int64_t c_in, int64_t c_out);
-int conv3x3_tc2_stat_slots(int64_t h);
+int conv3x3_tc2_stat_slots(int64_t h, int64_t w);
 cudaError_t conv3x3_tc2_plan(ConvTcPlan* p, const void* x, const void* w, void* y, int64_t nb, int64_t h, int64_t wd, int64_t c_in,
                              int64_t c_out, const EpiProgram& epi, int sm_count);
 cudaError_t launch_conv3x3_tc2(const ConvTcPlan& p, cudaStream_t s);

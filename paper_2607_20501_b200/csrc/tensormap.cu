@@ -85,15 +85,15 @@ cudaError_t encode_tmap_2d_bf16_store(CUtensorMap* out, const void* base, uint64
   return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
-// Output map of an NHWC bf16 tensor for the convolution's bulk stores: box 32 channels (64 bytes) x 32 pixels of one
-// image row, 64-byte swizzle.  Pixels past the row's end and rows past the image are clipped by the copy engine.
-cudaError_t encode_tmap_nhwc_bf16_store(CUtensorMap* out, const void* base, uint64_t nb, uint64_t h, uint64_t w, uint64_t c) {
+// Output map of an NHWC bf16 tensor for the convolution's bulk stores: box 32 channels (64 bytes) x box_pixels (<= 32)
+// pixels of one image row, 64-byte swizzle.  Pixels past the row's end and rows past the image are clipped by the copy engine.
+cudaError_t encode_tmap_nhwc_bf16_store(CUtensorMap* out, const void* base, uint64_t nb, uint64_t h, uint64_t w, uint64_t c, uint32_t box_pixels) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return cudaErrorNotSupported;
   if (((uintptr_t)base & 15) != 0 || (c * 2) % 16) return cudaErrorInvalidValue;
   cuuint64_t gdim[4] = {c, w, h, nb};
   cuuint64_t gstr[3] = {c * 2, w * c * 2, h * w * c * 2};
-  cuuint32_t bdim[4] = {32, 32, 1, 1};
+  cuuint32_t bdim[4] = {32, box_pixels, 1, 1};
   cuuint32_t estr[4] = {1, 1, 1, 1};
   CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), gdim, gstr, bdim, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                   CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);

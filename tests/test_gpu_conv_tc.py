@@ -23,8 +23,11 @@ def _bf16_round(x):
 
 # the last two: more tiles than CTA pairs with a last wave of at most half the pairs, which runs as units of half the
 # output channels each (320 and 150 tiles on 74 pairs; C_out 128 and 256)
+# ... and image rows wider than one tile's 62 pixels: 63 (a second segment of one pixel), 124 (two full segments), 125,
+# 200 (a ragged fourth), 112 x 112 feature maps
 SHAPES = [(1, 4, 4, 64, 32), (2, 8, 8, 64, 64), (3, 9, 7, 128, 128), (2, 13, 62, 64, 96), (1, 56, 56, 128, 128),
-          (5, 6, 10, 64, 256), (20, 64, 20, 64, 128), (25, 24, 9, 64, 256)]
+          (5, 6, 10, 64, 256), (20, 64, 20, 64, 128), (25, 24, 9, 64, 256),
+          (1, 8, 63, 64, 64), (2, 5, 124, 64, 32), (1, 9, 125, 128, 128), (1, 6, 200, 64, 96), (2, 112, 112, 64, 64)]
 
 
 @pytest.mark.parametrize("nb,h,w,c,co", SHAPES)
@@ -53,11 +56,12 @@ def test_conv_chain_matches_the_oracle(ctx, nb, h, w, c, co):
 
 
 @pytest.mark.parametrize("nb,h,w,c,co,g", [(2, 8, 8, 64, 64, 16), (3, 9, 7, 128, 128, 32), (2, 13, 62, 64, 128, 16), (1, 6, 10, 64, 256, 16),
-                                           (2, 5, 33, 64, 32, 1), (4, 56, 56, 128, 128, 32), (20, 64, 20, 64, 128, 32), (25, 24, 9, 64, 256, 8)])
+                                           (2, 5, 33, 64, 32, 1), (4, 56, 56, 128, 128, 32), (20, 64, 20, 64, 128, 32), (25, 24, 9, 64, 256, 8),
+                                           (1, 8, 63, 64, 64, 16), (2, 7, 130, 128, 128, 32), (1, 112, 112, 64, 64, 8)])
 def test_groupnorm_statistics_from_the_conv_epilogue(ctx, nb, h, w, c, co, g):
     """The fused form: the convolution's epilogue leaves per-(image, group) partial sums of what it stores
     and the normalisation reads only those (4, 8, 16 and 32 channels per group; image heights that do not
-    fill the last tile; widths that leave junk rows in the tile).  Swapped against the two-pass GroupNorm."""
+    fill the last tile; widths that leave junk rows in the tile; image rows of several segments).  Swapped against the two-pass GroupNorm."""
     wl = W.c3(2, NB=nb, H=h, W=w, C=c, CO=co, G=g)
     ref, _ = oracle(wl, [0])
     dw, out = run_gpu(ctx, wl, wl.partitions["fused"])
