@@ -107,7 +107,7 @@ __device__ __forceinline__ void chunk_stats(const float (&v)[32], bool valid, in
     a[2 * g + 1] = sq;
   }
   fold_rows<NV>(a, lane, 16);
-  constexpr int LOG = NV == 16 ? 4 : NV == 8 ? 3 : NV == 4 ? 2 : 1;
+  constexpr int LOG = NV == 32 ? 5 : NV == 16 ? 4 : NV == 8 ? 3 : NV == 4 ? 2 : 1;
   if ((lane & ((1 << (5 - LOG)) - 1)) == 0) dst[lane >> (5 - LOG)] = a[0];
 }
 
@@ -331,6 +331,7 @@ conv3x3_tc2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
         if (stats) {
           float* d = stat_dst + (c * 32 / cpg) * 2;
           switch (cpg) {
+            case 2: chunk_stats<2>(v, my_row >= 0, lane, d); break;
             case 4: chunk_stats<4>(v, my_row >= 0, lane, d); break;
             case 8: chunk_stats<8>(v, my_row >= 0, lane, d); break;
             case 16: chunk_stats<16>(v, my_row >= 0, lane, d); break;

@@ -498,7 +498,7 @@ bool conv_gn_tc2_match(const Module& m, int lo, int hi) {
   const int groups = m.ops[hi - 1].d.i[0];
   if (groups < 1 || c % groups) return false;
   const int64_t cpg = c / groups;
-  if (cpg != 4 && cpg != 8 && cpg != 16 && cpg != 32) return false;
+  if (cpg != 2 && cpg != 4 && cpg != 8 && cpg != 16 && cpg != 32) return false;
   return groupnorm_apply_partials_supported(dt(m), c, groups);
 }
 size_t conv_gn_tc2_scratch(const Module& m, int, int hi) {

@@ -132,7 +132,7 @@ struct ConvTcPlan {
   CUtensorMap tm_y, tm_y30; // the output, for the epilogue's bulk stores: boxes of 32 and of 30 pixels
   void* y = nullptr;
   // optional GroupNorm partial sums of the stored output: float [nb][conv3x3_tc2_stat_slots(h, w)][c_out / cpg][2]
-  // = (sum, sum of squares) per group of cpg adjacent channels (cpg in {4, 8, 16, 32}); null: none
+  // = (sum, sum of squares) per group of cpg adjacent channels (cpg in {2, 4, 8, 16, 32}); null: none
   float* stats = nullptr;
   int cpg = 0;
   int nb = 0, h = 0, w = 0, c_in = 0, c_out = 0;

@@ -57,10 +57,11 @@ def test_conv_chain_matches_the_oracle(ctx, nb, h, w, c, co):
 
 @pytest.mark.parametrize("nb,h,w,c,co,g", [(2, 8, 8, 64, 64, 16), (3, 9, 7, 128, 128, 32), (2, 13, 62, 64, 128, 16), (1, 6, 10, 64, 256, 16),
                                            (2, 5, 33, 64, 32, 1), (4, 56, 56, 128, 128, 32), (20, 64, 20, 64, 128, 32), (25, 24, 9, 64, 256, 8),
-                                           (1, 8, 63, 64, 64, 16), (2, 7, 130, 128, 128, 32), (1, 112, 112, 64, 64, 8)])
+                                           (1, 8, 63, 64, 64, 16), (2, 7, 130, 128, 128, 32), (1, 112, 112, 64, 64, 8),
+                                           (3, 10, 10, 64, 64, 32), (2, 9, 70, 128, 32, 16)])
 def test_groupnorm_statistics_from_the_conv_epilogue(ctx, nb, h, w, c, co, g):
     """The fused form: the convolution's epilogue leaves per-(image, group) partial sums of what it stores
-    and the normalisation reads only those (4, 8, 16 and 32 channels per group; image heights that do not
+    and the normalisation reads only those (2, 4, 8, 16 and 32 channels per group; image heights that do not
     fill the last tile; widths that leave junk rows in the tile; image rows of several segments).  Swapped against the two-pass GroupNorm."""
     wl = W.c3(2, NB=nb, H=h, W=w, C=c, CO=co, G=g)
     ref, _ = oracle(wl, [0])
