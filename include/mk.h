@@ -100,7 +100,7 @@ typedef struct mk_tensor_spec {
  *   CONV2D_3X3      NHWC cross-correlation, stride 1, zero pad 1; param 0 = W [C_out,3,3,C_in];
  *                                                       i[0] = C_out
  *   BIAS_ADD        y = x + b[last dim]                 param 0 = b
- *   RELU, GELU_TANH, SILU                               elementwise
+ *   RELU, GELU_TANH, GELU_ERF, SILU                     elementwise (GELU_ERF: 0.5 x (1 + erf(x / sqrt 2)), the exact form)
  *   SCALE           y = f[0] * x
  *   CLAMP           y = min(max(x, f[0]), f[1])
  *   RESIDUAL_ADD    y = x + in[1]                       (same shape).  i[0] = 1: the sum is stored as fp32
@@ -158,7 +158,8 @@ typedef enum {
   MK_OP_AVGPOOL2D = 17,
   MK_OP_MAXPOOL2D = 18,
   MK_OP_LPPOOL2D = 19,
-  MK_OP_LINEAR_FP8 = 20
+  MK_OP_LINEAR_FP8 = 20,
+  MK_OP_GELU_ERF = 21
 } mk_op_kind;
 
 /* Value numbering: module input k has id k; operator j produces id n_inputs + j.

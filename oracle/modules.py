@@ -33,6 +33,8 @@ def apply_op(op, vals, params):
         return O.relu(ins[0])
     if kind == "gelu_tanh":
         return O.gelu_tanh(ins[0])
+    if kind == "gelu_erf":
+        return O.gelu_erf(ins[0])
     if kind == "silu":
         return O.silu(ins[0])
     if kind == "scale":

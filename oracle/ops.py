@@ -103,6 +103,14 @@ def gelu_tanh(x):
     return 0.5 * x * (1.0 + np.tanh(GELU_C0 * (x + GELU_C1 * x * x * x)))
 
 
+def gelu_erf(x):
+    """0.5 * x * (1 + erf(x / sqrt 2)): the exact GELU the tanh form approximates (paper, appendix on numerical
+    precision: erf is the exact form)."""
+    import math
+    x = _f64(x)
+    return 0.5 * x * (1.0 + np.vectorize(math.erf, otypes=[np.float64])(x / math.sqrt(2.0)))
+
+
 def silu(x):
     """x / (1 + exp(-x))."""
     x = _f64(x)

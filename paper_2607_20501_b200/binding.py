@@ -31,7 +31,7 @@ MK_LAYOUT_ROW_MAJOR, MK_LAYOUT_TRANSPOSED = 0, 1
 MK_MAX_RANK = 4
 MK_PREV, MK_NONE = -1, -2
 OP = {
-    "linear": 1, "conv2d_3x3": 2, "bias_add": 3, "relu": 4, "gelu_tanh": 5, "silu": 6, "scale": 7,
+    "linear": 1, "conv2d_3x3": 2, "bias_add": 3, "relu": 4, "gelu_tanh": 5, "gelu_erf": 21, "silu": 6, "scale": 7,
     "clamp": 8, "residual_add": 9, "swiglu": 10, "layernorm": 11, "rmsnorm": 12, "groupnorm": 13,
     "softmax": 14, "attention_causal": 15, "attention": 16, "avgpool": 17, "maxpool": 18, "lppool": 19,
     "linear_fp8": 20,

@@ -34,6 +34,7 @@ bool is_eltwise(int32_t kind) {
     case MK_OP_BIAS_ADD:
     case MK_OP_RELU:
     case MK_OP_GELU_TANH:
+    case MK_OP_GELU_ERF:
     case MK_OP_SILU:
     case MK_OP_SCALE:
     case MK_OP_CLAMP:
@@ -129,6 +130,7 @@ mk_status infer_shapes(Module& m, std::string& err) {
       case MK_OP_BIAS_ADD:
       case MK_OP_RELU:
       case MK_OP_GELU_TANH:
+      case MK_OP_GELU_ERF:
       case MK_OP_SILU:
       case MK_OP_SCALE:
         break;
@@ -228,8 +230,8 @@ void contract_of(const Module& m, int lo, int hi, std::vector<int>& in_ids, std:
 static std::string kind_name(int32_t k) {
   static const char* names[] = {"?", "LINEAR", "CONV2D_3X3", "BIAS_ADD", "RELU", "GELU_TANH", "SILU", "SCALE", "CLAMP",
                                 "RESIDUAL_ADD", "SWIGLU", "LAYERNORM", "RMSNORM", "GROUPNORM", "SOFTMAX", "ATTENTION_CAUSAL", "ATTENTION",
-                                "AVGPOOL2D", "MAXPOOL2D", "LPPOOL2D"};
-  return (k >= 1 && k <= 19) ? names[k] : "?";
+                                "AVGPOOL2D", "MAXPOOL2D", "LPPOOL2D", "LINEAR_FP8", "GELU_ERF"};
+  return (k >= 1 && k <= 21) ? names[k] : "?";
 }
 
 mk_status default_binding(const Module& m, int lo, int hi, Binding& out, std::string& err) {
@@ -414,6 +416,7 @@ mk_status build_epi(const Module& m, int lo, int hi, const Resolved& r, EpiProgr
         e.kind = EPI_BIAS; e.ptr = op.param[0].ptr; e.ptr_dtype = p.dtype; break;
       case MK_OP_RELU: e.kind = EPI_RELU; break;
       case MK_OP_GELU_TANH: e.kind = EPI_GELU_TANH; break;
+      case MK_OP_GELU_ERF: e.kind = EPI_GELU_ERF; break;
       case MK_OP_SILU: e.kind = EPI_SILU; break;
       case MK_OP_SCALE: e.kind = EPI_SCALE; e.a = (float)op.d.f[0]; break;
       case MK_OP_CLAMP: e.kind = EPI_CLAMP; e.a = (float)op.d.f[0]; e.b = (float)op.d.f[1]; break;

@@ -135,6 +135,7 @@ __device__ __forceinline__ float gelu_tanh_f(float x) {
   const float u = 0.7978845608028654f * (x + 0.044715f * x * x * x);
   return 0.5f * x * (1.0f + tanhf(u));
 }
+__device__ __forceinline__ float gelu_erf_f(float x) { return 0.5f * x * (1.0f + erff(x * 0.7071067811865476f)); }
 __device__ __forceinline__ float silu_f(float x) { return x / (1.0f + __expf(-x)); }
 // hardware tanh (relative error ~2^-11): only where the result is stored as bf16 (half-ulp 2^-9)
 __device__ __forceinline__ float gelu_tanh_bf16_f(float x) {
@@ -157,6 +158,7 @@ __device__ __forceinline__ float epi_apply(const EpiProgram& p, float v, int64_t
       case EPI_BIAS: v += epi_ptr_ld(o.ptr, p.dtype, col); break;
       case EPI_RELU: v = fmaxf(v, 0.0f); break;
       case EPI_GELU_TANH: v = gelu_tanh_f(v); break;
+      case EPI_GELU_ERF: v = gelu_erf_f(v); break;
       case EPI_SILU: v = silu_f(v); break;
       case EPI_SCALE: v *= o.a; break;
       case EPI_CLAMP: v = fminf(fmaxf(v, o.a), o.b); break;
@@ -216,6 +218,10 @@ __device__ __forceinline__ void epi_apply_vec(const EpiProgram& p, float (&v)[NV
       case EPI_GELU_TANH:
 #pragma unroll
         for (int j = 0; j < NV; ++j) v[j] = sizeof(T) == 2 ? gelu_tanh_bf16_f(v[j]) : gelu_tanh_f(v[j]);
+        break;
+      case EPI_GELU_ERF:
+#pragma unroll
+        for (int j = 0; j < NV; ++j) v[j] = gelu_erf_f(v[j]);
         break;
       case EPI_SILU:
 #pragma unroll

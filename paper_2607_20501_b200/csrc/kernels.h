@@ -23,7 +23,8 @@ enum EpiKind : int32_t {
   EPI_SILU = 4,
   EPI_SCALE = 5,     // v *= a
   EPI_CLAMP = 6,     // v = min(max(v, a), b)
-  EPI_RESIDUAL = 7   // v += res[row * ld + col]  ptr = residual tensor, ld = output width
+  EPI_RESIDUAL = 7,  // v += res[row * ld + col]  ptr = residual tensor, ld = output width
+  EPI_GELU_ERF = 8   // 0.5 v (1 + erf(v / sqrt 2))
 };
 constexpr int EPI_MAX = 8;
 struct EpiOp {

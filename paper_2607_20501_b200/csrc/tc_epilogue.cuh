@@ -102,6 +102,10 @@ __device__ __forceinline__ void epi32(const EpiProgram& p, float (&v)[32], int64
 #pragma unroll
         for (int j = 0; j < 32; ++j) v[j] = gelu_fast(v[j]);
         break;
+      case EPI_GELU_ERF:
+#pragma unroll 4
+        for (int j = 0; j < 32; ++j) v[j] = gelu_erf_f(v[j]);
+        break;
       case EPI_SILU:
 #pragma unroll
         for (int j = 0; j < 32; ++j) v[j] = silu_fast(v[j]);

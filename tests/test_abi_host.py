@@ -237,8 +237,8 @@ def test_unmasked_attention_and_the_encoder_block_on_the_host(ctx):
     assert m.value_spec("x2_1") == (B.MK_BF16, (48, 256), 0)
     m.set_decomposition(w.partitions["fused_tails"])
     assert m.n_sub() == 14
-    # the attention submodule: both kernels that know the unmasked operator, not the one-tile causal kernel
-    assert m.impls(1) == ["attention_tc2", "attention_simt"]
+    # the attention submodule: every attention kernel knows the unmasked operator
+    assert m.impls(1) == ["attention_tc2", "attention_tc", "attention_simt"]
     ins, outs = m.contract(1)
     vid = m.value_id
     assert [n for n, _ in ins] == [vid["qkv_0"]] and [n for n, _ in outs] == [vid["att_0"]]
@@ -246,11 +246,15 @@ def test_unmasked_attention_and_the_encoder_block_on_the_host(ctx):
     ins, outs = m.contract(2)
     assert sorted(n for n, _ in ins) == sorted([vid["att_0"], vid["x"]]) and [n for n, _ in outs] == [vid["r1_0"]]
     assert m.bound_impl(2) == "gemm_tc" and m.bound_impl(3) == "rowop"      # 48 rows: the one-SM form
-    # head_dim 64: only the plain-ALU kernel is legal
+    # head_dim 64: the one-tile tensor-core kernel and the plain-ALU kernel; head_dim 32: the plain-ALU kernel alone
     w64 = W.c6(0, B=1, S=8, E=128, H=2, F=32, L=1)
     m64 = _mod(ctx, w64)
     m64.set_decomposition(w64.partitions["fused_tails"])
-    assert m64.impls(1) == ["attention_simt"]
+    assert m64.impls(1) == ["attention_tc", "attention_simt"]
+    w32 = W.c6(0, B=1, S=8, E=128, H=4, F=32, L=1)
+    m32 = _mod(ctx, w32)
+    m32.set_decomposition(w32.partitions["fused_tails"])
+    assert m32.impls(1) == ["attention_simt"]
     # a packed tensor of the wrong width is rejected at creation
     ops = [dict(o, attrs=dict(o["attrs"])) for o in w.ops]
     ops[2]["attrs"]["heads"] = 3

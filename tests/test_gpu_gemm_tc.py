@@ -87,3 +87,24 @@ def test_swiglu_and_residual_tails(ctx, t, e, f, impl):
     ref, inter = oracle(w, None)
     dw, _ = run_gpu(ctx, w, [0, 2], binds={0: impl, 1: impl}, keep=True)
     assert_parity(to_host_f64(dw.intermediate("h")), inter["h"], "bf16", "pairing")
+
+
+@pytest.mark.parametrize("dtype,impls", [("bf16", ("gemm_tc2", "gemm_tc", "gemm_simt")), ("f32", ("gemm_simt",))])
+def test_exact_gelu_in_the_epilogue(ctx, dtype, impls):
+    """LINEAR + bias + GELU_ERF (0.5 x (1 + erf(x / sqrt 2))) as one submodule on every GEMM kernel, and split after
+    the bias so that the activation runs as an elementwise pass."""
+    m, k, n = 300, 200, 264
+    rng = np.random.default_rng(9)
+    w = G.Workload("ge", dtype)
+    w.inputs["x"] = G.make("x", dtype, rng.standard_normal((m, k)).astype(np.float32))
+    w.params["W"] = G.make("W", dtype, (rng.standard_normal((k, n)) * (1.0 / k) ** 0.5 * 2).astype(np.float32))
+    w.params["b"] = G.make("b", dtype, (0.3 * rng.standard_normal(n)).astype(np.float32))
+    w.ops = [G._op("linear", "y0", ["x"], {"w": "W"}, n=n), G._op("bias_add", "y1", ["y0"], {"b": "b"}),
+             G._op("gelu_erf", "y", ["y1"])]
+    ref, _ = oracle(w, [0])
+    for impl in impls:
+        dw, out = run_gpu(ctx, w, [0], binds={0: impl})
+        assert dw.module.bound_impl(0) == impl
+        assert_parity(out, ref, dtype, f"{impl} fused")
+    _, out = run_gpu(ctx, w, [0, 2])
+    assert_parity(out, ref, dtype, "activation as its own pass")

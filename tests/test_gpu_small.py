@@ -167,9 +167,9 @@ def test_elementwise_ragged_and_swiglu(ctx, dtype):
         w.ops = [G._op("swiglu", "h", ["x"]), G._op("bias_add", "h1", ["h"], {"b": "b"}),
                  G._op("silu", "h2", ["h1"]), G._op("residual_add", "h3", ["h2", "r"]),
                  G._op("gelu_tanh", "h4", ["h3"]), G._op("scale", "h5", ["h4"], s=-1.5),
-                 G._op("clamp", "h6", ["h5"], lo=-0.75, hi=2.0), G._op("relu", "y", ["h6"])]
+                 G._op("clamp", "h6", ["h5"], lo=-0.75, hi=2.0), G._op("gelu_erf", "h7", ["h6"]), G._op("relu", "y", ["h7"])]
         ref, _ = oracle(w, [0])
-        for cuts in ([0], [0, 1, 4], list(range(8))):
+        for cuts in ([0], [0, 1, 4], list(range(9))):
             _, out = run_gpu(ctx, w, cuts)
             assert_parity(out, ref, dtype, f"{rows}x{cols} {cuts}")
 

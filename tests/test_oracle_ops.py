@@ -69,6 +69,26 @@ def test_bias_relu_scale_clamp_residual():
     assert np.array_equal(O.residual_add(x, -x), np.zeros_like(x))
 
 
+def test_gelu_erf_pins():
+    """The exact GELU is x times the standard normal's distribution function: pinned against scipy's normal CDF and
+    torch's own exact GELU (neither uses the oracle's erf call), the odd-part identity, the tails, and the value at 1."""
+    from scipy.stats import norm
+    x = np.linspace(-6, 6, 2001)
+    g = O.gelu_erf(x)
+    assert O.gelu_erf(np.array([0.0]))[0] == 0.0
+    assert np.allclose(g, x * norm.cdf(x), rtol=1e-13, atol=1e-15)
+    assert np.allclose(g, torch.nn.functional.gelu(torch.from_numpy(x)).numpy(), rtol=1e-13, atol=1e-15)
+    assert np.allclose(g - O.gelu_erf(-x), x, rtol=0, atol=1e-14)
+    assert abs(O.gelu_erf(np.array([1.0]))[0] - 0.8413447460685429) < 1e-15          # Phi(1)
+    assert abs(O.gelu_erf(np.array([10.0]))[0] - 10.0) < 1e-12 and abs(O.gelu_erf(np.array([-10.0]))[0]) < 1e-12
+    # not the tanh form (up to 5e-4 apart) and not the sigmoid form
+    assert 1e-5 < np.abs(g - O.gelu_tanh(x)).max() < 1e-3
+    assert np.abs(g - x / (1.0 + np.exp(-1.702 * x))).max() > 5e-3
+    # minimum near x = -0.7518 with value -0.1700 (a sign slip in the erf argument moves it to +0.75)
+    i = int(np.argmin(g))
+    assert abs(x[i] + 0.7518) < 0.01 and abs(g[i] + 0.16997) < 1e-4
+
+
 def test_gelu_tanh_pins():
     x = np.linspace(-6, 6, 2001)
     g = O.gelu_tanh(x)
