@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the composed forward (one JSON line on stdout).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload all|c1..c7]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload all|c1..c9]
 
 A step is one composed forward of the workload's module (every submodule of its default
 decomposition) over one batch of seeded synthetic input.  With no --workload the run covers the
@@ -44,7 +44,7 @@ NCU_TRAFFIC_BYTES = {"c2": 89.9e6,            # profiles/gemm_tc2_c2.md
                      "c4": 8 * 52.2e6,         # profiles/attention_tc2_c4.md
                      "c5": 259.7e6}            # profiles/gemm_tc2_decoder_c5.md
 
-DEFAULT_STEPS = {"c1": 2000, "c2": 200, "c3": 400, "c4": 100, "c5": 50, "c6": 100, "c7": 400, "c8": 200}
+DEFAULT_STEPS = {"c1": 2000, "c2": 200, "c3": 400, "c4": 100, "c5": 50, "c6": 100, "c7": 400, "c8": 200, "c9": 200}
 
 
 def full_workload(name, seed=0, batch=None, only_ops=None):
@@ -54,7 +54,7 @@ def full_workload(name, seed=0, batch=None, only_ops=None):
     kw = {}
     if batch is not None:
         kw = {"c1": {"M": batch}, "c2": {"M": batch}, "c3": {"NB": batch}, "c4": {"B": batch}, "c5": {"B": batch},
-              "c6": {"B": batch}, "c7": {"NB": batch}, "c8": {"M": batch}}[name]
+              "c6": {"B": batch}, "c7": {"NB": batch}, "c8": {"M": batch}, "c9": {"NB": batch}}[name]
     w = W.generate.WORKLOADS[name](seed, **kw)
     if only_ops is not None:
         w.ops = w.ops[:only_ops]
@@ -154,7 +154,7 @@ def oracle_sample(name, w, budget_s=12.0):
                 s.inputs[k] = Tensor(k, w.inputs[k].dtype, w.inputs[k].store[:rows])
             total = w.inputs["xq"].shape[0]
             what = f"first {rows} of {total} rows of X"
-        elif name in ("c3", "c7"):
+        elif name in ("c3", "c7", "c9"):
             s.inputs["x"] = Tensor("x", w.dtype, w.inputs["x"].store[:frac_units])
             total = w.inputs["x"].shape[0]
             what = f"first {frac_units} of {total} images"
@@ -175,7 +175,7 @@ def oracle_sample(name, w, budget_s=12.0):
             what = f"first {frac_units} of {total} batch elements"
         return s, total, what
 
-    probe_units = {"c1": 64, "c2": 64, "c3": 1, "c4": 1, "c5": 1, "c6": 1, "c7": 1, "c8": 64}[name]
+    probe_units = {"c1": 64, "c2": 64, "c3": 1, "c4": 1, "c5": 1, "c6": 1, "c7": 1, "c8": 64, "c9": 1}[name]
     s, total, _ = sub(probe_units)
     t0 = time.perf_counter()
     OM.run_workload(s, [0])
@@ -214,7 +214,7 @@ def submodule_work(w, module):
             _, xs, _ = module.value_spec(op["in"][0])
             _, ys, _ = module.value_spec(op["out"])
             if op["kind"] in ("linear", "linear_fp8"):
-                fl += 2.0 * xs[0] * xs[1] * op["attrs"]["n"]
+                fl += 2.0 * float(np.prod(xs)) * op["attrs"]["n"]
             elif op["kind"] == "conv2d_3x3":
                 fl += 2.0 * xs[0] * xs[1] * xs[2] * 9 * xs[3] * op["attrs"]["c_out"]
             elif op["kind"] in ("attention_causal", "attention"):
@@ -494,7 +494,7 @@ def measure_one(name, args, steps, ctx, rank, local, world, cpu_seconds):
     # (time, share, algorithmic work, roofline fraction of that subkernel)
     breakdown = None
     dominant = None
-    split_name = {"c1": "split", "c2": "split", "c3": "split2", "c4": "split3", "c5": "fused_tails", "c6": "fused_tails", "c7": "split2"}.get(name)
+    split_name = {"c1": "split", "c2": "split", "c3": "split2", "c4": "split3", "c5": "fused_tails", "c6": "fused_tails", "c7": "split2", "c9": "split3"}.get(name)
     if rank == 0 and split_name in w.partitions:
         pk_ = peaks()
         dw = sets[0]
@@ -699,7 +699,7 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default=None, choices=["all", "c1", "c2", "c3", "c4", "c5", "c6", "c7", "c8"],
+    ap.add_argument("--workload", default=None, choices=["all", "c1", "c2", "c3", "c4", "c5", "c6", "c7", "c8", "c9"],
                     help="default: all five modules of the workload list for the GPU arm (headline C5), c5 for the reference arm")
     ap.add_argument("--decomposition", default=None)
     ap.add_argument("--batch", type=int, default=None, help="smaller leading batch dimension (profiler captures)")

@@ -95,8 +95,9 @@ typedef struct mk_tensor_spec {
 } mk_tensor_spec;
 
 /* Operator kinds.  "x" is the operator's first input.
- *   LINEAR          y[M,N] = x[M,K] @ W[K,N]            param 0 = W (logical [K,N]); i[0] = N,
- *                                                       i[1] = mk_layout of W's storage
+ *   LINEAR          y[..., N] = x[..., K] @ W[K,N]      param 0 = W (logical [K,N]); i[0] = N,
+ *                   (rank >= 2; the leading dimensions   i[1] = mk_layout of W's storage
+ *                   are rows: on NHWC a 1 x 1 convolution)
  *   CONV2D_3X3      NHWC cross-correlation, stride 1, zero pad 1; param 0 = W [C_out,3,3,C_in];
  *                                                       i[0] = C_out
  *   BIAS_ADD        y = x + b[last dim]                 param 0 = b

@@ -115,10 +115,14 @@ mk_status infer_shapes(Module& m, std::string& err) {
         break;
       }
       case MK_OP_LINEAR: {
-        if (x.rank != 2) { err = at + "LINEAR takes a rank-2 input"; return MK_ERR_SHAPE_MISMATCH; }
+        // any rank >= 2: the contraction runs over the last dimension, the leading ones are rows (on an NHWC tensor
+        // this is the 1 x 1 convolution)
+        if (x.rank < 2) { err = at + "LINEAR takes an input of rank 2 or more"; return MK_ERR_SHAPE_MISMATCH; }
         if (d.i[0] < 1) { err = at + "LINEAR needs i[0] = N >= 1"; return MK_ERR_INVALID_ARG; }
         if (d.i[1] != MK_LAYOUT_ROW_MAJOR && d.i[1] != MK_LAYOUT_TRANSPOSED) { err = at + "LINEAR i[1] must be an mk_layout"; return MK_ERR_INVALID_ARG; }
-        y = make_spec(dtype, {x.shape[0], d.i[0]});
+        y = x;
+        y.dtype = dtype;
+        y.shape[x.rank - 1] = d.i[0];
         break;
       }
       case MK_OP_CONV2D_3X3: {

@@ -173,7 +173,7 @@ mk_status gemm_simt_emit(const Module& m, int lo, int hi, const Resolved& r, std
   const void* w = op.param[0].ptr;
   void* y = r.value_ptr[m.ops[hi - 1].out_id];
   const mk_tensor_spec& xs = m.vspec(op.in_id[0]);
-  const int64_t M = xs.shape[0], K = xs.shape[1], N = last_dim(m.vspec(m.ops[hi - 1].out_id));
+  const int64_t M = rows_of(xs), K = last_dim(xs), N = last_dim(m.vspec(m.ops[hi - 1].out_id));
   const bool wt = op.d.i[1] == MK_LAYOUT_TRANSPOSED;
   const int d = dt(m), od = dt_of(m.vspec(m.ops[hi - 1].out_id));
   out.push_back([=](cudaStream_t s) { return launch_gemm_simt(d, od, a, w, wt, y, M, N, K, sw, p, s); });
@@ -187,7 +187,7 @@ bool gemm_tc_match(const Module& m, int lo, int hi) {
   if (m.dtype != MK_BF16) return false;
   const Op& op = m.ops[lo];
   if (op.d.i[1] != MK_LAYOUT_TRANSPOSED) return false;
-  const int64_t K = m.vspec(op.in_id[0]).shape[1];
+  const int64_t K = last_dim(m.vspec(op.in_id[0]));
   const int64_t N = last_dim(m.vspec(m.ops[hi - 1].out_id));
   return K % 8 == 0 && N % 8 == 0;
 }
@@ -199,7 +199,7 @@ mk_status gemm_tc_emit_impl(const Module& m, int lo, int hi, const Resolved& r, 
   if (st != MK_OK) return st;
   const Op& op = m.ops[lo];
   const mk_tensor_spec& xs = m.vspec(op.in_id[0]);
-  const int64_t M = xs.shape[0], K = xs.shape[1], N = last_dim(m.vspec(m.ops[hi - 1].out_id));
+  const int64_t M = rows_of(xs), K = last_dim(xs), N = last_dim(m.vspec(m.ops[hi - 1].out_id));
   auto plan = std::make_shared<GemmTcPlan>();
   const void* a = r.value_ptr[op.in_id[0]];
   void* y = r.value_ptr[m.ops[hi - 1].out_id];
@@ -216,7 +216,7 @@ mk_status gemm_tc_emit(const Module& m, int lo, int hi, const Resolved& r, std::
 }
 // two-SM form: worth it once a tile pair has more than one CTA's worth of rows
 bool gemm_tc2_match(const Module& m, int lo, int hi) {
-  return gemm_tc_match(m, lo, hi) && m.vspec(m.ops[lo].in_id[0]).shape[0] > 128;
+  return gemm_tc_match(m, lo, hi) && rows_of(m.vspec(m.ops[lo].in_id[0])) > 128;
 }
 mk_status gemm_tc2_emit(const Module& m, int lo, int hi, const Resolved& r, std::vector<Launch>& out, std::string& err) {
   return gemm_tc_emit_impl(m, lo, hi, r, out, err, true);
@@ -230,7 +230,7 @@ bool gemm_fp8_simt_match(const Module& m, int lo, int hi) { return gemm_fp8_shap
 bool gemm_fp8_tc2_match(const Module& m, int lo, int hi) {
   if (!gemm_fp8_shape(m, lo, hi) || m.ops[lo].d.i[1] != MK_LAYOUT_TRANSPOSED) return false;
   const mk_tensor_spec& xs = m.vspec(m.ops[lo].in_id[0]);
-  return gemm_fp8_tc2_supported(xs.shape[0], m.ops[lo].d.i[0], xs.shape[1]);
+  return gemm_fp8_tc2_supported(rows_of(xs), m.ops[lo].d.i[0], last_dim(xs));
 }
 mk_status gemm_fp8_emit_impl(const Module& m, int lo, int hi, const Resolved& r, std::vector<Launch>& out, std::string& err, bool tc) {
   EpiProgram p;
@@ -238,7 +238,7 @@ mk_status gemm_fp8_emit_impl(const Module& m, int lo, int hi, const Resolved& r,
   if (st != MK_OK) return st;
   const Op& op = m.ops[lo];
   const mk_tensor_spec& xs = m.vspec(op.in_id[0]);
-  const int64_t M = xs.shape[0], K = xs.shape[1], N = op.d.i[0];
+  const int64_t M = rows_of(xs), K = last_dim(xs), N = op.d.i[0];
   const void* xq = r.value_ptr[op.in_id[0]];
   const float* sx = (const float*)r.value_ptr[op.in_id[1]];
   const void* wq = op.param[0].ptr;
@@ -279,7 +279,7 @@ bool gemm_rownorm_tc2_match(const Module& m, int lo, int hi) {
 }
 size_t gemm_rownorm_tc2_scratch_fn(const Module& m, int lo, int hi) {
   const mk_tensor_spec& xs = m.vspec(m.ops[lo].in_id[0]);
-  return gemm_rownorm_tc2_scratch(xs.shape[0], last_dim(m.vspec(m.ops[hi - 1].out_id)));
+  return gemm_rownorm_tc2_scratch(rows_of(xs), last_dim(m.vspec(m.ops[hi - 1].out_id)));
 }
 mk_status gemm_rownorm_tc2_emit(const Module& m, int lo, int hi, const Resolved& r, std::vector<Launch>& out, std::string& err) {
   bool sw; int t;
@@ -290,7 +290,7 @@ mk_status gemm_rownorm_tc2_emit(const Module& m, int lo, int hi, const Resolved&
   const Op& op = m.ops[lo];
   const Op& nop = m.ops[hi - 1];
   const mk_tensor_spec& xs = m.vspec(op.in_id[0]);
-  const int64_t M = xs.shape[0], K = xs.shape[1], N = last_dim(m.vspec(nop.out_id));
+  const int64_t M = rows_of(xs), K = last_dim(xs), N = last_dim(m.vspec(nop.out_id));
   const void* g = nop.param[0].set ? nop.param[0].ptr : nullptr;
   const void* b = nop.param[1].set ? nop.param[1].ptr : nullptr;
   auto plan = std::make_shared<GemmTcPlan>();
@@ -326,7 +326,7 @@ bool gemm_rownorm_cl_match(const Module& m, int lo, int hi) {
   if (op.d.i[1] != MK_LAYOUT_TRANSPOSED || !all_eltwise(m, lo + 1, hi - 1)) return false;
   if (m.vspec(m.ops[hi - 1].out_id).dtype != MK_BF16) return false;
   const mk_tensor_spec& xs = m.vspec(op.in_id[0]);
-  return gemm_rownorm_cl_supported(xs.shape[0], last_dim(m.vspec(m.ops[hi - 1].out_id)), xs.shape[1]);
+  return gemm_rownorm_cl_supported(rows_of(xs), last_dim(m.vspec(m.ops[hi - 1].out_id)), last_dim(xs));
 }
 mk_status gemm_rownorm_cl_emit(const Module& m, int lo, int hi, const Resolved& r, std::vector<Launch>& out, std::string& err) {
   EpiProgram p;
@@ -335,7 +335,7 @@ mk_status gemm_rownorm_cl_emit(const Module& m, int lo, int hi, const Resolved& 
   const Op& op = m.ops[lo];
   const Op& nop = m.ops[hi - 1];
   const mk_tensor_spec& xs = m.vspec(op.in_id[0]);
-  const int64_t M = xs.shape[0], K = xs.shape[1], N = last_dim(m.vspec(nop.out_id));
+  const int64_t M = rows_of(xs), K = last_dim(xs), N = last_dim(m.vspec(nop.out_id));
   const void* g = nop.param[0].set ? nop.param[0].ptr : nullptr;
   const void* b = nop.param[1].set ? nop.param[1].ptr : nullptr;
   const int pre = m.ops[hi - 2].out_id;
@@ -381,7 +381,7 @@ bool gemm_prenorm_find(const Module& m, int lo, int hi, int* norm_at, bool* swig
   if (*swiglu2) ++t;
   if (!all_eltwise(m, t, hi) || !out_is_module_dtype(m, hi)) return false;
   const mk_tensor_spec& xs = m.vspec(l1.in_id[0]);
-  const int64_t M = xs.shape[0], K1 = xs.shape[1], N1 = l1.d.i[0], N2 = last_dim(m.vspec(m.ops[hi - 1].out_id));
+  const int64_t M = rows_of(xs), K1 = last_dim(xs), N1 = l1.d.i[0], N2 = last_dim(m.vspec(m.ops[hi - 1].out_id));
   if (M <= 128 || K1 % 8 || N1 % 8 || N2 % 8) return false;
   *norm_at = r;
   *tail2_lo = t;
@@ -392,7 +392,7 @@ bool gemm_prenorm_match(const Module& m, int lo, int hi) {
   return gemm_prenorm_find(m, lo, hi, &r, &sw, &t);
 }
 size_t gemm_prenorm_scratch_fn(const Module& m, int lo, int) {
-  return gemm_prenorm_scratch(m.vspec(m.ops[lo].in_id[0]).shape[0], m.ops[lo].d.i[0]);
+  return gemm_prenorm_scratch(rows_of(m.vspec(m.ops[lo].in_id[0])), m.ops[lo].d.i[0]);
 }
 mk_status gemm_prenorm_emit(const Module& m, int lo, int hi, const Resolved& r, std::vector<Launch>& out, std::string& err) {
   int nr, t2; bool sw2;
@@ -405,7 +405,7 @@ mk_status gemm_prenorm_emit(const Module& m, int lo, int hi, const Resolved& r, 
   const Op& nop = m.ops[nr];
   const Op& l2 = m.ops[nr + 1];
   const mk_tensor_spec& xs = m.vspec(l1.in_id[0]);
-  const int64_t M = xs.shape[0], K1 = xs.shape[1], N1 = l1.d.i[0], N2 = last_dim(m.vspec(m.ops[hi - 1].out_id));
+  const int64_t M = rows_of(xs), K1 = last_dim(xs), N1 = l1.d.i[0], N2 = last_dim(m.vspec(m.ops[hi - 1].out_id));
   const int pre = m.ops[nr - 1].out_id;
   auto plan1 = std::make_shared<GemmTcPlan>();
   auto plan2 = std::make_shared<GemmTcPlan>();
@@ -437,7 +437,7 @@ mk_status linear_rownorm_emit(const Module& m, int lo, int hi, const Resolved& r
   const void* w = op.param[0].ptr;
   void* y = r.value_ptr[nop.out_id];
   const mk_tensor_spec& xs = m.vspec(op.in_id[0]);
-  const int64_t M = xs.shape[0], K = xs.shape[1], N = op.d.i[0];
+  const int64_t M = rows_of(xs), K = last_dim(xs), N = op.d.i[0];
   const bool wt = op.d.i[1] == MK_LAYOUT_TRANSPOSED;
   const void* g = nop.param[0].set ? nop.param[0].ptr : nullptr;
   const void* b = nop.param[1].set ? nop.param[1].ptr : nullptr;

@@ -194,7 +194,24 @@ def _hand_c8(w):
     return v, "y2"
 
 
+def _hand_c9(w):
+    i, p = _widen(w)
+    v = {}
+    v["a0"] = O.linear(i["x"], p["W1"])            # a LINEAR over the channel dimension of an NHWC tensor
+    v["a1"] = O.bias_add(v["a0"], p["b1"])
+    v["a2"] = O.relu(v["a1"])
+    v["c0"] = O.conv2d_3x3_nhwc(v["a2"], p["Wc"])
+    v["c1"] = O.bias_add(v["c0"], p["b2"])
+    v["c2"] = O.relu(v["c1"])
+    v["d0"] = O.linear(v["c2"], p["W3"])
+    v["d1"] = O.bias_add(v["d0"], p["b3"])
+    v["d2"] = O.residual_add(v["d1"], i["x"])
+    v["y"] = O.relu(v["d2"])
+    return v, "y"
+
+
 HAND = {
+    "c9": (lambda s: W.c9(s, NB=2, H=5, W=6, C=16, CM=8), _hand_c9),
     "c8": (lambda s: W.c8(s, M=24, K=256, N=136, bias=True), _hand_c8),
     "c1": (lambda s: W.c1(s), _hand_c1),
     "c2": (lambda s: W.c2(s, M=48, K=64, N=40), _hand_c2),

@@ -16,6 +16,7 @@ from .generate import (  # noqa: F401
     c6,
     c7,
     c8,
+    c9,
     e4m3_bits_to_f64,
     f32_to_e4m3_bits,
     f32_to_bf16_bits,

@@ -433,4 +433,36 @@ def c8(seed=0, M=4096, K=7168, N=4096, bias=False) -> Workload:
     return w
 
 
-WORKLOADS = {"c1": c1, "c2": c2, "c3": c3, "c4": c4, "c5": c5, "c6": c6, "c7": c7, "c8": c8}
+# --------------------------------------------------------------------------
+# C9: a residual bottleneck block on an NHWC feature map: 1 x 1 convolution (C -> CM) + bias + ReLU, 3 x 3
+# convolution (CM -> CM) + bias + ReLU, 1 x 1 convolution (CM -> C) + bias + skip connection + ReLU.  A 1 x 1
+# convolution is a LINEAR over the channel dimension, so the whole block is three tensor-core launches.
+# --------------------------------------------------------------------------
+def c9(seed=0, NB=32, H=56, W=56, C=256, CM=64, dtype="bf16") -> Workload:
+    w = Workload("c9", dtype)
+    w.inputs["x"] = make("x", dtype, _normal(seed, 0, (NB, H, W, C)))
+    w.params["W1"] = make("W1", dtype, _normal(seed, 1, (C, CM), std=(1.0 / C) ** 0.5))
+    w.params["b1"] = make("b1", dtype, _normal(seed, 2, (CM,), std=0.02))
+    w.params["Wc"] = make("Wc", dtype, _normal(seed, 3, (CM, 3, 3, CM), std=(2.0 / (9 * CM)) ** 0.5))
+    w.params["b2"] = make("b2", dtype, _normal(seed, 4, (CM,), std=0.02))
+    w.params["W3"] = make("W3", dtype, _normal(seed, 5, (CM, C), std=(2.0 / CM) ** 0.5))
+    w.params["b3"] = make("b3", dtype, _normal(seed, 6, (C,), std=0.02))
+    w.ops = [
+        _op("linear", "a0", ["x"], {"w": "W1"}, n=CM),
+        _op("bias_add", "a1", ["a0"], {"b": "b1"}),
+        _op("relu", "a2", ["a1"]),
+        _op("conv2d_3x3", "c0", ["a2"], {"w": "Wc"}, c_out=CM),
+        _op("bias_add", "c1", ["c0"], {"b": "b2"}),
+        _op("relu", "c2", ["c1"]),
+        _op("linear", "d0", ["c2"], {"w": "W3"}, n=C),
+        _op("bias_add", "d1", ["d0"], {"b": "b3"}),
+        _op("residual_add", "d2", ["d1", "x"]),
+        _op("relu", "y", ["d2"]),
+    ]
+    w.partitions = {"fused": [0], "split3": [0, 3, 6], "per_op": list(range(10))}
+    w.flops = 2.0 * NB * H * W * (C * CM + 9 * CM * CM + CM * C)
+    w.min_bytes = 2 * (2 * NB * H * W * C + 2 * C * CM + 9 * CM * CM + 2 * CM + C)
+    return w
+
+
+WORKLOADS = {"c1": c1, "c2": c2, "c3": c3, "c4": c4, "c5": c5, "c6": c6, "c7": c7, "c8": c8, "c9": c9}
