@@ -4,12 +4,19 @@
 
 Objects are rebuilt when their source or any header under csrc/ or include/ is
 newer.  nvcc cross-compiles without a GPU.
+
+The build reads ptxas' resource report and refuses a library in which one of the
+hot tensor-core kernels keeps a large stack frame: their epilogues hold 32
+accumulator values per thread in registers, and a single run-time index into that
+array (a partially unrolled loop is enough) moves it to local memory and more than
+doubles the epilogue's time without changing any result.
 """
 from __future__ import annotations
 
 import concurrent.futures as cf
 import glob
 import os
+import re
 import subprocess
 import sys
 
@@ -27,6 +34,42 @@ FLAGS = [
 ]
 
 
+# (source file, pattern on the mangled kernel name, largest stack frame in bytes).  The default GEMM instantiations
+# are <CG, SWIGLU, NORM=0, RING, PRE=0>; the row-norm and prefix variants spill at their register cap by design.
+STACK_LIMITS = [
+    ("gemm_tc.cu", r"gemm_tc_kernelILi[12]ELb[01]ELb0ELb[01]ELb0EE", 64),
+    ("conv3x3_tc2.cu", r"conv3x3_tc2_kernel", 64),
+    ("attention_tc2.cu", r"attention_tc2_kernel", 64),
+    ("groupnorm_cluster.cu", r"groupnorm_cluster_kernel", 64),
+]
+
+
+def stack_frames(report):
+    """{mangled kernel name: stack frame bytes} from the text ptxas -v prints."""
+    out, name = {}, None
+    for line in report.splitlines():
+        m = re.search(r"Compiling entry function '([^']+)'", line)
+        if m:
+            name = m.group(1)
+            continue
+        m = re.search(r"(\d+) bytes stack frame", line)
+        if m and name:
+            out[name] = int(m.group(1))
+            name = None
+    return out
+
+
+def check_stack(src, report):
+    bad = []
+    for fname, pat, limit in STACK_LIMITS:
+        if os.path.basename(src) != fname:
+            continue
+        for k, b in stack_frames(report).items():
+            if re.search(pat, k) and b > limit:
+                bad.append(f"{fname}: {k} keeps a {b}-byte stack frame (limit {limit})")
+    return bad
+
+
 def _sources():
     return sorted(glob.glob(os.path.join(CSRC, "*.cu")) + glob.glob(os.path.join(CSRC, "*.cpp")))
 
@@ -39,7 +82,7 @@ def _headers_mtime():
 
 def _compile(src, obj, verbose):
     cmd = [NVCC, *FLAGS, *os.environ.get("MK_NVCC_FLAGS", "").split(), "-x", "cu", "-c", src, "-o", obj]
-    if verbose:
+    if src.endswith(".cu"):
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")
     r = subprocess.run(cmd, capture_output=True, text=True)
@@ -61,6 +104,10 @@ def build(force=False, verbose=False):
                 sys.stderr.write(out)
             if rc != 0:
                 raise RuntimeError(f"nvcc failed on {src}")
+            bad = check_stack(src, out)
+            if bad:
+                os.remove(os.path.join(OBJ, os.path.basename(src) + ".o"))
+                raise RuntimeError("accumulators left the register file:\n  " + "\n  ".join(bad))
     if jobs or not os.path.exists(LIB):
         cmd = [NVCC, "-shared", "-o", LIB, *objs, "-gencode", "arch=compute_100a,code=sm_100a",
                "-Xcompiler", "-fPIC"]

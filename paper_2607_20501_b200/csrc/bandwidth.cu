@@ -475,11 +475,11 @@ constexpr int GN_MAX_C = 2048;
 #ifndef MK_GN_RESIDENT
 #define MK_GN_RESIDENT 2
 #endif
-constexpr int GN_RESIDENT = MK_GN_RESIDENT;
+constexpr int GN_RESIDENT = MK_GN_RESIDENT;    // CTAs per SM the two-pass kernels are compiled for
 #ifndef MK_GN_UN
-#define MK_GN_UN 8
+#define MK_GN_UN 4
 #endif
-constexpr int GN_UN = MK_GN_UN;               // independent 16-byte loads per thread and batch   // CTAs per SM the two-pass kernels are compiled for
+constexpr int GN_UN = MK_GN_UN;                // independent 16-byte loads per thread and batch (8 and 16 measured slower)
 
 int groupnorm_chunks(int64_t nb, int64_t hw, int sm_count) {
   // as many CTAs as are resident at once (GN_RESIDENT per SM: both kernels are built for it), never one more: a

@@ -103,8 +103,8 @@ __device__ __forceinline__ void epi32(const EpiProgram& p, float (&v)[32], int64
         for (int j = 0; j < 32; ++j) v[j] = gelu_fast(v[j]);
         break;
       case EPI_GELU_ERF:
-#pragma unroll 4
-        for (int j = 0; j < 32; ++j) v[j] = gelu_erf_f(v[j]);
+#pragma unroll
+        for (int j = 0; j < 32; ++j) v[j] = gelu_erf_f(v[j]);   // fully unrolled like the rest: a run-time index would put v in local memory
         break;
       case EPI_SILU:
 #pragma unroll
