@@ -367,7 +367,8 @@ conv3x3_tc2_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
       tc::tc_fence_before();
       __syncwarp();
       if (threadIdx.x == 64) CTR(5 + it * 8);  // epilogue: tile stored
-      if (lane == 0) tc::mbar_arrive_cluster(tc::map_to_cta(tc::smem_u32(&sh->tempty[acc]), 0));
+      // (a relaxed arrival: the warp's reads of tensor memory are over, nothing has to be published)
+      if (lane == 0) tc::mbar_arrive_cluster_relaxed(tc::map_to_cta(tc::smem_u32(&sh->tempty[acc]), 0));
     }
   }
 

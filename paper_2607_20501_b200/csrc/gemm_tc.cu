@@ -398,6 +398,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
         pre_rstd = rsqrtf(sq * pn.inv_n_in + pn.eps_in);
       }
+      if (threadIdx.x == 64) MK_TR(7 + it * 8);  // epilogue: bias in shared memory, about to wait for the accumulator
       ok = tc::mbar_wait(&sh->tfull[acc], (it >> 1) & 1, abort_flag, status, tc::WAIT_TMEM_FULL);
       ok = __all_sync(0xffffffffu, ok ? 1 : 0) != 0;
       if (!ok) break;
@@ -417,8 +418,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           if (lane == 0) tc::tma_store_wait_read();
           __syncwarp();
         }
+#ifdef MK_TRACE
+        ew.tr = (threadIdx.x == 64 && it == 2 && c == half + 2 && blockIdx.x == 0) ? &mk_tr[50] : nullptr;
+        if (ew.tr) ew.tr[-1] = (unsigned long long)clock64();
+#endif
         tc::tmem_ld32(t_row + c * 32, r);
         tc::tmem_ld_wait();
+#ifdef MK_TRACE
+        if (ew.tr) ew.tr[0] = (unsigned long long)clock64();
+#endif
         if (threadIdx.x == 64 && c == half + 2) MK_TR(5 + it * 8);  // epilogue: second chunk in registers
 #pragma unroll
         for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
@@ -492,9 +500,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       __syncwarp();
       if (threadIdx.x == 64) MK_TR(4 + it * 8);  // epilogue: tile stored
       if (lane == 0) {
-        if (CTAS == 2) tc::mbar_arrive_cluster(tc::map_to_cta(tc::smem_u32(&sh->tempty[acc]), 0));
+        // a relaxed arrival: what must be over are this warp's reads of tensor memory (tcgen05.wait::ld and the fence
+        // above), nothing written to memory has to be published; the release form at cluster scope held each warp
+        // for some two thousand cycles per tile
+        if (CTAS == 2) tc::mbar_arrive_cluster_relaxed(tc::map_to_cta(tc::smem_u32(&sh->tempty[acc]), 0));
         else tc::mbar_arrive(&sh->tempty[acc]);
       }
+      if (threadIdx.x == 64 && it) MK_TR(it * 8);  // epilogue: accumulator handed back
       if (NORM) {
         // partial sums of this warp's share of the rows, then count this warp in; the warp that completes the
         // block of 32 rows (2 * column tiles arrivals: both column halves of every tile) normalises it

@@ -258,9 +258,13 @@ __device__ __forceinline__ float ex2_fast(float x) {
 // ---------------------------------------------------------------- optional timeline (-DMK_TRACE builds only)
 #ifdef MK_TRACE
 __device__ __forceinline__ unsigned long long gtime() {
+#ifdef MK_TRACE_CLK
+  return (unsigned long long)clock64();   // SM cycles: cheap to read, comparable inside one CTA only
+#else
   unsigned long long t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
+#endif
 }
 #define MK_TR_DECL __shared__ unsigned long long mk_tr[96];
 #define MK_TR_INIT do { if (threadIdx.x == 0) { for (int i_ = 0; i_ < 96; ++i_) mk_tr[i_] = 0; mk_tr[0] = mk::tc::gtime(); mk_tr[95] = (unsigned long long)clock64(); } } while (0)

@@ -151,6 +151,12 @@ struct EpiWarp {
   bool res_f32, out_f32;
   bool store = true;   // false: chunk_out applies the program to v and stores nothing (the caller goes on with v)
   int lane;
+#ifdef MK_TRACE
+  unsigned long long* tr = nullptr;   // trace builds: where the chunk being timed leaves its clock readings (null: not timed)
+#define MK_TRC(k) do { if (tr) tr[k] = (unsigned long long)clock64(); } while (0)
+#else
+#define MK_TRC(k) do {} while (0)
+#endif
   __device__ __forceinline__ void init(uint8_t* warp_smem, const EpiProgram& p, int lane_, bool out_f32_) {
     stage = warp_smem;
     bias = warp_smem + EPI_WARP_STAGE;
@@ -223,12 +229,15 @@ struct EpiWarp {
     const int f = (lane >> 1) & 3;
 #pragma unroll
     for (int i = 0; i < 4; ++i) *reinterpret_cast<uint4*>(stage + lane * 64 + ((i ^ f) * 16)) = mine[i];
+    MK_TRC(4);
     tc::fence_proxy_async();
     __syncwarp();
+    MK_TRC(5);
     if (lane == 0) {
       tc::tma_store_2d(tm, stage, x, y);
       tc::tma_store_commit();
     }
+    MK_TRC(6);
   }
   // One chunk: program, pack, transposed coalesced store.
   //   v            the lane's fp32 values for columns [col0, col0 + 32) of its row
@@ -273,12 +282,15 @@ struct EpiWarp {
       if (lane == 0) tc::tma_store_wait_read();
       __syncwarp();
     }
+    MK_TRC(1);
     const int64_t my_row = rowmap(lane);
     uint8_t* out = reinterpret_cast<uint8_t*>(out_v);
     if (col0 + 32 <= n_cols) {
       uint4 ra[4], rb[4];
       const int res_mode = get(ra, rb);
+      MK_TRC(2);
       if (my_row >= 0) epi32(epi, v, my_row, col0, n_cols, bias_idx >= 0 ? bias + bias_off * 2 : nullptr, res_mode, ra, rb);
+      MK_TRC(3);
       uint4 mine[4];
       if (!store) {
         // program only
