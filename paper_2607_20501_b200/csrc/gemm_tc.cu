@@ -322,26 +322,36 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // staging so that the lane's read of its own 64-byte row is free of bank conflicts), one commit group per chunk.
     uint8_t* my_ring = res_ring + (warp - 2) * 2 * RES_SLOT_BYTES;
     int pf_u = unit_id, pf_c = half, res_slot = 0;
+    // what the cursor's tile fixes, recomputed when the cursor moves to another tile and not once per chunk: its first
+    // row of this warp, its first column, its number of chunks, and this lane's first source address
+    int64_t pf_r0 = 0, pf_cb = 0;
+    int pf_chunks = 0;
+    const uint8_t* pf_src = nullptr;
+    auto ring_tile = [&]() {
+      if (pf_u >= total_units) return;
+      int t, nhalf;
+      decode(pf_u, t, nhalf);
+      int mi, ni;
+      tile_coords(t, num_m, num_n, group_m, mi, ni);
+      pf_r0 = (int64_t)(mi * CTAS + (int)rank) * BM + q * 32;
+      pf_cb = (int64_t)ni * OUT_N + (nhalf > 0 ? BN / 2 : 0);
+      pf_chunks = nhalf < 0 ? CHUNKS : CHUNKS / 2;
+      pf_src = reinterpret_cast<const uint8_t*>(epi.op[ew.res_idx].ptr) + ((pf_r0 + (lane >> 2)) * (int64_t)N + pf_cb) * 2 + (lane & 3) * 16;
+    };
     auto ring_issue = [&](int slot) {
       if (pf_u < total_units) {
-        int t, nhalf;
-        decode(pf_u, t, nhalf);
-        int mi, ni;
-        tile_coords(t, num_m, num_n, group_m, mi, ni);
-        const int64_t r0 = (int64_t)(mi * CTAS + (int)rank) * BM + q * 32;
-        const int64_t c0 = (int64_t)ni * OUT_N + (nhalf > 0 ? BN / 2 : 0) + pf_c * 32;
-        if (c0 + 32 <= N) {
-          const uint8_t* res = reinterpret_cast<const uint8_t*>(epi.op[ew.res_idx].ptr);
+        if (pf_cb + pf_c * 32 + 32 <= N) {
           const int sub_row = lane >> 2, seg = lane & 3;
           const uint32_t dst0 = tc::smem_u32(my_ring + slot * RES_SLOT_BYTES);
+          const uint8_t* src = pf_src + pf_c * 64;
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             const int r = sub_row + 8 * i;
-            if (r0 + r < M) tc::cp_async16(dst0 + r * 64 + ((seg ^ ((r >> 1) & 3)) * 16), res + ((r0 + r) * (int64_t)N + c0) * 2 + seg * 16);
+            if (pf_r0 + r < M) tc::cp_async16(dst0 + r * 64 + ((seg ^ ((r >> 1) & 3)) * 16), src + (int64_t)(8 * i) * N * 2);
           }
         }
         pf_c += 2;
-        if (pf_c >= (nhalf < 0 ? CHUNKS : CHUNKS / 2)) { pf_u += num_units; pf_c = half; }
+        if (pf_c >= pf_chunks) { pf_u += num_units; pf_c = half; ring_tile(); }
       }
       tc::cp_async_commit();
     };
@@ -364,6 +374,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       res_slot ^= 1;
     };
     if (RING) {
+      ring_tile();
       ring_issue(0);
       ring_issue(1);
     }
@@ -376,7 +387,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int64_t row0 = (int64_t)(mi * CTAS + (int)rank) * BM + q * 32;
       auto rowmap = [&](int r) -> int64_t { const int64_t g = row0 + r; return g < M ? g : -1; };
       const int64_t col_base = (int64_t)ni * OUT_N + (nhalf > 0 ? BN / 2 : 0);
-      const int chunks_here = nhalf < 0 ? CHUNKS : CHUNKS / 2;
+      // chunks of this unit; without the ring (whose cursor counts every chunk of every tile) only those that begin inside N
+      const int chunks_unit = nhalf < 0 ? CHUNKS : CHUNKS / 2;
+      const int chunks_here = RING ? chunks_unit : (int)min((int64_t)chunks_unit, (N - col_base + 31) / 32);
       uint4 res_regs[8];
       ew.load_bias(epi, col_base, nhalf < 0 ? OUT_N : OUT_N / 2, N);
       if (!RING) ew.prefetch_res(epi, rowmap, col_base + half * 32, N, res_regs);
