@@ -169,6 +169,26 @@ __device__ __forceinline__ float epi_apply(const EpiProgram& p, float v, int64_t
   return v;
 }
 
+// The same with the value of one bias op (index pre_idx, -1: none) already in a register: kernels whose whole time is
+// latency ask for it in their first instructions instead of at the end.
+__device__ __forceinline__ float epi_apply_pre(const EpiProgram& p, float v, int64_t row, int64_t col, int64_t ld, int pre_idx, float pre_val) {
+  for (int i = 0; i < p.n; ++i) {
+    const EpiOp& o = p.op[i];
+    switch (o.kind) {
+      case EPI_BIAS: v += i == pre_idx ? pre_val : epi_ptr_ld(o.ptr, p.dtype, col); break;
+      case EPI_RELU: v = fmaxf(v, 0.0f); break;
+      case EPI_GELU_TANH: v = gelu_tanh_f(v); break;
+      case EPI_GELU_ERF: v = gelu_erf_f(v); break;
+      case EPI_SILU: v = silu_f(v); break;
+      case EPI_SCALE: v *= o.a; break;
+      case EPI_CLAMP: v = fminf(fmaxf(v, o.a), o.b); break;
+      case EPI_RESIDUAL: v += epi_ptr_ld(o.ptr, o.ptr_dtype, row * ld + col); break;
+      default: break;
+    }
+  }
+  return v;
+}
+
 // Run the program on NV consecutive columns of one row; col0 is a multiple of NV and the program's
 // pointers are 16-byte aligned, so bias and residual are fetched with 128-bit loads.
 template <typename T, int NV>

@@ -86,12 +86,15 @@ static cudaError_t gemm_simt_dispatch(const void* a, const void* w, bool wt, voi
 // The same fused chain on a thread-block cluster, for the small problems whose whole time is latency (N <= 256):
 // a cluster of eight CTAs owns eight rows, each CTA a slice of the columns, so a CTA loads an eighth of W
 // instead of all of it; the row statistics meet through distributed shared memory (every CTA writes its
-// partial sums into all eight CTAs' slots, one cluster barrier per statistic).  Two-pass LayerNorm
-// (mean, then centred squares), as in the single-CTA form.
+// (mean, M2) of its slice of each row into all eight CTAs' slots, one cluster barrier).  The merged variance is what
+// the single-CTA form's two passes give.
 // =====================================================================================================
 constexpr int LC_CL = 8;         // CTAs per cluster
 constexpr int LC_RB = 8;         // rows per cluster
-constexpr int LC_THREADS = 256;
+#ifndef MK_LC_THREADS
+#define MK_LC_THREADS 512
+#endif
+constexpr int LC_THREADS = MK_LC_THREADS;   // the threads beyond the CTA's outputs split K: more of them, shorter dot products
 constexpr int LC_MAXNC = 32;     // columns per CTA: N <= LC_CL * LC_MAXNC
 
 __device__ __forceinline__ void st_cluster_f32(uint32_t cluster_addr, float v) {
@@ -106,12 +109,17 @@ __global__ void __launch_bounds__(LC_THREADS) linear_rownorm_cluster_kernel(cons
                                                                             float eps) {
   extern __shared__ float smem[];
   const int KP = K + 1;                                    // odd pitch: threads of different columns hit different banks
-  float* xs = smem;                                        // [LC_RB][K]
-  float* ws = xs + LC_RB * K;                              // [NC][KP]: this CTA's columns of W, K contiguous
+  const int XP = K + 4;                                    // the rows a warp reads together start four banks apart
+  float* xs = smem;                                        // [LC_RB][XP]
+  float* ws = xs + LC_RB * XP;                             // [NC][KP]: this CTA's columns of W, K contiguous
   float* part = ws + NC * KP;                              // [KS][LC_RB * NC]
-  __shared__ float val[LC_RB][LC_MAXNC];                   // this CTA's outputs after the elementwise tail
-  __shared__ float slot[2][LC_CL][LC_RB];                  // row partial sums of every CTA of the cluster (two statistics)
-  __shared__ float stat[2][LC_RB];
+  __shared__ float slot[2][LC_CL][LC_RB];                  // every CTA's (mean, M2) of its slice of each row
+#ifdef MK_TRACE_C1
+  long long tr_[8]; tr_[0] = clock64();
+#define C1T(i) tr_[i] = clock64()
+#else
+#define C1T(i) do {} while (0)
+#endif
   pdl_launch_dependents();
   // A CTA may write into a peer's shared memory only once that peer is running: every CTA announces itself
   // here and waits for the others just before its first remote store, so the rendezvous costs nothing.
@@ -120,129 +128,158 @@ __global__ void __launch_bounds__(LC_THREADS) linear_rownorm_cluster_kernel(cons
   const uint32_t rank = tc::cluster_ctarank();
   const int m0 = (int)(blockIdx.x / LC_CL) * LC_RB, c0 = (int)rank * NC;
   const int nc = min(NC, N - c0) > 0 ? min(NC, N - c0) : 0;   // columns of this CTA that exist
-  // Everything that is read late - the norm's scale and shift, a bias vector inside the elementwise tail - is asked
-  // for now: a dependent global load at the end of this kernel would be a tenth of its whole duration.
-  float ga = 1.0f, be = 0.0f;
+  // Everything that is read late - the norm's scale and shift, the first bias vector of the elementwise tail - is
+  // asked for now: a dependent global load at the end of this kernel would be a tenth of its whole duration.
+  float ga = 1.0f, be = 0.0f, bias_v = 0.0f;
+  int bias_i = -1;
   {
     const int rj = threadIdx.x, j = rj % NC;
     if (rj < LC_RB * NC && j < nc) {
       if (gamma) ga = Elem<T>::ld(gamma + c0 + j);
       if (mode == ROW_LAYERNORM && beta) be = Elem<T>::ld(beta + c0 + j);
-      for (int i = 0; i < p.n; ++i)
-        if (p.op[i].kind == EPI_BIAS && p.op[i].ptr)
-          asm volatile("prefetch.global.L1 [%0];" ::"l"(reinterpret_cast<const char*>(p.op[i].ptr) + (size_t)(c0 + j) * sizeof(T)));
+      for (int i = 0; i < p.n && bias_i < 0; ++i)
+        if (p.op[i].kind == EPI_BIAS && p.op[i].ptr) bias_i = i;
+      if (bias_i >= 0) bias_v = epi_ptr_ld(p.op[bias_i].ptr, p.dtype, c0 + j);
     }
   }
   constexpr int VE = Elem<T>::VEC;
-  if (K % VE == 0) {
-    // 16-byte loads, all of a thread's in flight together: the whole kernel is a few round trips to L2 long
-    const int kv = K / VE;
-    for (int i = threadIdx.x; i < LC_RB * kv; i += LC_THREADS) {
-      const int r = i / kv, k = (i - r * kv) * VE;
-      float v[VE];
-      if (m0 + r < M) {
-        ld_vec(a + (int64_t)(m0 + r) * K + k, v);
-      } else {
+  // how W is read: 1 = 16-byte vectors along K (stored [N, K]), 2 = 16-byte vectors along N (stored [K, N]), 0 = scalars
+  const int wmode = wt ? (K % VE == 0 ? 1 : 0) : ((N % VE == 0 && NC % VE == 0 && nc % VE == 0) ? 2 : 0);
+  if (K % VE == 0 && wmode != 0) {
+    // 16-byte loads; a thread's load of X and its load of W are in flight together: the whole kernel is a few round
+    // trips to L2 long
+    const int kv = K / VE, nx = LC_RB * kv, nv = nc / VE;
+    const int nw = wmode == 1 ? nc * kv : K * nv;
+    for (int base = 0; base < max(nx, nw); base += LC_THREADS) {
+      const int i = base + threadIdx.x;
+      const bool hx = i < nx, hw = i < nw;
+      float vx[VE], vw[VE];
+      int r = 0, kx = 0, jw = 0, kw = 0;
+      if (hx) {
+        r = i / kv; kx = (i - r * kv) * VE;
+        if (m0 + r < M) {
+          ld_vec(a + (int64_t)(m0 + r) * K + kx, vx);
+        } else {
 #pragma unroll
-        for (int e = 0; e < VE; ++e) v[e] = 0.0f;
+          for (int e = 0; e < VE; ++e) vx[e] = 0.0f;
+        }
       }
+      if (hw) {
+        if (wmode == 1) { jw = i / kv; kw = (i - jw * kv) * VE; ld_vec(w + (int64_t)(c0 + jw) * K + kw, vw); }
+        else { kw = i / nv; jw = (i - kw * nv) * VE; ld_vec(w + (int64_t)kw * N + c0 + jw, vw); }
+      }
+      if (hx) {
 #pragma unroll
-      for (int e = 0; e < VE; ++e) xs[r * K + k + e] = v[e];
+        for (int e = 0; e < VE; ++e) xs[r * XP + kx + e] = vx[e];
+      }
+      if (hw) {
+#pragma unroll
+        for (int e = 0; e < VE; ++e) {
+          if (wmode == 1) ws[jw * KP + kw + e] = vw[e];
+          else ws[(jw + e) * KP + kw] = vw[e];
+        }
+      }
     }
   } else {
     for (int i = threadIdx.x; i < LC_RB * K; i += LC_THREADS) {
       const int r = i / K, k = i - r * K;
-      xs[i] = (m0 + r < M) ? Elem<T>::ld(a + (int64_t)(m0 + r) * K + k) : 0.0f;
+      xs[r * XP + k] = (m0 + r < M) ? Elem<T>::ld(a + (int64_t)(m0 + r) * K + k) : 0.0f;
     }
-  }
-  if (wt && K % VE == 0) {
-    const int kv = K / VE;
-    for (int i = threadIdx.x; i < nc * kv; i += LC_THREADS) {
-      const int j = i / kv, k = (i - j * kv) * VE;
-      float v[VE];
-      ld_vec(w + (int64_t)(c0 + j) * K + k, v);
-#pragma unroll
-      for (int e = 0; e < VE; ++e) ws[j * KP + k + e] = v[e];
-    }
-  } else if (wt) {
-    for (int i = threadIdx.x; i < nc * K; i += LC_THREADS) {
-      const int j = i / K, k = i - j * K;                   // consecutive threads walk K: contiguous in memory
-      ws[j * KP + k] = Elem<T>::ld(w + (int64_t)(c0 + j) * K + k);
-    }
-  } else {
-    for (int i = threadIdx.x; i < nc * K; i += LC_THREADS) {
-      const int k = i / nc, j = i - k * nc;                 // consecutive threads walk the columns: contiguous in memory
-      ws[j * KP + k] = Elem<T>::ld(w + (int64_t)k * N + c0 + j);
+    if (wt) {
+      for (int i = threadIdx.x; i < nc * K; i += LC_THREADS) {
+        const int j = i / K, k = i - j * K;                   // consecutive threads walk K: contiguous in memory
+        ws[j * KP + k] = Elem<T>::ld(w + (int64_t)(c0 + j) * K + k);
+      }
+    } else {
+      for (int i = threadIdx.x; i < nc * K; i += LC_THREADS) {
+        const int k = i / nc, j = i - k * nc;                 // consecutive threads walk the columns: contiguous in memory
+        ws[j * KP + k] = Elem<T>::ld(w + (int64_t)k * N + c0 + j);
+      }
     }
   }
   __syncthreads();
+  C1T(1);
   // outputs r * NC + j; the threads beyond them split K
   const int outs = LC_RB * NC;
   const int KS = LC_THREADS / outs > 0 ? LC_THREADS / outs : 1;
   for (int o = threadIdx.x; o < outs * KS; o += LC_THREADS) {
     const int ks = o / outs, rj = o - ks * outs, r = rj / NC, j = rj - r * NC;
     const int kper = (K + KS - 1) / KS, kb = ks * kper, ke = min(K, kb + kper);
-    float acc = 0.0f;
+    float acc = 0.0f, acc1 = 0.0f;   // two chains: the loop is bound by the latency of a dependent FMA
     if (j < nc) {
-      const float* xr = xs + r * K;
+      const float* xr = xs + r * XP;
       const float* wr = ws + j * KP;
-#pragma unroll 8
-      for (int k = kb; k < ke; ++k) acc = fmaf(xr[k], wr[k], acc);
+      int k = kb;
+#pragma unroll 4
+      for (; k + 1 < ke; k += 2) {
+        acc = fmaf(xr[k], wr[k], acc);
+        acc1 = fmaf(xr[k + 1], wr[k + 1], acc1);
+      }
+      if (k < ke) acc = fmaf(xr[k], wr[k], acc);
     }
-    part[ks * outs + rj] = acc;
+    part[ks * outs + rj] = acc + acc1;
   }
   __syncthreads();
-  for (int rj = threadIdx.x; rj < outs; rj += LC_THREADS) {
-    const int r = rj / NC, j = rj - r * NC;
-    float v = 0.0f;
+  C1T(2);
+  // from here on a thread owns one output (outs <= LC_THREADS): row r, column j of this CTA's slice, kept in a register
+  const int rj = threadIdx.x, r = rj / NC, j = rj - r * NC;
+  const bool has = rj < outs && j < nc;
+  float v = 0.0f;
+  if (has) {
     for (int q = 0; q < KS; ++q) v += part[q * outs + rj];       // fixed order
-    val[r][j] = j < nc ? epi_apply(p, v, m0 + r, c0 + j, N) : 0.0f;
+    v = epi_apply_pre(p, v, m0 + r, c0 + j, N, bias_i, bias_v);
   }
-  __syncthreads();
+  C1T(3);
   tc::cluster_wait();   // all eight CTAs of the cluster are resident from here on
-  const float inv_n = 1.0f / (float)N;
-  // statistic 0: the row sums (LayerNorm) -> mean
-  if (mode == ROW_LAYERNORM) {
-    if (threadIdx.x < LC_RB) {
-      float sm = 0.0f;
-      for (int j = 0; j < nc; ++j) sm += val[threadIdx.x][j];
-      const uint32_t local = tc::smem_u32(&slot[0][rank][threadIdx.x]);
-      for (uint32_t c = 0; c < LC_CL; ++c) st_cluster_f32(tc::map_to_cta(local, c), sm);
+  C1T(4);
+  // One exchange for both statistics.  LayerNorm: every CTA sends, per row, the mean of its columns and their squared
+  // deviations from that mean; the receiver merges the eight (count, mean, M2) triples, M2 = sum of M2_c + n_c *
+  // (mean_c - mean)^2, which is what a second pass about the global mean would have summed, so no second round is
+  // needed.  RMSNorm: the squares about zero.  A row's NC values sit in NC adjacent lanes (NC is a power of two <= 32).
+  if ((threadIdx.x & ~31) < outs) {
+    float mc = 0.0f, q;
+    if (mode == ROW_LAYERNORM) {
+      float sm = v;
+      for (int o = NC >> 1; o; o >>= 1) sm += __shfl_xor_sync(0xffffffffu, sm, o);
+      mc = nc > 0 ? sm / (float)nc : 0.0f;
+      const float d = has ? v - mc : 0.0f;
+      q = d * d;
+    } else {
+      q = v * v;
     }
-    tc::cluster_sync();
-    if (threadIdx.x < LC_RB) {
-      float sm = 0.0f;
-      for (int c = 0; c < LC_CL; ++c) sm += slot[0][c][threadIdx.x];   // the same order in every CTA
-      stat[0][threadIdx.x] = sm * inv_n;
+    for (int o = NC >> 1; o; o >>= 1) q += __shfl_xor_sync(0xffffffffu, q, o);
+    if (rj < outs) {
+      const uint32_t l0 = tc::smem_u32(&slot[0][rank][r]), l1 = tc::smem_u32(&slot[1][rank][r]);
+      for (uint32_t c = (uint32_t)j; c < LC_CL; c += (uint32_t)NC) {   // the row's lanes share the eight destinations
+        st_cluster_f32(tc::map_to_cta(l0, c), mc);
+        st_cluster_f32(tc::map_to_cta(l1, c), q);
+      }
     }
-  } else if (threadIdx.x < LC_RB) {
-    stat[0][threadIdx.x] = 0.0f;
   }
-  __syncthreads();
-  // statistic 1: centred squares -> 1 / sqrt(var + eps)  (RMSNorm: squares about zero)
-  if (threadIdx.x < LC_RB) {
-    const float mean = stat[0][threadIdx.x];
-    float q = 0.0f;
-    for (int j = 0; j < nc; ++j) { const float d = val[threadIdx.x][j] - mean; q += d * d; }
-    const uint32_t local = tc::smem_u32(&slot[1][rank][threadIdx.x]);
-    for (uint32_t c = 0; c < LC_CL; ++c) st_cluster_f32(tc::map_to_cta(local, c), q);
-  }
+  C1T(5);
   tc::cluster_sync();
-  if (threadIdx.x < LC_RB) {
-    float q = 0.0f;
-    for (int c = 0; c < LC_CL; ++c) q += slot[1][c][threadIdx.x];
-    stat[1][threadIdx.x] = rsqrtf(q * inv_n + eps);
-  }
-  __syncthreads();
-  for (int rj = threadIdx.x; rj < outs; rj += LC_THREADS) {
-    const int r = rj / NC, j = rj - r * NC;
-    if (j < nc && m0 + r < M) {
-      const int c = c0 + j;
-      const float o = (val[r][j] - stat[0][r]) * stat[1][r] * ga + be;
-      Elem<T>::st(y + (int64_t)(m0 + r) * N + c, o);
+  C1T(6);
+  if (has && m0 + r < M) {
+    float mean = 0.0f, m2 = 0.0f;
+    const float inv_n = 1.0f / (float)N;
+    if (mode == ROW_LAYERNORM) {
+      for (int c = 0; c < LC_CL; ++c) mean += (float)max(0, min(NC, N - c * NC)) * slot[0][c][r];   // the same order everywhere
+      mean *= inv_n;
+      for (int c = 0; c < LC_CL; ++c) {
+        const float d = slot[0][c][r] - mean;
+        m2 += slot[1][c][r] + (float)max(0, min(NC, N - c * NC)) * d * d;
+      }
+    } else {
+      for (int c = 0; c < LC_CL; ++c) m2 += slot[1][c][r];
     }
+    const float o = (v - mean) * rsqrtf(m2 * inv_n + eps) * ga + be;
+    Elem<T>::st(y + (int64_t)(m0 + r) * N + c0 + j, o);
   }
-  // nobody writes into a peer's shared memory after the second cluster barrier: a CTA may retire here
+#ifdef MK_TRACE_C1
+  C1T(7);
+  if (blockIdx.x == 0 && threadIdx.x == 0) printf("c1 loads %lld fma %lld tail %lld wait %lld stats %lld sync %lld out %lld\n", tr_[1]-tr_[0], tr_[2]-tr_[1], tr_[3]-tr_[2], tr_[4]-tr_[3], tr_[5]-tr_[4], tr_[6]-tr_[5], tr_[7]-tr_[6]);
+#endif
+  // nobody writes into a peer's shared memory after the cluster barrier: a CTA may retire here
 }
 
 template <typename T>
@@ -254,7 +291,7 @@ static cudaError_t linear_rownorm_cluster_launch(const void* a, const void* w, b
   while (pw < NC) pw *= 2;
   NC = pw;
   const int outs = LC_RB * NC, KS = LC_THREADS / outs > 0 ? LC_THREADS / outs : 1;
-  const size_t smem = sizeof(float) * ((size_t)LC_RB * k + (size_t)NC * (k + 1) + (size_t)KS * outs);
+  const size_t smem = sizeof(float) * ((size_t)LC_RB * (k + 4) + (size_t)NC * (k + 1) + (size_t)KS * outs);
   static SmemOptIn opt_in;   // one per instantiation (T)
   if (smem > 48 * 1024) {
     cudaError_t e = opt_in.ensure(smem, linear_rownorm_cluster_kernel<T>);
@@ -269,7 +306,7 @@ static cudaError_t linear_rownorm_cluster_launch(const void* a, const void* w, b
 static bool linear_rownorm_cluster_ok(int64_t m, int64_t n, int64_t k, int mode) {
   if (mode != ROW_LAYERNORM && mode != ROW_RMSNORM) return false;
   if (n > LC_CL * LC_MAXNC || n < LC_CL || k > 2048 || m > (1 << 20)) return false;
-  return sizeof(float) * ((size_t)(LC_RB + LC_MAXNC) * (k + 1) + LC_THREADS) <= 160 * 1024;
+  return sizeof(float) * ((size_t)(LC_RB + LC_MAXNC) * (k + 4) + LC_THREADS) <= 160 * 1024;
 }
 
 template <typename T>
