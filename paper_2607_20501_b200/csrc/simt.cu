@@ -101,6 +101,55 @@ __device__ __forceinline__ void st_cluster_f32(uint32_t cluster_addr, float v) {
   asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(cluster_addr), "f"(v) : "memory");
 }
 
+// The end of both cluster forms: thread (r, j) holds output v of row m0 + r, column c0 + j (has: that output exists;
+// in_outs: the thread is one of the CTA's LC_RB * NC output threads).  Called by every thread of the CTA.
+template <typename T>
+__device__ __forceinline__ void lc_norm_tail(float v, bool has, bool in_outs, int r, int j, int nc, int NC, int N, int M, int m0, int c0,
+                                             uint32_t rank, int mode, float eps, float ga, float be, float (&slot)[2][LC_CL][LC_RB],
+                                             T* __restrict__ y) {
+  // One exchange for both statistics.  LayerNorm: every CTA sends, per row, the mean of its columns and their squared
+  // deviations from that mean; the receiver merges the eight (count, mean, M2) triples, M2 = sum of M2_c + n_c *
+  // (mean_c - mean)^2, which is what a second pass about the global mean would have summed, so no second round is
+  // needed.  RMSNorm: the squares about zero.  A row's NC values sit in NC adjacent lanes (NC is a power of two <= 32).
+  if (__any_sync(0xffffffffu, in_outs)) {
+    float mc = 0.0f, q;
+    if (mode == ROW_LAYERNORM) {
+      float sm = v;
+      for (int o = NC >> 1; o; o >>= 1) sm += __shfl_xor_sync(0xffffffffu, sm, o);
+      mc = nc > 0 ? sm / (float)nc : 0.0f;
+      const float d = has ? v - mc : 0.0f;
+      q = d * d;
+    } else {
+      q = v * v;
+    }
+    for (int o = NC >> 1; o; o >>= 1) q += __shfl_xor_sync(0xffffffffu, q, o);
+    if (in_outs) {
+      const uint32_t l0 = tc::smem_u32(&slot[0][rank][r]), l1 = tc::smem_u32(&slot[1][rank][r]);
+      for (uint32_t c = (uint32_t)j; c < LC_CL; c += (uint32_t)NC) {   // the row's lanes share the eight destinations
+        st_cluster_f32(tc::map_to_cta(l0, c), mc);
+        st_cluster_f32(tc::map_to_cta(l1, c), q);
+      }
+    }
+  }
+  tc::cluster_sync();
+  if (has && m0 + r < M) {
+    float mean = 0.0f, m2 = 0.0f;
+    const float inv_n = 1.0f / (float)N;
+    if (mode == ROW_LAYERNORM) {
+      for (int c = 0; c < LC_CL; ++c) mean += (float)max(0, min(NC, N - c * NC)) * slot[0][c][r];   // the same order everywhere
+      mean *= inv_n;
+      for (int c = 0; c < LC_CL; ++c) {
+        const float d = slot[0][c][r] - mean;
+        m2 += slot[1][c][r] + (float)max(0, min(NC, N - c * NC)) * d * d;
+      }
+    } else {
+      for (int c = 0; c < LC_CL; ++c) m2 += slot[1][c][r];
+    }
+    const float o = (v - mean) * rsqrtf(m2 * inv_n + eps) * ga + be;
+    Elem<T>::st(y + (int64_t)(m0 + r) * N + c0 + j, o);
+  }
+}
+
 template <typename T>
 __global__ void __launch_bounds__(LC_THREADS) linear_rownorm_cluster_kernel(const T* __restrict__ a, const T* __restrict__ w, bool wt,
                                                                             T* __restrict__ y, int M, int N, int K, int NC,
@@ -108,8 +157,10 @@ __global__ void __launch_bounds__(LC_THREADS) linear_rownorm_cluster_kernel(cons
                                                                             const T* __restrict__ gamma, const T* __restrict__ beta,
                                                                             float eps) {
   extern __shared__ float smem[];
-  const int KP = K + 1;                                    // odd pitch: threads of different columns hit different banks
-  const int XP = K + 4;                                    // the rows a warp reads together start four banks apart
+  // row pitches of K + 4 floats: rows stay 16-byte aligned for the vector reads of the dot products, and the rows (of X)
+  // or columns (of W) that a quarter warp reads together start four banks apart
+  const int KP = K + 4;
+  const int XP = K + 4;
   float* xs = smem;                                        // [LC_RB][XP]
   float* ws = xs + LC_RB * XP;                             // [NC][KP]: this CTA's columns of W, K contiguous
   float* part = ws + NC * KP;                              // [KS][LC_RB * NC]
@@ -205,17 +256,29 @@ __global__ void __launch_bounds__(LC_THREADS) linear_rownorm_cluster_kernel(cons
   for (int o = threadIdx.x; o < outs * KS; o += LC_THREADS) {
     const int ks = o / outs, rj = o - ks * outs, r = rj / NC, j = rj - r * NC;
     const int kper = (K + KS - 1) / KS, kb = ks * kper, ke = min(K, kb + kper);
-    float acc = 0.0f, acc1 = 0.0f;   // two chains: the loop is bound by the latency of a dependent FMA
+    float acc = 0.0f, acc1 = 0.0f;   // two chains: a dependent FMA every four cycles is half of what the loop can issue
     if (j < nc) {
       const float* xr = xs + r * XP;
       const float* wr = ws + j * KP;
-      int k = kb;
+      if (((kb | ke | K) & 3) == 0) {   // K itself too: the row pitches are K + 4
+        // 16-byte reads: the dot products are bound by shared-memory wavefronts, and a vector read of X (two distinct
+        // rows per warp) costs one wavefront for four k where scalar reads cost four
+        for (int k = kb; k < ke; k += 4) {
+          const float4 xv = *reinterpret_cast<const float4*>(xr + k), wv = *reinterpret_cast<const float4*>(wr + k);
+          acc = fmaf(xv.x, wv.x, acc);
+          acc1 = fmaf(xv.y, wv.y, acc1);
+          acc = fmaf(xv.z, wv.z, acc);
+          acc1 = fmaf(xv.w, wv.w, acc1);
+        }
+      } else {
+        int k = kb;
 #pragma unroll 4
-      for (; k + 1 < ke; k += 2) {
-        acc = fmaf(xr[k], wr[k], acc);
-        acc1 = fmaf(xr[k + 1], wr[k + 1], acc1);
+        for (; k + 1 < ke; k += 2) {
+          acc = fmaf(xr[k], wr[k], acc);
+          acc1 = fmaf(xr[k + 1], wr[k + 1], acc1);
+        }
+        if (k < ke) acc = fmaf(xr[k], wr[k], acc);
       }
-      if (k < ke) acc = fmaf(xr[k], wr[k], acc);
     }
     part[ks * outs + rj] = acc + acc1;
   }
@@ -232,54 +295,100 @@ __global__ void __launch_bounds__(LC_THREADS) linear_rownorm_cluster_kernel(cons
   C1T(3);
   tc::cluster_wait();   // all eight CTAs of the cluster are resident from here on
   C1T(4);
-  // One exchange for both statistics.  LayerNorm: every CTA sends, per row, the mean of its columns and their squared
-  // deviations from that mean; the receiver merges the eight (count, mean, M2) triples, M2 = sum of M2_c + n_c *
-  // (mean_c - mean)^2, which is what a second pass about the global mean would have summed, so no second round is
-  // needed.  RMSNorm: the squares about zero.  A row's NC values sit in NC adjacent lanes (NC is a power of two <= 32).
-  if ((threadIdx.x & ~31) < outs) {
-    float mc = 0.0f, q;
-    if (mode == ROW_LAYERNORM) {
-      float sm = v;
-      for (int o = NC >> 1; o; o >>= 1) sm += __shfl_xor_sync(0xffffffffu, sm, o);
-      mc = nc > 0 ? sm / (float)nc : 0.0f;
-      const float d = has ? v - mc : 0.0f;
-      q = d * d;
-    } else {
-      q = v * v;
-    }
-    for (int o = NC >> 1; o; o >>= 1) q += __shfl_xor_sync(0xffffffffu, q, o);
-    if (rj < outs) {
-      const uint32_t l0 = tc::smem_u32(&slot[0][rank][r]), l1 = tc::smem_u32(&slot[1][rank][r]);
-      for (uint32_t c = (uint32_t)j; c < LC_CL; c += (uint32_t)NC) {   // the row's lanes share the eight destinations
-        st_cluster_f32(tc::map_to_cta(l0, c), mc);
-        st_cluster_f32(tc::map_to_cta(l1, c), q);
-      }
-    }
-  }
-  C1T(5);
-  tc::cluster_sync();
-  C1T(6);
-  if (has && m0 + r < M) {
-    float mean = 0.0f, m2 = 0.0f;
-    const float inv_n = 1.0f / (float)N;
-    if (mode == ROW_LAYERNORM) {
-      for (int c = 0; c < LC_CL; ++c) mean += (float)max(0, min(NC, N - c * NC)) * slot[0][c][r];   // the same order everywhere
-      mean *= inv_n;
-      for (int c = 0; c < LC_CL; ++c) {
-        const float d = slot[0][c][r] - mean;
-        m2 += slot[1][c][r] + (float)max(0, min(NC, N - c * NC)) * d * d;
-      }
-    } else {
-      for (int c = 0; c < LC_CL; ++c) m2 += slot[1][c][r];
-    }
-    const float o = (v - mean) * rsqrtf(m2 * inv_n + eps) * ga + be;
-    Elem<T>::st(y + (int64_t)(m0 + r) * N + c0 + j, o);
-  }
+  lc_norm_tail<T>(v, has, rj < outs, r, j, nc, NC, N, M, m0, c0, rank, mode, eps, ga, be, slot, y);
 #ifdef MK_TRACE_C1
   C1T(7);
   if (blockIdx.x == 0 && threadIdx.x == 0) printf("c1 loads %lld fma %lld tail %lld wait %lld stats %lld sync %lld out %lld\n", tr_[1]-tr_[0], tr_[2]-tr_[1], tr_[3]-tr_[2], tr_[4]-tr_[3], tr_[5]-tr_[4], tr_[6]-tr_[5], tr_[7]-tr_[6]);
 #endif
   // nobody writes into a peer's shared memory after the cluster barrier: a CTA may retire here
+}
+
+// The register form of the same kernel, for the shapes where it applies (K <= LC_KPER * LC_THREADS / NC, K a multiple of
+// LC_KPER): nothing is staged in shared memory.  A thread owns one column and LC_KPER consecutive k: it loads its
+// LC_KPER weights and the eight rows' LC_KPER activations straight into registers (all loads in flight at once; the
+// lanes that share a k slice read the same addresses of X, which the load unit serves as one request), multiplies, and
+// leaves eight partial sums in shared memory; an output thread adds its column's slices.  The staged form is bound by
+// shared-memory wavefronts in its dot products (two reads per FMA, the read of X a broadcast); this one has none.
+constexpr int LC_KPER = 8;
+
+template <typename T>
+__global__ void __launch_bounds__(LC_THREADS) linear_rownorm_cluster_reg_kernel(const T* __restrict__ a, const T* __restrict__ w, bool wt,
+                                                                                T* __restrict__ y, int M, int N, int K, int NC,
+                                                                                const __grid_constant__ EpiProgram p, int mode,
+                                                                                const T* __restrict__ gamma, const T* __restrict__ beta,
+                                                                                float eps) {
+  __shared__ float part[LC_THREADS * LC_RB];               // [k slice][LC_RB][NC]
+  __shared__ float slot[2][LC_CL][LC_RB];                  // every CTA's (mean, M2) of its slice of each row
+  pdl_launch_dependents();
+  tc::cluster_arrive();                                    // see the staged form: met again just before the remote stores
+  pdl_wait();
+  const uint32_t rank = tc::cluster_ctarank();
+  const int m0 = (int)(blockIdx.x / LC_CL) * LC_RB, c0 = (int)rank * NC;
+  const int nc = min(NC, N - c0) > 0 ? min(NC, N - c0) : 0;
+  const int outs = LC_RB * NC;
+  const int j = threadIdx.x % NC, sl = threadIdx.x / NC, kb = sl * LC_KPER;
+  float ga = 1.0f, be = 0.0f, bias_v = 0.0f;
+  int bias_i = -1;
+  if (threadIdx.x < outs && j < nc) {
+    if (gamma) ga = Elem<T>::ld(gamma + c0 + j);
+    if (mode == ROW_LAYERNORM && beta) be = Elem<T>::ld(beta + c0 + j);
+    for (int i = 0; i < p.n && bias_i < 0; ++i)
+      if (p.op[i].kind == EPI_BIAS && p.op[i].ptr) bias_i = i;
+    if (bias_i >= 0) bias_v = epi_ptr_ld(p.op[bias_i].ptr, p.dtype, c0 + j);
+  }
+  constexpr int VE = Elem<T>::VEC;
+  static_assert(LC_KPER % VE == 0, "a thread's k slice is whole 16-byte vectors");
+  float acc[LC_RB];
+#pragma unroll
+  for (int r = 0; r < LC_RB; ++r) acc[r] = 0.0f;
+  if (kb < K && j < nc) {
+    float wv[LC_KPER], xr[LC_RB][LC_KPER];
+    if (wt) {
+#pragma unroll
+      for (int e0 = 0; e0 < LC_KPER; e0 += VE) {
+        float t[VE];
+        ld_vec(w + (int64_t)(c0 + j) * K + kb + e0, t);
+#pragma unroll
+        for (int e = 0; e < VE; ++e) wv[e0 + e] = t[e];
+      }
+    } else {
+#pragma unroll
+      for (int e = 0; e < LC_KPER; ++e) wv[e] = Elem<T>::ld(w + (int64_t)(kb + e) * N + c0 + j);
+    }
+#pragma unroll
+    for (int r = 0; r < LC_RB; ++r) {
+#pragma unroll
+      for (int e0 = 0; e0 < LC_KPER; e0 += VE) {
+        float t[VE];
+        if (m0 + r < M) {
+          ld_vec(a + (int64_t)(m0 + r) * K + kb + e0, t);
+        } else {
+#pragma unroll
+          for (int e = 0; e < VE; ++e) t[e] = 0.0f;
+        }
+#pragma unroll
+        for (int e = 0; e < VE; ++e) xr[r][e0 + e] = t[e];
+      }
+    }
+#pragma unroll
+    for (int e = 0; e < LC_KPER; ++e) {
+#pragma unroll
+      for (int r = 0; r < LC_RB; ++r) acc[r] = fmaf(xr[r][e], wv[e], acc[r]);
+    }
+  }
+#pragma unroll
+  for (int r = 0; r < LC_RB; ++r) part[(sl * LC_RB + r) * NC + j] = acc[r];
+  __syncthreads();
+  const int rj = threadIdx.x, r = rj / NC;
+  const bool has = rj < outs && j < nc;
+  float v = 0.0f;
+  if (has) {
+    const int ns = K / LC_KPER;
+    for (int q = 0; q < ns; ++q) v += part[(q * LC_RB + r) * NC + j];   // fixed order
+    v = epi_apply_pre(p, v, m0 + r, c0 + j, N, bias_i, bias_v);
+  }
+  tc::cluster_wait();   // all eight CTAs of the cluster are resident from here on
+  lc_norm_tail<T>(v, has, rj < outs, r, j, nc, NC, N, M, m0, c0, rank, mode, eps, ga, be, slot, y);
 }
 
 template <typename T>
@@ -290,14 +399,19 @@ static cudaError_t linear_rownorm_cluster_launch(const void* a, const void* w, b
   int pw = 1;
   while (pw < NC) pw *= 2;
   NC = pw;
+  const unsigned grid = (unsigned)((m + LC_RB - 1) / LC_RB) * LC_CL;
+  if (k % LC_KPER == 0 && k <= (int64_t)LC_KPER * (LC_THREADS / NC) && (!wt || k % Elem<T>::VEC == 0)) {
+    LaunchCfg lc(PDL_ELTWISE, dim3(grid), dim3(LC_THREADS), 0, s, LC_CL);
+    return cudaLaunchKernelEx(&lc.cfg, linear_rownorm_cluster_reg_kernel<T>, (const T*)a, (const T*)w, wt, (T*)y, (int)m, (int)n, (int)k, NC, p,
+                              mode, (const T*)g, (const T*)b, eps);
+  }
   const int outs = LC_RB * NC, KS = LC_THREADS / outs > 0 ? LC_THREADS / outs : 1;
-  const size_t smem = sizeof(float) * ((size_t)LC_RB * (k + 4) + (size_t)NC * (k + 1) + (size_t)KS * outs);
+  const size_t smem = sizeof(float) * ((size_t)LC_RB * (k + 4) + (size_t)NC * (k + 4) + (size_t)KS * outs);
   static SmemOptIn opt_in;   // one per instantiation (T)
   if (smem > 48 * 1024) {
     cudaError_t e = opt_in.ensure(smem, linear_rownorm_cluster_kernel<T>);
     if (e != cudaSuccess) return e;
   }
-  const unsigned grid = (unsigned)((m + LC_RB - 1) / LC_RB) * LC_CL;
   LaunchCfg lc(PDL_ELTWISE, dim3(grid), dim3(LC_THREADS), smem, s, LC_CL);
   return cudaLaunchKernelEx(&lc.cfg, linear_rownorm_cluster_kernel<T>, (const T*)a, (const T*)w, wt, (T*)y, (int)m, (int)n, (int)k, NC, p, mode,
                             (const T*)g, (const T*)b, eps);

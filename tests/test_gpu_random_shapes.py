@@ -106,3 +106,24 @@ def test_small_fused_chain_with_random_shape(ctx, i):
     dw, out = run_gpu(ctx, w, [0], weight_layout=B.MK_LAYOUT_ROW_MAJOR if row_major else None)
     assert dw.module.bound_impl(0) == "linear_rownorm_simt"
     assert_parity(out, ref, dtype, f"M{m} K{k} N{n} {dtype} {norm} row_major={row_major}")
+
+
+# the small fused chain at the edges of its register form (K a multiple of 8 up to 8 * 512 / columns per CTA) and just
+# beyond them, where the staged form takes over: (M, K, N, dtype, norm, row-major weight)
+EDGE = [(64, 256, 128, "f32", "layernorm", False), (64, 256, 128, "f32", "layernorm", True), (61, 248, 100, "f32", "layernorm", True),
+        (9, 8, 8, "f32", "rmsnorm", False), (64, 264, 128, "f32", "layernorm", False), (64, 128, 256, "f32", "rmsnorm", True),
+        (64, 136, 256, "f32", "layernorm", False), (3, 512, 60, "f32", "layernorm", False), (3, 520, 60, "f32", "layernorm", True),
+        (17, 256, 128, "bf16", "layernorm", False), (17, 256, 128, "bf16", "rmsnorm", True), (40, 252, 128, "f32", "layernorm", False)]
+
+
+@pytest.mark.parametrize("m,k,n,dtype,norm,row_major", EDGE)
+def test_small_fused_chain_at_the_edges_of_its_register_form(ctx, m, k, n, dtype, norm, row_major):
+    from paper_2607_20501_b200 import binding as B
+    w = W.c1(900 + m + k + n, M=m, K=k, N=n, dtype=dtype)
+    if norm == "rmsnorm":
+        w.ops[-1] = dict(w.ops[-1], kind="rmsnorm", params={"gamma": "gamma"}, attrs={"eps": 1e-6})
+    ref, _ = oracle(w, [0])
+    dw, out = run_gpu(ctx, w, [0], weight_layout=B.MK_LAYOUT_ROW_MAJOR if row_major else None)
+    assert_parity(out, ref, dtype, f"M{m} K{k} N{n} {dtype} {norm} row_major={row_major}")
+    _, again = run_gpu(ctx, w, [0], weight_layout=B.MK_LAYOUT_ROW_MAJOR if row_major else None)
+    assert np.array_equal(out, again)     # every sum in a fixed order
