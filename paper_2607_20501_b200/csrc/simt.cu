@@ -107,6 +107,10 @@ template <typename T>
 __device__ __forceinline__ void lc_norm_tail(float v, bool has, bool in_outs, int r, int j, int nc, int NC, int N, int M, int m0, int c0,
                                              uint32_t rank, int mode, float eps, float ga, float be, float (&slot)[2][LC_CL][LC_RB],
                                              T* __restrict__ y) {
+  if (mode != ROW_LAYERNORM && mode != ROW_RMSNORM) {   // the chain without its norm (a tiny GEMM + elementwise tail)
+    if (has && m0 + r < M) Elem<T>::st(y + (int64_t)(m0 + r) * N + c0 + j, v);
+    return;
+  }
   // One exchange for both statistics.  LayerNorm: every CTA sends, per row, the mean of its columns and their squared
   // deviations from that mean; the receiver merges the eight (count, mean, M2) triples, M2 = sum of M2_c + n_c *
   // (mean_c - mean)^2, which is what a second pass about the global mean would have summed, so no second round is
@@ -418,7 +422,7 @@ static cudaError_t linear_rownorm_cluster_launch(const void* a, const void* w, b
 }
 // what the cluster form takes: a row norm with two statistics at most, few columns, operands that fit
 static bool linear_rownorm_cluster_ok(int64_t m, int64_t n, int64_t k, int mode) {
-  if (mode != ROW_LAYERNORM && mode != ROW_RMSNORM) return false;
+  if (mode != ROW_LAYERNORM && mode != ROW_RMSNORM && mode != -1) return false;   // -1: no norm, the column split alone
   if (n > LC_CL * LC_MAXNC || n < LC_CL || k > 2048 || m > (1 << 20)) return false;
   return sizeof(float) * ((size_t)(LC_RB + LC_MAXNC) * (k + 4) + LC_THREADS) <= 160 * 1024;
 }
