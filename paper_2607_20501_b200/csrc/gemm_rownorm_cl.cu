@@ -397,7 +397,8 @@ gemm_rownorm_cl_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
         }
         tc::tc_fence_before();
         __syncwarp();
-        if (lane == 0) tc::mbar_arrive_cluster(tc::map_to_cta(tc::smem_u32(&sh->tempty[slot]), leader_rank));
+        // (a relaxed arrival: the warp's reads of tensor memory are over, nothing has to be published)
+        if (lane == 0) tc::mbar_arrive_cluster_relaxed(tc::map_to_cta(tc::smem_u32(&sh->tempty[slot]), leader_rank));
       }
 #ifdef MK_TRACE_RN
       tr[6] = clock64();
