@@ -42,3 +42,18 @@ def test_one_by_one_convolution_is_exact_on_integers(ctx):
         dw, out = run_gpu(ctx, wl, [0], binds={0: impl})
         assert out.shape == (nb, h, w, n)
         assert np.array_equal(out, ref), impl
+
+
+def test_bottleneck_block_full_size_sampled_images(ctx):
+    """The benchmark's configuration ([32, 56, 56, 256] via 64 channels, default decomposition).  Images are independent
+    through every operator of the block, so the oracle checks whole images exactly."""
+    from oracle import modules as OM
+    wl = W.c9(0)
+    dw, out = run_gpu(ctx, wl, wl.partitions["fused"])
+    assert dw.module.n_sub() == 1 and dw.module.bound_impl(0) == "gemm_tc2+conv3x3_tc2+gemm_tc2"   # one submodule, three launches
+    assert out.shape == (32, 56, 56, 256) and np.isfinite(out).all()
+    params = {k: t.f64() for k, t in wl.params.items()}
+    x = wl.inputs["x"].f64()
+    for n in (0, 13, 31):
+        ref, _ = OM.run_module(wl.ops, {"x": x[n:n + 1]}, params, [0])
+        assert_parity(out[n:n + 1], ref, "bf16", f"c9 image {n}")
