@@ -609,6 +609,10 @@ cudaError_t plan_impl(GemmTcPlan* p, const void* a, const void* w_nk, void* y, b
       if (epi.op[i].kind == EPI_RESIDUAL) { idx = i; ++cnt; }
     p->res_ring = cnt == 1 && epi.op[idx].ptr_dtype == DT_BF16;
   }
+  // When the whole of W fits in L2 beside the A rows in flight (up to 48 MB), walking one tile row at a time is
+  // fastest: its column tiles run on neighbouring pairs at the same moment and share each A row while it passes
+  // (measured over groups of 1, 2, 4, 8, 16: 8192 x 2048 x 8192 185.7 ... 193.1 us, 8192 x 6144 x 2048 131.8 ... 133.7 us,
+  // 32768 x 2048 x 2048 177.3 ... 179.0 us; with 67 MB of W, 8192 x 16384 x 2048, the order turns round: 382.8 ... 352.4 us).
   // Tile rows walked together: their A rows (group_m x CTAS x 128 rows of K) plus the W slabs in flight should stay
   // in L2 for the walk across the columns.  With K = 8192 sixteen tile rows are 67 MB of A and the DRAM traffic
   // doubles (measured: 541 MB for 302 MB algorithmic); the budget below keeps a group's A rows under ~36 MB.
@@ -616,6 +620,7 @@ cudaError_t plan_impl(GemmTcPlan* p, const void* a, const void* w_nk, void* y, b
     int g = GROUP_M_MAX;
     const char* ov = getenv("MK_GEMM_GROUP_M");
     if (ov && ov[0]) g = atoi(ov);
+    else if ((int64_t)(swiglu ? 2 : 1) * n * k * 2 <= (int64_t)48 << 20) g = 1;   // W stays in L2 whatever the walk: see below
     else while (g > 2 && (int64_t)g * CTAS * BM * k * 2 > (int64_t)36 << 20) g /= 2;
     p->group_m = g < 1 ? 1 : g;
   }
