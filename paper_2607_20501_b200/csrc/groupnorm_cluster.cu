@@ -123,7 +123,7 @@ groupnorm_cluster_kernel(const T* __restrict__ x, T* __restrict__ y, int64_t hw,
     tc::fence_barrier_init();
   }
   __syncthreads();
-  tc::cluster_arrive();        // "this CTA runs": waited for before the first store into a peer's shared memory
+  tc::cluster_arrive_relaxed();        // "this CTA runs": waited for before the first store into a peer's shared memory
   pdl_launch_dependents();
   pdl_wait();                  // x may come from the kernel before this one
   const T* xin = x + (img * hw + p0) * c;

@@ -178,7 +178,7 @@ __global__ void __launch_bounds__(LC_THREADS) linear_rownorm_cluster_kernel(cons
   pdl_launch_dependents();
   // A CTA may write into a peer's shared memory only once that peer is running: every CTA announces itself
   // here and waits for the others just before its first remote store, so the rendezvous costs nothing.
-  tc::cluster_arrive();
+  tc::cluster_arrive_relaxed();
   pdl_wait();
   const uint32_t rank = tc::cluster_ctarank();
   const int m0 = (int)(blockIdx.x / LC_CL) * LC_RB, c0 = (int)rank * NC;
@@ -324,7 +324,7 @@ __global__ void __launch_bounds__(LC_THREADS) linear_rownorm_cluster_reg_kernel(
   __shared__ float part[LC_THREADS * LC_RB];               // [k slice][LC_RB][NC]
   __shared__ float slot[2][LC_CL][LC_RB];                  // every CTA's (mean, M2) of its slice of each row
   pdl_launch_dependents();
-  tc::cluster_arrive();                                    // see the staged form: met again just before the remote stores
+  tc::cluster_arrive_relaxed();                                    // see the staged form: met again just before the remote stores
   pdl_wait();
   const uint32_t rank = tc::cluster_ctarank();
   const int m0 = (int)(blockIdx.x / LC_CL) * LC_RB, c0 = (int)rank * NC;
